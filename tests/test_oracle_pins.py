@@ -1,0 +1,376 @@
+"""Pins for the fp64 oracle: each test fixes it to something other than itself - scalar
+textbook loops, brute force, closed forms, invariants, and the equivalences the paper
+states in Section 4.2 (split forward, prefill == decode loop, page omission == masking)."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import pie_oracle as orc
+from tests._util import SmallBatch, oracle_on, random_seqs, run_oracle
+from workloads import configs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "worked_example.txt")
+
+
+# ---------------------------------------------------------------- scalar textbook reference
+def textbook_attention(Q, K, V, allowed):
+    """Scalar-loop softmax attention over dense arrays: the definition, nothing else."""
+    q_len, H_q, D = Q.shape
+    G = H_q // K.shape[1]
+    O = np.zeros((q_len, H_q, D))
+    L = np.full((q_len, H_q), -math.inf)
+    for i in range(q_len):
+        for h in range(H_q):
+            js = [j for j in range(K.shape[0]) if allowed[i][j]]
+            if not js:
+                continue
+            s = [sum(float(Q[i, h, d]) * float(K[j, h // G, d]) for d in range(D)) / math.sqrt(D)
+                 for j in js]
+            Z = math.fsum(math.exp(x) for x in s)
+            for d in range(D):
+                O[i, h, d] = math.fsum(math.exp(x) * float(V[j, h // G, d]) for x, j in zip(s, js)) / Z
+            L[i, h] = math.log(Z)
+    return O, L
+
+
+def causal(q_len, kv_len):
+    return [[j <= kv_len - q_len + i for j in range(kv_len)] for i in range(q_len)]
+
+
+# p1 ------------------------------------------------------------------------------------
+@pytest.mark.parametrize("P", [8, 16])
+def test_p1_contiguous_causal_equals_textbook(P):
+    rng = np.random.RandomState(1)
+    shapes = [(1, 19), (5, 5), (7, 33)]
+    seqs = random_seqs(rng, shapes, H_q=4, H_kv=2, D=8)
+    O, L = oracle_on(SmallBatch(seqs, 4).paged(P, "contiguous"))
+    t = 0
+    for s, (q_len, kv_len) in zip(seqs, shapes):
+        Or, Lr = textbook_attention(s["Q"], s["K"], s["V"], causal(q_len, kv_len))
+        np.testing.assert_allclose(O[t:t + q_len], Or, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(L[t:t + q_len], Lr, rtol=0, atol=1e-12)
+        t += q_len
+
+
+# p2 ------------------------------------------------------------------------------------
+def test_p2_physical_page_permutation_is_bit_invariant():
+    rng = np.random.RandomState(2)
+    m = rng.rand(4, 50) < 0.6
+    m[:, 0] = True
+    seqs = random_seqs(rng, [(1, 37), (4, 50), (3, 16)], 4, 2, 16, masks=[None, m, None])
+    ref = oracle_on(SmallBatch(seqs, 4).paged(16, "contiguous"))
+    for order, seed in [("reversed", 0), ("random", 3), ("random", 4)]:
+        got = oracle_on(SmallBatch(seqs, 4).paged(16, order, seed=seed))
+        assert np.array_equal(ref[0], got[0]) and np.array_equal(ref[1], got[1])
+
+
+# p3 ------------------------------------------------------------------------------------
+def test_p3_page_size_is_bit_invariant():
+    rng = np.random.RandomState(3)
+    seqs = random_seqs(rng, [(1, 31), (6, 70), (2, 8)], 8, 1, 16)
+    ref = oracle_on(SmallBatch(seqs, 8).paged(8, "random", seed=1))
+    for P in (16, 32):
+        got = oracle_on(SmallBatch(seqs, 8).paged(P, "random", seed=P))
+        assert np.array_equal(ref[0], got[0]) and np.array_equal(ref[1], got[1])
+
+
+# p4 ------------------------------------------------------------------------------------
+def test_p4_one_hot_rows_return_that_v_row_exactly():
+    rng = np.random.RandomState(4)
+    kv_len, q_len = 45, 6
+    pick = rng.randint(0, kv_len, size=q_len)
+    m = np.zeros((q_len, kv_len), dtype=bool)
+    m[np.arange(q_len), pick] = True
+    seqs = random_seqs(rng, [(q_len, kv_len)], 4, 2, 16, masks=[m])
+    O, L = oracle_on(SmallBatch(seqs, 4).paged(16, "random"))
+    s = seqs[0]
+    for i in range(q_len):
+        for h in range(4):
+            assert np.array_equal(O[i, h], s["V"][pick[i], h // 2].astype(np.float64))
+            sc = float(np.dot(s["Q"][i, h].astype(np.float64), s["K"][pick[i], h // 2].astype(np.float64))) / 4.0
+            assert abs(L[i, h] - sc) < 1e-13
+
+
+# p5 ------------------------------------------------------------------------------------
+def test_p5_brute_force_all_masks_tiny():
+    rng = np.random.RandomState(5)
+    D = 4
+    for kv_len in (1, 2, 3, 4):
+        for q_len in (1, 2):
+            if q_len > kv_len:
+                continue
+            rows = list(itertools.product([False, True], repeat=kv_len))
+            for combo in itertools.islice(itertools.product(rows, repeat=q_len), 0, None, 3 if q_len == 2 else 1):
+                m = np.array(combo, dtype=bool)
+                seqs = random_seqs(rng, [(q_len, kv_len)], 2, 1, D, masks=[m])
+                O, L = oracle_on(SmallBatch(seqs, 2).paged(8))
+                Or, Lr = textbook_attention(seqs[0]["Q"], seqs[0]["K"], seqs[0]["V"], m)
+                np.testing.assert_allclose(O, Or, rtol=0, atol=1e-13)
+                assert np.array_equal(np.isneginf(L), np.isneginf(Lr))
+                fin = np.isfinite(Lr)
+                np.testing.assert_allclose(L[fin], Lr[fin], rtol=0, atol=1e-13)
+                for i in range(q_len):      # empty row: zero output, LSE = -inf
+                    if not m[i].any():
+                        assert not O[i].any() and np.isneginf(L[i]).all()
+
+
+# p6 ------------------------------------------------------------------------------------
+def test_p6_closed_forms():
+    rng = np.random.RandomState(6)
+    kv_len, q_len = 40, 3
+    m = rng.rand(q_len, kv_len) < 0.5
+    m[:, 5] = True
+    seqs = random_seqs(rng, [(q_len, kv_len)], 4, 2, 16, masks=[m])
+    base = seqs[0]
+    # Q = 0: uniform weights over the allowed set
+    z = dict(base, Q=np.zeros_like(base["Q"]))
+    O, L = oracle_on(SmallBatch([z], 4).paged(16))
+    for i in range(q_len):
+        for h in range(4):
+            np.testing.assert_allclose(O[i, h], base["V"][m[i], h // 2].astype(np.float64).mean(0), atol=1e-14)
+            assert abs(L[i, h] - math.log(m[i].sum())) < 1e-14
+    # all K rows equal: uniform weights again, LSE = score + ln|S|
+    kk = dict(base, K=np.broadcast_to(base["K"][:1], base["K"].shape).copy())
+    O2, L2 = oracle_on(SmallBatch([kk], 4).paged(16))
+    np.testing.assert_allclose(O2, O, atol=1e-13)
+    # V constant: output is that constant for any mask
+    c = rng.randn(2, 16).astype(np.float32)
+    vc = dict(base, V=np.broadcast_to(c, base["V"].shape).copy())
+    O3, _ = oracle_on(SmallBatch([vc], 4).paged(16))
+    for h in range(4):
+        np.testing.assert_allclose(O3[:, h], np.broadcast_to(c[h // 2].astype(np.float64), (q_len, 16)), atol=1e-14)
+    # V + u shifts O by u and leaves LSE alone (V on a 2^-10 grid so the shift is exact in fp32)
+    Vq = (np.round(base["V"].astype(np.float64) * 1024) / 1024).astype(np.float32)
+    O4, L4 = oracle_on(SmallBatch([dict(base, V=Vq)], 4).paged(16))
+    O5, L5 = oracle_on(SmallBatch([dict(base, V=(Vq.astype(np.float64) + 0.5).astype(np.float32))], 4).paged(16))
+    np.testing.assert_allclose(O5, O4 + 0.5, atol=1e-13)
+    np.testing.assert_array_equal(L5, L4)
+
+
+# p7 ------------------------------------------------------------------------------------
+def test_p7_lse_merge_identity():
+    rng = np.random.RandomState(7)
+    kv_len, q_len = 64, 4
+    full = rng.rand(q_len, kv_len) < 0.7
+    full[:, 0] = True
+    part = rng.randint(0, 3, size=kv_len)                 # three disjoint column classes
+    part[10:20] = 2
+    seqs = random_seqs(rng, [(q_len, kv_len)], 4, 2, 16, masks=[full])
+    O, L = oracle_on(SmallBatch(seqs, 4).paged(16))
+    Os, Ls = [], []
+    for c in range(3):
+        mc = full & (part[None, :] == c)
+        if c == 1:
+            mc[2, :] = False                              # an empty part for one row
+            full_row2 = full[2] & (part != 1)
+        s = dict(seqs[0], mask=mc)
+        o, l = oracle_on(SmallBatch([s], 4).paged(16))
+        Os.append(o), Ls.append(l)
+    # row 2 lost its class-1 columns: recompute the reference for that row's reduced set
+    f2 = full.copy()
+    f2[2] = full_row2
+    O, L = oracle_on(SmallBatch([dict(seqs[0], mask=f2)], 4).paged(16))
+    Om, Lm = orc.merge_partials(Os, Ls)
+    np.testing.assert_allclose(Om, O, atol=1e-13)
+    np.testing.assert_allclose(Lm, L, atol=1e-13)
+
+
+# p8 ------------------------------------------------------------------------------------
+def test_p8_split_forward_and_decode_loop_equal_one_prefill():
+    """Section 4.2: a 9-token prefill equals an 8-token forward that fills KvPages followed
+    by a 1-token forward that reads them; and prefill equals the token-by-token loop."""
+    rng = np.random.RandomState(8)
+    n, P, H_q, H_kv, D = 21, 8, 4, 2, 16
+    Q = rng.randn(n, H_q, D).astype(np.float32)
+    K = rng.randn(n, H_kv, D).astype(np.float32)
+    V = rng.randn(n, H_kv, D).astype(np.float32)
+    O_full, L_full = oracle_on(SmallBatch([dict(Q=Q, K=K, V=V)], H_q).paged(P, "random", seed=1))
+
+    npg = (n + P - 1) // P
+    pages = np.random.RandomState(9).permutation(npg + 2)[:npg]
+    pool = {int(p): (np.full((P, H_kv, D), np.nan, np.float32), np.full((P, H_kv, D), np.nan, np.float32))
+            for p in range(npg + 2)}
+
+    def step(lo, hi):
+        np_r = (hi + P - 1) // P
+        return orc.forward(pool, P, H_q, np.array([0, hi - lo]), np.array([0, np_r]), pages[:np_r],
+                           np.array([hi - (np_r - 1) * P]), Q[lo:hi], K[lo:hi], V[lo:hi])
+
+    O1, L1 = step(0, n - 1)          # fills the pages with n-1 tokens
+    O2, L2 = step(n - 1, n)          # one token reading them
+    np.testing.assert_allclose(np.concatenate([O1, O2]), O_full, atol=1e-14)
+    np.testing.assert_allclose(np.concatenate([L1, L2]), L_full, atol=1e-14)
+
+    for p in pool:                    # token-by-token from an empty cache
+        pool[p][0][:] = np.nan
+        pool[p][1][:] = np.nan
+    outs = [step(i, i + 1) for i in range(n)]
+    np.testing.assert_allclose(np.concatenate([o for o, _ in outs]), O_full, atol=1e-14)
+    np.testing.assert_allclose(np.concatenate([l for _, l in outs]), L_full, atol=1e-14)
+
+
+# p9 ------------------------------------------------------------------------------------
+def test_p9_page_omission_equals_masking():
+    rng = np.random.RandomState(10)
+    P, kv_len, H_q, H_kv, D = 8, 48, 4, 2, 16
+    seq = random_seqs(rng, [(1, kv_len)], H_q, H_kv, D)[0]
+    drop_pages = [1, 3]
+    keep = np.ones(kv_len, dtype=bool)
+    for p in drop_pages:
+        keep[p * P:(p + 1) * P] = False
+    O_mask, L_mask = oracle_on(SmallBatch([dict(seq, mask=keep[None, :])], H_q).paged(P, "random"))
+    short = dict(Q=seq["Q"], K=seq["K"][keep], V=seq["V"][keep])     # pages simply left out
+    O_omit, L_omit = oracle_on(SmallBatch([short], H_q).paged(P, "random", seed=5))
+    np.testing.assert_allclose(O_omit, O_mask, atol=1e-14)
+    np.testing.assert_allclose(L_omit, L_mask, atol=1e-14)
+
+
+# p10 -----------------------------------------------------------------------------------
+def test_p10_shared_pages_equal_private_copies():
+    wl = configs.small("shared_prefix_tree")
+    O, L, _ = run_oracle(wl)
+    # give every branch a private copy of its group's prefix pages via copy_kvpage
+    pool = wl.oracle_pool()
+    n_pre = wl.meta["prefix"] // wl.P
+    free = [p for p in range(wl.num_pages) if wl.page_owner[p] < 0]
+    idx = wl.page_indices.copy()
+    src, dst = [], []
+    for r in range(wl.R):
+        if r % wl.meta["branches"] == 0:
+            continue                                       # first branch keeps the original
+        base = wl.page_indptr[r]
+        for k in range(n_pre):
+            new = free.pop()
+            src.append(idx[base + k]), dst.append(new)
+            idx[base + k] = new
+    for p in dst:
+        pool[p] = (np.zeros((wl.P, wl.H_kv, wl.D), np.uint16), np.zeros((wl.P, wl.H_kv, wl.D), np.uint16))
+    n = len(src)
+    orc.copy_kvpage(pool, src, dst, [0] * n, [0] * n, [wl.P] * n)
+    from tests._util import bits
+    O2, L2 = orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, idx, wl.last_page_len,
+                         bits(wl.q()), bits(wl.k_new()), bits(wl.v_new()), wl.masks)
+    assert np.array_equal(O, O2) and np.array_equal(L, L2)
+
+
+def test_copy_kvpage_token_ranges():
+    P, H, D = 8, 2, 4
+    rng = np.random.RandomState(11)
+    pool = {p: (rng.randn(P, H, D).astype(np.float32), rng.randn(P, H, D).astype(np.float32)) for p in range(4)}
+    before = {p: (k.copy(), v.copy()) for p, (k, v) in pool.items()}
+    orc.copy_kvpage(pool, [0, 1], [2, 0], [1, 0], [3, 5], [4, 2])
+    for kv in (0, 1):
+        exp2 = before[2][kv].copy()
+        exp2[3:7] = before[0][kv][1:5]
+        exp0 = before[0][kv].copy()
+        exp0[5:7] = before[1][kv][0:2]
+        assert np.array_equal(pool[2][kv], exp2) and np.array_equal(pool[0][kv], exp0)
+        assert np.array_equal(pool[1][kv], before[1][kv]) and np.array_equal(pool[3][kv], before[3][kv])
+
+
+# p11 -----------------------------------------------------------------------------------
+def test_p11_tree_mask_equals_causal_path():
+    wl = configs.small("shared_prefix_tree")
+    O, L, pool = run_oracle(wl)
+    from tests._util import bits
+    q, k_new, v_new = bits(wl.q()), bits(wl.k_new()), bits(wl.v_new())
+    ctx = wl.meta["prefix"] + wl.meta["suffix"]
+    for r in (0, wl.R - 1):
+        par = wl.meta["parents"][r]
+        t0 = wl.qo_indptr[r]
+        pages = wl.pages_of(r)
+        Kc, Vc = orc.gather_kv(pool, wl.P, pages, ctx)      # context rows (post-append pool)
+        for n in (0, 5, len(par) - 1):
+            path = []
+            a = n
+            while a >= 0:
+                path.append(a)
+                a = par[a]
+            path = path[::-1]                                # root .. n
+            K = np.concatenate([Kc, orc.widen(k_new[t0 + np.array(path)])])
+            V = np.concatenate([Vc, orc.widen(v_new[t0 + np.array(path)])])
+            Or, Lr = textbook_free(orc.widen(q[t0 + n])[None], K, V)
+            np.testing.assert_allclose(O[t0 + n], Or[0], atol=1e-12)
+            np.testing.assert_allclose(L[t0 + n], Lr[0], atol=1e-12)
+
+
+def textbook_free(Q, K, V):
+    """Dense unmasked attention of the LAST query position over all rows, vectorised
+    differently from the oracle (einsum + logsumexp by hand)."""
+    q_len, H_q, D = Q.shape
+    G = H_q // K.shape[1]
+    Kh = np.repeat(K, G, axis=1)
+    Vh = np.repeat(V, G, axis=1)
+    s = np.einsum("ihd,jhd->ihj", Q, Kh) / math.sqrt(D)
+    Z = np.exp(s).sum(-1)
+    return np.einsum("ihj,jhd->ihd", np.exp(s), Vh) / Z[..., None], np.log(Z)
+
+
+# p12 -----------------------------------------------------------------------------------
+def test_p12_gqa_equals_repeated_mha():
+    rng = np.random.RandomState(12)
+    seqs = random_seqs(rng, [(3, 29), (1, 12)], 8, 2, 16)
+    O, L = oracle_on(SmallBatch(seqs, 8).paged(8, "random"))
+    rep = [dict(Q=s["Q"], K=np.repeat(s["K"], 4, axis=1), V=np.repeat(s["V"], 4, axis=1)) for s in seqs]
+    O2, L2 = oracle_on(SmallBatch(rep, 8).paged(8, "random"))
+    np.testing.assert_allclose(O2, O, atol=1e-14)
+    np.testing.assert_allclose(L2, L, atol=1e-14)
+
+
+# p13 -----------------------------------------------------------------------------------
+def test_p13_append_touches_exactly_the_new_rows_and_poison_is_harmless():
+    wl = configs.small("mixed_prefill_decode")
+    from tests._util import bits
+    pool = wl.oracle_pool(poison=True)
+    used = wl.used_pages()
+    before = {int(p): (pool[int(p)][0].copy(), pool[int(p)][1].copy()) for p in used}
+    O, L, _ = run_oracle(wl, pool=pool)
+    k_new, v_new = bits(wl.k_new()), bits(wl.v_new())
+    changed = 0
+    kv, ql = wl.kv_lens(), wl.q_lens()
+    expect = {}
+    for r in range(wl.R):
+        for i in range(ql[r]):
+            pos = kv[r] - ql[r] + i
+            expect[(int(wl.pages_of(r)[pos // wl.P]), int(pos % wl.P))] = wl.qo_indptr[r] + i
+    for p in used:
+        for slot in range(wl.P):
+            key = (int(p), slot)
+            for kvsel, new in ((0, k_new), (1, v_new)):
+                now, old = pool[int(p)][kvsel][slot], before[int(p)][kvsel][slot]
+                if key in expect:
+                    assert np.array_equal(now, new[expect[key]])
+                    changed += now.size
+                else:
+                    assert np.array_equal(now, old)
+    assert changed == wl.T * wl.H_kv * wl.D * 2
+    O2, L2, _ = run_oracle(wl, poison=False)                # NaN in unused slots changes nothing
+    assert np.isfinite(O).all()
+    assert np.array_equal(O, O2) and np.array_equal(L, L2)
+
+
+# golden --------------------------------------------------------------------------------
+def test_golden_worked_example():
+    vec, cases = {}, []
+    for line in open(GOLDEN):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        tok = line.split()
+        if tok[0] == "mask":
+            cases.append(([bool(int(tok[1])), bool(int(tok[2]))], [float(x) for x in tok[5:9]], float(tok[10])))
+        else:
+            vec[tok[0]] = np.array([float(x) for x in tok[1:]], dtype=np.float64)
+    assert len(cases) == 3
+    for mask, O_exp, L_exp in cases:
+        seq = dict(Q=vec["q"][None, None, :], K=np.stack([vec["k0"], vec["k1"]])[:, None, :],
+                   V=np.stack([vec["v0"], vec["v1"]])[:, None, :], mask=np.array([mask]))
+        args = SmallBatch([{k: (v.astype(np.float64) if k != "mask" else v) for k, v in seq.items()}], 1).paged(8)
+        for p in args["pool"]:      # keep fp64 storage so ln 3 is not rounded to fp32
+            args["pool"][p] = (args["pool"][p][0].astype(np.float64), args["pool"][p][1].astype(np.float64))
+        O, L = oracle_on(args)
+        np.testing.assert_allclose(O[0, 0], O_exp, atol=1e-14)
+        assert abs(L[0, 0] - L_exp) < 1e-14
