@@ -1,0 +1,190 @@
+/*
+ * pie_b200.h - C ABI of the B200-native batched `forward` attention handler.
+ *
+ * The calls follow the inference-layer handler API of the Pie paper (Table 1: alloc_kvpage,
+ * dealloc_kvpage, copy_kvpage, forward; Section 4.1 "Resources" for KvPages; Section 4.2
+ * "Forward API" for masks and positions; Section 5.2 for the batch the control layer hands
+ * to a handler).  One `forward` batch = many inferlets' calls coalesced: per request the new
+ * K/V rows are appended to its output KvPages and every query token attends over the
+ * request's page list under its mask.
+ *
+ * Conventions
+ *   - Every function returns PIE_OK (0) or a negative pie_status.  Nothing throws, aborts or
+ *     traps on the device.  pie_strerror() names a status.
+ *   - "host" / "device" below says where a pointer must live.  Index arrays given to the
+ *     planner are host memory, read during the call and not retained.
+ *   - Device work is enqueued on the caller's stream (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream) and is asynchronous unless stated otherwise.  Ordering
+ *     between calls is stream order (the paper's command-queue order).
+ *   - The KvPage pool is owned by the library; its layout is private.  Q / K_new / V_new /
+ *     output / LSE buffers are owned by the caller.
+ *   - Element type: bf16 or fp32 for Q, K, V and the output; LSE is always fp32.
+ */
+#ifndef PIE_B200_H_
+#define PIE_B200_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum pie_status {
+  PIE_OK = 0,
+  PIE_ERR_INVALID = -1,         /* bad argument (null pointer, size out of range, bad config)   */
+  PIE_ERR_NO_PAGES = -2,        /* pool exhausted; nothing was allocated                        */
+  PIE_ERR_BAD_PAGE = -3,        /* page id out of range, not allocated, or freed twice          */
+  PIE_ERR_CONFLICT = -4,        /* two batched calls touch the same KvPage slot, one writing    */
+  PIE_ERR_BATCH_TOO_LARGE = -5, /* more requests / query tokens than the configured maximum     */
+  PIE_ERR_MASK = -6,            /* mask range size != q_len * kv_len, or a byte not 0/1         */
+  PIE_ERR_CUDA = -7,            /* a CUDA runtime call failed (see pie_last_cuda_error)         */
+  PIE_ERR_NO_DEVICE = -8,       /* the context was created host-only (device = -1)              */
+  PIE_ERR_UNSUPPORTED = -9,     /* shape / type combination the kernels do not cover            */
+  PIE_ERR_DEVICE_TIMEOUT = -10  /* a bounded device-side wait gave up (results invalid)         */
+} pie_status;
+
+enum { PIE_DTYPE_BF16 = 0, PIE_DTYPE_F32 = 1 };
+
+/* Start-up configuration (Section 5.2 "Resource management": the pool is sized once at
+ * start-up; Section 5.2 "Batch scheduler": the backend has a maximum batch size). */
+typedef struct pie_config {
+  int32_t num_pages;        /* KvPages in the pool                                    */
+  int32_t page_size;        /* tokens per KvPage: 8, 16 or 32 (Section 4.1)            */
+  int32_t num_q_heads;      /* H_q                                                    */
+  int32_t num_kv_heads;     /* H_kv, divides H_q; kv head of q head h is h / (H_q/H_kv) */
+  int32_t head_dim;         /* D: 64 or 128                                           */
+  int32_t dtype;            /* PIE_DTYPE_BF16 or PIE_DTYPE_F32                         */
+  int32_t max_requests;     /* largest batch (requests) pie_plan_forward accepts       */
+  int32_t max_query_tokens; /* largest total of query tokens in one batch              */
+  int32_t device;           /* CUDA device ordinal; -1 = host-only context (planner,
+                               allocator and validation work; device calls return
+                               PIE_ERR_NO_DEVICE)                                      */
+} pie_config;
+
+typedef struct pie_ctx pie_ctx;
+typedef struct pie_plan pie_plan;
+
+const char* pie_strerror(int status);
+/* Text of the last CUDA error seen by this context ("" if none).  Host. */
+const char* pie_last_cuda_error(const pie_ctx* ctx);
+
+/* Create a context and its KvPage pool (Section 5.3: the inference layer holds the physical
+ * memory).  Allocates num_pages * page_size * 2 * H_kv * D elements on the device and
+ * zero-fills them once.  *out is set only on success.  Synchronous. */
+int pie_create(const pie_config* cfg, pie_ctx** out);
+/* Free the pool and everything the context owns.  Plans must be destroyed first. */
+int pie_destroy(pie_ctx* ctx);
+
+/* alloc_kvpage / dealloc_kvpage (Table 1).  Host free list; no device work.
+ * pie_alloc_kvpages writes n page ids to out_ids (host) or fails with PIE_ERR_NO_PAGES and
+ * allocates nothing (the caller applies the first-come-first-served policy of Section 5.2).
+ * Page contents are NOT cleared.  pie_dealloc_kvpages rejects ids that are out of range or
+ * not allocated (PIE_ERR_BAD_PAGE) without freeing any. */
+int pie_alloc_kvpages(pie_ctx* ctx, int32_t n, int32_t* out_ids);
+int pie_dealloc_kvpages(pie_ctx* ctx, int32_t n, const int32_t* ids);
+int pie_num_free_kvpages(const pie_ctx* ctx, int32_t* out);
+
+/* Write / read whole pages in the canonical layout  K[n][page_size][H_kv][D], V[same]
+ * (the save / restore side of export_kvpage / import_kvpage, Table 1; also how tests install
+ * context).  ids: host.  K, V: host memory if on_device == 0 (the call then synchronises the
+ * stream before returning), device memory if on_device == 1 (asynchronous). */
+int pie_kvpage_write(pie_ctx* ctx, int32_t n, const int32_t* ids, const void* K, const void* V,
+                     int on_device, void* stream);
+int pie_kvpage_read(pie_ctx* ctx, int32_t n, const int32_t* ids, void* K, void* V,
+                    int on_device, void* stream);
+
+/* copy_kvpage (Table 1: "copy KV cache contents at token-level").  For op k, rows
+ * [src_off[k], src_off[k]+ntok[k]) of page src[k] are copied (K and V, all heads, bit for bit)
+ * to rows starting at dst_off[k] of page dst[k].  All arrays: host, n entries.
+ * Errors: ranges outside a page or unallocated pages (PIE_ERR_BAD_PAGE / PIE_ERR_INVALID);
+ * two ops writing the same slot, or an op reading a slot another op of the same call writes
+ * (PIE_ERR_CONFLICT).  Asynchronous on `stream`. */
+int pie_copy_kvpage(pie_ctx* ctx, int32_t n, const int32_t* src, const int32_t* dst,
+                    const int32_t* src_off, const int32_t* dst_off, const int32_t* ntok,
+                    void* stream);
+
+/* One coalesced `forward` batch as the control layer hands it over (Section 5.2).
+ * Request r has q_len = qo_indptr[r+1]-qo_indptr[r] >= 1 new tokens and the page list
+ * page_indices[page_indptr[r] .. page_indptr[r+1]) (input KvPages followed by output KvPages;
+ * ids may repeat across requests: shared pages).  last_page_len[r] in [1, page_size] counts the
+ * filled slots of the last page AFTER the append, so the context length is
+ * kv_len = (num_pages_r - 1) * page_size + last_page_len[r] and the new tokens occupy
+ * positions kv_len - q_len .. kv_len - 1.
+ * Mask (Section 4.2): mask_indptr == NULL, or an empty range for request r, means "infer from
+ * positions": token i attends to positions <= kv_len - q_len + i.  Otherwise
+ * mask[mask_indptr[r] .. mask_indptr[r+1]) holds q_len * kv_len bytes, row major, 1 = attend,
+ * 0 = masked; it is the complete specification (not combined with causality) and is shared by
+ * all heads.  A row with no allowed position yields output 0 and LSE = -inf. */
+typedef struct pie_batch_desc {
+  int32_t num_requests;
+  const int32_t* qo_indptr;     /* [R+1], qo_indptr[0] == 0                       */
+  const int32_t* page_indptr;   /* [R+1], page_indptr[0] == 0                     */
+  const int32_t* page_indices;  /* [page_indptr[R]]                               */
+  const int32_t* last_page_len; /* [R]                                            */
+  const int64_t* mask_indptr;   /* [R+1] or NULL                                  */
+  const uint8_t* mask;          /* [mask_indptr[R]] or NULL                       */
+  uint32_t flags;               /* PIE_PLAN_* below, 0 for the default path       */
+} pie_batch_desc;
+
+enum {
+  PIE_PLAN_FORCE_SIMPLE = 1u,   /* run every request through the plain CUDA-core kernel   */
+  PIE_PLAN_NO_TENSOR_TILES = 2u /* keep prefill / tree requests off the tcgen05 tile path */
+};
+
+typedef struct pie_plan_info {
+  int32_t num_requests;
+  int32_t num_query_tokens;
+  int32_t num_split_items;      /* work items of the split-KV (decode) kernel      */
+  int32_t num_tile_items;       /* work items of the prefill / tree tile kernel    */
+  int32_t num_simple_rows;      /* (token, head) rows given to the plain kernel    */
+  int32_t num_merge_groups;     /* groups whose split partials the merge combines  */
+  int32_t launches;             /* kernels one pie_forward enqueues                */
+  int32_t reserved;
+  int64_t kept_pages;           /* pages left in the lists after dropping fully masked ones */
+  int64_t mask_words;           /* 32-bit words of packed mask                     */
+  int64_t workspace_bytes;      /* device scratch for split partials               */
+} pie_plan_info;
+
+/* Batch planner (host side of `forward`): validates the batch, infers or bit-packs the masks
+ * (LSB first, 32-bit words, rows padded to 128 bits), drops pages no query row attends to,
+ * splits the work across SMs, and uploads the result.  Errors: PIE_ERR_BAD_PAGE (id out of
+ * range / not allocated), PIE_ERR_INVALID (last_page_len outside [1,page_size], q_len < 1,
+ * kv_len < q_len, non-monotone indptr), PIE_ERR_CONFLICT (two requests append to the same
+ * slot, or one reads a slot another one writes: the vertical-batching rule of Section 5.2),
+ * PIE_ERR_BATCH_TOO_LARGE, PIE_ERR_MASK.  *out is set only on success.  The upload uses
+ * `stream`; the call returns after it completed. */
+int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pie_plan** out);
+int pie_plan_destroy(pie_plan* plan);
+int pie_plan_get_info(const pie_plan* plan, pie_plan_info* out);
+
+/* Planner introspection for tests: copy one of the plan's host-side arrays into buf (host).
+ * which: 0 = packed mask words (uint32), 1 = kept page list (int32 pairs: physical id,
+ * logical page | 0x80000000 if the page needs mask evaluation), 2 = append destinations
+ * (int32 per query token: page * page_size + slot).  *out_bytes receives the array size; data
+ * is copied only if cap_bytes is large enough. */
+int pie_plan_debug_read(const pie_plan* plan, int which, void* buf, int64_t cap_bytes,
+                        int64_t* out_bytes);
+
+/* forward (Table 1; Section 4.2).  Device pointers: q [T][H_q][D], k_new / v_new
+ * [T][H_kv][D], out [T][H_q][D] in the configured element type, lse [T][H_q] fp32 (natural log
+ * of the sum of exp of the scaled scores).  Enqueues on `stream`: append of the new rows into
+ * the pool, then attention (scale 1/sqrt(D)) reading the pool, then the merge of split
+ * partials.  The plan may be reused for repeated calls with the same batch structure. */
+int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new,
+                const void* v_new, void* out, float* lse, void* stream);
+
+/* The same call for callers whose tensors live in HOST memory: plans the batch, copies
+ * q / k_new / v_new to the device, runs pie_forward, copies out / lse back and synchronises.
+ * All pointers host (pinned memory makes the copies asynchronous with respect to the host,
+ * but the call still returns only after the results arrived). */
+int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, const void* k_new,
+                     const void* v_new, void* out, float* lse, void* stream);
+
+/* Device-side status word: 0, or PIE_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel
+ * gave up since the last call.  Synchronises `stream`, reads and clears the word. */
+int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PIE_B200_H_ */

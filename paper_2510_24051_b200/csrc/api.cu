@@ -1,0 +1,515 @@
+// C ABI entry points, the KvPage allocator, and the bit-exact data-movement kernels
+// (append of new K/V rows, token-level page copy, canonical page import / export).
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "pie_internal.h"
+
+// ------------------------------------------------------------------------------------ kernels
+namespace {
+
+// K1: append (Table 1 `forward`, output KvPages).  One thread moves one 16-byte chunk of one
+// new K or V row into the swizzled pool block of its destination (page, slot).
+__global__ void append_kernel(uint8_t* __restrict__ pool, const uint8_t* __restrict__ k_new,
+                              const uint8_t* __restrict__ v_new, const int32_t* __restrict__ append_dst,
+                              int T, PoolGeom g) {
+  const int chunks = g.row_bytes >> 4;
+  const int64_t per_tok = (int64_t)2 * g.n_kv_heads * chunks;
+  const int64_t total = (int64_t)T * per_tok;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int t = (int)(i / per_tok);
+    int rem = (int)(i - (int64_t)t * per_tok);
+    int kv = rem / (g.n_kv_heads * chunks);
+    rem -= kv * g.n_kv_heads * chunks;
+    int head = rem / chunks, c = rem - head * chunks;
+    const uint8_t* src = (kv ? v_new : k_new) + ((int64_t)t * g.n_kv_heads + head) * g.row_bytes + c * 16;
+    int dst = append_dst[t];
+    int page = dst / g.page_size, slot = dst - page * g.page_size;
+    uint8_t* d = pool + (int64_t)page * g.page_bytes + (int64_t)(head * 2 + kv) * g.block_bytes +
+                 pie_chunk_offset(g.slab_bytes, slot, c);
+    *reinterpret_cast<uint4*>(d) = *reinterpret_cast<const uint4*>(src);
+  }
+}
+
+// K2: copy_kvpage (Table 1).  ops[k] = {src, dst, src_off, dst_off, ntok}; one block per op.
+__global__ void copy_kernel(uint8_t* __restrict__ pool, const int32_t* __restrict__ ops, PoolGeom g) {
+  const int32_t* op = ops + blockIdx.x * 5;
+  const int src = op[0], dst = op[1], so = op[2], dof = op[3], n = op[4];
+  const int chunks = g.row_bytes >> 4;
+  const int per_tok = 2 * g.n_kv_heads * chunks;
+  for (int i = threadIdx.x; i < n * per_tok; i += blockDim.x) {
+    int t = i / per_tok, rem = i - t * per_tok;
+    int blk = rem / chunks, c = rem - blk * chunks;  // blk = head*2 + kv
+    const uint8_t* s = pool + (int64_t)src * g.page_bytes + (int64_t)blk * g.block_bytes +
+                       pie_chunk_offset(g.slab_bytes, so + t, c);
+    uint8_t* d = pool + (int64_t)dst * g.page_bytes + (int64_t)blk * g.block_bytes +
+                 pie_chunk_offset(g.slab_bytes, dof + t, c);
+    *reinterpret_cast<uint4*>(d) = *reinterpret_cast<const uint4*>(s);
+  }
+}
+
+// Canonical [n][slot][head][D] <-> pool layout, 16 bytes per thread.
+__global__ void page_io_kernel(uint8_t* __restrict__ pool, const int32_t* __restrict__ ids, uint8_t* K,
+                               uint8_t* V, int n, int write, PoolGeom g) {
+  const int chunks = g.row_bytes >> 4;
+  const int64_t per_page = (int64_t)g.page_size * g.n_kv_heads * chunks;
+  const int64_t total = (int64_t)n * per_page * 2;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int kv = (int)(i / ((int64_t)n * per_page));
+    int64_t j = i - (int64_t)kv * n * per_page;  // chunk index inside canonical K or V
+    int pg = (int)(j / per_page);
+    int rem = (int)(j - (int64_t)pg * per_page);
+    int slot = rem / (g.n_kv_heads * chunks);
+    rem -= slot * g.n_kv_heads * chunks;
+    int head = rem / chunks, c = rem - head * chunks;
+    uint8_t* canon = (kv ? V : K) + j * 16;
+    uint8_t* p = pool + (int64_t)ids[pg] * g.page_bytes + (int64_t)(head * 2 + kv) * g.block_bytes +
+                 pie_chunk_offset(g.slab_bytes, slot, c);
+    if (write) *reinterpret_cast<uint4*>(p) = *reinterpret_cast<const uint4*>(canon);
+    else *reinterpret_cast<uint4*>(canon) = *reinterpret_cast<const uint4*>(p);
+  }
+}
+
+int grid_for(int64_t work_items, int threads, int n_sms) {
+  int64_t blocks = (work_items + threads - 1) / threads;
+  return (int)std::max<int64_t>(1, std::min<int64_t>(blocks, (int64_t)n_sms * 8));
+}
+
+int ensure_buffer(pie_ctx* ctx, void** buf, size_t* cap, size_t need) {
+  if (*cap >= need) return PIE_OK;
+  if (*buf) PIE_CUDA(ctx, cudaFree(*buf));
+  *buf = nullptr;
+  *cap = 0;
+  size_t want = std::max(need, (size_t)1 << 20);
+  PIE_CUDA(ctx, cudaMalloc(buf, want));
+  *cap = want;
+  return PIE_OK;
+}
+
+bool page_ok(const pie_ctx* ctx, int32_t id) {
+  return id >= 0 && id < ctx->cfg.num_pages && ctx->allocated[id];
+}
+
+}  // namespace
+
+int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, const void* v_new, cudaStream_t s) {
+  if (plan->T == 0) return PIE_OK;
+  const PoolGeom& g = ctx->geom;
+  int64_t work = (int64_t)plan->T * 2 * g.n_kv_heads * (g.row_bytes >> 4);
+  append_kernel<<<grid_for(work, 256, ctx->n_sms), 256, 0, s>>>(ctx->pool, (const uint8_t*)k_new, (const uint8_t*)v_new,
+                                                                 plan->d_append_dst, plan->T, g);
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}
+
+int pie_launch_copy(pie_ctx* ctx, int n, const int32_t* d_ops, cudaStream_t s) {
+  copy_kernel<<<n, 256, 0, s>>>(ctx->pool, d_ops, ctx->geom);
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}
+
+int pie_launch_page_io(pie_ctx* ctx, int n, const int32_t* d_ids, void* K, void* V, bool write, cudaStream_t s) {
+  const PoolGeom& g = ctx->geom;
+  int64_t work = (int64_t)n * g.page_size * g.n_kv_heads * (g.row_bytes >> 4) * 2;
+  page_io_kernel<<<grid_for(work, 256, ctx->n_sms), 256, 0, s>>>(ctx->pool, d_ids, (uint8_t*)K, (uint8_t*)V, n,
+                                                                  write ? 1 : 0, g);
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}
+
+// ------------------------------------------------------------------------------------ C ABI
+extern "C" {
+
+const char* pie_strerror(int status) {
+  switch (status) {
+    case PIE_OK: return "ok";
+    case PIE_ERR_INVALID: return "invalid argument";
+    case PIE_ERR_NO_PAGES: return "out of KvPages";
+    case PIE_ERR_BAD_PAGE: return "bad KvPage id";
+    case PIE_ERR_CONFLICT: return "conflicting KvPage access inside one batch";
+    case PIE_ERR_BATCH_TOO_LARGE: return "batch exceeds the configured maximum";
+    case PIE_ERR_MASK: return "malformed mask";
+    case PIE_ERR_CUDA: return "CUDA error";
+    case PIE_ERR_NO_DEVICE: return "host-only context";
+    case PIE_ERR_UNSUPPORTED: return "unsupported shape or type";
+    case PIE_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+const char* pie_last_cuda_error(const pie_ctx* ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
+
+int pie_create(const pie_config* cfg, pie_ctx** out) {
+  if (!cfg || !out) return PIE_ERR_INVALID;
+  const int P = cfg->page_size, D = cfg->head_dim;
+  if (P != 8 && P != 16 && P != 32) return PIE_ERR_INVALID;
+  if (D != 64 && D != 128) return PIE_ERR_INVALID;
+  if (cfg->dtype != PIE_DTYPE_BF16 && cfg->dtype != PIE_DTYPE_F32) return PIE_ERR_INVALID;
+  if (cfg->num_pages < 1 || cfg->num_q_heads < 1 || cfg->num_kv_heads < 1) return PIE_ERR_INVALID;
+  if (cfg->num_q_heads % cfg->num_kv_heads) return PIE_ERR_INVALID;
+  if (cfg->max_requests < 1 || cfg->max_query_tokens < 1) return PIE_ERR_INVALID;
+  if ((int64_t)cfg->num_pages * P > 0x7FFFFFFF) return PIE_ERR_INVALID;
+  pie_ctx* ctx = new (std::nothrow) pie_ctx();
+  if (!ctx) return PIE_ERR_INVALID;
+  ctx->cfg = *cfg;
+  ctx->G = cfg->num_q_heads / cfg->num_kv_heads;
+  PoolGeom& g = ctx->geom;
+  g.page_size = P;
+  g.n_kv_heads = cfg->num_kv_heads;
+  g.head_dim = D;
+  g.esize = cfg->dtype == PIE_DTYPE_BF16 ? 2 : 4;
+  g.row_bytes = D * g.esize;
+  g.n_slabs = g.row_bytes / 128;
+  g.slab_bytes = P * 128;
+  g.block_bytes = P * g.row_bytes;
+  g.page_bytes = (int64_t)cfg->num_kv_heads * 2 * g.block_bytes;
+  ctx->allocated.assign(cfg->num_pages, 0);
+  ctx->free_list.resize(cfg->num_pages);
+  for (int i = 0; i < cfg->num_pages; ++i) ctx->free_list[i] = cfg->num_pages - 1 - i;  // pop from the back: 0,1,2,..
+  ctx->wmask.assign(cfg->num_pages, 0u);
+  ctx->writer.assign(cfg->num_pages, -1);
+  ctx->host_only = cfg->device < 0;
+  if (!ctx->host_only) {
+    auto fail = [&](cudaError_t e, const char* what) {
+      (void)e;
+      (void)what;
+      if (ctx->pool) cudaFree(ctx->pool);
+      if (ctx->d_status) cudaFree(ctx->d_status);
+      delete ctx;
+      return PIE_ERR_CUDA;
+    };
+    cudaError_t e;
+    if ((e = cudaSetDevice(cfg->device)) != cudaSuccess) return fail(e, "cudaSetDevice");
+    int sms = 0;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device)) != cudaSuccess)
+      return fail(e, "attr");
+    ctx->n_sms = sms;
+    size_t bytes = (size_t)cfg->num_pages * (size_t)g.page_bytes;
+    if ((e = cudaMalloc((void**)&ctx->pool, bytes)) != cudaSuccess) return fail(e, "cudaMalloc pool");
+    if ((e = cudaMemset(ctx->pool, 0, bytes)) != cudaSuccess) return fail(e, "memset");
+    if ((e = cudaMalloc((void**)&ctx->d_status, 256)) != cudaSuccess) return fail(e, "cudaMalloc status");
+    if ((e = cudaMemset(ctx->d_status, 0, 256)) != cudaSuccess) return fail(e, "memset");
+    if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "sync");
+  }
+  *out = ctx;
+  return PIE_OK;
+}
+
+int pie_destroy(pie_ctx* ctx) {
+  if (!ctx) return PIE_ERR_INVALID;
+  if (!ctx->host_only) {
+    cudaSetDevice(ctx->cfg.device);
+    cudaDeviceSynchronize();
+    if (ctx->pool) cudaFree(ctx->pool);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->d_stage) cudaFree(ctx->d_stage);
+    if (ctx->d_io) cudaFree(ctx->d_io);
+  }
+  delete ctx;
+  return PIE_OK;
+}
+
+int pie_alloc_kvpages(pie_ctx* ctx, int32_t n, int32_t* out_ids) {
+  if (!ctx || n < 0 || (n > 0 && !out_ids)) return PIE_ERR_INVALID;
+  if ((size_t)n > ctx->free_list.size()) return PIE_ERR_NO_PAGES;
+  for (int i = 0; i < n; ++i) {
+    int32_t id = ctx->free_list.back();
+    ctx->free_list.pop_back();
+    ctx->allocated[id] = 1;
+    out_ids[i] = id;
+  }
+  return PIE_OK;
+}
+
+int pie_dealloc_kvpages(pie_ctx* ctx, int32_t n, const int32_t* ids) {
+  if (!ctx || n < 0 || (n > 0 && !ids)) return PIE_ERR_INVALID;
+  for (int i = 0; i < n; ++i) {
+    if (!page_ok(ctx, ids[i])) return PIE_ERR_BAD_PAGE;
+    for (int j = 0; j < i; ++j)  // a repeated id inside one call is a double free
+      if (ids[j] == ids[i]) return PIE_ERR_BAD_PAGE;
+  }
+  for (int i = 0; i < n; ++i) {
+    ctx->allocated[ids[i]] = 0;
+    ctx->free_list.push_back(ids[i]);
+  }
+  return PIE_OK;
+}
+
+int pie_num_free_kvpages(const pie_ctx* ctx, int32_t* out) {
+  if (!ctx || !out) return PIE_ERR_INVALID;
+  *out = (int32_t)ctx->free_list.size();
+  return PIE_OK;
+}
+
+static int page_io(pie_ctx* ctx, int32_t n, const int32_t* ids, void* K, void* V, int on_device, void* stream,
+                   bool write) {
+  if (!ctx || n < 0 || (n > 0 && (!ids || !K || !V))) return PIE_ERR_INVALID;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  for (int i = 0; i < n; ++i)
+    if (!page_ok(ctx, ids[i])) return PIE_ERR_BAD_PAGE;
+  if (n == 0) return PIE_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  const size_t canon = (size_t)ctx->geom.page_size * ctx->geom.n_kv_heads * ctx->geom.row_bytes;  // K (or V) bytes per page
+  if (on_device) {
+    int rc = ensure_buffer(ctx, &ctx->d_stage, &ctx->stage_bytes, (size_t)n * 4);
+    if (rc) return rc;
+    PIE_CUDA(ctx, cudaMemcpyAsync(ctx->d_stage, ids, (size_t)n * 4, cudaMemcpyHostToDevice, s));
+    return pie_launch_page_io(ctx, n, (const int32_t*)ctx->d_stage, K, V, write, s);
+  }
+  const int chunk = (int)std::max<size_t>(1, std::min<size_t>((size_t)n, ((size_t)64 << 20) / canon));
+  size_t ids_bytes = ((size_t)chunk * 4 + 255) & ~(size_t)255;
+  int rc = ensure_buffer(ctx, &ctx->d_stage, &ctx->stage_bytes, ids_bytes + 2 * chunk * canon);
+  if (rc) return rc;
+  uint8_t* dK = (uint8_t*)ctx->d_stage + ids_bytes;
+  uint8_t* dV = dK + (size_t)chunk * canon;
+  for (int i0 = 0; i0 < n; i0 += chunk) {
+    int m = std::min(chunk, n - i0);
+    PIE_CUDA(ctx, cudaMemcpyAsync(ctx->d_stage, ids + i0, (size_t)m * 4, cudaMemcpyHostToDevice, s));
+    if (write) {
+      PIE_CUDA(ctx, cudaMemcpyAsync(dK, (const uint8_t*)K + (size_t)i0 * canon, (size_t)m * canon, cudaMemcpyHostToDevice, s));
+      PIE_CUDA(ctx, cudaMemcpyAsync(dV, (const uint8_t*)V + (size_t)i0 * canon, (size_t)m * canon, cudaMemcpyHostToDevice, s));
+    }
+    rc = pie_launch_page_io(ctx, m, (const int32_t*)ctx->d_stage, dK, dV, write, s);
+    if (rc) return rc;
+    if (!write) {
+      PIE_CUDA(ctx, cudaMemcpyAsync((uint8_t*)K + (size_t)i0 * canon, dK, (size_t)m * canon, cudaMemcpyDeviceToHost, s));
+      PIE_CUDA(ctx, cudaMemcpyAsync((uint8_t*)V + (size_t)i0 * canon, dV, (size_t)m * canon, cudaMemcpyDeviceToHost, s));
+    }
+    PIE_CUDA(ctx, cudaStreamSynchronize(s));
+  }
+  return PIE_OK;
+}
+
+int pie_kvpage_write(pie_ctx* ctx, int32_t n, const int32_t* ids, const void* K, const void* V, int on_device,
+                     void* stream) {
+  return page_io(ctx, n, ids, const_cast<void*>(K), const_cast<void*>(V), on_device, stream, true);
+}
+
+int pie_kvpage_read(pie_ctx* ctx, int32_t n, const int32_t* ids, void* K, void* V, int on_device, void* stream) {
+  return page_io(ctx, n, ids, K, V, on_device, stream, false);
+}
+
+int pie_copy_kvpage(pie_ctx* ctx, int32_t n, const int32_t* src, const int32_t* dst, const int32_t* src_off,
+                    const int32_t* dst_off, const int32_t* ntok, void* stream) {
+  if (!ctx || n < 0 || (n > 0 && (!src || !dst || !src_off || !dst_off || !ntok))) return PIE_ERR_INVALID;
+  const int P = ctx->cfg.page_size;
+  for (int k = 0; k < n; ++k) {
+    if (!page_ok(ctx, src[k]) || !page_ok(ctx, dst[k])) return PIE_ERR_BAD_PAGE;
+    if (ntok[k] < 0 || src_off[k] < 0 || dst_off[k] < 0 || src_off[k] + ntok[k] > P || dst_off[k] + ntok[k] > P)
+      return PIE_ERR_INVALID;
+  }
+  auto bits = [](int lo, int n_) -> uint32_t {
+    if (n_ <= 0) return 0u;
+    uint32_t m = (n_ >= 32) ? 0xFFFFFFFFu : ((1u << n_) - 1u);
+    return m << lo;
+  };
+  int status = PIE_OK;
+  for (int k = 0; k < n && status == PIE_OK; ++k) {
+    uint32_t m = bits(dst_off[k], ntok[k]);
+    if (ctx->wmask[dst[k]] & m) status = PIE_ERR_CONFLICT;
+    ctx->wmask[dst[k]] |= m;
+  }
+  for (int k = 0; k < n && status == PIE_OK; ++k)
+    if (ctx->wmask[src[k]] & bits(src_off[k], ntok[k])) status = PIE_ERR_CONFLICT;
+  for (int k = 0; k < n; ++k) ctx->wmask[dst[k]] = 0;
+  if (status != PIE_OK) return status;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  if (n == 0) return PIE_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  std::vector<int32_t> ops((size_t)n * 5);
+  for (int k = 0; k < n; ++k) {
+    ops[k * 5 + 0] = src[k];
+    ops[k * 5 + 1] = dst[k];
+    ops[k * 5 + 2] = src_off[k];
+    ops[k * 5 + 3] = dst_off[k];
+    ops[k * 5 + 4] = ntok[k];
+  }
+  int rc = ensure_buffer(ctx, &ctx->d_stage, &ctx->stage_bytes, ops.size() * 4);
+  if (rc) return rc;
+  PIE_CUDA(ctx, cudaMemcpyAsync(ctx->d_stage, ops.data(), ops.size() * 4, cudaMemcpyHostToDevice, s));
+  return pie_launch_copy(ctx, n, (const int32_t*)ctx->d_stage, s);
+}
+
+int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pie_plan** out) {
+  if (!ctx || !batch || !out) return PIE_ERR_INVALID;
+  pie_plan* plan = new (std::nothrow) pie_plan();
+  if (!plan) return PIE_ERR_INVALID;
+  plan->ctx = ctx;
+  int rc = pie_build_plan(ctx, batch, plan);
+  if (rc != PIE_OK) {
+    delete plan;
+    return rc;
+  }
+  if (!ctx->host_only && plan->R > 0) {
+    cudaStream_t s = (cudaStream_t)stream;
+    // one allocation, one upload: [reqs | kept | mask | append_dst | tok_req | simple_rows |
+    // split items, cta_ptr, merges | tile items, cta_ptr, merges] then the partial workspaces.
+    std::vector<uint8_t> host;
+    auto put = [&](const void* p, size_t bytes) {
+      size_t off = (host.size() + 255) & ~(size_t)255;
+      host.resize(off + bytes);
+      if (bytes) std::memcpy(host.data() + off, p, bytes);
+      return off;
+    };
+    size_t o_reqs = put(plan->reqs.data(), plan->reqs.size() * sizeof(PieReq));
+    size_t o_kept = put(plan->kept.data(), plan->kept.size() * 4);
+    size_t o_mask = put(plan->mask_words.data(), plan->mask_words.size() * 4);
+    size_t o_app = put(plan->append_dst.data(), plan->append_dst.size() * 4);
+    size_t o_tok = put(plan->tok_req.data(), plan->tok_req.size() * 4);
+    size_t o_simple = put(plan->simple_rows.data(), plan->simple_rows.size() * 4);
+    size_t o_li[2], o_lc[2], o_lm[2];
+    PieLaunchList* lls[2] = {&plan->split, &plan->tile};
+    for (int k = 0; k < 2; ++k) {
+      o_li[k] = put(lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
+      o_lc[k] = put(lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
+      o_lm[k] = put(lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
+    }
+    size_t upload = (host.size() + 255) & ~(size_t)255;
+    size_t total = upload;
+    size_t o_wo[2], o_wl[2];
+    const int D = ctx->cfg.head_dim;
+    for (int k = 0; k < 2; ++k) {
+      o_wo[k] = total;
+      total += (((size_t)lls[k]->n_slots * lls[k]->slot_rows * D * 4) + 255) & ~(size_t)255;
+      o_wl[k] = total;
+      total += (((size_t)lls[k]->n_slots * lls[k]->slot_rows * 4) + 255) & ~(size_t)255;
+    }
+    cudaError_t e = cudaSetDevice(ctx->cfg.device);
+    if (e == cudaSuccess) e = cudaMalloc(&plan->d_blob, std::max<size_t>(total, 256));
+    if (e == cudaSuccess && !host.empty())
+      e = cudaMemcpyAsync(plan->d_blob, host.data(), host.size(), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+      ctx->cuda_error = std::string("plan upload: ") + cudaGetErrorString(e);
+      if (plan->d_blob) cudaFree(plan->d_blob);
+      delete plan;
+      return PIE_ERR_CUDA;
+    }
+    uint8_t* base = (uint8_t*)plan->d_blob;
+    plan->d_reqs = (PieReq*)(base + o_reqs);
+    plan->d_kept = (int2*)(base + o_kept);
+    plan->d_mask = (uint32_t*)(base + o_mask);
+    plan->d_append_dst = (int32_t*)(base + o_app);
+    plan->d_tok_req = (int32_t*)(base + o_tok);
+    plan->d_simple_rows = (int32_t*)(base + o_simple);
+    for (int k = 0; k < 2; ++k) {
+      lls[k]->d_items = (PieItem*)(base + o_li[k]);
+      lls[k]->d_cta_ptr = (int32_t*)(base + o_lc[k]);
+      lls[k]->d_merges = (PieMerge*)(base + o_lm[k]);
+      lls[k]->d_ws_o = (float*)(base + o_wo[k]);
+      lls[k]->d_ws_lse = (float*)(base + o_wl[k]);
+    }
+  }
+  *out = plan;
+  return PIE_OK;
+}
+
+int pie_plan_destroy(pie_plan* plan) {
+  if (!plan) return PIE_ERR_INVALID;
+  if (plan->d_blob) {
+    cudaSetDevice(plan->ctx->cfg.device);
+    cudaFree(plan->d_blob);
+  }
+  delete plan;
+  return PIE_OK;
+}
+
+int pie_plan_get_info(const pie_plan* plan, pie_plan_info* out) {
+  if (!plan || !out) return PIE_ERR_INVALID;
+  *out = plan->info;
+  return PIE_OK;
+}
+
+int pie_plan_debug_read(const pie_plan* plan, int which, void* buf, int64_t cap_bytes, int64_t* out_bytes) {
+  if (!plan || !out_bytes) return PIE_ERR_INVALID;
+  const void* p = nullptr;
+  int64_t n = 0;
+  switch (which) {
+    case 0: p = plan->mask_words.data(); n = (int64_t)plan->mask_words.size() * 4; break;
+    case 1: p = plan->kept.data(); n = (int64_t)plan->kept.size() * 4; break;
+    case 2: p = plan->append_dst.data(); n = (int64_t)plan->append_dst.size() * 4; break;
+    default: return PIE_ERR_INVALID;
+  }
+  *out_bytes = n;
+  if (buf && cap_bytes >= n && n > 0) std::memcpy(buf, p, (size_t)n);
+  return PIE_OK;
+}
+
+int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new, const void* v_new, void* out,
+                float* lse, void* stream) {
+  if (!ctx || !plan || plan->ctx != ctx) return PIE_ERR_INVALID;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  if (plan->T == 0) return PIE_OK;
+  if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
+  cudaStream_t s = (cudaStream_t)stream;
+  PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  int rc = pie_launch_append(ctx, plan, k_new, v_new, s);
+  if (rc) return rc;
+  if (!plan->simple_rows.empty() && (rc = pie_launch_simple(ctx, plan, q, out, lse, s))) return rc;
+  if (!plan->split.items.empty() && (rc = pie_launch_split(ctx, plan, q, out, lse, s))) return rc;
+  if (!plan->tile.items.empty() && (rc = pie_launch_tiles(ctx, plan, q, out, lse, s))) return rc;
+  if (!plan->split.merges.empty() && (rc = pie_launch_merge(ctx, plan, plan->split, out, lse, s))) return rc;
+  if (!plan->tile.merges.empty() && (rc = pie_launch_merge(ctx, plan, plan->tile, out, lse, s))) return rc;
+  return PIE_OK;
+}
+
+int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, const void* k_new, const void* v_new,
+                     void* out, float* lse, void* stream) {
+  if (!ctx || !batch) return PIE_ERR_INVALID;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  pie_plan* plan = nullptr;
+  int rc = pie_plan_forward(ctx, batch, stream, &plan);
+  if (rc) return rc;
+  if (plan->T == 0) {
+    pie_plan_destroy(plan);
+    return PIE_OK;
+  }
+  if (!q || !k_new || !v_new || !out || !lse) {
+    pie_plan_destroy(plan);
+    return PIE_ERR_INVALID;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t T = plan->T, es = ctx->geom.esize, D = ctx->cfg.head_dim;
+  const size_t qb = (T * ctx->cfg.num_q_heads * D * es + 255) & ~(size_t)255;
+  const size_t kb = (T * ctx->cfg.num_kv_heads * D * es + 255) & ~(size_t)255;
+  const size_t lb = (T * ctx->cfg.num_q_heads * 4 + 255) & ~(size_t)255;
+  auto body = [&]() -> int {
+    int rc2 = ensure_buffer(ctx, &ctx->d_io, &ctx->io_bytes, 2 * qb + 2 * kb + lb);
+    if (rc2) return rc2;
+    uint8_t* dq = (uint8_t*)ctx->d_io;
+    uint8_t *dk = dq + qb, *dv = dk + kb, *dout = dv + kb, *dl = dout + qb;
+    PIE_CUDA(ctx, cudaMemcpyAsync(dq, q, T * ctx->cfg.num_q_heads * D * es, cudaMemcpyHostToDevice, s));
+    PIE_CUDA(ctx, cudaMemcpyAsync(dk, k_new, T * ctx->cfg.num_kv_heads * D * es, cudaMemcpyHostToDevice, s));
+    PIE_CUDA(ctx, cudaMemcpyAsync(dv, v_new, T * ctx->cfg.num_kv_heads * D * es, cudaMemcpyHostToDevice, s));
+    rc2 = pie_forward(ctx, plan, dq, dk, dv, dout, (float*)dl, stream);
+    if (rc2) return rc2;
+    PIE_CUDA(ctx, cudaMemcpyAsync(out, dout, T * ctx->cfg.num_q_heads * D * es, cudaMemcpyDeviceToHost, s));
+    PIE_CUDA(ctx, cudaMemcpyAsync(lse, dl, T * ctx->cfg.num_q_heads * 4, cudaMemcpyDeviceToHost, s));
+    PIE_CUDA(ctx, cudaStreamSynchronize(s));
+    return PIE_OK;
+  };
+  rc = body();
+  pie_plan_destroy(plan);
+  return rc;
+}
+
+int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out) {
+  if (!ctx || !out) return PIE_ERR_INVALID;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  cudaStream_t s = (cudaStream_t)stream;
+  PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  int v = 0;
+  PIE_CUDA(ctx, cudaMemcpyAsync(&v, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  PIE_CUDA(ctx, cudaStreamSynchronize(s));
+  if (v != 0) {
+    PIE_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int), s));
+    PIE_CUDA(ctx, cudaStreamSynchronize(s));
+  }
+  *out = v;
+  return PIE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,597 @@
+// Attention kernels of the `forward` handler (Section 4.2 "Forward API": attention over the
+// request's KvPages under an explicit or inferred mask):
+//   * attn_mma_kernel<SPLIT=true>  - decode: split-KV over scattered pages, HBM bound.  A
+//     producer warp streams (page, kv head) blocks into a deep shared-memory ring with bulk
+//     async copies; consumer warps take pages round-robin, run QK^T / PV on tensor cores with
+//     the grouped query heads stacked in the M dimension, and keep private online-softmax
+//     states that are merged once per work item.
+//   * attn_mma_kernel<SPLIT=false> - row tiles (prefill chunks, token trees): each consumer warp
+//     owns 16 query rows and every warp walks the same page stream.
+//   * merge_kernel                 - LSE-weighted merge of split partials.
+//   * simple_kernel                - plain CUDA-core kernel (fp32 pools and shapes the tile
+//     kernels do not cover); one warp per (token, head) row, sequential online softmax.
+#include <cuda_bf16.h>
+
+#include "pie_internal.h"
+
+namespace {
+
+// ------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after ~2 s, records the failure in the status word and returns false.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status) {
+  const uint64_t t0 = global_ns();
+  while (!mbar_try_wait(bar, parity)) {
+    if (global_ns() - t0 > 2000000000ull) {
+      atomicExch(status, (int)PIE_ERR_DEVICE_TIMEOUT);
+      return false;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, status);
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+constexpr float kNegInf = -__builtin_huge_valf();
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ------------------------------------------------------------------------------ tile kernel
+template <int D, int P, int NW, bool SPLIT, int NSTAGES>
+struct TileCfg {
+  static constexpr int BLK = P * D * 2;       // one K (or V) block, bytes
+  static constexpr int STAGE = 2 * BLK;       // K block then V block
+  static constexpr int SLAB = P * 128;
+  static constexpr int OROW = D + 8;          // padded fp32 row of the cross-warp merge area
+  static constexpr int MERGE_FLOATS = SPLIT ? NW * (16 * OROW + 32) : 0;
+  static constexpr int SMEM = NSTAGES * STAGE + 2 * NSTAGES * 8 + MERGE_FLOATS * 4 + 64;
+};
+
+template <int D, int P, int NW, bool SPLIT, int NSTAGES>
+__global__ void __launch_bounds__((NW + 1) * 32, 1) attn_mma_kernel(const AttnParams p) {
+  using C = TileCfg<D, P, NW, SPLIT, NSTAGES>;
+  constexpr int KSTEPS = D / 16;   // k-steps of QK^T, and 16-column groups of PV
+  constexpr int SUBS = P / 16;     // 16-token sub-tiles per page
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint8_t* stages = smem;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + NSTAGES * C::STAGE);
+  uint64_t* empty_bar = full_bar + NSTAGES;
+  float* merge = reinterpret_cast<float*>(empty_bar + NSTAGES);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NSTAGES; ++s) {
+      mbar_init(smem_u32(full_bar + s), 1);
+      mbar_init(smem_u32(empty_bar + s), SPLIT ? 1 : NW);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const int it0 = p.cta_ptr[blockIdx.x], it1 = p.cta_ptr[blockIdx.x + 1];
+
+  if (warp == NW) {
+    // ------------------------------------------------------------------ producer (one lane)
+    if (lane == 0) {
+      uint32_t cnt = 0;
+      for (int it = it0; it < it1; ++it) {
+        const PieItem item = p.items[it];
+        const uint8_t* base = p.pool + (int64_t)item.kv_head * C::STAGE;
+        for (int k = item.page_begin; k < item.page_end; ++k, ++cnt) {
+          const uint32_t s = cnt % NSTAGES, ph = (cnt / NSTAGES) & 1;
+          const int phys = p.kept[k].x;
+          mbar_wait(smem_u32(empty_bar + s), ph ^ 1, p.status);
+          mbar_expect_tx(smem_u32(full_bar + s), C::STAGE);
+          bulk_g2s(smem_u32(stages + s * C::STAGE), base + (int64_t)phys * p.page_bytes, C::STAGE,
+                   smem_u32(full_bar + s));
+        }
+      }
+    }
+    return;
+  }
+
+  // ---------------------------------------------------------------------- consumers
+  const int G = p.G;
+  const int r_lo = lane >> 2;            // this thread's rows: r_lo and r_lo + 8
+  const int cpair = (lane & 3) * 2;      // its columns inside an 8-wide block: cpair, cpair + 1
+  uint32_t cnt_base = 0;
+
+  for (int it = it0; it < it1; ++it) {
+    const PieItem item = p.items[it];
+    const PieReq rq = p.reqs[item.req];
+    const int rbase = item.row0 + (SPLIT ? 0 : warp * 16);
+    const int row_end = item.row0 + item.nrows;
+    const bool explicit_mask = rq.mask_row_words != 0;
+
+    bool valid[2];
+    int lim[2];
+    const uint32_t* mrow[2];
+    const __nv_bfloat16* qptr[2];
+    for (int r = 0; r < 2; ++r) {
+      const int gr = rbase + r_lo + r * 8;
+      valid[r] = gr < row_end;
+      const int tok = valid[r] ? gr / G : 0;
+      const int head = item.kv_head * G + (valid[r] ? gr % G : 0);
+      lim[r] = valid[r] ? rq.kv_len - rq.q_len + tok : -1;
+      mrow[r] = p.mask + rq.mask_word_off + (int64_t)tok * rq.mask_row_words;
+      qptr[r] = reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)(rq.q_start + tok) * p.n_q_heads + head) * D;
+    }
+    const bool warp_has_rows = rbase < row_end;
+
+    // Q fragments (A operand, 16 rows x D)
+    uint32_t qf[KSTEPS][4];
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        uint32_t lo = 0, hi = 0;
+        if (valid[r]) {
+          lo = *reinterpret_cast<const uint32_t*>(qptr[r] + ks * 16 + cpair);
+          hi = *reinterpret_cast<const uint32_t*>(qptr[r] + ks * 16 + 8 + cpair);
+        }
+        qf[ks][r] = lo;
+        qf[ks][2 + r] = hi;
+      }
+    }
+
+    float m_run[2] = {kNegInf, kNegInf}, l_run[2] = {0.f, 0.f};
+    float o[D / 8][4];
+#pragma unroll
+    for (int nb = 0; nb < D / 8; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
+
+    const int npages = item.page_end - item.page_begin;
+    for (int kk = 0; kk < npages; ++kk) {
+      if (SPLIT && (kk % NW) != warp) continue;
+      const uint32_t cnt = cnt_base + kk;
+      const uint32_t s = cnt % NSTAGES, ph = (cnt / NSTAGES) & 1;
+      const uint32_t lpf = (uint32_t)p.kept[item.page_begin + kk].y;
+      const int lp = (int)(lpf & ~PIE_KEPT_NEEDS_MASK);
+      const bool needs_mask = (lpf & PIE_KEPT_NEEDS_MASK) != 0;
+      mbar_wait(smem_u32(full_bar + s), ph, p.status);
+      const uint32_t kbase = smem_u32(stages + s * C::STAGE);
+      const uint32_t vbase = kbase + C::BLK;
+
+      if (lp == rq.last_logical && rq.last_page_len < P) {
+        // slots past the end of the context may hold anything: clear their V rows so that a
+        // zero probability times a NaN bit pattern cannot leak into the output
+        constexpr int CH = D * 2 / 16;
+        uint8_t* v = stages + s * C::STAGE + C::BLK;
+        const int nz = (P - rq.last_page_len) * CH;
+        for (int c = lane; c < nz; c += 32) {
+          const int t = rq.last_page_len + c / CH, ch = c % CH;
+          *reinterpret_cast<uint4*>(v + pie_chunk_offset(C::SLAB, t, ch)) = make_uint4(0, 0, 0, 0);
+        }
+        __syncwarp();
+      }
+
+      if (warp_has_rows) {
+#pragma unroll
+        for (int sub = 0; sub < SUBS; ++sub) {
+          const int j0 = lp * P + sub * 16;
+          uint32_t bits[2] = {0xFFFFu, 0xFFFFu};
+          if (needs_mask) {
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+              if (!valid[r]) bits[r] = 0;
+              else if (explicit_mask) bits[r] = (__ldg(mrow[r] + (j0 >> 5)) >> (j0 & 31)) & 0xFFFFu;
+              else bits[r] = lim[r] >= j0 + 15 ? 0xFFFFu : (lim[r] < j0 ? 0u : ((1u << (lim[r] - j0 + 1)) - 1u));
+            }
+            if (__all_sync(0xFFFFFFFFu, (bits[0] | bits[1]) == 0)) continue;  // nothing visible to this warp
+          }
+          // ---- S = Q K^T for 16 tokens
+          float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+          {
+            const int t = sub * 16 + ((lane >> 4) << 3) + (lane & 7);
+            const uint32_t rowaddr = kbase + t * 128;
+            const int csel = (lane >> 3) & 1;
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+              const int c = (ks & 3) * 2 + csel;
+              uint32_t b0, b1, b2, b3;
+              ldsm_x4(rowaddr + (ks >> 2) * C::SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
+              mma_bf16(sacc[0], qf[ks], b0, b1);
+              mma_bf16(sacc[1], qf[ks], b2, b3);
+            }
+          }
+          // ---- mask, online softmax (base-2 domain)
+          float mx[2] = {kNegInf, kNegInf};
+#pragma unroll
+          for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int r = e >> 1, col = nb * 8 + cpair + (e & 1);
+              float v = sacc[nb][e] * p.scale_log2;
+              if (needs_mask && !((bits[r] >> col) & 1u)) v = kNegInf;
+              sacc[nb][e] = v;
+              mx[r] = fmaxf(mx[r], v);
+            }
+          float alpha[2], m_use[2];
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], 1));
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], 2));
+            const float m_new = fmaxf(m_run[r], mx[r]);
+            m_use[r] = (m_new == kNegInf) ? 0.f : m_new;
+            alpha[r] = fast_exp2(m_run[r] - m_use[r]);
+            m_run[r] = m_new;
+          }
+          float psum[2] = {0.f, 0.f};
+#pragma unroll
+          for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float pv = fast_exp2(sacc[nb][e] - m_use[e >> 1]);
+              sacc[nb][e] = pv;
+              psum[e >> 1] += pv;
+            }
+          l_run[0] = l_run[0] * alpha[0] + psum[0];
+          l_run[1] = l_run[1] * alpha[1] + psum[1];
+#pragma unroll
+          for (int nb = 0; nb < D / 8; ++nb) {
+            o[nb][0] *= alpha[0];
+            o[nb][1] *= alpha[0];
+            o[nb][2] *= alpha[1];
+            o[nb][3] *= alpha[1];
+          }
+          uint32_t pa[4];
+          pa[0] = pack_bf16(sacc[0][0], sacc[0][1]);
+          pa[1] = pack_bf16(sacc[0][2], sacc[0][3]);
+          pa[2] = pack_bf16(sacc[1][0], sacc[1][1]);
+          pa[3] = pack_bf16(sacc[1][2], sacc[1][3]);
+          // ---- O += P V
+          {
+            const int t = sub * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
+            const uint32_t rowaddr = vbase + t * 128;
+            const int csel = lane >> 4;
+#pragma unroll
+            for (int db = 0; db < KSTEPS; ++db) {
+              const int c = (db & 3) * 2 + csel;
+              uint32_t b0, b1, b2, b3;
+              ldsm_x4_t(rowaddr + (db >> 2) * C::SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
+              mma_bf16(o[2 * db], pa, b0, b1);
+              mma_bf16(o[2 * db + 1], pa, b2, b3);
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(empty_bar + s));
+    }
+    cnt_base += npages;
+
+    // ---- row sums across the quad
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, l_run[r], 1);
+      l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, l_run[r], 2);
+    }
+
+    if constexpr (SPLIT) {
+      // ---- merge the NW private softmax states of this item
+      float* wm = merge + warp * (16 * C::OROW + 32);
+      float* wl = wm + 16;
+      float* wo = wm + 32;
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int row = r_lo + r * 8;
+        if ((lane & 3) == 0) {
+          wm[row] = m_run[r];
+          wl[row] = l_run[r];
+        }
+#pragma unroll
+        for (int nb = 0; nb < D / 8; ++nb)
+          *reinterpret_cast<float2*>(wo + row * C::OROW + nb * 8 + cpair) = make_float2(o[nb][2 * r], o[nb][2 * r + 1]);
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+      const int tid = threadIdx.x;
+      for (int e = tid; e < item.nrows * (D / 2); e += NW * 32) {
+        const int row = e / (D / 2), d = (e % (D / 2)) * 2;
+        float M = kNegInf;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) M = fmaxf(M, merge[w * (16 * C::OROW + 32) + row]);
+        float L = 0.f, a0 = 0.f, a1 = 0.f;
+        if (M != kNegInf) {
+#pragma unroll
+          for (int w = 0; w < NW; ++w) {
+            const float* b = merge + w * (16 * C::OROW + 32);
+            const float sc = fast_exp2(b[row] - M);
+            L += b[16 + row] * sc;
+            const float2 ov = *reinterpret_cast<const float2*>(b + 32 + row * C::OROW + d);
+            a0 += ov.x * sc;
+            a1 += ov.y * sc;
+          }
+        }
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : kNegInf;
+        const int gr = item.row0 + row;
+        const int tok = gr / G, head = item.kv_head * G + gr % G;
+        if (item.partial_slot < 0) {
+          const int64_t oi = ((int64_t)(rq.q_start + tok) * p.n_q_heads + head);
+          *reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D + d) = pack_bf16(a0 * inv, a1 * inv);
+          if (d == 0) p.lse[oi] = lse;
+        } else {
+          const int64_t si = (int64_t)item.partial_slot * 16 + row;
+          *reinterpret_cast<float2*>(p.ws_o + si * D + d) = make_float2(a0 * inv, a1 * inv);
+          if (d == 0) p.ws_lse[si] = lse;
+        }
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+    } else {
+      // ---- each warp owns its rows: write straight from registers
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        if (!valid[r]) continue;
+        const int gr = rbase + r_lo + r * 8;
+        const int tok = gr / G, head = item.kv_head * G + gr % G;
+        const float L = l_run[r];
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        const float lse = L > 0.f ? (m_run[r] + log2f(L)) * kLn2 : kNegInf;
+        if (item.partial_slot < 0) {
+          const int64_t oi = ((int64_t)(rq.q_start + tok) * p.n_q_heads + head);
+          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D;
+#pragma unroll
+          for (int nb = 0; nb < D / 8; ++nb)
+            *reinterpret_cast<uint32_t*>(dst + nb * 8 + cpair) = pack_bf16(o[nb][2 * r] * inv, o[nb][2 * r + 1] * inv);
+          if ((lane & 3) == 0) p.lse[oi] = lse;
+        } else {
+          const int64_t si = (int64_t)item.partial_slot * (NW * 16) + (gr - item.row0);
+          float* dst = p.ws_o + si * D;
+#pragma unroll
+          for (int nb = 0; nb < D / 8; ++nb)
+            *reinterpret_cast<float2*>(dst + nb * 8 + cpair) = make_float2(o[nb][2 * r] * inv, o[nb][2 * r + 1] * inv);
+          if ((lane & 3) == 0) p.ws_lse[si] = lse;
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------ merge kernel
+// lse = ln sum_c exp(lse_c), o = sum_c exp(lse_c - lse) o_c over the partial slots of a group.
+template <typename T>
+__global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* __restrict__ reqs,
+                             const float* __restrict__ ws_o, const float* __restrict__ ws_lse, T* __restrict__ out,
+                             float* __restrict__ lse_out, int slot_rows, int D, int n_q_heads, int G) {
+  const PieMerge mg = merges[blockIdx.x];
+  const PieReq rq = reqs[mg.req];
+  for (int e = threadIdx.x; e < mg.nrows * D; e += blockDim.x) {
+    const int row = e / D, d = e - row * D;
+    float M = kNegInf;
+    for (int c = 0; c < mg.nslots; ++c) M = fmaxf(M, ws_lse[(int64_t)(mg.slot0 + c) * slot_rows + row]);
+    float Z = 0.f, acc = 0.f;
+    if (M != kNegInf) {
+      for (int c = 0; c < mg.nslots; ++c) {
+        const int64_t si = (int64_t)(mg.slot0 + c) * slot_rows + row;
+        const float w = __expf(ws_lse[si] - M);
+        Z += w;
+        acc += w * ws_o[si * D + d];
+      }
+    }
+    const int gr = mg.row0 + row;
+    const int tok = gr / G, head = mg.kv_head * G + gr % G;
+    const int64_t oi = (int64_t)(rq.q_start + tok) * n_q_heads + head;
+    out[oi * D + d] = (T)(Z > 0.f ? acc / Z : 0.f);
+    if (d == 0) lse_out[oi] = Z > 0.f ? M + logf(Z) : kNegInf;
+  }
+}
+
+// ------------------------------------------------------------------------------ simple kernel
+template <typename T>
+__device__ __forceinline__ float to_f32(T v);
+template <>
+__device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T, int D>
+__global__ void simple_kernel(const uint8_t* __restrict__ pool, const T* __restrict__ q, T* __restrict__ out,
+                              float* __restrict__ lse_out, const PieReq* __restrict__ reqs,
+                              const int2* __restrict__ kept, const uint32_t* __restrict__ mask,
+                              const int32_t* __restrict__ tok_req, const int32_t* __restrict__ rows, int n_rows,
+                              PoolGeom g, int n_q_heads, int G, float scale) {
+  constexpr int EPL = D / 32;  // elements per lane
+  const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (wid >= n_rows) return;
+  const int row = rows[wid];
+  const int t = row / n_q_heads, h = row - t * n_q_heads;
+  const PieReq rq = reqs[tok_req[t]];
+  const int i = t - rq.q_start, kvh = h / G;
+  const int lim = rq.kv_len - rq.q_len + i;
+  const uint32_t* mrow = mask + rq.mask_word_off + (int64_t)i * rq.mask_row_words;
+  float qv[EPL], acc[EPL];
+  for (int e = 0; e < EPL; ++e) {
+    qv[e] = to_f32<T>(q[(int64_t)row * D + lane * EPL + e]);
+    acc[e] = 0.f;
+  }
+  const int byte_off = lane * EPL * (int)sizeof(T);
+  const int chunk = byte_off >> 4, within = byte_off & 15;
+  float m = kNegInf, l = 0.f;
+  for (int k = 0; k < rq.kept_count; ++k) {
+    const int2 kp = kept[rq.kept_start + k];
+    const int lp = (int)((uint32_t)kp.y & ~PIE_KEPT_NEEDS_MASK);
+    const uint8_t* blockK = pool + (int64_t)kp.x * g.page_bytes + (int64_t)(kvh * 2) * g.block_bytes;
+    const uint8_t* blockV = blockK + g.block_bytes;
+    for (int slot = 0; slot < g.page_size; ++slot) {
+      const int j = lp * g.page_size + slot;
+      if (j >= rq.kv_len) break;
+      const bool allowed = rq.mask_row_words ? ((mrow[j >> 5] >> (j & 31)) & 1u) : (j <= lim);
+      if (!allowed) continue;
+      const int off = pie_chunk_offset(g.slab_bytes, slot, chunk) + within;
+      const T* kp_ = reinterpret_cast<const T*>(blockK + off);
+      const T* vp_ = reinterpret_cast<const T*>(blockV + off);
+      float dot = 0.f;
+      for (int e = 0; e < EPL; ++e) dot += qv[e] * to_f32<T>(kp_[e]);
+      for (int sft = 16; sft > 0; sft >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, sft);
+      const float s = dot * scale;
+      const float m_new = fmaxf(m, s);
+      const float a = expf(m - m_new), pw = expf(s - m_new);
+      l = l * a + pw;
+      for (int e = 0; e < EPL; ++e) acc[e] = acc[e] * a + pw * to_f32<T>(vp_[e]);
+      m = m_new;
+    }
+  }
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  for (int e = 0; e < EPL; ++e) out[(int64_t)row * D + lane * EPL + e] = (T)(acc[e] * inv);
+  if (lane == 0) lse_out[row] = l > 0.f ? m + logf(l) : kNegInf;
+}
+
+// ------------------------------------------------------------------------------ launchers
+AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, const void* q, void* out,
+                       float* lse) {
+  AttnParams p{};
+  p.pool = ctx->pool;
+  p.q = q;
+  p.out = out;
+  p.lse = lse;
+  p.reqs = plan->d_reqs;
+  p.kept = plan->d_kept;
+  p.mask = plan->d_mask;
+  p.items = ll.d_items;
+  p.cta_ptr = ll.d_cta_ptr;
+  p.ws_o = ll.d_ws_o;
+  p.ws_lse = ll.d_ws_lse;
+  p.status = ctx->d_status;
+  p.page_bytes = ctx->geom.page_bytes;
+  p.n_q_heads = ctx->cfg.num_q_heads;
+  p.n_kv_heads = ctx->cfg.num_kv_heads;
+  p.G = ctx->G;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)ctx->cfg.head_dim);
+  return p;
+}
+
+template <int D, int P, int NW, bool SPLIT>
+int launch_tile_kernel(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
+  constexpr int NSTAGES = (128 * 1024) / (2 * P * D * 2);
+  using C = TileCfg<D, P, NW, SPLIT, NSTAGES>;
+  auto kern = attn_mma_kernel<D, P, NW, SPLIT, NSTAGES>;
+  static bool configured[8] = {};
+  int dev = ctx->cfg.device & 7;
+  if (!configured[dev]) {
+    PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+    configured[dev] = true;
+  }
+  kern<<<grid, (NW + 1) * 32, C::SMEM, s>>>(p);
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}
+
+template <bool SPLIT, int NW>
+int dispatch_tile(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
+  const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size;
+  if (D == 64 && P == 16) return launch_tile_kernel<64, 16, NW, SPLIT>(ctx, p, grid, s);
+  if (D == 128 && P == 16) return launch_tile_kernel<128, 16, NW, SPLIT>(ctx, p, grid, s);
+  if (D == 64 && P == 32) return launch_tile_kernel<64, 32, NW, SPLIT>(ctx, p, grid, s);
+  if (D == 128 && P == 32) return launch_tile_kernel<128, 32, NW, SPLIT>(ctx, p, grid, s);
+  return PIE_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+bool pie_split_supported(const pie_ctx* ctx) {
+  const pie_config& c = ctx->cfg;
+  return c.dtype == PIE_DTYPE_BF16 && (c.page_size == 16 || c.page_size == 32) && (c.head_dim == 64 || c.head_dim == 128) &&
+         ctx->G <= 16;
+}
+
+int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s) {
+  AttnParams p = make_params(ctx, plan, plan->split, q, out, lse);
+  return dispatch_tile<true, 8>(ctx, p, plan->split.grid, s);
+}
+
+int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s) {
+  AttnParams p = make_params(ctx, plan, plan->tile, q, out, lse);
+  return dispatch_tile<false, 4>(ctx, p, plan->tile.grid, s);
+}
+
+int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s) {
+  const int D = ctx->cfg.head_dim;
+  const int n = (int)ll.merges.size();
+  if (ctx->cfg.dtype == PIE_DTYPE_BF16)
+    merge_kernel<__nv_bfloat16><<<n, 256, 0, s>>>(ll.d_merges, plan->d_reqs, ll.d_ws_o, ll.d_ws_lse, (__nv_bfloat16*)out, lse,
+                                                   ll.slot_rows, D, ctx->cfg.num_q_heads, ctx->G);
+  else
+    merge_kernel<float><<<n, 256, 0, s>>>(ll.d_merges, plan->d_reqs, ll.d_ws_o, ll.d_ws_lse, (float*)out, lse, ll.slot_rows, D,
+                                           ctx->cfg.num_q_heads, ctx->G);
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}
+
+int pie_launch_simple(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s) {
+  const int n = (int)plan->simple_rows.size();
+  const int D = ctx->cfg.head_dim;
+  const float scale = 1.f / sqrtf((float)D);
+  const int threads = 128, grid = (n * 32 + threads - 1) / threads;
+#define PIE_SIMPLE(T, DD)                                                                                              \
+  simple_kernel<T, DD><<<grid, threads, 0, s>>>(ctx->pool, (const T*)q, (T*)out, lse, plan->d_reqs, plan->d_kept,      \
+                                                plan->d_mask, plan->d_tok_req, plan->d_simple_rows, n, ctx->geom,      \
+                                                ctx->cfg.num_q_heads, ctx->G, scale)
+  if (ctx->cfg.dtype == PIE_DTYPE_BF16) {
+    if (D == 64) PIE_SIMPLE(__nv_bfloat16, 64);
+    else PIE_SIMPLE(__nv_bfloat16, 128);
+  } else {
+    if (D == 64) PIE_SIMPLE(float, 64);
+    else PIE_SIMPLE(float, 128);
+  }
+#undef PIE_SIMPLE
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}

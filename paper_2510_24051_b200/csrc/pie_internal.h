@@ -1,0 +1,164 @@
+// Internal structures shared by the host code and the kernels of libpie_b200.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "pie_b200.h"
+
+// ---------------------------------------------------------------------------------------------
+// KvPage pool layout (private to the library).
+//
+//   pool[page][kv_head][K|V][slab][slot][128 bytes]
+//
+// A "block" is the K (or V) data of one (page, kv head): page_size rows of D elements.  Each
+// row is cut into 128-byte slabs; inside a slab the eight 16-byte chunks of row `slot` are
+// stored at chunk position (chunk ^ (slot & 7)).  This is exactly the 128-byte shared-memory
+// swizzle that ldmatrix and the tcgen05 matrix descriptors want, so a plain linear bulk copy of
+// a block lands in shared memory bank-conflict free and MMA ready, with no tensor map.
+// K and V of the same (page, head) are adjacent: one copy of 2 blocks feeds one attention step.
+// ---------------------------------------------------------------------------------------------
+struct PoolGeom {
+  int32_t page_size, n_kv_heads, head_dim, esize;
+  int32_t row_bytes;    // D * esize
+  int32_t n_slabs;      // row_bytes / 128
+  int32_t slab_bytes;   // page_size * 128
+  int32_t block_bytes;  // page_size * row_bytes
+  int64_t page_bytes;   // n_kv_heads * 2 * block_bytes
+};
+
+// Byte offset inside a block of the 16-byte chunk `chunk` (0 .. row_bytes/16) of row `slot`.
+__host__ __device__ inline int32_t pie_chunk_offset(int32_t slab_bytes, int32_t slot, int32_t chunk) {
+  return (chunk >> 3) * slab_bytes + slot * 128 + (((chunk & 7) ^ (slot & 7)) << 4);
+}
+
+// Per-request record read by the attention kernels.
+struct PieReq {
+  int32_t q_start;         // first query token (qo_indptr[r])
+  int32_t q_len;
+  int32_t kv_len;
+  int32_t kept_start;      // first entry in the kept-page list
+  int32_t kept_count;
+  int32_t mask_row_words;  // 0: causal mask inferred from positions
+  int64_t mask_word_off;   // first packed mask word of this request
+  int32_t last_logical;    // logical index of the last page
+  int32_t last_page_len;
+};
+
+// One unit of work of a tile kernel: rows [row0, row0+nrows) of the request's (token, head-in-
+// group) row space for one kv head, attended over kept pages [page_begin, page_end).
+struct PieItem {
+  int32_t req, kv_head, row0, nrows;
+  int32_t page_begin, page_end;  // absolute indices into the kept-page list
+  int32_t partial_slot;          // -1: write the final output; else slot of the fp32 partial
+  int32_t pad;
+};
+
+// A group of partial slots that the merge kernel combines into final rows.
+struct PieMerge {
+  int32_t req, kv_head, row0, nrows;
+  int32_t slot0, nslots;
+};
+
+#define PIE_KEPT_NEEDS_MASK 0x80000000u
+
+struct PieLaunchList {           // one tile-kernel launch (split-KV decode, or row tiles)
+  std::vector<PieItem> items;
+  std::vector<int32_t> cta_ptr;  // [grid+1] items of each CTA
+  std::vector<PieMerge> merges;
+  int32_t grid = 0;
+  int32_t n_slots = 0;
+  int32_t slot_rows = 0;
+  // device copies
+  PieItem* d_items = nullptr;
+  int32_t* d_cta_ptr = nullptr;
+  PieMerge* d_merges = nullptr;
+  float* d_ws_o = nullptr;       // [n_slots][slot_rows][D]
+  float* d_ws_lse = nullptr;     // [n_slots][slot_rows]
+};
+
+struct pie_plan {
+  pie_ctx* ctx = nullptr;
+  uint32_t flags = 0;
+  int32_t R = 0, T = 0;
+  std::vector<PieReq> reqs;
+  std::vector<int32_t> kept;        // pairs (phys, logical|flag)
+  std::vector<uint32_t> mask_words;
+  std::vector<int32_t> append_dst;  // [T] page*P + slot
+  std::vector<int32_t> tok_req;     // [T]
+  std::vector<int32_t> simple_rows; // (token*H_q + head) rows for the plain kernel
+  PieLaunchList split, tile;
+  pie_plan_info info{};
+  // device
+  void* d_blob = nullptr;           // one allocation holding every array below
+  PieReq* d_reqs = nullptr;
+  int2* d_kept = nullptr;
+  uint32_t* d_mask = nullptr;
+  int32_t* d_append_dst = nullptr;
+  int32_t* d_tok_req = nullptr;
+  int32_t* d_simple_rows = nullptr;
+};
+
+struct pie_ctx {
+  pie_config cfg{};
+  PoolGeom geom{};
+  int32_t G = 1;
+  int32_t n_sms = 148;
+  bool host_only = false;
+  // allocator
+  std::vector<int32_t> free_list;
+  std::vector<uint8_t> allocated;
+  // device
+  uint8_t* pool = nullptr;
+  int* d_status = nullptr;
+  void* d_stage = nullptr;  // staging for host <-> device calls
+  size_t stage_bytes = 0;
+  void* d_io = nullptr;     // q/k/v/out/lse staging of pie_forward_host
+  size_t io_bytes = 0;
+  std::string cuda_error;
+  // scratch for validation (sized num_pages)
+  std::vector<uint32_t> wmask;
+  std::vector<int32_t> writer;
+};
+
+// ---- kernels (defined in the .cu files) --------------------------------------------------------
+struct AttnParams {
+  const uint8_t* pool;
+  const void* q;
+  void* out;
+  float* lse;
+  const PieReq* reqs;
+  const int2* kept;
+  const uint32_t* mask;
+  const PieItem* items;
+  const int32_t* cta_ptr;
+  float* ws_o;
+  float* ws_lse;
+  int* status;
+  int64_t page_bytes;
+  int32_t n_q_heads, n_kv_heads, G;
+  float scale_log2;  // log2(e) / sqrt(D)
+};
+
+int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, const void* v_new, cudaStream_t s);
+int pie_launch_copy(pie_ctx* ctx, int n, const int32_t* d_ops, cudaStream_t s);
+int pie_launch_page_io(pie_ctx* ctx, int n, const int32_t* d_ids, void* K, void* V, bool write, cudaStream_t s);
+int pie_launch_simple(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);
+int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);
+int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);
+int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s);
+bool pie_split_supported(const pie_ctx* ctx);
+size_t pie_split_smem_bytes(const pie_ctx* ctx);
+
+int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);  // host part (planner.cc)
+
+#define PIE_CUDA(ctx, expr)                                   \
+  do {                                                        \
+    cudaError_t e__ = (expr);                                 \
+    if (e__ != cudaSuccess) {                                 \
+      (ctx)->cuda_error = std::string(#expr) + ": " + cudaGetErrorString(e__); \
+      return PIE_ERR_CUDA;                                    \
+    }                                                         \
+  } while (0)

@@ -1,0 +1,291 @@
+// Host batch planner: the control-layer side of one coalesced `forward` batch (Section 5.2
+// "Batch scheduler": a batch is a set of same-type calls that do not conflict; Section 4.2
+// "Forward API": explicit boolean masks or masks inferred from positions).
+//
+// Turns per-request page lists and masks into what the kernels read: per-request records,
+// bit-packed masks, a page list with fully masked pages removed, append destinations, and a
+// work partition that gives every SM an equal share of page visits.
+#include <algorithm>
+#include <cstring>
+
+#include "pie_internal.h"
+
+namespace {
+
+// Pack `n` bool bytes (each 0 or 1) into bits, LSB first.  Returns false on a byte > 1.
+bool pack_row(const uint8_t* src, int64_t n, uint32_t* dst) {
+  int64_t j = 0;
+  uint8_t bad = 0;
+  for (; j + 8 <= n; j += 8) {
+    uint64_t x;
+    std::memcpy(&x, src + j, 8);
+    bad |= (x & 0xFEFEFEFEFEFEFEFEull) != 0;
+    // gather the low bit of each byte into one byte (byte k -> bit k)
+    uint32_t b = (uint32_t)((x * 0x0102040810204080ull) >> 56) & 0xFFu;
+    dst[j >> 5] |= b << (j & 31);
+  }
+  for (; j < n; ++j) {
+    bad |= src[j] > 1;
+    dst[j >> 5] |= (uint32_t)(src[j] & 1) << (j & 31);
+  }
+  return bad == 0;
+}
+
+struct Unit {
+  int32_t req, kv_head, row0, nrows, page_begin, page_end;
+};
+
+// Give each of `grid` CTAs a contiguous, equal share of the page visits of `units` (taken in
+// order); a unit cut by a share boundary becomes several items whose fp32 partials are merged.
+void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_cta, int slot_rows,
+               PieLaunchList& ll) {
+  ll.items.clear();
+  ll.merges.clear();
+  ll.cta_ptr.clear();
+  ll.n_slots = 0;
+  ll.slot_rows = slot_rows;
+  ll.grid = 0;
+  if (units.empty()) return;
+  int64_t W = 0;
+  for (const Unit& u : units) W += u.page_end - u.page_begin;
+  int grid = (int)std::min<int64_t>(grid_max, std::max<int64_t>(1, W / std::max(1, min_pages_per_cta)));
+  ll.grid = grid;
+  std::vector<std::vector<PieItem>> per_cta(grid);
+  int64_t off = 0;
+  auto cta_of = [&](int64_t x) {  // share that holds page-visit x
+    if (W == 0) return 0;
+    int64_t c = (x * grid) / W;
+    while (c + 1 < grid && ((c + 1) * W) / grid <= x) ++c;
+    while (c > 0 && (c * W) / grid > x) --c;
+    return (int)std::min<int64_t>(c, grid - 1);
+  };
+  for (const Unit& u : units) {
+    int64_t n = u.page_end - u.page_begin;
+    if (n == 0) {
+      PieItem it{u.req, u.kv_head, u.row0, u.nrows, u.page_begin, u.page_begin, -1, 0};
+      per_cta[cta_of(std::min(off, W > 0 ? W - 1 : 0))].push_back(it);
+      continue;
+    }
+    // pieces: cut at share boundaries strictly inside (off, off+n)
+    std::vector<std::pair<int64_t, int>> cuts;  // (start offset, cta)
+    int64_t x = off;
+    while (x < off + n) {
+      int c = cta_of(x);
+      int64_t end = (c + 1 == grid) ? W : ((int64_t)(c + 1) * W) / grid;
+      if (end <= x) end = x + 1;
+      cuts.push_back({x, c});
+      x = std::min(end, off + n);
+    }
+    int np = (int)cuts.size();
+    int slot0 = ll.n_slots;
+    for (int k = 0; k < np; ++k) {
+      int64_t b = cuts[k].first, e = (k + 1 < np) ? cuts[k + 1].first : off + n;
+      PieItem it{u.req, u.kv_head, u.row0, u.nrows, (int32_t)(u.page_begin + (b - off)),
+                 (int32_t)(u.page_begin + (e - off)), np > 1 ? slot0 + k : -1, 0};
+      per_cta[cuts[k].second].push_back(it);
+    }
+    if (np > 1) {
+      ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, slot0, np});
+      ll.n_slots += np;
+    }
+    off += n;
+  }
+  ll.cta_ptr.push_back(0);
+  for (int c = 0; c < grid; ++c) {
+    for (const PieItem& it : per_cta[c]) ll.items.push_back(it);
+    ll.cta_ptr.push_back((int32_t)ll.items.size());
+  }
+}
+
+}  // namespace
+
+int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
+  const pie_config& cfg = ctx->cfg;
+  const int P = cfg.page_size, G = ctx->G;
+  const int R = b->num_requests;
+  if (R < 0) return PIE_ERR_INVALID;
+  if (R > cfg.max_requests) return PIE_ERR_BATCH_TOO_LARGE;
+  if (R > 0 && (!b->qo_indptr || !b->page_indptr || !b->page_indices || !b->last_page_len))
+    return PIE_ERR_INVALID;
+  plan->R = R;
+  plan->flags = b->flags;
+  plan->T = 0;
+  if (R == 0) {
+    plan->info = pie_plan_info{};
+    return PIE_OK;
+  }
+  if (b->qo_indptr[0] != 0 || b->page_indptr[0] != 0) return PIE_ERR_INVALID;
+  for (int r = 0; r < R; ++r) {
+    if (b->qo_indptr[r + 1] <= b->qo_indptr[r]) return PIE_ERR_INVALID;      // q_len >= 1
+    if (b->page_indptr[r + 1] <= b->page_indptr[r]) return PIE_ERR_INVALID;  // >= 1 page
+  }
+  const int T = b->qo_indptr[R];
+  if (T > cfg.max_query_tokens) return PIE_ERR_BATCH_TOO_LARGE;
+  plan->T = T;
+
+  // ---- per-request validation
+  plan->reqs.assign(R, PieReq{});
+  for (int r = 0; r < R; ++r) {
+    const int q_len = b->qo_indptr[r + 1] - b->qo_indptr[r];
+    const int np = b->page_indptr[r + 1] - b->page_indptr[r];
+    const int last = b->last_page_len[r];
+    if (last < 1 || last > P) return PIE_ERR_INVALID;
+    const int64_t kv_len64 = (int64_t)(np - 1) * P + last;
+    if (kv_len64 > 0x3FFFFFFF) return PIE_ERR_INVALID;
+    if (kv_len64 < q_len) return PIE_ERR_INVALID;
+    const int32_t* pages = b->page_indices + b->page_indptr[r];
+    for (int k = 0; k < np; ++k) {
+      if (pages[k] < 0 || pages[k] >= cfg.num_pages || !ctx->allocated[pages[k]]) return PIE_ERR_BAD_PAGE;
+    }
+    PieReq& q = plan->reqs[r];
+    q.q_start = b->qo_indptr[r];
+    q.q_len = q_len;
+    q.kv_len = (int32_t)kv_len64;
+    q.last_logical = np - 1;
+    q.last_page_len = last;
+  }
+
+  // ---- conflict rule: no slot is written twice, and no request reads a slot another writes
+  {
+    std::vector<int32_t> touched;
+    int status = PIE_OK;
+    auto slot_mask = [&](int lo, int hi) -> uint32_t {  // bits [lo, hi)
+      uint32_t m = (hi >= 32) ? 0xFFFFFFFFu : ((1u << hi) - 1u);
+      return m & ~((1u << lo) - 1u);
+    };
+    for (int r = 0; r < R && status == PIE_OK; ++r) {
+      const PieReq& q = plan->reqs[r];
+      const int32_t* pages = b->page_indices + b->page_indptr[r];
+      const int first = q.kv_len - q.q_len;
+      for (int lp = first / P; lp <= q.last_logical; ++lp) {
+        int lo = std::max(first - lp * P, 0), hi = std::min(q.kv_len - lp * P, P);
+        uint32_t m = slot_mask(lo, hi);
+        int32_t pg = pages[lp];
+        if (ctx->wmask[pg] & m) { status = PIE_ERR_CONFLICT; break; }
+        if (ctx->wmask[pg] == 0) { touched.push_back(pg); ctx->writer[pg] = r; }
+        else if (ctx->writer[pg] != r) ctx->writer[pg] = -2;
+        ctx->wmask[pg] |= m;
+      }
+    }
+    for (int r = 0; r < R && status == PIE_OK; ++r) {
+      const PieReq& q = plan->reqs[r];
+      const int32_t* pages = b->page_indices + b->page_indptr[r];
+      for (int lp = 0; lp <= q.last_logical; ++lp) {
+        int32_t pg = pages[lp];
+        uint32_t w = ctx->wmask[pg];
+        if (w == 0 || ctx->writer[pg] == r) continue;
+        uint32_t rd = slot_mask(0, lp == q.last_logical ? q.last_page_len : P);
+        if (w & rd) { status = PIE_ERR_CONFLICT; break; }
+      }
+    }
+    for (int32_t pg : touched) { ctx->wmask[pg] = 0; ctx->writer[pg] = -1; }
+    if (status != PIE_OK) return status;
+  }
+
+  // ---- masks: pack explicit ones, classify pages, build the kept-page list
+  plan->mask_words.clear();
+  plan->kept.clear();
+  const uint32_t full_bits = (P >= 32) ? 0xFFFFFFFFu : ((1u << P) - 1u);
+  for (int r = 0; r < R; ++r) {
+    PieReq& q = plan->reqs[r];
+    const int32_t* pages = b->page_indices + b->page_indptr[r];
+    const int np = q.last_logical + 1;
+    int64_t m0 = 0, m1 = 0;
+    if (b->mask_indptr) { m0 = b->mask_indptr[r]; m1 = b->mask_indptr[r + 1]; }
+    q.kept_start = (int32_t)(plan->kept.size() / 2);
+    if (m1 > m0) {
+      if (!b->mask || m1 - m0 != (int64_t)q.q_len * q.kv_len) return PIE_ERR_MASK;
+      const int row_words = ((q.kv_len + 127) / 128) * 4;
+      q.mask_row_words = row_words;
+      q.mask_word_off = (int64_t)plan->mask_words.size();
+      plan->mask_words.resize(plan->mask_words.size() + (size_t)row_words * q.q_len, 0u);
+      uint32_t* w = plan->mask_words.data() + q.mask_word_off;
+      for (int i = 0; i < q.q_len; ++i)
+        if (!pack_row(b->mask + m0 + (int64_t)i * q.kv_len, q.kv_len, w + (size_t)i * row_words))
+          return PIE_ERR_MASK;
+      for (int lp = 0; lp < np; ++lp) {
+        const int bit = lp * P;
+        uint32_t any = 0, all = full_bits;
+        for (int i = 0; i < q.q_len; ++i) {
+          uint32_t bits = (w[(size_t)i * row_words + (bit >> 5)] >> (bit & 31)) & full_bits;
+          any |= bits;
+          all &= bits;
+        }
+        if (!any) continue;  // no query row attends to this page: it is never fetched
+        plan->kept.push_back(pages[lp]);
+        plan->kept.push_back((int32_t)((uint32_t)lp | (all == full_bits ? 0u : PIE_KEPT_NEEDS_MASK)));
+      }
+    } else {
+      if (m1 < m0) return PIE_ERR_MASK;
+      q.mask_row_words = 0;
+      q.mask_word_off = 0;
+      const int lim0 = q.kv_len - q.q_len;  // last position the first query token sees
+      for (int lp = 0; lp < np; ++lp) {
+        plan->kept.push_back(pages[lp]);
+        plan->kept.push_back((int32_t)((uint32_t)lp | (lp * P + P - 1 <= lim0 ? 0u : PIE_KEPT_NEEDS_MASK)));
+      }
+    }
+    q.kept_count = (int32_t)(plan->kept.size() / 2) - q.kept_start;
+  }
+
+  // ---- append destinations
+  plan->append_dst.resize(T);
+  plan->tok_req.resize(T);
+  for (int r = 0; r < R; ++r) {
+    const PieReq& q = plan->reqs[r];
+    const int32_t* pages = b->page_indices + b->page_indptr[r];
+    for (int i = 0; i < q.q_len; ++i) {
+      int pos = q.kv_len - q.q_len + i;
+      plan->append_dst[q.q_start + i] = pages[pos / P] * P + pos % P;
+      plan->tok_req[q.q_start + i] = r;
+    }
+  }
+
+  // ---- route requests to kernels and partition the work
+  const bool tiles_ok = pie_split_supported(ctx) && !(b->flags & PIE_PLAN_FORCE_SIMPLE);
+  std::vector<Unit> split_units, tile_units;
+  plan->simple_rows.clear();
+  const int TILE_ROWS = 64;
+  for (int r = 0; r < R; ++r) {
+    const PieReq& q = plan->reqs[r];
+    const int rows = q.q_len * G;
+    if (!tiles_ok) {
+      for (int i = 0; i < q.q_len; ++i)
+        for (int h = 0; h < cfg.num_q_heads; ++h) plan->simple_rows.push_back((q.q_start + i) * cfg.num_q_heads + h);
+    } else if (rows <= 16) {
+      for (int g = 0; g < cfg.num_kv_heads; ++g)
+        split_units.push_back(Unit{r, g, 0, rows, q.kept_start, q.kept_start + q.kept_count});
+    } else {
+      for (int g = 0; g < cfg.num_kv_heads; ++g)
+        for (int row0 = 0; row0 < rows; row0 += TILE_ROWS) {
+          int nrows = std::min(TILE_ROWS, rows - row0);
+          int end = q.kept_count;
+          if (q.mask_row_words == 0) {  // causal: pages beyond the tile's last token are invisible
+            int i1 = (row0 + nrows - 1) / G;
+            int lim = q.kv_len - q.q_len + i1;
+            end = std::min(end, lim / P + 1);
+          }
+          tile_units.push_back(Unit{r, g, row0, nrows, q.kept_start, q.kept_start + end});
+        }
+    }
+  }
+  partition(split_units, ctx->n_sms, 8, 16, plan->split);
+  partition(tile_units, ctx->n_sms, 8, TILE_ROWS, plan->tile);
+
+  pie_plan_info& info = plan->info;
+  info = pie_plan_info{};
+  info.num_requests = R;
+  info.num_query_tokens = T;
+  info.num_split_items = (int32_t)plan->split.items.size();
+  info.num_tile_items = (int32_t)plan->tile.items.size();
+  info.num_simple_rows = (int32_t)plan->simple_rows.size();
+  info.num_merge_groups = (int32_t)(plan->split.merges.size() + plan->tile.merges.size());
+  info.kept_pages = (int64_t)plan->kept.size() / 2;
+  info.mask_words = (int64_t)plan->mask_words.size();
+  info.workspace_bytes = ((int64_t)plan->split.n_slots * plan->split.slot_rows +
+                          (int64_t)plan->tile.n_slots * plan->tile.slot_rows) * (cfg.head_dim + 1) * 4;
+  info.launches = 1 + (info.num_simple_rows ? 1 : 0) + (info.num_split_items ? 1 : 0) +
+                  (info.num_tile_items ? 1 : 0) + (plan->split.merges.empty() ? 0 : 1) +
+                  (plan->tile.merges.empty() ? 0 : 1);
+  return PIE_OK;
+}

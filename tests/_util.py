@@ -11,6 +11,14 @@ def bits(t):
     return synth.to_numpy_bits(t)
 
 
+def same_bits(a, b):
+    """Bitwise equality (NaN patterns included) of two arrays of the same storage type."""
+    a, b = np.ascontiguousarray(a), np.ascontiguousarray(b)
+    if a.dtype == np.float32:
+        a, b = a.view(np.uint32), b.view(np.uint32)
+    return a.shape == b.shape and np.array_equal(a, b)
+
+
 def run_oracle(wl, poison=False, requests=None, pool=None):
     """Oracle forward on a Workload; returns (O fp64, LSE fp64, pool after the append)."""
     pool = wl.oracle_pool(poison) if pool is None else pool

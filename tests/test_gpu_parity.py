@@ -1,0 +1,120 @@
+"""GPU parity: the CUDA path against the fp64 oracle, element by element, on the same seeded
+inputs, through the C ABI.  Tolerances: |O - O*| <= 2e-2 (bf16) / 1e-4 (fp32), |LSE - LSE*| <=
+1e-3, plus a per-request relative RMS gate; append and copy are bit exact."""
+import numpy as np
+import pytest
+import torch
+
+from tests._util import bits, run_oracle, same_bits
+from workloads import configs, synth
+
+pytestmark = pytest.mark.gpu
+
+SMALL = ["tiny_fp32", "batched_decode", "mixed_prefill_decode", "shared_prefix_tree", "long_context_policy"]
+
+
+def test_generator_is_bit_identical_on_cpu_and_gpu():
+    wl = configs.small("mixed_prefill_decode")
+    for f in (wl.q, wl.k_new, wl.v_new):
+        assert torch.equal(f("cpu"), f("cuda").cpu())
+    ids = wl.used_pages()[:7]
+    Kc, Vc = wl.context_pages(ids, "cpu", poison=True)
+    Kg, Vg = wl.context_pages(ids, "cuda", poison=True)
+    assert same_bits(bits(Kc), bits(Kg)) and same_bits(bits(Vc), bits(Vg))
+
+
+@pytest.mark.parametrize("name", SMALL)
+@pytest.mark.parametrize("flags", [0, 1])
+def test_small_configs_match_oracle(name, flags):
+    from tests._gpu import check_close, run_workload
+    wl = configs.small(name)
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    O, L, info, gp = run_workload(wl, poison=True, flags=flags, keep=True)
+    try:
+        check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        # append is bit exact: every used page equals the oracle's pool after the call
+        used = wl.used_pages()
+        K, V = gp.read_pages(used)
+        for n, p in enumerate(used):
+            Ko, Vo = pool[int(p)]
+            assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {p}"
+    finally:
+        gp.close()
+
+
+@pytest.mark.parametrize("name", SMALL[1:])
+def test_peaked_scores_match_oracle(name):
+    """Q scaled x4: the softmax concentrates and |O| = O(1), so a wrong kernel cannot hide
+    behind small outputs."""
+    from oracle import pie_oracle as orc
+    from tests._gpu import check_close, run_workload
+    wl = configs.small(name)
+    q4 = (wl.q().float() * 4).to(torch.bfloat16)
+    pool = wl.oracle_pool()
+    O_ref, L_ref = orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices,
+                               wl.last_page_len, bits(q4), bits(wl.k_new()), bits(wl.v_new()), wl.masks)
+    O, L, _ = run_workload(wl, q_scale=4.0)
+    check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
+
+
+def test_copy_kvpage_bit_exact_and_errors():
+    import paper_2510_24051_b200 as pie
+    from oracle import pie_oracle as orc
+    from tests._gpu import GpuPool
+    wl = configs.small("long_context_policy")
+    pool = wl.oracle_pool()
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        c = wl.copies
+        touched = np.unique(np.concatenate([c["src"], c["dst"]]))
+        gp.install(wl, pages=touched)
+        # whole-range copies of the workload plus token-level ones with shifted offsets
+        src = np.concatenate([c["src"], c["src"][:3]])
+        dst = np.concatenate([c["dst"], c["dst"][3:6]])
+        so = np.concatenate([c["src_off"], [1, 2, 5]])
+        do = np.concatenate([c["dst_off"], [9, 13, 10]])
+        nt = np.concatenate([np.minimum(c["ntok"], 9), [7, 3, 6]])
+        nt[3:6] = np.minimum(nt[3:6], 9)
+        orc.copy_kvpage(pool, src, dst, so, do, nt)
+        pie.pie_copy_kvpage(gp.ctx, src, dst, so, do, nt)
+        K, V = gp.read_pages(touched)
+        for n, p in enumerate(touched):
+            assert same_bits(K[n], pool[int(p)][0]) and same_bits(V[n], pool[int(p)][1])
+        with pytest.raises(pie.PieError) as e:      # two ops write the same slot
+            pie.pie_copy_kvpage(gp.ctx, [1, 2], [3, 3], [0, 0], [0, 4], [8, 8])
+        assert e.value.status == pie.PIE_ERR_CONFLICT
+        with pytest.raises(pie.PieError) as e:      # overlapping in-place shift
+            pie.pie_copy_kvpage(gp.ctx, [1], [1], [0], [4], [8])
+        assert e.value.status == pie.PIE_ERR_CONFLICT
+        with pytest.raises(pie.PieError) as e:
+            pie.pie_copy_kvpage(gp.ctx, [1], [2], [10], [0], [8])
+        assert e.value.status == pie.PIE_ERR_INVALID
+        pie.pie_copy_kvpage(gp.ctx, [], [], [], [], [])          # empty call is fine
+
+
+def test_forward_host_matches_device_call():
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs.small("mixed_prefill_decode")
+    O_ref, L_ref, _ = run_oracle(wl)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl)
+        q, k, v = (t.pin_memory() for t in (wl.q(), wl.k_new(), wl.v_new()))
+        out = torch.empty_like(q).pin_memory()
+        lse = torch.empty((wl.T, wl.H_q), dtype=torch.float32).pin_memory()
+        pie.pie_forward_host(gp.ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                             q, k, v, out, lse)
+        check_close(out.double().numpy(), lse.double().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+
+
+def test_repeat_calls_are_bitwise_deterministic():
+    from tests._gpu import GpuPool
+    import paper_2510_24051_b200 as pie
+    wl = configs.small("batched_decode")
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl)
+        plan = gp.plan(wl)
+        q, k, v = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
+        a = gp.forward(plan, q, k, v)
+        b = gp.forward(plan, q, k, v)
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+        pie.pie_plan_destroy(plan)
