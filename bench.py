@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the batched `forward` attention handler on synthetic workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one pass of the whole hot path over one coalesced batch: pie_forward (append of
+the new K/V rows, attention, merge of split partials) plus, for the long-context workload, the
+pie_copy_kvpage call that follows it.  Plans are built once (host planning time is reported
+separately as `plan_ms`); inputs are resident in HBM when the timed region starts.  The `e2e`
+figure repeats the measurement through pie_forward_host: planning, pinned-host -> device copies
+of Q/K/V and the device -> host read of the outputs are all inside its timed region.
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs its own batch
+of the same shape (requests are independent: no data-path collective); the time is the max over
+ranks and `value` counts all ranks' tokens (weak scaling).
+
+`--impl reference` times the fp64 CPU oracle on the same workload shape instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "attention tokens/s and achieved HBM GB/s / tensor TFLOPS vs B200 peak"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (null until a capture exists for that workload).
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def build_workloads(name, seed_offset=0):
+    """The list of batches a run cycles through (several page placements when one batch's KV is
+    small enough to live in L2), plus a note saying how L2 reuse is defeated."""
+    from workloads import configs
+    builder = configs.FULL[name]
+    seed = configs.SEED0 + list(configs.FULL).index(name) + 1 + 1000 * seed_offset
+    if name == "batched_decode":
+        probe = builder(seed=seed)
+        n_place = max(1, probe.num_pages // len(probe.page_indices))
+        wls = [builder(seed=seed, placement=i) for i in range(n_place)]
+        note = f"{n_place} rotating page placements ({n_place * probe.algorithmic_bytes()['kv'] / 1e9:.2f} GB of KV) > L2"
+    else:
+        wls = [builder(seed=seed)]
+        note = f"one placement; KV read per step {wls[0].algorithmic_bytes()['kv'] / 1e9:.2f} GB > L2"
+    return wls, note
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        self.rows, self.proc, self.device = [], None, device
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.device), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])), mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(wl, budget_s=20.0):
+    """Time the fp64 oracle on a bounded sample of the workload's requests (inputs pre-generated).
+    Returns (tokens, seconds, description, threads)."""
+    from oracle import pie_oracle as orc
+    from workloads import synth
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = 1
+    qb, kb, vb = (synth.to_numpy_bits(t) for t in (wl.q(), wl.k_new(), wl.v_new()))
+    # estimate cost per request from its score-matrix size, then take a prefix that fits the budget
+    cost = wl.q_lens() * wl.kept_tokens() * wl.H_q * wl.D * 4.0
+    rate = 2e9                                        # conservative fp64 flop/s incl. gather overhead
+    order = np.arange(wl.R)
+    n, acc = 0, 0.0
+    while n < wl.R and (n == 0 or acc + cost[order[n]] / rate <= budget_s):
+        acc += cost[order[n]] / rate
+        n += 1
+    sample = order[:n]
+    pool = wl.oracle_pool()
+    for r in sample:                                  # generate the pages outside the timed region
+        m = None if wl.masks is None else wl.masks[r]
+        npg = len(wl.pages_of(r))
+        if m is None:
+            need = np.ones(npg, bool)
+        else:
+            cols = np.zeros(npg * wl.P, bool)
+            cols[:m.shape[1]] = m.any(axis=0)
+            need = cols.reshape(npg, wl.P).any(axis=1)
+        for p in wl.pages_of(r)[need]:
+            pool[int(p)]
+    for r in range(wl.R):                             # pages the append writes
+        kv, ql = int(wl.kv_lens()[r]), int(wl.q_lens()[r])
+        for lp in range((kv - ql) // wl.P, len(wl.pages_of(r))):
+            pool[int(wl.pages_of(r)[lp])]
+    t0 = time.perf_counter()
+    orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                qb, kb, vb, wl.masks, requests=sample)
+    dt = time.perf_counter() - t0
+    tokens = int(wl.q_lens()[sample].sum())
+    return tokens, dt, f"first {n} of {wl.R} requests of {wl.name}, one pass", threads
+
+
+def run_reference(args):
+    """The reference arm: the fp64 CPU oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wls, _ = build_workloads(args.workload)
+    wl = wls[0]
+    times, tokens, desc, threads = [], 0, "", 1
+    budget = 8.0
+    for it in range(args.warmup + args.steps):
+        tokens, dt, desc, threads = oracle_sample(wl, budget_s=budget)
+        if it >= args.warmup:
+            times.append(dt)
+        if (it + 1) * dt > 150:                        # keep the whole run within a few minutes
+            break
+    dt = statistics.mean(times) if times else dt
+    val = tokens / dt
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": len(times) or 1, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "sample": desc},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="batched_decode")
+    ap.add_argument("--flags", type=int, default=0, help="PIE_PLAN_* flags (debug / A-B runs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2510_24051_b200 as pie
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    wls, l2_note = build_workloads(args.workload, seed_offset=rank)
+    wl0 = wls[0]
+    ctx = pie.pie_create(wl0.num_pages, wl0.P, wl0.H_q, wl0.H_kv, wl0.D, wl0.dtype, max(wl0.R, 1), max(wl0.T, 1), local)
+    ids = pie.pie_alloc_kvpages(ctx, wl0.num_pages)
+    assert np.array_equal(ids, np.arange(wl0.num_pages))
+    for wl in wls:                                     # install the pre-existing context (device generator)
+        used = wl.used_pages()
+        for i in range(0, len(used), 4096):
+            K, V = wl.context_pages(used[i:i + 4096], "cuda")
+            pie.pie_kvpage_write(ctx, used[i:i + 4096], K.contiguous(), V.contiguous())
+            torch.cuda.synchronize()
+            del K, V
+    plans, plan_ms = [], []
+    mask_args = [wl.mask_bytes() for wl in wls]
+    for wl, (mi, mb) in zip(wls, mask_args):
+        t0 = time.perf_counter()
+        plans.append(pie.pie_plan_forward(ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                                          mi, mb, args.flags))
+        plan_ms.append((time.perf_counter() - t0) * 1e3)
+    info = pie.pie_plan_get_info(plans[0])
+    q, k_new, v_new = wl0.q("cuda"), wl0.k_new("cuda"), wl0.v_new("cuda")
+    out = torch.empty_like(q)
+    lse = torch.empty((wl0.T, wl0.H_q), dtype=torch.float32, device="cuda")
+    copies = wl0.copies
+
+    def step(i):
+        pie.pie_forward(ctx, plans[i % len(plans)], q, k_new, v_new, out, lse)
+        if copies is not None:
+            pie.pie_copy_kvpage(ctx, copies["src"], copies["dst"], copies["src_off"], copies["dst_off"], copies["ntok"])
+
+    # ---------------------------------------------------------------- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    assert pie.pie_get_last_device_status(ctx) == 0, "a device-side wait timed out"
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    launches_per_step = info["launches"] + (1 if copies is not None else 0)
+
+    # ---------------------------------------------------------------- per-kernel timing (live)
+    pie.pie_set_kernel_timing(ctx, 1)
+    for i in range(args.steps):
+        step(i)
+    torch.cuda.synchronize()
+    ktimes = pie.pie_get_kernel_times(ctx)
+    pie.pie_set_kernel_timing(ctx, 0)
+
+    # ---------------------------------------------------------------- end to end (host buffers)
+    e2e = None
+    if not args.no_e2e:
+        hq, hk, hv = (t.cpu().pin_memory() for t in (q, k_new, v_new))
+        hout = torch.empty_like(hq).pin_memory()
+        hlse = torch.empty((wl0.T, wl0.H_q), dtype=torch.float32).pin_memory()
+        n_e2e = max(3, min(args.steps, 30))
+
+        def e2e_step(i):
+            wl = wls[i % len(wls)]
+            mi, mb = mask_args[i % len(wls)]
+            pie.pie_forward_host(ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                                 hq, hk, hv, hout, hlse, mi, mb, args.flags)
+            if copies is not None:
+                pie.pie_copy_kvpage(ctx, copies["src"], copies["dst"], copies["src_off"], copies["dst_off"], copies["ntok"])
+                torch.cuda.synchronize()
+
+        for i in range(3):
+            e2e_step(i)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([e2e_s], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
+        d2h = hout.numel() * hout.element_size() + hlse.numel() * 4
+        e2e = {"value": world * wl0.T * n_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": e2e_s / n_e2e * 1e3,
+               "includes": "host planning, pinned H2D of Q/K/V, forward, D2H of O/LSE"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---------------------------------------------------------------- roofline of the dominant kernel
+    peaks = load_peaks()
+    dom = max(("split", "tiles", "simple"), key=lambda k: ktimes[k][0])
+    dom_ms = ktimes[dom][0] / max(ktimes[dom][1], 1)
+    G = wl0.H_q // wl0.H_kv
+    rows = wl0.q_lens() * G
+    sel = rows <= 16 if dom == "split" else rows > 16
+    b_tok = 2 * wl0.H_kv * wl0.D * wl0.esize
+    if dom in ("split", "simple"):
+        kv_bytes = int(wl0.kept_tokens()[sel].sum()) * b_tok
+        qo_bytes = int(wl0.q_lens()[sel].sum()) * wl0.H_q * (2 * wl0.D * wl0.esize + 4)
+        mask_bytes = 0 if wl0.masks is None else sum((m.size + 7) // 8 for m, s in zip(wl0.masks, sel) if s and m is not None)
+        alg = kv_bytes + qo_bytes + mask_bytes
+        achieved = alg / (dom_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(wl0.name),
+                "algorithmic_bytes": alg, "kernel_ms": dom_ms, "peak_source": peaks["source"]}
+    else:
+        flops = 0
+        for r in np.nonzero(sel)[0]:
+            m = None if wl0.masks is None else wl0.masks[r]
+            ql, kv = int(wl0.q_lens()[r]), int(wl0.kv_lens()[r])
+            n = (ql * kv - ql * (ql - 1) // 2) if m is None else int(m.sum())
+            flops += 4 * wl0.D * wl0.H_q * n
+        achieved = flops / (dom_ms * 1e-3) / 1e12
+        peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        roof = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(wl0.name), "useful_flops": flops,
+                "kernel_ms": dom_ms, "peak_source": peaks["source"] + " (sustained)"}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        tokens, dt, desc, threads = oracle_sample(wl0)
+        cpu = {"value": tokens / dt, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc,
+               "seconds": dt}
+
+    ms_per_step = ms / args.steps
+    alg_bytes = wl0.algorithmic_bytes()
+    line = {
+        "metric": METRIC, "value": world * wl0.T / (ms_per_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": wl0.dtype, "data": "synthetic",
+        "config": {"workload": wl0.name, "requests": wl0.R, "query_tokens": wl0.T, "heads": f"{wl0.H_q}/{wl0.H_kv}",
+                   "head_dim": wl0.D, "page_size": wl0.P, "pool_pages": wl0.num_pages, "l2": l2_note,
+                   "plan_flags": args.flags},
+        "hbm_gbs_step": alg_bytes["total"] / (ms_per_step * 1e-3) / 1e9,
+        "algorithmic_bytes_step": alg_bytes, "useful_flops_step": wl0.useful_flops(),
+        "plan_ms": statistics.median(plan_ms), "plan_info": info,
+        "kernel_ms": {k: (v[0] / v[1] if v[1] else 0.0) for k, v in ktimes.items()},
+        "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    for p in plans:
+        pie.pie_plan_destroy(p)
+    pie.pie_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -184,6 +184,23 @@ int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, c
  * gave up since the last call.  Synchronises `stream`, reads and clears the word. */
 int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out);
 
+/* Per-kernel device timing for benchmarks.  While enabled, pie_forward and pie_copy_kvpage
+ * bracket each kernel they enqueue with CUDA events on the caller's stream.
+ * pie_get_kernel_times waits for the recorded events, adds the elapsed milliseconds and the
+ * launch counts per kernel kind into ms[PIE_NUM_KERNEL_KINDS] / launches[PIE_NUM_KERNEL_KINDS]
+ * (host arrays, overwritten), and forgets the records.  Off by default (no events, no cost). */
+enum {
+  PIE_KERNEL_APPEND = 0,
+  PIE_KERNEL_SIMPLE = 1,
+  PIE_KERNEL_SPLIT = 2,   /* split-KV decode attention   */
+  PIE_KERNEL_TILES = 3,   /* prefill / tree row tiles    */
+  PIE_KERNEL_MERGE = 4,
+  PIE_KERNEL_COPY = 5,
+  PIE_NUM_KERNEL_KINDS = 6
+};
+int pie_set_kernel_timing(pie_ctx* ctx, int enable);
+int pie_get_kernel_times(pie_ctx* ctx, float* ms, int32_t* launches);
+
 #ifdef __cplusplus
 }
 #endif

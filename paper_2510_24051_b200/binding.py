@@ -69,6 +69,8 @@ def _load():
         "pie_forward": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, vp]),
         "pie_forward_host": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
         "pie_get_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int)]),
+        "pie_set_kernel_timing": (C.c_int, [vp, C.c_int]),
+        "pie_get_kernel_times": (C.c_int, [vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)          # AttributeError here = the library lacks a declared symbol
@@ -221,3 +223,18 @@ def pie_get_last_device_status(ctx, stream=None):
     out = C.c_int()
     _check(lib.pie_get_last_device_status(ctx, _stream(stream), C.byref(out)), ctx)
     return out.value
+
+
+KERNEL_KINDS = ("append", "simple", "split", "tiles", "merge", "copy")
+
+
+def pie_set_kernel_timing(ctx, enable):
+    _check(lib.pie_set_kernel_timing(ctx, int(bool(enable))), ctx)
+
+
+def pie_get_kernel_times(ctx):
+    """{kind: (total ms, launches)} of the kernels recorded since timing was enabled / last read."""
+    ms = np.zeros(len(KERNEL_KINDS), dtype=np.float32)
+    n = np.zeros(len(KERNEL_KINDS), dtype=np.int32)
+    _check(lib.pie_get_kernel_times(ctx, ms.ctypes.data, n.ctypes.data), ctx)
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}

@@ -87,6 +87,26 @@ int ensure_buffer(pie_ctx* ctx, void** buf, size_t* cap, size_t need) {
   return PIE_OK;
 }
 
+// Runs `launch` bracketed by events when timing is on.
+template <typename F>
+int timed_launch(pie_ctx* ctx, int kind, cudaStream_t s, F&& launch) {
+  if (!ctx->timing) return launch();
+  cudaEvent_t ev[2];
+  for (int k = 0; k < 2; ++k) {
+    if (!ctx->free_events.empty()) {
+      ev[k] = ctx->free_events.back();
+      ctx->free_events.pop_back();
+    } else {
+      PIE_CUDA(ctx, cudaEventCreate(&ev[k]));
+    }
+  }
+  PIE_CUDA(ctx, cudaEventRecord(ev[0], s));
+  int rc = launch();
+  PIE_CUDA(ctx, cudaEventRecord(ev[1], s));
+  ctx->timed.push_back({kind, ev[0], ev[1]});
+  return rc;
+}
+
 bool page_ok(const pie_ctx* ctx, int32_t id) {
   return id >= 0 && id < ctx->cfg.num_pages && ctx->allocated[id];
 }
@@ -205,6 +225,11 @@ int pie_destroy(pie_ctx* ctx) {
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_stage) cudaFree(ctx->d_stage);
     if (ctx->d_io) cudaFree(ctx->d_io);
+    for (auto& t : ctx->timed) {
+      cudaEventDestroy(t.start);
+      cudaEventDestroy(t.stop);
+    }
+    for (auto e : ctx->free_events) cudaEventDestroy(e);
   }
   delete ctx;
   return PIE_OK;
@@ -330,7 +355,7 @@ int pie_copy_kvpage(pie_ctx* ctx, int32_t n, const int32_t* src, const int32_t* 
   int rc = ensure_buffer(ctx, &ctx->d_stage, &ctx->stage_bytes, ops.size() * 4);
   if (rc) return rc;
   PIE_CUDA(ctx, cudaMemcpyAsync(ctx->d_stage, ops.data(), ops.size() * 4, cudaMemcpyHostToDevice, s));
-  return pie_launch_copy(ctx, n, (const int32_t*)ctx->d_stage, s);
+  return timed_launch(ctx, PIE_KERNEL_COPY, s, [&] { return pie_launch_copy(ctx, n, (const int32_t*)ctx->d_stage, s); });
 }
 
 int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pie_plan** out) {
@@ -446,13 +471,23 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
   if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
   cudaStream_t s = (cudaStream_t)stream;
   PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
-  int rc = pie_launch_append(ctx, plan, k_new, v_new, s);
+  int rc = timed_launch(ctx, PIE_KERNEL_APPEND, s, [&] { return pie_launch_append(ctx, plan, k_new, v_new, s); });
   if (rc) return rc;
-  if (!plan->simple_rows.empty() && (rc = pie_launch_simple(ctx, plan, q, out, lse, s))) return rc;
-  if (!plan->split.items.empty() && (rc = pie_launch_split(ctx, plan, q, out, lse, s))) return rc;
-  if (!plan->tile.items.empty() && (rc = pie_launch_tiles(ctx, plan, q, out, lse, s))) return rc;
-  if (!plan->split.merges.empty() && (rc = pie_launch_merge(ctx, plan, plan->split, out, lse, s))) return rc;
-  if (!plan->tile.merges.empty() && (rc = pie_launch_merge(ctx, plan, plan->tile, out, lse, s))) return rc;
+  if (!plan->simple_rows.empty() &&
+      (rc = timed_launch(ctx, PIE_KERNEL_SIMPLE, s, [&] { return pie_launch_simple(ctx, plan, q, out, lse, s); })))
+    return rc;
+  if (!plan->split.items.empty() &&
+      (rc = timed_launch(ctx, PIE_KERNEL_SPLIT, s, [&] { return pie_launch_split(ctx, plan, q, out, lse, s); })))
+    return rc;
+  if (!plan->tile.items.empty() &&
+      (rc = timed_launch(ctx, PIE_KERNEL_TILES, s, [&] { return pie_launch_tiles(ctx, plan, q, out, lse, s); })))
+    return rc;
+  if (!plan->split.merges.empty() &&
+      (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s, [&] { return pie_launch_merge(ctx, plan, plan->split, out, lse, s); })))
+    return rc;
+  if (!plan->tile.merges.empty() &&
+      (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s, [&] { return pie_launch_merge(ctx, plan, plan->tile, out, lse, s); })))
+    return rc;
   return PIE_OK;
 }
 
@@ -509,6 +544,39 @@ int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out) {
     PIE_CUDA(ctx, cudaStreamSynchronize(s));
   }
   *out = v;
+  return PIE_OK;
+}
+
+int pie_set_kernel_timing(pie_ctx* ctx, int enable) {
+  if (!ctx) return PIE_ERR_INVALID;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  for (auto& t : ctx->timed) {
+    ctx->free_events.push_back(t.start);
+    ctx->free_events.push_back(t.stop);
+  }
+  ctx->timed.clear();
+  ctx->timing = enable != 0;
+  return PIE_OK;
+}
+
+int pie_get_kernel_times(pie_ctx* ctx, float* ms, int32_t* launches) {
+  if (!ctx || !ms || !launches) return PIE_ERR_INVALID;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  for (int k = 0; k < PIE_NUM_KERNEL_KINDS; ++k) {
+    ms[k] = 0.f;
+    launches[k] = 0;
+  }
+  PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  for (auto& t : ctx->timed) {
+    PIE_CUDA(ctx, cudaEventSynchronize(t.stop));
+    float e = 0.f;
+    PIE_CUDA(ctx, cudaEventElapsedTime(&e, t.start, t.stop));
+    ms[t.kind] += e;
+    launches[t.kind] += 1;
+    ctx->free_events.push_back(t.start);
+    ctx->free_events.push_back(t.stop);
+  }
+  ctx->timed.clear();
   return PIE_OK;
 }
 

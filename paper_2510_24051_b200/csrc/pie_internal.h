@@ -118,6 +118,11 @@ struct pie_ctx {
   void* d_io = nullptr;     // q/k/v/out/lse staging of pie_forward_host
   size_t io_bytes = 0;
   std::string cuda_error;
+  // optional per-kernel timing (pie_set_kernel_timing)
+  bool timing = false;
+  struct TimedLaunch { int kind; cudaEvent_t start, stop; };
+  std::vector<TimedLaunch> timed;
+  std::vector<cudaEvent_t> free_events;
   // scratch for validation (sized num_pages)
   std::vector<uint32_t> wmask;
   std::vector<int32_t> writer;
