@@ -170,6 +170,7 @@ int pie_create(const pie_config* cfg, pie_ctx** out) {
   if (cfg->num_q_heads % cfg->num_kv_heads) return PIE_ERR_INVALID;
   if (cfg->max_requests < 1 || cfg->max_query_tokens < 1) return PIE_ERR_INVALID;
   if ((int64_t)cfg->num_pages * P > 0x7FFFFFFF) return PIE_ERR_INVALID;
+  if ((int64_t)cfg->num_pages * cfg->num_kv_heads > 0x7FFFFFFF) return PIE_ERR_INVALID;
   pie_ctx* ctx = new (std::nothrow) pie_ctx();
   if (!ctx) return PIE_ERR_INVALID;
   ctx->cfg = *cfg;
@@ -385,12 +386,14 @@ int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pi
     size_t o_app = put(plan->append_dst.data(), plan->append_dst.size() * 4);
     size_t o_tok = put(plan->tok_req.data(), plan->tok_req.size() * 4);
     size_t o_simple = put(plan->simple_rows.data(), plan->simple_rows.size() * 4);
-    size_t o_li[2], o_lc[2], o_lm[2];
+    size_t o_li[2], o_lc[2], o_lm[2], o_ls[2], o_lp[2];
     PieLaunchList* lls[2] = {&plan->split, &plan->tile};
     for (int k = 0; k < 2; ++k) {
       o_li[k] = put(lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
       o_lc[k] = put(lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
       o_lm[k] = put(lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
+      o_ls[k] = put(lls[k]->stream.data(), lls[k]->stream.size() * 4);
+      o_lp[k] = put(lls[k]->stream_ptr.data(), lls[k]->stream_ptr.size() * 4);
     }
     size_t upload = (host.size() + 255) & ~(size_t)255;
     size_t total = upload;
@@ -424,6 +427,8 @@ int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pi
       lls[k]->d_items = (PieItem*)(base + o_li[k]);
       lls[k]->d_cta_ptr = (int32_t*)(base + o_lc[k]);
       lls[k]->d_merges = (PieMerge*)(base + o_lm[k]);
+      lls[k]->d_stream = (int2*)(base + o_ls[k]);
+      lls[k]->d_stream_ptr = (int32_t*)(base + o_lp[k]);
       lls[k]->d_ws_o = (float*)(base + o_wo[k]);
       lls[k]->d_ws_lse = (float*)(base + o_wl[k]);
     }

@@ -1,12 +1,11 @@
 // Attention kernels of the `forward` handler (Section 4.2 "Forward API": attention over the
 // request's KvPages under an explicit or inferred mask):
-//   * attn_mma_kernel<SPLIT=true>  - decode: split-KV over scattered pages, HBM bound.  A
-//     producer warp streams (page, kv head) blocks into a deep shared-memory ring with bulk
-//     async copies; consumer warps take pages round-robin, run QK^T / PV on tensor cores with
-//     the grouped query heads stacked in the M dimension, and keep private online-softmax
-//     states that are merged once per work item.
-//   * attn_mma_kernel<SPLIT=false> - row tiles (prefill chunks, token trees): each consumer warp
-//     owns 16 query rows and every warp walks the same page stream.
+//   * attn_split_kernel - decode: split-KV over scattered pages, HBM bound.  Every warp is an
+//     independent pipeline: it streams its share of (page, kv head) blocks into a private
+//     shared-memory ring with bulk async copies, runs QK^T / PV on tensor cores with the
+//     grouped query heads stacked in the M dimension, and writes a final row or an fp32 partial.
+//   * attn_tile_kernel  - row tiles (prefill chunks, token trees): each consumer warp owns 16
+//     query rows and every warp walks the same page stream filled by a producer warp.
 //   * merge_kernel                 - LSE-weighted merge of split partials.
 //   * simple_kernel                - plain CUDA-core kernel (fp32 pools and shapes the tile
 //     kernels do not cover); one warp per (token, head) row, sequential online softmax.
@@ -95,33 +94,295 @@ __device__ __forceinline__ float fast_exp2(float x) {
 constexpr float kNegInf = -__builtin_huge_valf();
 constexpr float kLn2 = 0.6931471805599453f;
 
-// ------------------------------------------------------------------------------ tile kernel
-template <int D, int P, int NW, bool SPLIT, int NSTAGES>
+// ------------------------------------------------------------------------------ warp-level core
+// One warp attends 16 query rows (row = query token * G + head-in-group, for one kv head) over a
+// stream of KvPage blocks.  Per thread: rows r_lo = lane/4 and r_lo + 8, columns cpair, cpair+1
+// of every 8-wide block (the m16n8k16 accumulator layout).
+template <int D>
+struct RowState {
+  uint32_t qf[D / 16][4];  // Q fragments (A operand)
+  float o[D / 8][4];       // un-normalised output accumulators
+  float m_run[2], l_run[2];
+  int lim[2];              // last visible position under the inferred causal mask (-1: no row)
+  const uint32_t* mrow[2]; // packed explicit mask row
+  bool valid[2];
+  bool explicit_mask;
+  bool any_rows;
+};
+
+template <int D>
+__device__ __forceinline__ void rows_init(RowState<D>& st, const AttnParams& p, const PieItem& item, const PieReq& rq,
+                                          int rbase, int lane) {
+  const int r_lo = lane >> 2, cpair = (lane & 3) * 2;
+  const int row_end = item.row0 + item.nrows;
+  st.explicit_mask = rq.mask_row_words != 0;
+  st.any_rows = rbase < row_end;
+  const __nv_bfloat16* qptr[2];
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int gr = rbase + r_lo + r * 8;
+    st.valid[r] = gr < row_end;
+    const int tok = st.valid[r] ? gr / p.G : 0;
+    const int head = item.kv_head * p.G + (st.valid[r] ? gr % p.G : 0);
+    st.lim[r] = st.valid[r] ? rq.kv_len - rq.q_len + tok : -1;
+    st.mrow[r] = p.mask + rq.mask_word_off + (int64_t)tok * rq.mask_row_words;
+    qptr[r] = reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)(rq.q_start + tok) * p.n_q_heads + head) * D;
+    st.m_run[r] = kNegInf;
+    st.l_run[r] = 0.f;
+  }
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      uint32_t lo = 0, hi = 0;
+      if (st.valid[r]) {
+        lo = __ldg(reinterpret_cast<const uint32_t*>(qptr[r] + ks * 16 + cpair));
+        hi = __ldg(reinterpret_cast<const uint32_t*>(qptr[r] + ks * 16 + 8 + cpair));
+      }
+      st.qf[ks][r] = lo;
+      st.qf[ks][2 + r] = hi;
+    }
+  }
+#pragma unroll
+  for (int nb = 0; nb < D / 8; ++nb) st.o[nb][0] = st.o[nb][1] = st.o[nb][2] = st.o[nb][3] = 0.f;
+}
+
+// Attend the warp's rows to one KvPage block resident in shared memory (K block then V block,
+// each [slab][slot][128 B] with the 16-byte chunks XOR-swizzled by slot & 7).
+template <int D, int P>
+__device__ __forceinline__ void page_compute(RowState<D>& st, uint8_t* stage, const PieReq& rq, uint32_t lpf,
+                                             float scale_log2, int lane) {
+  constexpr int KSTEPS = D / 16, SUBS = P / 16, BLK = P * D * 2, SLAB = P * 128;
+  const int cpair = (lane & 3) * 2;
+  const int lp = (int)(lpf & ~PIE_KEPT_NEEDS_MASK);
+  const bool needs_mask = (lpf & PIE_KEPT_NEEDS_MASK) != 0;
+  const uint32_t kbase = smem_u32(stage), vbase = kbase + BLK;
+
+  if (lp == rq.last_logical && rq.last_page_len < P) {
+    // slots past the end of the context may hold anything: clear their V rows so that a zero
+    // probability times a NaN bit pattern cannot leak into the output
+    constexpr int CH = D * 2 / 16;
+    const int nz = (P - rq.last_page_len) * CH;
+    for (int c = lane; c < nz; c += 32) {
+      const int t = rq.last_page_len + c / CH, ch = c % CH;
+      *reinterpret_cast<uint4*>(stage + BLK + pie_chunk_offset(SLAB, t, ch)) = make_uint4(0, 0, 0, 0);
+    }
+    __syncwarp();
+  }
+  if (!st.any_rows) return;
+
+#pragma unroll
+  for (int sub = 0; sub < SUBS; ++sub) {
+    const int j0 = lp * P + sub * 16;
+    uint32_t bits[2] = {0xFFFFu, 0xFFFFu};
+    if (needs_mask) {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        if (!st.valid[r]) bits[r] = 0;
+        else if (st.explicit_mask) bits[r] = (__ldg(st.mrow[r] + (j0 >> 5)) >> (j0 & 31)) & 0xFFFFu;
+        else bits[r] = st.lim[r] >= j0 + 15 ? 0xFFFFu : (st.lim[r] < j0 ? 0u : ((1u << (st.lim[r] - j0 + 1)) - 1u));
+      }
+      if (__all_sync(0xFFFFFFFFu, (bits[0] | bits[1]) == 0)) continue;  // nothing visible to this warp
+    }
+    // ---- S = Q K^T for 16 tokens
+    float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    {
+      const int t = sub * 16 + ((lane >> 4) << 3) + (lane & 7);
+      const uint32_t rowaddr = kbase + t * 128;
+      const int csel = (lane >> 3) & 1;
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        const int c = (ks & 3) * 2 + csel;
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4(rowaddr + (ks >> 2) * SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
+        mma_bf16(sacc[0], st.qf[ks], b0, b1);
+        mma_bf16(sacc[1], st.qf[ks], b2, b3);
+      }
+    }
+    // ---- mask, online softmax (base-2 domain)
+    float mx[2] = {kNegInf, kNegInf};
+#pragma unroll
+    for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int r = e >> 1, col = nb * 8 + cpair + (e & 1);
+        float v = sacc[nb][e] * scale_log2;
+        if (needs_mask && !((bits[r] >> col) & 1u)) v = kNegInf;
+        sacc[nb][e] = v;
+        mx[r] = fmaxf(mx[r], v);
+      }
+    float alpha[2], m_use[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], 2));
+      const float m_new = fmaxf(st.m_run[r], mx[r]);
+      m_use[r] = (m_new == kNegInf) ? 0.f : m_new;
+      alpha[r] = fast_exp2(st.m_run[r] - m_use[r]);
+      st.m_run[r] = m_new;
+    }
+    float psum[2] = {0.f, 0.f};
+#pragma unroll
+    for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float pv = fast_exp2(sacc[nb][e] - m_use[e >> 1]);
+        sacc[nb][e] = pv;
+        psum[e >> 1] += pv;
+      }
+    st.l_run[0] = st.l_run[0] * alpha[0] + psum[0];
+    st.l_run[1] = st.l_run[1] * alpha[1] + psum[1];
+#pragma unroll
+    for (int nb = 0; nb < D / 8; ++nb) {
+      st.o[nb][0] *= alpha[0];
+      st.o[nb][1] *= alpha[0];
+      st.o[nb][2] *= alpha[1];
+      st.o[nb][3] *= alpha[1];
+    }
+    uint32_t pa[4];
+    pa[0] = pack_bf16(sacc[0][0], sacc[0][1]);
+    pa[1] = pack_bf16(sacc[0][2], sacc[0][3]);
+    pa[2] = pack_bf16(sacc[1][0], sacc[1][1]);
+    pa[3] = pack_bf16(sacc[1][2], sacc[1][3]);
+    // ---- O += P V
+    {
+      const int t = sub * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
+      const uint32_t rowaddr = vbase + t * 128;
+      const int csel = lane >> 4;
+#pragma unroll
+      for (int db = 0; db < KSTEPS; ++db) {
+        const int c = (db & 3) * 2 + csel;
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4_t(rowaddr + (db >> 2) * SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
+        mma_bf16(st.o[2 * db], pa, b0, b1);
+        mma_bf16(st.o[2 * db + 1], pa, b2, b3);
+      }
+    }
+  }
+}
+
+// Normalise and store the warp's rows: final bf16 output + LSE, or an fp32 partial for the merge.
+template <int D>
+__device__ __forceinline__ void rows_store(RowState<D>& st, const AttnParams& p, const PieItem& item, const PieReq& rq,
+                                           int rbase, int slot_rows, int lane) {
+  const int r_lo = lane >> 2, cpair = (lane & 3) * 2;
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    st.l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, st.l_run[r], 1);
+    st.l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, st.l_run[r], 2);
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (!st.valid[r]) continue;
+    const int gr = rbase + r_lo + r * 8;
+    const int tok = gr / p.G, head = item.kv_head * p.G + gr % p.G;
+    const float L = st.l_run[r];
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    const float lse = L > 0.f ? (st.m_run[r] + log2f(L)) * kLn2 : kNegInf;
+    if (item.partial_slot < 0) {
+      const int64_t oi = ((int64_t)(rq.q_start + tok) * p.n_q_heads + head);
+      __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D;
+#pragma unroll
+      for (int nb = 0; nb < D / 8; ++nb)
+        *reinterpret_cast<uint32_t*>(dst + nb * 8 + cpair) = pack_bf16(st.o[nb][2 * r] * inv, st.o[nb][2 * r + 1] * inv);
+      if ((lane & 3) == 0) p.lse[oi] = lse;
+    } else {
+      const int64_t si = (int64_t)item.partial_slot * slot_rows + (gr - item.row0);
+      float* dst = p.ws_o + si * D;
+#pragma unroll
+      for (int nb = 0; nb < D / 8; ++nb)
+        *reinterpret_cast<float2*>(dst + nb * 8 + cpair) = make_float2(st.o[nb][2 * r] * inv, st.o[nb][2 * r + 1] * inv);
+      if ((lane & 3) == 0) p.ws_lse[si] = lse;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------ split-KV decode
+// Every warp is an independent pipeline over its own contiguous share of the batch's page
+// visits (the planner cuts the visits into equal shares, one per warp of the grid).  The warp
+// keeps DEPTH bulk copies in flight into a private ring and refills a stage as soon as it has
+// consumed it, so there is no producer warp, no empty barrier and no block-level sync.
+template <int D, int P, int NW, int DEPTH>
+struct SplitCfg {
+  static constexpr int STAGE = 2 * P * D * 2;
+  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * 8 + 64;
+};
+
+template <int D, int P, int NW, int DEPTH>
+__global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams p, int n_warps) {
+  using C = SplitCfg<D, P, NW, DEPTH>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int wg = blockIdx.x * NW + warp;
+  if (wg >= n_warps) return;
+  uint8_t* stages = smem + warp * DEPTH * C::STAGE;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + NW * DEPTH * C::STAGE) + warp * DEPTH;
+  if (lane == 0) {
+    for (int s = 0; s < DEPTH; ++s) mbar_init(smem_u32(full_bar + s), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+
+  const int it0 = p.cta_ptr[wg], it1 = p.cta_ptr[wg + 1];
+  const int s0 = p.stream_ptr[wg], n_total = p.stream_ptr[wg + 1] - s0;
+  const int2* stream = p.stream + s0;
+
+  // issue the copy of stream position n into ring stage n % DEPTH (lane 0)
+  auto issue = [&](int n, int2 e) {
+    const uint32_t s = n % DEPTH;
+    // order this warp's generic-proxy accesses to the stage before the async-proxy overwrite
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_expect_tx(smem_u32(full_bar + s), C::STAGE);
+    bulk_g2s(smem_u32(stages + s * C::STAGE), p.pool + (int64_t)e.x * C::STAGE, C::STAGE, smem_u32(full_bar + s));
+  };
+  if (lane == 0)
+    for (int n = 0; n < DEPTH && n < n_total; ++n) issue(n, __ldg(stream + n));
+
+  int n = 0;  // stream position
+  for (int it = it0; it < it1; ++it) {
+    const PieItem item = p.items[it];
+    const PieReq rq = p.reqs[item.req];
+    RowState<D> st;
+    rows_init<D>(st, p, item, rq, item.row0, lane);
+    const int n_end = n + (item.page_end - item.page_begin);
+    for (; n < n_end; ++n) {
+      const uint32_t s = n % DEPTH, ph = (n / DEPTH) & 1;
+      const uint32_t lpf = (uint32_t)__ldg(&stream[n].y);
+      int2 e_next = make_int2(0, 0);
+      if (lane == 0 && n + DEPTH < n_total) e_next = __ldg(stream + n + DEPTH);  // latency hides behind the wait
+      mbar_wait(smem_u32(full_bar + s), ph, p.status);
+      page_compute<D, P>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
+      __syncwarp();
+      if (lane == 0 && n + DEPTH < n_total) issue(n + DEPTH, e_next);
+    }
+    rows_store<D>(st, p, item, rq, item.row0, 16, lane);
+  }
+}
+
+// ------------------------------------------------------------------------------ row-tile kernel
+// Prefill chunks and token trees: NW consumer warps own 16 query rows each and all walk the same
+// page stream, which a producer warp keeps filled through a ring of full / empty barriers.
+template <int D, int P, int NW, int NSTAGES>
 struct TileCfg {
   static constexpr int BLK = P * D * 2;       // one K (or V) block, bytes
   static constexpr int STAGE = 2 * BLK;       // K block then V block
-  static constexpr int SLAB = P * 128;
-  static constexpr int OROW = D + 8;          // padded fp32 row of the cross-warp merge area
-  static constexpr int MERGE_FLOATS = SPLIT ? NW * (16 * OROW + 32) : 0;
-  static constexpr int SMEM = NSTAGES * STAGE + 2 * NSTAGES * 8 + MERGE_FLOATS * 4 + 64;
+  static constexpr int SMEM = NSTAGES * STAGE + 2 * NSTAGES * 8 + ((NSTAGES + 3) & ~3) * 4 + 64;
 };
 
-template <int D, int P, int NW, bool SPLIT, int NSTAGES>
-__global__ void __launch_bounds__((NW + 1) * 32, 1) attn_mma_kernel(const AttnParams p) {
-  using C = TileCfg<D, P, NW, SPLIT, NSTAGES>;
-  constexpr int KSTEPS = D / 16;   // k-steps of QK^T, and 16-column groups of PV
-  constexpr int SUBS = P / 16;     // 16-token sub-tiles per page
+template <int D, int P, int NW, int NSTAGES>
+__global__ void __launch_bounds__((NW + 1) * 32, 1) attn_tile_kernel(const AttnParams p) {
+  using C = TileCfg<D, P, NW, NSTAGES>;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* stages = smem;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + NSTAGES * C::STAGE);
   uint64_t* empty_bar = full_bar + NSTAGES;
-  float* merge = reinterpret_cast<float*>(empty_bar + NSTAGES);
+  uint32_t* meta = reinterpret_cast<uint32_t*>(empty_bar + NSTAGES);  // per stage: logical page | flag
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
       mbar_init(smem_u32(full_bar + s), 1);
-      mbar_init(smem_u32(empty_bar + s), SPLIT ? 1 : NW);
+      mbar_init(smem_u32(empty_bar + s), NW);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -130,278 +391,51 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) attn_mma_kernel(const AttnPa
   const int it0 = p.cta_ptr[blockIdx.x], it1 = p.cta_ptr[blockIdx.x + 1];
 
   if (warp == NW) {
-    // ------------------------------------------------------------------ producer (one lane)
-    if (lane == 0) {
-      uint32_t cnt = 0;
-      for (int it = it0; it < it1; ++it) {
-        const PieItem item = p.items[it];
-        const uint8_t* base = p.pool + (int64_t)item.kv_head * C::STAGE;
-        for (int k = item.page_begin; k < item.page_end; ++k, ++cnt) {
+    // ---- producer warp: LANES copies per step; stages of one step are distinct, and the warp
+    // re-converges after every step so that no lane runs ahead into a later ring phase
+    constexpr int LANES = NSTAGES / 2 < 32 ? NSTAGES / 2 : 32;
+    uint32_t cnt_base = 0;
+    for (int it = it0; it < it1; ++it) {
+      const PieItem item = p.items[it];
+      const uint8_t* base = p.pool + (int64_t)item.kv_head * C::STAGE;
+      const int npages = item.page_end - item.page_begin;
+      for (int k0 = 0; k0 < npages; k0 += LANES) {
+        const int kk = k0 + lane;
+        if (lane < LANES && kk < npages) {
+          const uint32_t cnt = cnt_base + kk;
           const uint32_t s = cnt % NSTAGES, ph = (cnt / NSTAGES) & 1;
-          const int phys = p.kept[k].x;
+          const int2 kp = __ldg(p.kept + item.page_begin + kk);
           mbar_wait(smem_u32(empty_bar + s), ph ^ 1, p.status);
+          meta[s] = (uint32_t)kp.y;
           mbar_expect_tx(smem_u32(full_bar + s), C::STAGE);
-          bulk_g2s(smem_u32(stages + s * C::STAGE), base + (int64_t)phys * p.page_bytes, C::STAGE,
+          bulk_g2s(smem_u32(stages + s * C::STAGE), base + (int64_t)kp.x * p.page_bytes, C::STAGE,
                    smem_u32(full_bar + s));
         }
+        __syncwarp();
       }
+      cnt_base += npages;
     }
     return;
   }
 
-  // ---------------------------------------------------------------------- consumers
-  const int G = p.G;
-  const int r_lo = lane >> 2;            // this thread's rows: r_lo and r_lo + 8
-  const int cpair = (lane & 3) * 2;      // its columns inside an 8-wide block: cpair, cpair + 1
-  uint32_t cnt_base = 0;
-
+  // ---- consumers
+  uint32_t cnt = 0;
   for (int it = it0; it < it1; ++it) {
     const PieItem item = p.items[it];
     const PieReq rq = p.reqs[item.req];
-    const int rbase = item.row0 + (SPLIT ? 0 : warp * 16);
-    const int row_end = item.row0 + item.nrows;
-    const bool explicit_mask = rq.mask_row_words != 0;
-
-    bool valid[2];
-    int lim[2];
-    const uint32_t* mrow[2];
-    const __nv_bfloat16* qptr[2];
-    for (int r = 0; r < 2; ++r) {
-      const int gr = rbase + r_lo + r * 8;
-      valid[r] = gr < row_end;
-      const int tok = valid[r] ? gr / G : 0;
-      const int head = item.kv_head * G + (valid[r] ? gr % G : 0);
-      lim[r] = valid[r] ? rq.kv_len - rq.q_len + tok : -1;
-      mrow[r] = p.mask + rq.mask_word_off + (int64_t)tok * rq.mask_row_words;
-      qptr[r] = reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)(rq.q_start + tok) * p.n_q_heads + head) * D;
-    }
-    const bool warp_has_rows = rbase < row_end;
-
-    // Q fragments (A operand, 16 rows x D)
-    uint32_t qf[KSTEPS][4];
-#pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) {
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        uint32_t lo = 0, hi = 0;
-        if (valid[r]) {
-          lo = *reinterpret_cast<const uint32_t*>(qptr[r] + ks * 16 + cpair);
-          hi = *reinterpret_cast<const uint32_t*>(qptr[r] + ks * 16 + 8 + cpair);
-        }
-        qf[ks][r] = lo;
-        qf[ks][2 + r] = hi;
-      }
-    }
-
-    float m_run[2] = {kNegInf, kNegInf}, l_run[2] = {0.f, 0.f};
-    float o[D / 8][4];
-#pragma unroll
-    for (int nb = 0; nb < D / 8; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
-
+    const int rbase = item.row0 + warp * 16;
+    RowState<D> st;
+    rows_init<D>(st, p, item, rq, rbase, lane);
     const int npages = item.page_end - item.page_begin;
-    for (int kk = 0; kk < npages; ++kk) {
-      if (SPLIT && (kk % NW) != warp) continue;
-      const uint32_t cnt = cnt_base + kk;
+    for (int kk = 0; kk < npages; ++kk, ++cnt) {
       const uint32_t s = cnt % NSTAGES, ph = (cnt / NSTAGES) & 1;
-      const uint32_t lpf = (uint32_t)p.kept[item.page_begin + kk].y;
-      const int lp = (int)(lpf & ~PIE_KEPT_NEEDS_MASK);
-      const bool needs_mask = (lpf & PIE_KEPT_NEEDS_MASK) != 0;
       mbar_wait(smem_u32(full_bar + s), ph, p.status);
-      const uint32_t kbase = smem_u32(stages + s * C::STAGE);
-      const uint32_t vbase = kbase + C::BLK;
-
-      if (lp == rq.last_logical && rq.last_page_len < P) {
-        // slots past the end of the context may hold anything: clear their V rows so that a
-        // zero probability times a NaN bit pattern cannot leak into the output
-        constexpr int CH = D * 2 / 16;
-        uint8_t* v = stages + s * C::STAGE + C::BLK;
-        const int nz = (P - rq.last_page_len) * CH;
-        for (int c = lane; c < nz; c += 32) {
-          const int t = rq.last_page_len + c / CH, ch = c % CH;
-          *reinterpret_cast<uint4*>(v + pie_chunk_offset(C::SLAB, t, ch)) = make_uint4(0, 0, 0, 0);
-        }
-        __syncwarp();
-      }
-
-      if (warp_has_rows) {
-#pragma unroll
-        for (int sub = 0; sub < SUBS; ++sub) {
-          const int j0 = lp * P + sub * 16;
-          uint32_t bits[2] = {0xFFFFu, 0xFFFFu};
-          if (needs_mask) {
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-              if (!valid[r]) bits[r] = 0;
-              else if (explicit_mask) bits[r] = (__ldg(mrow[r] + (j0 >> 5)) >> (j0 & 31)) & 0xFFFFu;
-              else bits[r] = lim[r] >= j0 + 15 ? 0xFFFFu : (lim[r] < j0 ? 0u : ((1u << (lim[r] - j0 + 1)) - 1u));
-            }
-            if (__all_sync(0xFFFFFFFFu, (bits[0] | bits[1]) == 0)) continue;  // nothing visible to this warp
-          }
-          // ---- S = Q K^T for 16 tokens
-          float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-          {
-            const int t = sub * 16 + ((lane >> 4) << 3) + (lane & 7);
-            const uint32_t rowaddr = kbase + t * 128;
-            const int csel = (lane >> 3) & 1;
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-              const int c = (ks & 3) * 2 + csel;
-              uint32_t b0, b1, b2, b3;
-              ldsm_x4(rowaddr + (ks >> 2) * C::SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
-              mma_bf16(sacc[0], qf[ks], b0, b1);
-              mma_bf16(sacc[1], qf[ks], b2, b3);
-            }
-          }
-          // ---- mask, online softmax (base-2 domain)
-          float mx[2] = {kNegInf, kNegInf};
-#pragma unroll
-          for (int nb = 0; nb < 2; ++nb)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int r = e >> 1, col = nb * 8 + cpair + (e & 1);
-              float v = sacc[nb][e] * p.scale_log2;
-              if (needs_mask && !((bits[r] >> col) & 1u)) v = kNegInf;
-              sacc[nb][e] = v;
-              mx[r] = fmaxf(mx[r], v);
-            }
-          float alpha[2], m_use[2];
-#pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], 1));
-            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], 2));
-            const float m_new = fmaxf(m_run[r], mx[r]);
-            m_use[r] = (m_new == kNegInf) ? 0.f : m_new;
-            alpha[r] = fast_exp2(m_run[r] - m_use[r]);
-            m_run[r] = m_new;
-          }
-          float psum[2] = {0.f, 0.f};
-#pragma unroll
-          for (int nb = 0; nb < 2; ++nb)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float pv = fast_exp2(sacc[nb][e] - m_use[e >> 1]);
-              sacc[nb][e] = pv;
-              psum[e >> 1] += pv;
-            }
-          l_run[0] = l_run[0] * alpha[0] + psum[0];
-          l_run[1] = l_run[1] * alpha[1] + psum[1];
-#pragma unroll
-          for (int nb = 0; nb < D / 8; ++nb) {
-            o[nb][0] *= alpha[0];
-            o[nb][1] *= alpha[0];
-            o[nb][2] *= alpha[1];
-            o[nb][3] *= alpha[1];
-          }
-          uint32_t pa[4];
-          pa[0] = pack_bf16(sacc[0][0], sacc[0][1]);
-          pa[1] = pack_bf16(sacc[0][2], sacc[0][3]);
-          pa[2] = pack_bf16(sacc[1][0], sacc[1][1]);
-          pa[3] = pack_bf16(sacc[1][2], sacc[1][3]);
-          // ---- O += P V
-          {
-            const int t = sub * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
-            const uint32_t rowaddr = vbase + t * 128;
-            const int csel = lane >> 4;
-#pragma unroll
-            for (int db = 0; db < KSTEPS; ++db) {
-              const int c = (db & 3) * 2 + csel;
-              uint32_t b0, b1, b2, b3;
-              ldsm_x4_t(rowaddr + (db >> 2) * C::SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
-              mma_bf16(o[2 * db], pa, b0, b1);
-              mma_bf16(o[2 * db + 1], pa, b2, b3);
-            }
-          }
-        }
-      }
+      const uint32_t lpf = meta[s];
+      page_compute<D, P>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(empty_bar + s));
     }
-    cnt_base += npages;
-
-    // ---- row sums across the quad
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, l_run[r], 1);
-      l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, l_run[r], 2);
-    }
-
-    if constexpr (SPLIT) {
-      // ---- merge the NW private softmax states of this item
-      float* wm = merge + warp * (16 * C::OROW + 32);
-      float* wl = wm + 16;
-      float* wo = wm + 32;
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const int row = r_lo + r * 8;
-        if ((lane & 3) == 0) {
-          wm[row] = m_run[r];
-          wl[row] = l_run[r];
-        }
-#pragma unroll
-        for (int nb = 0; nb < D / 8; ++nb)
-          *reinterpret_cast<float2*>(wo + row * C::OROW + nb * 8 + cpair) = make_float2(o[nb][2 * r], o[nb][2 * r + 1]);
-      }
-      asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
-      const int tid = threadIdx.x;
-      for (int e = tid; e < item.nrows * (D / 2); e += NW * 32) {
-        const int row = e / (D / 2), d = (e % (D / 2)) * 2;
-        float M = kNegInf;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) M = fmaxf(M, merge[w * (16 * C::OROW + 32) + row]);
-        float L = 0.f, a0 = 0.f, a1 = 0.f;
-        if (M != kNegInf) {
-#pragma unroll
-          for (int w = 0; w < NW; ++w) {
-            const float* b = merge + w * (16 * C::OROW + 32);
-            const float sc = fast_exp2(b[row] - M);
-            L += b[16 + row] * sc;
-            const float2 ov = *reinterpret_cast<const float2*>(b + 32 + row * C::OROW + d);
-            a0 += ov.x * sc;
-            a1 += ov.y * sc;
-          }
-        }
-        const float inv = L > 0.f ? 1.f / L : 0.f;
-        const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : kNegInf;
-        const int gr = item.row0 + row;
-        const int tok = gr / G, head = item.kv_head * G + gr % G;
-        if (item.partial_slot < 0) {
-          const int64_t oi = ((int64_t)(rq.q_start + tok) * p.n_q_heads + head);
-          *reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D + d) = pack_bf16(a0 * inv, a1 * inv);
-          if (d == 0) p.lse[oi] = lse;
-        } else {
-          const int64_t si = (int64_t)item.partial_slot * 16 + row;
-          *reinterpret_cast<float2*>(p.ws_o + si * D + d) = make_float2(a0 * inv, a1 * inv);
-          if (d == 0) p.ws_lse[si] = lse;
-        }
-      }
-      asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
-    } else {
-      // ---- each warp owns its rows: write straight from registers
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        if (!valid[r]) continue;
-        const int gr = rbase + r_lo + r * 8;
-        const int tok = gr / G, head = item.kv_head * G + gr % G;
-        const float L = l_run[r];
-        const float inv = L > 0.f ? 1.f / L : 0.f;
-        const float lse = L > 0.f ? (m_run[r] + log2f(L)) * kLn2 : kNegInf;
-        if (item.partial_slot < 0) {
-          const int64_t oi = ((int64_t)(rq.q_start + tok) * p.n_q_heads + head);
-          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D;
-#pragma unroll
-          for (int nb = 0; nb < D / 8; ++nb)
-            *reinterpret_cast<uint32_t*>(dst + nb * 8 + cpair) = pack_bf16(o[nb][2 * r] * inv, o[nb][2 * r + 1] * inv);
-          if ((lane & 3) == 0) p.lse[oi] = lse;
-        } else {
-          const int64_t si = (int64_t)item.partial_slot * (NW * 16) + (gr - item.row0);
-          float* dst = p.ws_o + si * D;
-#pragma unroll
-          for (int nb = 0; nb < D / 8; ++nb)
-            *reinterpret_cast<float2*>(dst + nb * 8 + cpair) = make_float2(o[nb][2 * r] * inv, o[nb][2 * r + 1] * inv);
-          if ((lane & 3) == 0) p.ws_lse[si] = lse;
-        }
-      }
-    }
+    rows_store<D>(st, p, item, rq, rbase, NW * 16, lane);
   }
 }
 
@@ -421,7 +455,9 @@ __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* 
     if (M != kNegInf) {
       for (int c = 0; c < mg.nslots; ++c) {
         const int64_t si = (int64_t)(mg.slot0 + c) * slot_rows + row;
-        const float w = __expf(ws_lse[si] - M);
+        const float l = ws_lse[si];
+        if (l == kNegInf) continue;  // an empty partial: its O rows were never written
+        const float w = __expf(l - M);
         Z += w;
         acc += w * ws_o[si * D + d];
       }
@@ -507,6 +543,8 @@ AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& 
   p.mask = plan->d_mask;
   p.items = ll.d_items;
   p.cta_ptr = ll.d_cta_ptr;
+  p.stream = ll.d_stream;
+  p.stream_ptr = ll.d_stream_ptr;
   p.ws_o = ll.d_ws_o;
   p.ws_lse = ll.d_ws_lse;
   p.status = ctx->d_status;
@@ -518,11 +556,26 @@ AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& 
   return p;
 }
 
-template <int D, int P, int NW, bool SPLIT>
-int launch_tile_kernel(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
+template <int D, int P, int NW, int DEPTH>
+int launch_split(pie_ctx* ctx, const AttnParams& p, int n_warps, cudaStream_t s) {
+  using C = SplitCfg<D, P, NW, DEPTH>;
+  auto kern = attn_split_kernel<D, P, NW, DEPTH>;
+  static bool configured[8] = {};
+  int dev = ctx->cfg.device & 7;
+  if (!configured[dev]) {
+    PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+    configured[dev] = true;
+  }
+  kern<<<(n_warps + NW - 1) / NW, NW * 32, C::SMEM, s>>>(p, n_warps);
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}
+
+template <int D, int P, int NW>
+int launch_tiles(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
   constexpr int NSTAGES = (128 * 1024) / (2 * P * D * 2);
-  using C = TileCfg<D, P, NW, SPLIT, NSTAGES>;
-  auto kern = attn_mma_kernel<D, P, NW, SPLIT, NSTAGES>;
+  using C = TileCfg<D, P, NW, NSTAGES>;
+  auto kern = attn_tile_kernel<D, P, NW, NSTAGES>;
   static bool configured[8] = {};
   int dev = ctx->cfg.device & 7;
   if (!configured[dev]) {
@@ -534,16 +587,6 @@ int launch_tile_kernel(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t
   return PIE_OK;
 }
 
-template <bool SPLIT, int NW>
-int dispatch_tile(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
-  const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size;
-  if (D == 64 && P == 16) return launch_tile_kernel<64, 16, NW, SPLIT>(ctx, p, grid, s);
-  if (D == 128 && P == 16) return launch_tile_kernel<128, 16, NW, SPLIT>(ctx, p, grid, s);
-  if (D == 64 && P == 32) return launch_tile_kernel<64, 32, NW, SPLIT>(ctx, p, grid, s);
-  if (D == 128 && P == 32) return launch_tile_kernel<128, 32, NW, SPLIT>(ctx, p, grid, s);
-  return PIE_ERR_UNSUPPORTED;
-}
-
 }  // namespace
 
 bool pie_split_supported(const pie_ctx* ctx) {
@@ -552,14 +595,30 @@ bool pie_split_supported(const pie_ctx* ctx) {
          ctx->G <= 16;
 }
 
+// Warps per block of the split-KV kernel (the planner sizes its shares with this).
+int pie_split_warps_per_block(const pie_ctx* ctx) {
+  return (ctx->cfg.page_size == 32 && ctx->cfg.head_dim == 128) ? 4 : 8;
+}
+
 int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s) {
   AttnParams p = make_params(ctx, plan, plan->split, q, out, lse);
-  return dispatch_tile<true, 8>(ctx, p, plan->split.grid, s);
+  const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size, n = plan->split.grid;
+  // ring depth: about 192 KB of copies in flight per SM
+  if (D == 64 && P == 16) return launch_split<64, 16, 8, 6>(ctx, p, n, s);
+  if (D == 128 && P == 16) return launch_split<128, 16, 8, 3>(ctx, p, n, s);
+  if (D == 64 && P == 32) return launch_split<64, 32, 8, 3>(ctx, p, n, s);
+  if (D == 128 && P == 32) return launch_split<128, 32, 4, 3>(ctx, p, n, s);
+  return PIE_ERR_UNSUPPORTED;
 }
 
 int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s) {
   AttnParams p = make_params(ctx, plan, plan->tile, q, out, lse);
-  return dispatch_tile<false, 4>(ctx, p, plan->tile.grid, s);
+  const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size, grid = plan->tile.grid;
+  if (D == 64 && P == 16) return launch_tiles<64, 16, 4>(ctx, p, grid, s);
+  if (D == 128 && P == 16) return launch_tiles<128, 16, 4>(ctx, p, grid, s);
+  if (D == 64 && P == 32) return launch_tiles<64, 32, 4>(ctx, p, grid, s);
+  if (D == 128 && P == 32) return launch_tiles<128, 32, 4>(ctx, p, grid, s);
+  return PIE_ERR_UNSUPPORTED;
 }
 
 int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s) {

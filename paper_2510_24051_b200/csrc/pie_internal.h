@@ -71,6 +71,12 @@ struct PieLaunchList {           // one tile-kernel launch (split-KV decode, or 
   int32_t grid = 0;
   int32_t n_slots = 0;
   int32_t slot_rows = 0;
+  // split-KV kernel only: the page visits of every share, flattened in item order.
+  // entry = (physical page * H_kv + kv head, logical page | needs-mask flag)
+  std::vector<int32_t> stream;
+  std::vector<int32_t> stream_ptr;  // [grid+1]
+  int2* d_stream = nullptr;
+  int32_t* d_stream_ptr = nullptr;
   // device copies
   PieItem* d_items = nullptr;
   int32_t* d_cta_ptr = nullptr;
@@ -139,6 +145,8 @@ struct AttnParams {
   const uint32_t* mask;
   const PieItem* items;
   const int32_t* cta_ptr;
+  const int2* stream;
+  const int32_t* stream_ptr;
   float* ws_o;
   float* ws_lse;
   int* status;
@@ -155,7 +163,7 @@ int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, void* ou
 int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);
 int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s);
 bool pie_split_supported(const pie_ctx* ctx);
-size_t pie_split_smem_bytes(const pie_ctx* ctx);
+int pie_split_warps_per_block(const pie_ctx* ctx);
 
 int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);  // host part (planner.cc)
 

@@ -269,7 +269,23 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
         }
     }
   }
-  partition(split_units, ctx->n_sms, 8, 16, plan->split);
+  // split-KV decode: one share per warp of a full grid (every warp is its own pipeline)
+  partition(split_units, ctx->n_sms * pie_split_warps_per_block(ctx), 4, 16, plan->split);
+  {
+    PieLaunchList& ll = plan->split;
+    ll.stream.clear();
+    ll.stream_ptr.assign(1, 0);
+    for (int c = 0; c < ll.grid; ++c) {
+      for (int k = ll.cta_ptr[c]; k < ll.cta_ptr[c + 1]; ++k) {
+        const PieItem& it = ll.items[k];
+        for (int e = it.page_begin; e < it.page_end; ++e) {
+          ll.stream.push_back(plan->kept[2 * e] * cfg.num_kv_heads + it.kv_head);
+          ll.stream.push_back(plan->kept[2 * e + 1]);
+        }
+      }
+      ll.stream_ptr.push_back((int32_t)(ll.stream.size() / 2));
+    }
+  }
   partition(tile_units, ctx->n_sms, 8, TILE_ROWS, plan->tile);
 
   pie_plan_info& info = plan->info;
