@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (null until a capture exists for that workload).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"batched_decode": 288_890_000}   # profiles/attn_split_kernel_batched_decode.md
 
 
 def load_peaks():
@@ -259,12 +259,9 @@ def main():
     ev1.record()
     barrier()
     ms = ev0.elapsed_time(ev1)
-    clocks = sampler.stop() if rank == 0 else None
     assert pie.pie_get_last_device_status(ctx) == 0, "a device-side wait timed out"
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2510_24051_b200 import shard
+    total_tokens, ms = shard.aggregate(wl0.T, ms)          # sum of tokens, slowest rank's time
     launches_per_step = info["launches"] + (1 if copies is not None else 0)
 
     # ---------------------------------------------------------------- per-kernel timing (live)
@@ -274,6 +271,7 @@ def main():
     torch.cuda.synchronize()
     ktimes = pie.pie_get_kernel_times(ctx)
     pie.pie_set_kernel_timing(ctx, 0)
+    clocks = sampler.stop() if rank == 0 else None         # covers both timed loops
 
     # ---------------------------------------------------------------- end to end (host buffers)
     e2e = None
@@ -354,7 +352,7 @@ def main():
     ms_per_step = ms / args.steps
     alg_bytes = wl0.algorithmic_bytes()
     line = {
-        "metric": METRIC, "value": world * wl0.T / (ms_per_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+        "metric": METRIC, "value": total_tokens / (ms_per_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": wl0.dtype, "data": "synthetic",
         "config": {"workload": wl0.name, "requests": wl0.R, "query_tokens": wl0.T, "heads": f"{wl0.H_q}/{wl0.H_kv}",

@@ -238,3 +238,7 @@ def pie_get_kernel_times(ctx):
     n = np.zeros(len(KERNEL_KINDS), dtype=np.int32)
     _check(lib.pie_get_kernel_times(ctx, ms.ctypes.data, n.ctypes.data), ctx)
     return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}
+
+
+def pie_last_cuda_error(ctx):
+    return lib.pie_last_cuda_error(ctx).decode()

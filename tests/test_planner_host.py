@@ -1,0 +1,137 @@
+"""Host logic of the library on a host-only context: allocator, batch validation (the
+vertical-batching conflict rule, size limits), mask packing, page dropping, append positions."""
+import numpy as np
+import pytest
+
+import paper_2510_24051_b200 as pie
+from workloads import configs
+
+
+@pytest.fixture
+def ctx():
+    c = pie.pie_create(256, 16, 8, 2, 64, "bf16", 8, 256, device=-1)
+    yield c
+    pie.pie_destroy(c)
+
+
+def status_of(fn, *a, **k):
+    try:
+        fn(*a, **k)
+    except pie.PieError as e:
+        return e.status
+    return pie.PIE_OK
+
+
+def test_allocator_fcfs_and_errors(ctx):
+    a = pie.pie_alloc_kvpages(ctx, 200)
+    assert len(set(a.tolist())) == 200 and pie.pie_num_free_kvpages(ctx) == 56
+    assert status_of(pie.pie_alloc_kvpages, ctx, 57) == pie.PIE_ERR_NO_PAGES      # nothing allocated
+    assert pie.pie_num_free_kvpages(ctx) == 56
+    pie.pie_dealloc_kvpages(ctx, a[:10])
+    assert pie.pie_num_free_kvpages(ctx) == 66
+    assert status_of(pie.pie_dealloc_kvpages, ctx, a[:1]) == pie.PIE_ERR_BAD_PAGE  # double free
+    assert status_of(pie.pie_dealloc_kvpages, ctx, [a[20], a[20]]) == pie.PIE_ERR_BAD_PAGE
+    assert status_of(pie.pie_dealloc_kvpages, ctx, [999]) == pie.PIE_ERR_BAD_PAGE
+    assert pie.pie_num_free_kvpages(ctx) == 66
+    assert len(pie.pie_alloc_kvpages(ctx, 0)) == 0
+
+
+def test_validation_errors(ctx):
+    ids = pie.pie_alloc_kvpages(ctx, 32)
+    ok = lambda **k: status_of(pie.pie_plan_forward, ctx, **k)
+    base = dict(qo_indptr=[0, 1, 3], page_indptr=[0, 2, 4], page_indices=ids[:4], last_page_len=[5, 16])
+    assert ok(**base) == pie.PIE_OK
+    assert ok(**dict(base, last_page_len=[0, 16])) == pie.PIE_ERR_INVALID
+    assert ok(**dict(base, last_page_len=[5, 17])) == pie.PIE_ERR_INVALID
+    assert ok(**dict(base, qo_indptr=[0, 0, 3])) == pie.PIE_ERR_INVALID            # q_len < 1
+    assert ok(qo_indptr=[0, 20], page_indptr=[0, 1], page_indices=ids[:1], last_page_len=[16]) == pie.PIE_ERR_INVALID  # kv_len < q_len
+    assert ok(**dict(base, page_indices=[ids[0], 250, ids[2], ids[3]])) == pie.PIE_ERR_BAD_PAGE  # not allocated
+    assert ok(**dict(base, page_indices=[ids[0], -1, ids[2], ids[3]])) == pie.PIE_ERR_BAD_PAGE
+    # batch size limits (the scheduler truncates; the library refuses)
+    R = 9
+    assert ok(qo_indptr=np.arange(R + 1), page_indptr=np.arange(R + 1), page_indices=ids[:R],
+              last_page_len=np.ones(R)) == pie.PIE_ERR_BATCH_TOO_LARGE
+    assert ok(qo_indptr=[0, 257], page_indptr=[0, 17], page_indices=ids[:17], last_page_len=[16]) == pie.PIE_ERR_BATCH_TOO_LARGE
+    # mask of the wrong size / with a byte that is not 0 or 1
+    assert ok(**dict(base, mask_indptr=[0, 0, 10], mask=np.ones(10, np.uint8))) == pie.PIE_ERR_MASK
+    m = np.ones(2 * 32, np.uint8)
+    assert ok(**dict(base, mask_indptr=[0, 0, 64], mask=m)) == pie.PIE_OK
+    m[5] = 2
+    assert ok(**dict(base, mask_indptr=[0, 0, 64], mask=m)) == pie.PIE_ERR_MASK
+    # an empty batch plans to nothing
+    assert ok(qo_indptr=[0], page_indptr=[0], page_indices=[], last_page_len=[]) == pie.PIE_OK
+
+
+def test_conflict_rule(ctx):
+    ids = pie.pie_alloc_kvpages(ctx, 8)
+    plan = lambda **k: status_of(pie.pie_plan_forward, ctx, **k)
+    # two requests append into the same slot of a shared last page
+    assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 2, 4], page_indices=[ids[0], ids[1], ids[2], ids[1]],
+                last_page_len=[4, 4]) == pie.PIE_ERR_CONFLICT
+    # request 1 reads (as context) a slot request 0 writes
+    assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 1, 3], page_indices=[ids[0], ids[0], ids[2]],
+                last_page_len=[4, 4]) == pie.PIE_ERR_CONFLICT
+    # sharing read-only pages is legal; so is reading slots below the other request's write
+    assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 2, 4], page_indices=[ids[0], ids[1], ids[0], ids[2]],
+                last_page_len=[4, 4]) == pie.PIE_OK
+    assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 1, 3], page_indices=[ids[0], ids[3], ids[0]],
+                last_page_len=[9, 3]) == pie.PIE_ERR_CONFLICT   # req 1 appends slot 2, req 0 reads slots 0..8
+    # a request that lists the same page twice and would write it through both positions
+    assert plan(qo_indptr=[0, 20], page_indptr=[0, 2], page_indices=[ids[4], ids[4]],
+                last_page_len=[16]) == pie.PIE_ERR_CONFLICT
+    # copy_kvpage conflicts are found on the host too
+    assert status_of(pie.pie_copy_kvpage, ctx, [ids[0], ids[1]], [ids[2], ids[2]], [0, 0], [0, 4], [8, 8]) == pie.PIE_ERR_CONFLICT
+    assert status_of(pie.pie_copy_kvpage, ctx, [ids[0]], [ids[0]], [0], [4], [8]) == pie.PIE_ERR_CONFLICT
+    assert status_of(pie.pie_copy_kvpage, ctx, [ids[0]], [ids[1]], [10], [0], [8]) == pie.PIE_ERR_INVALID
+    assert status_of(pie.pie_copy_kvpage, ctx, [ids[0]], [200], [0], [0], [8]) == pie.PIE_ERR_BAD_PAGE
+
+
+@pytest.mark.parametrize("name", ["tiny_fp32", "shared_prefix_tree", "long_context_policy", "mixed_prefill_decode"])
+def test_plan_arrays_match_numpy(name):
+    wl = configs.small(name)
+    ctx = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+    try:
+        pie.pie_alloc_kvpages(ctx, wl.num_pages)
+        mi, mb = wl.mask_bytes()
+        plan = pie.pie_plan_forward(ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len, mi, mb)
+        info = pie.pie_plan_get_info(plan)
+        words = pie.pie_plan_debug_read(plan, 0)
+        kept = pie.pie_plan_debug_read(plan, 1).reshape(-1, 2)
+        app = pie.pie_plan_debug_read(plan, 2)
+        pie.pie_plan_destroy(plan)
+    finally:
+        pie.pie_destroy(ctx)
+    kv, ql, P = wl.kv_lens(), wl.q_lens(), wl.P
+    # append destinations = the oracle's positions
+    exp = []
+    for r in range(wl.R):
+        for i in range(ql[r]):
+            pos = kv[r] - ql[r] + i
+            exp.append(int(wl.pages_of(r)[pos // P]) * P + pos % P)
+    assert app.tolist() == exp
+    # packed masks: LSB first, rows padded to 128 bits; kept pages: exactly those some row attends to
+    woff, koff = 0, 0
+    for r in range(wl.R):
+        m = None if wl.masks is None else wl.masks[r]
+        npg = len(wl.pages_of(r))
+        if m is None:
+            keep = np.ones(npg, bool)
+            lim0 = kv[r] - ql[r]
+            needs = np.array([lp * P + P - 1 > lim0 for lp in range(npg)])
+        else:
+            rw = ((kv[r] + 127) // 128) * 4
+            padded = np.zeros((ql[r], rw * 32), np.uint8)
+            padded[:, :kv[r]] = m
+            expw = np.packbits(padded, axis=1, bitorder="little").view(np.uint32).reshape(ql[r], rw)
+            assert np.array_equal(words[woff:woff + ql[r] * rw].reshape(ql[r], rw), expw)
+            woff += ql[r] * rw
+            pg = padded[:, :npg * P].reshape(ql[r], npg, P)
+            keep = pg.any(axis=(0, 2))
+            needs = ~pg.all(axis=(0, 2))
+        n = int(keep.sum())
+        got = kept[koff:koff + n]
+        assert np.array_equal(got[:, 0], wl.pages_of(r)[keep])
+        assert np.array_equal(got[:, 1] & 0x7FFFFFFF, np.nonzero(keep)[0])
+        assert np.array_equal((got[:, 1] < 0), needs[keep])
+        koff += n
+    assert koff == info["kept_pages"] and woff == info["mask_words"]
