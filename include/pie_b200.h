@@ -184,6 +184,34 @@ int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, c
  * gave up since the last call.  Synchronises `stream`, reads and clears the word. */
 int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out);
 
+/* forward for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for the embedding application, not for the method.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they run a batch: code
+ * running under a memory manager that owns the whole device heap, code that must not trigger the
+ * implicit synchronisation of cudaMalloc / cudaFree inside a latency-critical serving loop, or
+ * code running after its allocator has been frozen.  pie_plan_forward allocates the device copy
+ * of the plan and the fp32 scratch of the split-KV kernels; this call does the same work as
+ * pie_plan_forward + pie_forward but keeps both in one fixed array that is part of the library
+ * image (a file-scope `static __device__` array of PIE_STATIC_SCRATCH_BYTES bytes; every GPU that
+ * loads the library holds it until the process exits).  It calls no cudaMalloc, no cudaFree and
+ * no allocating library routine; host-side planning uses ordinary host memory.
+ *
+ *   - Arguments, results and errors are those of pie_forward, with `batch` (host) as in
+ *     pie_plan_forward; q / k_new / v_new / out / lse are device pointers owned by the caller.
+ *   - A batch whose plan arrays plus split partials need more than PIE_STATIC_SCRATCH_BYTES is
+ *     refused with PIE_ERR_BATCH_TOO_LARGE and nothing is enqueued.
+ *   - The first call on a device looks up the array's device address (one cudaGetSymbolAddress,
+ *     with that device current); make that first call before any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents.  Nothing in it has
+ *     to start at zero (each call overwrites the plan arrays it reads and writes every partial
+ *     before reading it), but two calls whose device work overlaps - different streams, or
+ *     different contexts on the same GPU - race on it: keep them in one stream order. */
+enum { PIE_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 };
+int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* batch, const void* q,
+                               const void* k_new, const void* v_new, void* out, float* lse,
+                               void* stream);
+
 /* Per-kernel device timing for benchmarks.  While enabled, pie_forward and pie_copy_kvpage
  * bracket each kernel they enqueue with CUDA events on the caller's stream.
  * pie_get_kernel_times waits for the recorded events, adds the elapsed milliseconds and the

@@ -69,6 +69,7 @@ def _load():
         "pie_forward": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, vp]),
         "pie_forward_host": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
         "pie_get_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int)]),
+        "pie_forward_static_scratch": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
         "pie_set_kernel_timing": (C.c_int, [vp, C.c_int]),
         "pie_get_kernel_times": (C.c_int, [vp, vp, vp]),
     }
@@ -242,3 +243,16 @@ def pie_get_kernel_times(ctx):
 
 def pie_last_cuda_error(ctx):
     return lib.pie_last_cuda_error(ctx).decode()
+
+
+PIE_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def pie_forward_static_scratch(ctx, qo_indptr, page_indptr, page_indices, last_page_len, q, k_new, v_new,
+                               out, lse, mask_indptr=None, mask=None, flags=0, stream=None):
+    """forward for callers that cannot allocate device memory: plan arrays and split partials go
+    to the library's fixed device array (at most PIE_STATIC_SCRATCH_BYTES, else
+    PIE_ERR_BATCH_TOO_LARGE).  Tensors are device tensors; calls must not overlap on the GPU."""
+    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags)
+    _check(lib.pie_forward_static_scratch(ctx, C.byref(d), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
+                                          _ptr(lse), _stream(stream)), ctx)

@@ -11,6 +11,8 @@
 //     kernels do not cover); one warp per (token, head) row, sequential online softmax.
 #include <cuda_bf16.h>
 
+#include <cstring>
+
 #include "pie_internal.h"
 
 namespace {
@@ -652,5 +654,95 @@ int pie_launch_simple(pie_ctx* ctx, const pie_plan* plan, const void* q, void* o
   }
 #undef PIE_SIMPLE
   PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}
+
+
+// ------------------------------------------------------------------------------ forward without allocation
+// Scratch for pie_forward_static_scratch: the uploaded plan arrays and the fp32 split partials
+// live in this file-scope array instead of a cudaMalloc'd buffer.  Every GPU that loads the
+// library holds it until the process exits.  In host code the name below is only a stand-in
+// for the symbol; its device address is looked up once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char pie_static_scratch[PIE_STATIC_SCRATCH_BYTES];
+static void* g_static_scratch_addr[64] = {};  // per device ordinal, filled on first use
+
+extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, const void* k_new,
+                                          const void* v_new, void* out, float* lse, void* stream) {
+  if (!ctx || !batch) return PIE_ERR_INVALID;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  const int dev = ctx->cfg.device;
+  if (dev < 0 || dev >= 64) return PIE_ERR_INVALID;
+  cudaStream_t s = (cudaStream_t)stream;
+  PIE_CUDA(ctx, cudaSetDevice(dev));
+  if (!g_static_scratch_addr[dev]) {  // set-up, once per device, with that device current
+    void* ptr = nullptr;
+    PIE_CUDA(ctx, cudaGetSymbolAddress(&ptr, pie_static_scratch));
+    g_static_scratch_addr[dev] = ptr;
+  }
+  uint8_t* base = static_cast<uint8_t*>(g_static_scratch_addr[dev]);
+
+  pie_plan plan;  // host-side only; its device pointers will point into the static scratch
+  plan.ctx = ctx;
+  int rc = pie_build_plan(ctx, batch, &plan);
+  if (rc != PIE_OK) return rc;
+  if (plan.T == 0) return PIE_OK;
+  if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
+
+  std::vector<uint8_t> host;
+  auto put = [&](const void* ptr, size_t bytes) {
+    size_t off = (host.size() + 255) & ~(size_t)255;
+    host.resize(off + bytes);
+    if (bytes) memcpy(host.data() + off, ptr, bytes);
+    return off;
+  };
+  const size_t o_reqs = put(plan.reqs.data(), plan.reqs.size() * sizeof(PieReq));
+  const size_t o_kept = put(plan.kept.data(), plan.kept.size() * 4);
+  const size_t o_mask = put(plan.mask_words.data(), plan.mask_words.size() * 4);
+  const size_t o_app = put(plan.append_dst.data(), plan.append_dst.size() * 4);
+  const size_t o_tok = put(plan.tok_req.data(), plan.tok_req.size() * 4);
+  const size_t o_simple = put(plan.simple_rows.data(), plan.simple_rows.size() * 4);
+  PieLaunchList* lls[2] = {&plan.split, &plan.tile};
+  size_t o_li[2], o_lc[2], o_lm[2], o_ls[2], o_lp[2], o_wo[2], o_wl[2];
+  for (int k = 0; k < 2; ++k) {
+    o_li[k] = put(lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
+    o_lc[k] = put(lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
+    o_lm[k] = put(lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
+    o_ls[k] = put(lls[k]->stream.data(), lls[k]->stream.size() * 4);
+    o_lp[k] = put(lls[k]->stream_ptr.data(), lls[k]->stream_ptr.size() * 4);
+  }
+  size_t total = (host.size() + 255) & ~(size_t)255;
+  const int D = ctx->cfg.head_dim;
+  for (int k = 0; k < 2; ++k) {
+    o_wo[k] = total;
+    total += (((size_t)lls[k]->n_slots * lls[k]->slot_rows * D * 4) + 255) & ~(size_t)255;
+    o_wl[k] = total;
+    total += (((size_t)lls[k]->n_slots * lls[k]->slot_rows * 4) + 255) & ~(size_t)255;
+  }
+  if (total > (size_t)PIE_STATIC_SCRATCH_BYTES) return PIE_ERR_BATCH_TOO_LARGE;  // plan + partials exceed the static scratch
+
+  // Nothing in the scratch has to start at zero: every plan array is overwritten by this copy
+  // and every partial row is written by the attention kernel before the merge reads it.
+  PIE_CUDA(ctx, cudaMemcpyAsync(base, host.data(), host.size(), cudaMemcpyHostToDevice, s));
+  plan.d_reqs = (PieReq*)(base + o_reqs);
+  plan.d_kept = (int2*)(base + o_kept);
+  plan.d_mask = (uint32_t*)(base + o_mask);
+  plan.d_append_dst = (int32_t*)(base + o_app);
+  plan.d_tok_req = (int32_t*)(base + o_tok);
+  plan.d_simple_rows = (int32_t*)(base + o_simple);
+  for (int k = 0; k < 2; ++k) {
+    lls[k]->d_items = (PieItem*)(base + o_li[k]);
+    lls[k]->d_cta_ptr = (int32_t*)(base + o_lc[k]);
+    lls[k]->d_merges = (PieMerge*)(base + o_lm[k]);
+    lls[k]->d_stream = (int2*)(base + o_ls[k]);
+    lls[k]->d_stream_ptr = (int32_t*)(base + o_lp[k]);
+    lls[k]->d_ws_o = (float*)(base + o_wo[k]);
+    lls[k]->d_ws_lse = (float*)(base + o_wl[k]);
+  }
+  if ((rc = pie_launch_append(ctx, &plan, k_new, v_new, s))) return rc;
+  if (!plan.simple_rows.empty() && (rc = pie_launch_simple(ctx, &plan, q, out, lse, s))) return rc;
+  if (!plan.split.items.empty() && (rc = pie_launch_split(ctx, &plan, q, out, lse, s))) return rc;
+  if (!plan.tile.items.empty() && (rc = pie_launch_tiles(ctx, &plan, q, out, lse, s))) return rc;
+  if (!plan.split.merges.empty() && (rc = pie_launch_merge(ctx, &plan, plan.split, out, lse, s))) return rc;
+  if (!plan.tile.merges.empty() && (rc = pie_launch_merge(ctx, &plan, plan.tile, out, lse, s))) return rc;
   return PIE_OK;
 }
