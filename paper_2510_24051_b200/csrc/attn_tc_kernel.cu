@@ -1,0 +1,552 @@
+// Prefill / token-tree attention on the 5th-generation tensor cores (Section 4.2 "Forward API":
+// chunked prefill, speculative-tree verification under explicit masks).
+//
+// One CTA per SM walks its share of work items.  An item is up to 256 rows (row = query token *
+// G + head-in-group, one kv head) = two 128-row Q tiles, attended over the item's kept pages in
+// KV tiles of 128 tokens.  Roles (384 threads):
+//   warps 0-3 / 4-7  softmax warpgroup of Q tile 0 / 1: one row per thread.  Reads S from TMEM,
+//                    masks, exponentiates, writes bf16 P back over S in TMEM, keeps the running
+//                    (max, sum), rescales O in TMEM only when the row max grew by more than 2^8,
+//                    and runs the epilogue.
+//   warp 8           producer: linear bulk copies of page blocks into the K / V stage rings.  The
+//                    pool's storage order is the 128-byte-swizzled canonical operand layout, so a
+//                    page block drops into its 16-row band of the tile with no tensor map.
+//   warp 9           MMA issuer (one lane): S_t = Q_t K^T, O_t += P_t V with tcgen05.mma,
+//                    accumulators and P in TMEM; completion is tracked with tcgen05.commit.
+// TMEM (512 columns): S0 | S1 | O0 | O1; P_t overlays the first 64 columns of S_t.
+#include <cuda_bf16.h>
+
+#include "pie_internal.h"
+
+namespace {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Gives up after ~1 s, or at once when any wait of this launch already gave up
+// (the status word is set), so a broken pipeline drains in bounded time instead of hanging.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status) {
+  const uint64_t t0 = global_ns();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*reinterpret_cast<volatile int*>(status) != 0) return false;
+    if (global_ns() - t0 > 1000000000ull) {
+      atomicExch(status, (int)PIE_ERR_DEVICE_TIMEOUT);
+      return false;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, status);
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M x N, A K-major, B K- or MN-major.
+__device__ __forceinline__ uint32_t instr_desc(int M, int N, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d_tmem),
+               "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+               : "memory");
+}
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d_tmem),
+               "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
+               : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%"
+      "31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%"
+      "32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+               "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+               "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+constexpr float kNegInf = -__builtin_huge_valf();
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kTileM = 128;   // rows per Q tile
+constexpr int kTileN = 128;   // tokens per KV tile
+
+template <int D, int P>
+struct TcCfg {
+  static constexpr int NSLAB = D / 64;                 // 128-byte slabs per row
+  static constexpr int PPT = kTileN / P;               // pages per KV tile
+  static constexpr int SLAB_TILE = kTileN * 128;       // bytes of one slab of a 128-row tile (16 KB)
+  static constexpr int SLAB_PAGE = P * 128;            // bytes of one slab of a page block
+  static constexpr int BLK = P * D * 2;                // K (or V) block of one page and head
+  static constexpr int QTILE = kTileM * D * 2;
+  static constexpr int KVTILE = kTileN * D * 2;
+  static constexpr int STAGES = D == 128 ? 2 : 4;
+  static constexpr int NBAR = 4 * STAGES + 10;
+  static constexpr int SMEM = 2 * QTILE + 2 * STAGES * KVTILE + NBAR * 8 + 64;
+};
+
+template <int D, int P>
+__global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
+  using C = TcCfg<D, P>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + 2 * C::QTILE;
+  uint8_t* sV = sK + C::STAGES * C::KVTILE;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + C::STAGES * C::KVTILE);
+  uint64_t* k_full = bars;
+  uint64_t* k_empty = k_full + C::STAGES;
+  uint64_t* v_full = k_empty + C::STAGES;
+  uint64_t* v_empty = v_full + C::STAGES;
+  uint64_t* q_full = v_empty + C::STAGES;  // [2]
+  uint64_t* s_full = q_full + 2;           // [2]
+  uint64_t* p_full = s_full + 2;           // [2]
+  uint64_t* o_done = p_full + 2;           // [2]
+  uint64_t* o_free = o_done + 2;           // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_free + 2);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) {
+      mbar_init(smem_u32(k_full + s), 1);
+      mbar_init(smem_u32(k_empty + s), 1);
+      mbar_init(smem_u32(v_full + s), 1);
+      mbar_init(smem_u32(v_empty + s), 1);
+    }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(smem_u32(q_full + t), kTileM);
+      mbar_init(smem_u32(s_full + t), 1);
+      mbar_init(smem_u32(p_full + t), kTileM);
+      mbar_init(smem_u32(o_done + t), 1);
+      mbar_init(smem_u32(o_free + t), kTileM);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  const int it0 = p.cta_ptr[blockIdx.x], it1 = p.cta_ptr[blockIdx.x + 1];
+
+  if (warp >= 8) {
+    if (warp == 8) {
+      // ================================================================ producer
+      uint32_t tile_cnt = 0;
+      for (int it = it0; it < it1; ++it) {
+        const PieItem item = p.items[it];
+        const uint8_t* base = p.pool + (int64_t)item.kv_head * (2 * C::BLK);
+        const int npages = item.page_end - item.page_begin;
+        const int ntiles = (npages + C::PPT - 1) / C::PPT;
+        for (int j = 0; j < ntiles; ++j, ++tile_cnt) {
+          const uint32_t s = tile_cnt % C::STAGES, ph = (tile_cnt / C::STAGES) & 1;
+          const int nvalid = min(C::PPT, npages - j * C::PPT);
+          const int ncopies = nvalid * C::NSLAB;
+          int phys = 0;
+          if (lane < nvalid) phys = __ldg(&p.kept[item.page_begin + j * C::PPT + lane].x);
+          // ---- K
+          mbar_wait(smem_u32(k_empty + s), ph ^ 1, p.status);
+          if (lane == 0) mbar_expect_tx(smem_u32(k_full + s), nvalid * C::BLK);
+          __syncwarp();
+          const int pg = lane / C::NSLAB, sl = lane % C::NSLAB;     // copy `lane`: page pg of the tile, slab sl
+          const int ph_pg = __shfl_sync(0xFFFFFFFFu, phys, pg);      // (at most PPT * NSLAB <= 32 copies per tile)
+          if (lane < ncopies)
+            bulk_g2s(smem_u32(sK + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
+                     base + (int64_t)ph_pg * p.page_bytes + sl * C::SLAB_PAGE, C::SLAB_PAGE, smem_u32(k_full + s));
+          __syncwarp();
+          // ---- V
+          mbar_wait(smem_u32(v_empty + s), ph ^ 1, p.status);
+          if (lane == 0) mbar_expect_tx(smem_u32(v_full + s), nvalid * C::BLK);
+          __syncwarp();
+          if (lane < ncopies)
+            bulk_g2s(smem_u32(sV + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
+                     base + (int64_t)ph_pg * p.page_bytes + C::BLK + sl * C::SLAB_PAGE, C::SLAB_PAGE,
+                     smem_u32(v_full + s));
+          __syncwarp();
+        }
+      }
+    } else if (warp == 9) {
+      // ================================================================ MMA issuer
+      uint32_t tile_cnt = 0;
+      uint32_t n_items[2] = {0, 0};   // items in which Q tile t took part (phase of q_full / o_done / o_free)
+      uint32_t n_tiles[2] = {0, 0};   // KV tiles Q tile t went through (phase of s_full / p_full)
+      const uint32_t idesc_pv = instr_desc(kTileM, D, 1);
+      for (int it = it0; it < it1; ++it) {
+        const PieItem item = p.items[it];
+        const PieReq rq = p.reqs[item.req];
+        const int npages = item.page_end - item.page_begin;
+        const int ntiles = (npages + C::PPT - 1) / C::PPT;
+        const int nt = item.nrows > kTileM ? 2 : 1;
+        if (ntiles == 0) continue;  // the softmax warpgroups write zeros / -inf on their own
+        for (int t = 0; t < nt; ++t) {
+          mbar_wait(smem_u32(q_full + t), n_items[t] & 1, p.status);
+          mbar_wait(smem_u32(o_free + t), (n_items[t] & 1) ^ 1, p.status);  // previous epilogue has drained O_t
+          ++n_items[t];
+        }
+        tc_fence_after();
+
+        auto issue_s = [&](int t, int j, uint32_t cnt) {
+          const uint32_t s = cnt % C::STAGES;
+          const int nvalid = min(C::PPT, npages - j * C::PPT);
+          const uint32_t idesc = instr_desc(kTileM, nvalid * P, 0);
+          const uint32_t qa = smem_u32(sQ + t * C::QTILE), kb = smem_u32(sK + s * C::KVTILE);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t off = (ks >> 2) * C::SLAB_TILE + (ks & 3) * 32;
+            umma_ss(tmem + t * 128, smem_desc(qa + off, 16, 1024), smem_desc(kb + off, 16, 1024), idesc, ks > 0);
+          }
+          umma_commit(smem_u32(s_full + t));
+        };
+
+        // prologue: S_t(0)
+        {
+          const uint32_t s = tile_cnt % C::STAGES, ph = (tile_cnt / C::STAGES) & 1;
+          mbar_wait(smem_u32(k_full + s), ph, p.status);
+          tc_fence_after();
+          if (lane == 0) {
+            for (int t = 0; t < nt; ++t) issue_s(t, 0, tile_cnt);
+            umma_commit(smem_u32(k_empty + s));
+          }
+          __syncwarp();
+        }
+        for (int j = 0; j < ntiles; ++j) {
+          const uint32_t cnt = tile_cnt + j;
+          const uint32_t s = cnt % C::STAGES, ph = (cnt / C::STAGES) & 1;
+          const int nvalid = min(C::PPT, npages - j * C::PPT);
+          mbar_wait(smem_u32(v_full + s), ph, p.status);
+          // clear V rows past the end of the context in the request's last page (may hold NaN patterns)
+          if (rq.last_page_len < P) {
+            const int pg = lane < nvalid ? (int)((uint32_t)__ldg(&p.kept[item.page_begin + j * C::PPT + lane].y) & ~PIE_KEPT_NEEDS_MASK) : -1;
+            const unsigned hit = __ballot_sync(0xFFFFFFFFu, pg == rq.last_logical);
+            if (hit) {
+              const int pgi = __ffs(hit) - 1;
+              constexpr int CH = D * 2 / 16;
+              const int nz = (P - rq.last_page_len) * CH;
+              for (int c = lane; c < nz; c += 32) {
+                const int tkn = pgi * P + rq.last_page_len + c / CH, ch = c % CH;
+                *reinterpret_cast<uint4*>(sV + s * C::KVTILE + (ch >> 3) * C::SLAB_TILE + tkn * 128 +
+                                          (((ch & 7) ^ (tkn & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+              }
+              fence_async_smem();
+              __syncwarp();
+            }
+          }
+          tc_fence_after();
+          for (int t = 0; t < nt; ++t) {
+            mbar_wait(smem_u32(p_full + t), n_tiles[t] & 1, p.status);
+            ++n_tiles[t];
+            tc_fence_after();
+            if (lane == 0) {
+              const uint32_t vb = smem_u32(sV + s * C::KVTILE);
+              const int ksteps = nvalid * P / 16;
+              for (int ks = 0; ks < ksteps; ++ks)
+                umma_ts(tmem + 256 + t * D, tmem + t * 128 + ks * 8, smem_desc(vb + ks * 2048, C::SLAB_TILE, 1024),
+                        idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+              if (t == nt - 1) umma_commit(smem_u32(v_empty + s));
+              if (j + 1 == ntiles) umma_commit(smem_u32(o_done + t));
+            }
+            __syncwarp();
+            if (j + 1 < ntiles) {
+              const uint32_t cn = cnt + 1;
+              const uint32_t sn = cn % C::STAGES, phn = (cn / C::STAGES) & 1;
+              if (t == 0) {
+                mbar_wait(smem_u32(k_full + sn), phn, p.status);
+                tc_fence_after();
+              }
+              if (lane == 0) {
+                issue_s(t, j + 1, cn);
+                if (t == nt - 1) umma_commit(smem_u32(k_empty + sn));
+              }
+              __syncwarp();
+            }
+          }
+        }
+        tile_cnt += ntiles;
+      }
+    }
+  } else {
+    // ================================================================ softmax warpgroups
+    const int t = warp >> 2;                       // Q tile of this warpgroup
+    const int rho = (warp & 3) * 32 + lane;        // row inside the tile = TMEM lane
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + t * 128 + lane_sel, tO = tmem + 256 + t * D + lane_sel;
+    uint32_t my_items = 0, my_tiles = 0;   // phases of the per-item / per-tile barriers of this Q tile
+    for (int it = it0; it < it1; ++it) {
+      const PieItem item = p.items[it];
+      const PieReq rq = p.reqs[item.req];
+      const int npages = item.page_end - item.page_begin;
+      const int ntiles = (npages + C::PPT - 1) / C::PPT;
+      const int nt = item.nrows > kTileM ? 2 : 1;
+      if (t >= nt) continue;
+      const int gr = item.row0 + t * kTileM + rho;
+      const bool valid = gr < item.row0 + item.nrows;
+      const int tok = valid ? gr / p.G : 0;
+      const int head = item.kv_head * p.G + (valid ? gr % p.G : 0);
+      const int64_t oi = (int64_t)(rq.q_start + tok) * p.n_q_heads + head;
+      const int lim = valid ? rq.kv_len - rq.q_len + tok : -1;
+      const uint32_t* mrow = p.mask + rq.mask_word_off + (int64_t)tok * rq.mask_row_words;
+      const bool explicit_mask = rq.mask_row_words != 0;
+      float m_ref = kNegInf, l_sum = 0.f;
+
+      if (ntiles > 0) {
+        // ---- Q row -> shared memory (K-major, 128-byte swizzle)
+        const uint4* qsrc = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.q) + oi * D);
+        uint8_t* qdst = sQ + t * C::QTILE;
+#pragma unroll
+        for (int ch = 0; ch < D * 2 / 16; ++ch) {
+          const uint4 v = valid ? __ldg(qsrc + ch) : make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(qdst + (ch >> 3) * C::SLAB_TILE + rho * 128 + (((ch & 7) ^ (rho & 7)) << 4)) = v;
+        }
+        fence_async_smem();
+        mbar_arrive(smem_u32(q_full + t));
+
+        for (int j = 0; j < ntiles; ++j) {
+          const int nvalid = min(C::PPT, npages - j * C::PPT);
+          const int my_tile_in_item = j;
+          // page records of this KV tile (logical page | needs-mask flag); same addresses for all threads
+          uint32_t bits[C::PPT];   // allowed positions of this row inside each page of the tile
+          bool tile_mask = nvalid < C::PPT;
+#pragma unroll
+          for (int g = 0; g < C::PPT; ++g) {
+            const uint32_t lpf = g < nvalid ? (uint32_t)__ldg(&p.kept[item.page_begin + j * C::PPT + g].y) : 0u;
+            bits[g] = 0xFFFFFFFFu;
+            if (g >= nvalid || !valid) {
+              bits[g] = 0u;
+              tile_mask = true;
+            } else if (lpf & PIE_KEPT_NEEDS_MASK) {
+              const int j0 = (int)(lpf & ~PIE_KEPT_NEEDS_MASK) * P;
+              if (explicit_mask) bits[g] = __ldg(mrow + (j0 >> 5)) >> (j0 & 31);
+              else bits[g] = lim >= j0 + P - 1 ? 0xFFFFFFFFu : (lim < j0 ? 0u : ((1u << (lim - j0 + 1)) - 1u));
+              tile_mask = true;
+            }
+          }
+          mbar_wait(smem_u32(s_full + t), my_tiles & 1, p.status);
+          ++my_tiles;
+          tc_fence_after();
+          // ---- pass 1: row maximum of the (masked) raw scores, 64 columns at a time
+          float mraw = kNegInf;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float a[64];
+            tmem_ld32(tS + h * 64, reinterpret_cast<uint32_t*>(a));
+            tmem_ld32(tS + h * 64 + 32, reinterpret_cast<uint32_t*>(a) + 32);
+            tmem_wait_ld();
+            if (tile_mask) {
+#pragma unroll
+              for (int c = 0; c < 64; ++c)
+                if (!((bits[(h * 64 + c) / P] >> ((h * 64 + c) % P)) & 1u)) a[c] = kNegInf;
+            }
+#pragma unroll
+            for (int c = 0; c < 64; ++c) mraw = fmaxf(mraw, a[c]);
+          }
+          const float m_tile = mraw * p.scale_log2;   // -inf stays -inf
+          const float m_new = fmaxf(m_ref, m_tile);
+          if (my_tile_in_item == 0) {
+            m_ref = m_new;
+          } else {
+            const bool grow = m_new > m_ref + 8.f;     // also true when m_ref is -inf and m_new is finite
+            if (__any_sync(0xFFFFFFFFu, grow)) {
+              // rare: bring O_t (complete up to the previous tile: S_t of this tile was issued after
+              // it) to the new reference maximum
+              const float f = (m_ref == kNegInf) ? 1.f : fast_exp2(m_ref - m_new);
+              if (m_new != kNegInf) m_ref = m_new;
+              l_sum *= f;
+#pragma unroll
+              for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t o[32];
+                tmem_ld32(tO + c0, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
+                tmem_st32(tO + c0, o);
+              }
+              tmem_wait_st();
+            }
+          }
+          // ---- pass 2: P = exp2(S * scale - m_ref) as bf16 over the first 64 columns of S_t
+          const float neg_m = (m_ref == kNegInf) ? 0.f : -m_ref;
+          float psum = 0.f;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float a[64];
+            tmem_ld32(tS + h * 64, reinterpret_cast<uint32_t*>(a));
+            tmem_ld32(tS + h * 64 + 32, reinterpret_cast<uint32_t*>(a) + 32);
+            tmem_wait_ld();
+            if (tile_mask) {
+#pragma unroll
+              for (int c = 0; c < 64; ++c)
+                if (!((bits[(h * 64 + c) / P] >> ((h * 64 + c) % P)) & 1u)) a[c] = kNegInf;
+            }
+            uint32_t pk[32];
+#pragma unroll
+            for (int c = 0; c < 64; c += 2) {
+              const float p0 = fast_exp2(fmaf(a[c], p.scale_log2, neg_m));
+              const float p1 = fast_exp2(fmaf(a[c + 1], p.scale_log2, neg_m));
+              psum += p0 + p1;
+              pk[c >> 1] = pack_bf16(p0, p1);
+            }
+            tmem_st32(tS + h * 32, pk);
+          }
+          l_sum += psum;
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(smem_u32(p_full + t));
+        }
+        mbar_wait(smem_u32(o_done + t), my_items & 1, p.status);
+        ++my_items;
+        tc_fence_after();
+      }
+
+      // ---- epilogue: normalise, store
+      const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+      const float lse = l_sum > 0.f ? (m_ref + log2f(l_sum)) * kLn2 : kNegInf;
+#pragma unroll
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t o[32];
+        if (ntiles > 0) {
+          tmem_ld32(tO + c0, o);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = 0u;
+        }
+        if (valid) {
+          if (item.partial_slot < 0) {
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D + c0);
+#pragma unroll
+            for (int c = 0; c < 32; c += 8)
+              dst[c >> 3] = make_uint4(pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv),
+                                       pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv),
+                                       pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv),
+                                       pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv));
+          } else {
+            float4* dst = reinterpret_cast<float4*>(p.ws_o + ((int64_t)item.partial_slot * 256 + (gr - item.row0)) * D + c0);
+#pragma unroll
+            for (int c = 0; c < 32; c += 4)
+              dst[c >> 2] = make_float4(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv,
+                                        __uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+          }
+        }
+      }
+      if (valid) {
+        if (item.partial_slot < 0) p.lse[oi] = lse;
+        else p.ws_lse[(int64_t)item.partial_slot * 256 + (gr - item.row0)] = lse;
+      }
+      if (ntiles > 0) {
+        tc_fence_before();
+        mbar_arrive(smem_u32(o_free + t));
+      }
+    }
+  }
+
+  // ---- teardown: everyone is done with TMEM before it is released
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+}
+
+}  // namespace
+
+bool pie_tc_supported(const pie_ctx* ctx) {
+  const pie_config& c = ctx->cfg;
+  return c.dtype == PIE_DTYPE_BF16 && (c.page_size == 16 || c.page_size == 32) && (c.head_dim == 64 || c.head_dim == 128);
+}
+
+template <int D, int P>
+static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
+  using C = TcCfg<D, P>;
+  auto kern = attn_tc_kernel<D, P>;
+  static bool configured[8] = {};
+  int dev = ctx->cfg.device & 7;
+  if (!configured[dev]) {
+    PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+    configured[dev] = true;
+  }
+  kern<<<grid, 384, C::SMEM, s>>>(p);
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}
+
+int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
+  const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size;
+  if (D == 128 && P == 16) return launch_tc<128, 16>(ctx, p, grid, s);
+  if (D == 64 && P == 16) return launch_tc<64, 16>(ctx, p, grid, s);
+  if (D == 128 && P == 32) return launch_tc<128, 32>(ctx, p, grid, s);
+  if (D == 64 && P == 32) return launch_tc<64, 32>(ctx, p, grid, s);
+  return PIE_ERR_UNSUPPORTED;
+}

@@ -96,6 +96,7 @@ struct pie_plan {
   std::vector<int32_t> tok_req;     // [T]
   std::vector<int32_t> simple_rows; // (token*H_q + head) rows for the plain kernel
   PieLaunchList split, tile;
+  bool tile_tc = false;             // row tiles run on the tcgen05 kernel (256-row items)
   pie_plan_info info{};
   // device
   void* d_blob = nullptr;           // one allocation holding every array below
@@ -164,6 +165,8 @@ int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* ou
 int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s);
 bool pie_split_supported(const pie_ctx* ctx);
 int pie_split_warps_per_block(const pie_ctx* ctx);
+bool pie_tc_supported(const pie_ctx* ctx);
+int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s);
 
 int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);  // host part (planner.cc)
 

@@ -245,7 +245,8 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   const bool tiles_ok = pie_split_supported(ctx) && !(b->flags & PIE_PLAN_FORCE_SIMPLE);
   std::vector<Unit> split_units, tile_units;
   plan->simple_rows.clear();
-  const int TILE_ROWS = 64;
+  plan->tile_tc = pie_tc_supported(ctx) && !(b->flags & PIE_PLAN_NO_TENSOR_TILES);
+  const int TILE_ROWS = plan->tile_tc ? 256 : 64;   // two 128-row tcgen05 tiles, or four 16-row warps
   for (int r = 0; r < R; ++r) {
     const PieReq& q = plan->reqs[r];
     const int rows = q.q_len * G;
@@ -286,7 +287,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       ll.stream_ptr.push_back((int32_t)(ll.stream.size() / 2));
     }
   }
-  partition(tile_units, ctx->n_sms, 8, TILE_ROWS, plan->tile);
+  partition(tile_units, ctx->n_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, plan->tile);
 
   pie_plan_info& info = plan->info;
   info = pie_plan_info{};

@@ -24,7 +24,7 @@ def test_generator_is_bit_identical_on_cpu_and_gpu():
 
 
 @pytest.mark.parametrize("name", SMALL)
-@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("flags", [0, 1, 2])
 def test_small_configs_match_oracle(name, flags):
     from tests._gpu import check_close, run_workload
     wl = configs.small(name)
