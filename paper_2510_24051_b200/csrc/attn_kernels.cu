@@ -447,10 +447,14 @@ template <typename T>
 __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* __restrict__ reqs,
                              const float* __restrict__ ws_o, const float* __restrict__ ws_lse, T* __restrict__ out,
                              float* __restrict__ lse_out, int slot_rows, int D, int n_q_heads, int G) {
+  // block (x, y): merge group x, rows [16 y, 16 y + 16) of it
   const PieMerge mg = merges[blockIdx.x];
+  const int r0 = blockIdx.y * 16;
+  if (r0 >= mg.nrows) return;
   const PieReq rq = reqs[mg.req];
-  for (int e = threadIdx.x; e < mg.nrows * D; e += blockDim.x) {
-    const int row = e / D, d = e - row * D;
+  const int nr = min(16, mg.nrows - r0);
+  for (int e = threadIdx.x; e < nr * D; e += blockDim.x) {
+    const int row = r0 + e / D, d = e % D;
     float M = kNegInf;
     for (int c = 0; c < mg.nslots; ++c) M = fmaxf(M, ws_lse[(int64_t)(mg.slot0 + c) * slot_rows + row]);
     float Z = 0.f, acc = 0.f;
@@ -626,7 +630,7 @@ int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* ou
 
 int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s) {
   const int D = ctx->cfg.head_dim;
-  const int n = (int)ll.merges.size();
+  const dim3 n((unsigned)ll.merges.size(), (unsigned)((ll.slot_rows + 15) / 16));
   if (ctx->cfg.dtype == PIE_DTYPE_BF16)
     merge_kernel<__nv_bfloat16><<<n, 256, 0, s>>>(ll.d_merges, plan->d_reqs, ll.d_ws_o, ll.d_ws_lse, (__nv_bfloat16*)out, lse,
                                                    ll.slot_rows, D, ctx->cfg.num_q_heads, ctx->G);

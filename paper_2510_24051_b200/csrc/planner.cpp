@@ -35,10 +35,25 @@ struct Unit {
   int32_t req, kv_head, row0, nrows, page_begin, page_end;
 };
 
-// Give each of `grid` CTAs a contiguous, equal share of the page visits of `units` (taken in
-// order); a unit cut by a share boundary becomes several items whose fp32 partials are merged.
+// Finish a launch list from per-CTA item vectors.
+void flatten(std::vector<std::vector<PieItem>>& per_cta, PieLaunchList& ll) {
+  ll.cta_ptr.push_back(0);
+  for (auto& v : per_cta) {
+    for (const PieItem& it : v) ll.items.push_back(it);
+    ll.cta_ptr.push_back((int32_t)ll.items.size());
+  }
+}
+
+// Give each of `grid` CTAs (or warps) a share of the page visits of `units`.
+//  * Many units, none of them large against a share: whole units are dealt out in order, each to
+//    the least-loaded CTA (equal units => round robin).  Units that are neighbours in the batch
+//    (heads of one request, branches that share a prefix) then run at the same time on different
+//    SMs, so shared pages are fetched from HBM once and served from L2 afterwards; nothing is
+//    split, so nothing needs merging.
+//  * Otherwise: contiguous equal shares; a unit cut by a share boundary becomes several items
+//    whose fp32 partials are merged.
 void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_cta, int slot_rows,
-               PieLaunchList& ll) {
+               bool allow_whole_units, PieLaunchList& ll) {
   ll.items.clear();
   ll.merges.clear();
   ll.cta_ptr.clear();
@@ -46,11 +61,32 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
   ll.slot_rows = slot_rows;
   ll.grid = 0;
   if (units.empty()) return;
-  int64_t W = 0;
-  for (const Unit& u : units) W += u.page_end - u.page_begin;
+  int64_t W = 0, max_unit = 0;
+  for (const Unit& u : units) {
+    W += u.page_end - u.page_begin;
+    max_unit = std::max<int64_t>(max_unit, u.page_end - u.page_begin);
+  }
   int grid = (int)std::min<int64_t>(grid_max, std::max<int64_t>(1, W / std::max(1, min_pages_per_cta)));
   ll.grid = grid;
   std::vector<std::vector<PieItem>> per_cta(grid);
+
+  if (allow_whole_units && (int64_t)units.size() >= 4 * (int64_t)grid && max_unit * 8 <= W / grid) {
+    // least-loaded-first list scheduling; a binary heap keyed on (load, cta)
+    std::vector<std::pair<int64_t, int>> heap(grid);
+    for (int c = 0; c < grid; ++c) heap[c] = {0, c};
+    auto cmp = [](const std::pair<int64_t, int>& a, const std::pair<int64_t, int>& b) { return a > b; };
+    std::make_heap(heap.begin(), heap.end(), cmp);
+    for (const Unit& u : units) {
+      std::pop_heap(heap.begin(), heap.end(), cmp);
+      auto& top = heap.back();
+      per_cta[top.second].push_back(PieItem{u.req, u.kv_head, u.row0, u.nrows, u.page_begin, u.page_end, -1, 0});
+      top.first += std::max<int64_t>(1, u.page_end - u.page_begin);
+      std::push_heap(heap.begin(), heap.end(), cmp);
+    }
+    flatten(per_cta, ll);
+    return;
+  }
+
   int64_t off = 0;
   auto cta_of = [&](int64_t x) {  // share that holds page-visit x
     if (W == 0) return 0;
@@ -90,11 +126,7 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
     }
     off += n;
   }
-  ll.cta_ptr.push_back(0);
-  for (int c = 0; c < grid; ++c) {
-    for (const PieItem& it : per_cta[c]) ll.items.push_back(it);
-    ll.cta_ptr.push_back((int32_t)ll.items.size());
-  }
+  flatten(per_cta, ll);
 }
 
 }  // namespace
@@ -271,7 +303,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     }
   }
   // split-KV decode: one share per warp of a full grid (every warp is its own pipeline)
-  partition(split_units, ctx->n_sms * pie_split_warps_per_block(ctx), 4, 16, plan->split);
+  partition(split_units, ctx->n_sms * pie_split_warps_per_block(ctx), 4, 16, false, plan->split);
   {
     PieLaunchList& ll = plan->split;
     ll.stream.clear();
@@ -287,7 +319,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       ll.stream_ptr.push_back((int32_t)(ll.stream.size() / 2));
     }
   }
-  partition(tile_units, ctx->n_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, plan->tile);
+  partition(tile_units, ctx->n_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile);
 
   pie_plan_info& info = plan->info;
   info = pie_plan_info{};
