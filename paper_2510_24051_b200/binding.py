@@ -154,7 +154,7 @@ def pie_num_free_kvpages(ctx):
 
 
 def _on_device(t):
-    return 0 if isinstance(t, np.ndarray) or not t.is_cuda else 1
+    return 0 if t is None or isinstance(t, np.ndarray) or not t.is_cuda else 1
 
 
 def pie_kvpage_write(ctx, ids, K, V, stream=None):
