@@ -111,6 +111,78 @@ bool page_ok(const pie_ctx* ctx, int32_t id) {
   return id >= 0 && id < ctx->cfg.num_pages && ctx->allocated[id];
 }
 
+// Device image of a plan: every array the kernels read, 256-byte aligned, followed by the fp32
+// partial workspaces of the two tile launches.
+struct PlanLayout {
+  size_t reqs, kept, mask, app, tok, simple, items[2], cta[2], merges[2], ws_o[2], ws_lse[2];
+  size_t upload, total;
+};
+
+PlanLayout plan_layout(const pie_ctx* ctx, const pie_plan* plan) {
+  PlanLayout L{};
+  size_t off = 0;
+  auto place = [&](size_t bytes) {
+    size_t o = off;
+    off = (off + bytes + 255) & ~(size_t)255;
+    return o;
+  };
+  L.reqs = place(plan->reqs.size() * sizeof(PieReq));
+  L.kept = place(plan->kept.size() * 4);
+  L.mask = place(plan->mask_words.size() * 4);
+  L.app = place(plan->append_dst.size() * 4);
+  L.tok = place(plan->tok_req.size() * 4);
+  L.simple = place(plan->simple_rows.size() * 4);
+  const PieLaunchList* lls[2] = {&plan->split, &plan->tile};
+  for (int k = 0; k < 2; ++k) {
+    L.items[k] = place(lls[k]->items.size() * sizeof(PieItem));
+    L.cta[k] = place(lls[k]->cta_ptr.size() * 4);
+    L.merges[k] = place(lls[k]->merges.size() * sizeof(PieMerge));
+  }
+  L.upload = off;
+  const size_t D = ctx->cfg.head_dim;
+  for (int k = 0; k < 2; ++k) {
+    L.ws_o[k] = place((size_t)lls[k]->n_slots * lls[k]->slot_rows * D * 4);
+    L.ws_lse[k] = place((size_t)lls[k]->n_slots * lls[k]->slot_rows * 4);
+  }
+  L.total = off;
+  return L;
+}
+
+void plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
+  auto cp = [&](size_t off, const void* p, size_t bytes) {
+    if (bytes) std::memcpy(dst + off, p, bytes);
+  };
+  cp(L.reqs, plan->reqs.data(), plan->reqs.size() * sizeof(PieReq));
+  cp(L.kept, plan->kept.data(), plan->kept.size() * 4);
+  cp(L.mask, plan->mask_words.data(), plan->mask_words.size() * 4);
+  cp(L.app, plan->append_dst.data(), plan->append_dst.size() * 4);
+  cp(L.tok, plan->tok_req.data(), plan->tok_req.size() * 4);
+  cp(L.simple, plan->simple_rows.data(), plan->simple_rows.size() * 4);
+  const PieLaunchList* lls[2] = {&plan->split, &plan->tile};
+  for (int k = 0; k < 2; ++k) {
+    cp(L.items[k], lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
+    cp(L.cta[k], lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
+    cp(L.merges[k], lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
+  }
+}
+
+void plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base) {
+  plan->d_reqs = (PieReq*)(base + L.reqs);
+  plan->d_kept = (int2*)(base + L.kept);
+  plan->d_mask = (uint32_t*)(base + L.mask);
+  plan->d_append_dst = (int32_t*)(base + L.app);
+  plan->d_tok_req = (int32_t*)(base + L.tok);
+  plan->d_simple_rows = (int32_t*)(base + L.simple);
+  PieLaunchList* lls[2] = {&plan->split, &plan->tile};
+  for (int k = 0; k < 2; ++k) {
+    lls[k]->d_items = (PieItem*)(base + L.items[k]);
+    lls[k]->d_cta_ptr = (int32_t*)(base + L.cta[k]);
+    lls[k]->d_merges = (PieMerge*)(base + L.merges[k]);
+    lls[k]->d_ws_o = (float*)(base + L.ws_o[k]);
+    lls[k]->d_ws_lse = (float*)(base + L.ws_lse[k]);
+  }
+}
+
 }  // namespace
 
 int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, const void* v_new, cudaStream_t s) {
@@ -226,12 +298,14 @@ int pie_destroy(pie_ctx* ctx) {
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_stage) cudaFree(ctx->d_stage);
     if (ctx->d_io) cudaFree(ctx->d_io);
+    if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
     for (auto& t : ctx->timed) {
       cudaEventDestroy(t.start);
       cudaEventDestroy(t.stop);
     }
     for (auto e : ctx->free_events) cudaEventDestroy(e);
   }
+  delete ctx->host_plan;
   delete ctx;
   return PIE_OK;
 }
@@ -371,44 +445,13 @@ int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pi
   }
   if (!ctx->host_only && plan->R > 0) {
     cudaStream_t s = (cudaStream_t)stream;
-    // one allocation, one upload: [reqs | kept | mask | append_dst | tok_req | simple_rows |
-    // split items, cta_ptr, merges | tile items, cta_ptr, merges] then the partial workspaces.
-    std::vector<uint8_t> host;
-    auto put = [&](const void* p, size_t bytes) {
-      size_t off = (host.size() + 255) & ~(size_t)255;
-      host.resize(off + bytes);
-      if (bytes) std::memcpy(host.data() + off, p, bytes);
-      return off;
-    };
-    size_t o_reqs = put(plan->reqs.data(), plan->reqs.size() * sizeof(PieReq));
-    size_t o_kept = put(plan->kept.data(), plan->kept.size() * 4);
-    size_t o_mask = put(plan->mask_words.data(), plan->mask_words.size() * 4);
-    size_t o_app = put(plan->append_dst.data(), plan->append_dst.size() * 4);
-    size_t o_tok = put(plan->tok_req.data(), plan->tok_req.size() * 4);
-    size_t o_simple = put(plan->simple_rows.data(), plan->simple_rows.size() * 4);
-    size_t o_li[2], o_lc[2], o_lm[2], o_ls[2], o_lp[2];
-    PieLaunchList* lls[2] = {&plan->split, &plan->tile};
-    for (int k = 0; k < 2; ++k) {
-      o_li[k] = put(lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
-      o_lc[k] = put(lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
-      o_lm[k] = put(lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
-      o_ls[k] = put(lls[k]->stream.data(), lls[k]->stream.size() * 4);
-      o_lp[k] = put(lls[k]->stream_ptr.data(), lls[k]->stream_ptr.size() * 4);
-    }
-    size_t upload = (host.size() + 255) & ~(size_t)255;
-    size_t total = upload;
-    size_t o_wo[2], o_wl[2];
-    const int D = ctx->cfg.head_dim;
-    for (int k = 0; k < 2; ++k) {
-      o_wo[k] = total;
-      total += (((size_t)lls[k]->n_slots * lls[k]->slot_rows * D * 4) + 255) & ~(size_t)255;
-      o_wl[k] = total;
-      total += (((size_t)lls[k]->n_slots * lls[k]->slot_rows * 4) + 255) & ~(size_t)255;
-    }
+    const PlanLayout L = plan_layout(ctx, plan);
+    std::vector<uint8_t> host(L.upload);
+    plan_fill(plan, L, host.data());
     cudaError_t e = cudaSetDevice(ctx->cfg.device);
-    if (e == cudaSuccess) e = cudaMalloc(&plan->d_blob, std::max<size_t>(total, 256));
-    if (e == cudaSuccess && !host.empty())
-      e = cudaMemcpyAsync(plan->d_blob, host.data(), host.size(), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMalloc(&plan->d_blob, std::max<size_t>(L.total, 256));
+    if (e == cudaSuccess && L.upload)
+      e = cudaMemcpyAsync(plan->d_blob, host.data(), L.upload, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
       ctx->cuda_error = std::string("plan upload: ") + cudaGetErrorString(e);
@@ -416,22 +459,7 @@ int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pi
       delete plan;
       return PIE_ERR_CUDA;
     }
-    uint8_t* base = (uint8_t*)plan->d_blob;
-    plan->d_reqs = (PieReq*)(base + o_reqs);
-    plan->d_kept = (int2*)(base + o_kept);
-    plan->d_mask = (uint32_t*)(base + o_mask);
-    plan->d_append_dst = (int32_t*)(base + o_app);
-    plan->d_tok_req = (int32_t*)(base + o_tok);
-    plan->d_simple_rows = (int32_t*)(base + o_simple);
-    for (int k = 0; k < 2; ++k) {
-      lls[k]->d_items = (PieItem*)(base + o_li[k]);
-      lls[k]->d_cta_ptr = (int32_t*)(base + o_lc[k]);
-      lls[k]->d_merges = (PieMerge*)(base + o_lm[k]);
-      lls[k]->d_stream = (int2*)(base + o_ls[k]);
-      lls[k]->d_stream_ptr = (int32_t*)(base + o_lp[k]);
-      lls[k]->d_ws_o = (float*)(base + o_wo[k]);
-      lls[k]->d_ws_lse = (float*)(base + o_wl[k]);
-    }
+    plan_bind(plan, L, (uint8_t*)plan->d_blob);
   }
   *out = plan;
   return PIE_OK;
@@ -500,40 +528,47 @@ int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, c
                      void* out, float* lse, void* stream) {
   if (!ctx || !batch) return PIE_ERR_INVALID;
   if (ctx->host_only) return PIE_ERR_NO_DEVICE;
-  pie_plan* plan = nullptr;
-  int rc = pie_plan_forward(ctx, batch, stream, &plan);
+  // The context keeps one plan object, one pinned staging buffer and one device arena for this
+  // entry point and reuses them call after call: no allocation in the steady state.
+  if (!ctx->host_plan) ctx->host_plan = new (std::nothrow) pie_plan();
+  pie_plan* plan = ctx->host_plan;
+  if (!plan) return PIE_ERR_INVALID;
+  plan->ctx = ctx;
+  int rc = pie_build_plan(ctx, batch, plan);
   if (rc) return rc;
-  if (plan->T == 0) {
-    pie_plan_destroy(plan);
-    return PIE_OK;
-  }
-  if (!q || !k_new || !v_new || !out || !lse) {
-    pie_plan_destroy(plan);
-    return PIE_ERR_INVALID;
-  }
+  if (plan->T == 0) return PIE_OK;
+  if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
   cudaStream_t s = (cudaStream_t)stream;
+  PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  const PlanLayout L = plan_layout(ctx, plan);
   const size_t T = plan->T, es = ctx->geom.esize, D = ctx->cfg.head_dim;
-  const size_t qb = (T * ctx->cfg.num_q_heads * D * es + 255) & ~(size_t)255;
-  const size_t kb = (T * ctx->cfg.num_kv_heads * D * es + 255) & ~(size_t)255;
-  const size_t lb = (T * ctx->cfg.num_q_heads * 4 + 255) & ~(size_t)255;
-  auto body = [&]() -> int {
-    int rc2 = ensure_buffer(ctx, &ctx->d_io, &ctx->io_bytes, 2 * qb + 2 * kb + lb);
-    if (rc2) return rc2;
-    uint8_t* dq = (uint8_t*)ctx->d_io;
-    uint8_t *dk = dq + qb, *dv = dk + kb, *dout = dv + kb, *dl = dout + qb;
-    PIE_CUDA(ctx, cudaMemcpyAsync(dq, q, T * ctx->cfg.num_q_heads * D * es, cudaMemcpyHostToDevice, s));
-    PIE_CUDA(ctx, cudaMemcpyAsync(dk, k_new, T * ctx->cfg.num_kv_heads * D * es, cudaMemcpyHostToDevice, s));
-    PIE_CUDA(ctx, cudaMemcpyAsync(dv, v_new, T * ctx->cfg.num_kv_heads * D * es, cudaMemcpyHostToDevice, s));
-    rc2 = pie_forward(ctx, plan, dq, dk, dv, dout, (float*)dl, stream);
-    if (rc2) return rc2;
-    PIE_CUDA(ctx, cudaMemcpyAsync(out, dout, T * ctx->cfg.num_q_heads * D * es, cudaMemcpyDeviceToHost, s));
-    PIE_CUDA(ctx, cudaMemcpyAsync(lse, dl, T * ctx->cfg.num_q_heads * 4, cudaMemcpyDeviceToHost, s));
-    PIE_CUDA(ctx, cudaStreamSynchronize(s));
-    return PIE_OK;
-  };
-  rc = body();
-  pie_plan_destroy(plan);
-  return rc;
+  const size_t q_bytes = T * ctx->cfg.num_q_heads * D * es, kv_bytes = T * ctx->cfg.num_kv_heads * D * es;
+  const size_t lse_bytes = T * ctx->cfg.num_q_heads * 4;
+  auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  const size_t o_q = al(L.total), o_k = o_q + al(q_bytes), o_v = o_k + al(kv_bytes), o_out = o_v + al(kv_bytes),
+               o_lse = o_out + al(q_bytes), need = o_lse + al(lse_bytes);
+  if ((rc = ensure_buffer(ctx, &ctx->d_io, &ctx->io_bytes, need))) return rc;
+  if (ctx->h_stage_bytes < L.upload) {
+    if (ctx->h_stage) PIE_CUDA(ctx, cudaFreeHost(ctx->h_stage));
+    ctx->h_stage = nullptr;
+    ctx->h_stage_bytes = 0;
+    const size_t want = std::max(L.upload * 2, (size_t)1 << 20);
+    PIE_CUDA(ctx, cudaMallocHost(&ctx->h_stage, want));
+    ctx->h_stage_bytes = want;
+  }
+  uint8_t* base = (uint8_t*)ctx->d_io;
+  plan_fill(plan, L, (uint8_t*)ctx->h_stage);
+  plan_bind(plan, L, base);
+  PIE_CUDA(ctx, cudaMemcpyAsync(base, ctx->h_stage, L.upload, cudaMemcpyHostToDevice, s));
+  PIE_CUDA(ctx, cudaMemcpyAsync(base + o_q, q, q_bytes, cudaMemcpyHostToDevice, s));
+  PIE_CUDA(ctx, cudaMemcpyAsync(base + o_k, k_new, kv_bytes, cudaMemcpyHostToDevice, s));
+  PIE_CUDA(ctx, cudaMemcpyAsync(base + o_v, v_new, kv_bytes, cudaMemcpyHostToDevice, s));
+  if ((rc = pie_forward(ctx, plan, base + o_q, base + o_k, base + o_v, base + o_out, (float*)(base + o_lse), stream)))
+    return rc;
+  PIE_CUDA(ctx, cudaMemcpyAsync(out, base + o_out, q_bytes, cudaMemcpyDeviceToHost, s));
+  PIE_CUDA(ctx, cudaMemcpyAsync(lse, base + o_lse, lse_bytes, cudaMemcpyDeviceToHost, s));
+  PIE_CUDA(ctx, cudaStreamSynchronize(s));
+  return PIE_OK;
 }
 
 int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out) {

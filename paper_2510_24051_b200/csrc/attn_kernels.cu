@@ -326,36 +326,72 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   __syncwarp();
 
   const int it0 = p.cta_ptr[wg], it1 = p.cta_ptr[wg + 1];
-  const int s0 = p.stream_ptr[wg], n_total = p.stream_ptr[wg + 1] - s0;
-  const int2* stream = p.stream + s0;
 
-  // issue the copy of stream position n into ring stage n % DEPTH (lane 0)
-  auto issue = [&](int n, int2 e) {
+  // Prefetch cursor: the page visit DEPTH positions ahead of the one being consumed.  It walks
+  // the same item list; the next item's record is fetched one item early so that crossing an
+  // item boundary costs no memory latency.
+  int pf_it = it0 - 1, pf_k = 0, pf_end = 0, pf_head = 0;
+  int nx_begin = 0, nx_end = 0, nx_head = 0;
+  if (it0 < it1) {
+    const PieItem f = p.items[it0];
+    nx_begin = f.page_begin;
+    nx_end = f.page_end;
+    nx_head = f.kv_head;
+  }
+  bool pf_live = true;
+  auto pf_settle = [&]() {  // move to the next non-empty item while the current one is used up
+    while (pf_live && pf_k >= pf_end) {
+      if (pf_it + 1 >= it1) {
+        pf_live = false;
+        break;
+      }
+      ++pf_it;
+      pf_k = nx_begin;
+      pf_end = nx_end;
+      pf_head = nx_head;
+      if (pf_it + 1 < it1) {
+        const PieItem f = p.items[pf_it + 1];
+        nx_begin = f.page_begin;
+        nx_end = f.page_end;
+        nx_head = f.kv_head;
+      }
+    }
+  };
+  // issue the copy of (physical page, head) into ring stage n % DEPTH (lane 0)
+  auto issue = [&](int n, int phys, int head) {
     const uint32_t s = n % DEPTH;
     // order this warp's generic-proxy accesses to the stage before the async-proxy overwrite
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     mbar_expect_tx(smem_u32(full_bar + s), C::STAGE);
-    bulk_g2s(smem_u32(stages + s * C::STAGE), p.pool + (int64_t)e.x * C::STAGE, C::STAGE, smem_u32(full_bar + s));
+    bulk_g2s(smem_u32(stages + s * C::STAGE), p.pool + ((int64_t)phys * p.n_kv_heads + head) * C::STAGE, C::STAGE,
+             smem_u32(full_bar + s));
   };
-  if (lane == 0)
-    for (int n = 0; n < DEPTH && n < n_total; ++n) issue(n, __ldg(stream + n));
+  pf_settle();
+  for (int n = 0; n < DEPTH && pf_live; ++n) {  // prologue: fill the ring
+    const int phys = __ldg(&p.kept[pf_k].x);
+    if (lane == 0) issue(n, phys, pf_head);
+    ++pf_k;
+    pf_settle();
+  }
 
-  int n = 0;  // stream position
+  int n = 0;  // visits consumed so far (ring position)
   for (int it = it0; it < it1; ++it) {
     const PieItem item = p.items[it];
     const PieReq rq = p.reqs[item.req];
     RowState<D> st;
     rows_init<D>(st, p, item, rq, item.row0, lane);
-    const int n_end = n + (item.page_end - item.page_begin);
-    for (; n < n_end; ++n) {
+    for (int k = item.page_begin; k < item.page_end; ++k, ++n) {
       const uint32_t s = n % DEPTH, ph = (n / DEPTH) & 1;
-      const uint32_t lpf = (uint32_t)__ldg(&stream[n].y);
-      int2 e_next = make_int2(0, 0);
-      if (lane == 0 && n + DEPTH < n_total) e_next = __ldg(stream + n + DEPTH);  // latency hides behind the wait
+      const uint32_t lpf = (uint32_t)__ldg(&p.kept[k].y);
+      const int phys_next = pf_live ? __ldg(&p.kept[pf_k].x) : 0;  // latency hides behind the wait
       mbar_wait(smem_u32(full_bar + s), ph, p.status);
       page_compute<D, P>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
       __syncwarp();
-      if (lane == 0 && n + DEPTH < n_total) issue(n + DEPTH, e_next);
+      if (pf_live) {
+        if (lane == 0) issue(n + DEPTH, phys_next, pf_head);
+        ++pf_k;
+        pf_settle();
+      }
     }
     rows_store<D>(st, p, item, rq, item.row0, 16, lane);
   }
@@ -549,8 +585,6 @@ AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& 
   p.mask = plan->d_mask;
   p.items = ll.d_items;
   p.cta_ptr = ll.d_cta_ptr;
-  p.stream = ll.d_stream;
-  p.stream_ptr = ll.d_stream_ptr;
   p.ws_o = ll.d_ws_o;
   p.ws_lse = ll.d_ws_lse;
   p.status = ctx->d_status;
@@ -707,13 +741,11 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   const size_t o_tok = put(plan.tok_req.data(), plan.tok_req.size() * 4);
   const size_t o_simple = put(plan.simple_rows.data(), plan.simple_rows.size() * 4);
   PieLaunchList* lls[2] = {&plan.split, &plan.tile};
-  size_t o_li[2], o_lc[2], o_lm[2], o_ls[2], o_lp[2], o_wo[2], o_wl[2];
+  size_t o_li[2], o_lc[2], o_lm[2], o_wo[2], o_wl[2];
   for (int k = 0; k < 2; ++k) {
     o_li[k] = put(lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
     o_lc[k] = put(lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
     o_lm[k] = put(lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
-    o_ls[k] = put(lls[k]->stream.data(), lls[k]->stream.size() * 4);
-    o_lp[k] = put(lls[k]->stream_ptr.data(), lls[k]->stream_ptr.size() * 4);
   }
   size_t total = (host.size() + 255) & ~(size_t)255;
   const int D = ctx->cfg.head_dim;
@@ -738,8 +770,6 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
     lls[k]->d_items = (PieItem*)(base + o_li[k]);
     lls[k]->d_cta_ptr = (int32_t*)(base + o_lc[k]);
     lls[k]->d_merges = (PieMerge*)(base + o_lm[k]);
-    lls[k]->d_stream = (int2*)(base + o_ls[k]);
-    lls[k]->d_stream_ptr = (int32_t*)(base + o_lp[k]);
     lls[k]->d_ws_o = (float*)(base + o_wo[k]);
     lls[k]->d_ws_lse = (float*)(base + o_wl[k]);
   }

@@ -71,12 +71,6 @@ struct PieLaunchList {           // one tile-kernel launch (split-KV decode, or 
   int32_t grid = 0;
   int32_t n_slots = 0;
   int32_t slot_rows = 0;
-  // split-KV kernel only: the page visits of every share, flattened in item order.
-  // entry = (physical page * H_kv + kv head, logical page | needs-mask flag)
-  std::vector<int32_t> stream;
-  std::vector<int32_t> stream_ptr;  // [grid+1]
-  int2* d_stream = nullptr;
-  int32_t* d_stream_ptr = nullptr;
   // device copies
   PieItem* d_items = nullptr;
   int32_t* d_cta_ptr = nullptr;
@@ -91,6 +85,7 @@ struct pie_plan {
   int32_t R = 0, T = 0;
   std::vector<PieReq> reqs;
   std::vector<int32_t> kept;        // pairs (phys, logical|flag)
+  std::vector<int32_t> kept_scratch; // planner scratch (per-request slices before packing)
   std::vector<uint32_t> mask_words;
   std::vector<int32_t> append_dst;  // [T] page*P + slot
   std::vector<int32_t> tok_req;     // [T]
@@ -108,6 +103,7 @@ struct pie_plan {
   int32_t* d_simple_rows = nullptr;
 };
 
+struct pie_plan;
 struct pie_ctx {
   pie_config cfg{};
   PoolGeom geom{};
@@ -122,8 +118,11 @@ struct pie_ctx {
   int* d_status = nullptr;
   void* d_stage = nullptr;  // staging for host <-> device calls
   size_t stage_bytes = 0;
-  void* d_io = nullptr;     // q/k/v/out/lse staging of pie_forward_host
+  void* d_io = nullptr;     // device arena of pie_forward_host: plan image + q/k/v/out/lse
   size_t io_bytes = 0;
+  void* h_stage = nullptr;  // pinned host staging of the plan image (pie_forward_host)
+  size_t h_stage_bytes = 0;
+  pie_plan* host_plan = nullptr;  // reused plan object of pie_forward_host
   std::string cuda_error;
   // optional per-kernel timing (pie_set_kernel_timing)
   bool timing = false;
@@ -146,8 +145,6 @@ struct AttnParams {
   const uint32_t* mask;
   const PieItem* items;
   const int32_t* cta_ptr;
-  const int2* stream;
-  const int32_t* stream_ptr;
   float* ws_o;
   float* ws_lse;
   int* status;

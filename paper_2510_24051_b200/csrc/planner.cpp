@@ -6,7 +6,9 @@
 // bit-packed masks, a page list with fully masked pages removed, append destinations, and a
 // work partition that gives every SM an equal share of page visits.
 #include <algorithm>
+#include <atomic>
 #include <cstring>
+#include <thread>
 
 #include "pie_internal.h"
 
@@ -35,15 +37,6 @@ struct Unit {
   int32_t req, kv_head, row0, nrows, page_begin, page_end;
 };
 
-// Finish a launch list from per-CTA item vectors.
-void flatten(std::vector<std::vector<PieItem>>& per_cta, PieLaunchList& ll) {
-  ll.cta_ptr.push_back(0);
-  for (auto& v : per_cta) {
-    for (const PieItem& it : v) ll.items.push_back(it);
-    ll.cta_ptr.push_back((int32_t)ll.items.size());
-  }
-}
-
 // Give each of `grid` CTAs (or warps) a share of the page visits of `units`.
 //  * Many units, none of them large against a share: whole units are dealt out in order, each to
 //    the least-loaded CTA (equal units => round robin).  Units that are neighbours in the batch
@@ -66,28 +59,47 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
     W += u.page_end - u.page_begin;
     max_unit = std::max<int64_t>(max_unit, u.page_end - u.page_begin);
   }
-  int grid = (int)std::min<int64_t>(grid_max, std::max<int64_t>(1, W / std::max(1, min_pages_per_cta)));
+  const int grid = (int)std::min<int64_t>(grid_max, std::max<int64_t>(1, W / std::max(1, min_pages_per_cta)));
   ll.grid = grid;
-  std::vector<std::vector<PieItem>> per_cta(grid);
 
   if (allow_whole_units && (int64_t)units.size() >= 4 * (int64_t)grid && max_unit * 8 <= W / grid) {
-    // least-loaded-first list scheduling; a binary heap keyed on (load, cta)
+    // least-loaded-first list scheduling (binary heap keyed on (load, cta)), then a counting sort
     std::vector<std::pair<int64_t, int>> heap(grid);
     for (int c = 0; c < grid; ++c) heap[c] = {0, c};
     auto cmp = [](const std::pair<int64_t, int>& a, const std::pair<int64_t, int>& b) { return a > b; };
     std::make_heap(heap.begin(), heap.end(), cmp);
-    for (const Unit& u : units) {
+    std::vector<int32_t> owner(units.size());
+    ll.cta_ptr.assign(grid + 1, 0);
+    for (size_t k = 0; k < units.size(); ++k) {
       std::pop_heap(heap.begin(), heap.end(), cmp);
       auto& top = heap.back();
-      per_cta[top.second].push_back(PieItem{u.req, u.kv_head, u.row0, u.nrows, u.page_begin, u.page_end, -1, 0});
-      top.first += std::max<int64_t>(1, u.page_end - u.page_begin);
+      owner[k] = top.second;
+      ++ll.cta_ptr[top.second + 1];
+      top.first += std::max<int64_t>(1, units[k].page_end - units[k].page_begin);
       std::push_heap(heap.begin(), heap.end(), cmp);
     }
-    flatten(per_cta, ll);
+    for (int c = 0; c < grid; ++c) ll.cta_ptr[c + 1] += ll.cta_ptr[c];
+    std::vector<int32_t> fill(ll.cta_ptr.begin(), ll.cta_ptr.end() - 1);
+    ll.items.resize(units.size());
+    for (size_t k = 0; k < units.size(); ++k) {
+      const Unit& u = units[k];
+      ll.items[fill[owner[k]]++] = PieItem{u.req, u.kv_head, u.row0, u.nrows, u.page_begin, u.page_end, -1, 0};
+    }
     return;
   }
 
-  int64_t off = 0;
+  // Contiguous shares.  Walking the units in order visits the shares in order too, so the items
+  // come out already grouped by CTA.
+  ll.items.reserve(units.size() + grid);
+  ll.cta_ptr.reserve(grid + 1);
+  ll.cta_ptr.push_back(0);
+  int cur = 0;  // CTA whose item range is open
+  auto open_cta = [&](int c) {
+    while (cur < c) {
+      ll.cta_ptr.push_back((int32_t)ll.items.size());
+      ++cur;
+    }
+  };
   auto cta_of = [&](int64_t x) {  // share that holds page-visit x
     if (W == 0) return 0;
     int64_t c = (x * grid) / W;
@@ -95,38 +107,36 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
     while (c > 0 && (c * W) / grid > x) --c;
     return (int)std::min<int64_t>(c, grid - 1);
   };
+  int64_t off = 0;
   for (const Unit& u : units) {
-    int64_t n = u.page_end - u.page_begin;
+    const int64_t n = u.page_end - u.page_begin;
     if (n == 0) {
-      PieItem it{u.req, u.kv_head, u.row0, u.nrows, u.page_begin, u.page_begin, -1, 0};
-      per_cta[cta_of(std::min(off, W > 0 ? W - 1 : 0))].push_back(it);
+      open_cta(std::max(cur, cta_of(std::min(off, W > 0 ? W - 1 : 0))));
+      ll.items.push_back(PieItem{u.req, u.kv_head, u.row0, u.nrows, u.page_begin, u.page_begin, -1, 0});
       continue;
     }
-    // pieces: cut at share boundaries strictly inside (off, off+n)
-    std::vector<std::pair<int64_t, int>> cuts;  // (start offset, cta)
+    const int first_item = (int)ll.items.size();
     int64_t x = off;
-    while (x < off + n) {
-      int c = cta_of(x);
+    while (x < off + n) {  // pieces: cut at share boundaries strictly inside (off, off+n)
+      const int c = cta_of(x);
       int64_t end = (c + 1 == grid) ? W : ((int64_t)(c + 1) * W) / grid;
       if (end <= x) end = x + 1;
-      cuts.push_back({x, c});
-      x = std::min(end, off + n);
+      end = std::min(end, off + n);
+      open_cta(c);
+      ll.items.push_back(PieItem{u.req, u.kv_head, u.row0, u.nrows, (int32_t)(u.page_begin + (x - off)),
+                                 (int32_t)(u.page_begin + (end - off)), -1, 0});
+      x = end;
     }
-    int np = (int)cuts.size();
-    int slot0 = ll.n_slots;
-    for (int k = 0; k < np; ++k) {
-      int64_t b = cuts[k].first, e = (k + 1 < np) ? cuts[k + 1].first : off + n;
-      PieItem it{u.req, u.kv_head, u.row0, u.nrows, (int32_t)(u.page_begin + (b - off)),
-                 (int32_t)(u.page_begin + (e - off)), np > 1 ? slot0 + k : -1, 0};
-      per_cta[cuts[k].second].push_back(it);
-    }
+    const int np = (int)ll.items.size() - first_item;
     if (np > 1) {
-      ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, slot0, np});
+      for (int k = 0; k < np; ++k) ll.items[first_item + k].partial_slot = ll.n_slots + k;
+      ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, ll.n_slots, np});
       ll.n_slots += np;
     }
     off += n;
   }
-  flatten(per_cta, ll);
+  open_cta(grid - 1);
+  ll.cta_ptr.push_back((int32_t)ll.items.size());
 }
 
 }  // namespace
@@ -214,27 +224,46 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     if (status != PIE_OK) return status;
   }
 
-  // ---- masks: pack explicit ones, classify pages, build the kept-page list
-  plan->mask_words.clear();
+  // ---- masks: pack explicit ones, classify pages, build the kept-page list.
+  // Word offsets are fixed first; then requests are independent, so large batches (tens of MB of
+  // mask bytes) are packed by several host threads, each writing its own requests' slices.
   plan->kept.clear();
   const uint32_t full_bits = (P >= 32) ? 0xFFFFFFFFu : ((1u << P) - 1u);
+  int64_t n_words = 0, mask_bytes_total = 0;
   for (int r = 0; r < R; ++r) {
+    PieReq& q = plan->reqs[r];
+    int64_t m0 = 0, m1 = 0;
+    if (b->mask_indptr) { m0 = b->mask_indptr[r]; m1 = b->mask_indptr[r + 1]; }
+    if (m1 < m0) return PIE_ERR_MASK;
+    if (m1 > m0) {
+      if (!b->mask || m1 - m0 != (int64_t)q.q_len * q.kv_len) return PIE_ERR_MASK;
+      q.mask_row_words = ((q.kv_len + 127) / 128) * 4;
+      q.mask_word_off = n_words;
+      n_words += (int64_t)q.mask_row_words * q.q_len;
+      mask_bytes_total += m1 - m0;
+    } else {
+      q.mask_row_words = 0;
+      q.mask_word_off = 0;
+    }
+  }
+  plan->mask_words.assign((size_t)n_words, 0u);
+  // every request first writes its kept pages into its own slice of a scratch array (sized for
+  // "all pages kept"); the slices are then packed together in request order
+  std::vector<int32_t>& scratch = plan->kept_scratch;
+  scratch.resize(2 * (size_t)b->page_indptr[R]);
+  std::atomic<int> bad_mask{0};
+  auto do_request = [&](int r) {
     PieReq& q = plan->reqs[r];
     const int32_t* pages = b->page_indices + b->page_indptr[r];
     const int np = q.last_logical + 1;
-    int64_t m0 = 0, m1 = 0;
-    if (b->mask_indptr) { m0 = b->mask_indptr[r]; m1 = b->mask_indptr[r + 1]; }
-    q.kept_start = (int32_t)(plan->kept.size() / 2);
-    if (m1 > m0) {
-      if (!b->mask || m1 - m0 != (int64_t)q.q_len * q.kv_len) return PIE_ERR_MASK;
-      const int row_words = ((q.kv_len + 127) / 128) * 4;
-      q.mask_row_words = row_words;
-      q.mask_word_off = (int64_t)plan->mask_words.size();
-      plan->mask_words.resize(plan->mask_words.size() + (size_t)row_words * q.q_len, 0u);
+    int32_t* kept = scratch.data() + 2 * (size_t)b->page_indptr[r];
+    int nk = 0;
+    if (q.mask_row_words) {
+      const int row_words = q.mask_row_words;
+      const uint8_t* src = b->mask + b->mask_indptr[r];
       uint32_t* w = plan->mask_words.data() + q.mask_word_off;
       for (int i = 0; i < q.q_len; ++i)
-        if (!pack_row(b->mask + m0 + (int64_t)i * q.kv_len, q.kv_len, w + (size_t)i * row_words))
-          return PIE_ERR_MASK;
+        if (!pack_row(src + (int64_t)i * q.kv_len, q.kv_len, w + (size_t)i * row_words)) bad_mask.store(1);
       for (int lp = 0; lp < np; ++lp) {
         const int bit = lp * P;
         uint32_t any = 0, all = full_bits;
@@ -244,20 +273,47 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
           all &= bits;
         }
         if (!any) continue;  // no query row attends to this page: it is never fetched
-        plan->kept.push_back(pages[lp]);
-        plan->kept.push_back((int32_t)((uint32_t)lp | (all == full_bits ? 0u : PIE_KEPT_NEEDS_MASK)));
+        kept[2 * nk] = pages[lp];
+        kept[2 * nk + 1] = (int32_t)((uint32_t)lp | (all == full_bits ? 0u : PIE_KEPT_NEEDS_MASK));
+        ++nk;
       }
     } else {
-      if (m1 < m0) return PIE_ERR_MASK;
-      q.mask_row_words = 0;
-      q.mask_word_off = 0;
       const int lim0 = q.kv_len - q.q_len;  // last position the first query token sees
       for (int lp = 0; lp < np; ++lp) {
-        plan->kept.push_back(pages[lp]);
-        plan->kept.push_back((int32_t)((uint32_t)lp | (lp * P + P - 1 <= lim0 ? 0u : PIE_KEPT_NEEDS_MASK)));
+        kept[2 * lp] = pages[lp];
+        kept[2 * lp + 1] = (int32_t)((uint32_t)lp | (lp * P + P - 1 <= lim0 ? 0u : PIE_KEPT_NEEDS_MASK));
       }
+      nk = np;
     }
-    q.kept_count = (int32_t)(plan->kept.size() / 2) - q.kept_start;
+    q.kept_count = nk;
+  };
+  int n_threads = 1;
+  if (mask_bytes_total > (4 << 20)) {
+    n_threads = (int)std::min<int64_t>({(int64_t)std::max(1u, std::thread::hardware_concurrency()), 16, (int64_t)R});
+  }
+  if (n_threads <= 1) {
+    for (int r = 0; r < R; ++r) do_request(r);
+  } else {
+    std::atomic<int> next{0};
+    std::vector<std::thread> pool;
+    for (int t = 0; t < n_threads; ++t)
+      pool.emplace_back([&] {
+        for (int r = next.fetch_add(1); r < R; r = next.fetch_add(1)) do_request(r);
+      });
+    for (auto& th : pool) th.join();
+  }
+  if (bad_mask.load()) return PIE_ERR_MASK;
+  {
+    size_t total = 0;
+    for (int r = 0; r < R; ++r) total += (size_t)plan->reqs[r].kept_count;
+    plan->kept.resize(2 * total);
+    size_t at = 0;
+    for (int r = 0; r < R; ++r) {
+      PieReq& q = plan->reqs[r];
+      q.kept_start = (int32_t)at;
+      std::memcpy(plan->kept.data() + 2 * at, scratch.data() + 2 * (size_t)b->page_indptr[r], 8 * (size_t)q.kept_count);
+      at += (size_t)q.kept_count;
+    }
   }
 
   // ---- append destinations
@@ -304,21 +360,6 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   }
   // split-KV decode: one share per warp of a full grid (every warp is its own pipeline)
   partition(split_units, ctx->n_sms * pie_split_warps_per_block(ctx), 4, 16, false, plan->split);
-  {
-    PieLaunchList& ll = plan->split;
-    ll.stream.clear();
-    ll.stream_ptr.assign(1, 0);
-    for (int c = 0; c < ll.grid; ++c) {
-      for (int k = ll.cta_ptr[c]; k < ll.cta_ptr[c + 1]; ++k) {
-        const PieItem& it = ll.items[k];
-        for (int e = it.page_begin; e < it.page_end; ++e) {
-          ll.stream.push_back(plan->kept[2 * e] * cfg.num_kv_heads + it.kv_head);
-          ll.stream.push_back(plan->kept[2 * e + 1]);
-        }
-      }
-      ll.stream_ptr.push_back((int32_t)(ll.stream.size() / 2));
-    }
-  }
   partition(tile_units, ctx->n_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile);
 
   pie_plan_info& info = plan->info;

@@ -42,14 +42,20 @@ def test_static_scratch_forward_matches_planned_forward(name):
 def test_static_scratch_rejects_batches_beyond_its_size():
     import paper_2510_24051_b200 as pie
     from tests._gpu import GpuPool
-    from workloads import configs
-    # 600 long decode requests need far more than 16 MiB of partials + page streams
-    wl = configs.batched_decode(R=600, lo=3000, hi=4000, num_pages=160000)
-    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
-        q, k, v = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
+    # 72 requests x 64 query tokens x 32,768 context positions of explicit mask pack to 18.9 MB of
+    # mask words: more than the 16 MiB array on their own, whatever else the plan holds
+    R, q_len, kv_len, P, H_q, H_kv, D = 72, 64, 32768, 16, 4, 2, 64
+    npg = kv_len // P
+    assert R * q_len * kv_len // 8 > pie.PIE_STATIC_SCRATCH_BYTES
+    with GpuPool(R * npg, P, H_q, H_kv, D, "bf16") as gp:
+        qo = np.arange(R + 1) * q_len
+        pi = np.arange(R + 1) * npg
+        mask = np.ones(R * q_len * kv_len, dtype=np.uint8)
+        mi = np.arange(R + 1, dtype=np.int64) * q_len * kv_len
+        q = torch.zeros((R * q_len, H_q, D), dtype=torch.bfloat16, device="cuda")
+        k = torch.zeros((R * q_len, H_kv, D), dtype=torch.bfloat16, device="cuda")
         out = torch.empty_like(q)
-        lse = torch.empty((wl.T, wl.H_q), dtype=torch.float32, device="cuda")
+        lse = torch.empty((R * q_len, H_q), dtype=torch.float32, device="cuda")
         with pytest.raises(pie.PieError) as e:
-            pie.pie_forward_static_scratch(gp.ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices,
-                                           wl.last_page_len, q, k, v, out, lse)
+            pie.pie_forward_static_scratch(gp.ctx, qo, pi, np.arange(R * npg), np.full(R, P), q, k, k, out, lse, mi, mask)
         assert e.value.status == pie.PIE_ERR_BATCH_TOO_LARGE
