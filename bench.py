@@ -190,6 +190,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="batched_decode")
     ap.add_argument("--flags", type=int, default=0, help="PIE_PLAN_* flags (debug / A-B runs)")
+    ap.add_argument("--opt", action="append", default=[], help="pie_set_option as K=V (tuning runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -220,6 +221,9 @@ def main():
     ctx = pie.pie_create(wl0.num_pages, wl0.P, wl0.H_q, wl0.H_kv, wl0.D, wl0.dtype, max(wl0.R, 1), max(wl0.T, 1), local)
     ids = pie.pie_alloc_kvpages(ctx, wl0.num_pages)
     assert np.array_equal(ids, np.arange(wl0.num_pages))
+    for kv in args.opt:
+        k, v = kv.split("=")
+        pie.pie_set_option(ctx, int(k), int(v))
     for wl in wls:                                     # install the pre-existing context (device generator)
         used = wl.used_pages()
         for i in range(0, len(used), 4096):

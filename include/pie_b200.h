@@ -212,6 +212,17 @@ int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* batch, const 
                                const void* k_new, const void* v_new, void* out, float* lse,
                                void* stream);
 
+/* Tuning knobs (all optional; 0 restores the default).  They affect plans made afterwards.
+ *   PIE_OPT_SPLIT_SMS  SMs the split-KV decode kernel may use (default: all).
+ *   PIE_OPT_TILE_SMS   SMs the prefill / tree kernel may use (default: all).
+ *   PIE_OPT_OVERLAP    mixed batches: 0 = default (the decode kernel, then the prefill / tree
+ *                      kernel), 1 = side by side on disjoint SM sets, the second on an internal
+ *                      stream that forks from and joins the caller's stream.  Pays only when the
+ *                      tensor-bound part is long against the HBM-bound part: the decode kernel
+ *                      needs about 60 % of the SMs to keep the memory system saturated. */
+enum { PIE_OPT_SPLIT_SMS = 0, PIE_OPT_TILE_SMS = 1, PIE_OPT_OVERLAP = 2, PIE_NUM_OPTIONS = 3 };
+int pie_set_option(pie_ctx* ctx, int option, int value);
+
 /* Per-kernel device timing for benchmarks.  While enabled, pie_forward and pie_copy_kvpage
  * bracket each kernel they enqueue with CUDA events on the caller's stream.
  * pie_get_kernel_times waits for the recorded events, adds the elapsed milliseconds and the

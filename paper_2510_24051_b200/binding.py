@@ -70,6 +70,7 @@ def _load():
         "pie_forward_host": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
         "pie_get_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int)]),
         "pie_forward_static_scratch": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
+        "pie_set_option": (C.c_int, [vp, C.c_int, C.c_int]),
         "pie_set_kernel_timing": (C.c_int, [vp, C.c_int]),
         "pie_get_kernel_times": (C.c_int, [vp, vp, vp]),
     }
@@ -256,3 +257,10 @@ def pie_forward_static_scratch(ctx, qo_indptr, page_indptr, page_indices, last_p
     d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags)
     _check(lib.pie_forward_static_scratch(ctx, C.byref(d), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
                                           _ptr(lse), _stream(stream)), ctx)
+
+
+PIE_OPT_SPLIT_SMS, PIE_OPT_TILE_SMS, PIE_OPT_OVERLAP = 0, 1, 2
+
+
+def pie_set_option(ctx, option, value):
+    _check(lib.pie_set_option(ctx, option, value), ctx)

@@ -114,7 +114,7 @@ bool page_ok(const pie_ctx* ctx, int32_t id) {
 // Device image of a plan: every array the kernels read, 256-byte aligned, followed by the fp32
 // partial workspaces of the two tile launches.
 struct PlanLayout {
-  size_t reqs, kept, mask, app, tok, simple, items[2], cta[2], merges[2], ws_o[2], ws_lse[2];
+  size_t reqs, kept, mask, app, tok, simple, items[2], cta[2], merges[2], ctr[2], ws_o[2], ws_lse[2];
   size_t upload, total;
 };
 
@@ -137,6 +137,7 @@ PlanLayout plan_layout(const pie_ctx* ctx, const pie_plan* plan) {
     L.items[k] = place(lls[k]->items.size() * sizeof(PieItem));
     L.cta[k] = place(lls[k]->cta_ptr.size() * 4);
     L.merges[k] = place(lls[k]->merges.size() * sizeof(PieMerge));
+    L.ctr[k] = place(8);
   }
   L.upload = off;
   const size_t D = ctx->cfg.head_dim;
@@ -163,6 +164,7 @@ void plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
     cp(L.items[k], lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
     cp(L.cta[k], lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
     cp(L.merges[k], lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
+    std::memset(dst + L.ctr[k], 0, 8);  // work counters start at zero; the kernel re-arms them itself
   }
 }
 
@@ -178,6 +180,7 @@ void plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base) {
     lls[k]->d_items = (PieItem*)(base + L.items[k]);
     lls[k]->d_cta_ptr = (int32_t*)(base + L.cta[k]);
     lls[k]->d_merges = (PieMerge*)(base + L.merges[k]);
+    lls[k]->d_work_ctr = (int32_t*)(base + L.ctr[k]);
     lls[k]->d_ws_o = (float*)(base + L.ws_o[k]);
     lls[k]->d_ws_lse = (float*)(base + L.ws_lse[k]);
   }
@@ -299,6 +302,9 @@ int pie_destroy(pie_ctx* ctx) {
     if (ctx->d_stage) cudaFree(ctx->d_stage);
     if (ctx->d_io) cudaFree(ctx->d_io);
     if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
+    if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     for (auto& t : ctx->timed) {
       cudaEventDestroy(t.start);
       cudaEventDestroy(t.stop);
@@ -509,18 +515,36 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
   if (!plan->simple_rows.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_SIMPLE, s, [&] { return pie_launch_simple(ctx, plan, q, out, lse, s); })))
     return rc;
+  const bool side = plan->overlap && !plan->split.items.empty() && !plan->tile.items.empty();
+  cudaStream_t s2 = s;
+  if (side) {
+    // fork: the tile kernel (and its merge) runs on the context's side stream, next to the
+    // decode kernel on the caller's stream; both joined again before the call returns
+    if (!ctx->side_stream) {
+      PIE_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking));
+      PIE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
+      PIE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming));
+    }
+    s2 = ctx->side_stream;
+    PIE_CUDA(ctx, cudaEventRecord(ctx->ev_fork, s));
+    PIE_CUDA(ctx, cudaStreamWaitEvent(s2, ctx->ev_fork, 0));
+  }
+  if (!plan->tile.items.empty() &&
+      (rc = timed_launch(ctx, PIE_KERNEL_TILES, s2, [&] { return pie_launch_tiles(ctx, plan, q, out, lse, s2); })))
+    return rc;
+  if (!plan->tile.merges.empty() &&
+      (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s2, [&] { return pie_launch_merge(ctx, plan, plan->tile, out, lse, s2); })))
+    return rc;
   if (!plan->split.items.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_SPLIT, s, [&] { return pie_launch_split(ctx, plan, q, out, lse, s); })))
-    return rc;
-  if (!plan->tile.items.empty() &&
-      (rc = timed_launch(ctx, PIE_KERNEL_TILES, s, [&] { return pie_launch_tiles(ctx, plan, q, out, lse, s); })))
     return rc;
   if (!plan->split.merges.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s, [&] { return pie_launch_merge(ctx, plan, plan->split, out, lse, s); })))
     return rc;
-  if (!plan->tile.merges.empty() &&
-      (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s, [&] { return pie_launch_merge(ctx, plan, plan->tile, out, lse, s); })))
-    return rc;
+  if (side) {
+    PIE_CUDA(ctx, cudaEventRecord(ctx->ev_join, s2));
+    PIE_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_join, 0));
+  }
   return PIE_OK;
 }
 
@@ -584,6 +608,12 @@ int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out) {
     PIE_CUDA(ctx, cudaStreamSynchronize(s));
   }
   *out = v;
+  return PIE_OK;
+}
+
+int pie_set_option(pie_ctx* ctx, int option, int value) {
+  if (!ctx || option < 0 || option >= PIE_NUM_OPTIONS || value < 0) return PIE_ERR_INVALID;
+  ctx->options[option] = value;
   return PIE_OK;
 }
 

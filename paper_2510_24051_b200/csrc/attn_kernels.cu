@@ -169,6 +169,8 @@ __device__ __forceinline__ void page_compute(RowState<D>& st, uint8_t* stage, co
       const int t = rq.last_page_len + c / CH, ch = c % CH;
       *reinterpret_cast<uint4*>(stage + BLK + pie_chunk_offset(SLAB, t, ch)) = make_uint4(0, 0, 0, 0);
     }
+    // these generic-proxy writes must be ordered before the bulk copy that later refills the stage
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
   }
   if (!st.any_rows) return;
@@ -300,100 +302,168 @@ __device__ __forceinline__ void rows_store(RowState<D>& st, const AttnParams& p,
 }
 
 // ------------------------------------------------------------------------------ split-KV decode
-// Every warp is an independent pipeline over its own contiguous share of the batch's page
-// visits (the planner cuts the visits into equal shares, one per warp of the grid).  The warp
-// keeps DEPTH bulk copies in flight into a private ring and refills a stage as soon as it has
-// consumed it, so there is no producer warp, no empty barrier and no block-level sync.
+// Every warp is an independent pipeline.  The planner cuts every (request, kv head) into chunks
+// of pages - large ones first, small ones for the tail - and the warps of the grid take chunks
+// from a global counter as they go, so SMs that get less memory bandwidth simply take fewer
+// chunks and all of them finish together.  A warp keeps DEPTH bulk copies in flight into a
+// private ring and refills a stage as soon as it has consumed it: no producer warp, no empty
+// barrier, no block-level sync.  The chunk after the current one is taken a few pages early so
+// that neither the atomic nor the chunk record is ever waited for.
 template <int D, int P, int NW, int DEPTH>
 struct SplitCfg {
   static constexpr int STAGE = 2 * P * D * 2;
-  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * 8 + 64;
+  static constexpr int QUEUE = 8;  // chunk ids a warp has started fetching but not finished (<= DEPTH + 2)
+  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * 12 + NW * QUEUE * 4 + 64;
 };
 
 template <int D, int P, int NW, int DEPTH>
-__global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams p, int n_warps) {
+__global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams p, int n_items, int n_warps) {
   using C = SplitCfg<D, P, NW, DEPTH>;
+  static_assert(DEPTH + 2 <= C::QUEUE, "queue too small");
   extern __shared__ __align__(1024) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int wg = blockIdx.x * NW + warp;
-  if (wg >= n_warps) return;
   uint8_t* stages = smem + warp * DEPTH * C::STAGE;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + NW * DEPTH * C::STAGE) + warp * DEPTH;
+  volatile uint32_t* meta = reinterpret_cast<uint32_t*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 8) + warp * DEPTH;
+  volatile int* queue = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 12) + warp * C::QUEUE;
   if (lane == 0) {
     for (int s = 0; s < DEPTH; ++s) mbar_init(smem_u32(full_bar + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
 
-  const int it0 = p.cta_ptr[wg], it1 = p.cta_ptr[wg + 1];
+  // ---- prefetch side: a cursor DEPTH page visits ahead of the consumer
+  int q_head = 0, q_tail = 0;                       // queue of chunk ids, pushed here, popped by the consumer
+  int pf_k = 0, pf_end = 0, pf_head = 0;            // cursor inside its current chunk
+  int nx_begin = 0, nx_end = 0, nx_head = 0, nx_idx = -1;  // record of the chunk after it (when nx_idx >= 0)
+  int grabbed = 0;                                  // lane 0: result of an atomic whose value is not needed yet
+  bool grab_pending = false, exhausted = false, pf_live = true;
 
-  // Prefetch cursor: the page visit DEPTH positions ahead of the one being consumed.  It walks
-  // the same item list; the next item's record is fetched one item early so that crossing an
-  // item boundary costs no memory latency.
-  int pf_it = it0 - 1, pf_k = 0, pf_end = 0, pf_head = 0;
-  int nx_begin = 0, nx_end = 0, nx_head = 0;
-  if (it0 < it1) {
-    const PieItem f = p.items[it0];
-    nx_begin = f.page_begin;
-    nx_end = f.page_end;
-    nx_head = f.kv_head;
+  // Small launches use fixed shares instead (cta_ptr != nullptr): warp w owns items
+  // [cta_ptr[w], cta_ptr[w+1]) and "taking" is just counting through them.
+  const bool fixed_shares = p.cta_ptr != nullptr;
+  const int wg = blockIdx.x * NW + warp;
+  int own_next = 0, own_end = 0;
+  if (fixed_shares && wg < p.n_shares) {
+    own_next = p.cta_ptr[wg];
+    own_end = p.cta_ptr[wg + 1];
   }
-  bool pf_live = true;
-  auto pf_settle = [&]() {  // move to the next non-empty item while the current one is used up
+  auto take = [&]() {  // synchronous: next chunk id for this warp
+    if (fixed_shares) return own_next < own_end ? own_next++ : n_items;
+    int v = 0;
+    if (lane == 0) v = atomicAdd(p.work_ctr, 1);
+    return __shfl_sync(0xFFFFFFFFu, v, 0);
+  };
+  auto load_next_record = [&](int idx) {
+    if (idx >= n_items) {
+      exhausted = true;
+      return;
+    }
+    const int4 r0 = __ldg(reinterpret_cast<const int4*>(p.items + idx));      // req, kv_head, row0, nrows
+    const int2 r1 = __ldg(reinterpret_cast<const int2*>(p.items + idx) + 2);  // page_begin, page_end
+    nx_head = r0.y;
+    nx_begin = r1.x;
+    nx_end = r1.y;
+    nx_idx = idx;
+  };
+  auto pf_settle = [&]() {  // enter the next chunk while the current one is used up
     while (pf_live && pf_k >= pf_end) {
-      if (pf_it + 1 >= it1) {
+      if (nx_idx < 0 && !exhausted) {  // start-up, or chunks shorter than the look-ahead
+        const int idx = grab_pending ? __shfl_sync(0xFFFFFFFFu, grabbed, 0) : take();
+        grab_pending = false;
+        load_next_record(idx);
+      }
+      if (nx_idx < 0) {
         pf_live = false;
         break;
       }
-      ++pf_it;
       pf_k = nx_begin;
       pf_end = nx_end;
       pf_head = nx_head;
-      if (pf_it + 1 < it1) {
-        const PieItem f = p.items[pf_it + 1];
-        nx_begin = f.page_begin;
-        nx_end = f.page_end;
-        nx_head = f.kv_head;
-      }
+      if (lane == 0) queue[q_tail % C::QUEUE] = nx_idx;
+      ++q_tail;
+      nx_idx = -1;
+      __syncwarp();
     }
   };
-  // issue the copy of (physical page, head) into ring stage n % DEPTH (lane 0)
-  auto issue = [&](int n, int phys, int head) {
+  auto pf_lookahead = [&]() {  // two steps, a few pages apart, so that nothing is waited for
+    if (!pf_live || nx_idx >= 0 || exhausted) return;
+    const int left = pf_end - pf_k;
+    if (!grab_pending) {
+      if (left <= 4) {
+        if (fixed_shares) grabbed = own_next < own_end ? own_next++ : n_items;
+        else if (lane == 0) grabbed = atomicAdd(p.work_ctr, 1);
+        grab_pending = true;
+      }
+    } else if (left <= 2) {
+      const int idx = __shfl_sync(0xFFFFFFFFu, grabbed, 0);
+      grab_pending = false;
+      load_next_record(idx);
+    }
+  };
+  // (The stage was last read with ldmatrix by this same warp, and those reads have returned
+  // their registers before the warp gets here, so the overwrite needs no proxy fence; the one
+  // generic-proxy write to a stage, clearing rows of a last page, fences for itself.)
+  auto issue = [&](int n, int2 rec, int head) {
     const uint32_t s = n % DEPTH;
-    // order this warp's generic-proxy accesses to the stage before the async-proxy overwrite
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    meta[s] = (uint32_t)rec.y;  // logical page | needs-mask flag, read back by the warp after the wait
     mbar_expect_tx(smem_u32(full_bar + s), C::STAGE);
-    bulk_g2s(smem_u32(stages + s * C::STAGE), p.pool + ((int64_t)phys * p.n_kv_heads + head) * C::STAGE, C::STAGE,
+    bulk_g2s(smem_u32(stages + s * C::STAGE), p.pool + ((int64_t)rec.x * p.n_kv_heads + head) * C::STAGE, C::STAGE,
              smem_u32(full_bar + s));
   };
+
   pf_settle();
   for (int n = 0; n < DEPTH && pf_live; ++n) {  // prologue: fill the ring
-    const int phys = __ldg(&p.kept[pf_k].x);
-    if (lane == 0) issue(n, phys, pf_head);
+    const int2 rec = __ldg(&p.kept[pf_k]);
+    if (lane == 0) issue(n, rec, pf_head);
     ++pf_k;
+    pf_lookahead();
     pf_settle();
   }
 
+  // ---- consumer side
   int n = 0;  // visits consumed so far (ring position)
-  for (int it = it0; it < it1; ++it) {
-    const PieItem item = p.items[it];
-    const PieReq rq = p.reqs[item.req];
+  while (q_head < q_tail) {
+    const int idx = queue[q_head % C::QUEUE];
+    ++q_head;
+    const PieItem item = p.items[idx];
+    PieReq rq;  // the chunk carries its request's record
+    rq.q_start = item.q_start;
+    rq.q_len = item.q_len;
+    rq.kv_len = item.kv_len;
+    rq.kept_start = 0;
+    rq.kept_count = 0;
+    rq.mask_row_words = item.mask_row_words;
+    rq.mask_word_off = item.mask_word_off;
+    rq.last_logical = item.last_logical;
+    rq.last_page_len = item.last_page_len;
     RowState<D> st;
     rows_init<D>(st, p, item, rq, item.row0, lane);
     for (int k = item.page_begin; k < item.page_end; ++k, ++n) {
       const uint32_t s = n % DEPTH, ph = (n / DEPTH) & 1;
-      const uint32_t lpf = (uint32_t)__ldg(&p.kept[k].y);
-      const int phys_next = pf_live ? __ldg(&p.kept[pf_k].x) : 0;  // latency hides behind the wait
+      int2 rec_next = make_int2(0, 0);
+      if (pf_live) rec_next = __ldg(&p.kept[pf_k]);  // latency hides behind the wait
       mbar_wait(smem_u32(full_bar + s), ph, p.status);
+      const uint32_t lpf = meta[s];
       page_compute<D, P>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
       __syncwarp();
       if (pf_live) {
-        if (lane == 0) issue(n + DEPTH, phys_next, pf_head);
+        if (lane == 0) issue(n + DEPTH, rec_next, pf_head);
         ++pf_k;
+        pf_lookahead();
         pf_settle();
       }
     }
-    rows_store<D>(st, p, item, rq, item.row0, 16, lane);
+    rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);
+  }
+
+  // ---- the last warp of the grid to finish re-arms the counters for the next launch
+  if (lane == 0 && !fixed_shares) {
+    __threadfence();
+    if (atomicAdd(p.work_ctr + 1, 1) == n_warps - 1) {
+      p.work_ctr[0] = 0;
+      p.work_ctr[1] = 0;
+    }
   }
 }
 
@@ -479,37 +549,55 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) attn_tile_kernel(const AttnP
 
 // ------------------------------------------------------------------------------ merge kernel
 // lse = ln sum_c exp(lse_c), o = sum_c exp(lse_c - lse) o_c over the partial slots of a group.
-template <typename T>
+template <typename T, int D>
 __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* __restrict__ reqs,
                              const float* __restrict__ ws_o, const float* __restrict__ ws_lse, T* __restrict__ out,
-                             float* __restrict__ lse_out, int slot_rows, int D, int n_q_heads, int G) {
-  // block (x, y): merge group x, rows [16 y, 16 y + 16) of it
+                             float* __restrict__ lse_out, int slot_rows, int n_q_heads, int G) {
+  // One warp per (merge group, row).  Lanes share the slots for the max and the weights, then each
+  // lane owns D/32 consecutive columns and the slot loop issues independent, coalesced row loads.
+  // (Every partial row is written by its kernel, with zeros when its part of the context was empty.)
+  constexpr int EPL = D / 32;
   const PieMerge mg = merges[blockIdx.x];
-  const int r0 = blockIdx.y * 16;
-  if (r0 >= mg.nrows) return;
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= mg.nrows) return;
   const PieReq rq = reqs[mg.req];
-  const int nr = min(16, mg.nrows - r0);
-  for (int e = threadIdx.x; e < nr * D; e += blockDim.x) {
-    const int row = r0 + e / D, d = e % D;
-    float M = kNegInf;
-    for (int c = 0; c < mg.nslots; ++c) M = fmaxf(M, ws_lse[(int64_t)(mg.slot0 + c) * slot_rows + row]);
-    float Z = 0.f, acc = 0.f;
-    if (M != kNegInf) {
-      for (int c = 0; c < mg.nslots; ++c) {
-        const int64_t si = (int64_t)(mg.slot0 + c) * slot_rows + row;
-        const float l = ws_lse[si];
-        if (l == kNegInf) continue;  // an empty partial: its O rows were never written
-        const float w = __expf(l - M);
-        Z += w;
-        acc += w * ws_o[si * D + d];
+  const float* lse_in = ws_lse + (int64_t)mg.slot0 * slot_rows + row;
+  const float* o_in = ws_o + ((int64_t)mg.slot0 * slot_rows + row) * D + lane * EPL;
+  const int64_t slot_stride = (int64_t)slot_rows * D;
+  float M = kNegInf;
+  for (int c = lane; c < mg.nslots; c += 32) M = fmaxf(M, lse_in[(int64_t)c * slot_rows]);
+  for (int sft = 16; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));
+  float Z = 0.f, acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  for (int base = 0; base < mg.nslots; base += 32) {
+    const int c = base + lane;
+    float w = 0.f;
+    if (c < mg.nslots && M != kNegInf) w = __expf(lse_in[(int64_t)c * slot_rows] - M);  // exp(-inf) = 0
+    Z += w;
+    const int cnt = min(32, mg.nslots - base);
+#pragma unroll 4
+    for (int u = 0; u < cnt; ++u) {
+      const float wu = __shfl_sync(0xFFFFFFFFu, w, u);
+      const float* src = o_in + (base + u) * slot_stride;
+      if constexpr (EPL == 4) {
+        const float4 v = *reinterpret_cast<const float4*>(src);
+        acc[0] += wu * v.x, acc[1] += wu * v.y, acc[2] += wu * v.z, acc[3] += wu * v.w;
+      } else {
+        const float2 v = *reinterpret_cast<const float2*>(src);
+        acc[0] += wu * v.x, acc[1] += wu * v.y;
       }
     }
-    const int gr = mg.row0 + row;
-    const int tok = gr / G, head = mg.kv_head * G + gr % G;
-    const int64_t oi = (int64_t)(rq.q_start + tok) * n_q_heads + head;
-    out[oi * D + d] = (T)(Z > 0.f ? acc / Z : 0.f);
-    if (d == 0) lse_out[oi] = Z > 0.f ? M + logf(Z) : kNegInf;
   }
+  for (int sft = 16; sft > 0; sft >>= 1) Z += __shfl_xor_sync(0xFFFFFFFFu, Z, sft);
+  const int gr = mg.row0 + row;
+  const int tok = gr / G, head = mg.kv_head * G + gr % G;
+  const int64_t oi = (int64_t)(rq.q_start + tok) * n_q_heads + head;
+  const float inv = Z > 0.f ? 1.f / Z : 0.f;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) out[oi * D + lane * EPL + e] = (T)(acc[e] * inv);
+  if (lane == 0) lse_out[oi] = Z > 0.f ? M + logf(Z) : kNegInf;
 }
 
 // ------------------------------------------------------------------------------ simple kernel
@@ -584,7 +672,10 @@ AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& 
   p.kept = plan->d_kept;
   p.mask = plan->d_mask;
   p.items = ll.d_items;
-  p.cta_ptr = ll.d_cta_ptr;
+  p.cta_ptr = ll.cta_ptr.empty() ? nullptr : ll.d_cta_ptr;
+  p.n_shares = ll.cta_ptr.empty() ? 0 : (int)ll.cta_ptr.size() - 1;
+  p.work_ctr = ll.d_work_ctr;
+  p.slot_rows = ll.slot_rows;
   p.ws_o = ll.d_ws_o;
   p.ws_lse = ll.d_ws_lse;
   p.status = ctx->d_status;
@@ -597,7 +688,7 @@ AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& 
 }
 
 template <int D, int P, int NW, int DEPTH>
-int launch_split(pie_ctx* ctx, const AttnParams& p, int n_warps, cudaStream_t s) {
+int launch_split(pie_ctx* ctx, const AttnParams& p, int n_items, int n_warps, cudaStream_t s) {
   using C = SplitCfg<D, P, NW, DEPTH>;
   auto kern = attn_split_kernel<D, P, NW, DEPTH>;
   static bool configured[8] = {};
@@ -606,7 +697,8 @@ int launch_split(pie_ctx* ctx, const AttnParams& p, int n_warps, cudaStream_t s)
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
     configured[dev] = true;
   }
-  kern<<<(n_warps + NW - 1) / NW, NW * 32, C::SMEM, s>>>(p, n_warps);
+  const int blocks = (n_warps + NW - 1) / NW;
+  kern<<<blocks, NW * 32, C::SMEM, s>>>(p, n_items, blocks * NW);
   PIE_CUDA(ctx, cudaGetLastError());
   return PIE_OK;
 }
@@ -642,12 +734,12 @@ int pie_split_warps_per_block(const pie_ctx* ctx) {
 
 int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s) {
   AttnParams p = make_params(ctx, plan, plan->split, q, out, lse);
-  const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size, n = plan->split.grid;
+  const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size, n = plan->split.grid, ni = (int)plan->split.items.size();
   // ring depth: about 192 KB of copies in flight per SM
-  if (D == 64 && P == 16) return launch_split<64, 16, 8, 6>(ctx, p, n, s);
-  if (D == 128 && P == 16) return launch_split<128, 16, 8, 3>(ctx, p, n, s);
-  if (D == 64 && P == 32) return launch_split<64, 32, 8, 3>(ctx, p, n, s);
-  if (D == 128 && P == 32) return launch_split<128, 32, 4, 3>(ctx, p, n, s);
+  if (D == 64 && P == 16) return launch_split<64, 16, 8, 6>(ctx, p, ni, n, s);
+  if (D == 128 && P == 16) return launch_split<128, 16, 8, 3>(ctx, p, ni, n, s);
+  if (D == 64 && P == 32) return launch_split<64, 32, 8, 3>(ctx, p, ni, n, s);
+  if (D == 128 && P == 32) return launch_split<128, 32, 4, 3>(ctx, p, ni, n, s);
   return PIE_ERR_UNSUPPORTED;
 }
 
@@ -664,13 +756,19 @@ int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* ou
 
 int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s) {
   const int D = ctx->cfg.head_dim;
-  const dim3 n((unsigned)ll.merges.size(), (unsigned)((ll.slot_rows + 15) / 16));
-  if (ctx->cfg.dtype == PIE_DTYPE_BF16)
-    merge_kernel<__nv_bfloat16><<<n, 256, 0, s>>>(ll.d_merges, plan->d_reqs, ll.d_ws_o, ll.d_ws_lse, (__nv_bfloat16*)out, lse,
-                                                   ll.slot_rows, D, ctx->cfg.num_q_heads, ctx->G);
-  else
-    merge_kernel<float><<<n, 256, 0, s>>>(ll.d_merges, plan->d_reqs, ll.d_ws_o, ll.d_ws_lse, (float*)out, lse, ll.slot_rows, D,
-                                           ctx->cfg.num_q_heads, ctx->G);
+  const int wpb = ll.slot_rows >= 8 ? 8 : 4;  // warps (= rows) per block
+  const dim3 n((unsigned)ll.merges.size(), (unsigned)((ll.slot_rows + wpb - 1) / wpb));
+#define PIE_MERGE(T, DD)                                                                                          \
+  merge_kernel<T, DD><<<n, wpb * 32, 0, s>>>(ll.d_merges, plan->d_reqs, ll.d_ws_o, ll.d_ws_lse, (T*)out, lse, \
+                                             ll.slot_rows, ctx->cfg.num_q_heads, ctx->G)
+  if (ctx->cfg.dtype == PIE_DTYPE_BF16) {
+    if (D == 64) PIE_MERGE(__nv_bfloat16, 64);
+    else PIE_MERGE(__nv_bfloat16, 128);
+  } else {
+    if (D == 64) PIE_MERGE(float, 64);
+    else PIE_MERGE(float, 128);
+  }
+#undef PIE_MERGE
   PIE_CUDA(ctx, cudaGetLastError());
   return PIE_OK;
 }
@@ -722,7 +820,10 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
 
   pie_plan plan;  // host-side only; its device pointers will point into the static scratch
   plan.ctx = ctx;
+  const int saved_overlap = ctx->options[PIE_OPT_OVERLAP];
+  ctx->options[PIE_OPT_OVERLAP] = 0;  // this entry point enqueues its kernels one after the other
   int rc = pie_build_plan(ctx, batch, &plan);
+  ctx->options[PIE_OPT_OVERLAP] = saved_overlap;
   if (rc != PIE_OK) return rc;
   if (plan.T == 0) return PIE_OK;
   if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
@@ -741,10 +842,12 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   const size_t o_tok = put(plan.tok_req.data(), plan.tok_req.size() * 4);
   const size_t o_simple = put(plan.simple_rows.data(), plan.simple_rows.size() * 4);
   PieLaunchList* lls[2] = {&plan.split, &plan.tile};
-  size_t o_li[2], o_lc[2], o_lm[2], o_wo[2], o_wl[2];
+  size_t o_li[2], o_lc[2], o_lm[2], o_wo[2], o_wl[2], o_ctr[2];
+  const int32_t zero_ctr[2] = {0, 0};  // work counters of the split-KV kernel start at zero
   for (int k = 0; k < 2; ++k) {
     o_li[k] = put(lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
     o_lc[k] = put(lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
+    o_ctr[k] = put(zero_ctr, sizeof(zero_ctr));
     o_lm[k] = put(lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
   }
   size_t total = (host.size() + 255) & ~(size_t)255;
@@ -770,6 +873,7 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
     lls[k]->d_items = (PieItem*)(base + o_li[k]);
     lls[k]->d_cta_ptr = (int32_t*)(base + o_lc[k]);
     lls[k]->d_merges = (PieMerge*)(base + o_lm[k]);
+    lls[k]->d_work_ctr = (int32_t*)(base + o_ctr[k]);
     lls[k]->d_ws_o = (float*)(base + o_wo[k]);
     lls[k]->d_ws_lse = (float*)(base + o_wl[k]);
   }

@@ -53,8 +53,11 @@ struct PieItem {
   int32_t req, kv_head, row0, nrows;
   int32_t page_begin, page_end;  // absolute indices into the kept-page list
   int32_t partial_slot;          // -1: write the final output; else slot of the fp32 partial
-  int32_t pad;
+  // copy of the request record, so that a kernel can start an item from this one 64-byte line
+  int32_t q_start, q_len, kv_len, mask_row_words, last_logical, last_page_len, pad;
+  int64_t mask_word_off;
 };
+static_assert(sizeof(PieItem) == 64, "PieItem is one 64-byte line");
 
 // A group of partial slots that the merge kernel combines into final rows.
 struct PieMerge {
@@ -75,6 +78,7 @@ struct PieLaunchList {           // one tile-kernel launch (split-KV decode, or 
   PieItem* d_items = nullptr;
   int32_t* d_cta_ptr = nullptr;
   PieMerge* d_merges = nullptr;
+  int32_t* d_work_ctr = nullptr; // [2] dynamic-scheduling counters (split-KV kernel), zero between launches
   float* d_ws_o = nullptr;       // [n_slots][slot_rows][D]
   float* d_ws_lse = nullptr;     // [n_slots][slot_rows]
 };
@@ -92,6 +96,7 @@ struct pie_plan {
   std::vector<int32_t> simple_rows; // (token*H_q + head) rows for the plain kernel
   PieLaunchList split, tile;
   bool tile_tc = false;             // row tiles run on the tcgen05 kernel (256-row items)
+  bool overlap = false;             // decode and tile kernels run side by side on disjoint SM sets
   pie_plan_info info{};
   // device
   void* d_blob = nullptr;           // one allocation holding every array below
@@ -124,6 +129,9 @@ struct pie_ctx {
   size_t h_stage_bytes = 0;
   pie_plan* host_plan = nullptr;  // reused plan object of pie_forward_host
   std::string cuda_error;
+  int options[PIE_NUM_OPTIONS] = {0, 0, 0};
+  cudaStream_t side_stream = nullptr;  // second stream of overlapped mixed batches
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   // optional per-kernel timing (pie_set_kernel_timing)
   bool timing = false;
   struct TimedLaunch { int kind; cudaEvent_t start, stop; };
@@ -145,6 +153,9 @@ struct AttnParams {
   const uint32_t* mask;
   const PieItem* items;
   const int32_t* cta_ptr;
+  int32_t* work_ctr;
+  int32_t n_shares;   // split-KV kernel with fixed shares: entries of cta_ptr minus one
+  int32_t slot_rows;
   float* ws_o;
   float* ws_lse;
   int* status;

@@ -37,6 +37,18 @@ struct Unit {
   int32_t req, kv_head, row0, nrows, page_begin, page_end;
 };
 
+PieItem make_item(const Unit& u, int32_t page_begin, int32_t page_end) {
+  PieItem it{};
+  it.req = u.req;
+  it.kv_head = u.kv_head;
+  it.row0 = u.row0;
+  it.nrows = u.nrows;
+  it.page_begin = page_begin;
+  it.page_end = page_end;
+  it.partial_slot = -1;
+  return it;
+}
+
 // Give each of `grid` CTAs (or warps) a share of the page visits of `units`.
 //  * Many units, none of them large against a share: whole units are dealt out in order, each to
 //    the least-loaded CTA (equal units => round robin).  Units that are neighbours in the batch
@@ -83,7 +95,7 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
     ll.items.resize(units.size());
     for (size_t k = 0; k < units.size(); ++k) {
       const Unit& u = units[k];
-      ll.items[fill[owner[k]]++] = PieItem{u.req, u.kv_head, u.row0, u.nrows, u.page_begin, u.page_end, -1, 0};
+      ll.items[fill[owner[k]]++] = make_item(u, u.page_begin, u.page_end);
     }
     return;
   }
@@ -112,7 +124,7 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
     const int64_t n = u.page_end - u.page_begin;
     if (n == 0) {
       open_cta(std::max(cur, cta_of(std::min(off, W > 0 ? W - 1 : 0))));
-      ll.items.push_back(PieItem{u.req, u.kv_head, u.row0, u.nrows, u.page_begin, u.page_begin, -1, 0});
+      ll.items.push_back(make_item(u, u.page_begin, u.page_begin));
       continue;
     }
     const int first_item = (int)ll.items.size();
@@ -123,8 +135,7 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
       if (end <= x) end = x + 1;
       end = std::min(end, off + n);
       open_cta(c);
-      ll.items.push_back(PieItem{u.req, u.kv_head, u.row0, u.nrows, (int32_t)(u.page_begin + (x - off)),
-                                 (int32_t)(u.page_begin + (end - off)), -1, 0});
+      ll.items.push_back(make_item(u, (int32_t)(u.page_begin + (x - off)), (int32_t)(u.page_begin + (end - off))));
       x = end;
     }
     const int np = (int)ll.items.size() - first_item;
@@ -137,6 +148,51 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
   }
   open_cta(grid - 1);
   ll.cta_ptr.push_back((int32_t)ll.items.size());
+}
+
+// Split-KV decode: cut every unit into chunks that the warps of the grid take from a global
+// counter at run time.  Units in the first 80 % of the page visits get large chunks (about a
+// third of a warp's fair share), the rest small ones, and the large chunks come first in the
+// list, so the end of the launch is filled with short pieces of work.
+void chunk_units(const std::vector<Unit>& units, int n_warps, PieLaunchList& ll) {
+  ll.items.clear();
+  ll.merges.clear();
+  ll.cta_ptr.clear();
+  ll.n_slots = 0;
+  ll.slot_rows = 1;
+  ll.grid = 0;
+  if (units.empty()) return;
+  int64_t W = 0;
+  for (const Unit& u : units) {
+    W += u.page_end - u.page_begin;
+    ll.slot_rows = std::max(ll.slot_rows, u.nrows);
+  }
+  const int64_t share = std::max<int64_t>(1, W / std::max(1, n_warps));
+  const int c_big = (int)std::min<int64_t>(128, std::max<int64_t>(4, share / 3));
+  const int c_small = std::min(16, std::max(2, c_big / 4));
+  const int64_t tail_start = W - W / 5;
+  std::vector<PieItem> small;
+  int64_t off = 0;
+  for (const Unit& u : units) {
+    const int n = u.page_end - u.page_begin;
+    const bool tail = off >= tail_start;
+    const int c = tail ? c_small : c_big;
+    const int nchunks = (n + c - 1) / c;
+    std::vector<PieItem>& dst = tail ? small : ll.items;
+    for (int k = 0; k < nchunks; ++k) {  // chunks of equal size (+-1 page)
+      const int b = (int)((int64_t)n * k / nchunks), e = (int)((int64_t)n * (k + 1) / nchunks);
+      PieItem it = make_item(u, u.page_begin + b, u.page_begin + e);
+      if (nchunks > 1) it.partial_slot = ll.n_slots + k;
+      dst.push_back(it);
+    }
+    if (nchunks > 1) {
+      ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, ll.n_slots, nchunks});
+      ll.n_slots += nchunks;
+    }
+    off += n;
+  }
+  ll.items.insert(ll.items.end(), small.begin(), small.end());
+  ll.grid = (int)std::min<int64_t>(n_warps, (int64_t)ll.items.size());
 }
 
 }  // namespace
@@ -338,7 +394,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   for (int r = 0; r < R; ++r) {
     const PieReq& q = plan->reqs[r];
     const int rows = q.q_len * G;
-    if (!tiles_ok) {
+    if (!tiles_ok || q.kept_count == 0) {  // (a request with no attendable page only needs zeros / -inf written)
       for (int i = 0; i < q.q_len; ++i)
         for (int h = 0; h < cfg.num_q_heads; ++h) plan->simple_rows.push_back((q.q_start + i) * cfg.num_q_heads + h);
     } else if (rows <= 16) {
@@ -358,10 +414,58 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
         }
     }
   }
-  // split-KV decode: one share per warp of a full grid (every warp is its own pipeline)
-  partition(split_units, ctx->n_sms * pie_split_warps_per_block(ctx), 4, 16, false, plan->split);
-  partition(tile_units, ctx->n_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile);
+  // SM budget of the two tile kernels.  On request (PIE_OPT_OVERLAP) a mixed batch runs them side
+  // by side: the decode kernel is HBM bound and saturates the memory system from roughly 60 % of
+  // the SMs, so it keeps at least that many and otherwise a share proportional to its estimated
+  // time; the rest go to the tensor-bound prefill / tree kernel.
+  int split_sms = ctx->options[PIE_OPT_SPLIT_SMS] > 0 ? std::min(ctx->options[PIE_OPT_SPLIT_SMS], ctx->n_sms) : ctx->n_sms;
+  int tile_sms = ctx->options[PIE_OPT_TILE_SMS] > 0 ? std::min(ctx->options[PIE_OPT_TILE_SMS], ctx->n_sms) : ctx->n_sms;
+  plan->overlap = false;
+  if (!split_units.empty() && !tile_units.empty() && plan->tile_tc && ctx->options[PIE_OPT_OVERLAP] == 1 &&
+      ctx->options[PIE_OPT_SPLIT_SMS] == 0 && ctx->options[PIE_OPT_TILE_SMS] == 0 && ctx->n_sms >= 16) {
+    double split_bytes = 0, tile_flops = 0;
+    for (const Unit& u : split_units) split_bytes += (double)(u.page_end - u.page_begin) * 2.0 * P * cfg.head_dim * 2.0;
+    for (const Unit& u : tile_units) tile_flops += (double)(u.page_end - u.page_begin) * P * 4.0 * cfg.head_dim * 256.0;
+    const double t_split = split_bytes / 6.0e12, t_tile = tile_flops / 1.0e15;  // whole-chip estimates, seconds
+    const int floor_split = (ctx->n_sms * 5) / 8;
+    int n_split = (int)(ctx->n_sms * t_split / (t_split + t_tile) + 0.5);
+    n_split = std::max(n_split, floor_split);
+    n_split = std::min(n_split, ctx->n_sms - 8);
+    split_sms = n_split;
+    tile_sms = ctx->n_sms - n_split;
+    plan->overlap = true;
+  }
+  // split-KV decode.  Long launches: chunks taken dynamically by the warps of the grid (evens out
+  // SMs that get different shares of the memory bandwidth).  Short launches: fixed equal shares,
+  // one per warp - fewer pieces, fewer partials to merge, and the per-chunk overheads matter more
+  // than the balance.
+  {
+    const int n_warps = split_sms * pie_split_warps_per_block(ctx);
+    int64_t W = 0;
+    int max_rows = 1;
+    for (const Unit& u : split_units) {
+      W += u.page_end - u.page_begin;
+      max_rows = std::max(max_rows, u.nrows);
+    }
+    if (W >= (int64_t)200 * n_warps) {
+      chunk_units(split_units, n_warps, plan->split);
+    } else {
+      partition(split_units, n_warps, 4, max_rows, false, plan->split);
+    }
+  }
+  partition(tile_units, tile_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile);
 
+  for (PieLaunchList* ll : {&plan->split, &plan->tile})
+    for (PieItem& it : ll->items) {
+      const PieReq& q = plan->reqs[it.req];
+      it.q_start = q.q_start;
+      it.q_len = q.q_len;
+      it.kv_len = q.kv_len;
+      it.mask_row_words = q.mask_row_words;
+      it.last_logical = q.last_logical;
+      it.last_page_len = q.last_page_len;
+      it.mask_word_off = q.mask_word_off;
+    }
   pie_plan_info& info = plan->info;
   info = pie_plan_info{};
   info.num_requests = R;

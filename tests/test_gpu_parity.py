@@ -118,3 +118,20 @@ def test_repeat_calls_are_bitwise_deterministic():
         b = gp.forward(plan, q, k, v)
         assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
         pie.pie_plan_destroy(plan)
+
+
+def test_mixed_batch_side_by_side_option_matches_oracle():
+    """PIE_OPT_OVERLAP: decode and prefill kernels on disjoint SM sets, forked / joined streams."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs.small("mixed_prefill_decode")
+    O_ref, L_ref, _ = run_oracle(wl)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl)
+        pie.pie_set_option(gp.ctx, pie.PIE_OPT_OVERLAP, 1)
+        plan = gp.plan(wl)
+        q, k, v = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
+        for _ in range(3):
+            out, lse = gp.forward(plan, q, k, v)
+            check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        pie.pie_plan_destroy(plan)
