@@ -126,6 +126,36 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
                "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
                : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                 "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr));
+}
+// packed fp32x2 arithmetic (two independent fp32 lanes in one 64-bit register) and 3-input max
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0,%1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -246,6 +276,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
       uint32_t n_items[2] = {0, 0};   // items in which Q tile t took part (phase of q_full / o_done / o_free)
       uint32_t n_tiles[2] = {0, 0};   // KV tiles Q tile t went through (phase of s_full / p_full)
       const uint32_t idesc_pv = instr_desc(kTileM, D, 1);
+      const uint64_t k_desc0 = smem_desc(smem_u32(sK), 16, 1024);            // K-major
+      const uint64_t v_desc0 = smem_desc(smem_u32(sV), C::SLAB_TILE, 1024);  // MN-major: LBO = slab stride
+      const uint64_t q_desc0 = smem_desc(smem_u32(sQ), 16, 1024);
       for (int it = it0; it < it1; ++it) {
         const PieItem item = p.items[it];
         const PieReq rq = p.reqs[item.req];
@@ -260,15 +293,17 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
         }
         tc_fence_after();
 
+        // Descriptors are built once (per kernel for the K / V stages, per item for Q); a k-step only
+        // adds its byte offset >> 4 to the start-address field.
         auto issue_s = [&](int t, int j, uint32_t cnt) {
           const uint32_t s = cnt % C::STAGES;
           const int nvalid = min(C::PPT, npages - j * C::PPT);
           const uint32_t idesc = instr_desc(kTileM, nvalid * P, 0);
-          const uint32_t qa = smem_u32(sQ + t * C::QTILE), kb = smem_u32(sK + s * C::KVTILE);
+          const uint64_t qd = q_desc0 + (uint64_t)(t * (C::QTILE >> 4)), kd = k_desc0 + (uint64_t)(s * (C::KVTILE >> 4));
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
-            const uint32_t off = (ks >> 2) * C::SLAB_TILE + (ks & 3) * 32;
-            umma_ss(tmem + t * 128, smem_desc(qa + off, 16, 1024), smem_desc(kb + off, 16, 1024), idesc, ks > 0);
+            const uint64_t off = (uint64_t)(((ks >> 2) * C::SLAB_TILE + (ks & 3) * 32) >> 4);
+            umma_ss(tmem + t * 128, qd + off, kd + off, idesc, ks > 0);
           }
           umma_commit(smem_u32(s_full + t));
         };
@@ -312,11 +347,12 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
             ++n_tiles[t];
             tc_fence_after();
             if (lane == 0) {
-              const uint32_t vb = smem_u32(sV + s * C::KVTILE);
+              const uint64_t vd = v_desc0 + (uint64_t)(s * (C::KVTILE >> 4));
               const int ksteps = nvalid * P / 16;
-              for (int ks = 0; ks < ksteps; ++ks)
-                umma_ts(tmem + 256 + t * D, tmem + t * 128 + ks * 8, smem_desc(vb + ks * 2048, C::SLAB_TILE, 1024),
-                        idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll 8
+              for (int ks = 0; ks < ksteps; ++ks)   // 16 token rows = 2048 bytes per k-step
+                umma_ts(tmem + 256 + t * D, tmem + t * 128 + ks * 8, vd + (uint64_t)(ks * 128), idesc_pv,
+                        (j > 0 || ks > 0) ? 1u : 0u);
               if (t == nt - 1) umma_commit(smem_u32(v_empty + s));
               if (j + 1 == ntiles) umma_commit(smem_u32(o_done + t));
             }
@@ -398,69 +434,79 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
           mbar_wait(smem_u32(s_full + t), my_tiles & 1, p.status);
           ++my_tiles;
           tc_fence_after();
-          // ---- pass 1: row maximum of the (masked) raw scores, 64 columns at a time
-          float mraw = kNegInf;
+          // ---- one pass over the row in 32-column chunks (online softmax with a lagging reference):
+          // P = exp2(S * scale - m_ref) goes back as bf16 over the first 64 columns of S_t.  m_ref may
+          // lag the true running maximum by up to 2^8; when a chunk exceeds that (rare after the first
+          // chunk of an item), O_t, the sums and the P chunks already written for this tile are brought
+          // to the new reference.  Scale-and-shift and the row sum use packed fp32x2 arithmetic.
+          uint64_t psum2 = pack_f32x2(0.f, 0.f);
+          const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+          float xbuf[2][32];   // double buffer: chunk k+1 is in flight while chunk k is processed
+          tmem_ld32(tS, reinterpret_cast<uint32_t*>(xbuf[0]));
+          tmem_wait_ld();
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            float a[64];
-            tmem_ld32(tS + h * 64, reinterpret_cast<uint32_t*>(a));
-            tmem_ld32(tS + h * 64 + 32, reinterpret_cast<uint32_t*>(a) + 32);
-            tmem_wait_ld();
+          for (int k = 0; k < kTileN / 32; ++k) {
+            float* x = xbuf[k & 1];
+            if (k + 1 < kTileN / 32) tmem_ld32(tS + (k + 1) * 32, reinterpret_cast<uint32_t*>(xbuf[(k + 1) & 1]));
             if (tile_mask) {
 #pragma unroll
-              for (int c = 0; c < 64; ++c)
-                if (!((bits[(h * 64 + c) / P] >> ((h * 64 + c) % P)) & 1u)) a[c] = kNegInf;
+              for (int c = 0; c < 32; ++c)
+                if (!((bits[(k * 32 + c) / P] >> ((k * 32 + c) % P)) & 1u)) x[c] = kNegInf;
             }
+            float cmax = kNegInf;
 #pragma unroll
-            for (int c = 0; c < 64; ++c) mraw = fmaxf(mraw, a[c]);
-          }
-          const float m_tile = mraw * p.scale_log2;   // -inf stays -inf
-          const float m_new = fmaxf(m_ref, m_tile);
-          if (my_tile_in_item == 0) {
-            m_ref = m_new;
-          } else {
-            const bool grow = m_new > m_ref + 8.f;     // also true when m_ref is -inf and m_new is finite
-            if (__any_sync(0xFFFFFFFFu, grow)) {
-              // rare: bring O_t (complete up to the previous tile: S_t of this tile was issued after
-              // it) to the new reference maximum
+            for (int c = 0; c < 32; c += 2) cmax = max3(cmax, x[c], x[c + 1]);
+            const float m_new = fmaxf(m_ref, cmax * p.scale_log2);   // -inf stays -inf
+            if (__any_sync(0xFFFFFFFFu, m_new > m_ref + 8.f)) {       // also when m_ref is -inf and m_new finite
               const float f = (m_ref == kNegInf) ? 1.f : fast_exp2(m_ref - m_new);
               if (m_new != kNegInf) m_ref = m_new;
               l_sum *= f;
+              psum2 = fma_f32x2(psum2, pack_f32x2(f, f), pack_f32x2(0.f, 0.f));
+              if (my_tile_in_item > 0) {   // O_t is complete up to the previous tile (S_t of this tile was issued after it)
+#pragma unroll 1
+                for (int c0 = 0; c0 < D; c0 += 16) {
+                  uint32_t o[16];
+                  tmem_ld16(tO + c0, o);
+                  tmem_wait_ld();
 #pragma unroll
-              for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t o[32];
-                tmem_ld32(tO + c0, o);
+                  for (int c = 0; c < 16; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
+                  tmem_st16(tO + c0, o);
+                }
+              }
+#pragma unroll 1
+              for (int kk = 0; kk < k; ++kk) {   // P chunks of this tile written under the old reference
+                uint32_t pp[16];
+                tmem_wait_st();
+                tmem_ld16(tS + kk * 16, pp);
                 tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
-                tmem_st32(tO + c0, o);
+                for (int c = 0; c < 16; ++c) {
+                  const float lo = __uint_as_float(pp[c] << 16) * f, hi = __uint_as_float(pp[c] & 0xFFFF0000u) * f;
+                  pp[c] = pack_bf16(lo, hi);
+                }
+                tmem_st16(tS + kk * 16, pp);
               }
               tmem_wait_st();
             }
-          }
-          // ---- pass 2: P = exp2(S * scale - m_ref) as bf16 over the first 64 columns of S_t
-          const float neg_m = (m_ref == kNegInf) ? 0.f : -m_ref;
-          float psum = 0.f;
+            const float neg_m = (m_ref == kNegInf) ? 0.f : -m_ref;
+            const uint64_t negm2 = pack_f32x2(neg_m, neg_m);
+            uint32_t pk[16];
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            float a[64];
-            tmem_ld32(tS + h * 64, reinterpret_cast<uint32_t*>(a));
-            tmem_ld32(tS + h * 64 + 32, reinterpret_cast<uint32_t*>(a) + 32);
-            tmem_wait_ld();
-            if (tile_mask) {
-#pragma unroll
-              for (int c = 0; c < 64; ++c)
-                if (!((bits[(h * 64 + c) / P] >> ((h * 64 + c) % P)) & 1u)) a[c] = kNegInf;
-            }
-            uint32_t pk[32];
-#pragma unroll
-            for (int c = 0; c < 64; c += 2) {
-              const float p0 = fast_exp2(fmaf(a[c], p.scale_log2, neg_m));
-              const float p1 = fast_exp2(fmaf(a[c + 1], p.scale_log2, neg_m));
-              psum += p0 + p1;
+            for (int c = 0; c < 32; c += 2) {
+              float e0, e1;
+              unpack_f32x2(fma_f32x2(pack_f32x2(x[c], x[c + 1]), scale2, negm2), e0, e1);
+              const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+              psum2 = add_f32x2(psum2, pack_f32x2(p0, p1));
               pk[c >> 1] = pack_bf16(p0, p1);
             }
-            tmem_st32(tS + h * 32, pk);
+            tmem_st16(tS + k * 16, pk);   // columns [16k, 16k+16): below every S column still to be read
+            if (k + 1 < kTileN / 32) tmem_wait_ld();
+          }
+          float psum;
+          {
+            float s0, s1;
+            unpack_f32x2(psum2, s0, s1);
+            psum = s0 + s1;
           }
           l_sum += psum;
           tmem_wait_st();
