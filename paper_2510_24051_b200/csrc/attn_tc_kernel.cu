@@ -47,15 +47,22 @@ __device__ __forceinline__ uint64_t global_ns() {
 // Bounded wait.  Gives up after ~1 s, or at once when any wait of this launch already gave up
 // (the status word is set), so a broken pipeline drains in bounded time instead of hanging.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status) {
-  const uint64_t t0 = global_ns();
-  while (!mbar_try_wait(bar, parity)) {
-    if (*reinterpret_cast<volatile int*>(status) != 0) return false;
-    if (global_ns() - t0 > 1000000000ull) {
-      atomicExch(status, (int)PIE_ERR_DEVICE_TIMEOUT);
-      return false;
+  // Poll tightly (try_wait itself parks the thread for a while when the phase is not complete);
+  // the clock and the status word - a global load - are looked at only every 256 polls, so a
+  // completed barrier is noticed at once.
+  uint64_t t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0) {
+      if (*reinterpret_cast<volatile int*>(status) != 0) return false;  // another wait of this launch gave up
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > 1000000000ull) {
+        atomicExch(status, (int)PIE_ERR_DEVICE_TIMEOUT);
+        return false;
+      }
     }
   }
-  return true;
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
