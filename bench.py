@@ -149,12 +149,15 @@ def oracle_sample(wl, budget_s=20.0):
         kv, ql = int(wl.kv_lens()[r]), int(wl.q_lens()[r])
         for lp in range((kv - ql) // wl.P, len(wl.pages_of(r))):
             pool[int(wl.pages_of(r)[lp])]
-    t0 = time.perf_counter()
-    orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
-                qb, kb, vb, wl.masks, requests=sample)
-    dt = time.perf_counter() - t0
+    times = []
+    while not times or (sum(times) < min(budget_s, 10.0) and len(times) < 20):   # repeat short passes
+        t0 = time.perf_counter()
+        orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                    qb, kb, vb, wl.masks, requests=sample)
+        times.append(time.perf_counter() - t0)
+    dt = statistics.mean(times)
     tokens = int(wl.q_lens()[sample].sum())
-    return tokens, dt, f"first {n} of {wl.R} requests of {wl.name}, one pass", threads
+    return tokens, dt, f"first {n} of {wl.R} requests of {wl.name}, mean of {len(times)} passes", threads
 
 
 def run_reference(args):

@@ -103,6 +103,17 @@ int pie_copy_kvpage(pie_ctx* ctx, int32_t n, const int32_t* src, const int32_t* 
                     const int32_t* src_off, const int32_t* dst_off, const int32_t* ntok,
                     void* stream);
 
+/* mask_kvpage (Table 1: "masks the KV cache in a token-level manner"; used by the attention-sink,
+ * windowed- and hierarchical-attention inferlets of Section 7).  Sets the persistent visibility
+ * mask of n pages: bit s of masks[k] set = slot s of page ids[k] may be attended to.  The mask
+ * stays with the page until it is set again; allocating a page resets it to all-visible.
+ * In forward a position is attended iff the batch mask (explicit or inferred) allows it AND its
+ * page-mask bit is set; a page none of whose slots is visible to a request is never fetched
+ * (the same as leaving the page out of the list, Section 4.2).  Host bookkeeping only; it
+ * affects plans made afterwards.  ids, masks: host, n entries.  PIE_ERR_BAD_PAGE if a page is
+ * out of range or not allocated (nothing is changed then). */
+int pie_mask_kvpage(pie_ctx* ctx, int32_t n, const int32_t* ids, const uint32_t* masks);
+
 /* One coalesced `forward` batch as the control layer hands it over (Section 5.2).
  * Request r has q_len = qo_indptr[r+1]-qo_indptr[r] >= 1 new tokens and the page list
  * page_indices[page_indptr[r] .. page_indptr[r+1]) (input KvPages followed by output KvPages;

@@ -15,6 +15,7 @@ KvPages; Section 4.2 "Forward API" for masks, positions and the append-then-read
                 with an explicit boolean mask (true = attend) or, when none is given, the
                 causal mask inferred from positions; grouped-query heads (kv = q // G);
   4. copy     - token-range copy of K and V rows between pages, bit for bit.
+  5. page masks (`mask_kvpage`) - persistent per-page token masks ANDed into the allowed set.
 
 All floating point is fp64 on exactly widened inputs.  There is no tiling, no online
 softmax and no reordering: a reader can check each function against the definition by eye.
@@ -146,8 +147,27 @@ def attend(q_r: np.ndarray, K: np.ndarray, V: np.ndarray, allowed: np.ndarray):
     return O, LSE
 
 
+def apply_page_masks(allowed: np.ndarray, pages, P: int, page_masks) -> np.ndarray:
+    """Persistent per-page token masks (Table 1 `mask_kvpage`): position j of a request stays
+    attendable only if slot j % P of its page pages[j // P] is visible.  page_masks maps a page id
+    to a bool [P] array (true = visible); pages without an entry are fully visible."""
+    if not page_masks:
+        return allowed
+    out = allowed.copy()
+    kv_len = allowed.shape[1]
+    for lp, page in enumerate(pages):
+        pm = page_masks.get(int(page))
+        if pm is None:
+            continue
+        lo, hi = lp * P, min((lp + 1) * P, kv_len)
+        if lo >= kv_len:
+            break
+        out[:, lo:hi] &= np.asarray(pm, dtype=bool)[None, : hi - lo]
+    return out
+
+
 def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
-            q, k_new, v_new, masks=None, append=True, requests=None):
+            q, k_new, v_new, masks=None, append=True, requests=None, page_masks=None):
     """One batched `forward`: append, then gather and attend for every request.
 
     q [T, H_q, D], k_new/v_new [T, H_kv, D] in the storage type; masks is None or a list
@@ -167,6 +187,7 @@ def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
         pages = page_indices[page_indptr[r]:page_indptr[r + 1]]
         kv_len = kv_len_of(len(pages), int(last_page_len[r]), P)
         allowed = allowed_matrix(t1 - t0, kv_len, None if masks is None else masks[r])
+        allowed = apply_page_masks(allowed, pages, P, page_masks)
         K, V = gather_kv(pool, P, pages, kv_len, needed=allowed.any(axis=0))
         O[t0:t1], LSE[t0:t1] = attend(widen(q[t0:t1]), K, V, allowed)
     return O, LSE

@@ -59,6 +59,7 @@ def _load():
         "pie_alloc_kvpages": (C.c_int, [vp, i32, vp]),
         "pie_dealloc_kvpages": (C.c_int, [vp, i32, vp]),
         "pie_num_free_kvpages": (C.c_int, [vp, C.POINTER(i32)]),
+        "pie_mask_kvpage": (C.c_int, [vp, i32, vp, vp]),
         "pie_kvpage_write": (C.c_int, [vp, i32, vp, vp, vp, C.c_int, vp]),
         "pie_kvpage_read": (C.c_int, [vp, i32, vp, vp, vp, C.c_int, vp]),
         "pie_copy_kvpage": (C.c_int, [vp, i32, vp, vp, vp, vp, vp, vp]),
@@ -264,3 +265,11 @@ PIE_OPT_SPLIT_SMS, PIE_OPT_TILE_SMS, PIE_OPT_OVERLAP = 0, 1, 2
 
 def pie_set_option(ctx, option, value):
     _check(lib.pie_set_option(ctx, option, value), ctx)
+
+
+def pie_mask_kvpage(ctx, ids, masks):
+    """Persistent per-page token masks: bit s of masks[k] set = slot s of page ids[k] visible."""
+    ids = _i32(ids)
+    m = np.ascontiguousarray(masks, dtype=np.uint32)
+    assert len(m) == len(ids)
+    _check(lib.pie_mask_kvpage(ctx, len(ids), ids.ctypes.data, m.ctypes.data), ctx)

@@ -261,6 +261,7 @@ int pie_create(const pie_config* cfg, pie_ctx** out) {
   g.block_bytes = P * g.row_bytes;
   g.page_bytes = (int64_t)cfg->num_kv_heads * 2 * g.block_bytes;
   ctx->allocated.assign(cfg->num_pages, 0);
+  ctx->page_mask.assign(cfg->num_pages, 0xFFFFFFFFu);
   ctx->free_list.resize(cfg->num_pages);
   for (int i = 0; i < cfg->num_pages; ++i) ctx->free_list[i] = cfg->num_pages - 1 - i;  // pop from the back: 0,1,2,..
   ctx->wmask.assign(cfg->num_pages, 0u);
@@ -323,6 +324,10 @@ int pie_alloc_kvpages(pie_ctx* ctx, int32_t n, int32_t* out_ids) {
     int32_t id = ctx->free_list.back();
     ctx->free_list.pop_back();
     ctx->allocated[id] = 1;
+    if (ctx->page_mask[id] != 0xFFFFFFFFu) {  // a fresh page is fully visible
+      ctx->page_mask[id] = 0xFFFFFFFFu;
+      --ctx->n_masked_pages;
+    }
     out_ids[i] = id;
   }
   return PIE_OK;
@@ -338,6 +343,21 @@ int pie_dealloc_kvpages(pie_ctx* ctx, int32_t n, const int32_t* ids) {
   for (int i = 0; i < n; ++i) {
     ctx->allocated[ids[i]] = 0;
     ctx->free_list.push_back(ids[i]);
+  }
+  return PIE_OK;
+}
+
+int pie_mask_kvpage(pie_ctx* ctx, int32_t n, const int32_t* ids, const uint32_t* masks) {
+  if (!ctx || n < 0 || (n > 0 && (!ids || !masks))) return PIE_ERR_INVALID;
+  for (int i = 0; i < n; ++i)
+    if (!page_ok(ctx, ids[i])) return PIE_ERR_BAD_PAGE;
+  const int P = ctx->cfg.page_size;
+  const uint32_t full = P >= 32 ? 0xFFFFFFFFu : ((1u << P) - 1u);
+  for (int i = 0; i < n; ++i) {
+    const uint32_t m = ((masks[i] & full) == full) ? 0xFFFFFFFFu : (masks[i] & full);
+    uint32_t& cur = ctx->page_mask[ids[i]];
+    ctx->n_masked_pages += (m != 0xFFFFFFFFu) - (cur != 0xFFFFFFFFu);
+    cur = m;
   }
   return PIE_OK;
 }

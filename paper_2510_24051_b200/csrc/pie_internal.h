@@ -118,6 +118,8 @@ struct pie_ctx {
   // allocator
   std::vector<int32_t> free_list;
   std::vector<uint8_t> allocated;
+  std::vector<uint32_t> page_mask;   // mask_kvpage: bit s = slot s visible (all ones by default)
+  int64_t n_masked_pages = 0;        // pages whose mask hides at least one slot
   // device
   uint8_t* pool = nullptr;
   int* d_status = nullptr;

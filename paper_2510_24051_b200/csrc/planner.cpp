@@ -291,8 +291,13 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     int64_t m0 = 0, m1 = 0;
     if (b->mask_indptr) { m0 = b->mask_indptr[r]; m1 = b->mask_indptr[r + 1]; }
     if (m1 < m0) return PIE_ERR_MASK;
-    if (m1 > m0) {
-      if (!b->mask || m1 - m0 != (int64_t)q.q_len * q.kv_len) return PIE_ERR_MASK;
+    bool page_masked = false;  // some page of the request carries a mask_kvpage mask
+    if (ctx->n_masked_pages > 0) {
+      const int32_t* pages = b->page_indices + b->page_indptr[r];
+      for (int lp = 0; lp <= q.last_logical && !page_masked; ++lp) page_masked = ctx->page_mask[pages[lp]] != 0xFFFFFFFFu;
+    }
+    if (m1 > m0 && (!b->mask || m1 - m0 != (int64_t)q.q_len * q.kv_len)) return PIE_ERR_MASK;
+    if (m1 > m0 || page_masked) {  // the request gets packed mask rows (given, or causal AND page masks)
       q.mask_row_words = ((q.kv_len + 127) / 128) * 4;
       q.mask_word_off = n_words;
       n_words += (int64_t)q.mask_row_words * q.q_len;
@@ -316,10 +321,29 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     int nk = 0;
     if (q.mask_row_words) {
       const int row_words = q.mask_row_words;
-      const uint8_t* src = b->mask + b->mask_indptr[r];
       uint32_t* w = plan->mask_words.data() + q.mask_word_off;
-      for (int i = 0; i < q.q_len; ++i)
-        if (!pack_row(src + (int64_t)i * q.kv_len, q.kv_len, w + (size_t)i * row_words)) bad_mask.store(1);
+      const bool given = b->mask_indptr && b->mask_indptr[r + 1] > b->mask_indptr[r];
+      if (given) {
+        const uint8_t* src = b->mask + b->mask_indptr[r];
+        for (int i = 0; i < q.q_len; ++i)
+          if (!pack_row(src + (int64_t)i * q.kv_len, q.kv_len, w + (size_t)i * row_words)) bad_mask.store(1);
+      } else {  // inferred causal rows, written out because page masks will be ANDed in
+        for (int i = 0; i < q.q_len; ++i) {
+          const int nbits = q.kv_len - q.q_len + i + 1;  // positions 0 .. lim
+          uint32_t* row = w + (size_t)i * row_words;
+          for (int k = 0; k < nbits / 32; ++k) row[k] = 0xFFFFFFFFu;
+          if (nbits & 31) row[nbits / 32] = (1u << (nbits & 31)) - 1u;
+        }
+      }
+      if (ctx->n_masked_pages > 0) {
+        for (int lp = 0; lp < np; ++lp) {
+          const uint32_t pm = ctx->page_mask[pages[lp]];
+          if (pm == 0xFFFFFFFFu) continue;
+          const int bit = lp * P;
+          const uint32_t clear = ~pm & full_bits;
+          for (int i = 0; i < q.q_len; ++i) w[(size_t)i * row_words + (bit >> 5)] &= ~(clear << (bit & 31));
+        }
+      }
       for (int lp = 0; lp < np; ++lp) {
         const int bit = lp * P;
         uint32_t any = 0, all = full_bits;

@@ -89,3 +89,13 @@ def test_full_long_context_policy_with_copy():
             assert same_bits(Ks[0][:n], Kd[0][:n]) and same_bits(Vs[0][:n], Vd[0][:n])
     finally:
         gp.close()
+
+
+def test_large_single_requests():
+    """Index arithmetic at the large end: a 131,071-token decode (8,192 pages, many split chunks and a
+    ragged last page) and a 300-token prefill chunk over a 20,000-token prefix in one batch."""
+    from workloads.configs import _assemble
+    wl = _assemble("large", 0x50494500 + 77, 32, 8, 128, 16, "bf16", 9600, [1, 300], [131071, 20300], None)
+    info, gp = _sampled_check(wl, sample=[0, 1])
+    gp.close()
+    assert info["num_split_items"] > 100 and info["num_tile_items"] > 0

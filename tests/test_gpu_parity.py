@@ -135,3 +135,29 @@ def test_mixed_batch_side_by_side_option_matches_oracle():
             out, lse = gp.forward(plan, q, k, v)
             check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
         pie.pie_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("name", ["batched_decode", "mixed_prefill_decode", "shared_prefix_tree", "long_context_policy", "tiny_fp32"])
+@pytest.mark.parametrize("flags", [0, 2])
+def test_mask_kvpage_matches_oracle(name, flags):
+    """Persistent page masks: random token masks on a third of the pages, some pages hidden entirely."""
+    import paper_2510_24051_b200 as pie
+    from oracle import pie_oracle as orc
+    from tests._gpu import GpuPool, check_close
+    wl = configs.small(name)
+    rng = np.random.RandomState(99)
+    used = wl.used_pages()
+    chosen = used[rng.rand(len(used)) < 0.35]
+    bits_ = rng.randint(0, 1 << wl.P, size=len(chosen), dtype=np.int64)
+    bits_[rng.rand(len(chosen)) < 0.3] = 0                      # hidden pages
+    page_masks = {int(p): np.array([(int(b) >> s) & 1 for s in range(wl.P)], bool) for p, b in zip(chosen, bits_)}
+    pool = wl.oracle_pool()
+    O_ref, L_ref = orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                               bits(wl.q()), bits(wl.k_new()), bits(wl.v_new()), wl.masks, page_masks=page_masks)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl)
+        pie.pie_mask_kvpage(gp.ctx, chosen, bits_.astype(np.uint32))
+        plan = gp.plan(wl, flags)
+        out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+        pie.pie_plan_destroy(plan)
+        check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype)

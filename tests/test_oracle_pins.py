@@ -374,3 +374,47 @@ def test_golden_worked_example():
         O, L = oracle_on(args)
         np.testing.assert_allclose(O[0, 0], O_exp, atol=1e-14)
         assert abs(L[0, 0] - L_exp) < 1e-14
+
+
+# mask_kvpage ---------------------------------------------------------------------------
+def test_page_masks_equal_textbook_with_columns_removed_and_page_omission():
+    """Persistent page masks (Table 1 `mask_kvpage`): attention with per-page token masks equals the
+    scalar textbook computation over (batch mask AND page-mask) columns; a page with every slot hidden
+    equals leaving the page out of the list (Section 4.2)."""
+    rng = np.random.RandomState(21)
+    P, H_q, H_kv, D = 8, 4, 2, 8
+    shapes = [(1, 37), (5, 30)]
+    m1 = rng.rand(5, 30) < 0.7
+    m1[:, 3] = True
+    seqs = random_seqs(rng, shapes, H_q, H_kv, D, masks=[None, m1])
+    args = SmallBatch(seqs, H_q).paged(P, "random", seed=2)
+    pages0 = args["page_indices"][args["page_indptr"][0]:args["page_indptr"][1]]
+    pages1 = args["page_indices"][args["page_indptr"][1]:args["page_indptr"][2]]
+    page_masks = {int(pages0[1]): rng.rand(P) < 0.5, int(pages0[3]): np.zeros(P, bool),
+                  int(pages1[0]): rng.rand(P) < 0.5, int(pages1[2]): np.zeros(P, bool)}
+    O, L = orc.forward(**args, page_masks=page_masks)
+    t = 0
+    for s, (q_len, kv_len), pages in zip(seqs, shapes, (pages0, pages1)):
+        allowed = np.array(causal(q_len, kv_len)) if s.get("mask") is None else s["mask"].copy()
+        col = np.ones(kv_len, bool)
+        for lp, pg in enumerate(pages):
+            if int(pg) in page_masks:
+                col[lp * P:(lp + 1) * P] = page_masks[int(pg)][: max(0, min(P, kv_len - lp * P))]
+        allowed = allowed & col[None, :]
+        Or, Lr = textbook_attention(s["Q"], s["K"], s["V"], allowed)
+        np.testing.assert_allclose(O[t:t + q_len], Or, atol=1e-12)
+        fin = np.isfinite(Lr)
+        assert np.array_equal(np.isfinite(L[t:t + q_len]), fin)
+        np.testing.assert_allclose(L[t:t + q_len][fin], Lr[fin], atol=1e-12)
+        t += q_len
+    # hidden page == omitted page, for a decode whose hidden page is a full, earlier one
+    seq = random_seqs(rng, [(1, 5 * P)], H_q, H_kv, D)[0]
+    a = SmallBatch([seq], H_q).paged(P, "random", seed=3)
+    hidden = int(a["page_indices"][2])
+    O_h, L_h = orc.forward(**a, page_masks={hidden: np.zeros(P, bool)})
+    keep = np.ones(5 * P, bool)
+    keep[2 * P:3 * P] = False
+    short = dict(Q=seq["Q"], K=seq["K"][keep], V=seq["V"][keep])
+    O_o, L_o = oracle_on(SmallBatch([short], H_q).paged(P, "random", seed=4))
+    np.testing.assert_allclose(O_h, O_o, atol=1e-14)
+    np.testing.assert_allclose(L_h, L_o, atol=1e-14)

@@ -135,3 +135,44 @@ def test_plan_arrays_match_numpy(name):
         assert np.array_equal((got[:, 1] < 0), needs[keep])
         koff += n
     assert koff == info["kept_pages"] and woff == info["mask_words"]
+
+
+def test_mask_kvpage_is_anded_into_packed_rows_and_drops_hidden_pages():
+    wl = configs.small("mixed_prefill_decode")
+    ctx = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+    try:
+        pie.pie_alloc_kvpages(ctx, wl.num_pages)
+        rng = np.random.RandomState(5)
+        r = 4                                             # a decode request with several pages
+        pages = wl.pages_of(r)
+        pm = {int(pages[0]): 0x0000, int(pages[1]): 0x0F0F, int(pages[2]): 0xFFFF}
+        pie.pie_mask_kvpage(ctx, list(pm), list(pm.values()))
+        assert status_of(pie.pie_mask_kvpage, ctx, [wl.num_pages + 5], [1]) == pie.PIE_ERR_BAD_PAGE
+        plan = pie.pie_plan_forward(ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len)
+        words = pie.pie_plan_debug_read(plan, 0)
+        kept = pie.pie_plan_debug_read(plan, 1).reshape(-1, 2)
+        pie.pie_plan_destroy(plan)
+        kv, ql, P = int(wl.kv_lens()[r]), int(wl.q_lens()[r]), wl.P
+        assert ql == 1
+        rw = ((kv + 127) // 128) * 4
+        assert len(words) == rw                           # only the page-masked request got packed rows
+        exp = np.zeros(rw * 32, np.uint8)
+        exp[:kv] = 1                                      # inferred causal row of a decode: everything
+        exp[0:P] = 0
+        exp[P:2 * P] = [(0x0F0F >> s) & 1 for s in range(P)]
+        assert np.array_equal(words, np.packbits(exp, bitorder="little").view(np.uint32))
+        k0 = int(np.sum(np.diff(wl.page_indptr)[:r]))     # earlier requests keep all their pages
+        mine = kept[k0:k0 + len(pages) - 1]
+        assert np.array_equal(mine[:, 0], pages[1:])      # the fully hidden first page is dropped
+        assert mine[0, 1] < 0 and mine[1, 1] >= 0         # partially hidden page needs mask bits, visible one not
+        # re-allocating a page resets its mask
+        pie.pie_dealloc_kvpages(ctx, [pages[1]])
+        again = pie.pie_alloc_kvpages(ctx, 1)
+        assert again[0] == pages[1]
+        plan = pie.pie_plan_forward(ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len)
+        w2 = pie.pie_plan_debug_read(plan, 0)
+        pie.pie_plan_destroy(plan)
+        exp[P:2 * P] = 1
+        assert np.array_equal(w2, np.packbits(exp, bitorder="little").view(np.uint32))
+    finally:
+        pie.pie_destroy(ctx)
