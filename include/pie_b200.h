@@ -161,7 +161,9 @@ typedef struct pie_plan_info {
  * splits the work across SMs, and uploads the result.  Errors: PIE_ERR_BAD_PAGE (id out of
  * range / not allocated), PIE_ERR_INVALID (last_page_len outside [1,page_size], q_len < 1,
  * kv_len < q_len, non-monotone indptr), PIE_ERR_CONFLICT (two requests append to the same
- * slot, or one reads a slot another one writes: the vertical-batching rule of Section 5.2),
+ * slot, or a request reads a slot that a LATER request of the batch appends: the
+ * vertical-batching rule of Section 5.2; reading rows an EARLIER request appends is legal,
+ * because the whole batch is appended before any request attends),
  * PIE_ERR_BATCH_TOO_LARGE, PIE_ERR_MASK.  *out is set only on success.  The upload uses
  * `stream`; the call returns after it completed. */
 int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pie_plan** out);
@@ -222,6 +224,36 @@ enum { PIE_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 };
 int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* batch, const void* q,
                                const void* k_new, const void* v_new, void* out, float* lse,
                                void* stream);
+
+/* ---- Batch scheduler of the control layer (Section 5.2 "Batch scheduler", Section 6.1) ------------
+ * Host-only bookkeeping that decides WHICH pending calls form the next batch; it does not touch
+ * the device.  Calls are submitted to command queues (Section 4.1 "Command queue": order inside a
+ * queue is dependency order; queues carry a priority).  pie_sched_next_batch - to be called the
+ * moment the GPU reports idle (work-conserving dispatch) - forms one batch:
+ *   1. API type: the one whose oldest eligible call has waited longest (eligible = the run of
+ *      consecutive same-type calls at the head of a queue);
+ *   2. vertical batching: a queue contributes its head run, in order, up to (not including) the
+ *      first call that writes a KvPage already written by a call of this batch;
+ *   3. horizontal batching: all queues whose head call has that type take part, higher priority
+ *      first (ties: lower queue id), so that
+ *   4. the batch is cut from the tail at min(max_batch_calls, cap).
+ * Chosen calls leave their queues; tags (caller's handles) come back in batch order, with their
+ * queue ids if out_queues != NULL.  *out_n = 0 and *out_type = -1 when nothing is pending.
+ * Types are small integers chosen by the caller (< PIE_SCHED_MAX_TYPES); write_pages lists the
+ * KvPages a call writes (forward: its output pages; copy_kvpage: its destinations).  A request
+ * reading rows that an EARLIER call of the same batch appends is not a conflict: pie_forward
+ * appends the whole batch before attending (the two-call split of Section 4.2 runs as one batch). */
+enum { PIE_SCHED_MAX_TYPES = 16 };
+typedef struct pie_sched pie_sched;
+int pie_sched_create(int32_t max_batch_calls, pie_sched** out);
+int pie_sched_destroy(pie_sched* s);
+int pie_sched_create_queue(pie_sched* s, int32_t priority, int32_t* out_queue);
+int pie_sched_set_queue_priority(pie_sched* s, int32_t queue, int32_t priority);
+int pie_sched_submit(pie_sched* s, int32_t queue, int32_t type, int32_t n_write, const int32_t* write_pages,
+                     int64_t arrival_ns, int64_t tag);
+int pie_sched_pending(const pie_sched* s, int32_t* out);
+int pie_sched_next_batch(pie_sched* s, int32_t* out_type, int32_t cap, int64_t* out_tags, int32_t* out_queues,
+                         int32_t* out_n);
 
 /* Tuning knobs (all optional; 0 restores the default).  They affect plans made afterwards.
  *   PIE_OPT_SPLIT_SMS  SMs the split-KV decode kernel may use (default: all).

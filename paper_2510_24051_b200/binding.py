@@ -72,6 +72,13 @@ def _load():
         "pie_get_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int)]),
         "pie_forward_static_scratch": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
         "pie_set_option": (C.c_int, [vp, C.c_int, C.c_int]),
+        "pie_sched_create": (C.c_int, [i32, C.POINTER(vp)]),
+        "pie_sched_destroy": (C.c_int, [vp]),
+        "pie_sched_create_queue": (C.c_int, [vp, i32, C.POINTER(i32)]),
+        "pie_sched_set_queue_priority": (C.c_int, [vp, i32, i32]),
+        "pie_sched_submit": (C.c_int, [vp, i32, i32, i32, vp, C.c_int64, C.c_int64]),
+        "pie_sched_pending": (C.c_int, [vp, C.POINTER(i32)]),
+        "pie_sched_next_batch": (C.c_int, [vp, C.POINTER(i32), i32, vp, vp, C.POINTER(i32)]),
         "pie_set_kernel_timing": (C.c_int, [vp, C.c_int]),
         "pie_get_kernel_times": (C.c_int, [vp, vp, vp]),
     }
@@ -273,3 +280,45 @@ def pie_mask_kvpage(ctx, ids, masks):
     m = np.ascontiguousarray(masks, dtype=np.uint32)
     assert len(m) == len(ids)
     _check(lib.pie_mask_kvpage(ctx, len(ids), ids.ctypes.data, m.ctypes.data), ctx)
+
+
+# ------------------------------------------------------------------ batch scheduler (host only)
+def pie_sched_create(max_batch_calls):
+    s = C.c_void_p()
+    _check(lib.pie_sched_create(max_batch_calls, C.byref(s)))
+    return s
+
+
+def pie_sched_destroy(s):
+    _check(lib.pie_sched_destroy(s))
+
+
+def pie_sched_create_queue(s, priority=0):
+    q = C.c_int32()
+    _check(lib.pie_sched_create_queue(s, priority, C.byref(q)))
+    return q.value
+
+
+def pie_sched_set_queue_priority(s, queue, priority):
+    _check(lib.pie_sched_set_queue_priority(s, queue, priority))
+
+
+def pie_sched_submit(s, queue, call_type, write_pages, arrival_ns, tag):
+    w = _i32(write_pages)
+    _check(lib.pie_sched_submit(s, queue, call_type, len(w), w.ctypes.data, arrival_ns, tag))
+
+
+def pie_sched_pending(s):
+    n = C.c_int32()
+    _check(lib.pie_sched_pending(s, C.byref(n)))
+    return n.value
+
+
+def pie_sched_next_batch(s, cap=1 << 20):
+    """(type, [tags], [queue ids]) of the next batch; (-1, [], []) when nothing is pending."""
+    cap = min(cap, 1 << 20)
+    tags = np.zeros(cap, dtype=np.int64)
+    qs = np.zeros(cap, dtype=np.int32)
+    t, n = C.c_int32(), C.c_int32()
+    _check(lib.pie_sched_next_batch(s, C.byref(t), cap, tags.ctypes.data, qs.ctypes.data, C.byref(n)))
+    return t.value, tags[:n.value].tolist(), qs[:n.value].tolist()

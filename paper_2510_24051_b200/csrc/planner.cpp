@@ -243,9 +243,12 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     q.last_page_len = last;
   }
 
-  // ---- conflict rule: no slot is written twice, and no request reads a slot another writes
+  // ---- conflict rule: no slot is written twice, and no request reads a slot that a later request
+  // of the batch writes (rows appended by an earlier request are visible: append precedes attention)
   {
     std::vector<int32_t> touched;
+    struct SharedWrite { int32_t page, req; uint32_t mask; };
+    std::vector<SharedWrite> shared;  // pages written by more than one request: who wrote which slots
     int status = PIE_OK;
     auto slot_mask = [&](int lo, int hi) -> uint32_t {  // bits [lo, hi)
       uint32_t m = (hi >= 32) ? 0xFFFFFFFFu : ((1u << hi) - 1u);
@@ -260,8 +263,16 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
         uint32_t m = slot_mask(lo, hi);
         int32_t pg = pages[lp];
         if (ctx->wmask[pg] & m) { status = PIE_ERR_CONFLICT; break; }
-        if (ctx->wmask[pg] == 0) { touched.push_back(pg); ctx->writer[pg] = r; }
-        else if (ctx->writer[pg] != r) ctx->writer[pg] = -2;
+        if (ctx->wmask[pg] == 0) {
+          touched.push_back(pg);
+          ctx->writer[pg] = r;
+        } else {
+          if (ctx->writer[pg] >= 0) {  // second writer of this page: start the per-writer record
+            shared.push_back(SharedWrite{pg, ctx->writer[pg], ctx->wmask[pg]});
+            ctx->writer[pg] = -2;
+          }
+          shared.push_back(SharedWrite{pg, r, m});
+        }
         ctx->wmask[pg] |= m;
       }
     }
@@ -272,7 +283,13 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
         int32_t pg = pages[lp];
         uint32_t w = ctx->wmask[pg];
         if (w == 0 || ctx->writer[pg] == r) continue;
+        if (ctx->writer[pg] >= 0 && ctx->writer[pg] < r) continue;  // written by an earlier request: visible
         uint32_t rd = slot_mask(0, lp == q.last_logical ? q.last_page_len : P);
+        if (ctx->writer[pg] == -2) {  // several writers: only slots written by LATER requests conflict
+          w = 0;
+          for (const SharedWrite& sw : shared)
+            if (sw.page == pg && sw.req > r) w |= sw.mask;
+        }
         if (w & rd) { status = PIE_ERR_CONFLICT; break; }
       }
     }

@@ -161,3 +161,37 @@ def test_mask_kvpage_matches_oracle(name, flags):
         out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
         pie.pie_plan_destroy(plan)
         check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype)
+
+
+def test_split_forward_batched_together_equals_one_prefill():
+    """Section 4.2: `forward([], iemb[:-1], kv)` and `forward(kv, iemb[-1:], oemb)` may be batched
+    together (vertical batching).  As ONE batch - request 0 fills the pages, request 1 lists the same
+    pages and reads the rows request 0 appends - the outputs equal a single 9-token prefill."""
+    import paper_2510_24051_b200 as pie
+    from oracle import pie_oracle as orc
+    from tests._gpu import TOL_LSE, TOL_O
+    n, P, H_q, H_kv, D = 41, 16, 8, 2, 128
+    g = torch.Generator().manual_seed(5)
+    q = torch.randn(n, H_q, D, generator=g).to(torch.bfloat16)
+    k = torch.randn(n, H_kv, D, generator=g).to(torch.bfloat16)
+    v = torch.randn(n, H_kv, D, generator=g).to(torch.bfloat16)
+    ctx = pie.pie_create(16, P, H_q, H_kv, D, "bf16", 4, 64, 0)
+    try:
+        ids = pie.pie_alloc_kvpages(ctx, 8)
+        pages = ids[[5, 2, 7]]
+        # oracle: one prefill of n tokens into empty pages
+        pool = {int(p): (np.zeros((P, H_kv, D), np.uint16), np.zeros((P, H_kv, D), np.uint16)) for p in pages}
+        O_ref, L_ref = orc.forward(pool, P, H_q, np.array([0, n]), np.array([0, 3]), pages, np.array([n - 2 * P]),
+                                   bits(q), bits(k), bits(v))
+        # GPU: request 0 = first n-1 tokens (writes them), request 1 = last token, same page list
+        plan = pie.pie_plan_forward(ctx, [0, n - 1, n], [0, 3, 6], np.concatenate([pages, pages]),
+                                    [n - 1 - 2 * P, n - 2 * P])
+        out = torch.empty((n, H_q, D), dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty((n, H_q), dtype=torch.float32, device="cuda")
+        pie.pie_forward(ctx, plan, q.cuda(), k.cuda(), v.cuda(), out, lse)
+        torch.cuda.synchronize()
+        pie.pie_plan_destroy(plan)
+        assert (out.double().cpu().numpy() - O_ref).__abs__().max() <= TOL_O["bf16"]
+        assert np.abs(lse.double().cpu().numpy() - L_ref).max() <= TOL_LSE
+    finally:
+        pie.pie_destroy(ctx)

@@ -68,14 +68,18 @@ def test_conflict_rule(ctx):
     # two requests append into the same slot of a shared last page
     assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 2, 4], page_indices=[ids[0], ids[1], ids[2], ids[1]],
                 last_page_len=[4, 4]) == pie.PIE_ERR_CONFLICT
-    # request 1 reads (as context) a slot request 0 writes
+    # request 1 reads (as context) a slot the EARLIER request 0 appends: legal, the whole batch is
+    # appended before anyone attends (the split forward of Section 4.2 as one batch) ...
     assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 1, 3], page_indices=[ids[0], ids[0], ids[2]],
+                last_page_len=[4, 4]) == pie.PIE_OK
+    # ... but reading a slot that a LATER request of the batch appends is a conflict
+    assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 2, 3], page_indices=[ids[0], ids[2], ids[0]],
                 last_page_len=[4, 4]) == pie.PIE_ERR_CONFLICT
     # sharing read-only pages is legal; so is reading slots below the other request's write
     assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 2, 4], page_indices=[ids[0], ids[1], ids[0], ids[2]],
                 last_page_len=[4, 4]) == pie.PIE_OK
     assert plan(qo_indptr=[0, 1, 2], page_indptr=[0, 1, 3], page_indices=[ids[0], ids[3], ids[0]],
-                last_page_len=[9, 3]) == pie.PIE_ERR_CONFLICT   # req 1 appends slot 2, req 0 reads slots 0..8
+                last_page_len=[9, 3]) == pie.PIE_ERR_CONFLICT   # req 1 appends slot 2, the earlier req 0 reads slots 0..8
     # a request that lists the same page twice and would write it through both positions
     assert plan(qo_indptr=[0, 20], page_indptr=[0, 2], page_indices=[ids[4], ids[4]],
                 last_page_len=[16]) == pie.PIE_ERR_CONFLICT
