@@ -14,6 +14,8 @@ namespace {
 __global__ void append_kernel(uint8_t* __restrict__ pool, const uint8_t* __restrict__ k_new,
                               const uint8_t* __restrict__ v_new, const int32_t* __restrict__ append_dst,
                               int T, PoolGeom g) {
+  pie_pdl_launch_dependents();
+  pie_pdl_wait();
   const int chunks = g.row_bytes >> 4;
   const int64_t per_tok = (int64_t)2 * g.n_kv_heads * chunks;
   const int64_t total = (int64_t)T * per_tok;
@@ -34,6 +36,8 @@ __global__ void append_kernel(uint8_t* __restrict__ pool, const uint8_t* __restr
 
 // K2: copy_kvpage (Table 1).  ops[k] = {src, dst, src_off, dst_off, ntok}; one block per op.
 __global__ void copy_kernel(uint8_t* __restrict__ pool, const int32_t* __restrict__ ops, PoolGeom g) {
+  pie_pdl_launch_dependents();
+  pie_pdl_wait();
   const int32_t* op = ops + blockIdx.x * 5;
   const int src = op[0], dst = op[1], so = op[2], dof = op[3], n = op[4];
   const int chunks = g.row_bytes >> 4;
@@ -192,15 +196,13 @@ int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, con
   if (plan->T == 0) return PIE_OK;
   const PoolGeom& g = ctx->geom;
   int64_t work = (int64_t)plan->T * 2 * g.n_kv_heads * (g.row_bytes >> 4);
-  append_kernel<<<grid_for(work, 256, ctx->n_sms), 256, 0, s>>>(ctx->pool, (const uint8_t*)k_new, (const uint8_t*)v_new,
-                                                                 plan->d_append_dst, plan->T, g);
-  PIE_CUDA(ctx, cudaGetLastError());
+  PIE_CUDA(ctx, pie_launch_pdl(append_kernel, dim3(grid_for(work, 256, ctx->n_sms)), dim3(256), 0, s, ctx->pool,
+                               (const uint8_t*)k_new, (const uint8_t*)v_new, (const int32_t*)plan->d_append_dst, plan->T, g));
   return PIE_OK;
 }
 
 int pie_launch_copy(pie_ctx* ctx, int n, const int32_t* d_ops, cudaStream_t s) {
-  copy_kernel<<<n, 256, 0, s>>>(ctx->pool, d_ops, ctx->geom);
-  PIE_CUDA(ctx, cudaGetLastError());
+  PIE_CUDA(ctx, pie_launch_pdl(copy_kernel, dim3(n), dim3(256), 0, s, ctx->pool, d_ops, ctx->geom));
   return PIE_OK;
 }
 

@@ -335,11 +335,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + NW * DEPTH * C::STAGE) + warp * DEPTH;
   volatile uint32_t* meta = reinterpret_cast<uint32_t*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 8) + warp * DEPTH;
   volatile int* queue = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 12) + warp * C::QUEUE;
+  pie_pdl_launch_dependents();
   if (lane == 0) {
     for (int s = 0; s < DEPTH; ++s) mbar_init(smem_u32(full_bar + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
+  pie_pdl_wait();  // the append (and whatever produced Q) must be complete before the first copy / Q load
 
   // ---- prefetch side: a cursor DEPTH page visits ahead of the consumer
   int q_head = 0, q_tail = 0;                       // queue of chunk ids, pushed here, popped by the consumer
@@ -503,7 +505,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) attn_tile_kernel(const AttnP
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  pie_pdl_launch_dependents();
   __syncthreads();
+  pie_pdl_wait();
 
   const int it0 = p.cta_ptr[blockIdx.x], it1 = p.cta_ptr[blockIdx.x + 1];
 
@@ -566,6 +570,8 @@ __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* 
   // lane owns D/32 consecutive columns and the slot loop issues independent, coalesced row loads.
   // (Every partial row is written by its kernel, with zeros when its part of the context was empty.)
   constexpr int EPL = D / 32;
+  pie_pdl_launch_dependents();
+  pie_pdl_wait();
   const PieMerge mg = merges[blockIdx.x];
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -624,6 +630,8 @@ __global__ void simple_kernel(const uint8_t* __restrict__ pool, const T* __restr
                               const int32_t* __restrict__ tok_req, const int32_t* __restrict__ rows, int n_rows,
                               PoolGeom g, int n_q_heads, int G, float scale) {
   constexpr int EPL = D / 32;  // elements per lane
+  pie_pdl_launch_dependents();
+  pie_pdl_wait();
   const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (wid >= n_rows) return;
   const int row = rows[wid];
@@ -707,8 +715,7 @@ int launch_split(pie_ctx* ctx, const AttnParams& p, int n_items, int n_warps, cu
     configured[dev] = true;
   }
   const int blocks = (n_warps + NW - 1) / NW;
-  kern<<<blocks, NW * 32, C::SMEM, s>>>(p, n_items, blocks * NW);
-  PIE_CUDA(ctx, cudaGetLastError());
+  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(blocks), dim3(NW * 32), C::SMEM, s, p, n_items, blocks * NW));
   return PIE_OK;
 }
 
@@ -723,8 +730,7 @@ int launch_tiles(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
     configured[dev] = true;
   }
-  kern<<<grid, (NW + 1) * 32, C::SMEM, s>>>(p);
-  PIE_CUDA(ctx, cudaGetLastError());
+  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3((NW + 1) * 32), C::SMEM, s, p));
   return PIE_OK;
 }
 
@@ -768,8 +774,9 @@ int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll
   const int wpb = ll.slot_rows >= 8 ? 8 : 4;  // warps (= rows) per block
   const dim3 n((unsigned)ll.merges.size(), (unsigned)((ll.slot_rows + wpb - 1) / wpb));
 #define PIE_MERGE(T, DD)                                                                                          \
-  merge_kernel<T, DD><<<n, wpb * 32, 0, s>>>(ll.d_merges, plan->d_reqs, ll.d_ws_o, ll.d_ws_lse, (T*)out, lse, \
-                                             ll.slot_rows, ctx->cfg.num_q_heads, ctx->G)
+  PIE_CUDA(ctx, pie_launch_pdl(merge_kernel<T, DD>, n, dim3(wpb * 32), 0, s, (const PieMerge*)ll.d_merges,      \
+                               (const PieReq*)plan->d_reqs, (const float*)ll.d_ws_o, (const float*)ll.d_ws_lse, \
+                               (T*)out, lse, ll.slot_rows, ctx->cfg.num_q_heads, ctx->G))
   if (ctx->cfg.dtype == PIE_DTYPE_BF16) {
     if (D == 64) PIE_MERGE(__nv_bfloat16, 64);
     else PIE_MERGE(__nv_bfloat16, 128);
@@ -788,9 +795,10 @@ int pie_launch_simple(pie_ctx* ctx, const pie_plan* plan, const void* q, void* o
   const float scale = 1.f / sqrtf((float)D);
   const int threads = 128, grid = (n * 32 + threads - 1) / threads;
 #define PIE_SIMPLE(T, DD)                                                                                              \
-  simple_kernel<T, DD><<<grid, threads, 0, s>>>(ctx->pool, (const T*)q, (T*)out, lse, plan->d_reqs, plan->d_kept,      \
-                                                plan->d_mask, plan->d_tok_req, plan->d_simple_rows, n, ctx->geom,      \
-                                                ctx->cfg.num_q_heads, ctx->G, scale)
+  PIE_CUDA(ctx, pie_launch_pdl(simple_kernel<T, DD>, dim3(grid), dim3(threads), 0, s, (const uint8_t*)ctx->pool,     \
+                               (const T*)q, (T*)out, lse, (const PieReq*)plan->d_reqs, (const int2*)plan->d_kept,     \
+                               (const uint32_t*)plan->d_mask, (const int32_t*)plan->d_tok_req,                         \
+                               (const int32_t*)plan->d_simple_rows, n, ctx->geom, ctx->cfg.num_q_heads, ctx->G, scale))
   if (ctx->cfg.dtype == PIE_DTYPE_BF16) {
     if (D == 64) PIE_SIMPLE(__nv_bfloat16, 64);
     else PIE_SIMPLE(__nv_bfloat16, 128);

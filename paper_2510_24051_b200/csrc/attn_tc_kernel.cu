@@ -234,10 +234,12 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  pie_pdl_launch_dependents();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pie_pdl_wait();  // the append (and whatever produced Q) is complete from here on
 
   const int it0 = p.cta_ptr[blockIdx.x], it1 = p.cta_ptr[blockIdx.x + 1];
 
@@ -590,8 +592,7 @@ static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
     configured[dev] = true;
   }
-  kern<<<grid, 384, C::SMEM, s>>>(p);
-  PIE_CUDA(ctx, cudaGetLastError());
+  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3(384), C::SMEM, s, p));
   return PIE_OK;
 }
 

@@ -188,3 +188,28 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);  // h
       return PIE_ERR_CUDA;                                    \
     }                                                         \
   } while (0)
+
+// Programmatic dependent launch: every kernel of the path is launched with the stream-serialisation
+// attribute, lets its successor start launching at once (pie_pdl_launch_dependents) and waits for its
+// predecessor's results only where it first needs them (pie_pdl_wait), so launch latencies and
+// prologues overlap the previous kernel's tail.  pie_pdl_wait returns once every earlier grid of the
+// stream has completed and its writes are visible.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pie_pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pie_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t pie_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
