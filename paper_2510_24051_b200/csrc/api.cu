@@ -168,7 +168,10 @@ void plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
     cp(L.items[k], lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
     cp(L.cta[k], lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
     cp(L.merges[k], lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
-    std::memset(dst + L.ctr[k], 0, 8);  // work counters start at zero; the kernel re-arms them itself
+    {
+      const int32_t ctr0[2] = {lls[k]->n_static, 0};  // next dynamic item, finished warps; the kernel re-arms them
+      std::memcpy(dst + L.ctr[k], ctr0, 8);
+    }
   }
 }
 

@@ -350,17 +350,17 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   int grabbed = 0;                                  // lane 0: result of an atomic whose value is not needed yet
   bool grab_pending = false, exhausted = false, pf_live = true;
 
-  // Small launches use fixed shares instead (cta_ptr != nullptr): warp w owns items
-  // [cta_ptr[w], cta_ptr[w+1]) and "taking" is just counting through them.
-  const bool fixed_shares = p.cta_ptr != nullptr;
+  // Short launches give every warp a fixed share first (cta_ptr != nullptr: warp w owns items
+  // [cta_ptr[w], cta_ptr[w+1])) and leave only the last part of the work, cut into small chunks
+  // [n_static, n_items), to the counter: few pieces and partials, yet no SM is left waiting at the end.
   const int wg = blockIdx.x * NW + warp;
   int own_next = 0, own_end = 0;
-  if (fixed_shares && wg < p.n_shares) {
+  if (p.cta_ptr != nullptr && wg < p.n_shares) {
     own_next = p.cta_ptr[wg];
     own_end = p.cta_ptr[wg + 1];
   }
   auto take = [&]() {  // synchronous: next chunk id for this warp
-    if (fixed_shares) return own_next < own_end ? own_next++ : n_items;
+    if (own_next < own_end) return own_next++;
     int v = 0;
     if (lane == 0) v = atomicAdd(p.work_ctr, 1);
     return __shfl_sync(0xFFFFFFFFu, v, 0);
@@ -402,7 +402,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
     const int left = pf_end - pf_k;
     if (!grab_pending) {
       if (left <= 4) {
-        if (fixed_shares) grabbed = own_next < own_end ? own_next++ : n_items;
+        if (own_next < own_end) grabbed = own_next++;
         else if (lane == 0) grabbed = atomicAdd(p.work_ctr, 1);
         grab_pending = true;
       }
@@ -469,10 +469,10 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   }
 
   // ---- the last warp of the grid to finish re-arms the counters for the next launch
-  if (lane == 0 && !fixed_shares) {
+  if (lane == 0) {
     __threadfence();
     if (atomicAdd(p.work_ctr + 1, 1) == n_warps - 1) {
-      p.work_ctr[0] = 0;
+      p.work_ctr[0] = p.n_static;
       p.work_ctr[1] = 0;
     }
   }
@@ -691,6 +691,7 @@ AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& 
   p.items = ll.d_items;
   p.cta_ptr = ll.cta_ptr.empty() ? nullptr : ll.d_cta_ptr;
   p.n_shares = ll.cta_ptr.empty() ? 0 : (int)ll.cta_ptr.size() - 1;
+  p.n_static = ll.n_static;
   p.work_ctr = ll.d_work_ctr;
   p.slot_rows = ll.slot_rows;
   p.ws_o = ll.d_ws_o;
@@ -860,11 +861,13 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   const size_t o_simple = put(plan.simple_rows.data(), plan.simple_rows.size() * 4);
   PieLaunchList* lls[2] = {&plan.split, &plan.tile};
   size_t o_li[2], o_lc[2], o_lm[2], o_wo[2], o_wl[2], o_ctr[2];
-  const int32_t zero_ctr[2] = {0, 0};  // work counters of the split-KV kernel start at zero
   for (int k = 0; k < 2; ++k) {
     o_li[k] = put(lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
     o_lc[k] = put(lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
-    o_ctr[k] = put(zero_ctr, sizeof(zero_ctr));
+    {
+      const int32_t ctr0[2] = {lls[k]->n_static, 0};  // the dynamic part of the item list starts here
+      o_ctr[k] = put(ctr0, sizeof(ctr0));
+    }
     o_lm[k] = put(lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
   }
   size_t total = (host.size() + 255) & ~(size_t)255;

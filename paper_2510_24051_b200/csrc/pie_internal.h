@@ -74,6 +74,7 @@ struct PieLaunchList {           // one tile-kernel launch (split-KV decode, or 
   int32_t grid = 0;
   int32_t n_slots = 0;
   int32_t slot_rows = 0;
+  int32_t n_static = 0;          // split-KV: items [n_static, size) are taken from the work counter
   // device copies
   PieItem* d_items = nullptr;
   int32_t* d_cta_ptr = nullptr;
@@ -157,6 +158,7 @@ struct AttnParams {
   const int32_t* cta_ptr;
   int32_t* work_ctr;
   int32_t n_shares;   // split-KV kernel with fixed shares: entries of cta_ptr minus one
+  int32_t n_static;   // first item that is taken dynamically (items before it belong to fixed shares)
   int32_t slot_rows;
   float* ws_o;
   float* ws_lse;

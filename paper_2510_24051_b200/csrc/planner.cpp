@@ -65,6 +65,7 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
   ll.n_slots = 0;
   ll.slot_rows = slot_rows;
   ll.grid = 0;
+  ll.n_static = 0;
   if (units.empty()) return;
   int64_t W = 0, max_unit = 0;
   for (const Unit& u : units) {
@@ -161,6 +162,7 @@ void chunk_units(const std::vector<Unit>& units, int n_warps, PieLaunchList& ll)
   ll.n_slots = 0;
   ll.slot_rows = 1;
   ll.grid = 0;
+  ll.n_static = 0;
   if (units.empty()) return;
   int64_t W = 0;
   for (const Unit& u : units) {
@@ -491,7 +493,10 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     if (W >= (int64_t)200 * n_warps) {
       chunk_units(split_units, n_warps, plan->split);
     } else {
+      // fixed equal shares, nothing left to the counter (a dynamic tail of small chunks was measured:
+      // the extra partials cost more in the merge than the better balance gains on a 50 us launch)
       partition(split_units, n_warps, 4, max_rows, false, plan->split);
+      plan->split.n_static = (int32_t)plan->split.items.size();
     }
   }
   partition(tile_units, tile_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile);
