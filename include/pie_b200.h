@@ -59,6 +59,13 @@ typedef struct pie_config {
   int32_t device;           /* CUDA device ordinal; -1 = host-only context (planner,
                                allocator and validation work; device calls return
                                PIE_ERR_NO_DEVICE)                                      */
+  float rope_theta;         /* 0: Q / K arrive position-encoded (default).  > 0: rotary
+                               position embedding inside the path with this base (Llama-3:
+                               500000): forward rotates Q for the attention and rotates each
+                               new K row before storing it, at the token's position
+                               (rotate-half form: pairs (i, i + D/2), angle pos * theta^(-2i/D)).
+                               `forward` "operates based on explicit sequence positions"
+                               (Section 4.2); the paper gives no formula.               */
 } pie_config;
 
 typedef struct pie_ctx pie_ctx;
@@ -135,6 +142,9 @@ typedef struct pie_batch_desc {
   const int64_t* mask_indptr;   /* [R+1] or NULL                                  */
   const uint8_t* mask;          /* [mask_indptr[R]] or NULL                       */
   uint32_t flags;               /* PIE_PLAN_* below, 0 for the default path       */
+  const int32_t* positions;     /* [T] explicit position of every new token, or NULL for the
+                                   default kv_len - q_len + i.  Used only when the context
+                                   was created with rope_theta > 0.                 */
 } pie_batch_desc;
 
 enum {

@@ -53,6 +53,48 @@ def kv_len_of(num_pages_r: int, last_page_len_r: int, P: int) -> int:
     return (num_pages_r - 1) * P + last_page_len_r
 
 
+# --------------------------------------------------------------------------- positions (RoPE)
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary position embedding in the rotate-half form used by the Llama family: for i < D/2,
+    with angle a = pos * theta**(-2i/D),
+        y[i]       = x[i] cos a - x[i + D/2] sin a
+        y[i + D/2] = x[i + D/2] cos a + x[i] sin a.
+    x [T, H, D] fp64, pos [T] integers.  (`forward` "operates based on explicit sequence positions",
+    Section 4.2; the paper gives no formula, this is the reading built here.)"""
+    T, H, D = x.shape
+    half = D // 2
+    inv_freq = theta ** (-2.0 * np.arange(half, dtype=np.float64) / D)
+    ang = np.asarray(pos, dtype=np.float64)[:, None] * inv_freq[None, :]          # [T, D/2]
+    c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    y = np.empty_like(x)
+    y[..., :half] = x[..., :half] * c - x[..., half:] * s
+    y[..., half:] = x[..., half:] * c + x[..., :half] * s
+    return y
+
+
+def to_storage(x64: np.ndarray, like: np.ndarray) -> np.ndarray:
+    """Round fp64 values to the storage type of `like` (fp32, or bf16 bit patterns, both round to
+    nearest even; bf16 goes through fp32)."""
+    if like.dtype == np.float64:   # fp64 storage (pins only): nothing to round
+        return x64
+    f32 = x64.astype(np.float32)
+    if like.dtype == np.uint16:
+        u = f32.view(np.uint32)
+        return ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+    return f32.astype(like.dtype)
+
+
+def default_positions(qo_indptr, page_indptr, last_page_len, P) -> np.ndarray:
+    """Position of every new token when none is given: the last q_len positions of its context."""
+    R = len(qo_indptr) - 1
+    pos = np.zeros(int(qo_indptr[R]), dtype=np.int64)
+    for r in range(R):
+        q_len = int(qo_indptr[r + 1] - qo_indptr[r])
+        kv_len = kv_len_of(int(page_indptr[r + 1] - page_indptr[r]), int(last_page_len[r]), P)
+        pos[qo_indptr[r]:qo_indptr[r + 1]] = kv_len - q_len + np.arange(q_len)
+    return pos
+
+
 # --------------------------------------------------------------------------- step 1: append
 def append_kv(pool, P, qo_indptr, page_indptr, page_indices, last_page_len, k_new, v_new):
     """Store the new K/V rows of every request in its pages (Table 1 `forward`, output
@@ -167,7 +209,8 @@ def apply_page_masks(allowed: np.ndarray, pages, P: int, page_masks) -> np.ndarr
 
 
 def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
-            q, k_new, v_new, masks=None, append=True, requests=None, page_masks=None):
+            q, k_new, v_new, masks=None, append=True, requests=None, page_masks=None,
+            rope_theta=None, positions=None):
     """One batched `forward`: append, then gather and attend for every request.
 
     q [T, H_q, D], k_new/v_new [T, H_kv, D] in the storage type; masks is None or a list
@@ -178,6 +221,14 @@ def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
     R = len(qo_indptr) - 1
     T = int(qo_indptr[R])
     D = q.shape[-1]
+    q64 = widen(q)
+    if rope_theta:
+        # positions inside the path: Q is rotated for the attention, K is rotated before it is stored
+        # (the pages hold position-encoded keys)
+        pos = default_positions(qo_indptr, page_indptr, last_page_len, P) if positions is None else np.asarray(positions)
+        # (both rotated operands are values of the element type: the attention consumes bf16 / fp32 Q and K)
+        q64 = widen(to_storage(rope(q64, pos, rope_theta), np.asarray(q)))
+        k_new = to_storage(rope(widen(k_new), pos, rope_theta), k_new)
     if append:
         append_kv(pool, P, qo_indptr, page_indptr, page_indices, last_page_len, k_new, v_new)
     O = np.zeros((T, H_q, D), dtype=np.float64)
@@ -189,7 +240,7 @@ def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
         allowed = allowed_matrix(t1 - t0, kv_len, None if masks is None else masks[r])
         allowed = apply_page_masks(allowed, pages, P, page_masks)
         K, V = gather_kv(pool, P, pages, kv_len, needed=allowed.any(axis=0))
-        O[t0:t1], LSE[t0:t1] = attend(widen(q[t0:t1]), K, V, allowed)
+        O[t0:t1], LSE[t0:t1] = attend(q64[t0:t1], K, V, allowed)
     return O, LSE
 
 

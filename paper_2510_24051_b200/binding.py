@@ -24,13 +24,13 @@ PIE_ERR_UNSUPPORTED, PIE_ERR_DEVICE_TIMEOUT = -9, -10
 class pie_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "num_pages", "page_size", "num_q_heads", "num_kv_heads", "head_dim", "dtype",
-        "max_requests", "max_query_tokens", "device")]
+        "max_requests", "max_query_tokens", "device")] + [("rope_theta", C.c_float)]
 
 
 class pie_batch_desc(C.Structure):
     _fields_ = [("num_requests", C.c_int32), ("qo_indptr", C.c_void_p), ("page_indptr", C.c_void_p),
                 ("page_indices", C.c_void_p), ("last_page_len", C.c_void_p), ("mask_indptr", C.c_void_p),
-                ("mask", C.c_void_p), ("flags", C.c_uint32)]
+                ("mask", C.c_void_p), ("flags", C.c_uint32), ("positions", C.c_void_p)]
 
 
 class pie_plan_info(C.Structure):
@@ -132,10 +132,10 @@ def pie_strerror(status):
 
 
 def pie_create(num_pages, page_size, num_q_heads, num_kv_heads, head_dim, dtype, max_requests,
-               max_query_tokens, device=0):
+               max_query_tokens, device=0, rope_theta=0.0):
     dt = {"bf16": PIE_DTYPE_BF16, "f32": PIE_DTYPE_F32}.get(dtype, dtype)
     cfg = pie_config(num_pages, page_size, num_q_heads, num_kv_heads, head_dim, dt, max_requests,
-                     max_query_tokens, device)
+                     max_query_tokens, device, rope_theta)
     ctx = C.c_void_p()
     _check(lib.pie_create(C.byref(cfg), C.byref(ctx)))
     return ctx
@@ -181,19 +181,20 @@ def pie_copy_kvpage(ctx, src, dst, src_off, dst_off, ntok, stream=None):
     _check(lib.pie_copy_kvpage(ctx, len(a[0]), *[x.ctypes.data for x in a], _stream(stream)), ctx)
 
 
-def _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags):
+def _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions=None):
     keep = [_i32(qo_indptr), _i32(page_indptr), _i32(page_indices), _i32(last_page_len)]
     mi = None if mask_indptr is None else np.ascontiguousarray(mask_indptr, dtype=np.int64)
     mk = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
-    keep += [mi, mk]
+    ps = None if positions is None else _i32(positions)
+    keep += [mi, mk, ps]
     d = pie_batch_desc(len(keep[0]) - 1, keep[0].ctypes.data, keep[1].ctypes.data, keep[2].ctypes.data,
-                       keep[3].ctypes.data, _ptr(mi), _ptr(mk), flags)
+                       keep[3].ctypes.data, _ptr(mi), _ptr(mk), flags, _ptr(ps))
     return d, keep
 
 
 def pie_plan_forward(ctx, qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr=None,
-                     mask=None, flags=0, stream=None):
-    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags)
+                     mask=None, flags=0, stream=None, positions=None):
+    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions)
     plan = C.c_void_p()
     _check(lib.pie_plan_forward(ctx, C.byref(d), _stream(stream), C.byref(plan)), ctx)
     return plan

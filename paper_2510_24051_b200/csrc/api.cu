@@ -1,6 +1,7 @@
 // C ABI entry points, the KvPage allocator, and the bit-exact data-movement kernels
 // (append of new K/V rows, token-level page copy, canonical page import / export).
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <new>
 
@@ -118,7 +119,7 @@ bool page_ok(const pie_ctx* ctx, int32_t id) {
 // Device image of a plan: every array the kernels read, 256-byte aligned, followed by the fp32
 // partial workspaces of the two tile launches.
 struct PlanLayout {
-  size_t reqs, kept, mask, app, tok, simple, items[2], cta[2], merges[2], ctr[2], ws_o[2], ws_lse[2];
+  size_t reqs, kept, mask, app, tok, pos, simple, items[2], cta[2], merges[2], ctr[2], ws_o[2], ws_lse[2];
   size_t upload, total;
 };
 
@@ -135,6 +136,7 @@ PlanLayout plan_layout(const pie_ctx* ctx, const pie_plan* plan) {
   L.mask = place(plan->mask_words.size() * 4);
   L.app = place(plan->append_dst.size() * 4);
   L.tok = place(plan->tok_req.size() * 4);
+  L.pos = place(plan->positions.size() * 4);
   L.simple = place(plan->simple_rows.size() * 4);
   const PieLaunchList* lls[2] = {&plan->split, &plan->tile};
   for (int k = 0; k < 2; ++k) {
@@ -162,6 +164,7 @@ void plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
   cp(L.mask, plan->mask_words.data(), plan->mask_words.size() * 4);
   cp(L.app, plan->append_dst.data(), plan->append_dst.size() * 4);
   cp(L.tok, plan->tok_req.data(), plan->tok_req.size() * 4);
+  cp(L.pos, plan->positions.data(), plan->positions.size() * 4);
   cp(L.simple, plan->simple_rows.data(), plan->simple_rows.size() * 4);
   const PieLaunchList* lls[2] = {&plan->split, &plan->tile};
   for (int k = 0; k < 2; ++k) {
@@ -181,6 +184,7 @@ void plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base) {
   plan->d_mask = (uint32_t*)(base + L.mask);
   plan->d_append_dst = (int32_t*)(base + L.app);
   plan->d_tok_req = (int32_t*)(base + L.tok);
+  plan->d_positions = (int32_t*)(base + L.pos);
   plan->d_simple_rows = (int32_t*)(base + L.simple);
   PieLaunchList* lls[2] = {&plan->split, &plan->tile};
   for (int k = 0; k < 2; ++k) {
@@ -202,6 +206,16 @@ int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, con
   PIE_CUDA(ctx, pie_launch_pdl(append_kernel, dim3(grid_for(work, 256, ctx->n_sms)), dim3(256), 0, s, ctx->pool,
                                (const uint8_t*)k_new, (const uint8_t*)v_new, (const int32_t*)plan->d_append_dst, plan->T, g));
   return PIE_OK;
+}
+
+int pie_append_and_q(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new, const void* v_new, cudaStream_t s,
+                     const void** q_eff) {
+  *q_eff = q;
+  if (ctx->cfg.rope_theta > 0.f) {  // positions inside the path: rotated K goes to the pages, attention reads rotated Q
+    *q_eff = ctx->d_qrot;
+    return pie_launch_rope(ctx, plan, q, k_new, v_new, s);
+  }
+  return pie_launch_append(ctx, plan, k_new, v_new, s);
 }
 
 int pie_launch_copy(pie_ctx* ctx, int n, const int32_t* d_ops, cudaStream_t s) {
@@ -249,6 +263,7 @@ int pie_create(const pie_config* cfg, pie_ctx** out) {
   if (cfg->num_pages < 1 || cfg->num_q_heads < 1 || cfg->num_kv_heads < 1) return PIE_ERR_INVALID;
   if (cfg->num_q_heads % cfg->num_kv_heads) return PIE_ERR_INVALID;
   if (cfg->max_requests < 1 || cfg->max_query_tokens < 1) return PIE_ERR_INVALID;
+  if (!(cfg->rope_theta >= 0.f)) return PIE_ERR_INVALID;
   if ((int64_t)cfg->num_pages * P > 0x7FFFFFFF) return PIE_ERR_INVALID;
   if ((int64_t)cfg->num_pages * cfg->num_kv_heads > 0x7FFFFFFF) return PIE_ERR_INVALID;
   pie_ctx* ctx = new (std::nothrow) pie_ctx();
@@ -278,6 +293,8 @@ int pie_create(const pie_config* cfg, pie_ctx** out) {
       (void)what;
       if (ctx->pool) cudaFree(ctx->pool);
       if (ctx->d_status) cudaFree(ctx->d_status);
+      if (ctx->d_qrot) cudaFree(ctx->d_qrot);
+      if (ctx->d_inv_freq) cudaFree(ctx->d_inv_freq);
       delete ctx;
       return PIE_ERR_CUDA;
     };
@@ -292,6 +309,15 @@ int pie_create(const pie_config* cfg, pie_ctx** out) {
     if ((e = cudaMemset(ctx->pool, 0, bytes)) != cudaSuccess) return fail(e, "memset");
     if ((e = cudaMalloc((void**)&ctx->d_status, 256)) != cudaSuccess) return fail(e, "cudaMalloc status");
     if ((e = cudaMemset(ctx->d_status, 0, 256)) != cudaSuccess) return fail(e, "memset");
+    if (cfg->rope_theta > 0.f) {
+      const size_t qb = (size_t)cfg->max_query_tokens * cfg->num_q_heads * g.row_bytes;
+      std::vector<double> inv((size_t)D / 2);
+      for (int i = 0; i < D / 2; ++i) inv[i] = std::pow((double)cfg->rope_theta, -2.0 * i / D);
+      if ((e = cudaMalloc(&ctx->d_qrot, qb)) != cudaSuccess) return fail(e, "cudaMalloc qrot");
+      if ((e = cudaMalloc((void**)&ctx->d_inv_freq, inv.size() * 8)) != cudaSuccess) return fail(e, "cudaMalloc inv_freq");
+      if ((e = cudaMemcpy(ctx->d_inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice)) != cudaSuccess)
+        return fail(e, "upload inv_freq");
+    }
     if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "sync");
   }
   *out = ctx;
@@ -308,6 +334,8 @@ int pie_destroy(pie_ctx* ctx) {
     if (ctx->d_stage) cudaFree(ctx->d_stage);
     if (ctx->d_io) cudaFree(ctx->d_io);
     if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
+    if (ctx->d_qrot) cudaFree(ctx->d_qrot);
+    if (ctx->d_inv_freq) cudaFree(ctx->d_inv_freq);
     if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
@@ -535,7 +563,8 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
   if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
   cudaStream_t s = (cudaStream_t)stream;
   PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
-  int rc = timed_launch(ctx, PIE_KERNEL_APPEND, s, [&] { return pie_launch_append(ctx, plan, k_new, v_new, s); });
+  const void* q_in = q;
+  int rc = timed_launch(ctx, PIE_KERNEL_APPEND, s, [&] { return pie_append_and_q(ctx, plan, q_in, k_new, v_new, s, &q); });
   if (rc) return rc;
   if (!plan->simple_rows.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_SIMPLE, s, [&] { return pie_launch_simple(ctx, plan, q, out, lse, s); })))

@@ -803,6 +803,7 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   const size_t o_mask = put(plan.mask_words.data(), plan.mask_words.size() * 4);
   const size_t o_app = put(plan.append_dst.data(), plan.append_dst.size() * 4);
   const size_t o_tok = put(plan.tok_req.data(), plan.tok_req.size() * 4);
+  const size_t o_pos = put(plan.positions.data(), plan.positions.size() * 4);
   const size_t o_simple = put(plan.simple_rows.data(), plan.simple_rows.size() * 4);
   PieLaunchList* lls[2] = {&plan.split, &plan.tile};
   size_t o_li[2], o_lc[2], o_lm[2], o_wo[2], o_wl[2], o_ctr[2];
@@ -833,6 +834,7 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   plan.d_mask = (uint32_t*)(base + o_mask);
   plan.d_append_dst = (int32_t*)(base + o_app);
   plan.d_tok_req = (int32_t*)(base + o_tok);
+  plan.d_positions = (int32_t*)(base + o_pos);
   plan.d_simple_rows = (int32_t*)(base + o_simple);
   for (int k = 0; k < 2; ++k) {
     lls[k]->d_items = (PieItem*)(base + o_li[k]);
@@ -842,7 +844,7 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
     lls[k]->d_ws_o = (float*)(base + o_wo[k]);
     lls[k]->d_ws_lse = (float*)(base + o_wl[k]);
   }
-  if ((rc = pie_launch_append(ctx, &plan, k_new, v_new, s))) return rc;
+  if ((rc = pie_append_and_q(ctx, &plan, q, k_new, v_new, s, &q))) return rc;
   if (!plan.simple_rows.empty() && (rc = pie_launch_simple(ctx, &plan, q, out, lse, s))) return rc;
   if (!plan.split.items.empty() && (rc = pie_launch_split(ctx, &plan, q, out, lse, s))) return rc;
   if (!plan.tile.items.empty() && (rc = pie_launch_tiles(ctx, &plan, q, out, lse, s))) return rc;

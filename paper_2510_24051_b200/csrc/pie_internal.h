@@ -94,6 +94,7 @@ struct pie_plan {
   std::vector<uint32_t> mask_words;
   std::vector<int32_t> append_dst;  // [T] page*P + slot
   std::vector<int32_t> tok_req;     // [T]
+  std::vector<int32_t> positions;   // [T] position of every new token (RoPE contexts only)
   std::vector<int32_t> simple_rows; // (token*H_q + head) rows for the plain kernel
   PieLaunchList split, tile;
   bool tile_tc = false;             // row tiles run on the tcgen05 kernel (256-row items)
@@ -106,6 +107,7 @@ struct pie_plan {
   uint32_t* d_mask = nullptr;
   int32_t* d_append_dst = nullptr;
   int32_t* d_tok_req = nullptr;
+  int32_t* d_positions = nullptr;
   int32_t* d_simple_rows = nullptr;
 };
 
@@ -128,6 +130,8 @@ struct pie_ctx {
   size_t stage_bytes = 0;
   void* d_io = nullptr;     // device arena of pie_forward_host: plan image + q/k/v/out/lse
   size_t io_bytes = 0;
+  void* d_qrot = nullptr;        // rotated copy of Q (RoPE contexts): [max_query_tokens][H_q][D]
+  double* d_inv_freq = nullptr;  // [D/2] theta^(-2i/D)
   void* h_stage = nullptr;  // pinned host staging of the plan image (pie_forward_host)
   size_t h_stage_bytes = 0;
   pie_plan* host_plan = nullptr;  // reused plan object of pie_forward_host
@@ -169,6 +173,11 @@ struct AttnParams {
 };
 
 int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, const void* v_new, cudaStream_t s);
+// RoPE contexts: append with rotated K and a rotated copy of Q (rope.cu); *q_eff is what attention reads
+int pie_launch_rope(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new, const void* v_new, cudaStream_t s);
+// append (plain or RoPE) and the Q the attention kernels must read
+int pie_append_and_q(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new, const void* v_new, cudaStream_t s,
+                     const void** q_eff);
 int pie_launch_copy(pie_ctx* ctx, int n, const int32_t* d_ops, cudaStream_t s);
 int pie_launch_page_io(pie_ctx* ctx, int n, const int32_t* d_ids, void* K, void* V, bool write, cudaStream_t s);
 int pie_launch_simple(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);

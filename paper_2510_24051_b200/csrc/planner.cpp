@@ -418,6 +418,8 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   // ---- append destinations
   plan->append_dst.resize(T);
   plan->tok_req.resize(T);
+  plan->positions.clear();
+  if (cfg.rope_theta > 0.f) plan->positions.resize(T);
   for (int r = 0; r < R; ++r) {
     const PieReq& q = plan->reqs[r];
     const int32_t* pages = b->page_indices + b->page_indptr[r];
@@ -425,6 +427,11 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       int pos = q.kv_len - q.q_len + i;
       plan->append_dst[q.q_start + i] = pages[pos / P] * P + pos % P;
       plan->tok_req[q.q_start + i] = r;
+      if (cfg.rope_theta > 0.f) {
+        const int p_i = b->positions ? b->positions[q.q_start + i] : pos;
+        if (p_i < 0) return PIE_ERR_INVALID;
+        plan->positions[q.q_start + i] = p_i;
+      }
     }
   }
 

@@ -195,3 +195,58 @@ def test_split_forward_batched_together_equals_one_prefill():
         assert np.abs(lse.double().cpu().numpy() - L_ref).max() <= TOL_LSE
     finally:
         pie.pie_destroy(ctx)
+
+
+@pytest.mark.parametrize("name", ["tiny_fp32", "batched_decode", "mixed_prefill_decode", "shared_prefix_tree"])
+@pytest.mark.parametrize("explicit_pos", [False, True])
+def test_rope_inside_the_path_matches_oracle(name, explicit_pos):
+    """Contexts created with rope_theta: K rows are rotated before they are stored, Q for the attention;
+    positions default to the last q_len context positions or are given per token."""
+    import paper_2510_24051_b200 as pie
+    from oracle import pie_oracle as orc
+    from tests._gpu import TDTYPE, check_close
+    wl = configs.small(name)
+    theta = 500000.0
+    pos = None
+    if explicit_pos:                                        # e.g. positions continuing after dropped context
+        pos = orc.default_positions(wl.qo_indptr, wl.page_indptr, wl.last_page_len, wl.P) + 12345
+    pool = wl.oracle_pool()
+    O_ref, L_ref = orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                               bits(wl.q()), bits(wl.k_new()), bits(wl.v_new()), wl.masks, rope_theta=theta, positions=pos)
+    ctx = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, 0, rope_theta=theta)
+    try:
+        pie.pie_alloc_kvpages(ctx, wl.num_pages)
+        used = wl.used_pages()
+        K, V = wl.context_pages(used, "cuda")
+        pie.pie_kvpage_write(ctx, used, K.contiguous(), V.contiguous())
+        mi, mb = wl.mask_bytes()
+        plan = pie.pie_plan_forward(ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len, mi, mb,
+                                    positions=pos)
+        q = wl.q("cuda")
+        out = torch.empty_like(q)
+        lse = torch.empty((wl.T, wl.H_q), dtype=torch.float32, device="cuda")
+        pie.pie_forward(ctx, plan, q, wl.k_new("cuda"), wl.v_new("cuda"), out, lse)
+        torch.cuda.synchronize()
+        assert pie.pie_get_last_device_status(ctx) == 0
+        pie.pie_plan_destroy(plan)
+        check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        # stored pages: V bit exact; K (rotated in fp32 on the GPU, fp64 in the oracle) within one unit in the
+        # last place of the storage type, and mostly identical
+        Kg = torch.empty((len(used), wl.P, wl.H_kv, wl.D), dtype=TDTYPE[wl.dtype], device="cuda")
+        Vg = torch.empty_like(Kg)
+        pie.pie_kvpage_read(ctx, used, Kg, Vg)
+        torch.cuda.synchronize()
+        Kg, Vg = bits(Kg), bits(Vg)
+        Ko = np.stack([pool[int(p)][0] for p in used])
+        Vo = np.stack([pool[int(p)][1] for p in used])
+        assert same_bits(Vg, Vo)
+        a, b = orc.widen(Kg), orc.widen(Ko)
+        if wl.dtype == "bf16":     # a rounding flip at most: one unit in the last place of the stored value
+            # (or the fp32 rotation error itself where the two products cancel to almost nothing)
+            bad = np.abs(a - b) > np.maximum(np.abs(b) * 2.0 ** -7, 2e-6)
+            assert not bad.any(), (int(bad.sum()), a[bad][:4], b[bad][:4])
+            assert (a != b).mean() < 0.02
+        else:                      # fp32 sine / cosine and products: a few 1e-7 of the row's magnitude
+            assert np.abs(a - b).max() <= 2e-6
+    finally:
+        pie.pie_destroy(ctx)

@@ -418,3 +418,42 @@ def test_page_masks_equal_textbook_with_columns_removed_and_page_omission():
     O_o, L_o = oracle_on(SmallBatch([short], H_q).paged(P, "random", seed=4))
     np.testing.assert_allclose(O_h, O_o, atol=1e-14)
     np.testing.assert_allclose(L_h, L_o, atol=1e-14)
+
+
+# RoPE ----------------------------------------------------------------------------------
+def test_rope_pins():
+    """Rotary positions inside the path: hand-derived quarter turn, identity at position 0, norm
+    preservation, and the defining property - scores depend only on position differences, so
+    shifting every position of a request by a constant leaves its attention output unchanged."""
+    # D = 2, theta arbitrary: one pair, angle = pos.  (1, 0) at pos = pi/2 (as a float) -> (cos, sin)
+    x = np.array([[[1.0, 0.0]]])
+    y = orc.rope(x, np.array([1]), 10000.0)
+    np.testing.assert_allclose(y[0, 0], [math.cos(1.0), math.sin(1.0)], atol=1e-15)
+    # D = 4: second pair turns at theta^(-1/2)
+    x = np.array([[[1.0, 2.0, 0.0, 0.0]]])
+    y = orc.rope(x, np.array([3]), 100.0)
+    np.testing.assert_allclose(y[0, 0], [math.cos(3.0), 2 * math.cos(0.3), math.sin(3.0), 2 * math.sin(0.3)], atol=1e-14)
+    rng = np.random.RandomState(31)
+    x = rng.randn(5, 3, 16)
+    assert np.array_equal(orc.rope(x, np.zeros(5, int), 500000.0), x)                       # position 0: identity
+    y = orc.rope(x, rng.randint(0, 100000, 5), 500000.0)
+    np.testing.assert_allclose((y[..., :8] ** 2 + y[..., 8:] ** 2), (x[..., :8] ** 2 + x[..., 8:] ** 2), rtol=1e-12)
+    # relative-position property through the whole forward (fp64 storage so nothing is rounded)
+    P, H_q, H_kv, D, n = 8, 4, 2, 16, 19
+    Q, K, V = rng.randn(n, H_q, D), rng.randn(n, H_kv, D), rng.randn(n, H_kv, D)
+    outs = []
+    for shift in (0, 1000):
+        pool = {p: (np.zeros((P, H_kv, D)), np.zeros((P, H_kv, D))) for p in range(3)}
+        outs.append(orc.forward(pool, P, H_q, np.array([0, n]), np.array([0, 3]), np.array([2, 0, 1]), np.array([n - 2 * P]),
+                                Q, K, V, rope_theta=10000.0, positions=np.arange(n) + shift))
+    np.testing.assert_allclose(outs[0][0], outs[1][0], atol=1e-10)
+    np.testing.assert_allclose(outs[0][1], outs[1][1], atol=1e-10)
+    # and against the textbook computation on explicitly rotated dense arrays
+    Qr, Kr = orc.rope(Q, np.arange(n), 10000.0), orc.rope(K, np.arange(n), 10000.0)
+    Or, Lr = textbook_attention(Qr, Kr, V, causal(n, n))
+    np.testing.assert_allclose(outs[0][0], Or, atol=1e-12)
+    np.testing.assert_allclose(outs[0][1], Lr, atol=1e-12)
+    # to_storage: bf16 bit patterns round to nearest even
+    v = np.array([1.0, 1.00390625, 1.01171875, -2.5])          # 1 + 2^-8 is a tie -> even (1.0); 1 + 3*2^-8 -> 1.015625
+    b = orc.to_storage(v, np.zeros(1, np.uint16))
+    np.testing.assert_array_equal(orc.widen(b), [1.0, 1.0, 1.015625, -2.5])
