@@ -333,6 +333,7 @@ int pie_destroy(pie_ctx* ctx) {
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_stage) cudaFree(ctx->d_stage);
     if (ctx->d_io) cudaFree(ctx->d_io);
+    if (ctx->d_planbuf) cudaFree(ctx->d_planbuf);
     if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
     if (ctx->d_qrot) cudaFree(ctx->d_qrot);
     if (ctx->d_inv_freq) cudaFree(ctx->d_inv_freq);
@@ -606,26 +607,57 @@ int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, c
                      void* out, float* lse, void* stream) {
   if (!ctx || !batch) return PIE_ERR_INVALID;
   if (ctx->host_only) return PIE_ERR_NO_DEVICE;
-  // The context keeps one plan object, one pinned staging buffer and one device arena for this
-  // entry point and reuses them call after call: no allocation in the steady state.
+  // The context keeps one plan object, one pinned staging buffer and two device arenas (tensors,
+  // plan image) for this entry point and reuses them call after call: no allocation in the
+  // steady state.  The Q / K / V uploads are started first, so the DMA runs while the host plans.
   if (!ctx->host_plan) ctx->host_plan = new (std::nothrow) pie_plan();
   pie_plan* plan = ctx->host_plan;
   if (!plan) return PIE_ERR_INVALID;
   plan->ctx = ctx;
-  int rc = pie_build_plan(ctx, batch, plan);
-  if (rc) return rc;
-  if (plan->T == 0) return PIE_OK;
-  if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
   cudaStream_t s = (cudaStream_t)stream;
   PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
-  const PlanLayout L = plan_layout(ctx, plan);
-  const size_t T = plan->T, es = ctx->geom.esize, D = ctx->cfg.head_dim;
-  const size_t q_bytes = T * ctx->cfg.num_q_heads * D * es, kv_bytes = T * ctx->cfg.num_kv_heads * D * es;
-  const size_t lse_bytes = T * ctx->cfg.num_q_heads * 4;
+  const int R = batch->num_requests;
+  const bool early = R > 0 && R <= ctx->cfg.max_requests && batch->qo_indptr && batch->qo_indptr[R] > 0 &&
+                     batch->qo_indptr[R] <= ctx->cfg.max_query_tokens && q && k_new && v_new && out && lse;
+  const size_t es = ctx->geom.esize, D = ctx->cfg.head_dim;
   auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
-  const size_t o_q = al(L.total), o_k = o_q + al(q_bytes), o_v = o_k + al(kv_bytes), o_out = o_v + al(kv_bytes),
-               o_lse = o_out + al(q_bytes), need = o_lse + al(lse_bytes);
-  if ((rc = ensure_buffer(ctx, &ctx->d_io, &ctx->io_bytes, need))) return rc;
+  size_t T = 0, q_bytes = 0, kv_bytes = 0, lse_bytes = 0, o_k = 0, o_v = 0, o_out = 0, o_lse = 0;
+  auto io_layout = [&](size_t tokens) {
+    T = tokens;
+    q_bytes = T * ctx->cfg.num_q_heads * D * es;
+    kv_bytes = T * ctx->cfg.num_kv_heads * D * es;
+    lse_bytes = T * ctx->cfg.num_q_heads * 4;
+    o_k = al(q_bytes);
+    o_v = o_k + al(kv_bytes);
+    o_out = o_v + al(kv_bytes);
+    o_lse = o_out + al(q_bytes);
+    return o_lse + al(lse_bytes);
+  };
+  auto upload_inputs = [&]() -> int {
+    uint8_t* io = (uint8_t*)ctx->d_io;
+    PIE_CUDA(ctx, cudaMemcpyAsync(io, q, q_bytes, cudaMemcpyHostToDevice, s));
+    PIE_CUDA(ctx, cudaMemcpyAsync(io + o_k, k_new, kv_bytes, cudaMemcpyHostToDevice, s));
+    PIE_CUDA(ctx, cudaMemcpyAsync(io + o_v, v_new, kv_bytes, cudaMemcpyHostToDevice, s));
+    return PIE_OK;
+  };
+  int rc;
+  if (early) {
+    if ((rc = ensure_buffer(ctx, &ctx->d_io, &ctx->io_bytes, io_layout((size_t)batch->qo_indptr[R])))) return rc;
+    if ((rc = upload_inputs())) return rc;
+  }
+  rc = pie_build_plan(ctx, batch, plan);
+  if (rc) {
+    if (early) cudaStreamSynchronize(s);  // the caller's buffers must outlive the copies already queued
+    return rc;
+  }
+  if (plan->T == 0) return PIE_OK;
+  if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
+  if (!early) {
+    if ((rc = ensure_buffer(ctx, &ctx->d_io, &ctx->io_bytes, io_layout((size_t)plan->T)))) return rc;
+    if ((rc = upload_inputs())) return rc;
+  }
+  const PlanLayout L = plan_layout(ctx, plan);
+  if ((rc = ensure_buffer(ctx, &ctx->d_planbuf, &ctx->planbuf_bytes, L.total))) return rc;
   if (ctx->h_stage_bytes < L.upload) {
     if (ctx->h_stage) PIE_CUDA(ctx, cudaFreeHost(ctx->h_stage));
     ctx->h_stage = nullptr;
@@ -634,17 +666,13 @@ int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, c
     PIE_CUDA(ctx, cudaMallocHost(&ctx->h_stage, want));
     ctx->h_stage_bytes = want;
   }
-  uint8_t* base = (uint8_t*)ctx->d_io;
+  uint8_t* io = (uint8_t*)ctx->d_io;
   plan_fill(plan, L, (uint8_t*)ctx->h_stage);
-  plan_bind(plan, L, base);
-  PIE_CUDA(ctx, cudaMemcpyAsync(base, ctx->h_stage, L.upload, cudaMemcpyHostToDevice, s));
-  PIE_CUDA(ctx, cudaMemcpyAsync(base + o_q, q, q_bytes, cudaMemcpyHostToDevice, s));
-  PIE_CUDA(ctx, cudaMemcpyAsync(base + o_k, k_new, kv_bytes, cudaMemcpyHostToDevice, s));
-  PIE_CUDA(ctx, cudaMemcpyAsync(base + o_v, v_new, kv_bytes, cudaMemcpyHostToDevice, s));
-  if ((rc = pie_forward(ctx, plan, base + o_q, base + o_k, base + o_v, base + o_out, (float*)(base + o_lse), stream)))
-    return rc;
-  PIE_CUDA(ctx, cudaMemcpyAsync(out, base + o_out, q_bytes, cudaMemcpyDeviceToHost, s));
-  PIE_CUDA(ctx, cudaMemcpyAsync(lse, base + o_lse, lse_bytes, cudaMemcpyDeviceToHost, s));
+  plan_bind(plan, L, (uint8_t*)ctx->d_planbuf);
+  PIE_CUDA(ctx, cudaMemcpyAsync(ctx->d_planbuf, ctx->h_stage, L.upload, cudaMemcpyHostToDevice, s));
+  if ((rc = pie_forward(ctx, plan, io, io + o_k, io + o_v, io + o_out, (float*)(io + o_lse), stream))) return rc;
+  PIE_CUDA(ctx, cudaMemcpyAsync(out, io + o_out, q_bytes, cudaMemcpyDeviceToHost, s));
+  PIE_CUDA(ctx, cudaMemcpyAsync(lse, io + o_lse, lse_bytes, cudaMemcpyDeviceToHost, s));
   PIE_CUDA(ctx, cudaStreamSynchronize(s));
   return PIE_OK;
 }

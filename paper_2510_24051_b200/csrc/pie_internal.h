@@ -128,8 +128,10 @@ struct pie_ctx {
   int* d_status = nullptr;
   void* d_stage = nullptr;  // staging for host <-> device calls
   size_t stage_bytes = 0;
-  void* d_io = nullptr;     // device arena of pie_forward_host: plan image + q/k/v/out/lse
+  void* d_io = nullptr;     // device arena of pie_forward_host: q/k/v/out/lse
   size_t io_bytes = 0;
+  void* d_planbuf = nullptr;  // device arena of pie_forward_host: plan image + partial workspaces
+  size_t planbuf_bytes = 0;
   void* d_qrot = nullptr;        // rotated copy of Q (RoPE contexts): [max_query_tokens][H_q][D]
   double* d_inv_freq = nullptr;  // [D/2] theta^(-2i/D)
   void* h_stage = nullptr;  // pinned host staging of the plan image (pie_forward_host)

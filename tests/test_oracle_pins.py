@@ -457,3 +457,10 @@ def test_rope_pins():
     v = np.array([1.0, 1.00390625, 1.01171875, -2.5])          # 1 + 2^-8 is a tie -> even (1.0); 1 + 3*2^-8 -> 1.015625
     b = orc.to_storage(v, np.zeros(1, np.uint16))
     np.testing.assert_array_equal(orc.widen(b), [1.0, 1.0, 1.015625, -2.5])
+
+
+def test_default_positions_are_the_last_q_len_context_positions():
+    # request 0: 2 pages of 8, last page holds 3 -> kv_len 11, 1 new token -> position 10
+    # request 1: 3 pages, last holds 8 -> kv_len 24, 4 new tokens -> positions 20..23
+    pos = orc.default_positions(np.array([0, 1, 5]), np.array([0, 2, 5]), np.array([3, 8]), 8)
+    assert pos.tolist() == [10, 20, 21, 22, 23]
