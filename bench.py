@@ -197,6 +197,8 @@ def main():
     ap.add_argument("--workload", default="batched_decode")
     ap.add_argument("--flags", type=int, default=0, help="PIE_PLAN_* flags (debug / A-B runs)")
     ap.add_argument("--opt", action="append", default=[], help="pie_set_option as K=V (tuning runs)")
+    ap.add_argument("--graph", type=int, default=0,
+                    help="1: replay one captured CUDA graph per step (measured: no gain, the loop is GPU bound), 0: eager launches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -256,6 +258,28 @@ def main():
             pie.pie_copy_kvpage(ctx, copies["src"], copies["dst"], copies["src_off"], copies["dst_off"], copies["ntok"])
 
     # ---------------------------------------------------------------- device-resident timing
+    eager_step = step
+    use_graph = args.graph == 1 and copies is None
+    if use_graph:
+        # pie_forward only enqueues kernels on the caller's stream, so a step is captured once per
+        # page placement and replayed: no host launch cost inside the timed loop
+        cap = torch.cuda.Stream()
+        cap.wait_stream(torch.cuda.current_stream())
+        graphs = []
+        with torch.cuda.stream(cap):
+            for i in range(len(plans)):
+                eager_step(i)
+            cap.synchronize()
+            for i in range(len(plans)):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=cap):
+                    eager_step(i)
+                graphs.append(g)
+        torch.cuda.current_stream().wait_stream(cap)
+
+        def step(i):
+            graphs[i % len(graphs)].replay()
+
     for i in range(args.warmup):
         step(i)
     barrier()
@@ -277,7 +301,7 @@ def main():
     # ---------------------------------------------------------------- per-kernel timing (live)
     pie.pie_set_kernel_timing(ctx, 1)
     for i in range(args.steps):
-        step(i)
+        eager_step(i)
     torch.cuda.synchronize()
     ktimes = pie.pie_get_kernel_times(ctx)
     pie.pie_set_kernel_timing(ctx, 0)
@@ -367,7 +391,7 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": wl0.dtype, "data": "synthetic",
         "config": {"workload": wl0.name, "requests": wl0.R, "query_tokens": wl0.T, "heads": f"{wl0.H_q}/{wl0.H_kv}",
                    "head_dim": wl0.D, "page_size": wl0.P, "pool_pages": wl0.num_pages, "l2": l2_note,
-                   "plan_flags": args.flags},
+                   "plan_flags": args.flags, "launch": "cuda graph replay" if use_graph else "eager"},
         "hbm_gbs_step": alg_bytes["total"] / (ms_per_step * 1e-3) / 1e9,
         "algorithmic_bytes_step": alg_bytes, "useful_flops_step": wl0.useful_flops(),
         "plan_ms": statistics.median(plan_ms), "plan_info": info,

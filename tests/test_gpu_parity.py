@@ -250,3 +250,35 @@ def test_rope_inside_the_path_matches_oracle(name, explicit_pos):
             assert np.abs(a - b).max() <= 2e-6
     finally:
         pie.pie_destroy(ctx)
+
+
+def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
+    """pie_forward only enqueues kernels on the caller's stream (no allocation, no synchronisation), so a
+    decode step can be captured once and replayed; the replay must reproduce the eager result bit for bit."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool
+    wl = configs.small("mixed_prefill_decode")
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl)
+        plan = gp.plan(wl)
+        q, k, v = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
+        ref_out, ref_lse = gp.forward(plan, q, k, v)
+        out = torch.zeros_like(ref_out)
+        lse = torch.zeros_like(ref_lse)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            pie.pie_forward(gp.ctx, plan, q, k, v, out, lse)          # warm-up on the capture stream
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                pie.pie_forward(gp.ctx, plan, q, k, v, out, lse)
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(3):
+            out.zero_()
+            lse.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(out, ref_out) and torch.equal(lse, ref_lse)
+        assert pie.pie_get_last_device_status(gp.ctx) == 0
+        pie.pie_plan_destroy(plan)
