@@ -19,6 +19,10 @@
  *   - The KvPage pool is owned by the library; its layout is private.  Q / K_new / V_new /
  *     output / LSE buffers are owned by the caller.
  *   - Element type: bf16 or fp32 for Q, K, V and the output; LSE is always fp32.
+ *   - Threads: a context (and its plans and scheduler objects) must not be used from two host
+ *     threads at the same time.  A plan owns the scratch of its split partials, so two
+ *     pie_forward calls on the SAME plan must not overlap on the GPU (same stream order is fine);
+ *     different plans may run concurrently on different streams.
  */
 #ifndef PIE_B200_H_
 #define PIE_B200_H_

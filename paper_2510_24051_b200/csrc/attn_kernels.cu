@@ -286,7 +286,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
-  pie_pdl_wait();  // the append (and whatever produced Q) must be complete before the first copy / Q load
 
   // ---- prefetch side: a cursor DEPTH page visits ahead of the consumer
   int q_head = 0, q_tail = 0;                       // queue of chunk ids, pushed here, popped by the consumer
@@ -368,8 +367,26 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
              smem_u32(full_bar + s));
   };
 
-  pf_settle();
-  for (int n = 0; n < DEPTH && pf_live; ++n) {  // prologue: fill the ring
+  // Prologue.  The plan arrays are not written by the kernels that precede this one in the stream, so
+  // a warp with a fixed share walks its first DEPTH page records BEFORE waiting for those kernels:
+  // under programmatic dependent launch this runs while the previous kernel drains.  The work
+  // counter, the pool, Q and every output are touched only after the wait.
+  int2 pre_rec[DEPTH];
+  int n_pre = 0;
+  if (own_next < own_end) {
+    pf_settle();  // enters the first item of the fixed share (no counter access)
+    n_pre = min(DEPTH, pf_end - pf_k);
+#pragma unroll
+    for (int i = 0; i < DEPTH; ++i)
+      if (i < n_pre) pre_rec[i] = __ldg(&p.kept[pf_k + i]);
+  }
+  pie_pdl_wait();  // the append (and whatever produced Q) is complete from here on
+#pragma unroll
+  for (int i = 0; i < DEPTH; ++i)
+    if (i < n_pre && lane == 0) issue(i, pre_rec[i], pf_head);
+  pf_k += n_pre;
+  pf_settle();  // (may take from the counter now)
+  for (int n = n_pre; n < DEPTH && pf_live; ++n) {  // rest of the ring
     const int2 rec = __ldg(&p.kept[pf_k]);
     if (lane == 0) issue(n, rec, pf_head);
     ++pf_k;
