@@ -3,17 +3,22 @@
 //
 // One CTA per SM walks its share of work items.  An item is up to 256 rows (row = query token *
 // G + head-in-group, one kv head) = two 128-row Q tiles, attended over the item's kept pages in
-// KV tiles of 128 tokens.  Roles (384 threads):
-//   warps 0-3 / 4-7  softmax warpgroup of Q tile 0 / 1: one row per thread.  Reads S from TMEM,
-//                    masks, exponentiates, writes bf16 P back over S in TMEM, keeps the running
-//                    (max, sum), rescales O in TMEM only when the row max grew by more than 2^8,
-//                    and runs the epilogue.
+// KV tiles of 128 tokens that are handled as two halves of 64 columns.  Roles (320 threads):
+//   warps 0-3 / 4-7  softmax warpgroup of Q tile 0 / 1: one row per thread.  Reads a half of S
+//                    from TMEM, masks, exponentiates, writes bf16 P back over that half of S,
+//                    keeps the running (max, sum), rescales O in TMEM only when the row max grew
+//                    by more than 2^8, and runs the epilogue.
 //   warp 8           producer: linear bulk copies of page blocks into the K / V stage rings.  The
 //                    pool's storage order is the 128-byte-swizzled canonical operand layout, so a
 //                    page block drops into its 16-row band of the tile with no tensor map.
-//   warp 9           MMA issuer (one lane): S_t = Q_t K^T, O_t += P_t V with tcgen05.mma,
+//   warp 9, lane 0   MMA issuer: S_t^h = Q_t K_h^T (N = 64), O_t += P_t^h V_h with tcgen05.mma,
 //                    accumulators and P in TMEM; completion is tracked with tcgen05.commit.
-// TMEM (512 columns): S0 | S1 | O0 | O1; P_t overlays the first 64 columns of S_t.
+// The tensor pipe takes instructions synchronously from the issuing thread (measured: a group of
+// eight MMAs returns after ~8 x 64 cycles and any other work of that thread is idle pipe time), so
+// the issuer is a single thread that does nothing but wait, issue and commit.  The two halves
+// break the chain S -> softmax -> PV -> next S of a Q tile: while a warpgroup works on one half,
+// the PV of the other half and the next S into the columns it frees are already running.
+// TMEM (512 columns): S0a S0b | S1a S1b | O0 | O1; P_t^h overlays the first 32 columns of S_t^h.
 #include <cuda_bf16.h>
 
 #include "pie_internal.h"
@@ -55,6 +60,19 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// A load that stays where it is written (the compiler neither sinks it to its first use nor
+// merges it with a later one).
+__device__ __forceinline__ uint32_t ldg_early(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+// One lane of the (converged) warp, the same one every time.
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred P;\nelect.sync _|P, 0xffffffff;\nselp.u32 %0, 1, 0, P;\n}\n" : "=r"(pred));
+  return pred;
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -65,17 +83,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%"
-      "32};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
-      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
@@ -127,25 +134,28 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 constexpr float kNegInf = -__builtin_huge_valf();
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr int kTileM = 128;   // rows per Q tile
-constexpr int kTileN = 128;   // tokens per KV tile
+constexpr int kTileM = 128;    // rows per Q tile
+constexpr int kTileN = 128;    // tokens per KV tile (one stage of the K / V rings)
+constexpr int kHalf = 64;      // columns per half tile: the unit handed between softmax and MMA
+constexpr int kThreads = 320;
 
 template <int D, int P>
 struct TcCfg {
   static constexpr int NSLAB = D / 64;                 // 128-byte slabs per row
   static constexpr int PPT = kTileN / P;               // pages per KV tile
+  static constexpr int PPH = kHalf / P;                // pages per half
   static constexpr int SLAB_TILE = kTileN * 128;       // bytes of one slab of a 128-row tile (16 KB)
   static constexpr int SLAB_PAGE = P * 128;            // bytes of one slab of a page block
   static constexpr int BLK = P * D * 2;                // K (or V) block of one page and head
   static constexpr int QTILE = kTileM * D * 2;
   static constexpr int KVTILE = kTileN * D * 2;
   static constexpr int STAGES = D == 128 ? 2 : 4;
-  static constexpr int NBAR = 4 * STAGES + 10;
+  static constexpr int NBAR = 4 * STAGES + 17;
   static constexpr int SMEM = 2 * QTILE + 2 * STAGES * KVTILE + NBAR * 8 + 64;
 };
 
 template <int D, int P>
-__global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p) {
   using C = TcCfg<D, P>;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* sQ = smem;
@@ -156,12 +166,14 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
   uint64_t* k_empty = k_full + C::STAGES;
   uint64_t* v_full = k_empty + C::STAGES;
   uint64_t* v_empty = v_full + C::STAGES;
-  uint64_t* q_full = v_empty + C::STAGES;  // [2]
-  uint64_t* s_full = q_full + 2;           // [2]
-  uint64_t* p_full = s_full + 2;           // [2]
-  uint64_t* o_done = p_full + 2;           // [2]
-  uint64_t* o_free = o_done + 2;           // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_free + 2);
+  uint64_t* q_full = v_empty + C::STAGES;  // [2]      Q tile t is in shared memory
+  uint64_t* s_full = q_full + 2;           // [2][2]   S_t^h is complete in TMEM
+  uint64_t* p_full = s_full + 4;           // [2][2]   P_t^h is written (128 arrivals)
+  uint64_t* pv_done = p_full + 4;          // [2]      one phase per PV group of Q tile t
+  uint64_t* o_done = pv_done + 2;          // [2]      last PV of the item is complete
+  uint64_t* o_free = o_done + 2;           // [2]      the epilogue has read O_t (128 arrivals)
+  uint64_t* v_land = o_free + 2;           // [1]      producer-private: V tile that needs its tail cleared
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(v_land + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -173,11 +185,15 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
     }
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(q_full + t), kTileM);
-      mbar_init(smem_u32(s_full + t), 1);
-      mbar_init(smem_u32(p_full + t), kTileM);
+      for (int h = 0; h < 2; ++h) {
+        mbar_init(smem_u32(s_full + 2 * t + h), 1);
+        mbar_init(smem_u32(p_full + 2 * t + h), kTileM);
+      }
+      mbar_init(smem_u32(pv_done + t), 1);
       mbar_init(smem_u32(o_done + t), 1);
       mbar_init(smem_u32(o_free + t), kTileM);
     }
+    mbar_init(smem_u32(v_land), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 8) {
@@ -193,141 +209,179 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
 
   const int it0 = p.cta_ptr[blockIdx.x], it1 = p.cta_ptr[blockIdx.x + 1];
 
-  if (warp >= 8) {
-    if (warp == 8) {
-      // ================================================================ producer
-      uint32_t tile_cnt = 0;
-      for (int it = it0; it < it1; ++it) {
-        const PieItem item = p.items[it];
-        const uint8_t* base = p.pool + (int64_t)item.kv_head * (2 * C::BLK);
-        const int npages = item.page_end - item.page_begin;
-        const int ntiles = (npages + C::PPT - 1) / C::PPT;
-        for (int j = 0; j < ntiles; ++j, ++tile_cnt) {
-          const uint32_t s = tile_cnt % C::STAGES, ph = (tile_cnt / C::STAGES) & 1;
-          const int nvalid = min(C::PPT, npages - j * C::PPT);
-          const int ncopies = nvalid * C::NSLAB;
-          int phys = 0;
-          if (lane < nvalid) phys = __ldg(&p.kept[item.page_begin + j * C::PPT + lane].x);
-          // ---- K
-          mbar_wait(smem_u32(k_empty + s), ph ^ 1, p.status);
-          if (lane == 0) mbar_expect_tx(smem_u32(k_full + s), nvalid * C::BLK);
+  if (warp == 8) {
+    // ================================================================ producer
+    uint32_t tile_cnt = 0, land_cnt = 0;
+    for (int it = it0; it < it1; ++it) {
+      const PieItem item = p.items[it];
+      const uint8_t* base = p.pool + (int64_t)item.kv_head * (2 * C::BLK);
+      const int npages = item.page_end - item.page_begin;
+      const int ntiles = (npages + C::PPT - 1) / C::PPT;
+      const bool ragged = item.last_page_len < P;   // slots past the end of the context may hold anything
+      for (int j = 0; j < ntiles; ++j, ++tile_cnt) {
+        const uint32_t s = tile_cnt % C::STAGES, ph = (tile_cnt / C::STAGES) & 1;
+        const int nvalid = min(C::PPT, npages - j * C::PPT);
+        const int ncopies = nvalid * C::NSLAB;
+        int2 rec = make_int2(0, -1);
+        if (lane < nvalid) rec = __ldg(&p.kept[item.page_begin + j * C::PPT + lane]);
+        const int pg = lane / C::NSLAB, sl = lane % C::NSLAB;   // copy `lane`: page pg of the tile, slab sl
+        const int ph_pg = __shfl_sync(0xFFFFFFFFu, rec.x, pg);   // (at most PPT * NSLAB <= 32 copies per tile)
+        // ---- K
+        mbar_wait(smem_u32(k_empty + s), ph ^ 1, p.status);
+        if (lane == 0) mbar_expect_tx(smem_u32(k_full + s), nvalid * C::BLK);
+        __syncwarp();
+        if (lane < ncopies)
+          bulk_g2s(smem_u32(sK + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
+                   base + (int64_t)ph_pg * p.page_bytes + sl * C::SLAB_PAGE, C::SLAB_PAGE, smem_u32(k_full + s));
+        __syncwarp();
+        // ---- V.  A tile that holds the request's partly filled last page lands on a private
+        // barrier first: the rows past the end of the context are cleared (they may hold NaN
+        // patterns, and 0 x NaN would poison O) before the tile is handed to the MMA thread.
+        mbar_wait(smem_u32(v_empty + s), ph ^ 1, p.status);
+        unsigned hit = 0;
+        if (ragged) hit = __ballot_sync(0xFFFFFFFFu, lane < nvalid && (int)((uint32_t)rec.y & ~PIE_KEPT_NEEDS_MASK) == item.last_logical);
+        const uint32_t vbar = hit ? smem_u32(v_land) : smem_u32(v_full + s);
+        if (lane == 0) mbar_expect_tx(vbar, nvalid * C::BLK);
+        __syncwarp();
+        if (lane < ncopies)
+          bulk_g2s(smem_u32(sV + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
+                   base + (int64_t)ph_pg * p.page_bytes + C::BLK + sl * C::SLAB_PAGE, C::SLAB_PAGE, vbar);
+        __syncwarp();
+        if (hit) {
+          mbar_wait(smem_u32(v_land), land_cnt & 1, p.status);
+          ++land_cnt;
+          const int pgi = __ffs(hit) - 1;
+          constexpr int CH = D * 2 / 16;
+          const int nz = (P - item.last_page_len) * CH;
+          for (int c = lane; c < nz; c += 32) {
+            const int tkn = pgi * P + item.last_page_len + c / CH, ch = c % CH;
+            *reinterpret_cast<uint4*>(sV + s * C::KVTILE + (ch >> 3) * C::SLAB_TILE + tkn * 128 + (((ch & 7) ^ (tkn & 7)) << 4)) =
+                make_uint4(0, 0, 0, 0);
+          }
+          fence_async_smem();
           __syncwarp();
-          const int pg = lane / C::NSLAB, sl = lane % C::NSLAB;     // copy `lane`: page pg of the tile, slab sl
-          const int ph_pg = __shfl_sync(0xFFFFFFFFu, phys, pg);      // (at most PPT * NSLAB <= 32 copies per tile)
-          if (lane < ncopies)
-            bulk_g2s(smem_u32(sK + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
-                     base + (int64_t)ph_pg * p.page_bytes + sl * C::SLAB_PAGE, C::SLAB_PAGE, smem_u32(k_full + s));
-          __syncwarp();
-          // ---- V
-          mbar_wait(smem_u32(v_empty + s), ph ^ 1, p.status);
-          if (lane == 0) mbar_expect_tx(smem_u32(v_full + s), nvalid * C::BLK);
-          __syncwarp();
-          if (lane < ncopies)
-            bulk_g2s(smem_u32(sV + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
-                     base + (int64_t)ph_pg * p.page_bytes + C::BLK + sl * C::SLAB_PAGE, C::SLAB_PAGE,
-                     smem_u32(v_full + s));
-          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(v_full + s));
         }
       }
-    } else if (warp == 9) {
-      // ================================================================ MMA issuer
+    }
+  } else if (warp == 9) {
+    // ================================================================ MMA issuer
+    // One elected lane runs the whole role.  (Electing the lane, rather than testing the lane id,
+    // lets the compiler keep descriptors and loop state in uniform registers; measured, it halves
+    // the cost of issuing an MMA.)  Everything between two batches of MMAs is time the tensor pipe
+    // may run dry, so interior KV tiles take a fully unrolled path with constant offsets.
+    if (elect_one()) {
       uint32_t tile_cnt = 0;
-      uint32_t n_items[2] = {0, 0};   // items in which Q tile t took part (phase of q_full / o_done / o_free)
-      uint32_t n_tiles[2] = {0, 0};   // KV tiles Q tile t went through (phase of s_full / p_full)
+      uint32_t item_ph = 0;   // bit t: phase of q_full / o_free of Q tile t
+      uint32_t half_ph = 0;   // bit 2t+h: phase of p_full[t][h]
       const uint32_t idesc_pv = instr_desc(kTileM, D, 1);
+      const uint32_t idesc_s = instr_desc(kTileM, kHalf, 0);
       const uint64_t k_desc0 = smem_desc(smem_u32(sK), 16, 1024);            // K-major
       const uint64_t v_desc0 = smem_desc(smem_u32(sV), C::SLAB_TILE, 1024);  // MN-major: LBO = slab stride
       const uint64_t q_desc0 = smem_desc(smem_u32(sQ), 16, 1024);
+      const uint32_t bar_p = smem_u32(p_full), bar_s = smem_u32(s_full), bar_pv = smem_u32(pv_done);
       for (int it = it0; it < it1; ++it) {
-        const PieItem item = p.items[it];
-        const PieReq rq = p.reqs[item.req];
-        const int npages = item.page_end - item.page_begin;
+        const PieItem* ip = p.items + it;
+        const int npages = __ldg(&ip->page_end) - __ldg(&ip->page_begin);
+        const int nrows = __ldg(&ip->nrows);
+        if (npages == 0) continue;  // the softmax warpgroups write zeros / -inf on their own
         const int ntiles = (npages + C::PPT - 1) / C::PPT;
-        const int nt = item.nrows > kTileM ? 2 : 1;
-        if (ntiles == 0) continue;  // the softmax warpgroups write zeros / -inf on their own
+        const int nhalf = (npages + C::PPH - 1) / C::PPH;           // halves of the item
+        const int last_cols = (npages - (nhalf - 1) * C::PPH) * P;  // columns of the last half
+        const int nt = nrows > kTileM ? 2 : 1;
         for (int t = 0; t < nt; ++t) {
-          mbar_wait(smem_u32(q_full + t), n_items[t] & 1, p.status);
-          mbar_wait(smem_u32(o_free + t), (n_items[t] & 1) ^ 1, p.status);  // previous epilogue has drained O_t
-          ++n_items[t];
+          mbar_wait(smem_u32(q_full + t), (item_ph >> t) & 1, p.status);
+          mbar_wait(smem_u32(o_free + t), ((item_ph >> t) & 1) ^ 1, p.status);  // previous epilogue has drained O_t
+          item_ph ^= 1u << t;
         }
         tc_fence_after();
 
         // Descriptors are built once (per kernel for the K / V stages, per item for Q); a k-step only
         // adds its byte offset >> 4 to the start-address field.
-        auto issue_s = [&](int t, int j, uint32_t cnt) {
-          const uint32_t s = cnt % C::STAGES;
-          const int nvalid = min(C::PPT, npages - j * C::PPT);
-          const uint32_t idesc = instr_desc(kTileM, nvalid * P, 0);
-          const uint64_t qd = q_desc0 + (uint64_t)(t * (C::QTILE >> 4)), kd = k_desc0 + (uint64_t)(s * (C::KVTILE >> 4));
+        auto issue_s = [&](int t, int i, uint32_t stage) {   // S_t^h = Q_t K_h^T for half i of the item (h = i & 1)
+          const int h = i & 1;
+          const uint32_t idesc = instr_desc(kTileM, i + 1 < nhalf ? kHalf : last_cols, 0);
+          const uint64_t qd = q_desc0 + (uint64_t)(t * (C::QTILE >> 4));
+          const uint64_t kd = k_desc0 + (uint64_t)(stage * (C::KVTILE >> 4) + h * ((kHalf * 128) >> 4));
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
             const uint64_t off = (uint64_t)(((ks >> 2) * C::SLAB_TILE + (ks & 3) * 32) >> 4);
-            umma_ss(tmem + t * 128, qd + off, kd + off, idesc, ks > 0);
+            umma_ss(tmem + t * 128 + h * kHalf, qd + off, kd + off, idesc, ks > 0);
           }
-          umma_commit(smem_u32(s_full + t));
+          umma_commit(bar_s + 8 * (2 * t + h));
         };
 
-        // prologue: S_t(0)
+        // prologue: both halves of S_t for the first KV tile
         {
           const uint32_t s = tile_cnt % C::STAGES, ph = (tile_cnt / C::STAGES) & 1;
           mbar_wait(smem_u32(k_full + s), ph, p.status);
           tc_fence_after();
-          if (lane == 0) {
-            for (int t = 0; t < nt; ++t) issue_s(t, 0, tile_cnt);
-            umma_commit(smem_u32(k_empty + s));
-          }
-          __syncwarp();
+          for (int h = 0; h < min(2, nhalf); ++h)
+            for (int t = 0; t < nt; ++t) issue_s(t, h, s);
+          umma_commit(smem_u32(k_empty + s));
         }
         for (int j = 0; j < ntiles; ++j) {
           const uint32_t cnt = tile_cnt + j;
           const uint32_t s = cnt % C::STAGES, ph = (cnt / C::STAGES) & 1;
-          const int nvalid = min(C::PPT, npages - j * C::PPT);
+          const uint32_t sn = (cnt + 1) % C::STAGES, phn = ((cnt + 1) / C::STAGES) & 1;
           mbar_wait(smem_u32(v_full + s), ph, p.status);
-          // clear V rows past the end of the context in the request's last page (may hold NaN patterns)
-          if (rq.last_page_len < P) {
-            const int pg = lane < nvalid ? (int)((uint32_t)__ldg(&p.kept[item.page_begin + j * C::PPT + lane].y) & ~PIE_KEPT_NEEDS_MASK) : -1;
-            const unsigned hit = __ballot_sync(0xFFFFFFFFu, pg == rq.last_logical);
-            if (hit) {
-              const int pgi = __ffs(hit) - 1;
-              constexpr int CH = D * 2 / 16;
-              const int nz = (P - rq.last_page_len) * CH;
-              for (int c = lane; c < nz; c += 32) {
-                const int tkn = pgi * P + rq.last_page_len + c / CH, ch = c % CH;
-                *reinterpret_cast<uint4*>(sV + s * C::KVTILE + (ch >> 3) * C::SLAB_TILE + tkn * 128 +
-                                          (((ch & 7) ^ (tkn & 7)) << 4)) = make_uint4(0, 0, 0, 0);
-              }
-              fence_async_smem();
-              __syncwarp();
-            }
-          }
-          tc_fence_after();
-          for (int t = 0; t < nt; ++t) {
-            mbar_wait(smem_u32(p_full + t), n_tiles[t] & 1, p.status);
-            ++n_tiles[t];
-            tc_fence_after();
-            if (lane == 0) {
-              const uint64_t vd = v_desc0 + (uint64_t)(s * (C::KVTILE >> 4));
-              const int ksteps = nvalid * P / 16;
-#pragma unroll 8
-              for (int ks = 0; ks < ksteps; ++ks)   // 16 token rows = 2048 bytes per k-step
-                umma_ts(tmem + 256 + t * D, tmem + t * 128 + ks * 8, vd + (uint64_t)(ks * 128), idesc_pv,
-                        (j > 0 || ks > 0) ? 1u : 0u);
-              if (t == nt - 1) umma_commit(smem_u32(v_empty + s));
-              if (j + 1 == ntiles) umma_commit(smem_u32(o_done + t));
-            }
-            __syncwarp();
-            if (j + 1 < ntiles) {
-              const uint32_t cn = cnt + 1;
-              const uint32_t sn = cn % C::STAGES, phn = (cn / C::STAGES) & 1;
-              if (t == 0) {
-                mbar_wait(smem_u32(k_full + sn), phn, p.status);
+          if (nt == 2 && j > 0 && 2 * j + 5 <= nhalf) {
+            // ---- interior tile: this tile and the next both have two full halves
+            mbar_wait(smem_u32(k_full + sn), phn, p.status);
+            const uint64_t vd0 = v_desc0 + (uint64_t)(s * (C::KVTILE >> 4));
+            const uint64_t kd0 = k_desc0 + (uint64_t)(sn * (C::KVTILE >> 4));
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll
+              for (int t = 0; t < 2; ++t) {
+                mbar_wait(bar_p + 8 * (2 * t + h), (half_ph >> (2 * t + h)) & 1, p.status);
                 tc_fence_after();
+                const uint32_t dO = tmem + 256 + t * D, dS = tmem + t * 128 + h * kHalf;
+#pragma unroll
+                for (int ks = 0; ks < kHalf / 16; ++ks)   // 16 token rows = 2048 bytes per k-step
+                  umma_ts(dO, dS + ks * 8, vd0 + (uint64_t)((h * (kHalf / 16) + ks) * 128), idesc_pv, 1u);
+                umma_commit(bar_pv + 8 * t);
+                if (h == 1 && t == 1) umma_commit(smem_u32(v_empty + s));
+                const uint64_t qd = q_desc0 + (uint64_t)(t * (C::QTILE >> 4));
+                const uint64_t kd = kd0 + (uint64_t)(h * ((kHalf * 128) >> 4));
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                  const uint64_t off = (uint64_t)(((ks >> 2) * C::SLAB_TILE + (ks & 3) * 32) >> 4);
+                  umma_ss(dS, qd + off, kd + off, idesc_s, ks > 0);
+                }
+                umma_commit(bar_s + 8 * (2 * t + h));
+                if (h == 1 && t == 1) umma_commit(smem_u32(k_empty + sn));
               }
-              if (lane == 0) {
-                issue_s(t, j + 1, cn);
-                if (t == nt - 1) umma_commit(smem_u32(k_empty + sn));
+            }
+            half_ph ^= 0xFu;
+            continue;
+          }
+          // ---- first / last tiles of an item, ragged halves, single Q tile
+          const int nh = min(2, nhalf - 2 * j);                            // halves of this tile
+          const int nhn = j + 1 < ntiles ? min(2, nhalf - 2 * j - 2) : 0;   // halves of the next one
+          bool k_ready = false;
+          for (int h = 0; h < nh; ++h) {
+            const int i = 2 * j + h;
+            const int ksteps = (i + 1 < nhalf ? kHalf : last_cols) / 16;
+            for (int t = 0; t < nt; ++t) {
+              mbar_wait(bar_p + 8 * (2 * t + h), (half_ph >> (2 * t + h)) & 1, p.status);
+              half_ph ^= 1u << (2 * t + h);
+              if (h < nhn && !k_ready) {
+                mbar_wait(smem_u32(k_full + sn), phn, p.status);
+                k_ready = true;
               }
-              __syncwarp();
+              tc_fence_after();
+              const uint64_t vd = v_desc0 + (uint64_t)(s * (C::KVTILE >> 4) + h * (kHalf / 16) * 128);
+              const uint32_t dO = tmem + 256 + t * D, aP = tmem + t * 128 + h * kHalf;
+              for (int ks = 0; ks < ksteps; ++ks)
+                umma_ts(dO, aP + ks * 8, vd + (uint64_t)(ks * 128), idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
+              umma_commit(bar_pv + 8 * t);
+              if (h == nh - 1 && t == nt - 1) umma_commit(smem_u32(v_empty + s));
+              if (i + 1 == nhalf) umma_commit(smem_u32(o_done + t));
+              if (h < nhn) {   // S_t^h of the next tile goes into the columns this PV frees
+                issue_s(t, i + 2, sn);
+                if (h == nhn - 1 && t == nt - 1) umma_commit(smem_u32(k_empty + sn));
+              }
             }
           }
         }
@@ -340,25 +394,26 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
     const int rho = (warp & 3) * 32 + lane;        // row inside the tile = TMEM lane
     const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + t * 128 + lane_sel, tO = tmem + 256 + t * D + lane_sel;
-    uint32_t my_items = 0, my_tiles = 0;   // phases of the per-item / per-tile barriers of this Q tile
+    uint32_t my_items = 0;   // phase of o_done
+    uint32_t s_ph = 0;       // bit h: phase of s_full[t][h]
+    uint32_t n_arr = 0;      // p_full arrivals so far = PV groups of this Q tile issued or about to be
     for (int it = it0; it < it1; ++it) {
       const PieItem item = p.items[it];
-      const PieReq rq = p.reqs[item.req];
       const int npages = item.page_end - item.page_begin;
-      const int ntiles = (npages + C::PPT - 1) / C::PPT;
+      const int nhalf = (npages + C::PPH - 1) / C::PPH;
       const int nt = item.nrows > kTileM ? 2 : 1;
       if (t >= nt) continue;
       const int gr = item.row0 + t * kTileM + rho;
       const bool valid = gr < item.row0 + item.nrows;
       const int tok = valid ? gr / p.G : 0;
       const int head = item.kv_head * p.G + (valid ? gr % p.G : 0);
-      const int64_t oi = (int64_t)(rq.q_start + tok) * p.n_q_heads + head;
-      const int lim = valid ? rq.kv_len - rq.q_len + tok : -1;
-      const uint32_t* mrow = p.mask + rq.mask_word_off + (int64_t)tok * rq.mask_row_words;
-      const bool explicit_mask = rq.mask_row_words != 0;
+      const int64_t oi = (int64_t)(item.q_start + tok) * p.n_q_heads + head;
+      const int lim = valid ? item.kv_len - item.q_len + tok : -1;
+      const uint32_t* mrow = p.mask + item.mask_word_off + (int64_t)tok * item.mask_row_words;
+      const bool explicit_mask = item.mask_row_words != 0;
       float m_ref = kNegInf, l_sum = 0.f;
 
-      if (ntiles > 0) {
+      if (nhalf > 0) {
         // ---- Q row -> shared memory (K-major, 128-byte swizzle)
         const uint4* qsrc = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.q) + oi * D);
         uint8_t* qdst = sQ + t * C::QTILE;
@@ -370,58 +425,97 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
         fence_async_smem();
         mbar_arrive(smem_u32(q_full + t));
 
-        for (int j = 0; j < ntiles; ++j) {
-          const int nvalid = min(C::PPT, npages - j * C::PPT);
-          const int my_tile_in_item = j;
-          // page records of this KV tile (logical page | needs-mask flag); same addresses for all threads
-          uint32_t bits[C::PPT];   // allowed positions of this row inside each page of the tile
-          bool tile_mask = nvalid < C::PPT;
+        // Page records (logical page | needs-mask flag; same addresses for all threads) and the
+        // allowed-position bits of this row run two halves ahead of the softmax.  The loads are
+        // volatile so that they are issued here and not next to their first use, where their
+        // latency would be exposed on every half.
+        const int2* krec = p.kept + item.page_begin;
+        auto load_recs = [&](int i, uint32_t* rec) {
 #pragma unroll
-          for (int g = 0; g < C::PPT; ++g) {
-            const uint32_t lpf = g < nvalid ? (uint32_t)__ldg(&p.kept[item.page_begin + j * C::PPT + g].y) : 0u;
+          for (int g = 0; g < C::PPH; ++g) {
+            const int pg = i * C::PPH + g;
+            rec[g] = 0xFFFFFFFFu;   // all ones: no such page
+            if (pg < npages) rec[g] = ldg_early(reinterpret_cast<const uint32_t*>(&krec[pg].y));
+          }
+        };
+        auto make_bits = [&](const uint32_t* rec, uint32_t* bits) -> bool {
+          uint32_t any = valid ? 0u : PIE_KEPT_NEEDS_MASK;
+#pragma unroll
+          for (int g = 0; g < C::PPH; ++g) any |= rec[g];
+          if (!(any & PIE_KEPT_NEEDS_MASK)) return false;   // common case: every page fully visible (warp-uniform unless rows are padding)
+#pragma unroll
+          for (int g = 0; g < C::PPH; ++g) {
+            const uint32_t lpf = rec[g];
             bits[g] = 0xFFFFFFFFu;
-            if (g >= nvalid || !valid) {
+            if (lpf == 0xFFFFFFFFu || !valid) {
               bits[g] = 0u;
-              tile_mask = true;
             } else if (lpf & PIE_KEPT_NEEDS_MASK) {
               const int j0 = (int)(lpf & ~PIE_KEPT_NEEDS_MASK) * P;
-              if (explicit_mask) bits[g] = __ldg(mrow + (j0 >> 5)) >> (j0 & 31);
+              if (explicit_mask) bits[g] = ldg_early(mrow + (j0 >> 5)) >> (j0 & 31);
               else bits[g] = lim >= j0 + P - 1 ? 0xFFFFFFFFu : (lim < j0 ? 0u : ((1u << (lim - j0 + 1)) - 1u));
-              tile_mask = true;
             }
           }
-          mbar_wait(smem_u32(s_full + t), my_tiles & 1, p.status);
-          ++my_tiles;
+          return true;
+        };
+        uint32_t rec_nxt[C::PPH], bits_nxt[C::PPH], bits[C::PPH];
+#pragma unroll
+        for (int g = 0; g < C::PPH; ++g) bits_nxt[g] = 0xFFFFFFFFu;
+        bool mask_nxt;
+        load_recs(0, rec_nxt);
+        mask_nxt = make_bits(rec_nxt, bits_nxt);
+        load_recs(1, rec_nxt);
+
+        for (int i = 0; i < nhalf; ++i) {
+          const int h = i & 1;
+          const uint32_t tSh = tS + h * kHalf;
+          const bool half_mask = mask_nxt;
+#pragma unroll
+          for (int g = 0; g < C::PPH; ++g) bits[g] = bits_nxt[g];
+          mask_nxt = make_bits(rec_nxt, bits_nxt);   // half i + 1 (all "no such page" past the end)
+          load_recs(i + 2, rec_nxt);
+
+          mbar_wait(smem_u32(s_full + 2 * t + h), (s_ph >> h) & 1, p.status);
+          s_ph ^= 1u << h;
           tc_fence_after();
-          // ---- one pass over the row in 32-column chunks (online softmax with a lagging reference):
-          // P = exp2(S * scale - m_ref) goes back as bf16 over the first 64 columns of S_t.  m_ref may
+          // ---- one pass over the half in 32-column chunks (online softmax with a lagging reference):
+          // P = exp2(S * scale - m_ref) goes back as bf16 over the first 32 columns of S_t^h.  m_ref may
           // lag the true running maximum by up to 2^8; when a chunk exceeds that (rare after the first
-          // chunk of an item), O_t, the sums and the P chunks already written for this tile are brought
+          // chunk of an item), O_t, the sums and the P chunk already written for this half are brought
           // to the new reference.  Scale-and-shift and the row sum use packed fp32x2 arithmetic.
-          uint64_t psum2 = pack_f32x2(0.f, 0.f);
+          uint64_t psum_a = pack_f32x2(0.f, 0.f), psum_b = pack_f32x2(0.f, 0.f);
           const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
-          float xbuf[2][32];   // double buffer: chunk k+1 is in flight while chunk k is processed
-          tmem_ld32(tS, reinterpret_cast<uint32_t*>(xbuf[0]));
+          float xbuf[2][32];   // double buffer: chunk 1 is in flight while chunk 0 is processed
+          tmem_ld32(tSh, reinterpret_cast<uint32_t*>(xbuf[0]));
           tmem_wait_ld();
 #pragma unroll
-          for (int k = 0; k < kTileN / 32; ++k) {
+          for (int k = 0; k < kHalf / 32; ++k) {
             float* x = xbuf[k & 1];
-            if (k + 1 < kTileN / 32) tmem_ld32(tS + (k + 1) * 32, reinterpret_cast<uint32_t*>(xbuf[(k + 1) & 1]));
-            if (tile_mask) {
+            if (k + 1 < kHalf / 32) tmem_ld32(tSh + (k + 1) * 32, reinterpret_cast<uint32_t*>(xbuf[(k + 1) & 1]));
+            if (half_mask) {
 #pragma unroll
               for (int c = 0; c < 32; ++c)
                 if (!((bits[(k * 32 + c) / P] >> ((k * 32 + c) % P)) & 1u)) x[c] = kNegInf;
             }
-            float cmax = kNegInf;
+            float cm0 = max3(x[0], x[1], x[2]), cm1 = max3(x[3], x[4], x[5]);   // two chains
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) cmax = max3(cmax, x[c], x[c + 1]);
+            for (int c = 6; c < 30; c += 4) {
+              cm0 = max3(cm0, x[c], x[c + 1]);
+              cm1 = max3(cm1, x[c + 2], x[c + 3]);
+            }
+            const float cmax = fmaxf(max3(cm0, x[30], x[31]), cm1);
             const float m_new = fmaxf(m_ref, cmax * p.scale_log2);   // -inf stays -inf
             if (__any_sync(0xFFFFFFFFu, m_new > m_ref + 8.f)) {       // also when m_ref is -inf and m_new finite
               const float f = (m_ref == kNegInf) ? 1.f : fast_exp2(m_ref - m_new);
               if (m_new != kNegInf) m_ref = m_new;
               l_sum *= f;
-              psum2 = fma_f32x2(psum2, pack_f32x2(f, f), pack_f32x2(0.f, 0.f));
-              if (my_tile_in_item > 0) {   // O_t is complete up to the previous tile (S_t of this tile was issued after it)
+              psum_a = fma_f32x2(psum_a, pack_f32x2(f, f), pack_f32x2(0.f, 0.f));
+              psum_b = fma_f32x2(psum_b, pack_f32x2(f, f), pack_f32x2(0.f, 0.f));
+              if (i > 0) {
+                // O_t holds the PV groups of halves 0..i-1; the latest may still be running.  All but
+                // the latest are known complete (S_t^h of this half was issued after them), so the
+                // barrier is at most one phase behind and the parity wait is unambiguous.
+                mbar_wait(smem_u32(pv_done + t), (n_arr - 1) & 1, p.status);
+                tc_fence_after();
 #pragma unroll 1
                 for (int c0 = 0; c0 < D; c0 += 16) {
                   uint32_t o[16];
@@ -433,17 +527,17 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
                 }
               }
 #pragma unroll 1
-              for (int kk = 0; kk < k; ++kk) {   // P chunks of this tile written under the old reference
+              for (int kk = 0; kk < k; ++kk) {   // P chunks of this half written under the old reference
                 uint32_t pp[16];
                 tmem_wait_st();
-                tmem_ld16(tS + kk * 16, pp);
+                tmem_ld16(tSh + kk * 16, pp);
                 tmem_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                   const float lo = __uint_as_float(pp[c] << 16) * f, hi = __uint_as_float(pp[c] & 0xFFFF0000u) * f;
                   pp[c] = pack_bf16(lo, hi);
                 }
-                tmem_st16(tS + kk * 16, pp);
+                tmem_st16(tSh + kk * 16, pp);
               }
               tmem_wait_st();
             }
@@ -451,26 +545,28 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
             const uint64_t negm2 = pack_f32x2(neg_m, neg_m);
             uint32_t pk[16];
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              float e0, e1;
+            for (int c = 0; c < 32; c += 4) {
+              float e0, e1, e2, e3;
               unpack_f32x2(fma_f32x2(pack_f32x2(x[c], x[c + 1]), scale2, negm2), e0, e1);
-              const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
-              psum2 = add_f32x2(psum2, pack_f32x2(p0, p1));
+              unpack_f32x2(fma_f32x2(pack_f32x2(x[c + 2], x[c + 3]), scale2, negm2), e2, e3);
+              const float p0 = fast_exp2(e0), p1 = fast_exp2(e1), p2 = fast_exp2(e2), p3 = fast_exp2(e3);
+              psum_a = add_f32x2(psum_a, pack_f32x2(p0, p1));
+              psum_b = add_f32x2(psum_b, pack_f32x2(p2, p3));
               pk[c >> 1] = pack_bf16(p0, p1);
+              pk[(c >> 1) + 1] = pack_bf16(p2, p3);
             }
-            tmem_st16(tS + k * 16, pk);   // columns [16k, 16k+16): below every S column still to be read
-            if (k + 1 < kTileN / 32) tmem_wait_ld();
+            tmem_st16(tSh + k * 16, pk);   // columns [16k, 16k+16): below every S column still to be read
+            if (k + 1 < kHalf / 32) tmem_wait_ld();
           }
-          float psum;
           {
             float s0, s1;
-            unpack_f32x2(psum2, s0, s1);
-            psum = s0 + s1;
+            unpack_f32x2(add_f32x2(psum_a, psum_b), s0, s1);
+            l_sum += s0 + s1;
           }
-          l_sum += psum;
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(smem_u32(p_full + t));
+          mbar_arrive(smem_u32(p_full + 2 * t + h));
+          ++n_arr;
         }
         mbar_wait(smem_u32(o_done + t), my_items & 1, p.status);
         ++my_items;
@@ -483,7 +579,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
 #pragma unroll
       for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t o[32];
-        if (ntiles > 0) {
+        if (nhalf > 0) {
           tmem_ld32(tO + c0, o);
           tmem_wait_ld();
         } else {
@@ -512,7 +608,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
         if (item.partial_slot < 0) p.lse[oi] = lse;
         else p.ws_lse[(int64_t)item.partial_slot * 256 + (gr - item.row0)] = lse;
       }
-      if (ntiles > 0) {
+      if (nhalf > 0) {
         tc_fence_before();
         mbar_arrive(smem_u32(o_free + t));
       }
@@ -526,7 +622,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const AttnParams p) {
 }
 
 }  // namespace
-
 bool pie_tc_supported(const pie_ctx* ctx) {
   const pie_config& c = ctx->cfg;
   return c.dtype == PIE_DTYPE_BF16 && (c.page_size == 16 || c.page_size == 32) && (c.head_dim == 64 || c.head_dim == 128);
@@ -542,7 +637,7 @@ static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
     configured[dev] = true;
   }
-  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3(384), C::SMEM, s, p));
+  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3(kThreads), C::SMEM, s, p));
   return PIE_OK;
 }
 
