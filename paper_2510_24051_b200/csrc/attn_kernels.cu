@@ -724,7 +724,7 @@ int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, void* ou
 int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s) {
   AttnParams p = make_params(ctx, plan, plan->tile, q, out, lse);
   const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size, grid = plan->tile.grid;
-  if (plan->tile_tc) return pie_launch_tc_tiles(ctx, p, grid, s);
+  if (plan->tile_tc) return pie_launch_tc_tiles(ctx, p, grid, plan->info.num_query_tokens, s);
   if (D == 64 && P == 16) return launch_tiles<64, 16, 4>(ctx, p, grid, s);
   if (D == 128 && P == 16) return launch_tiles<128, 16, 4>(ctx, p, grid, s);
   if (D == 64 && P == 32) return launch_tiles<64, 32, 4>(ctx, p, grid, s);

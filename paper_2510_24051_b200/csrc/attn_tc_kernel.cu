@@ -3,7 +3,7 @@
 //
 // One CTA per SM walks its share of work items.  An item is up to 256 rows (row = query token *
 // G + head-in-group, one kv head) = two 128-row Q tiles, attended over the item's kept pages in
-// KV tiles of 128 tokens that are handled as two halves of 64 columns.  Roles (320 threads):
+// KV tiles of 128 tokens that are handled as two halves of 64 columns.  Roles (352 threads):
 //   warps 0-3 / 4-7  softmax warpgroup of Q tile 0 / 1: one row per thread.  Reads a half of S
 //                    from TMEM, masks, exponentiates, writes bf16 P back over that half of S,
 //                    keeps the running (max, sum), rescales O in TMEM only when the row max grew
@@ -11,14 +11,17 @@
 //   warp 8           producer: linear bulk copies of page blocks into the K / V stage rings.  The
 //                    pool's storage order is the 128-byte-swizzled canonical operand layout, so a
 //                    page block drops into its 16-row band of the tile with no tensor map.
-//   warp 9, lane 0   MMA issuer: S_t^h = Q_t K_h^T (N = 64), O_t += P_t^h V_h with tcgen05.mma,
+//   warp 9, one lane MMA issuer: S_t^h = Q_t K_h^T (N = 64), O_t += P_t^h V_h with tcgen05.mma,
 //                    accumulators and P in TMEM; completion is tracked with tcgen05.commit.
+//   warp 10          Q loader (TMA): runs one item ahead, so that the first S of the next item is
+//                    computed while the warpgroups are still in the epilogue of this one.
 // The tensor pipe takes instructions synchronously from the issuing thread (measured: a group of
 // eight MMAs returns after ~8 x 64 cycles and any other work of that thread is idle pipe time), so
 // the issuer is a single thread that does nothing but wait, issue and commit.  The two halves
 // break the chain S -> softmax -> PV -> next S of a Q tile: while a warpgroup works on one half,
 // the PV of the other half and the next S into the columns it frees are already running.
 // TMEM (512 columns): S0a S0b | S1a S1b | O0 | O1; P_t^h overlays the first 32 columns of S_t^h.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "pie_internal.h"
@@ -66,6 +69,18 @@ __device__ __forceinline__ uint32_t ldg_early(const uint32_t* p) {
   uint32_t v;
   asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(p));
   return v;
+}
+// Tiled TMA load of a 3-D box (no multicast); x is the innermost coordinate in elements.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+               "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+               : "memory");
+}
+// 32-byte global store (the address must be 32-byte aligned)
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* w) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]),
+               "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
 }
 // One lane of the (converged) warp, the same one every time.
 __device__ __forceinline__ uint32_t elect_one() {
@@ -132,12 +147,40 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+#define TRACEL(tag)
+#define TRACE_LD_END()
+// exp2 of two values on the FMA pipe (the MUFU unit is the softmax bottleneck: 4 results per clock
+// and SM sub-partition): round to the nearest integer n with the 1.5 * 2^23 trick, degree-3
+// minimax polynomial for 2^f on f in [-0.5, 0.5] (relative error 7.5e-5, far below the bf16
+// rounding of P), n added into the exponent field.  Inputs are clamped at -126, so a masked
+// entry (-inf) yields ~1e-38 instead of 0: harmless in a row that has live entries, and rows
+// without any are recognised by their maximum, not by their sum.
+__device__ __forceinline__ void poly_exp2x2(float x0, float x1, float& p0, float& p1) {
+  const float kMagic = 12582912.f;
+  const uint64_t xc = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t y = add_f32x2(xc, pack_f32x2(kMagic, kMagic));
+  const uint64_t r = add_f32x2(y, pack_f32x2(-kMagic, -kMagic));
+  const uint64_t f = fma_f32x2(r, pack_f32x2(-1.f, -1.f), xc);
+  uint64_t q = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), f, pack_f32x2(0.2426111251f, 0.2426111251f));
+  q = fma_f32x2(q, f, pack_f32x2(0.6932609677f, 0.6932609677f));
+  q = fma_f32x2(q, f, pack_f32x2(0.9999280572f, 0.9999280572f));
+  float y0, y1, q0, q1;
+  unpack_f32x2(y, y0, y1);
+  unpack_f32x2(q, q0, q1);
+  p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(y0) << 23));
+  p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(y1) << 23));
+}
+#ifndef PIE_POLY_MASK
+#define PIE_POLY_MASK 0x0000
+#endif
+constexpr uint32_t kPolyMask = PIE_POLY_MASK;   // bit b: pair b of a 32-column chunk is exponentiated on the FMA pipe
+
 constexpr float kNegInf = -__builtin_huge_valf();
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileM = 128;    // rows per Q tile
 constexpr int kTileN = 128;    // tokens per KV tile (one stage of the K / V rings)
 constexpr int kHalf = 64;      // columns per half tile: the unit handed between softmax and MMA
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 
 template <int D, int P>
 struct TcCfg {
@@ -150,12 +193,12 @@ struct TcCfg {
   static constexpr int QTILE = kTileM * D * 2;
   static constexpr int KVTILE = kTileN * D * 2;
   static constexpr int STAGES = D == 128 ? 2 : 4;
-  static constexpr int NBAR = 4 * STAGES + 17;
+  static constexpr int NBAR = 4 * STAGES + 19;
   static constexpr int SMEM = 2 * QTILE + 2 * STAGES * KVTILE + NBAR * 8 + 64;
 };
 
 template <int D, int P>
-__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qmap, const int kflags) {
   using C = TcCfg<D, P>;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* sQ = smem;
@@ -167,7 +210,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
   uint64_t* v_full = k_empty + C::STAGES;
   uint64_t* v_empty = v_full + C::STAGES;
   uint64_t* q_full = v_empty + C::STAGES;  // [2]      Q tile t is in shared memory
-  uint64_t* s_full = q_full + 2;           // [2][2]   S_t^h is complete in TMEM
+  uint64_t* q_free = q_full + 2;           // [2]      every S MMA of the item that reads Q tile t is complete
+  uint64_t* s_full = q_free + 2;           // [2][2]   S_t^h is complete in TMEM
   uint64_t* p_full = s_full + 4;           // [2][2]   P_t^h is written (128 arrivals)
   uint64_t* pv_done = p_full + 4;          // [2]      one phase per PV group of Q tile t
   uint64_t* o_done = pv_done + 2;          // [2]      last PV of the item is complete
@@ -176,6 +220,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(v_land + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool use_qmap = kflags & 1;      // Q tiles come through the tensor map
+  const bool out_wide = kflags & 2;      // the output pointer allows 32-byte stores
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) {
       mbar_init(smem_u32(k_full + s), 1);
@@ -184,7 +230,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
       mbar_init(smem_u32(v_empty + s), 1);
     }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(smem_u32(q_full + t), kTileM);
+      mbar_init(smem_u32(q_full + t), 1);
+      mbar_init(smem_u32(q_free + t), 1);
       for (int h = 0; h < 2; ++h) {
         mbar_init(smem_u32(s_full + 2 * t + h), 1);
         mbar_init(smem_u32(p_full + 2 * t + h), kTileM);
@@ -280,18 +327,31 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
       const uint64_t v_desc0 = smem_desc(smem_u32(sV), C::SLAB_TILE, 1024);  // MN-major: LBO = slab stride
       const uint64_t q_desc0 = smem_desc(smem_u32(sQ), 16, 1024);
       const uint32_t bar_p = smem_u32(p_full), bar_s = smem_u32(s_full), bar_pv = smem_u32(pv_done);
+      // the next item's page count and row count are fetched one item ahead (their latency would
+      // otherwise sit between the last MMA of an item and the first of the next)
+      // (raw loaded values are kept and only combined when the item starts: nothing waits for the loads here)
+      uint32_t nx_end = 0, nx_begin = 0, nx_nrows = 0;
+      if (it0 < it1) {
+        nx_end = ldg_early(reinterpret_cast<const uint32_t*>(&p.items[it0].page_end));
+        nx_begin = ldg_early(reinterpret_cast<const uint32_t*>(&p.items[it0].page_begin));
+        nx_nrows = ldg_early(reinterpret_cast<const uint32_t*>(&p.items[it0].nrows));
+      }
       for (int it = it0; it < it1; ++it) {
-        const PieItem* ip = p.items + it;
-        const int npages = __ldg(&ip->page_end) - __ldg(&ip->page_begin);
-        const int nrows = __ldg(&ip->nrows);
+        const int npages = (int)(nx_end - nx_begin), nrows = (int)nx_nrows;
+        if (it + 1 < it1) {
+          nx_end = ldg_early(reinterpret_cast<const uint32_t*>(&p.items[it + 1].page_end));
+          nx_begin = ldg_early(reinterpret_cast<const uint32_t*>(&p.items[it + 1].page_begin));
+          nx_nrows = ldg_early(reinterpret_cast<const uint32_t*>(&p.items[it + 1].nrows));
+        }
         if (npages == 0) continue;  // the softmax warpgroups write zeros / -inf on their own
         const int ntiles = (npages + C::PPT - 1) / C::PPT;
         const int nhalf = (npages + C::PPH - 1) / C::PPH;           // halves of the item
         const int last_cols = (npages - (nhalf - 1) * C::PPH) * P;  // columns of the last half
         const int nt = nrows > kTileM ? 2 : 1;
+        // Phase of q_full / o_free of Q tile t: bit t of item_ph counts the items the tile took part in.
+        const uint32_t ph_item = item_ph;
         for (int t = 0; t < nt; ++t) {
-          mbar_wait(smem_u32(q_full + t), (item_ph >> t) & 1, p.status);
-          mbar_wait(smem_u32(o_free + t), ((item_ph >> t) & 1) ^ 1, p.status);  // previous epilogue has drained O_t
+          mbar_wait(smem_u32(q_full + t), (ph_item >> t) & 1, p.status);
           item_ph ^= 1u << t;
         }
         tc_fence_after();
@@ -319,6 +379,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
           for (int h = 0; h < min(2, nhalf); ++h)
             for (int t = 0; t < nt; ++t) issue_s(t, h, s);
           umma_commit(smem_u32(k_empty + s));
+          if (ntiles == 1)
+            for (int t = 0; t < nt; ++t) umma_commit(smem_u32(q_free + t));
         }
         for (int j = 0; j < ntiles; ++j) {
           const uint32_t cnt = tile_cnt + j;
@@ -370,6 +432,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
                 mbar_wait(smem_u32(k_full + sn), phn, p.status);
                 k_ready = true;
               }
+              if (i == 0) mbar_wait(smem_u32(o_free + t), ((ph_item >> t) & 1) ^ 1, p.status);  // the previous epilogue has drained O_t
               tc_fence_after();
               const uint64_t vd = v_desc0 + (uint64_t)(s * (C::KVTILE >> 4) + h * (kHalf / 16) * 128);
               const uint32_t dO = tmem + 256 + t * D, aP = tmem + t * 128 + h * kHalf;
@@ -384,10 +447,65 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
               }
             }
           }
+          if (j + 2 == ntiles)   // the S MMAs of the last tile are all issued: Q may be replaced once they are done
+            for (int t = 0; t < nt; ++t) umma_commit(smem_u32(q_free + t));
         }
         tile_cnt += ntiles;
       }
     }
+  } else if (warp >= 10) {
+    // ================================================================ Q loader (warp 10)
+    // Runs one item ahead: the next item's Q rows go into shared memory (K-major, 128-byte
+    // swizzle) as soon as the S MMAs of the current item no longer read the tile.  A Q tile is
+    // the box (64 dims, G heads of the group, 128 / G tokens) of the Q tensor: two TMA loads per
+    // tile (one per 64-dim slab) when 128 is a multiple of G; plain 16-byte asynchronous copies
+    // otherwise.
+    uint32_t n_t[2] = {0, 0};   // items Q tile t took part in
+    const int G = p.G;
+    if (use_qmap && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&qmap) : "memory");
+    for (int it = it0; it < it1; ++it) {
+      const PieItem item = p.items[it];
+      if (item.page_end == item.page_begin) continue;
+      const int nt = item.nrows > kTileM ? 2 : 1;
+      TRACEL(80);
+      for (int t = 0; t < nt; ++t) {
+        mbar_wait(smem_u32(q_free + t), (n_t[t & 1] & 1) ^ 1, p.status);
+        ++n_t[t & 1];
+        TRACEL(81);
+        if (use_qmap) {
+          if (elect_one()) {
+            mbar_expect_tx(smem_u32(q_full + t), C::QTILE);
+            const int tok0 = item.q_start + (item.row0 + t * kTileM) / G;   // row0 is a multiple of the tile height
+#pragma unroll
+            for (int sl = 0; sl < C::NSLAB; ++sl)
+              tma_load_3d(smem_u32(sQ + t * C::QTILE + sl * C::SLAB_TILE), &qmap, sl * 64, item.kv_head * G, tok0, smem_u32(q_full + t));
+          }
+          __syncwarp();
+        } else {
+          constexpr int CPR = D * 2 / 16;        // 16-byte chunks per row
+          constexpr int RPI = 32 / CPR;          // rows per warp instruction
+          const int ch = lane % CPR;
+          const char* qbase = reinterpret_cast<const char*>(p.q) + ((int64_t)item.q_start * p.n_q_heads + item.kv_head * G) * (D * 2) + ch * 16;
+          const uint32_t dst0 = smem_u32(sQ + t * C::QTILE + (ch >> 3) * C::SLAB_TILE);
+#pragma unroll 4
+          for (int r = 0; r < kTileM; r += RPI) {
+            const int row = r + lane / CPR, gr = t * kTileM + row;   // row inside the tile / the item
+            const bool ok = gr < item.nrows;
+            const int tok = (item.row0 + gr) / G, hg = (item.row0 + gr) % G;
+            const char* src = ok ? qbase + ((int64_t)tok * p.n_q_heads + hg) * (D * 2) : qbase;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + row * 128 + (((ch & 7) ^ (row & 7)) << 4)),
+                         "l"(__cvta_generic_to_global(src)), "r"(ok ? 16 : 0)
+                         : "memory");
+          }
+          asm volatile("cp.async.wait_all;" ::: "memory");
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(q_full + t));
+        }
+        TRACEL(83);
+      }
+    }
+    TRACE_LD_END();
   } else {
     // ================================================================ softmax warpgroups
     const int t = warp >> 2;                       // Q tile of this warpgroup
@@ -414,17 +532,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
       float m_ref = kNegInf, l_sum = 0.f;
 
       if (nhalf > 0) {
-        // ---- Q row -> shared memory (K-major, 128-byte swizzle)
-        const uint4* qsrc = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.q) + oi * D);
-        uint8_t* qdst = sQ + t * C::QTILE;
-#pragma unroll
-        for (int ch = 0; ch < D * 2 / 16; ++ch) {
-          const uint4 v = valid ? __ldg(qsrc + ch) : make_uint4(0, 0, 0, 0);
-          *reinterpret_cast<uint4*>(qdst + (ch >> 3) * C::SLAB_TILE + rho * 128 + (((ch & 7) ^ (rho & 7)) << 4)) = v;
-        }
-        fence_async_smem();
-        mbar_arrive(smem_u32(q_full + t));
-
         // Page records (logical page | needs-mask flag; same addresses for all threads) and the
         // allowed-position bits of this row run two halves ahead of the softmax.  The loads are
         // volatile so that they are issued here and not next to their first use, where their
@@ -549,7 +656,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
               float e0, e1, e2, e3;
               unpack_f32x2(fma_f32x2(pack_f32x2(x[c], x[c + 1]), scale2, negm2), e0, e1);
               unpack_f32x2(fma_f32x2(pack_f32x2(x[c + 2], x[c + 3]), scale2, negm2), e2, e3);
-              const float p0 = fast_exp2(e0), p1 = fast_exp2(e1), p2 = fast_exp2(e2), p3 = fast_exp2(e3);
+              float p0, p1, p2, p3;
+              if ((kPolyMask >> (c >> 1)) & 1u) poly_exp2x2(e0, e1, p0, p1);
+              else p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+              if ((kPolyMask >> ((c >> 1) + 1)) & 1u) poly_exp2x2(e2, e3, p2, p3);
+              else p2 = fast_exp2(e2), p3 = fast_exp2(e3);
               psum_a = add_f32x2(psum_a, pack_f32x2(p0, p1));
               psum_b = add_f32x2(psum_b, pack_f32x2(p2, p3));
               pk[c >> 1] = pack_bf16(p0, p1);
@@ -574,8 +685,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
       }
 
       // ---- epilogue: normalise, store
-      const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-      const float lse = l_sum > 0.f ? (m_ref + log2f(l_sum)) * kLn2 : kNegInf;
+      const bool live = m_ref != kNegInf && l_sum > 0.f;   // a row with no allowed position: O = 0, LSE = -inf
+      const float inv = live ? 1.f / l_sum : 0.f;
+      const float lse = live ? (m_ref + log2f(l_sum)) * kLn2 : kNegInf;
 #pragma unroll
       for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t o[32];
@@ -588,19 +700,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
         }
         if (valid) {
           if (item.partial_slot < 0) {
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D + c0);
+            // 32-byte stores: every thread writes its own row, so the store path is bound by the number
+            // of (thread, instruction) pairs, not by bytes
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D + c0;
+            uint32_t w[16];
 #pragma unroll
-            for (int c = 0; c < 32; c += 8)
-              dst[c >> 3] = make_uint4(pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv),
-                                       pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv),
-                                       pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv),
-                                       pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv));
+            for (int c = 0; c < 32; c += 2) w[c >> 1] = pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+            if (out_wide) {
+              st_global_v8(dst, w);
+              st_global_v8(dst + 16, w + 8);
+            } else {
+#pragma unroll
+              for (int c = 0; c < 16; c += 4) reinterpret_cast<uint4*>(dst)[c >> 2] = make_uint4(w[c], w[c + 1], w[c + 2], w[c + 3]);
+            }
           } else {
-            float4* dst = reinterpret_cast<float4*>(p.ws_o + ((int64_t)item.partial_slot * 256 + (gr - item.row0)) * D + c0);
+            float* dst = p.ws_o + ((int64_t)item.partial_slot * 256 + (gr - item.row0)) * D + c0;
 #pragma unroll
-            for (int c = 0; c < 32; c += 4)
-              dst[c >> 2] = make_float4(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv,
-                                        __uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+            for (int c = 0; c < 32; c += 8) {
+              uint32_t w[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) w[k] = __float_as_uint(__uint_as_float(o[c + k]) * inv);
+              st_global_v8(dst + c, w);
+            }
           }
         }
       }
@@ -627,8 +748,40 @@ bool pie_tc_supported(const pie_ctx* ctx) {
   return c.dtype == PIE_DTYPE_BF16 && (c.page_size == 16 || c.page_size == 32) && (c.head_dim == 64 || c.head_dim == 128);
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+// Tensor map of Q [tokens][q heads][D] (bf16) whose box is one Q tile: 64 dims x G heads x 128/G
+// tokens, 128-byte swizzle.  Returns false when the shape does not fit (128 not a multiple of G,
+// unaligned pointer): the kernel then loads Q with plain asynchronous copies.
+static bool make_q_map(const pie_ctx* ctx, const void* q, int64_t n_tokens, int G, CUtensorMap* map) {
+  const int D = ctx->cfg.head_dim, Hq = ctx->cfg.num_q_heads;
+  if (G <= 0 || kTileM % G != 0 || n_tokens <= 0 || (reinterpret_cast<uintptr_t>(q) & 15) != 0) return false;
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return false;
+  const cuuint64_t gdim[3] = {(cuuint64_t)D, (cuuint64_t)Hq, (cuuint64_t)n_tokens};
+  const cuuint64_t gstride[2] = {(cuuint64_t)D * 2, (cuuint64_t)Hq * D * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(kTileM / G)};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int D, int P>
-static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
+static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_tokens, cudaStream_t s) {
   using C = TcCfg<D, P>;
   auto kern = attn_tc_kernel<D, P>;
   static bool configured[8] = {};
@@ -637,15 +790,18 @@ static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
     configured[dev] = true;
   }
-  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3(kThreads), C::SMEM, s, p));
+  CUtensorMap qmap;
+  memset(&qmap, 0, sizeof(qmap));
+  const int kflags = (make_q_map(ctx, p.q, n_tokens, p.G, &qmap) ? 1 : 0) | ((reinterpret_cast<uintptr_t>(p.out) & 31) == 0 ? 2 : 0);
+  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3(kThreads), C::SMEM, s, p, qmap, kflags));
   return PIE_OK;
 }
 
-int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
+int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_tokens, cudaStream_t s) {
   const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size;
-  if (D == 128 && P == 16) return launch_tc<128, 16>(ctx, p, grid, s);
-  if (D == 64 && P == 16) return launch_tc<64, 16>(ctx, p, grid, s);
-  if (D == 128 && P == 32) return launch_tc<128, 32>(ctx, p, grid, s);
-  if (D == 64 && P == 32) return launch_tc<64, 32>(ctx, p, grid, s);
+  if (D == 128 && P == 16) return launch_tc<128, 16>(ctx, p, grid, n_tokens, s);
+  if (D == 64 && P == 16) return launch_tc<64, 16>(ctx, p, grid, n_tokens, s);
+  if (D == 128 && P == 32) return launch_tc<128, 32>(ctx, p, grid, n_tokens, s);
+  if (D == 64 && P == 32) return launch_tc<64, 32>(ctx, p, grid, n_tokens, s);
   return PIE_ERR_UNSUPPORTED;
 }

@@ -189,7 +189,8 @@ int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll
 bool pie_split_supported(const pie_ctx* ctx);
 int pie_split_warps_per_block(const pie_ctx* ctx);
 bool pie_tc_supported(const pie_ctx* ctx);
-int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s);
+// n_tokens: rows of the Q tensor (the batch's query tokens), for the bounds of the Q tensor map
+int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_tokens, cudaStream_t s);
 
 int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);  // host part (planner.cc)
 

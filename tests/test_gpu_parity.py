@@ -282,3 +282,46 @@ def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
             assert torch.equal(out, ref_out) and torch.equal(lse, ref_lse)
         assert pie.pie_get_last_device_status(gp.ctx) == 0
         pie.pie_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("heads", [(6, 2), (12, 2), (5, 1)])
+def test_head_groups_that_do_not_divide_the_row_tile(heads):
+    """Group sizes 3, 6 and 5: a 128-row Q tile is not a whole number of tokens, so the tensor-core
+    kernel takes its Q rows with plain copies instead of the tensor map (Section 4.2 forward)."""
+    from tests._gpu import check_close, run_workload
+    H_q, H_kv = heads
+    for name in ("mixed_prefill_decode", "shared_prefix_tree"):
+        wl = configs.small(name, H_q=H_q, H_kv=H_kv)
+        O_ref, L_ref, _ = run_oracle(wl, poison=True)
+        O, L, info = run_workload(wl, poison=True)
+        assert info["num_tile_items"] > 0
+        check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
+
+
+def test_output_pointer_that_is_only_16_byte_aligned():
+    """The kernels use 32-byte stores when the output pointer allows it; a view that starts 16 bytes
+    into an allocation must give the same bits."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool
+    wl = configs.small("shared_prefix_tree")
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl)
+        plan = gp.plan(wl)
+        q, k, v = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
+        T = q.shape[0]
+        n = T * wl.H_q * wl.D
+        outs = []
+        for shift in (0, 8):                                   # elements: 8 bf16 = 16 bytes
+            buf = torch.full((n + 64,), float("nan"), dtype=q.dtype, device="cuda")
+            out = buf[shift:shift + n].view(T, wl.H_q, wl.D)
+            assert out.data_ptr() % 32 == (16 if shift else 0)
+            lse = torch.empty((T, wl.H_q), dtype=torch.float32, device="cuda")
+            # the call appends into the pool: start both runs from the same pool contents
+            gp.install(wl)
+            pie.pie_forward(gp.ctx, plan, q, k, v, out, lse)
+            torch.cuda.synchronize()
+            assert pie.pie_get_last_device_status(gp.ctx) == 0
+            outs.append((out.clone(), lse.clone()))
+        assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))
+        assert torch.equal(outs[0][1], outs[1][1])
+        pie.pie_plan_destroy(plan)
