@@ -196,7 +196,9 @@ int pie_plan_debug_read(const pie_plan* plan, int which, void* buf, int64_t cap_
  * [T][H_kv][D], out [T][H_q][D] in the configured element type, lse [T][H_q] fp32 (natural log
  * of the sum of exp of the scaled scores).  Enqueues on `stream`: append of the new rows into
  * the pool, then attention (scale 1/sqrt(D)) reading the pool, then the merge of split
- * partials.  The plan may be reused for repeated calls with the same batch structure. */
+ * partials.  The plan may be reused for repeated calls with the same batch structure.
+ * All five pointers must be 16-byte aligned (rows are moved in 16-byte pieces); an `out` that
+ * is 32-byte aligned is written with wider stores, with identical results. */
 int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new,
                 const void* v_new, void* out, float* lse, void* stream);
 
