@@ -360,6 +360,8 @@ def main():
         qo_bytes = int(wl0.q_lens()[sel].sum()) * wl0.H_q * (2 * wl0.D * wl0.esize + 4)
         mask_bytes = 0 if wl0.masks is None else sum((m.size + 7) // 8 for m, s in zip(wl0.masks, sel) if s and m is not None)
         alg = kv_bytes + qo_bytes + mask_bytes
+        if dom == "split" and ktimes["append"][1] == 0:   # fused append: the split-KV kernel also moves the new rows
+            alg += int(wl0.q_lens()[sel].sum()) * b_tok * 2
         achieved = alg / (dom_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(wl0.name),

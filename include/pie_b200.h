@@ -278,8 +278,13 @@ int pie_sched_next_batch(pie_sched* s, int32_t* out_type, int32_t cap, int64_t* 
  *                      kernel), 1 = side by side on disjoint SM sets, the second on an internal
  *                      stream that forks from and joins the caller's stream.  Pays only when the
  *                      tensor-bound part is long against the HBM-bound part: the decode kernel
- *                      needs about 60 % of the SMs to keep the memory system saturated. */
-enum { PIE_OPT_SPLIT_SMS = 0, PIE_OPT_TILE_SMS = 1, PIE_OPT_OVERLAP = 2, PIE_NUM_OPTIONS = 3 };
+ *                      needs about 60 % of the SMs to keep the memory system saturated.
+ *   PIE_OPT_NO_FUSION  1 = always launch the append kernel.  By default (0) a decode batch
+ *                      (every request one new token, all on the split-KV kernel, no request
+ *                      listing a page another one appends to) lets the attention kernel write
+ *                      the new K/V rows itself, which saves the append launch; results and
+ *                      pool contents are bit-identical either way. */
+enum { PIE_OPT_SPLIT_SMS = 0, PIE_OPT_TILE_SMS = 1, PIE_OPT_OVERLAP = 2, PIE_OPT_NO_FUSION = 3, PIE_NUM_OPTIONS = 4 };
 int pie_set_option(pie_ctx* ctx, int option, int value);
 
 /* Per-kernel device timing for benchmarks.  While enabled, pie_forward and pie_copy_kvpage

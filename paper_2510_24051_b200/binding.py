@@ -268,7 +268,7 @@ def pie_forward_static_scratch(ctx, qo_indptr, page_indptr, page_indices, last_p
                                           _ptr(lse), _stream(stream)), ctx)
 
 
-PIE_OPT_SPLIT_SMS, PIE_OPT_TILE_SMS, PIE_OPT_OVERLAP = 0, 1, 2
+PIE_OPT_SPLIT_SMS, PIE_OPT_TILE_SMS, PIE_OPT_OVERLAP, PIE_OPT_NO_FUSION = 0, 1, 2, 3
 
 
 def pie_set_option(ctx, option, value):

@@ -211,6 +211,7 @@ int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, con
 int pie_append_and_q(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new, const void* v_new, cudaStream_t s,
                      const void** q_eff) {
   *q_eff = q;
+  if (plan->append_fused) return PIE_OK;  // the split-KV kernel writes the new rows itself
   if (ctx->cfg.rope_theta > 0.f) {  // positions inside the path: rotated K goes to the pages, attention reads rotated Q
     *q_eff = ctx->d_qrot;
     return pie_launch_rope(ctx, plan, q, k_new, v_new, s);
@@ -565,7 +566,8 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
   cudaStream_t s = (cudaStream_t)stream;
   PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
   const void* q_in = q;
-  int rc = timed_launch(ctx, PIE_KERNEL_APPEND, s, [&] { return pie_append_and_q(ctx, plan, q_in, k_new, v_new, s, &q); });
+  int rc = plan->append_fused ? PIE_OK  // (q stays q_in: the split-KV kernel writes the new rows itself)
+                              : timed_launch(ctx, PIE_KERNEL_APPEND, s, [&] { return pie_append_and_q(ctx, plan, q_in, k_new, v_new, s, &q); });
   if (rc) return rc;
   if (!plan->simple_rows.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_SIMPLE, s, [&] { return pie_launch_simple(ctx, plan, q, out, lse, s); })))
@@ -591,7 +593,7 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
       (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s2, [&] { return pie_launch_merge(ctx, plan, plan->tile, out, lse, s2); })))
     return rc;
   if (!plan->split.items.empty() &&
-      (rc = timed_launch(ctx, PIE_KERNEL_SPLIT, s, [&] { return pie_launch_split(ctx, plan, q, out, lse, s); })))
+      (rc = timed_launch(ctx, PIE_KERNEL_SPLIT, s, [&] { return pie_launch_split(ctx, plan, q, k_new, v_new, out, lse, s); })))
     return rc;
   if (!plan->split.merges.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s, [&] { return pie_launch_merge(ctx, plan, plan->split, out, lse, s); })))

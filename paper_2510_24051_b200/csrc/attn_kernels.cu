@@ -267,7 +267,7 @@ template <int D, int P, int NW, int DEPTH>
 struct SplitCfg {
   static constexpr int STAGE = 2 * P * D * 2;
   static constexpr int QUEUE = 8;  // chunk ids a warp has started fetching but not finished (<= DEPTH + 2)
-  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * 12 + NW * QUEUE * 4 + 64;
+  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * 16 + NW * QUEUE * 4 + 64;
 };
 
 template <int D, int P, int NW, int DEPTH>
@@ -279,7 +279,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   uint8_t* stages = smem + warp * DEPTH * C::STAGE;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + NW * DEPTH * C::STAGE) + warp * DEPTH;
   volatile uint32_t* meta = reinterpret_cast<uint32_t*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 8) + warp * DEPTH;
-  volatile int* queue = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 12) + warp * C::QUEUE;
+  volatile int* meta_phys = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 12) + warp * DEPTH;
+  volatile int* queue = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 16) + warp * C::QUEUE;
   pie_pdl_launch_dependents();
   if (lane == 0) {
     for (int s = 0; s < DEPTH; ++s) mbar_init(smem_u32(full_bar + s), 1);
@@ -362,6 +363,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   auto issue = [&](int n, int2 rec, int head) {
     const uint32_t s = n % DEPTH;
     meta[s] = (uint32_t)rec.y;  // logical page | needs-mask flag, read back by the warp after the wait
+    meta_phys[s] = rec.x;       // physical page (the fused append writes its row back to it)
     mbar_expect_tx(smem_u32(full_bar + s), C::STAGE);
     bulk_g2s(smem_u32(stages + s * C::STAGE), p.pool + ((int64_t)rec.x * p.n_kv_heads + head) * C::STAGE, C::STAGE,
              smem_u32(full_bar + s));
@@ -410,6 +412,16 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
     rq.mask_word_off = item.mask_word_off;
     rq.last_logical = item.last_logical;
     rq.last_page_len = item.last_page_len;
+    // Fused append (decode batches): this piece ends with the request's last page, so this warp
+    // also owns the request's one new K/V row of its kv head.  The row's 16-byte chunks are
+    // fetched now (lanes [0, CH): K, [CH, 2 CH): V) and written, once the page has landed, into
+    // the staged copy and into the pool at the same offset (the stage is an image of the block).
+    constexpr int CH = D * 2 / 16;
+    const bool do_append = (item.flags & PIE_ITEM_APPEND) != 0;
+    uint4 new_chunk = make_uint4(0, 0, 0, 0);
+    if (do_append && lane < 2 * CH)
+      new_chunk = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(lane < CH ? p.k_new : p.v_new) +
+                                                       ((int64_t)item.q_start * p.n_kv_heads + item.kv_head) * (D * 2)) + (lane % CH));
     RowState<D> st;
     rows_init<D>(st, p, item, rq, item.row0, lane);
     for (int k = item.page_begin; k < item.page_end; ++k, ++n) {
@@ -418,6 +430,17 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
       if (pf_live) rec_next = __ldg(&p.kept[pf_k]);  // latency hides behind the wait
       mbar_wait(smem_u32(full_bar + s), ph, p.status);
       const uint32_t lpf = meta[s];
+      if (do_append && (int)(lpf & ~PIE_KEPT_NEEDS_MASK) == item.last_logical) {
+        if (lane < 2 * CH) {
+          const int off = (lane < CH ? 0 : C::STAGE / 2) + pie_chunk_offset(P * 128, item.last_page_len - 1, lane % CH);
+          *reinterpret_cast<uint4*>(stages + s * C::STAGE + off) = new_chunk;
+          const int phys = meta_phys[s];
+          *reinterpret_cast<uint4*>(const_cast<uint8_t*>(p.pool) + ((int64_t)phys * p.n_kv_heads + item.kv_head) * C::STAGE + off) = new_chunk;
+        }
+        // the generic-proxy write must be ordered before the bulk copy that later refills the stage
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+      }
       page_compute<D, P>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
       __syncwarp();
       if (pf_live) {
@@ -710,8 +733,11 @@ int pie_split_warps_per_block(const pie_ctx* ctx) {
   return (ctx->cfg.page_size == 32 && ctx->cfg.head_dim == 128) ? 4 : 8;
 }
 
-int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s) {
+int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new, const void* v_new, void* out,
+                     float* lse, cudaStream_t s) {
   AttnParams p = make_params(ctx, plan, plan->split, q, out, lse);
+  p.k_new = k_new;
+  p.v_new = v_new;
   const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size, n = plan->split.grid, ni = (int)plan->split.items.size();
   // ring depth: about 192 KB of copies in flight per SM
   if (D == 64 && P == 16) return launch_split<64, 16, 8, 6>(ctx, p, ni, n, s);
@@ -800,10 +826,12 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
 
   pie_plan plan;  // host-side only; its device pointers will point into the static scratch
   plan.ctx = ctx;
-  const int saved_overlap = ctx->options[PIE_OPT_OVERLAP];
-  ctx->options[PIE_OPT_OVERLAP] = 0;  // this entry point enqueues its kernels one after the other
+  const int saved_overlap = ctx->options[PIE_OPT_OVERLAP], saved_fusion = ctx->options[PIE_OPT_NO_FUSION];
+  ctx->options[PIE_OPT_OVERLAP] = 0;    // this entry point enqueues its kernels one after the other
+  ctx->options[PIE_OPT_NO_FUSION] = 1;  // and keeps the separate append launch
   int rc = pie_build_plan(ctx, batch, &plan);
   ctx->options[PIE_OPT_OVERLAP] = saved_overlap;
+  ctx->options[PIE_OPT_NO_FUSION] = saved_fusion;
   if (rc != PIE_OK) return rc;
   if (plan.T == 0) return PIE_OK;
   if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
@@ -863,7 +891,7 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   }
   if ((rc = pie_append_and_q(ctx, &plan, q, k_new, v_new, s, &q))) return rc;
   if (!plan.simple_rows.empty() && (rc = pie_launch_simple(ctx, &plan, q, out, lse, s))) return rc;
-  if (!plan.split.items.empty() && (rc = pie_launch_split(ctx, &plan, q, out, lse, s))) return rc;
+  if (!plan.split.items.empty() && (rc = pie_launch_split(ctx, &plan, q, k_new, v_new, out, lse, s))) return rc;
   if (!plan.tile.items.empty() && (rc = pie_launch_tiles(ctx, &plan, q, out, lse, s))) return rc;
   if (!plan.split.merges.empty() && (rc = pie_launch_merge(ctx, &plan, plan.split, out, lse, s))) return rc;
   if (!plan.tile.merges.empty() && (rc = pie_launch_merge(ctx, &plan, plan.tile, out, lse, s))) return rc;

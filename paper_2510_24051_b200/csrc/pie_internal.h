@@ -54,10 +54,14 @@ struct PieItem {
   int32_t page_begin, page_end;  // absolute indices into the kept-page list
   int32_t partial_slot;          // -1: write the final output; else slot of the fp32 partial
   // copy of the request record, so that a kernel can start an item from this one 64-byte line
-  int32_t q_start, q_len, kv_len, mask_row_words, last_logical, last_page_len, pad;
+  int32_t q_start, q_len, kv_len, mask_row_words, last_logical, last_page_len;
+  uint32_t flags;                // PIE_ITEM_*
   int64_t mask_word_off;
 };
 static_assert(sizeof(PieItem) == 64, "PieItem is one 64-byte line");
+// The split-KV warp that owns this item also writes the request's one new K/V row (decode batches
+// whose append is fused into the attention kernel): into the pool and into its staged copy of the page.
+#define PIE_ITEM_APPEND 1u
 
 // A group of partial slots that the merge kernel combines into final rows.
 struct PieMerge {
@@ -99,6 +103,7 @@ struct pie_plan {
   PieLaunchList split, tile;
   bool tile_tc = false;             // row tiles run on the tcgen05 kernel (256-row items)
   bool overlap = false;             // decode and tile kernels run side by side on disjoint SM sets
+  bool append_fused = false;        // the split-KV kernel writes the new K/V rows itself (no append launch)
   pie_plan_info info{};
   // device
   void* d_blob = nullptr;           // one allocation holding every array below
@@ -138,7 +143,7 @@ struct pie_ctx {
   size_t h_stage_bytes = 0;
   pie_plan* host_plan = nullptr;  // reused plan object of pie_forward_host
   std::string cuda_error;
-  int options[PIE_NUM_OPTIONS] = {0, 0, 0};
+  int options[PIE_NUM_OPTIONS] = {0, 0, 0, 0};
   cudaStream_t side_stream = nullptr;  // second stream of overlapped mixed batches
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   // optional per-kernel timing (pie_set_kernel_timing)
@@ -168,6 +173,8 @@ struct AttnParams {
   int32_t slot_rows;
   float* ws_o;
   float* ws_lse;
+  const void* k_new;         // fused append: new rows [T][H_kv][D]
+  const void* v_new;
   int* status;
   int64_t page_bytes;
   int32_t n_q_heads, n_kv_heads, G;
@@ -183,7 +190,8 @@ int pie_append_and_q(pie_ctx* ctx, const pie_plan* plan, const void* q, const vo
 int pie_launch_copy(pie_ctx* ctx, int n, const int32_t* d_ops, cudaStream_t s);
 int pie_launch_page_io(pie_ctx* ctx, int n, const int32_t* d_ids, void* K, void* V, bool write, cudaStream_t s);
 int pie_launch_simple(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);
-int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);
+int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k_new, const void* v_new, void* out,
+                     float* lse, cudaStream_t s);
 int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);
 int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s);
 bool pie_split_supported(const pie_ctx* ctx);

@@ -245,6 +245,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     q.last_page_len = last;
   }
 
+  bool cross_read = false;  // some request lists a page that another request of the batch appends to
   // ---- conflict rule: no slot is written twice, and no request reads a slot that a later request
   // of the batch writes (rows appended by an earlier request are visible: append precedes attention)
   {
@@ -252,6 +253,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     struct SharedWrite { int32_t page, req; uint32_t mask; };
     std::vector<SharedWrite> shared;  // pages written by more than one request: who wrote which slots
     int status = PIE_OK;
+    cross_read = false;
     auto slot_mask = [&](int lo, int hi) -> uint32_t {  // bits [lo, hi)
       uint32_t m = (hi >= 32) ? 0xFFFFFFFFu : ((1u << hi) - 1u);
       return m & ~((1u << lo) - 1u);
@@ -285,6 +287,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
         int32_t pg = pages[lp];
         uint32_t w = ctx->wmask[pg];
         if (w == 0 || ctx->writer[pg] == r) continue;
+        cross_read = true;  // a page one request appends to is in another request's list
         if (ctx->writer[pg] >= 0 && ctx->writer[pg] < r) continue;  // written by an earlier request: visible
         uint32_t rd = slot_mask(0, lp == q.last_logical ? q.last_page_len : P);
         if (ctx->writer[pg] == -2) {  // several writers: only slots written by LATER requests conflict
@@ -508,9 +511,27 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   }
   partition(tile_units, tile_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile);
 
+  // ---- fused append of the decode path (PIE_OPT_NO_FUSION switches it off): when every request brings exactly one new token, all of them run on the split-KV
+  // kernel, their last page is in the kept list and no request lists a page another one appends
+  // to, the warp that attends a request's last page also writes the new K/V row (into the pool
+  // and into its staged copy), and the append launch is dropped.
+  const int no_fusion = ctx->options[PIE_OPT_NO_FUSION];
+  plan->append_fused = false;
+  if (!(no_fusion & 1) && ctx->cfg.rope_theta <= 0.f && !cross_read && !plan->split.items.empty() &&
+      plan->tile.items.empty() && plan->simple_rows.empty()) {
+    bool ok = true;
+    for (int r = 0; r < R && ok; ++r) {
+      const PieReq& q = plan->reqs[r];
+      ok = q.q_len == 1 && q.kept_count > 0 &&
+           (int)((uint32_t)plan->kept[2 * (size_t)(q.kept_start + q.kept_count - 1) + 1] & ~PIE_KEPT_NEEDS_MASK) == q.last_logical;
+    }
+    plan->append_fused = ok;
+  }
   for (PieLaunchList* ll : {&plan->split, &plan->tile})
     for (PieItem& it : ll->items) {
       const PieReq& q = plan->reqs[it.req];
+      it.flags = 0;
+      if (ll == &plan->split && plan->append_fused && it.page_end == q.kept_start + q.kept_count) it.flags |= PIE_ITEM_APPEND;
       it.q_start = q.q_start;
       it.q_len = q.q_len;
       it.kv_len = q.kv_len;
@@ -531,7 +552,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   info.mask_words = (int64_t)plan->mask_words.size();
   info.workspace_bytes = ((int64_t)plan->split.n_slots * plan->split.slot_rows +
                           (int64_t)plan->tile.n_slots * plan->tile.slot_rows) * (cfg.head_dim + 1) * 4;
-  info.launches = 1 + (info.num_simple_rows ? 1 : 0) + (info.num_split_items ? 1 : 0) +
+  info.launches = (plan->append_fused ? 0 : 1) + (info.num_simple_rows ? 1 : 0) + (info.num_split_items ? 1 : 0) +
                   (info.num_tile_items ? 1 : 0) + (plan->split.merges.empty() ? 0 : 1) +
                   (plan->tile.merges.empty() ? 0 : 1);
   return PIE_OK;

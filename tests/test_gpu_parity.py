@@ -325,3 +325,33 @@ def test_output_pointer_that_is_only_16_byte_aligned():
         assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))
         assert torch.equal(outs[0][1], outs[1][1])
         pie.pie_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("name", ["batched_decode", "long_context_policy"])
+def test_fused_append_equals_the_separate_launch(name):
+    """Decode batches let the split-KV kernel write the new K/V rows itself (one launch fewer);
+    switching the fusion off must give the same bits in O, LSE and the pool."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs.small(name)
+    results = []
+    for no_fusion in (0, 1):
+        with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+            pie.pie_set_option(gp.ctx, pie.PIE_OPT_NO_FUSION, no_fusion)
+            gp.install(wl, poison=True)
+            plan = gp.plan(wl)
+            info = pie.pie_plan_get_info(plan)
+            out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+            K, V = gp.read_pages(wl.used_pages())
+            pie.pie_plan_destroy(plan)
+            results.append((info["launches"], out.view(torch.int16).cpu(), lse.cpu(), K, V))
+    fused, plain = results
+    assert plain[0] == fused[0] + 1
+    assert torch.equal(fused[1], plain[1]) and torch.equal(fused[2], plain[2])
+    assert same_bits(fused[3], plain[3]) and same_bits(fused[4], plain[4])
+    # and the fused run matches the oracle like any other
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    check_close(fused[1].view(torch.bfloat16).double().numpy(), fused[2].double().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+    for n, pg in enumerate(wl.used_pages()):
+        Ko, Vo = pool[int(pg)]
+        assert same_bits(fused[3][n], Ko) and same_bits(fused[4][n], Vo), f"page {pg}"
