@@ -153,7 +153,9 @@ typedef struct pie_batch_desc {
 
 enum {
   PIE_PLAN_FORCE_SIMPLE = 1u,   /* run every request through the plain CUDA-core kernel   */
-  PIE_PLAN_NO_TENSOR_TILES = 2u /* keep prefill / tree requests off the tcgen05 tile path */
+  PIE_PLAN_NO_TENSOR_TILES = 2u, /* keep prefill / tree requests off the tcgen05 tile path */
+  PIE_PLAN_NO_CASCADE = 4u,     /* never attend a shared prefix once for a group of requests */
+  PIE_PLAN_CASCADE_ALWAYS = 8u  /* cascade every shared prefix, however small the saving (tests, tuning) */
 };
 
 typedef struct pie_plan_info {

@@ -14,7 +14,7 @@ import numpy as np
 from . import build as _build
 
 PIE_DTYPE_BF16, PIE_DTYPE_F32 = 0, 1
-PIE_PLAN_FORCE_SIMPLE, PIE_PLAN_NO_TENSOR_TILES = 1, 2
+PIE_PLAN_FORCE_SIMPLE, PIE_PLAN_NO_TENSOR_TILES, PIE_PLAN_NO_CASCADE, PIE_PLAN_CASCADE_ALWAYS = 1, 2, 4, 8
 PIE_OK = 0
 PIE_ERR_INVALID, PIE_ERR_NO_PAGES, PIE_ERR_BAD_PAGE, PIE_ERR_CONFLICT = -1, -2, -3, -4
 PIE_ERR_BATCH_TOO_LARGE, PIE_ERR_MASK, PIE_ERR_CUDA, PIE_ERR_NO_DEVICE = -5, -6, -7, -8

@@ -550,10 +550,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) attn_tile_kernel(const AttnP
 template <typename T, int D>
 __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* __restrict__ reqs,
                              const float* __restrict__ ws_o, const float* __restrict__ ws_lse, T* __restrict__ out,
-                             float* __restrict__ lse_out, int slot_rows, int n_q_heads, int G) {
+                             float* __restrict__ lse_out, int slot_rows, int n_q_heads, int G,
+                             const float* __restrict__ x_ws_o, const float* __restrict__ x_ws_lse, int x_slot_rows) {
   // One warp per (merge group, row).  Lanes share the slots for the max and the weights, then each
   // lane owns D/32 consecutive columns and the slot loop issues independent, coalesced row loads.
   // (Every partial row is written by its kernel, with zeros when its part of the context was empty.)
+  // A group may name further partials of its rows in the row-tile launch's workspace (x_*: the
+  // shared-prefix cascade); they are combined after the group's own slots.
   constexpr int EPL = D / 32;
   pie_pdl_launch_dependents();
   pie_pdl_wait();
@@ -562,25 +565,32 @@ __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* 
   const int row = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= mg.nrows) return;
   const PieReq rq = reqs[mg.req];
-  const float* lse_in = ws_lse + (int64_t)mg.slot0 * slot_rows + row;
-  const float* o_in = ws_o + ((int64_t)mg.slot0 * slot_rows + row) * D + lane * EPL;
-  const int64_t slot_stride = (int64_t)slot_rows * D;
+  const int ntot = mg.nslots + mg.x_nslots;
+  // source c: own slot c, or cascade slot c - nslots
+  auto lse_of = [&](int c) -> float {
+    return c < mg.nslots ? ws_lse[(int64_t)(mg.slot0 + c) * slot_rows + row]
+                         : x_ws_lse[(int64_t)(mg.x_slot0 + c - mg.nslots) * x_slot_rows + mg.x_row0 + row];
+  };
+  auto row_of = [&](int c) -> const float* {
+    return c < mg.nslots ? ws_o + ((int64_t)(mg.slot0 + c) * slot_rows + row) * D + lane * EPL
+                         : x_ws_o + ((int64_t)(mg.x_slot0 + c - mg.nslots) * x_slot_rows + mg.x_row0 + row) * D + lane * EPL;
+  };
   float M = kNegInf;
-  for (int c = lane; c < mg.nslots; c += 32) M = fmaxf(M, lse_in[(int64_t)c * slot_rows]);
+  for (int c = lane; c < ntot; c += 32) M = fmaxf(M, lse_of(c));
   for (int sft = 16; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));
   float Z = 0.f, acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  for (int base = 0; base < mg.nslots; base += 32) {
+  for (int base = 0; base < ntot; base += 32) {
     const int c = base + lane;
     float w = 0.f;
-    if (c < mg.nslots && M != kNegInf) w = __expf(lse_in[(int64_t)c * slot_rows] - M);  // exp(-inf) = 0
+    if (c < ntot && M != kNegInf) w = __expf(lse_of(c) - M);  // exp(-inf) = 0
     Z += w;
-    const int cnt = min(32, mg.nslots - base);
+    const int cnt = min(32, ntot - base);
 #pragma unroll 4
     for (int u = 0; u < cnt; ++u) {
       const float wu = __shfl_sync(0xFFFFFFFFu, w, u);
-      const float* src = o_in + (base + u) * slot_stride;
+      const float* src = row_of(base + u);
       if constexpr (EPL == 4) {
         const float4 v = *reinterpret_cast<const float4*>(src);
         acc[0] += wu * v.x, acc[1] += wu * v.y, acc[2] += wu * v.z, acc[3] += wu * v.w;
@@ -765,7 +775,8 @@ int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll
 #define PIE_MERGE(T, DD)                                                                                          \
   PIE_CUDA(ctx, pie_launch_pdl(merge_kernel<T, DD>, n, dim3(wpb * 32), 0, s, (const PieMerge*)ll.d_merges,      \
                                (const PieReq*)plan->d_reqs, (const float*)ll.d_ws_o, (const float*)ll.d_ws_lse, \
-                               (T*)out, lse, ll.slot_rows, ctx->cfg.num_q_heads, ctx->G))
+                               (T*)out, lse, ll.slot_rows, ctx->cfg.num_q_heads, ctx->G,                         \
+                               (const float*)plan->tile.d_ws_o, (const float*)plan->tile.d_ws_lse, plan->tile.slot_rows))
   if (ctx->cfg.dtype == PIE_DTYPE_BF16) {
     if (D == 64) PIE_MERGE(__nv_bfloat16, 64);
     else PIE_MERGE(__nv_bfloat16, 128);

@@ -67,6 +67,10 @@ static_assert(sizeof(PieItem) == 64, "PieItem is one 64-byte line");
 struct PieMerge {
   int32_t req, kv_head, row0, nrows;
   int32_t slot0, nslots;
+  // Shared-prefix cascade: further partials of the same rows, written by the row-tile launch for a
+  // group of requests at once.  They sit in that launch's workspace, slots [x_slot0, x_slot0 +
+  // x_nslots), where this group's rows start at row x_row0 of the slot (x_nslots = 0: none).
+  int32_t x_slot0, x_nslots, x_row0;
 };
 
 #define PIE_KEPT_NEEDS_MASK 0x80000000u

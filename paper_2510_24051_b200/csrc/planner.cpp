@@ -35,7 +35,12 @@ bool pack_row(const uint8_t* src, int64_t n, uint32_t* dst) {
 
 struct Unit {
   int32_t req, kv_head, row0, nrows, page_begin, page_end;
+  // shared-prefix cascade (defaults: a plain unit)
+  int32_t x_slot0 = -1, x_nslots = 0, x_row0 = 0;  // cascade partials that cover this unit's rows
+  bool force_partial = false;                      // write fp32 partials even when the unit is not cut
+  bool cascade = false;                            // the unit IS a cascade piece: slots, but no merge group of its own
 };
+typedef std::vector<std::pair<int32_t, int32_t>> UnitSlots;  // per unit: (first slot, slots), (-1, 0) if none
 
 PieItem make_item(const Unit& u, int32_t page_begin, int32_t page_end) {
   PieItem it{};
@@ -58,7 +63,8 @@ PieItem make_item(const Unit& u, int32_t page_begin, int32_t page_end) {
 //  * Otherwise: contiguous equal shares; a unit cut by a share boundary becomes several items
 //    whose fp32 partials are merged.
 void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_cta, int slot_rows,
-               bool allow_whole_units, PieLaunchList& ll) {
+               bool allow_whole_units, PieLaunchList& ll, UnitSlots* slots_out = nullptr) {
+  if (slots_out) slots_out->assign(units.size(), std::make_pair(-1, 0));
   ll.items.clear();
   ll.merges.clear();
   ll.cta_ptr.clear();
@@ -96,7 +102,14 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
     ll.items.resize(units.size());
     for (size_t k = 0; k < units.size(); ++k) {
       const Unit& u = units[k];
-      ll.items[fill[owner[k]]++] = make_item(u, u.page_begin, u.page_end);
+      PieItem it = make_item(u, u.page_begin, u.page_end);
+      if (u.force_partial || u.cascade) {
+        it.partial_slot = ll.n_slots;
+        if (slots_out) (*slots_out)[k] = {ll.n_slots, 1};
+        if (!u.cascade) ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, ll.n_slots, 1, u.x_slot0, u.x_nslots, u.x_row0});
+        ++ll.n_slots;
+      }
+      ll.items[fill[owner[k]]++] = it;
     }
     return;
   }
@@ -121,7 +134,8 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
     return (int)std::min<int64_t>(c, grid - 1);
   };
   int64_t off = 0;
-  for (const Unit& u : units) {
+  for (size_t ui = 0; ui < units.size(); ++ui) {
+    const Unit& u = units[ui];
     const int64_t n = u.page_end - u.page_begin;
     if (n == 0) {
       open_cta(std::max(cur, cta_of(std::min(off, W > 0 ? W - 1 : 0))));
@@ -140,9 +154,10 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
       x = end;
     }
     const int np = (int)ll.items.size() - first_item;
-    if (np > 1) {
+    if (np > 1 || u.force_partial || u.cascade) {
       for (int k = 0; k < np; ++k) ll.items[first_item + k].partial_slot = ll.n_slots + k;
-      ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, ll.n_slots, np});
+      if (slots_out) (*slots_out)[ui] = {ll.n_slots, np};
+      if (!u.cascade) ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, ll.n_slots, np, u.x_slot0, u.x_nslots, u.x_row0});
       ll.n_slots += np;
     }
     off += n;
@@ -184,11 +199,11 @@ void chunk_units(const std::vector<Unit>& units, int n_warps, PieLaunchList& ll)
     for (int k = 0; k < nchunks; ++k) {  // chunks of equal size (+-1 page)
       const int b = (int)((int64_t)n * k / nchunks), e = (int)((int64_t)n * (k + 1) / nchunks);
       PieItem it = make_item(u, u.page_begin + b, u.page_begin + e);
-      if (nchunks > 1) it.partial_slot = ll.n_slots + k;
+      if (nchunks > 1 || u.force_partial) it.partial_slot = ll.n_slots + k;
       dst.push_back(it);
     }
-    if (nchunks > 1) {
-      ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, ll.n_slots, nchunks});
+    if (nchunks > 1 || u.force_partial) {
+      ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, ll.n_slots, nchunks, u.x_slot0, u.x_nslots, u.x_row0});
       ll.n_slots += nchunks;
     }
     off += n;
@@ -444,6 +459,69 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   plan->simple_rows.clear();
   plan->tile_tc = pie_tc_supported(ctx) && !(b->flags & PIE_PLAN_NO_TENSOR_TILES);
   const int TILE_ROWS = plan->tile_tc ? 256 : 64;   // two 128-row tcgen05 tiles, or four 16-row warps
+
+  // Shared-prefix cascade (decode-shaped requests): consecutive requests whose page lists start
+  // with the same physical pages - parallel samples, beams, branches of one prompt - have their
+  // rows gathered and attended to that prefix ONCE, as row tiles of a virtual request on the
+  // row-tile kernel; every request then attends only its private pages on the split-KV kernel,
+  // and the merge combines the two partials.  The prefix is read from HBM once per group instead
+  // of once per request.  (Requests with many rows of their own, e.g. token trees, already fill
+  // whole row tiles and find the shared pages in L2: gathering them would only add partials.)
+  struct Cascade { int32_t first, n, L, vreq; };
+  std::vector<Cascade> cascades;
+  std::vector<int32_t> casc_of(R, -1);
+  if (tiles_ok && !(b->flags & PIE_PLAN_NO_CASCADE)) {
+    const bool always = (b->flags & PIE_PLAN_CASCADE_ALWAYS) != 0;
+    const int min_n = always ? 2 : 4, min_L = always ? 1 : 16;
+    auto clean_prefix = [&](const PieReq& q) {  // leading kept pages that are fully visible and in place
+      int c = 0;
+      while (c < q.kept_count - 1 && plan->kept[2 * (size_t)(q.kept_start + c) + 1] == c) ++c;  // (flag bit clear, logical == index)
+      return c;
+    };
+    int64_t saved = 0;
+    for (int r = 0; r < R;) {
+      const PieReq& q0 = plan->reqs[r];
+      const int rows = q0.q_len * G;
+      if (rows > 16 || TILE_ROWS % rows != 0 || q0.kept_count < 2) { ++r; continue; }
+      int L = clean_prefix(q0), e = r + 1;
+      for (; e < R && L >= min_L; ++e) {
+        const PieReq& q = plan->reqs[e];
+        if (q.q_len != q0.q_len || q.kept_count < 2) break;
+        int c = 0;
+        const int cmax = std::min(L, clean_prefix(q));
+        while (c < cmax && plan->kept[2 * (size_t)(q.kept_start + c)] == plan->kept[2 * (size_t)(q0.kept_start + c)]) ++c;
+        if (c < min_L) break;
+        L = c;
+      }
+      if (e - r >= min_n && L >= min_L) {
+        cascades.push_back(Cascade{r, e - r, L, 0});
+        saved += (int64_t)(e - r - 1) * L * cfg.num_kv_heads;
+        r = e;
+      } else {
+        ++r;
+      }
+    }
+    // worth a second launch and a merge only when enough page reads disappear
+    if (!always && saved < 2048) cascades.clear();
+    for (size_t c = 0; c < cascades.size(); ++c) {
+      Cascade& cs = cascades[c];
+      const PieReq& q0 = plan->reqs[cs.first];
+      PieReq v{};   // the virtual request: all rows of the group, the shared pages, everything visible
+      v.q_start = q0.q_start;
+      v.q_len = q0.q_len * cs.n;
+      v.kv_len = v.q_len + cs.L * P;
+      v.kept_start = q0.kept_start;
+      v.kept_count = cs.L;
+      v.mask_row_words = 0;
+      v.mask_word_off = 0;
+      v.last_logical = cs.L - 1;
+      v.last_page_len = P;
+      cs.vreq = (int32_t)plan->reqs.size();
+      plan->reqs.push_back(v);
+      for (int k = 0; k < cs.n; ++k) casc_of[cs.first + k] = (int32_t)c;
+    }
+  }
+  std::vector<int32_t> casc_unit0(cascades.size(), 0);  // first tile unit of every cascade
   for (int r = 0; r < R; ++r) {
     const PieReq& q = plan->reqs[r];
     const int rows = q.q_len * G;
@@ -451,8 +529,10 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       for (int i = 0; i < q.q_len; ++i)
         for (int h = 0; h < cfg.num_q_heads; ++h) plan->simple_rows.push_back((q.q_start + i) * cfg.num_q_heads + h);
     } else if (rows <= 16) {
-      for (int g = 0; g < cfg.num_kv_heads; ++g)
-        split_units.push_back(Unit{r, g, 0, rows, q.kept_start, q.kept_start + q.kept_count});
+      if (casc_of[r] < 0)
+        for (int g = 0; g < cfg.num_kv_heads; ++g)
+          split_units.push_back(Unit{r, g, 0, rows, q.kept_start, q.kept_start + q.kept_count});
+      // (requests of a cascade get their split units below, once the cascade's slots are known)
     } else {
       for (int g = 0; g < cfg.num_kv_heads; ++g)
         for (int row0 = 0; row0 < rows; row0 += TILE_ROWS) {
@@ -466,6 +546,18 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
           tile_units.push_back(Unit{r, g, row0, nrows, q.kept_start, q.kept_start + end});
         }
     }
+  }
+  for (size_t c = 0; c < cascades.size(); ++c) {
+    const Cascade& cs = cascades[c];
+    const PieReq& v = plan->reqs[cs.vreq];
+    const int vrows = v.q_len * G;
+    casc_unit0[c] = (int32_t)tile_units.size();
+    for (int g = 0; g < cfg.num_kv_heads; ++g)
+      for (int row0 = 0; row0 < vrows; row0 += TILE_ROWS) {
+        Unit u{cs.vreq, g, row0, std::min(TILE_ROWS, vrows - row0), v.kept_start, v.kept_start + cs.L};
+        u.cascade = true;
+        tile_units.push_back(u);
+      }
   }
   // SM budget of the two tile kernels.  On request (PIE_OPT_OVERLAP) a mixed batch runs them side
   // by side: the decode kernel is HBM bound and saturates the memory system from roughly 60 % of
@@ -488,6 +580,30 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     tile_sms = ctx->n_sms - n_split;
     plan->overlap = true;
   }
+  // row tiles first: the cascade pieces get their partial slots, which the split units of the
+  // cascaded requests then name as further sources of their merge groups
+  UnitSlots tile_slots;
+  partition(tile_units, tile_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile, &tile_slots);
+  for (size_t c = 0; c < cascades.size(); ++c) {
+    const Cascade& cs = cascades[c];
+    const PieReq& v = plan->reqs[cs.vreq];
+    const int tiles_per_head = (v.q_len * G + TILE_ROWS - 1) / TILE_ROWS;
+    for (int k = 0; k < cs.n; ++k) {
+      const int r = cs.first + k;
+      const PieReq& q = plan->reqs[r];
+      const int rows = q.q_len * G, vr0 = (q.q_start - v.q_start) * G;   // first virtual row of the request
+      for (int g = 0; g < cfg.num_kv_heads; ++g) {
+        Unit u{r, g, 0, rows, q.kept_start + cs.L, q.kept_start + q.kept_count};
+        const auto& sl = tile_slots[(size_t)casc_unit0[c] + (size_t)g * tiles_per_head + vr0 / TILE_ROWS];
+        u.x_slot0 = sl.first;
+        u.x_nslots = sl.second;
+        u.x_row0 = vr0 % TILE_ROWS;
+        u.force_partial = true;
+        split_units.push_back(u);
+      }
+    }
+  }
+  if (!cascades.empty()) plan->overlap = false;  // the split merge reads the row-tile launch's partials
   // split-KV decode.  Long launches: chunks taken dynamically by the warps of the grid (evens out
   // SMs that get different shares of the memory bandwidth).  Short launches: fixed equal shares,
   // one per warp - fewer pieces, fewer partials to merge, and the per-chunk overheads matter more
@@ -509,7 +625,6 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       plan->split.n_static = (int32_t)plan->split.items.size();
     }
   }
-  partition(tile_units, tile_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile);
 
   // ---- fused append of the decode path (PIE_OPT_NO_FUSION switches it off): when every request brings exactly one new token, all of them run on the split-KV
   // kernel, their last page is in the kept list and no request lists a page another one appends

@@ -59,6 +59,15 @@ def test_full_mixed_prefill_decode():
     assert info["num_split_items"] > 0 and info["num_tile_items"] > 0
 
 
+def test_full_shared_prefix_decode_cascade():
+    wl = configs.shared_prefix_decode()
+    B = wl.meta["branches"]
+    sample = [0, 1, B - 1, B, 5 * B + 7, wl.R - 1] + list(range(3, wl.R, 61))
+    info, gp = _sampled_check(wl, sample=sample)
+    gp.close()
+    assert info["num_tile_items"] > 0 and info["num_merge_groups"] == wl.R * wl.H_kv   # the planner chose the cascade
+
+
 def test_full_shared_prefix_tree():
     wl = configs.shared_prefix_tree()
     info, gp = _sampled_check(wl, sample=[0, 17, 255])

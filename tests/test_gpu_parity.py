@@ -355,3 +355,26 @@ def test_fused_append_equals_the_separate_launch(name):
     for n, pg in enumerate(wl.used_pages()):
         Ko, Vo = pool[int(pg)]
         assert same_bits(fused[3][n], Ko) and same_bits(fused[4][n], Vo), f"page {pg}"
+
+
+@pytest.mark.parametrize("flags", [8, 4, 0, 8 | 2])
+def test_shared_prefix_cascade_matches_oracle(flags):
+    """Branches that decode from a shared prompt: with the cascade the prompt's pages are attended
+    once per group (row-tile kernel over the gathered rows) and each request's private pages by the
+    split-KV kernel, merged on LSE (Section 4.2: forked contexts share KvPages).  Flags: 8 = cascade
+    however small the saving, 4 = never, 0 = the planner's own choice (this small batch: none)."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import check_close, run_workload
+    wl = configs.small("shared_prefix_decode")
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    O, L, info, gp = run_workload(wl, poison=True, flags=flags, keep=True)
+    try:
+        assert (info["num_tile_items"] > 0) == bool(flags & 8)
+        check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        used = wl.used_pages()
+        K, V = gp.read_pages(used)
+        for n, p in enumerate(used):
+            Ko, Vo = pool[int(p)]
+            assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {p}"
+    finally:
+        gp.close()

@@ -180,3 +180,37 @@ def test_mask_kvpage_is_anded_into_packed_rows_and_drops_hidden_pages():
         assert np.array_equal(w2, np.packbits(exp, bitorder="little").view(np.uint32))
     finally:
         pie.pie_destroy(ctx)
+
+
+def test_shared_prefix_cascade_planning():
+    """Decode requests that share a prompt's pages: the planner gathers their rows into row-tile
+    work on the shared pages (once per group and kv head) and leaves each request only its
+    private pages on the split-KV path; every (request, kv head) becomes a merge group."""
+    def plan_info(wl, flags):
+        c = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+        try:
+            pie.pie_alloc_kvpages(c, wl.num_pages)
+            mi, mb = wl.mask_bytes()
+            plan = pie.pie_plan_forward(c, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len, mi, mb, flags)
+            info = pie.pie_plan_get_info(plan)
+            pie.pie_plan_destroy(plan)
+            return info
+        finally:
+            pie.pie_destroy(c)
+
+    small = configs.small("shared_prefix_decode")
+    forced = plan_info(small, pie.PIE_PLAN_CASCADE_ALWAYS)
+    assert forced["num_tile_items"] >= small.meta["groups"] * small.H_kv      # one row tile per (group, kv head), maybe cut
+    assert forced["num_merge_groups"] == small.R * small.H_kv
+    assert forced["launches"] == 4                                             # append, row tiles, split-KV, merge
+    for flags in (0, pie.PIE_PLAN_NO_CASCADE):                                 # too small a saving / switched off
+        info = plan_info(small, flags)
+        assert info["num_tile_items"] == 0
+    full = configs.shared_prefix_decode()
+    auto = plan_info(full, 0)
+    off = plan_info(full, pie.PIE_PLAN_NO_CASCADE)
+    assert auto["num_tile_items"] > 0 and off["num_tile_items"] == 0
+    assert auto["num_merge_groups"] == full.R * full.H_kv
+    # the tree workload keeps its requests whole: many rows each, shared pages served from L2
+    tree_wl = configs.small("shared_prefix_tree")
+    assert plan_info(tree_wl, pie.PIE_PLAN_CASCADE_ALWAYS) == plan_info(tree_wl, pie.PIE_PLAN_NO_CASCADE)

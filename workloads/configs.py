@@ -352,6 +352,53 @@ def long_context_policy(seed=SEED0 + 5, R=256, lo=16384, hi=32768, sink=4, windo
     return wl
 
 
+# ------------------------------------------------------------------------------- shared-prefix decode
+def shared_prefix_decode(seed=SEED0 + 6, groups=16, branches=32, prefix=4096, priv_lo=16, priv_hi=256,
+                         num_pages=16384, H_q=32, H_kv=8, D=128, P=16, dtype="bf16"):
+    """Parallel generation from shared prompts (fork / join, beams, samples of one prompt): every
+    group's branches share the prompt's pages and each decodes one token after a private
+    continuation of its own, seeded log-uniform length in [priv_lo, priv_hi].  Not one of the five
+    baseline configurations: the workload of the shared-prefix cascade."""
+    assert prefix % P == 0
+    R = groups * branches
+    n_pre = prefix // P
+    u = synth.uniform_unit(seed, 11, (R,))
+    priv = np.floor(np.exp(np.log(priv_lo) + u * (np.log(priv_hi + 1) - np.log(priv_lo)))).astype(np.int64)
+    priv = np.clip(priv, priv_lo, priv_hi)
+    perm = synth.permutation(seed, 10, num_pages)
+    owner = np.full(num_pages, -1, dtype=np.int64)
+    logical = np.zeros(num_pages, dtype=np.int64)
+    fill = np.zeros(num_pages, dtype=np.int64)
+    cur = 0
+    pre_ids = []
+    for g in range(groups):
+        ids = perm[cur:cur + n_pre]
+        cur += n_pre
+        owner[ids], logical[ids], fill[ids] = g, np.arange(n_pre), P
+        pre_ids.append(ids)
+    lists, npages, last = [], [], []
+    for g in range(groups):
+        for b in range(branches):
+            rid = g * branches + b
+            n_priv = int((priv[rid] + 1 + P - 1) // P)     # private context + the new token
+            assert cur + n_priv <= num_pages, "pool too small"
+            ids = perm[cur:cur + n_priv]
+            cur += n_priv
+            owner[ids] = 1000 + rid
+            logical[ids] = n_pre + np.arange(n_priv)
+            fill[ids] = np.clip(priv[rid] - np.arange(n_priv) * P, 0, P)
+            lists.append(np.concatenate([pre_ids[g], ids]))
+            npages.append(n_pre + n_priv)
+            last.append(priv[rid] + 1 - (n_priv - 1) * P)
+    assert cur <= num_pages, "pool too small"
+    return Workload(
+        name="shared_prefix_decode", seed=seed, H_q=H_q, H_kv=H_kv, D=D, P=P, dtype=dtype,
+        num_pages=num_pages, qo_indptr=_csr(np.ones(R, dtype=np.int64)), page_indptr=_csr(np.array(npages)),
+        page_indices=np.concatenate(lists).astype(np.int32), last_page_len=np.array(last, dtype=np.int32),
+        masks=None, page_owner=owner, page_logical=logical, page_fill=fill,
+        meta={"groups": groups, "branches": branches, "prefix": prefix})
+
+
 FULL = {
     "tiny_fp32": tiny_fp32,
     "batched_decode": batched_decode,
@@ -359,6 +406,8 @@ FULL = {
     "shared_prefix_tree": shared_prefix_tree,
     "long_context_policy": long_context_policy,
 }
+# further workloads (not baseline configurations)
+EXTRA = {"shared_prefix_decode": shared_prefix_decode}
 
 
 def small(name, **kw):
@@ -376,4 +425,6 @@ def small(name, **kw):
                                   num_pages=256, **kw)
     if name == "long_context_policy":
         return long_context_policy(R=6, lo=1500, hi=4000, window=256, **kw)
+    if name == "shared_prefix_decode":
+        return shared_prefix_decode(groups=3, branches=5, prefix=320, priv_lo=3, priv_hi=70, num_pages=256, **kw)
     raise KeyError(name)
