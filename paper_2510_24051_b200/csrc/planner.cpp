@@ -115,8 +115,10 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
   }
 
   // Contiguous shares.  Walking the units in order visits the shares in order too, so the items
-  // come out already grouped by CTA.
+  // come out already grouped by CTA; share c covers page visits [c W / grid, (c + 1) W / grid),
+  // and its end is recomputed only when the walk crosses it (no division per piece).
   ll.items.reserve(units.size() + grid);
+  ll.merges.reserve(std::min<size_t>(units.size(), (size_t)grid));
   ll.cta_ptr.reserve(grid + 1);
   ll.cta_ptr.push_back(0);
   int cur = 0;  // CTA whose item range is open
@@ -126,27 +128,29 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
       ++cur;
     }
   };
-  auto cta_of = [&](int64_t x) {  // share that holds page-visit x
-    if (W == 0) return 0;
-    int64_t c = (x * grid) / W;
-    while (c + 1 < grid && ((c + 1) * W) / grid <= x) ++c;
-    while (c > 0 && (c * W) / grid > x) --c;
-    return (int)std::min<int64_t>(c, grid - 1);
+  int c = 0;                                             // share that holds the walk's position
+  int64_t c_end = grid == 1 ? W : W / grid;              // its end
+  auto advance_to = [&](int64_t x) {                     // make c the share that holds page visit x
+    while (c + 1 < grid && x >= c_end) {
+      ++c;
+      c_end = (c + 1 == grid) ? W : ((int64_t)(c + 1) * W) / grid;
+    }
   };
   int64_t off = 0;
   for (size_t ui = 0; ui < units.size(); ++ui) {
     const Unit& u = units[ui];
     const int64_t n = u.page_end - u.page_begin;
     if (n == 0) {
-      open_cta(std::max(cur, cta_of(std::min(off, W > 0 ? W - 1 : 0))));
+      advance_to(std::min(off, W > 0 ? W - 1 : 0));
+      open_cta(std::max(cur, c));
       ll.items.push_back(make_item(u, u.page_begin, u.page_begin));
       continue;
     }
     const int first_item = (int)ll.items.size();
     int64_t x = off;
     while (x < off + n) {  // pieces: cut at share boundaries strictly inside (off, off+n)
-      const int c = cta_of(x);
-      int64_t end = (c + 1 == grid) ? W : ((int64_t)(c + 1) * W) / grid;
+      advance_to(x);
+      int64_t end = c_end;
       if (end <= x) end = x + 1;
       end = std::min(end, off + n);
       open_cta(c);
