@@ -281,11 +281,14 @@ int pie_sched_next_batch(pie_sched* s, int32_t* out_type, int32_t cap, int64_t* 
  *                      stream that forks from and joins the caller's stream.  Pays only when the
  *                      tensor-bound part is long against the HBM-bound part: the decode kernel
  *                      needs about 60 % of the SMs to keep the memory system saturated.
- *   PIE_OPT_NO_FUSION  1 = always launch the append kernel.  By default (0) a decode batch
- *                      (every request one new token, all on the split-KV kernel, no request
- *                      listing a page another one appends to) lets the attention kernel write
- *                      the new K/V rows itself, which saves the append launch; results and
- *                      pool contents are bit-identical either way. */
+ *   PIE_OPT_NO_FUSION  bit mask of fusions of the decode path to switch off (default 0: both on;
+ *                      results are identical up to fp32 summation order, pool contents bit-identical).
+ *                      Bit 0: always launch the append kernel.  By default a decode batch (every
+ *                      request one new token, all on the split-KV kernel, no request listing a
+ *                      page another one appends to) lets the attention kernel write the new K/V
+ *                      rows itself.  Bit 1: always merge split partials with the merge kernel.  By
+ *                      default short decode launches keep all pieces of a (request, kv head)
+ *                      inside one thread block, which merges them itself. */
 enum { PIE_OPT_SPLIT_SMS = 0, PIE_OPT_TILE_SMS = 1, PIE_OPT_OVERLAP = 2, PIE_OPT_NO_FUSION = 3, PIE_NUM_OPTIONS = 4 };
 int pie_set_option(pie_ctx* ctx, int option, int value);
 

@@ -255,6 +255,62 @@ __device__ __forceinline__ void rows_store(RowState<D>& st, const AttnParams& p,
   }
 }
 
+// The warp holding the first piece of a block-local group: combine its own rows (still in
+// registers) with the fp32 partials of the other pieces, slots slot0 + 1 .. slot0 + np - 1, and
+// store the final rows.  lse = ln sum_c exp(lse_c), o = sum_c exp(lse_c - lse) o_c, pieces in
+// slot order (the same fixed order as the merge kernel, so results do not depend on timing).
+template <int D>
+__device__ __forceinline__ void rows_merge_store(RowState<D>& st, const AttnParams& p, const PieItem& item, const PieReq& rq,
+                                                 int np, int slot_rows, int lane) {
+  const int r_lo = lane >> 2, cpair = (lane & 3) * 2;
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    st.l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, st.l_run[r], 1);
+    st.l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, st.l_run[r], 2);
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (!st.valid[r]) continue;
+    const int row = r_lo + r * 8;   // row inside the unit (item.row0 == 0 for split-KV units)
+    const int gr = item.row0 + row;
+    const int tok = gr / p.G, head = item.kv_head * p.G + gr % p.G;
+    const float L = st.l_run[r];
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    const float lse0 = L > 0.f ? (st.m_run[r] + log2f(L)) * kLn2 : kNegInf;
+    float M = lse0;
+    for (int c = 1; c < np; ++c) M = fmaxf(M, __ldcg(p.ws_lse + (int64_t)(item.partial_slot + c) * slot_rows + row));
+    float w0 = 0.f, Z = 0.f;
+    if (M != kNegInf) w0 = __expf(lse0 - M);
+    Z = w0;
+    const float s0 = w0 * inv;      // own rows are un-normalised: weight times 1 / l
+#pragma unroll
+    for (int nb = 0; nb < D / 8; ++nb) {
+      st.o[nb][2 * r] *= s0;
+      st.o[nb][2 * r + 1] *= s0;
+    }
+    for (int c = 1; c < np; ++c) {
+      const int64_t si = (int64_t)(item.partial_slot + c) * slot_rows + row;
+      float wc = 0.f;
+      if (M != kNegInf) wc = __expf(__ldcg(p.ws_lse + si) - M);
+      Z += wc;
+      const float* src = p.ws_o + si * D;
+#pragma unroll
+      for (int nb = 0; nb < D / 8; ++nb) {
+        const float2 v = __ldcg(reinterpret_cast<const float2*>(src + nb * 8 + cpair));
+        st.o[nb][2 * r] += wc * v.x;
+        st.o[nb][2 * r + 1] += wc * v.y;
+      }
+    }
+    const float invZ = Z > 0.f ? 1.f / Z : 0.f;
+    const int64_t oi = ((int64_t)(rq.q_start + tok) * p.n_q_heads + head);
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D;
+#pragma unroll
+    for (int nb = 0; nb < D / 8; ++nb)
+      *reinterpret_cast<uint32_t*>(dst + nb * 8 + cpair) = pack_bf16(st.o[nb][2 * r] * invZ, st.o[nb][2 * r + 1] * invZ);
+    if ((lane & 3) == 0) p.lse[oi] = Z > 0.f ? M + logf(Z) : kNegInf;
+  }
+}
+
 // ------------------------------------------------------------------------------ split-KV decode
 // Every warp is an independent pipeline.  The planner cuts every (request, kv head) into chunks
 // of pages - large ones first, small ones for the tail - and the warps of the grid take chunks
@@ -267,7 +323,7 @@ template <int D, int P, int NW, int DEPTH>
 struct SplitCfg {
   static constexpr int STAGE = 2 * P * D * 2;
   static constexpr int QUEUE = 8;  // chunk ids a warp has started fetching but not finished (<= DEPTH + 2)
-  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * 16 + NW * QUEUE * 4 + 64;
+  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * 16 + NW * QUEUE * 4 + PIE_MAX_LOCAL_GROUPS * 4 + 64;
 };
 
 template <int D, int P, int NW, int DEPTH>
@@ -281,6 +337,9 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   volatile uint32_t* meta = reinterpret_cast<uint32_t*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 8) + warp * DEPTH;
   volatile int* meta_phys = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 12) + warp * DEPTH;
   volatile int* queue = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 16) + warp * C::QUEUE;
+  int* local_cnt = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 16 + NW * C::QUEUE * 4);  // block-local merge groups
+  if (threadIdx.x < PIE_MAX_LOCAL_GROUPS) local_cnt[threadIdx.x] = 0;
+  __syncthreads();   // the only block-wide sync of the kernel (counters are zero before any warp counts itself in)
   pie_pdl_launch_dependents();
   if (lane == 0) {
     for (int s = 0; s < DEPTH; ++s) mbar_init(smem_u32(full_bar + s), 1);
@@ -450,7 +509,37 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
         pf_settle();
       }
     }
-    rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);
+    if (!(item.flags & PIE_ITEM_LOCAL_PIECE)) {
+      rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);
+    } else {
+      const int gid = (item.flags >> 8) & 0xFF, np = (item.flags >> 16) & 0xFF;
+      if (!(item.flags & PIE_ITEM_LOCAL_MERGER)) {
+        rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);   // fp32 partial
+        __threadfence_block();   // the merging warp runs on this SM: block scope is enough
+        __syncwarp();
+        if (lane == 0) atomicAdd(local_cnt + gid, 1);
+      } else {
+        // wait (bounded) until the other pieces of the group have been written
+        if (lane == 0) {
+          volatile int* cnt = local_cnt + gid;
+          uint64_t t0 = 0;
+          for (uint32_t spin = 1; *cnt < np - 1; ++spin) {
+            if ((spin & 255u) == 0) {
+              if (*reinterpret_cast<volatile int*>(p.status) != 0) break;
+              const uint64_t now = global_ns();
+              if (t0 == 0) t0 = now;
+              if (now - t0 > 1000000000ull) {
+                atomicExch(p.status, (int)PIE_ERR_DEVICE_TIMEOUT);
+                break;
+              }
+            }
+          }
+        }
+        __syncwarp();
+        __threadfence_block();
+        rows_merge_store<D>(st, p, item, rq, np, p.slot_rows, lane);
+      }
+    }
   }
 
   // ---- the last warp of the grid to finish re-arms the counters for the next launch
@@ -837,12 +926,10 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
 
   pie_plan plan;  // host-side only; its device pointers will point into the static scratch
   plan.ctx = ctx;
-  const int saved_overlap = ctx->options[PIE_OPT_OVERLAP], saved_fusion = ctx->options[PIE_OPT_NO_FUSION];
-  ctx->options[PIE_OPT_OVERLAP] = 0;    // this entry point enqueues its kernels one after the other
-  ctx->options[PIE_OPT_NO_FUSION] = 1;  // and keeps the separate append launch
+  const int saved_overlap = ctx->options[PIE_OPT_OVERLAP];
+  ctx->options[PIE_OPT_OVERLAP] = 0;  // this entry point enqueues its kernels one after the other
   int rc = pie_build_plan(ctx, batch, &plan);
   ctx->options[PIE_OPT_OVERLAP] = saved_overlap;
-  ctx->options[PIE_OPT_NO_FUSION] = saved_fusion;
   if (rc != PIE_OK) return rc;
   if (plan.T == 0) return PIE_OK;
   if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;

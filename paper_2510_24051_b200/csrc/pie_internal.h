@@ -62,6 +62,15 @@ static_assert(sizeof(PieItem) == 64, "PieItem is one 64-byte line");
 // The split-KV warp that owns this item also writes the request's one new K/V row (decode batches
 // whose append is fused into the attention kernel): into the pool and into its staged copy of the page.
 #define PIE_ITEM_APPEND 1u
+// Split-KV, fixed shares: a (request, kv head) cut into pieces that all belong to warps of ONE
+// thread block is merged inside the kernel.  Every piece but the first writes its fp32 partial and
+// counts itself in on a shared-memory counter (block-scope fence, no device-wide one); the warp
+// with the first piece - its last item, so it finishes last - waits for the count and combines
+// the partials with its own registers.  flags: bits 8-15 = the group's counter in the block,
+// bits 16-23 = number of pieces.
+#define PIE_ITEM_LOCAL_PIECE 2u
+#define PIE_ITEM_LOCAL_MERGER 4u
+#define PIE_MAX_LOCAL_GROUPS 8
 
 // A group of partial slots that the merge kernel combines into final rows.
 struct PieMerge {

@@ -170,6 +170,151 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
   ll.cta_ptr.push_back((int32_t)ll.items.size());
 }
 
+// Split-KV decode, short launches: fixed shares with block-local merges.  Whole units are first
+// dealt to thread blocks (largest first, each to the least-loaded block, then units are moved from
+// the fullest block to the emptiest while that lowers the maximum); inside a block its units'
+// page visits are cut into one contiguous equal share per warp.  A unit cut by a share boundary
+// therefore has all its pieces in one block, and the kernel merges them itself (PIE_ITEM_LOCAL_*):
+// no partial needs the merge launch.  Returns false (and leaves `ll` unusable) when whole units
+// cannot be dealt evenly enough - few or very unequal units - where cutting them across blocks
+// balances better than the merge launch costs.
+bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int min_pages_per_warp, int slot_rows,
+                     PieLaunchList& ll) {
+  ll.items.clear();
+  ll.merges.clear();
+  ll.cta_ptr.clear();
+  ll.n_slots = 0;
+  ll.slot_rows = slot_rows;
+  ll.grid = 0;
+  ll.n_static = 0;
+  if (units.empty()) return true;
+  auto size_of = [&](int32_t k) { return (int64_t)std::max(1, units[k].page_end - units[k].page_begin); };
+  int64_t W = 0;
+  for (size_t k = 0; k < units.size(); ++k) W += size_of((int32_t)k);
+  const int n_ctas = (int)std::min<int64_t>(ctas_max, std::max<int64_t>(1, W / std::max(1, min_pages_per_warp * NW)));
+  // Largest first.  Units arrive in runs of equal size (the kv heads of one request), so the runs
+  // are sorted, not the units: equivalent to a stable sort of the units by size, descending.
+  const int n_units = (int)units.size();
+  std::vector<uint64_t> runs;   // (~size) << 32 | first unit of the run
+  runs.reserve(n_units / 4 + 1);
+  for (int k = 0; k < n_units;) {
+    int e = k + 1;
+    while (e < n_units && size_of(e) == size_of(k)) ++e;
+    runs.push_back(((uint64_t)(0xFFFFFFFFu - (uint32_t)size_of(k)) << 32) | (uint32_t)k);
+    k = e;
+  }
+  std::sort(runs.begin(), runs.end());
+  // Min-heap of (load << 16 | block) keys; dealing a unit replaces the top key and sifts it down.
+  std::vector<uint64_t> heap(n_ctas);
+  for (int c = 0; c < n_ctas; ++c) heap[c] = (uint64_t)c;   // all loads zero: already a heap
+  std::vector<int64_t> load(n_ctas, 0);
+  std::vector<int32_t> head(n_ctas, -1), next(n_units, -1);   // members of a block: singly linked lists
+  for (uint64_t run : runs) {
+    const int k0 = (int)(uint32_t)run;
+    const int64_t sz = size_of(k0);
+    for (int k = k0; k < n_units && size_of(k) == sz; ++k) {
+      const int c = (int)(heap[0] & 0xFFFF);
+      next[k] = head[c];
+      head[c] = k;
+      load[c] += sz;
+      const uint64_t key = ((uint64_t)load[c] << 16) | (uint64_t)c;
+      int i = 0;
+      for (;;) {   // sift down
+        int ch = 2 * i + 1;
+        if (ch >= n_ctas) break;
+        if (ch + 1 < n_ctas && heap[ch + 1] < heap[ch]) ++ch;
+        if (heap[ch] >= key) break;
+        heap[i] = heap[ch];
+        i = ch;
+      }
+      heap[i] = key;
+    }
+  }
+  // refinement: move a unit from the fullest block to the emptiest one while that lowers the maximum
+  for (int iter = 0; iter < 48; ++iter) {
+    int hi = 0, lo = 0;
+    for (int c = 1; c < n_ctas; ++c) {
+      if (load[c] > load[hi]) hi = c;
+      if (load[c] < load[lo]) lo = c;
+    }
+    if (load[hi] * n_ctas * 100 <= W * 101) break;   // within 1 % of the average: good enough
+    const int64_t gap = load[hi] - load[lo];
+    int best = -1, best_prev = -1;
+    int64_t best_sz = 0;
+    for (int k = head[hi], prev = -1; k >= 0; prev = k, k = next[k]) {   // the largest unit that still leaves `lo` below the old maximum
+      const int64_t sz = size_of(k);
+      if (sz < gap && sz > best_sz) {
+        best = k;
+        best_prev = prev;
+        best_sz = sz;
+      }
+    }
+    if (best < 0) break;
+    if (best_prev < 0) head[hi] = next[best];
+    else next[best_prev] = next[best];
+    next[best] = head[lo];
+    head[lo] = best;
+    load[hi] -= best_sz;
+    load[lo] += best_sz;
+  }
+  int64_t max_load = 0;
+  for (int c = 0; c < n_ctas; ++c) max_load = std::max(max_load, load[c]);
+  if (max_load * n_ctas * 100 > W * 105) return false;   // the fullest block holds more than 5 % above the average
+
+  ll.items.reserve(units.size() + (size_t)n_ctas * NW);
+  ll.cta_ptr.reserve((size_t)n_ctas * NW + 1);
+  ll.cta_ptr.push_back(0);
+  std::vector<int32_t> members;
+  for (int c = 0; c < n_ctas; ++c) {
+    members.clear();
+    for (int k = head[c]; k >= 0; k = next[k]) members.push_back(k);
+    std::sort(members.begin(), members.end());      // batch order inside a block
+    const int64_t Wc = load[c];
+    const int nw = (int)std::min<int64_t>(NW, std::max<int64_t>(1, Wc / std::max(1, min_pages_per_warp)));
+    int w = 0;                                      // warp whose item range is open
+    int64_t w_end = nw == 1 ? Wc : Wc / nw, off = 0;
+    int local_groups = 0;
+    auto advance_to = [&](int64_t x) {
+      while (w + 1 < nw && x >= w_end) {
+        ll.cta_ptr.push_back((int32_t)ll.items.size());
+        ++w;
+        w_end = (w + 1 == nw) ? Wc : ((int64_t)(w + 1) * Wc) / nw;
+      }
+    };
+    for (int32_t ui : members) {
+      const Unit& u = units[ui];
+      const int64_t n = size_of(ui);
+      const int first_item = (int)ll.items.size();
+      if (u.page_end == u.page_begin) {
+        advance_to(off);
+        ll.items.push_back(make_item(u, u.page_begin, u.page_begin));
+      } else {
+        int64_t x = off;
+        while (x < off + n) {
+          advance_to(x);
+          const int64_t end = std::min(std::max(w_end, x + 1), off + n);
+          ll.items.push_back(make_item(u, (int32_t)(u.page_begin + (x - off)), (int32_t)(u.page_begin + (end - off))));
+          x = end;
+        }
+      }
+      const int np = (int)ll.items.size() - first_item;
+      if (np > 1) {   // (at most NW - 1 cut units per block, np <= NW)
+        for (int k = 0; k < np; ++k) {
+          PieItem& it = ll.items[first_item + k];
+          it.partial_slot = ll.n_slots + k;
+          it.flags |= PIE_ITEM_LOCAL_PIECE | (k == 0 ? PIE_ITEM_LOCAL_MERGER : 0u) | ((uint32_t)local_groups << 8) | ((uint32_t)np << 16);
+        }
+        ll.n_slots += np;
+        ++local_groups;
+      }
+      off += n;
+    }
+    for (; w < NW; ++w) ll.cta_ptr.push_back((int32_t)ll.items.size());   // close this block's warps (idle ones: empty ranges)
+  }
+  ll.grid = n_ctas * NW;
+  return true;
+}
+
 // Split-KV decode: cut every unit into chunks that the warps of the grid take from a global
 // counter at run time.  Units in the first 80 % of the page visits get large chunks (about a
 // third of a warp's fair share), the rest small ones, and the large chunks come first in the
@@ -625,7 +770,11 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     } else {
       // fixed equal shares, nothing left to the counter (a dynamic tail of small chunks was measured:
       // the extra partials cost more in the merge than the better balance gains on a 50 us launch)
-      partition(split_units, n_warps, 4, max_rows, false, plan->split);
+      bool plain = true;   // cascade pieces bring partials of another launch: those groups need the merge kernel
+      for (const Unit& u : split_units) plain = plain && !u.force_partial;
+      if (!plain || (ctx->options[PIE_OPT_NO_FUSION] & 2) ||
+          !partition_local(split_units, split_sms, pie_split_warps_per_block(ctx), 4, max_rows, plan->split))
+        partition(split_units, n_warps, 4, max_rows, false, plan->split);
       plan->split.n_static = (int32_t)plan->split.items.size();
     }
   }
@@ -649,7 +798,6 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   for (PieLaunchList* ll : {&plan->split, &plan->tile})
     for (PieItem& it : ll->items) {
       const PieReq& q = plan->reqs[it.req];
-      it.flags = 0;
       if (ll == &plan->split && plan->append_fused && it.page_end == q.kept_start + q.kept_count) it.flags |= PIE_ITEM_APPEND;
       it.q_start = q.q_start;
       it.q_len = q.q_len;

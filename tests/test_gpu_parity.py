@@ -328,33 +328,36 @@ def test_output_pointer_that_is_only_16_byte_aligned():
 
 
 @pytest.mark.parametrize("name", ["batched_decode", "long_context_policy"])
-def test_fused_append_equals_the_separate_launch(name):
-    """Decode batches let the split-KV kernel write the new K/V rows itself (one launch fewer);
-    switching the fusion off must give the same bits in O, LSE and the pool."""
+def test_decode_fusions_equal_the_separate_launches(name):
+    """Decode batches let the split-KV kernel write the new K/V rows itself and (short launches)
+    merge the pieces of a (request, kv head) inside one thread block; PIE_OPT_NO_FUSION switches
+    either off.  The append fusion must not change a bit of O, LSE or the pool; the merge fusion
+    only changes the fp32 summation order, so it is held to the oracle tolerance."""
     import paper_2510_24051_b200 as pie
     from tests._gpu import GpuPool, check_close
     wl = configs.small(name)
-    results = []
-    for no_fusion in (0, 1):
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    res = {}
+    for no_fusion in (0, 1, 2, 3):
         with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
             pie.pie_set_option(gp.ctx, pie.PIE_OPT_NO_FUSION, no_fusion)
             gp.install(wl, poison=True)
             plan = gp.plan(wl)
             info = pie.pie_plan_get_info(plan)
             out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+            out2, lse2 = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))   # plan reuse
+            assert torch.equal(out.view(torch.int16), out2.view(torch.int16)) and torch.equal(lse, lse2)
             K, V = gp.read_pages(wl.used_pages())
             pie.pie_plan_destroy(plan)
-            results.append((info["launches"], out.view(torch.int16).cpu(), lse.cpu(), K, V))
-    fused, plain = results
-    assert plain[0] == fused[0] + 1
-    assert torch.equal(fused[1], plain[1]) and torch.equal(fused[2], plain[2])
-    assert same_bits(fused[3], plain[3]) and same_bits(fused[4], plain[4])
-    # and the fused run matches the oracle like any other
-    O_ref, L_ref, pool = run_oracle(wl, poison=True)
-    check_close(fused[1].view(torch.bfloat16).double().numpy(), fused[2].double().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
-    for n, pg in enumerate(wl.used_pages()):
-        Ko, Vo = pool[int(pg)]
-        assert same_bits(fused[3][n], Ko) and same_bits(fused[4][n], Vo), f"page {pg}"
+        check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        for n, pg in enumerate(wl.used_pages()):
+            Ko, Vo = pool[int(pg)]
+            assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {pg}"
+        res[no_fusion] = (info["launches"], out.view(torch.int16).cpu(), lse.cpu())
+    for a, b2 in ((0, 1), (2, 3)):                         # the append fusion alone: identical bits, one launch fewer
+        assert res[b2][0] == res[a][0] + 1
+        assert torch.equal(res[a][1], res[b2][1]) and torch.equal(res[a][2], res[b2][2])
+    assert res[3][0] == 3 and res[0][0] <= 2              # append + split-KV + merge against split-KV (+ merge if dynamic)
 
 
 @pytest.mark.parametrize("flags", [8, 4, 0, 8 | 2])
@@ -378,3 +381,30 @@ def test_shared_prefix_cascade_matches_oracle(flags):
             assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {p}"
     finally:
         gp.close()
+
+
+@pytest.mark.parametrize("sms", [6, 16])
+def test_block_local_merge_matches_oracle(sms):
+    """Short decode launches deal whole (request, kv head) units to thread blocks and cut them only
+    between warps of one block, which then merges the pieces itself: no merge launch.  Few SMs
+    make the small batch balance well enough for that path to be chosen."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs.small("batched_decode")
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        pie.pie_set_option(gp.ctx, pie.PIE_OPT_SPLIT_SMS, sms)
+        gp.install(wl, poison=True)
+        plan = gp.plan(wl)
+        info = pie.pie_plan_get_info(plan)
+        assert info["num_merge_groups"] == 0 and info["launches"] == 1        # fused append, in-kernel merge
+        assert info["num_split_items"] > wl.R * wl.H_kv                        # units were cut
+        out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+        out2, lse2 = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+        assert torch.equal(out.view(torch.int16), out2.view(torch.int16)) and torch.equal(lse, lse2)
+        pie.pie_plan_destroy(plan)
+        check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        K, V = gp.read_pages(wl.used_pages())
+        for n, pg in enumerate(wl.used_pages()):
+            Ko, Vo = pool[int(pg)]
+            assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {pg}"
