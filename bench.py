@@ -353,7 +353,12 @@ def main():
     dom = max(("split", "tiles", "simple"), key=lambda k: ktimes[k][0])
     dom_ms = ktimes[dom][0] / max(ktimes[dom][1], 1)
     dom_timing = "events around each launch of the kernel"
-    if launches_per_step == 1 and args.gpus == 1:
+    if info.get("side_by_side_sms", 0) > 0:
+        # decode and prefill kernels run at the same time on disjoint SM sets: per-kernel events overlap, so the
+        # step is rated as a whole against the HBM roofline of its decode part (the prefill part is tensor work)
+        dom, dom_ms = "split", ms / args.steps
+        dom_timing = "timed region / steps (decode and prefill kernels side by side)"
+    elif launches_per_step == 1 and args.gpus == 1:
         # the step IS this one kernel: its launch duration is the timed region divided by the launches (the events
         # around single launches keep consecutive launches from overlapping their prologues and report more)
         dom_ms = min(dom_ms, ms / args.steps)

@@ -166,7 +166,7 @@ typedef struct pie_plan_info {
   int32_t num_simple_rows;      /* (token, head) rows given to the plain kernel    */
   int32_t num_merge_groups;     /* groups whose split partials the merge combines  */
   int32_t launches;             /* kernels one pie_forward enqueues                */
-  int32_t reserved;
+  int32_t side_by_side_sms;     /* SMs given to the row-tile kernel when it runs next to the decode kernel (0: one after the other) */
   int64_t kept_pages;           /* pages left in the lists after dropping fully masked ones */
   int64_t mask_words;           /* 32-bit words of packed mask                     */
   int64_t workspace_bytes;      /* device scratch for split partials               */
@@ -276,11 +276,15 @@ int pie_sched_next_batch(pie_sched* s, int32_t* out_type, int32_t cap, int64_t* 
 /* Tuning knobs (all optional; 0 restores the default).  They affect plans made afterwards.
  *   PIE_OPT_SPLIT_SMS  SMs the split-KV decode kernel may use (default: all).
  *   PIE_OPT_TILE_SMS   SMs the prefill / tree kernel may use (default: all).
- *   PIE_OPT_OVERLAP    mixed batches: 0 = default (the decode kernel, then the prefill / tree
- *                      kernel), 1 = side by side on disjoint SM sets, the second on an internal
- *                      stream that forks from and joins the caller's stream.  Pays only when the
- *                      tensor-bound part is long against the HBM-bound part: the decode kernel
- *                      needs about 60 % of the SMs to keep the memory system saturated.
+ *   PIE_OPT_OVERLAP    mixed batches (decode requests and prefill / tree requests in one call):
+ *                      0 = automatic (default): the HBM-bound decode kernel and the tensor-bound
+ *                      prefill / tree kernel run side by side on disjoint SM sets - the second on an
+ *                      internal stream that forks from and joins the caller's stream - when a model
+ *                      of the two kernels (the decode kernel keeps the memory system saturated
+ *                      with about 60 % of the SMs) predicts at least 10 % over running them one
+ *                      after the other; 1 = side by side whenever both kinds are present;
+ *                      2 = never.  With 1 and PIE_OPT_SPLIT_SMS and PIE_OPT_TILE_SMS both set,
+ *                      those are the two SM sets.
  *   PIE_OPT_NO_FUSION  bit mask of fusions of the decode path to switch off (default 0: both on;
  *                      results are identical up to fp32 summation order, pool contents bit-identical).
  *                      Bit 0: always launch the append kernel.  By default a decode batch (every

@@ -586,15 +586,24 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
     PIE_CUDA(ctx, cudaEventRecord(ctx->ev_fork, s));
     PIE_CUDA(ctx, cudaStreamWaitEvent(s2, ctx->ev_fork, 0));
   }
-  if (!plan->tile.items.empty() &&
-      (rc = timed_launch(ctx, PIE_KERNEL_TILES, s2, [&] { return pie_launch_tiles(ctx, plan, q, out, lse, s2); })))
-    return rc;
-  if (!plan->tile.merges.empty() &&
-      (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s2, [&] { return pie_launch_merge(ctx, plan, plan->tile, out, lse, s2); })))
-    return rc;
+  auto launch_tiles = [&]() -> int {
+    int r = PIE_OK;
+    if (!plan->tile.items.empty() &&
+        (r = timed_launch(ctx, PIE_KERNEL_TILES, s2, [&] { return pie_launch_tiles(ctx, plan, q, out, lse, s2); })))
+      return r;
+    if (!plan->tile.merges.empty() &&
+        (r = timed_launch(ctx, PIE_KERNEL_MERGE, s2, [&] { return pie_launch_merge(ctx, plan, plan->tile, out, lse, s2); })))
+      return r;
+    return PIE_OK;
+  };
+  // Side by side, the decode kernel is enqueued first: measured on B200, a running row-tile kernel
+  // keeps the decode kernel's blocks from being dispatched until it ends, while the other order
+  // lets both run.  One after the other, the row tiles go first (cascade partials feed the split merge).
+  if (!side && (rc = launch_tiles())) return rc;
   if (!plan->split.items.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_SPLIT, s, [&] { return pie_launch_split(ctx, plan, q, k_new, v_new, out, lse, s); })))
     return rc;
+  if (side && (rc = launch_tiles())) return rc;
   if (!plan->split.merges.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s, [&] { return pie_launch_merge(ctx, plan, plan->split, out, lse, s); })))
     return rc;

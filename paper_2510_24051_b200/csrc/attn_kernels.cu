@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   int* local_cnt = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 16 + NW * C::QUEUE * 4);  // block-local merge groups
   if (threadIdx.x < PIE_MAX_LOCAL_GROUPS) local_cnt[threadIdx.x] = 0;
   __syncthreads();   // the only block-wide sync of the kernel (counters are zero before any warp counts itself in)
-  pie_pdl_launch_dependents();
+  if (!p.late_trigger) pie_pdl_launch_dependents();
   if (lane == 0) {
     for (int s = 0; s < DEPTH; ++s) mbar_init(smem_u32(full_bar + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -542,6 +542,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
     }
   }
 
+  if (p.late_trigger) pie_pdl_launch_dependents();
   // ---- the last warp of the grid to finish re-arms the counters for the next launch
   if (lane == 0) {
     __threadfence();
@@ -786,6 +787,7 @@ AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& 
   p.n_kv_heads = ctx->cfg.num_kv_heads;
   p.G = ctx->G;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)ctx->cfg.head_dim);
+  p.late_trigger = plan->overlap ? 1 : 0;
   return p;
 }
 
@@ -927,7 +929,7 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   pie_plan plan;  // host-side only; its device pointers will point into the static scratch
   plan.ctx = ctx;
   const int saved_overlap = ctx->options[PIE_OPT_OVERLAP];
-  ctx->options[PIE_OPT_OVERLAP] = 0;  // this entry point enqueues its kernels one after the other
+  ctx->options[PIE_OPT_OVERLAP] = 2;  // this entry point enqueues its kernels one after the other
   int rc = pie_build_plan(ctx, batch, &plan);
   ctx->options[PIE_OPT_OVERLAP] = saved_overlap;
   if (rc != PIE_OK) return rc;

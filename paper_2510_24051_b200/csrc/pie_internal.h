@@ -192,6 +192,10 @@ struct AttnParams {
   int64_t page_bytes;
   int32_t n_q_heads, n_kv_heads, G;
   float scale_log2;  // log2(e) / sqrt(D)
+  // 1: signal dependent launches only when a block is done.  Side by side with another kernel an
+  // early signal would let the NEXT kernel of the stream (a merge) occupy the SMs meant for the
+  // neighbour with blocks that only wait; alone, the early signal hides the next launch.
+  int32_t late_trigger;
 };
 
 int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, const void* v_new, cudaStream_t s);

@@ -715,19 +715,36 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   int split_sms = ctx->options[PIE_OPT_SPLIT_SMS] > 0 ? std::min(ctx->options[PIE_OPT_SPLIT_SMS], ctx->n_sms) : ctx->n_sms;
   int tile_sms = ctx->options[PIE_OPT_TILE_SMS] > 0 ? std::min(ctx->options[PIE_OPT_TILE_SMS], ctx->n_sms) : ctx->n_sms;
   plan->overlap = false;
-  if (!split_units.empty() && !tile_units.empty() && plan->tile_tc && ctx->options[PIE_OPT_OVERLAP] == 1 &&
-      ctx->options[PIE_OPT_SPLIT_SMS] == 0 && ctx->options[PIE_OPT_TILE_SMS] == 0 && ctx->n_sms >= 16) {
-    double split_bytes = 0, tile_flops = 0;
-    for (const Unit& u : split_units) split_bytes += (double)(u.page_end - u.page_begin) * 2.0 * P * cfg.head_dim * 2.0;
-    for (const Unit& u : tile_units) tile_flops += (double)(u.page_end - u.page_begin) * P * 4.0 * cfg.head_dim * 256.0;
-    const double t_split = split_bytes / 6.0e12, t_tile = tile_flops / 1.0e15;  // whole-chip estimates, seconds
-    const int floor_split = (ctx->n_sms * 5) / 8;
-    int n_split = (int)(ctx->n_sms * t_split / (t_split + t_tile) + 0.5);
-    n_split = std::max(n_split, floor_split);
-    n_split = std::min(n_split, ctx->n_sms - 8);
-    split_sms = n_split;
-    tile_sms = ctx->n_sms - n_split;
-    plan->overlap = true;
+  if (!split_units.empty() && !tile_units.empty() && plan->tile_tc && ctx->options[PIE_OPT_OVERLAP] != 2 && ctx->n_sms >= 16) {
+    if (ctx->options[PIE_OPT_SPLIT_SMS] > 0 && ctx->options[PIE_OPT_TILE_SMS] > 0) {
+      plan->overlap = ctx->options[PIE_OPT_OVERLAP] == 1 && split_sms + tile_sms <= ctx->n_sms;   // explicit budgets, on request
+    } else {
+      // Model: the decode kernel moves `split_bytes` at the chip's copy rate as long as it has about
+      // 60 % of the SMs, and proportionally slower below that; the row-tile kernel's time scales with
+      // 1 / SMs.  Take the budget that minimises the later finish, and run side by side only if that
+      // beats one kernel after the other.
+      double split_bytes = 0, tile_flops = 0;
+      for (const Unit& u : split_units) split_bytes += (double)(u.page_end - u.page_begin) * 2.0 * P * cfg.head_dim * 2.0;
+      for (const Unit& u : tile_units) tile_flops += (double)(u.page_end - u.page_begin) * P * 4.0 * cfg.head_dim * u.nrows;
+      const double t_split = split_bytes / 6.4e12, t_tile = tile_flops / 0.48e15;  // whole-chip estimates, seconds (rates measured on the mixed workload)
+      const double sat = 0.6 * ctx->n_sms;                                         // SMs that saturate the memory system
+      int best_nt = 0;
+      double best_t = 1e30;
+      for (int nt = 8; nt <= ctx->n_sms - 16; nt += 2) {
+        const int ns = ctx->n_sms - nt;
+        const double ts = t_split * std::max(1.0, sat / ns), tt = t_tile * ctx->n_sms / nt;
+        const double t = std::max(ts, tt);
+        if (t < best_t) {
+          best_t = t;
+          best_nt = nt;
+        }
+      }
+      if (best_nt > 0 && (ctx->options[PIE_OPT_OVERLAP] == 1 || (best_t < 0.90 * (t_split + t_tile) && t_split + t_tile > 150e-6))) {
+        tile_sms = best_nt;
+        split_sms = ctx->n_sms - best_nt;
+        plan->overlap = true;
+      }
+    }
   }
   // row tiles first: the cascade pieces get their partial slots, which the split units of the
   // cascaded requests then name as further sources of their merge groups
@@ -819,6 +836,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   info.mask_words = (int64_t)plan->mask_words.size();
   info.workspace_bytes = ((int64_t)plan->split.n_slots * plan->split.slot_rows +
                           (int64_t)plan->tile.n_slots * plan->tile.slot_rows) * (cfg.head_dim + 1) * 4;
+  info.side_by_side_sms = plan->overlap ? plan->tile.grid : 0;
   info.launches = (plan->append_fused ? 0 : 1) + (info.num_simple_rows ? 1 : 0) + (info.num_split_items ? 1 : 0) +
                   (info.num_tile_items ? 1 : 0) + (plan->split.merges.empty() ? 0 : 1) +
                   (plan->tile.merges.empty() ? 0 : 1);
