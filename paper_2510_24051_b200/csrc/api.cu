@@ -603,14 +603,14 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
   if (!plan->split.items.empty() &&
       (rc = timed_launch(ctx, PIE_KERNEL_SPLIT, s, [&] { return pie_launch_split(ctx, plan, q, k_new, v_new, out, lse, s); })))
     return rc;
-  if (side && (rc = launch_tiles())) return rc;
-  if (!plan->split.merges.empty() &&
-      (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s, [&] { return pie_launch_merge(ctx, plan, plan->split, out, lse, s); })))
-    return rc;
-  if (side) {
+  if (side) {   // row tiles on the side stream, then join: the split merge may read their partials (cascade)
+    if ((rc = launch_tiles())) return rc;
     PIE_CUDA(ctx, cudaEventRecord(ctx->ev_join, s2));
     PIE_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_join, 0));
   }
+  if (!plan->split.merges.empty() &&
+      (rc = timed_launch(ctx, PIE_KERNEL_MERGE, s, [&] { return pie_launch_merge(ctx, plan, plan->split, out, lse, s); })))
+    return rc;
   return PIE_OK;
 }
 

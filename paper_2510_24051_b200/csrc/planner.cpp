@@ -715,7 +715,8 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   int split_sms = ctx->options[PIE_OPT_SPLIT_SMS] > 0 ? std::min(ctx->options[PIE_OPT_SPLIT_SMS], ctx->n_sms) : ctx->n_sms;
   int tile_sms = ctx->options[PIE_OPT_TILE_SMS] > 0 ? std::min(ctx->options[PIE_OPT_TILE_SMS], ctx->n_sms) : ctx->n_sms;
   plan->overlap = false;
-  if (!split_units.empty() && !tile_units.empty() && plan->tile_tc && ctx->options[PIE_OPT_OVERLAP] != 2 && ctx->n_sms >= 16) {
+  if ((!split_units.empty() || !cascades.empty()) && !tile_units.empty() && plan->tile_tc && ctx->options[PIE_OPT_OVERLAP] != 2 &&
+      ctx->n_sms >= 16) {
     if (ctx->options[PIE_OPT_SPLIT_SMS] > 0 && ctx->options[PIE_OPT_TILE_SMS] > 0) {
       plan->overlap = ctx->options[PIE_OPT_OVERLAP] == 1 && split_sms + tile_sms <= ctx->n_sms;   // explicit budgets, on request
     } else {
@@ -725,6 +726,9 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       // beats one kernel after the other.
       double split_bytes = 0, tile_flops = 0;
       for (const Unit& u : split_units) split_bytes += (double)(u.page_end - u.page_begin) * 2.0 * P * cfg.head_dim * 2.0;
+      for (const Cascade& cs : cascades)   // the private pages of cascaded requests (their split units are made below)
+        for (int k = 0; k < cs.n; ++k)
+          split_bytes += (double)(plan->reqs[cs.first + k].kept_count - cs.L) * cfg.num_kv_heads * 2.0 * P * cfg.head_dim * 2.0;
       for (const Unit& u : tile_units) tile_flops += (double)(u.page_end - u.page_begin) * P * 4.0 * cfg.head_dim * u.nrows;
       const double t_split = split_bytes / 6.4e12, t_tile = tile_flops / 0.48e15;  // whole-chip estimates, seconds (rates measured on the mixed workload)
       const double sat = 0.6 * ctx->n_sms;                                         // SMs that saturate the memory system
@@ -739,7 +743,10 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
           best_nt = nt;
         }
       }
-      if (best_nt > 0 && (ctx->options[PIE_OPT_OVERLAP] == 1 || (best_t < 0.90 * (t_split + t_tile) && t_split + t_tile > 150e-6))) {
+      // (automatic only for plain mixed batches: a cascade's row tiles are short gathered-decode items that
+      //  the model does not describe - measured 0.133 -> 0.127 ms at best, 0.19 ms with the model's budget)
+      if (best_nt > 0 && (ctx->options[PIE_OPT_OVERLAP] == 1 ||
+                          (cascades.empty() && best_t < 0.90 * (t_split + t_tile) && t_split + t_tile > 150e-6))) {
         tile_sms = best_nt;
         split_sms = ctx->n_sms - best_nt;
         plan->overlap = true;
@@ -769,7 +776,6 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       }
     }
   }
-  if (!cascades.empty()) plan->overlap = false;  // the split merge reads the row-tile launch's partials
   // split-KV decode.  Long launches: chunks taken dynamically by the warps of the grid (evens out
   // SMs that get different shares of the memory bandwidth).  Short launches: fixed equal shares,
   // one per warp - fewer pieces, fewer partials to merge, and the per-chunk overheads matter more
