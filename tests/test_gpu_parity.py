@@ -252,15 +252,20 @@ def test_rope_inside_the_path_matches_oracle(name, explicit_pos):
         pie.pie_destroy(ctx)
 
 
-def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
-    """pie_forward only enqueues kernels on the caller's stream (no allocation, no synchronisation), so a
-    decode step can be captured once and replayed; the replay must reproduce the eager result bit for bit."""
+@pytest.mark.parametrize("side_by_side", [0, 1])
+def test_forward_can_be_captured_in_a_cuda_graph_and_replayed(side_by_side):
+    """pie_forward only enqueues kernels (no allocation, no synchronisation), so a step can be captured
+    once and replayed; the replay must reproduce the eager result bit for bit.  With the decode and
+    prefill kernels side by side the capture includes the fork to and the join from the internal stream."""
     import paper_2510_24051_b200 as pie
     from tests._gpu import GpuPool
     wl = configs.small("mixed_prefill_decode")
     with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
         gp.install(wl)
+        if side_by_side:
+            pie.pie_set_option(gp.ctx, pie.PIE_OPT_OVERLAP, 1)
         plan = gp.plan(wl)
+        assert (pie.pie_plan_get_info(plan)["side_by_side_sms"] > 0) == bool(side_by_side)
         q, k, v = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
         ref_out, ref_lse = gp.forward(plan, q, k, v)
         out = torch.zeros_like(ref_out)
