@@ -35,7 +35,10 @@ __global__ void append_kernel(uint8_t* __restrict__ pool, const uint8_t* __restr
   }
 }
 
-// K2: copy_kvpage (Table 1).  ops[k] = {src, dst, src_off, dst_off, ntok}; one block per op.
+// K2: copy_kvpage (Table 1).  ops[k] = {src, dst, src_off, dst_off, ntok}; kCopySplit blocks per
+// op, 16 bytes per thread and step, four loads in flight before the first store (the copy is pure
+// latency: a page is a few tens of KB).
+constexpr int kCopySplit = 4;
 __global__ void copy_kernel(uint8_t* __restrict__ pool, const int32_t* __restrict__ ops, PoolGeom g) {
   pie_pdl_launch_dependents();
   pie_pdl_wait();
@@ -43,14 +46,20 @@ __global__ void copy_kernel(uint8_t* __restrict__ pool, const int32_t* __restric
   const int src = op[0], dst = op[1], so = op[2], dof = op[3], n = op[4];
   const int chunks = g.row_bytes >> 4;
   const int per_tok = 2 * g.n_kv_heads * chunks;
-  for (int i = threadIdx.x; i < n * per_tok; i += blockDim.x) {
-    int t = i / per_tok, rem = i - t * per_tok;
-    int blk = rem / chunks, c = rem - blk * chunks;  // blk = head*2 + kv
-    const uint8_t* s = pool + (int64_t)src * g.page_bytes + (int64_t)blk * g.block_bytes +
-                       pie_chunk_offset(g.slab_bytes, so + t, c);
-    uint8_t* d = pool + (int64_t)dst * g.page_bytes + (int64_t)blk * g.block_bytes +
-                 pie_chunk_offset(g.slab_bytes, dof + t, c);
-    *reinterpret_cast<uint4*>(d) = *reinterpret_cast<const uint4*>(s);
+  const int total = n * per_tok, stride = blockDim.x * kCopySplit;
+  auto addr = [&](int i, int page, int off) -> int64_t {
+    const int t = i / per_tok, rem = i - t * per_tok;
+    const int blk = rem / chunks, c = rem - blk * chunks;  // blk = head*2 + kv
+    return (int64_t)page * g.page_bytes + (int64_t)blk * g.block_bytes + pie_chunk_offset(g.slab_bytes, off + t, c);
+  };
+  for (int i0 = blockIdx.y * blockDim.x + threadIdx.x; i0 < total; i0 += 4 * stride) {
+    uint4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (i0 + k * stride < total) v[k] = *reinterpret_cast<const uint4*>(pool + addr(i0 + k * stride, src, so));
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (i0 + k * stride < total) *reinterpret_cast<uint4*>(pool + addr(i0 + k * stride, dst, dof)) = v[k];
   }
 }
 
@@ -220,7 +229,7 @@ int pie_append_and_q(pie_ctx* ctx, const pie_plan* plan, const void* q, const vo
 }
 
 int pie_launch_copy(pie_ctx* ctx, int n, const int32_t* d_ops, cudaStream_t s) {
-  PIE_CUDA(ctx, pie_launch_pdl(copy_kernel, dim3(n), dim3(256), 0, s, ctx->pool, d_ops, ctx->geom));
+  PIE_CUDA(ctx, pie_launch_pdl(copy_kernel, dim3(n, kCopySplit), dim3(256), 0, s, ctx->pool, d_ops, ctx->geom));
   return PIE_OK;
 }
 
