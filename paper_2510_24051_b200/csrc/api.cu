@@ -125,14 +125,12 @@ bool page_ok(const pie_ctx* ctx, int32_t id) {
   return id >= 0 && id < ctx->cfg.num_pages && ctx->allocated[id];
 }
 
+}  // namespace
+
 // Device image of a plan: every array the kernels read, 256-byte aligned, followed by the fp32
 // partial workspaces of the two tile launches.
-struct PlanLayout {
-  size_t reqs, kept, mask, app, tok, pos, simple, items[2], cta[2], merges[2], ctr[2], ws_o[2], ws_lse[2];
-  size_t upload, total;
-};
 
-PlanLayout plan_layout(const pie_ctx* ctx, const pie_plan* plan) {
+PlanLayout pie_plan_layout(const pie_ctx* ctx, const pie_plan* plan) {
   PlanLayout L{};
   size_t off = 0;
   auto place = [&](size_t bytes) {
@@ -164,7 +162,7 @@ PlanLayout plan_layout(const pie_ctx* ctx, const pie_plan* plan) {
   return L;
 }
 
-void plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
+void pie_plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
   auto cp = [&](size_t off, const void* p, size_t bytes) {
     if (bytes) std::memcpy(dst + off, p, bytes);
   };
@@ -187,7 +185,7 @@ void plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
   }
 }
 
-void plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base) {
+void pie_plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base) {
   plan->d_reqs = (PieReq*)(base + L.reqs);
   plan->d_kept = (int2*)(base + L.kept);
   plan->d_mask = (uint32_t*)(base + L.mask);
@@ -206,7 +204,6 @@ void plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base) {
   }
 }
 
-}  // namespace
 
 int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, const void* v_new, cudaStream_t s) {
   if (plan->T == 0) return PIE_OK;
@@ -515,9 +512,9 @@ int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pi
   }
   if (!ctx->host_only && plan->R > 0) {
     cudaStream_t s = (cudaStream_t)stream;
-    const PlanLayout L = plan_layout(ctx, plan);
+    const PlanLayout L = pie_plan_layout(ctx, plan);
     std::vector<uint8_t> host(L.upload);
-    plan_fill(plan, L, host.data());
+    pie_plan_fill(plan, L, host.data());
     cudaError_t e = cudaSetDevice(ctx->cfg.device);
     if (e == cudaSuccess) e = cudaMalloc(&plan->d_blob, std::max<size_t>(L.total, 256));
     if (e == cudaSuccess && L.upload)
@@ -529,7 +526,7 @@ int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pi
       delete plan;
       return PIE_ERR_CUDA;
     }
-    plan_bind(plan, L, (uint8_t*)plan->d_blob);
+    pie_plan_bind(plan, L, (uint8_t*)plan->d_blob);
   }
   *out = plan;
   return PIE_OK;
@@ -676,7 +673,7 @@ int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, c
     if ((rc = ensure_buffer(ctx, &ctx->d_io, &ctx->io_bytes, io_layout((size_t)plan->T)))) return rc;
     if ((rc = upload_inputs())) return rc;
   }
-  const PlanLayout L = plan_layout(ctx, plan);
+  const PlanLayout L = pie_plan_layout(ctx, plan);
   if ((rc = ensure_buffer(ctx, &ctx->d_planbuf, &ctx->planbuf_bytes, L.total))) return rc;
   if (ctx->h_stage_bytes < L.upload) {
     if (ctx->h_stage) PIE_CUDA(ctx, cudaFreeHost(ctx->h_stage));
@@ -687,8 +684,8 @@ int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, c
     ctx->h_stage_bytes = want;
   }
   uint8_t* io = (uint8_t*)ctx->d_io;
-  plan_fill(plan, L, (uint8_t*)ctx->h_stage);
-  plan_bind(plan, L, (uint8_t*)ctx->d_planbuf);
+  pie_plan_fill(plan, L, (uint8_t*)ctx->h_stage);
+  pie_plan_bind(plan, L, (uint8_t*)ctx->d_planbuf);
   PIE_CUDA(ctx, cudaMemcpyAsync(ctx->d_planbuf, ctx->h_stage, L.upload, cudaMemcpyHostToDevice, s));
   if ((rc = pie_forward(ctx, plan, io, io + o_k, io + o_v, io + o_out, (float*)(io + o_lse), stream))) return rc;
   PIE_CUDA(ctx, cudaMemcpyAsync(out, io + o_out, q_bytes, cudaMemcpyDeviceToHost, s));

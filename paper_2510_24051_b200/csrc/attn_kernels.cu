@@ -936,59 +936,14 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   if (plan.T == 0) return PIE_OK;
   if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
 
-  std::vector<uint8_t> host;
-  auto put = [&](const void* ptr, size_t bytes) {
-    size_t off = (host.size() + 255) & ~(size_t)255;
-    host.resize(off + bytes);
-    if (bytes) memcpy(host.data() + off, ptr, bytes);
-    return off;
-  };
-  const size_t o_reqs = put(plan.reqs.data(), plan.reqs.size() * sizeof(PieReq));
-  const size_t o_kept = put(plan.kept.data(), plan.kept.size() * 4);
-  const size_t o_mask = put(plan.mask_words.data(), plan.mask_words.size() * 4);
-  const size_t o_app = put(plan.append_dst.data(), plan.append_dst.size() * 4);
-  const size_t o_tok = put(plan.tok_req.data(), plan.tok_req.size() * 4);
-  const size_t o_pos = put(plan.positions.data(), plan.positions.size() * 4);
-  const size_t o_simple = put(plan.simple_rows.data(), plan.simple_rows.size() * 4);
-  PieLaunchList* lls[2] = {&plan.split, &plan.tile};
-  size_t o_li[2], o_lc[2], o_lm[2], o_wo[2], o_wl[2], o_ctr[2];
-  for (int k = 0; k < 2; ++k) {
-    o_li[k] = put(lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
-    o_lc[k] = put(lls[k]->cta_ptr.data(), lls[k]->cta_ptr.size() * 4);
-    {
-      const int32_t ctr0[2] = {lls[k]->n_static, 0};  // the dynamic part of the item list starts here
-      o_ctr[k] = put(ctr0, sizeof(ctr0));
-    }
-    o_lm[k] = put(lls[k]->merges.data(), lls[k]->merges.size() * sizeof(PieMerge));
-  }
-  size_t total = (host.size() + 255) & ~(size_t)255;
-  const int D = ctx->cfg.head_dim;
-  for (int k = 0; k < 2; ++k) {
-    o_wo[k] = total;
-    total += (((size_t)lls[k]->n_slots * lls[k]->slot_rows * D * 4) + 255) & ~(size_t)255;
-    o_wl[k] = total;
-    total += (((size_t)lls[k]->n_slots * lls[k]->slot_rows * 4) + 255) & ~(size_t)255;
-  }
-  if (total > (size_t)PIE_STATIC_SCRATCH_BYTES) return PIE_ERR_BATCH_TOO_LARGE;  // plan + partials exceed the static scratch
-
+  const PlanLayout L = pie_plan_layout(ctx, &plan);
+  if (L.total > (size_t)PIE_STATIC_SCRATCH_BYTES) return PIE_ERR_BATCH_TOO_LARGE;  // plan + partials exceed the static scratch
   // Nothing in the scratch has to start at zero: every plan array is overwritten by this copy
-  // and every partial row is written by the attention kernel before the merge reads it.
+  // and every partial row is written by the attention kernel before a merge reads it.
+  std::vector<uint8_t> host(L.upload);
+  pie_plan_fill(&plan, L, host.data());
   PIE_CUDA(ctx, cudaMemcpyAsync(base, host.data(), host.size(), cudaMemcpyHostToDevice, s));
-  plan.d_reqs = (PieReq*)(base + o_reqs);
-  plan.d_kept = (int2*)(base + o_kept);
-  plan.d_mask = (uint32_t*)(base + o_mask);
-  plan.d_append_dst = (int32_t*)(base + o_app);
-  plan.d_tok_req = (int32_t*)(base + o_tok);
-  plan.d_positions = (int32_t*)(base + o_pos);
-  plan.d_simple_rows = (int32_t*)(base + o_simple);
-  for (int k = 0; k < 2; ++k) {
-    lls[k]->d_items = (PieItem*)(base + o_li[k]);
-    lls[k]->d_cta_ptr = (int32_t*)(base + o_lc[k]);
-    lls[k]->d_merges = (PieMerge*)(base + o_lm[k]);
-    lls[k]->d_work_ctr = (int32_t*)(base + o_ctr[k]);
-    lls[k]->d_ws_o = (float*)(base + o_wo[k]);
-    lls[k]->d_ws_lse = (float*)(base + o_wl[k]);
-  }
+  pie_plan_bind(&plan, L, base);
   if ((rc = pie_append_and_q(ctx, &plan, q, k_new, v_new, s, &q))) return rc;
   if (!plan.simple_rows.empty() && (rc = pie_launch_simple(ctx, &plan, q, out, lse, s))) return rc;
   if (!plan.split.items.empty() && (rc = pie_launch_split(ctx, &plan, q, k_new, v_new, out, lse, s))) return rc;

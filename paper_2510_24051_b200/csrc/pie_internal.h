@@ -217,6 +217,18 @@ bool pie_tc_supported(const pie_ctx* ctx);
 // n_tokens: rows of the Q tensor (the batch's query tokens), for the bounds of the Q tensor map
 int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_tokens, cudaStream_t s);
 
+// Device image of a plan (every array the kernels read, 256-byte aligned, then the fp32 partial
+// workspaces of the two tile launches): offsets, host-side fill of the uploaded part, binding of the
+// plan's device pointers to an image at `base`.
+struct PlanLayout {
+  size_t reqs, kept, mask, app, tok, pos, simple, items[2], cta[2], merges[2], ctr[2], ws_o[2], ws_lse[2];
+  size_t upload, total;
+};
+
+PlanLayout pie_plan_layout(const pie_ctx* ctx, const pie_plan* plan);
+void pie_plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst);
+void pie_plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base);
+
 int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);  // host part (planner.cc)
 
 #define PIE_CUDA(ctx, expr)                                   \
