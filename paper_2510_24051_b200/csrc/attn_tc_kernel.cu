@@ -147,34 +147,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-#define TRACEL(tag)
-#define TRACE_LD_END()
-// exp2 of two values on the FMA pipe (the MUFU unit is the softmax bottleneck: 4 results per clock
-// and SM sub-partition): round to the nearest integer n with the 1.5 * 2^23 trick, degree-3
-// minimax polynomial for 2^f on f in [-0.5, 0.5] (relative error 7.5e-5, far below the bf16
-// rounding of P), n added into the exponent field.  Inputs are clamped at -126, so a masked
-// entry (-inf) yields ~1e-38 instead of 0: harmless in a row that has live entries, and rows
-// without any are recognised by their maximum, not by their sum.
-__device__ __forceinline__ void poly_exp2x2(float x0, float x1, float& p0, float& p1) {
-  const float kMagic = 12582912.f;
-  const uint64_t xc = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-  const uint64_t y = add_f32x2(xc, pack_f32x2(kMagic, kMagic));
-  const uint64_t r = add_f32x2(y, pack_f32x2(-kMagic, -kMagic));
-  const uint64_t f = fma_f32x2(r, pack_f32x2(-1.f, -1.f), xc);
-  uint64_t q = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), f, pack_f32x2(0.2426111251f, 0.2426111251f));
-  q = fma_f32x2(q, f, pack_f32x2(0.6932609677f, 0.6932609677f));
-  q = fma_f32x2(q, f, pack_f32x2(0.9999280572f, 0.9999280572f));
-  float y0, y1, q0, q1;
-  unpack_f32x2(y, y0, y1);
-  unpack_f32x2(q, q0, q1);
-  p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(y0) << 23));
-  p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(y1) << 23));
-}
-#ifndef PIE_POLY_MASK
-#define PIE_POLY_MASK 0x0000
-#endif
-constexpr uint32_t kPolyMask = PIE_POLY_MASK;   // bit b: pair b of a 32-column chunk is exponentiated on the FMA pipe
-
 constexpr float kNegInf = -__builtin_huge_valf();
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileM = 128;    // rows per Q tile
@@ -467,11 +439,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
       const PieItem item = p.items[it];
       if (item.page_end == item.page_begin) continue;
       const int nt = item.nrows > kTileM ? 2 : 1;
-      TRACEL(80);
       for (int t = 0; t < nt; ++t) {
         mbar_wait(smem_u32(q_free + t), (n_t[t & 1] & 1) ^ 1, p.status);
         ++n_t[t & 1];
-        TRACEL(81);
         if (use_qmap) {
           if (elect_one()) {
             mbar_expect_tx(smem_u32(q_full + t), C::QTILE);
@@ -502,10 +472,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(q_full + t));
         }
-        TRACEL(83);
       }
     }
-    TRACE_LD_END();
   } else {
     // ================================================================ softmax warpgroups
     const int t = warp >> 2;                       // Q tile of this warpgroup
@@ -656,11 +624,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
               float e0, e1, e2, e3;
               unpack_f32x2(fma_f32x2(pack_f32x2(x[c], x[c + 1]), scale2, negm2), e0, e1);
               unpack_f32x2(fma_f32x2(pack_f32x2(x[c + 2], x[c + 3]), scale2, negm2), e2, e3);
-              float p0, p1, p2, p3;
-              if ((kPolyMask >> (c >> 1)) & 1u) poly_exp2x2(e0, e1, p0, p1);
-              else p0 = fast_exp2(e0), p1 = fast_exp2(e1);
-              if ((kPolyMask >> ((c >> 1) + 1)) & 1u) poly_exp2x2(e2, e3, p2, p3);
-              else p2 = fast_exp2(e2), p3 = fast_exp2(e3);
+              const float p0 = fast_exp2(e0), p1 = fast_exp2(e1), p2 = fast_exp2(e2), p3 = fast_exp2(e3);
               psum_a = add_f32x2(psum_a, pack_f32x2(p0, p1));
               psum_b = add_f32x2(psum_b, pack_f32x2(p2, p3));
               pk[c >> 1] = pack_bf16(p0, p1);
