@@ -183,14 +183,23 @@ typedef struct pie_plan_info {
  * PIE_ERR_BATCH_TOO_LARGE, PIE_ERR_MASK.  *out is set only on success.  The upload uses
  * `stream`; the call returns after it completed. */
 int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pie_plan** out);
+/* Ends the plan's life.  The context keeps a few destroyed plans - host arrays, pinned upload
+ * image and device arrays - and pie_plan_forward reuses them, so a loop that plans every step
+ * stops allocating after its first steps (no cudaMalloc, no cudaFree and its device-wide
+ * synchronisation per batch).  The call does not wait: it marks the point behind the plan's
+ * latest pie_forward on that forward's stream, and the reuse waits for that point.  Destroy a
+ * plan only when no captured graph that holds its forward will be launched again, and before
+ * the stream of its latest forward is destroyed.  pie_destroy releases the kept plans. */
 int pie_plan_destroy(pie_plan* plan);
 int pie_plan_get_info(const pie_plan* plan, pie_plan_info* out);
 
 /* Planner introspection for tests: copy one of the plan's host-side arrays into buf (host).
  * which: 0 = packed mask words (uint32), 1 = kept page list (int32 pairs: physical id,
  * logical page | 0x80000000 if the page needs mask evaluation), 2 = append destinations
- * (int32 per query token: page * page_size + slot).  *out_bytes receives the array size; data
- * is copied only if cap_bytes is large enough. */
+ * (int32 per query token: page * page_size + slot), 3 = the plan's whole upload image (request
+ * records, kept pages, masks, append destinations, work items, share boundaries, merge groups
+ * and counters in device layout, gaps zeroed; size a multiple of 4).  *out_bytes receives the
+ * array size; data is copied only if cap_bytes is large enough. */
 int pie_plan_debug_read(const pie_plan* plan, int which, void* buf, int64_t cap_bytes,
                         int64_t* out_bytes);
 

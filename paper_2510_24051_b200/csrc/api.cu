@@ -354,6 +354,14 @@ int pie_destroy(pie_ctx* ctx) {
     for (auto e : ctx->free_events) cudaEventDestroy(e);
   }
   delete ctx->host_plan;
+  for (pie_plan* plan : ctx->parked_plans) {
+    if (!ctx->host_only) {
+      if (plan->d_blob) cudaFree(plan->d_blob);
+      if (plan->h_image) cudaFreeHost(plan->h_image);
+      if (plan->idle) cudaEventDestroy(plan->idle);
+    }
+    delete plan;
+  }
   delete ctx;
   return PIE_OK;
 }
@@ -500,45 +508,109 @@ int pie_copy_kvpage(pie_ctx* ctx, int32_t n, const int32_t* src, const int32_t* 
   return timed_launch(ctx, PIE_KERNEL_COPY, s, [&] { return pie_launch_copy(ctx, n, (const int32_t*)ctx->d_stage, s); });
 }
 
+// Plans are recycled: pie_plan_destroy parks up to kParkedPlans objects in the context, with their
+// host vectors, pinned image and device arrays, and pie_plan_forward takes one back.  A serving
+// loop that plans every step therefore stops allocating after its first steps: no cudaMalloc and
+// no cudaFree (with its device-wide synchronisation) per batch.
+static const size_t kParkedPlans = 4;
+
+static void release_plan(pie_plan* plan) {
+  if (plan->d_blob || plan->h_image || plan->idle) {
+    cudaSetDevice(plan->ctx->cfg.device);
+    if (plan->d_blob) cudaFree(plan->d_blob);   // (synchronises: nothing can still be reading the arrays afterwards)
+    if (plan->h_image) cudaFreeHost(plan->h_image);
+    if (plan->idle) cudaEventDestroy(plan->idle);
+  }
+  delete plan;
+}
+
 int pie_plan_forward(pie_ctx* ctx, const pie_batch_desc* batch, void* stream, pie_plan** out) {
   if (!ctx || !batch || !out) return PIE_ERR_INVALID;
-  pie_plan* plan = new (std::nothrow) pie_plan();
+  pie_plan* plan = nullptr;
+  if (!ctx->parked_plans.empty()) {
+    plan = ctx->parked_plans.back();
+    ctx->parked_plans.pop_back();
+  } else {
+    plan = new (std::nothrow) pie_plan();
+  }
   if (!plan) return PIE_ERR_INVALID;
   plan->ctx = ctx;
+  auto give_back = [&]() {   // the object goes back as it came: its device arrays were not touched
+    if (ctx->parked_plans.size() < kParkedPlans) ctx->parked_plans.push_back(plan);
+    else release_plan(plan);
+  };
   int rc = pie_build_plan(ctx, batch, plan);
   if (rc != PIE_OK) {
-    delete plan;
+    give_back();
     return rc;
   }
   if (!ctx->host_only && plan->R > 0) {
     cudaStream_t s = (cudaStream_t)stream;
     const PlanLayout L = pie_plan_layout(ctx, plan);
-    std::vector<uint8_t> host(L.upload);
-    pie_plan_fill(plan, L, host.data());
     cudaError_t e = cudaSetDevice(ctx->cfg.device);
-    if (e == cudaSuccess) e = cudaMalloc(&plan->d_blob, std::max<size_t>(L.total, 256));
-    if (e == cudaSuccess && L.upload)
-      e = cudaMemcpyAsync(plan->d_blob, host.data(), L.upload, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && plan->idle_pending) {   // the forward that last read the device arrays must be over
+      e = cudaEventSynchronize(plan->idle);
+      plan->idle_pending = false;
+    }
+    if (e == cudaSuccess && plan->h_image_bytes < L.upload) {
+      if (plan->h_image) cudaFreeHost(plan->h_image);
+      plan->h_image = nullptr;
+      plan->h_image_bytes = 0;
+      const size_t want = std::max(L.upload + L.upload / 4, (size_t)1 << 16);
+      e = cudaMallocHost(&plan->h_image, want);
+      if (e == cudaSuccess) plan->h_image_bytes = want;
+    }
+    if (e == cudaSuccess && plan->d_blob_bytes < L.total) {
+      if (plan->d_blob) cudaFree(plan->d_blob);
+      plan->d_blob = nullptr;
+      plan->d_blob_bytes = 0;
+      const size_t want = std::max(L.total + L.total / 4, (size_t)1 << 16);
+      e = cudaMalloc(&plan->d_blob, want);
+      if (e == cudaSuccess) plan->d_blob_bytes = want;
+    }
+    if (e == cudaSuccess) {
+      pie_plan_fill(plan, L, (uint8_t*)plan->h_image);
+      if (L.upload) e = cudaMemcpyAsync(plan->d_blob, plan->h_image, L.upload, cudaMemcpyHostToDevice, s);
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
       ctx->cuda_error = std::string("plan upload: ") + cudaGetErrorString(e);
-      if (plan->d_blob) cudaFree(plan->d_blob);
-      delete plan;
+      release_plan(plan);
       return PIE_ERR_CUDA;
     }
     pie_plan_bind(plan, L, (uint8_t*)plan->d_blob);
   }
+  plan->used = false;
+  plan->many_streams = false;
   *out = plan;
   return PIE_OK;
 }
 
 int pie_plan_destroy(pie_plan* plan) {
   if (!plan) return PIE_ERR_INVALID;
-  if (plan->d_blob) {
-    cudaSetDevice(plan->ctx->cfg.device);
-    cudaFree(plan->d_blob);
+  pie_ctx* ctx = plan->ctx;
+  if (!ctx || ctx->parked_plans.size() >= kParkedPlans) {
+    release_plan(plan);
+    return PIE_OK;
   }
-  delete plan;
+  if (plan->used && plan->d_blob) {
+    // a forward may still be reading the device arrays: mark the point behind it on its stream
+    cudaSetDevice(ctx->cfg.device);
+    cudaError_t e = cudaSuccess;
+    if (plan->many_streams) e = cudaErrorInvalidValue;   // forwards on several streams: one event cannot follow them all
+    if (e == cudaSuccess && !plan->idle) e = cudaEventCreateWithFlags(&plan->idle, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventRecord(plan->idle, plan->last_stream);
+    if (e == cudaSuccess) {
+      plan->idle_pending = true;
+    } else {   // (e.g. the stream no longer exists) fall back to waiting for the whole device
+      cudaGetLastError();
+      cudaDeviceSynchronize();
+      plan->idle_pending = false;
+    }
+  }
+  plan->used = false;
+  plan->many_streams = false;
+  ctx->parked_plans.push_back(plan);
   return PIE_OK;
 }
 
@@ -552,6 +624,15 @@ int pie_plan_debug_read(const pie_plan* plan, int which, void* buf, int64_t cap_
   if (!plan || !out_bytes) return PIE_ERR_INVALID;
   const void* p = nullptr;
   int64_t n = 0;
+  if (which == 3) {   // the whole image as it is uploaded: every array the kernels read, in device layout
+    const PlanLayout L = pie_plan_layout(plan->ctx, plan);
+    *out_bytes = (int64_t)L.upload;
+    if (buf && cap_bytes >= (int64_t)L.upload && L.upload > 0) {
+      std::memset(buf, 0, L.upload);   // (alignment gaps between the arrays)
+      pie_plan_fill(plan, L, (uint8_t*)buf);
+    }
+    return PIE_OK;
+  }
   switch (which) {
     case 0: p = plan->mask_words.data(); n = (int64_t)plan->mask_words.size() * 4; break;
     case 1: p = plan->kept.data(); n = (int64_t)plan->kept.size() * 4; break;
@@ -571,6 +652,10 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
   if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
   cudaStream_t s = (cudaStream_t)stream;
   PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  // (a recycled plan's device arrays are rewritten only behind the forwards that read them)
+  if (plan->used && plan->last_stream != s) plan->many_streams = true;
+  plan->last_stream = s;
+  plan->used = true;
   const void* q_in = q;
   int rc = plan->append_fused ? PIE_OK  // (q stays q_in: the split-KV kernel writes the new rows itself)
                               : timed_launch(ctx, PIE_KERNEL_APPEND, s, [&] { return pie_append_and_q(ctx, plan, q_in, k_new, v_new, s, &q); });

@@ -120,6 +120,16 @@ struct pie_plan {
   pie_plan_info info{};
   // device
   void* d_blob = nullptr;           // one allocation holding every array below
+  size_t d_blob_bytes = 0;
+  void* h_image = nullptr;          // pinned host copy of the uploaded part (pie_plan_forward)
+  size_t h_image_bytes = 0;
+  // recycling (pie_plan_destroy parks the object, pie_plan_forward takes it back): the device
+  // arrays may be overwritten only after the last forward that read them has finished
+  mutable cudaStream_t last_stream = nullptr;   // stream of the latest pie_forward with this plan
+  mutable bool used = false;                    // some pie_forward has read the device arrays
+  mutable bool many_streams = false;            // ... and not all of them on last_stream
+  cudaEvent_t idle = nullptr;                   // recorded behind that forward when the plan is parked
+  bool idle_pending = false;
   PieReq* d_reqs = nullptr;
   int2* d_kept = nullptr;
   uint32_t* d_mask = nullptr;
@@ -155,6 +165,7 @@ struct pie_ctx {
   void* h_stage = nullptr;  // pinned host staging of the plan image (pie_forward_host)
   size_t h_stage_bytes = 0;
   pie_plan* host_plan = nullptr;  // reused plan object of pie_forward_host
+  std::vector<pie_plan*> parked_plans;  // destroyed plans kept for reuse: host arrays, pinned image, device arrays
   std::string cuda_error;
   int options[PIE_NUM_OPTIONS] = {0, 0, 0, 0};
   cudaStream_t side_stream = nullptr;  // second stream of overlapped mixed batches

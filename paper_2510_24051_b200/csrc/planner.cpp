@@ -9,27 +9,51 @@
 #include <atomic>
 #include <cstring>
 #include <thread>
+#if defined(__SSE2__)
+#include <emmintrin.h>
+#endif
 
 #include "pie_internal.h"
 
 namespace {
 
-// Pack `n` bool bytes (each 0 or 1) into bits, LSB first.  Returns false on a byte > 1.
-bool pack_row(const uint8_t* src, int64_t n, uint32_t* dst) {
+// Pack `n` bool bytes (each 0 or 1) into bits, LSB first, and zero the rest of the row: all
+// `row_words` words of `dst` are written (the destination need not be cleared beforehand).
+// Returns false on a byte > 1.
+bool pack_row(const uint8_t* src, int64_t n, uint32_t* dst, int row_words) {
   int64_t j = 0;
   uint8_t bad = 0;
-  for (; j + 8 <= n; j += 8) {
-    uint64_t x;
-    std::memcpy(&x, src + j, 8);
-    bad |= (x & 0xFEFEFEFEFEFEFEFEull) != 0;
-    // gather the low bit of each byte into one byte (byte k -> bit k)
-    uint32_t b = (uint32_t)((x * 0x0102040810204080ull) >> 56) & 0xFFu;
-    dst[j >> 5] |= b << (j & 31);
+#if defined(__SSE2__)
+  // 32 bytes -> one word: bit 0 of every byte moved to its sign bit, then gathered by movemask
+  __m128i bad_v = _mm_setzero_si128();
+  const __m128i not_bool = _mm_set1_epi8((char)0xFE);
+  for (; j + 32 <= n; j += 32) {
+    const __m128i a = _mm_loadu_si128((const __m128i*)(src + j)), c = _mm_loadu_si128((const __m128i*)(src + j + 16));
+    bad_v = _mm_or_si128(bad_v, _mm_and_si128(_mm_or_si128(a, c), not_bool));
+    const uint32_t lo = (uint32_t)_mm_movemask_epi8(_mm_slli_epi16(a, 7)), hi = (uint32_t)_mm_movemask_epi8(_mm_slli_epi16(c, 7));
+    dst[j >> 5] = lo | (hi << 16);
   }
-  for (; j < n; ++j) {
-    bad |= src[j] > 1;
-    dst[j >> 5] |= (uint32_t)(src[j] & 1) << (j & 31);
+  bad |= _mm_movemask_epi8(_mm_cmpeq_epi8(bad_v, _mm_setzero_si128())) != 0xFFFF;
+#endif
+  int64_t k = j >> 5;   // next word to write (j is a multiple of 32 here)
+  while (j < n) {
+    uint32_t word = 0;
+    const int64_t word_end = std::min<int64_t>(j + 32, n);
+    int sh = 0;
+    for (; j + 8 <= word_end; j += 8, sh += 8) {
+      uint64_t x;
+      std::memcpy(&x, src + j, 8);
+      bad |= (x & 0xFEFEFEFEFEFEFEFEull) != 0;
+      // gather the low bit of each byte into one byte (byte k -> bit k)
+      word |= ((uint32_t)((x * 0x0102040810204080ull) >> 56) & 0xFFu) << sh;
+    }
+    for (; j < word_end; ++j, ++sh) {
+      bad |= src[j] > 1;
+      word |= (uint32_t)(src[j] & 1) << sh;
+    }
+    dst[k++] = word;
   }
+  for (; k < row_words; ++k) dst[k] = 0u;
   return bad == 0;
 }
 
@@ -180,14 +204,16 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
 // balances better than the merge launch costs.
 bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int min_pages_per_warp, int slot_rows,
                      PieLaunchList& ll) {
-  ll.items.clear();
   ll.merges.clear();
-  ll.cta_ptr.clear();
   ll.n_slots = 0;
   ll.slot_rows = slot_rows;
   ll.grid = 0;
   ll.n_static = 0;
-  if (units.empty()) return true;
+  if (units.empty()) {
+    ll.items.clear();
+    ll.cta_ptr.clear();
+    return true;
+  }
   auto size_of = [&](int32_t k) { return (int64_t)std::max(1, units[k].page_end - units[k].page_begin); };
   int64_t W = 0;
   for (size_t k = 0; k < units.size(); ++k) W += size_of((int32_t)k);
@@ -261,9 +287,26 @@ bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int m
   for (int c = 0; c < n_ctas; ++c) max_load = std::max(max_load, load[c]);
   if (max_load * n_ctas * 100 > W * 105) return false;   // the fullest block holds more than 5 % above the average
 
-  ll.items.reserve(units.size() + (size_t)n_ctas * NW);
-  ll.cta_ptr.reserve((size_t)n_ctas * NW + 1);
-  ll.cta_ptr.push_back(0);
+  // (items and warp ranges are written through plain pointers into arrays sized for the worst case,
+  //  every unit whole plus one extra piece per warp; a reused plan keeps the arrays, and every field
+  //  of an item is written here or when the request records are copied in, so nothing is cleared)
+  ll.items.resize(units.size() + (size_t)n_ctas * NW);
+  ll.cta_ptr.resize((size_t)n_ctas * NW + 1);
+  PieItem* const items = ll.items.data();
+  int32_t* const ptr = ll.cta_ptr.data();
+  int32_t n_items = 0, n_ptr = 0, n_slots = 0;
+  ptr[n_ptr++] = 0;
+  auto emit = [&](const Unit& u, int32_t page_begin, int32_t page_end) {
+    PieItem& it = items[n_items++];
+    it.req = u.req;
+    it.kv_head = u.kv_head;
+    it.row0 = u.row0;
+    it.nrows = u.nrows;
+    it.page_begin = page_begin;
+    it.page_end = page_end;
+    it.partial_slot = -1;
+    it.flags = 0;
+  };
   std::vector<int32_t> members;
   for (int c = 0; c < n_ctas; ++c) {
     members.clear();
@@ -272,45 +315,54 @@ bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int m
     const int64_t Wc = load[c];
     const int nw = (int)std::min<int64_t>(NW, std::max<int64_t>(1, Wc / std::max(1, min_pages_per_warp)));
     int w = 0;                                      // warp whose item range is open
-    int64_t w_end = nw == 1 ? Wc : Wc / nw, off = 0;
+    // share w ends at floor((w + 1) Wc / nw) = (w + 1) q + floor((w + 1) rem / nw): stepped, one division per block
+    const int64_t q_share = Wc / nw, rem_share = Wc % nw;
+    int64_t w_end = q_share, acc = rem_share, off = 0;
     int local_groups = 0;
     auto advance_to = [&](int64_t x) {
       while (w + 1 < nw && x >= w_end) {
-        ll.cta_ptr.push_back((int32_t)ll.items.size());
+        ptr[n_ptr++] = n_items;
         ++w;
-        w_end = (w + 1 == nw) ? Wc : ((int64_t)(w + 1) * Wc) / nw;
+        acc += rem_share;
+        w_end += q_share;
+        if (acc >= nw) {
+          acc -= nw;
+          ++w_end;
+        }
       }
     };
     for (int32_t ui : members) {
       const Unit& u = units[ui];
       const int64_t n = size_of(ui);
-      const int first_item = (int)ll.items.size();
+      const int first_item = n_items;
       if (u.page_end == u.page_begin) {
         advance_to(off);
-        ll.items.push_back(make_item(u, u.page_begin, u.page_begin));
+        emit(u, u.page_begin, u.page_begin);
       } else {
         int64_t x = off;
         while (x < off + n) {
           advance_to(x);
           const int64_t end = std::min(std::max(w_end, x + 1), off + n);
-          ll.items.push_back(make_item(u, (int32_t)(u.page_begin + (x - off)), (int32_t)(u.page_begin + (end - off))));
+          emit(u, (int32_t)(u.page_begin + (x - off)), (int32_t)(u.page_begin + (end - off)));
           x = end;
         }
       }
-      const int np = (int)ll.items.size() - first_item;
+      const int np = n_items - first_item;
       if (np > 1) {   // (at most NW - 1 cut units per block, np <= NW)
         for (int k = 0; k < np; ++k) {
-          PieItem& it = ll.items[first_item + k];
-          it.partial_slot = ll.n_slots + k;
+          PieItem& it = items[first_item + k];
+          it.partial_slot = n_slots + k;
           it.flags |= PIE_ITEM_LOCAL_PIECE | (k == 0 ? PIE_ITEM_LOCAL_MERGER : 0u) | ((uint32_t)local_groups << 8) | ((uint32_t)np << 16);
         }
-        ll.n_slots += np;
+        n_slots += np;
         ++local_groups;
       }
       off += n;
     }
-    for (; w < NW; ++w) ll.cta_ptr.push_back((int32_t)ll.items.size());   // close this block's warps (idle ones: empty ranges)
+    for (; w < NW; ++w) ptr[n_ptr++] = n_items;   // close this block's warps (idle ones: empty ranges)
   }
+  ll.items.resize((size_t)n_items);
+  ll.n_slots = n_slots;
   ll.grid = n_ctas * NW;
   return true;
 }
@@ -320,7 +372,7 @@ bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int m
 // third of a warp's fair share), the rest small ones, and the large chunks come first in the
 // list, so the end of the launch is filled with short pieces of work.
 void chunk_units(const std::vector<Unit>& units, int n_warps, PieLaunchList& ll) {
-  ll.items.clear();
+  if (units.empty()) ll.items.clear();
   ll.merges.clear();
   ll.cta_ptr.clear();
   ll.n_slots = 0;
@@ -337,27 +389,59 @@ void chunk_units(const std::vector<Unit>& units, int n_warps, PieLaunchList& ll)
   const int c_big = (int)std::min<int64_t>(128, std::max<int64_t>(4, share / 3));
   const int c_small = std::min(16, std::max(2, c_big / 4));
   const int64_t tail_start = W - W / 5;
-  std::vector<PieItem> small;
+  // first pass: how many large and small chunks there will be (the small ones go behind the large ones)
+  size_t n_big = 0, n_small = 0, n_groups = 0;
+  {
+    int64_t off = 0;
+    for (const Unit& u : units) {
+      const int n = u.page_end - u.page_begin;
+      const bool tail = off >= tail_start;
+      const int c = tail ? c_small : c_big;
+      const int nchunks = (n + c - 1) / c;
+      (tail ? n_small : n_big) += (size_t)nchunks;
+      n_groups += (nchunks > 1 || u.force_partial) ? 1 : 0;
+      off += n;
+    }
+  }
+  ll.items.resize(n_big + n_small);   // (every field of an item is written here or when the request records are copied in)
+  ll.merges.reserve(n_groups);
+  PieItem* big = ll.items.data();
+  PieItem* small = ll.items.data() + n_big;
   int64_t off = 0;
   for (const Unit& u : units) {
     const int n = u.page_end - u.page_begin;
     const bool tail = off >= tail_start;
     const int c = tail ? c_small : c_big;
     const int nchunks = (n + c - 1) / c;
-    std::vector<PieItem>& dst = tail ? small : ll.items;
-    for (int k = 0; k < nchunks; ++k) {  // chunks of equal size (+-1 page)
-      const int b = (int)((int64_t)n * k / nchunks), e = (int)((int64_t)n * (k + 1) / nchunks);
-      PieItem it = make_item(u, u.page_begin + b, u.page_begin + e);
-      if (nchunks > 1 || u.force_partial) it.partial_slot = ll.n_slots + k;
-      dst.push_back(it);
+    PieItem*& dst = tail ? small : big;
+    const bool partial = nchunks > 1 || u.force_partial;
+    // chunks of equal size (+-1 page): chunk k covers [floor(n k / nchunks), floor(n (k + 1) / nchunks)), stepped without divisions
+    const int base = nchunks ? n / nchunks : 0, rem = nchunks ? n % nchunks : 0;
+    int bgn = 0, acc = 0;
+    for (int k = 0; k < nchunks; ++k) {
+      int end = bgn + base;
+      acc += rem;
+      if (acc >= nchunks) {
+        acc -= nchunks;
+        ++end;
+      }
+      PieItem& it = *dst++;
+      it.req = u.req;
+      it.kv_head = u.kv_head;
+      it.row0 = u.row0;
+      it.nrows = u.nrows;
+      it.page_begin = u.page_begin + bgn;
+      it.page_end = u.page_begin + end;
+      it.partial_slot = partial ? ll.n_slots + k : -1;
+      it.flags = 0;
+      bgn = end;
     }
-    if (nchunks > 1 || u.force_partial) {
+    if (partial) {
       ll.merges.push_back(PieMerge{u.req, u.kv_head, u.row0, u.nrows, ll.n_slots, nchunks, u.x_slot0, u.x_nslots, u.x_row0});
       ll.n_slots += nchunks;
     }
     off += n;
   }
-  ll.items.insert(ll.items.end(), small.begin(), small.end());
   ll.grid = (int)std::min<int64_t>(n_warps, (int64_t)ll.items.size());
 }
 
@@ -398,9 +482,12 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     if (kv_len64 > 0x3FFFFFFF) return PIE_ERR_INVALID;
     if (kv_len64 < q_len) return PIE_ERR_INVALID;
     const int32_t* pages = b->page_indices + b->page_indptr[r];
-    for (int k = 0; k < np; ++k) {
-      if (pages[k] < 0 || pages[k] >= cfg.num_pages || !ctx->allocated[pages[k]]) return PIE_ERR_BAD_PAGE;
-    }
+    uint32_t max_id = 0;   // (negative ids wrap to large values)
+    for (int k = 0; k < np; ++k) max_id = std::max(max_id, (uint32_t)pages[k]);
+    if (max_id >= (uint32_t)cfg.num_pages) return PIE_ERR_BAD_PAGE;
+    uint8_t all_allocated = 1;
+    for (int k = 0; k < np; ++k) all_allocated &= ctx->allocated[pages[k]];
+    if (!all_allocated) return PIE_ERR_BAD_PAGE;
     PieReq& q = plan->reqs[r];
     q.q_start = b->qo_indptr[r];
     q.q_len = q_len;
@@ -447,7 +534,11 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     for (int r = 0; r < R && status == PIE_OK; ++r) {
       const PieReq& q = plan->reqs[r];
       const int32_t* pages = b->page_indices + b->page_indptr[r];
-      for (int lp = 0; lp <= q.last_logical; ++lp) {
+      // (common case first: none of the pages the request only reads is written by anybody)
+      const int first_written = (q.kv_len - q.q_len) / P;
+      uint32_t any_written = 0;
+      for (int lp = 0; lp < first_written; ++lp) any_written |= ctx->wmask[pages[lp]];
+      for (int lp = any_written ? 0 : first_written; lp <= q.last_logical; ++lp) {
         int32_t pg = pages[lp];
         uint32_t w = ctx->wmask[pg];
         if (w == 0 || ctx->writer[pg] == r) continue;
@@ -493,17 +584,24 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       q.mask_word_off = 0;
     }
   }
-  plan->mask_words.assign((size_t)n_words, 0u);
+  plan->mask_words.resize((size_t)n_words);   // (every row is written in full below: nothing to clear)
   // every request first writes its kept pages into its own slice of a scratch array (sized for
   // "all pages kept"); the slices are then packed together in request order
-  std::vector<int32_t>& scratch = plan->kept_scratch;
+  int n_threads = 1;
+  if (mask_bytes_total > (4 << 20)) {
+    n_threads = (int)std::min<int64_t>({(int64_t)std::max(1u, std::thread::hardware_concurrency()), 16, (int64_t)R});
+  }
+  // (one thread: the requests are visited in order, so each writes straight behind its predecessor
+  //  in the final list and nothing is packed afterwards)
+  std::vector<int32_t>& scratch = n_threads > 1 ? plan->kept_scratch : plan->kept;
   scratch.resize(2 * (size_t)b->page_indptr[R]);
   std::atomic<int> bad_mask{0};
+  size_t kept_at = 0;   // single-threaded: pages kept so far
   auto do_request = [&](int r) {
     PieReq& q = plan->reqs[r];
     const int32_t* pages = b->page_indices + b->page_indptr[r];
     const int np = q.last_logical + 1;
-    int32_t* kept = scratch.data() + 2 * (size_t)b->page_indptr[r];
+    int32_t* kept = scratch.data() + 2 * (n_threads > 1 ? (size_t)b->page_indptr[r] : kept_at);
     int nk = 0;
     if (q.mask_row_words) {
       const int row_words = q.mask_row_words;
@@ -512,13 +610,15 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       if (given) {
         const uint8_t* src = b->mask + b->mask_indptr[r];
         for (int i = 0; i < q.q_len; ++i)
-          if (!pack_row(src + (int64_t)i * q.kv_len, q.kv_len, w + (size_t)i * row_words)) bad_mask.store(1);
+          if (!pack_row(src + (int64_t)i * q.kv_len, q.kv_len, w + (size_t)i * row_words, row_words)) bad_mask.store(1);
       } else {  // inferred causal rows, written out because page masks will be ANDed in
         for (int i = 0; i < q.q_len; ++i) {
           const int nbits = q.kv_len - q.q_len + i + 1;  // positions 0 .. lim
           uint32_t* row = w + (size_t)i * row_words;
-          for (int k = 0; k < nbits / 32; ++k) row[k] = 0xFFFFFFFFu;
-          if (nbits & 31) row[nbits / 32] = (1u << (nbits & 31)) - 1u;
+          int k = 0;
+          for (; k < nbits / 32; ++k) row[k] = 0xFFFFFFFFu;
+          if (nbits & 31) row[k++] = (1u << (nbits & 31)) - 1u;
+          for (; k < row_words; ++k) row[k] = 0u;
         }
       }
       if (ctx->n_masked_pages > 0) {
@@ -530,14 +630,25 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
           for (int i = 0; i < q.q_len; ++i) w[(size_t)i * row_words + (bit >> 5)] &= ~(clear << (bit & 31));
         }
       }
+      // OR and AND of all rows, word by word (contiguous passes over the rows), then one look per page
+      std::vector<uint32_t> col(2 * (size_t)row_words);
+      uint32_t* const any_w = col.data();
+      uint32_t* const all_w = col.data() + row_words;
+      for (int k = 0; k < row_words; ++k) {
+        any_w[k] = 0u;
+        all_w[k] = 0xFFFFFFFFu;
+      }
+      for (int i = 0; i < q.q_len; ++i) {
+        const uint32_t* row = w + (size_t)i * row_words;
+        for (int k = 0; k < row_words; ++k) {
+          any_w[k] |= row[k];
+          all_w[k] &= row[k];
+        }
+      }
       for (int lp = 0; lp < np; ++lp) {
         const int bit = lp * P;
-        uint32_t any = 0, all = full_bits;
-        for (int i = 0; i < q.q_len; ++i) {
-          uint32_t bits = (w[(size_t)i * row_words + (bit >> 5)] >> (bit & 31)) & full_bits;
-          any |= bits;
-          all &= bits;
-        }
+        const uint32_t any = (any_w[bit >> 5] >> (bit & 31)) & full_bits;
+        const uint32_t all = (all_w[bit >> 5] >> (bit & 31)) & full_bits;
         if (!any) continue;  // no query row attends to this page: it is never fetched
         kept[2 * nk] = pages[lp];
         kept[2 * nk + 1] = (int32_t)((uint32_t)lp | (all == full_bits ? 0u : PIE_KEPT_NEEDS_MASK));
@@ -552,11 +663,11 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       nk = np;
     }
     q.kept_count = nk;
+    if (n_threads <= 1) {
+      q.kept_start = (int32_t)kept_at;
+      kept_at += (size_t)nk;
+    }
   };
-  int n_threads = 1;
-  if (mask_bytes_total > (4 << 20)) {
-    n_threads = (int)std::min<int64_t>({(int64_t)std::max(1u, std::thread::hardware_concurrency()), 16, (int64_t)R});
-  }
   if (n_threads <= 1) {
     for (int r = 0; r < R; ++r) do_request(r);
   } else {
@@ -569,7 +680,9 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     for (auto& th : pool) th.join();
   }
   if (bad_mask.load()) return PIE_ERR_MASK;
-  {
+  if (n_threads <= 1) {
+    plan->kept.resize(2 * kept_at);
+  } else {
     size_t total = 0;
     for (int r = 0; r < R; ++r) total += (size_t)plan->reqs[r].kept_count;
     plan->kept.resize(2 * total);
@@ -631,7 +744,11 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     for (int r = 0; r < R;) {
       const PieReq& q0 = plan->reqs[r];
       const int rows = q0.q_len * G;
-      if (rows > 16 || TILE_ROWS % rows != 0 || q0.kept_count < 2) { ++r; continue; }
+      if (rows > 16 || TILE_ROWS % rows != 0 || q0.kept_count < 2 || r + 1 >= R || plan->reqs[r + 1].kept_count < 2 ||
+          plan->kept[2 * (size_t)plan->reqs[r + 1].kept_start] != plan->kept[2 * (size_t)q0.kept_start]) {  // (no neighbour with the same first page: no run starts here)
+        ++r;
+        continue;
+      }
       int L = clean_prefix(q0), e = r + 1;
       for (; e < R && L >= min_L; ++e) {
         const PieReq& q = plan->reqs[e];

@@ -413,3 +413,45 @@ def test_block_local_merge_matches_oracle(sms):
         for n, pg in enumerate(wl.used_pages()):
             Ko, Vo = pool[int(pg)]
             assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {pg}"
+
+
+@pytest.mark.parametrize("name", ["mixed_prefill_decode", "long_context_policy"])
+def test_plan_per_step_loop_with_recycled_plans_matches_oracle(name):
+    """A serving loop plans every step and destroys the plan right after enqueueing its forward:
+    the context hands the same plan objects (pinned image, device arrays) out again.  Forwards run
+    on a non-blocking side stream while the uploads use another one, so only the library's own
+    ordering keeps a reused device image from being overwritten under a running kernel."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs.small(name)
+    O_ref, L_ref, _ = run_oracle(wl)
+    mi, mb = wl.mask_bytes()
+
+    def batch(k):   # the first k requests
+        npg = int(wl.page_indptr[k])
+        args = [wl.qo_indptr[:k + 1], wl.page_indptr[:k + 1], wl.page_indices[:npg], wl.last_page_len[:k]]
+        if mi is not None:
+            args += [mi[:k + 1], mb[:int(mi[k])]]
+        return args
+
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl)
+        q, k_new, v_new = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
+        run, up = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+        sizes = [wl.R, max(1, wl.R // 2), wl.R, 1, max(1, wl.R - 1), wl.R, wl.R, max(1, wl.R // 3)] * 2
+        results = []
+        for k in sizes:
+            T = int(wl.qo_indptr[k])
+            plan = pie.pie_plan_forward(gp.ctx, *batch(k), stream=up.cuda_stream)
+            out = torch.full((T, wl.H_q, wl.D), float("nan"), dtype=q.dtype, device="cuda")
+            lse = torch.full((T, wl.H_q), float("nan"), dtype=torch.float32, device="cuda")
+            run.wait_stream(torch.cuda.current_stream())      # (the fills above)
+            pie.pie_forward(gp.ctx, plan, q[:T], k_new[:T], v_new[:T], out, lse, stream=run.cuda_stream)
+            pie.pie_plan_destroy(plan)                        # no synchronisation in between
+            results.append((T, out, lse))
+        torch.cuda.synchronize()
+        assert pie.pie_get_last_device_status(gp.ctx) == 0
+        for T, out, lse in results:
+            check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref[:T], L_ref[:T], wl.dtype,
+                        wl.qo_indptr[:np.searchsorted(wl.qo_indptr, T) + 1])

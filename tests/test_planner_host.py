@@ -214,3 +214,60 @@ def test_shared_prefix_cascade_planning():
     # the tree workload keeps its requests whole: many rows each, shared pages served from L2
     tree_wl = configs.small("shared_prefix_tree")
     assert plan_info(tree_wl, pie.PIE_PLAN_CASCADE_ALWAYS) == plan_info(tree_wl, pie.PIE_PLAN_NO_CASCADE)
+
+
+@pytest.mark.parametrize("name", ["long_context_policy", "shared_prefix_tree", "mixed_prefill_decode", "batched_decode"])
+def test_recycled_plans_equal_fresh_ones(name):
+    """pie_plan_destroy parks the plan object and pie_plan_forward reuses it: whatever batch the object held
+    before, the image a reused object produces must be byte for byte the one a new context produces."""
+    wl = configs.small(name)
+    mi, mb = wl.mask_bytes()
+
+    def batch(k):   # the first k requests of the workload
+        npg = int(wl.page_indptr[k])
+        args = [wl.qo_indptr[:k + 1], wl.page_indptr[:k + 1], wl.page_indices[:npg], wl.last_page_len[:k]]
+        if mi is not None:
+            args += [mi[:k + 1], mb[:int(mi[k])]]
+        return args
+
+    def new_ctx():
+        ctx = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+        pie.pie_alloc_kvpages(ctx, wl.num_pages)
+        return ctx
+
+    def image(ctx, k):
+        plan = pie.pie_plan_forward(ctx, *batch(k))
+        img, info = pie.pie_plan_debug_read(plan, 3), pie.pie_plan_get_info(plan)
+        pie.pie_plan_destroy(plan)
+        return img, info
+
+    sizes = [wl.R, max(1, wl.R // 2), 1, wl.R, max(1, wl.R - 1)]
+    fresh = []
+    for k in sizes:
+        ctx = new_ctx()
+        try:
+            fresh.append(image(ctx, k))
+        finally:
+            pie.pie_destroy(ctx)
+    ctx = new_ctx()
+    try:
+        # a failed plan in between must leave the parked object usable
+        bad = batch(wl.R)
+        bad[3] = np.asarray(bad[3]).copy()
+        bad[3][0] = wl.P + 1
+        for k, (img0, info0) in zip(sizes, fresh):
+            img, info = image(ctx, k)
+            assert info == info0
+            assert img.shape == img0.shape and np.array_equal(img, img0), f"first {k} requests"
+            with pytest.raises(pie.PieError):
+                pie.pie_plan_forward(ctx, *bad)
+        # several live plans at once, destroyed in another order than they were made
+        plans = [pie.pie_plan_forward(ctx, *batch(k)) for k in sizes]
+        for p, (img0, _) in zip(plans, fresh):
+            assert np.array_equal(pie.pie_plan_debug_read(p, 3), img0)
+        for p in plans[::2] + plans[1::2]:
+            pie.pie_plan_destroy(p)
+        img, _ = image(ctx, sizes[1])
+        assert np.array_equal(img, fresh[1][0])
+    finally:
+        pie.pie_destroy(ctx)
