@@ -24,6 +24,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "pie_internal.h"
 #include "ptx_helpers.cuh"
 
@@ -532,22 +534,35 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
           }
           return true;
         };
+        // Halves that lie inside the item's clean prefix (pages every row of the tile sees in full,
+        // counted by the planner) need neither records nor bits; the look-ahead starts two halves
+        // before the first half that does.
+        const int clean_halves = (int)(item.flags >> PIE_ITEM_CLEAN_SHIFT) / C::PPH;
         uint32_t rec_nxt[C::PPH], bits_nxt[C::PPH], bits[C::PPH];
 #pragma unroll
         for (int g = 0; g < C::PPH; ++g) bits_nxt[g] = 0xFFFFFFFFu;
-        bool mask_nxt;
-        load_recs(0, rec_nxt);
-        mask_nxt = make_bits(rec_nxt, bits_nxt);
-        load_recs(1, rec_nxt);
+        bool mask_nxt = false;
+        if (clean_halves <= 0) {
+          load_recs(0, rec_nxt);
+          mask_nxt = make_bits(rec_nxt, bits_nxt);
+        }
+        if (clean_halves <= 1) load_recs(1, rec_nxt);
 
-        for (int i = 0; i < nhalf; ++i) {
+        // One half of the item.  The body exists twice: a lean copy for the halves of the clean
+        // prefix (no records, no bits, no masking code in the loop) and the general one.
+        auto do_half = [&](const int i, auto masked_tag) {
+          constexpr bool kMasked = decltype(masked_tag)::value;
           const int h = i & 1;
           const uint32_t tSh = tS + h * kHalf;
-          const bool half_mask = mask_nxt;
+          bool half_mask = false;
+          if constexpr (kMasked) {
+            half_mask = mask_nxt;
 #pragma unroll
-          for (int g = 0; g < C::PPH; ++g) bits[g] = bits_nxt[g];
-          mask_nxt = make_bits(rec_nxt, bits_nxt);   // half i + 1 (all "no such page" past the end)
-          load_recs(i + 2, rec_nxt);
+            for (int g = 0; g < C::PPH; ++g) bits[g] = bits_nxt[g];
+            mask_nxt = false;
+            if (i + 1 >= clean_halves) mask_nxt = make_bits(rec_nxt, bits_nxt);   // half i + 1 (all "no such page" past the end)
+            if (i + 2 >= clean_halves) load_recs(i + 2, rec_nxt);
+          }
 
           mbar_wait(smem_u32(s_full + 2 * t + h), (s_ph >> h) & 1, p.status);
           s_ph ^= 1u << h;
@@ -566,7 +581,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
           for (int k = 0; k < kHalf / 32; ++k) {
             float* x = xbuf[k & 1];
             if (k + 1 < kHalf / 32) tmem_ld32(tSh + (k + 1) * 32, reinterpret_cast<uint32_t*>(xbuf[(k + 1) & 1]));
-            if (half_mask) {
+            if (kMasked && half_mask) {
 #pragma unroll
               for (int c = 0; c < 32; ++c)
                 if (!((bits[(k * 32 + c) / P] >> ((k * 32 + c) % P)) & 1u)) x[c] = kNegInf;
@@ -642,7 +657,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
           tc_fence_before();
           mbar_arrive(smem_u32(p_full + 2 * t + h));
           ++n_arr;
-        }
+        };
+        const int n_lean = min(nhalf, max(0, clean_halves - 2));   // (the look-ahead of the general loop starts two halves early)
+        for (int i = 0; i < n_lean; ++i) do_half(i, std::false_type{});
+        for (int i = n_lean; i < nhalf; ++i) do_half(i, std::true_type{});
         mbar_wait(smem_u32(o_done + t), my_items & 1, p.status);
         ++my_items;
         tc_fence_after();

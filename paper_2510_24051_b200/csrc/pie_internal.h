@@ -71,6 +71,9 @@ static_assert(sizeof(PieItem) == 64, "PieItem is one 64-byte line");
 #define PIE_ITEM_LOCAL_PIECE 2u
 #define PIE_ITEM_LOCAL_MERGER 4u
 #define PIE_MAX_LOCAL_GROUPS 8
+// Row-tile items: flags >> PIE_ITEM_CLEAN_SHIFT = number of leading pages of the item that every
+// row of the tile sees in full (no page record and no mask word needs to be looked at for them).
+#define PIE_ITEM_CLEAN_SHIFT 8
 
 // A group of partial slots that the merge kernel combines into final rows.
 struct PieMerge {
@@ -108,6 +111,7 @@ struct pie_plan {
   std::vector<PieReq> reqs;
   std::vector<int32_t> kept;        // pairs (phys, logical|flag)
   std::vector<int32_t> kept_scratch; // planner scratch (per-request slices before packing)
+  std::vector<int32_t> clean_kept;   // [R] kept pages of the request before the first one some row sees only in part
   std::vector<uint32_t> mask_words;
   std::vector<int32_t> append_dst;  // [T] page*P + slot
   std::vector<int32_t> tok_req;     // [T]

@@ -596,13 +596,14 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   std::vector<int32_t>& scratch = n_threads > 1 ? plan->kept_scratch : plan->kept;
   scratch.resize(2 * (size_t)b->page_indptr[R]);
   std::atomic<int> bad_mask{0};
+  plan->clean_kept.resize(R);
   size_t kept_at = 0;   // single-threaded: pages kept so far
   auto do_request = [&](int r) {
     PieReq& q = plan->reqs[r];
     const int32_t* pages = b->page_indices + b->page_indptr[r];
     const int np = q.last_logical + 1;
     int32_t* kept = scratch.data() + 2 * (n_threads > 1 ? (size_t)b->page_indptr[r] : kept_at);
-    int nk = 0;
+    int nk = 0, first_flagged = -1;   // (first kept page some row sees only in part: explicit masks)
     if (q.mask_row_words) {
       const int row_words = q.mask_row_words;
       uint32_t* w = plan->mask_words.data() + q.mask_word_off;
@@ -652,6 +653,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
         if (!any) continue;  // no query row attends to this page: it is never fetched
         kept[2 * nk] = pages[lp];
         kept[2 * nk + 1] = (int32_t)((uint32_t)lp | (all == full_bits ? 0u : PIE_KEPT_NEEDS_MASK));
+        if (all != full_bits && first_flagged < 0) first_flagged = nk;
         ++nk;
       }
     } else {
@@ -663,6 +665,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       nk = np;
     }
     q.kept_count = nk;
+    plan->clean_kept[r] = first_flagged < 0 ? nk : first_flagged;
     if (n_threads <= 1) {
       q.kept_start = (int32_t)kept_at;
       kept_at += (size_t)nk;
@@ -939,6 +942,16 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     for (PieItem& it : ll->items) {
       const PieReq& q = plan->reqs[it.req];
       if (ll == &plan->split && plan->append_fused && it.page_end == q.kept_start + q.kept_count) it.flags |= PIE_ITEM_APPEND;
+      if (ll == &plan->tile) {
+        // leading pages of the item that every row of the tile sees in full: the kernel evaluates no
+        // mask there.  Inferred causal masks: the pages below the first row's limit; explicit masks:
+        // the kept pages before the first one that some row sees only in part.
+        int64_t clean_end;   // in the request's kept list
+        if (q.mask_row_words == 0) clean_end = ((int64_t)q.kv_len - q.q_len + it.row0 / G + 1) / P;
+        else clean_end = it.req < R ? plan->clean_kept[it.req] : q.kept_count;
+        const int64_t clean = std::min<int64_t>(std::max<int64_t>(clean_end - (it.page_begin - q.kept_start), 0), it.page_end - it.page_begin);
+        it.flags = (uint32_t)clean << PIE_ITEM_CLEAN_SHIFT;
+      }
       it.q_start = q.q_start;
       it.q_len = q.q_len;
       it.kv_len = q.kv_len;
