@@ -548,6 +548,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
         }
         if (clean_halves <= 1) load_recs(1, rec_nxt);
 
+        // P = exp2(x * scale - m) for one chunk of 32 columns: bf16 pairs into pk, the sums onto sa / sb.
+        auto exp_chunk = [&](const float* x, const uint64_t scale2, const uint64_t negm2, uint64_t& sa, uint64_t& sb, uint32_t* pk) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 4) {
+            float e0, e1, e2, e3;
+            unpack_f32x2(fma_f32x2(pack_f32x2(x[c], x[c + 1]), scale2, negm2), e0, e1);
+            unpack_f32x2(fma_f32x2(pack_f32x2(x[c + 2], x[c + 3]), scale2, negm2), e2, e3);
+            const float p0 = fast_exp2(e0), p1 = fast_exp2(e1), p2 = fast_exp2(e2), p3 = fast_exp2(e3);
+            sa = add_f32x2(sa, pack_f32x2(p0, p1));
+            sb = add_f32x2(sb, pack_f32x2(p2, p3));
+            pk[c >> 1] = pack_bf16(p0, p1);
+            pk[(c >> 1) + 1] = pack_bf16(p2, p3);
+          }
+        };
         // One half of the item.  The body exists twice: a lean copy for the halves of the clean
         // prefix (no records, no bits, no masking code in the loop) and the general one.
         auto do_half = [&](const int i, auto masked_tag) {
@@ -585,6 +599,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
 #pragma unroll
               for (int c = 0; c < 32; ++c)
                 if (!((bits[(k * 32 + c) / P] >> ((k * 32 + c) % P)) & 1u)) x[c] = kNegInf;
+            }
+            // Lean copy: no maximum is taken while the sums stay small.  The exponentials are computed
+            // against the current reference straight away; the chunk's sum bounds its largest term, so a
+            // sum below 2^16 proves that no score runs ahead of the reference by more than 16 binades
+            // (fp32 sums and bf16 P keep their relative precision at any such lag).  Otherwise - or when a
+            // row of the warp has no reference yet - the chunk is redone the careful way below.
+            if constexpr (!kMasked) {
+              if (__all_sync(0xFFFFFFFFu, m_ref != kNegInf)) {
+                const uint64_t negm2 = pack_f32x2(-m_ref, -m_ref);
+                uint64_t ca = pack_f32x2(0.f, 0.f), cb = pack_f32x2(0.f, 0.f);
+                uint32_t pk[16];
+                exp_chunk(x, scale2, negm2, ca, cb, pk);
+                float s0, s1;
+                unpack_f32x2(add_f32x2(ca, cb), s0, s1);
+                if (!__any_sync(0xFFFFFFFFu, !(s0 + s1 <= 65536.f))) {   // (also catches inf and NaN)
+                  psum_a = add_f32x2(psum_a, ca);
+                  psum_b = add_f32x2(psum_b, cb);
+                  tmem_st16(tSh + k * 16, pk);
+                  if (k + 1 < kHalf / 32) tmem_wait_ld();
+                  continue;
+                }
+              }
             }
             float cm0 = max3(x[0], x[1], x[2]), cm1 = max3(x[3], x[4], x[5]);   // two chains
 #pragma unroll
@@ -634,17 +670,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
             const float neg_m = (m_ref == kNegInf) ? 0.f : -m_ref;
             const uint64_t negm2 = pack_f32x2(neg_m, neg_m);
             uint32_t pk[16];
-#pragma unroll
-            for (int c = 0; c < 32; c += 4) {
-              float e0, e1, e2, e3;
-              unpack_f32x2(fma_f32x2(pack_f32x2(x[c], x[c + 1]), scale2, negm2), e0, e1);
-              unpack_f32x2(fma_f32x2(pack_f32x2(x[c + 2], x[c + 3]), scale2, negm2), e2, e3);
-              const float p0 = fast_exp2(e0), p1 = fast_exp2(e1), p2 = fast_exp2(e2), p3 = fast_exp2(e3);
-              psum_a = add_f32x2(psum_a, pack_f32x2(p0, p1));
-              psum_b = add_f32x2(psum_b, pack_f32x2(p2, p3));
-              pk[c >> 1] = pack_bf16(p0, p1);
-              pk[(c >> 1) + 1] = pack_bf16(p2, p3);
-            }
+            exp_chunk(x, scale2, negm2, psum_a, psum_b, pk);
             tmem_st16(tSh + k * 16, pk);   // columns [16k, 16k+16): below every S column still to be read
             if (k + 1 < kHalf / 32) tmem_wait_ld();
           }

@@ -88,13 +88,15 @@ def build_case(P, H_q, H_kv, D, dtype, order, seed):
     return args, reqs, total
 
 
-def run_gpu(args, total, H_kv, D, dtype, flags=0):
+def run_gpu(args, total, H_kv, D, dtype, flags=0, options=None):
     import paper_2510_24051_b200 as pie
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     P, H_q = args["P"], args["H_q"]
     T = len(args["q"])
     ctx = pie.pie_create(total, P, H_q, H_kv, D, dtype, len(args["last_page_len"]), T, 0)
     try:
+        for opt, value in (options or {}).items():
+            pie.pie_set_option(ctx, opt, value)
         ids = pie.pie_alloc_kvpages(ctx, total)
         K = torch.from_numpy(np.stack([args["pool"][int(p)][0] for p in ids])).to(tdt).cuda()
         V = torch.from_numpy(np.stack([args["pool"][int(p)][1] for p in ids])).to(tdt).cuda()
@@ -102,7 +104,8 @@ def run_gpu(args, total, H_kv, D, dtype, flags=0):
         ptr = np.zeros(len(args["masks"]) + 1, np.int64)
         for r, m in enumerate(args["masks"]):
             ptr[r + 1] = ptr[r] + (0 if m is None else m.size)
-        buf = np.concatenate([m.reshape(-1).astype(np.uint8) for m in args["masks"] if m is not None])
+        given = [m.reshape(-1).astype(np.uint8) for m in args["masks"] if m is not None]
+        buf = np.concatenate(given) if given else np.zeros(0, np.uint8)
         plan = pie.pie_plan_forward(ctx, args["qo_indptr"], args["page_indptr"], args["page_indices"],
                                     args["last_page_len"], ptr, buf, flags)
         q, k, v = (torch.from_numpy(args[n]).to(tdt).cuda() for n in ("q", "k_new", "v_new"))

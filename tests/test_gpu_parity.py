@@ -455,3 +455,43 @@ def test_plan_per_step_loop_with_recycled_plans_matches_oracle(name):
         for T, out, lse in results:
             check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref[:T], L_ref[:T], wl.dtype,
                         wl.qo_indptr[:np.searchsorted(wl.qo_indptr, T) + 1])
+
+
+@pytest.mark.parametrize("D", [128, 64])
+def test_scores_that_keep_outgrowing_the_running_reference(D):
+    """Row tiles whose scores climb a staircase along the context: every step is a jump of ~20
+    binades, far beyond what the lagging softmax reference tolerates, in the middle of pages that
+    need no mask (where the kernel takes no maximum as long as the sums stay small).  Rows with a
+    negative gain see falling scores instead and share warps with the climbing ones."""
+    from oracle import pie_oracle as orc
+    from tests._gpu import TOL_LSE, TOL_O
+    from tests._util import SmallBatch
+    from tests.test_gpu_matrix import _bf16_round, run_gpu
+    rng = np.random.RandomState(7 + D)
+    H_q, H_kv, P = 8, 2, 16
+    seqs = []
+    for q_len, kv_len in [(64, 1400), (40, 900), (1, 300), (33, 33)]:
+        pos = np.arange(kv_len)
+        stairs = (pos // 96) * (14.0 * np.sqrt(D) / D)          # +14 nats of score per step for a gain of 1
+        u = np.ones(D, np.float32)
+        K = stairs[:, None, None] * u[None, None, :] + 0.5 * rng.randn(kv_len, H_kv, D)
+        gain = rng.choice([1.0, 0.7, -0.8, 0.0], size=(q_len, H_q, 1))
+        Q = gain * u[None, None, :] + 0.5 * rng.randn(q_len, H_q, D)
+        seqs.append(dict(Q=_bf16_round(Q.astype(np.float32)), K=_bf16_round(K.astype(np.float32)),
+                         V=_bf16_round(rng.randn(kv_len, H_kv, D).astype(np.float32))))
+    args = SmallBatch(seqs, H_q).paged(P, "random", seed=3)
+    total = len(args["pool"])
+    O_ref, L_ref = orc.forward(**{k: (v if k != "pool" else {p: (a.copy(), b.copy()) for p, (a, b) in v.items()})
+                                  for k, v in args.items()})
+    args["masks"] = [None] * len(seqs)
+    import paper_2510_24051_b200 as pie
+    # (two thread blocks for the row tiles: the items stay long, ten and more steps of the staircase each)
+    for flags, options in ((0, {pie.PIE_OPT_TILE_SMS: 2}), (0, None), (2, None)):
+        O, L, info = run_gpu(args, total, H_kv, D, "bf16", flags, options)
+        if flags == 0:
+            assert info["num_tile_items"] > 0
+        if options:
+            assert info["num_tile_items"] <= 8
+        assert np.isfinite(O).all()
+        assert np.abs(O - O_ref).max() <= TOL_O["bf16"]
+        assert np.abs(L - L_ref).max() <= TOL_LSE
