@@ -198,7 +198,11 @@ int pie_plan_get_info(const pie_plan* plan, pie_plan_info* out);
  * logical page | 0x80000000 if the page needs mask evaluation), 2 = append destinations
  * (int32 per query token: page * page_size + slot), 3 = the plan's whole upload image (request
  * records, kept pages, masks, append destinations, work items, share boundaries, merge groups
- * and counters in device layout, gaps zeroed; size a multiple of 4).  *out_bytes receives the
+ * and counters in device layout, gaps zeroed; size a multiple of 4), 4 / 5 = the work items of
+ * the split-KV / row-tile launch (16 int32 each: request, kv head, first row, rows, first and
+ * end kept page, partial slot or -1, six fields of the request record, flags - for row-tile
+ * items flags >> 8 = leading pages every row of the tile sees in full -, mask word offset as two
+ * words).  *out_bytes receives the
  * array size; data is copied only if cap_bytes is large enough. */
 int pie_plan_debug_read(const pie_plan* plan, int which, void* buf, int64_t cap_bytes,
                         int64_t* out_bytes);

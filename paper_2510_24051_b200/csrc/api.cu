@@ -637,6 +637,8 @@ int pie_plan_debug_read(const pie_plan* plan, int which, void* buf, int64_t cap_
     case 0: p = plan->mask_words.data(); n = (int64_t)plan->mask_words.size() * 4; break;
     case 1: p = plan->kept.data(); n = (int64_t)plan->kept.size() * 4; break;
     case 2: p = plan->append_dst.data(); n = (int64_t)plan->append_dst.size() * 4; break;
+    case 4: p = plan->split.items.data(); n = (int64_t)plan->split.items.size() * (int64_t)sizeof(PieItem); break;
+    case 5: p = plan->tile.items.data(); n = (int64_t)plan->tile.items.size() * (int64_t)sizeof(PieItem); break;
     default: return PIE_ERR_INVALID;
   }
   *out_bytes = n;

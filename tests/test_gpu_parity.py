@@ -495,3 +495,40 @@ def test_scores_that_keep_outgrowing_the_running_reference(D):
         assert np.isfinite(O).all()
         assert np.abs(O - O_ref).max() <= TOL_O["bf16"]
         assert np.abs(L - L_ref).max() <= TOL_LSE
+
+
+def test_prefill_under_a_kv_policy_with_a_long_clean_prefix():
+    """Prefill chunks under application masks that drop whole pages (kept and logical page indices differ),
+    with the first partly hidden page far into the context: the kernel runs the pages before it without
+    looking at any mask, and must pick the masks up exactly where the planner says."""
+    from oracle import pie_oracle as orc
+    from tests._gpu import TOL_LSE, TOL_O
+    from tests._util import SmallBatch, random_seqs
+    from tests.test_gpu_matrix import _bf16_round, run_gpu
+    import paper_2510_24051_b200 as pie
+    rng = np.random.RandomState(23)
+    P, H_q, H_kv, D = 16, 8, 2, 128
+    shapes = [(48, 48 + 61 * P + 3), (33, 33 + 40 * P), (64, 64 + 52 * P + 9)]
+    masks = []
+    for n, (q_len, kv_len) in enumerate(shapes):
+        pos = kv_len - q_len + np.arange(q_len)
+        m = np.arange(kv_len)[None, :] <= pos[:, None]
+        for pg in rng.choice(24, size=4, replace=False):              # dropped for every row
+            m[:, pg * P:(pg + 1) * P] = False
+        m[rng.randint(q_len), (30 + 3 * n) * P + 5] = False           # first slot that only some rows see
+        m[:, (34 + n) * P:(35 + n) * P] &= rng.rand(q_len, P) < 0.7   # and a page hidden at random
+        masks.append(m)
+    seqs = random_seqs(rng, shapes, H_q, H_kv, D, masks=masks)
+    for s in seqs:
+        for k in ("Q", "K", "V"):
+            s[k] = _bf16_round(s[k])
+    args = SmallBatch(seqs, H_q).paged(P, "random", seed=5)
+    total = len(args["pool"])
+    O_ref, L_ref = orc.forward(**{k: (v if k != "pool" else {p: (a.copy(), b.copy()) for p, (a, b) in v.items()})
+                                  for k, v in args.items()})
+    for options in ({pie.PIE_OPT_TILE_SMS: 3}, None):
+        O, L, info = run_gpu(args, total, H_kv, D, "bf16", 0, options)
+        assert info["num_tile_items"] > 0 and info["kept_pages"] < sum((kv + P - 1) // P for _, kv in shapes)
+        assert np.isfinite(O).all()
+        assert np.abs(O - O_ref).max() <= TOL_O["bf16"]
+        assert np.abs(L - L_ref).max() <= TOL_LSE

@@ -271,3 +271,97 @@ def test_recycled_plans_equal_fresh_ones(name):
         assert np.array_equal(img, fresh[1][0])
     finally:
         pie.pie_destroy(ctx)
+
+
+def _check_clean_prefix(P, H_q, H_kv, D, qo_indptr, page_indptr, page_indices, last_page_len, masks, num_pages):
+    R, T = len(last_page_len), int(qo_indptr[-1])
+    ctx = pie.pie_create(num_pages, P, H_q, H_kv, D, "bf16", R, T, device=-1)
+    try:
+        pie.pie_alloc_kvpages(ctx, num_pages)
+        mi = mb = None
+        if masks is not None and any(m is not None for m in masks):
+            mi = np.zeros(R + 1, np.int64)
+            for r, m in enumerate(masks):
+                mi[r + 1] = mi[r] + (0 if m is None else np.asarray(m).size)
+            mb = np.concatenate([np.asarray(m).reshape(-1).astype(np.uint8) for m in masks if m is not None])
+        plan = pie.pie_plan_forward(ctx, qo_indptr, page_indptr, page_indices, last_page_len, mi, mb)
+        items = pie.pie_plan_debug_read(plan, 5).reshape(-1, 16)
+        kept = pie.pie_plan_debug_read(plan, 1).reshape(-1, 2)
+        info = pie.pie_plan_get_info(plan)
+        pie.pie_plan_destroy(plan)
+    finally:
+        pie.pie_destroy(ctx)
+    assert len(items) == info["num_tile_items"] > 0
+    G = H_q // H_kv
+    ql = np.diff(qo_indptr)
+    kv = (np.diff(page_indptr) - 1) * P + np.asarray(last_page_len)
+    n_clean_items = 0
+    for it in items:
+        r, row0, nrows, pb, pe = int(it[0]), int(it[2]), int(it[3]), int(it[4]), int(it[5])
+        clean = int(np.uint32(it[13])) >> 8
+        assert 0 <= clean <= pe - pb
+        if r >= R:
+            continue                                    # (virtual request of a shared-prefix cascade: all visible)
+        toks = np.arange(row0 // G, (row0 + nrows - 1) // G + 1)
+        m = None if masks is None or masks[r] is None else np.asarray(masks[r]).astype(bool)
+
+        def full(page_logical, rows):                   # every slot of the page allowed for every given row
+            j = page_logical * P + np.arange(P)
+            if (j >= kv[r]).any():
+                return False
+            if m is None:
+                return bool((j[None, :] <= (kv[r] - ql[r] + rows)[:, None]).all())
+            return bool(m[rows][:, j].all())
+
+        logical = kept[pb:pe, 1] & 0x7FFFFFFF
+        n_tile = 0
+        while n_tile < pe - pb and full(int(logical[n_tile]), toks):
+            n_tile += 1
+        assert clean <= n_tile, (r, row0, clean, n_tile)  # never a page with a hidden slot
+        if m is None:
+            assert clean == n_tile                      # causal: exactly the pages below the first row's limit
+        else:
+            n_req = 0
+            while n_req < pe - pb and full(int(logical[n_req]), np.arange(ql[r])):
+                n_req += 1
+            # the planner counts from the start of the request's kept list, so an item that begins behind the
+            # first partly hidden page reports none
+            assert clean in (n_req, 0)
+        n_clean_items += clean > 0
+    return n_clean_items
+
+
+@pytest.mark.parametrize("name", ["mixed_prefill_decode", "shared_prefix_tree"])
+def test_clean_page_prefix_of_row_tile_items(name):
+    """Row-tile items carry the number of leading pages that every row of the tile sees in full; the
+    kernel evaluates no mask there, so the count must never include a page with a hidden slot.  Checked
+    against the mask definition: exact for inferred causal masks, and equal to the request-wide count
+    (clipped to the item) for explicit ones."""
+    wl = configs.small(name)
+    assert _check_clean_prefix(wl.P, wl.H_q, wl.H_kv, wl.D, wl.qo_indptr, wl.page_indptr, wl.page_indices,
+                               wl.last_page_len, wl.masks, wl.num_pages) > 0
+
+
+def test_clean_page_prefix_with_dropped_and_partly_hidden_pages():
+    """Explicit masks of an application KV policy on prefill chunks: whole pages dropped (they leave the kept
+    list, so kept and logical indices differ), then a page one row sees only in part, then more visible pages."""
+    rng = np.random.RandomState(11)
+    P, H_q, H_kv, D = 16, 8, 2, 64
+    shapes = [(24, 24 + 37 * P), (40, 40 + 20 * P + 5), (17, 17 + 9 * P)]
+    masks, qo, pi, idx, last = [], [0], [0], [], []
+    for n, (q_len, kv_len) in enumerate(shapes):
+        pos = kv_len - q_len + np.arange(q_len)
+        m = np.arange(kv_len)[None, :] <= pos[:, None]
+        npg = (kv_len + P - 1) // P
+        for pg in rng.choice(npg - 4, size=3, replace=False):      # dropped for every row
+            m[:, pg * P:(pg + 1) * P] = False
+        if n < 2:
+            m[rng.randint(q_len), (5 + n) * P + 3] = False          # one slot hidden from one row
+        masks.append(m)
+        qo.append(qo[-1] + q_len)
+        pi.append(pi[-1] + npg)
+        idx.extend(range(pi[-2], pi[-1]))
+        last.append(kv_len - (npg - 1) * P)
+    masks[2] = None                                                  # and one inferred causal request
+    assert _check_clean_prefix(P, H_q, H_kv, D, np.array(qo), np.array(pi), np.array(idx), np.array(last), masks,
+                               pi[-1] + 2) > 0
