@@ -10,28 +10,48 @@
 // ------------------------------------------------------------------------------------ kernels
 namespace {
 
-// K1: append (Table 1 `forward`, output KvPages).  One thread moves one 16-byte chunk of one
-// new K or V row into the swizzled pool block of its destination (page, slot).
+// K1: append (Table 1 `forward`, output KvPages).  One thread moves one 16-byte chunk of one new K
+// or V row into the swizzled pool block of its destination (page, slot).  A thread keeps its place
+// inside a token (K or V, head, chunk: found once, with shifts - chunks per row and page size are
+// powers of two) and walks over tokens, four at a time so that four loads are in flight before
+// the first store.  tok_shift > 0: a token has fewer chunks than the block has threads and every
+// block covers 2^tok_shift tokens per step.
+constexpr int kAppendUnroll = 4;
 __global__ void append_kernel(uint8_t* __restrict__ pool, const uint8_t* __restrict__ k_new,
                               const uint8_t* __restrict__ v_new, const int32_t* __restrict__ append_dst,
-                              int T, PoolGeom g) {
+                              int T, PoolGeom g, int chunk_shift, int page_shift, int tok_shift) {
   pie_pdl_launch_dependents();
   pie_pdl_wait();
-  const int chunks = g.row_bytes >> 4;
-  const int64_t per_tok = (int64_t)2 * g.n_kv_heads * chunks;
-  const int64_t total = (int64_t)T * per_tok;
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    int t = (int)(i / per_tok);
-    int rem = (int)(i - (int64_t)t * per_tok);
-    int kv = rem / (g.n_kv_heads * chunks);
-    rem -= kv * g.n_kv_heads * chunks;
-    int head = rem / chunks, c = rem - head * chunks;
-    const uint8_t* src = (kv ? v_new : k_new) + ((int64_t)t * g.n_kv_heads + head) * g.row_bytes + c * 16;
-    int dst = append_dst[t];
-    int page = dst / g.page_size, slot = dst - page * g.page_size;
-    uint8_t* d = pool + (int64_t)page * g.page_bytes + (int64_t)(head * 2 + kv) * g.block_bytes +
-                 pie_chunk_offset(g.slab_bytes, slot, c);
-    *reinterpret_cast<uint4*>(d) = *reinterpret_cast<const uint4*>(src);
+  const int per_tok = (2 * g.n_kv_heads) << chunk_shift;     // chunks per token
+  const int lanes = blockDim.x >> tok_shift;                 // threads that work on one token
+  const int tl = threadIdx.x / lanes;                        // token of this thread inside the block's group
+  const int j0 = threadIdx.x - tl * lanes;
+  const int n_groups = (T + (1 << tok_shift) - 1) >> tok_shift;
+  for (int j = j0; j < per_tok; j += lanes) {                // (one pass unless a token has more chunks than the block has threads)
+    const int c = j & ((1 << chunk_shift) - 1), hk = j >> chunk_shift;
+    const int kv = hk >= g.n_kv_heads ? 1 : 0, head = hk - kv * g.n_kv_heads;
+    const uint8_t* src0 = (kv ? v_new : k_new) + (int64_t)head * g.row_bytes + c * 16;
+    const int64_t tok_stride = (int64_t)g.n_kv_heads * g.row_bytes;
+    uint8_t* dst0 = pool + (int64_t)(head * 2 + kv) * g.block_bytes;
+    for (int grp = blockIdx.x; grp < n_groups; grp += kAppendUnroll * gridDim.x) {
+      uint4 v[kAppendUnroll];
+      int dst[kAppendUnroll];
+#pragma unroll
+      for (int u = 0; u < kAppendUnroll; ++u) {
+        const int t = ((grp + u * (int)gridDim.x) << tok_shift) + tl;
+        dst[u] = -1;
+        if (grp + u * (int)gridDim.x < n_groups && t < T) {
+          dst[u] = append_dst[t];
+          v[u] = *reinterpret_cast<const uint4*>(src0 + t * tok_stride);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kAppendUnroll; ++u) {
+        if (dst[u] < 0) continue;
+        const int page = dst[u] >> page_shift, slot = dst[u] & ((1 << page_shift) - 1);
+        *reinterpret_cast<uint4*>(dst0 + (int64_t)page * g.page_bytes + pie_chunk_offset(g.slab_bytes, slot, c)) = v[u];
+      }
+    }
   }
 }
 
@@ -208,9 +228,19 @@ void pie_plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base) {
 int pie_launch_append(pie_ctx* ctx, const pie_plan* plan, const void* k_new, const void* v_new, cudaStream_t s) {
   if (plan->T == 0) return PIE_OK;
   const PoolGeom& g = ctx->geom;
-  int64_t work = (int64_t)plan->T * 2 * g.n_kv_heads * (g.row_bytes >> 4);
-  PIE_CUDA(ctx, pie_launch_pdl(append_kernel, dim3(grid_for(work, 256, ctx->n_sms)), dim3(256), 0, s, ctx->pool,
-                               (const uint8_t*)k_new, (const uint8_t*)v_new, (const int32_t*)plan->d_append_dst, plan->T, g));
+  auto log2i = [](int x) {
+    int l = 0;
+    while ((1 << l) < x) ++l;
+    return l;
+  };
+  const int chunk_shift = log2i(g.row_bytes >> 4), page_shift = log2i(g.page_size);   // (both powers of two: D 64 / 128, page size 8 / 16 / 32)
+  const int per_tok = (2 * g.n_kv_heads) << chunk_shift;
+  int tok_shift = 0;   // tokens per block and step: as many as fit into 256 threads, a power of two
+  while ((per_tok << (tok_shift + 1)) <= 256) ++tok_shift;
+  const int n_groups = (plan->T + (1 << tok_shift) - 1) >> tok_shift;
+  const int grid = std::max(1, std::min((n_groups + kAppendUnroll - 1) / kAppendUnroll, ctx->n_sms * 8));
+  PIE_CUDA(ctx, pie_launch_pdl(append_kernel, dim3(grid), dim3(256), 0, s, ctx->pool, (const uint8_t*)k_new, (const uint8_t*)v_new,
+                               (const int32_t*)plan->d_append_dst, plan->T, g, chunk_shift, page_shift, tok_shift));
   return PIE_OK;
 }
 
