@@ -210,13 +210,19 @@ def apply_page_masks(allowed: np.ndarray, pages, P: int, page_masks) -> np.ndarr
 
 def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
             q, k_new, v_new, masks=None, append=True, requests=None, page_masks=None,
-            rope_theta=None, positions=None):
+            rope_theta=None, positions=None, out_lens=None):
     """One batched `forward`: append, then gather and attend for every request.
 
     q [T, H_q, D], k_new/v_new [T, H_kv, D] in the storage type; masks is None or a list
     with, per request, None (inferred causal) or a bool [q_len, kv_len] matrix.
     `requests` restricts step 3 to some request ids (rows of the others stay 0 / -inf); the
     append is always done for the whole batch.  Returns O [T, H_q, D] fp64, LSE [T, H_q].
+
+    out_lens (Section 4.2 "Forward API": a call populates output Embeds and/or output KvPages;
+    its listing stores 8 tokens with no output and produces 1 output from 9 inputs): request r
+    produces outputs for its LAST out_lens[r] query tokens only - 0 = the rows are stored and
+    nothing else.  Rows that produce no output come back as NaN (O and LSE); every row is
+    appended and keeps its own position and mask row.
     """
     R = len(qo_indptr) - 1
     T = int(qo_indptr[R])
@@ -239,8 +245,13 @@ def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
         kv_len = kv_len_of(len(pages), int(last_page_len[r]), P)
         allowed = allowed_matrix(t1 - t0, kv_len, None if masks is None else masks[r])
         allowed = apply_page_masks(allowed, pages, P, page_masks)
+        first = 0 if out_lens is None else (t1 - t0) - int(out_lens[r])   # first query token that produces an output
+        O[t0:t0 + first], LSE[t0:t0 + first] = np.nan, np.nan
+        if first == t1 - t0:
+            continue
+        allowed = allowed[first:]
         K, V = gather_kv(pool, P, pages, kv_len, needed=allowed.any(axis=0))
-        O[t0:t1], LSE[t0:t1] = attend(q64[t0:t1], K, V, allowed)
+        O[t0 + first:t1], LSE[t0 + first:t1] = attend(q64[t0 + first:t1], K, V, allowed)
     return O, LSE
 
 

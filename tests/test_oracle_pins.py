@@ -464,3 +464,48 @@ def test_default_positions_are_the_last_q_len_context_positions():
     # request 1: 3 pages, last holds 8 -> kv_len 24, 4 new tokens -> positions 20..23
     pos = orc.default_positions(np.array([0, 1, 5]), np.array([0, 2, 5]), np.array([3, 8]), 8)
     assert pos.tolist() == [10, 20, 21, 22, 23]
+
+
+def test_out_lens_follow_the_papers_listing_and_the_textbook():
+    """Section 4.2 listing: `forward([], iemb, [], oemb)` gives ONE output from nine inputs, and the
+    same result comes from `forward([], iemb[:-1], kv)` (rows stored, no output) followed by
+    `forward(kv, iemb[-1:], oemb)`.  Rows with an output equal scalar-loop textbook attention of that
+    row; rows without come back as NaN; the stored rows do not depend on how many outputs were asked for."""
+    rng = np.random.RandomState(31)
+    P, H_q, H_kv, D = 8, 4, 2, 8
+    shapes = [(9, 9), (5, 21), (3, 17), (1, 12)]
+    out_lens = [1, 0, 2, 1]
+    m = rng.rand(3, 17) < 0.6
+    m[:, 0] = True
+    seqs = random_seqs(rng, shapes, H_q, H_kv, D, masks=[None, None, m, None])
+    args = SmallBatch(seqs, H_q).paged(P, "random", seed=2)
+    pool_a = {p: (a.copy(), b.copy()) for p, (a, b) in args["pool"].items()}
+    pool_b = {p: (a.copy(), b.copy()) for p, (a, b) in args["pool"].items()}
+    O_all, L_all = orc.forward(**dict(args, pool=pool_a))
+    O, L = orc.forward(**dict(args, pool=pool_b), out_lens=out_lens)
+    for p in pool_a:                                   # every row is stored either way
+        assert np.array_equal(pool_a[p][0], pool_b[p][0], equal_nan=True)
+        assert np.array_equal(pool_a[p][1], pool_b[p][1], equal_nan=True)
+    t = 0
+    for s, (q_len, kv_len), ol in zip(seqs, shapes, out_lens):
+        first = q_len - ol
+        assert np.isnan(O[t:t + first]).all() and np.isnan(L[t:t + first]).all()
+        allowed = s["mask"] if "mask" in s else np.array(causal(q_len, kv_len))
+        Or, Lr = textbook_attention(s["Q"][first:], s["K"], s["V"], np.asarray(allowed)[first:])
+        np.testing.assert_allclose(O[t + first:t + q_len], Or, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(L[t + first:t + q_len], Lr, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(O[t + first:t + q_len], O_all[t + first:t + q_len], rtol=0, atol=1e-13)
+        t += q_len
+
+    # the listing itself: 8 tokens stored with no output, then one token that reads them
+    s0 = seqs[0]
+    npg = 2
+    pool = {p: (np.full((P, H_kv, D), np.nan, np.float32), np.full((P, H_kv, D), np.nan, np.float32)) for p in range(3)}
+    pages = np.array([2, 0])
+    Oa, La = orc.forward(pool, P, H_q, np.array([0, 8]), np.array([0, 1]), pages[:1], np.array([8]),
+                         s0["Q"][:8], s0["K"][:8], s0["V"][:8], out_lens=[0])
+    assert np.isnan(Oa).all() and np.isnan(La).all()
+    Ob, Lb = orc.forward(pool, P, H_q, np.array([0, 1]), np.array([0, npg]), pages, np.array([1]),
+                         s0["Q"][8:], s0["K"][8:], s0["V"][8:])
+    np.testing.assert_allclose(Ob[0], O[8], atol=1e-14)
+    np.testing.assert_allclose(Lb[0], L[8], atol=1e-14)
