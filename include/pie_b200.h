@@ -149,6 +149,13 @@ typedef struct pie_batch_desc {
   const int32_t* positions;     /* [T] explicit position of every new token, or NULL for the
                                    default kv_len - q_len + i.  Used only when the context
                                    was created with rope_theta > 0.                 */
+  const int32_t* out_len;       /* [R] or NULL.  Section 4.2: a forward call fills output Embeds
+                                   and / or output KvPages.  Request r produces outputs (out, lse)
+                                   for its LAST out_len[r] query tokens only, 0 <= out_len[r] <=
+                                   q_len; 0 = its rows are stored and nothing is attended.  All
+                                   q_len rows are appended and keep their positions and mask rows;
+                                   out / lse rows of tokens without output are left untouched.
+                                   NULL = every token produces an output.             */
 } pie_batch_desc;
 
 enum {

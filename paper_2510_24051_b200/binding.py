@@ -30,7 +30,7 @@ class pie_config(C.Structure):
 class pie_batch_desc(C.Structure):
     _fields_ = [("num_requests", C.c_int32), ("qo_indptr", C.c_void_p), ("page_indptr", C.c_void_p),
                 ("page_indices", C.c_void_p), ("last_page_len", C.c_void_p), ("mask_indptr", C.c_void_p),
-                ("mask", C.c_void_p), ("flags", C.c_uint32), ("positions", C.c_void_p)]
+                ("mask", C.c_void_p), ("flags", C.c_uint32), ("positions", C.c_void_p), ("out_len", C.c_void_p)]
 
 
 class pie_plan_info(C.Structure):
@@ -181,20 +181,21 @@ def pie_copy_kvpage(ctx, src, dst, src_off, dst_off, ntok, stream=None):
     _check(lib.pie_copy_kvpage(ctx, len(a[0]), *[x.ctypes.data for x in a], _stream(stream)), ctx)
 
 
-def _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions=None):
+def _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions=None, out_len=None):
     keep = [_i32(qo_indptr), _i32(page_indptr), _i32(page_indices), _i32(last_page_len)]
     mi = None if mask_indptr is None else np.ascontiguousarray(mask_indptr, dtype=np.int64)
     mk = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
     ps = None if positions is None else _i32(positions)
-    keep += [mi, mk, ps]
+    ol = None if out_len is None else _i32(out_len)
+    keep += [mi, mk, ps, ol]
     d = pie_batch_desc(len(keep[0]) - 1, keep[0].ctypes.data, keep[1].ctypes.data, keep[2].ctypes.data,
-                       keep[3].ctypes.data, _ptr(mi), _ptr(mk), flags, _ptr(ps))
+                       keep[3].ctypes.data, _ptr(mi), _ptr(mk), flags, _ptr(ps), _ptr(ol))
     return d, keep
 
 
 def pie_plan_forward(ctx, qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr=None,
-                     mask=None, flags=0, stream=None, positions=None):
-    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions)
+                     mask=None, flags=0, stream=None, positions=None, out_len=None):
+    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions, out_len)
     plan = C.c_void_p()
     _check(lib.pie_plan_forward(ctx, C.byref(d), _stream(stream), C.byref(plan)), ctx)
     return plan
@@ -224,8 +225,8 @@ def pie_forward(ctx, plan, q, k_new, v_new, out, lse, stream=None):
 
 
 def pie_forward_host(ctx, qo_indptr, page_indptr, page_indices, last_page_len, q, k_new, v_new, out,
-                     lse, mask_indptr=None, mask=None, flags=0, stream=None):
-    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags)
+                     lse, mask_indptr=None, mask=None, flags=0, stream=None, out_len=None):
+    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, None, out_len)
     _check(lib.pie_forward_host(ctx, C.byref(d), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse),
                                 _stream(stream)), ctx)
 
@@ -259,11 +260,11 @@ PIE_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
 def pie_forward_static_scratch(ctx, qo_indptr, page_indptr, page_indices, last_page_len, q, k_new, v_new,
-                               out, lse, mask_indptr=None, mask=None, flags=0, stream=None):
+                               out, lse, mask_indptr=None, mask=None, flags=0, stream=None, out_len=None):
     """forward for callers that cannot allocate device memory: plan arrays and split partials go
     to the library's fixed device array (at most PIE_STATIC_SCRATCH_BYTES, else
     PIE_ERR_BATCH_TOO_LARGE).  Tensors are device tensors; calls must not overlap on the GPU."""
-    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags)
+    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, None, out_len)
     _check(lib.pie_forward_static_scratch(ctx, C.byref(d), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
                                           _ptr(lse), _stream(stream)), ctx)
 

@@ -481,6 +481,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     const int64_t kv_len64 = (int64_t)(np - 1) * P + last;
     if (kv_len64 > 0x3FFFFFFF) return PIE_ERR_INVALID;
     if (kv_len64 < q_len) return PIE_ERR_INVALID;
+    if (b->out_len && (b->out_len[r] < 0 || b->out_len[r] > q_len)) return PIE_ERR_INVALID;
     const int32_t* pages = b->page_indices + b->page_indptr[r];
     uint32_t max_id = 0;   // (negative ids wrap to large values)
     for (int k = 0; k < np; ++k) max_id = std::max(max_id, (uint32_t)pages[k]);
@@ -718,6 +719,24 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     }
   }
 
+  // ---- output Embeds for the last out_len tokens only (Section 4.2: a call fills output Embeds and / or
+  // output KvPages): from here on a request is its attention view - the query tokens that produce an
+  // output.  They keep their positions and mask rows (kv_len is unchanged, so the inferred causal limit
+  // kv_len - q_len + i of view token i is the one of the original token); a request with out_len 0 is
+  // stored and not attended at all.
+  bool all_rows_out = true;
+  if (b->out_len) {
+    for (int r = 0; r < R; ++r) {
+      PieReq& q = plan->reqs[r];
+      const int skip = q.q_len - b->out_len[r];
+      if (skip == 0) continue;
+      all_rows_out = false;
+      q.q_start += skip;
+      q.mask_word_off += (int64_t)skip * q.mask_row_words;
+      q.q_len = b->out_len[r];
+    }
+  }
+
   // ---- route requests to kernels and partition the work
   const bool tiles_ok = pie_split_supported(ctx) && !(b->flags & PIE_PLAN_FORCE_SIMPLE);
   std::vector<Unit> split_units, tile_units;
@@ -735,7 +754,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   struct Cascade { int32_t first, n, L, vreq; };
   std::vector<Cascade> cascades;
   std::vector<int32_t> casc_of(R, -1);
-  if (tiles_ok && !(b->flags & PIE_PLAN_NO_CASCADE)) {
+  if (tiles_ok && !(b->flags & PIE_PLAN_NO_CASCADE) && all_rows_out) {   // (the gathered rows of a group must be consecutive query tokens)
     const bool always = (b->flags & PIE_PLAN_CASCADE_ALWAYS) != 0;
     const int min_n = always ? 2 : 4, min_L = always ? 1 : 16;
     auto clean_prefix = [&](const PieReq& q) {  // leading kept pages that are fully visible and in place
@@ -747,7 +766,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
     for (int r = 0; r < R;) {
       const PieReq& q0 = plan->reqs[r];
       const int rows = q0.q_len * G;
-      if (rows > 16 || TILE_ROWS % rows != 0 || q0.kept_count < 2 || r + 1 >= R || plan->reqs[r + 1].kept_count < 2 ||
+      if (rows == 0 || rows > 16 || TILE_ROWS % rows != 0 || q0.kept_count < 2 || r + 1 >= R || plan->reqs[r + 1].kept_count < 2 ||
           plan->kept[2 * (size_t)plan->reqs[r + 1].kept_start] != plan->kept[2 * (size_t)q0.kept_start]) {  // (no neighbour with the same first page: no run starts here)
         ++r;
         continue;
@@ -794,6 +813,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   for (int r = 0; r < R; ++r) {
     const PieReq& q = plan->reqs[r];
     const int rows = q.q_len * G;
+    if (rows == 0) continue;               // (stored only: no output row)
     if (!tiles_ok || q.kept_count == 0) {  // (a request with no attendable page only needs zeros / -inf written)
       for (int i = 0; i < q.q_len; ++i)
         for (int h = 0; h < cfg.num_q_heads; ++h) plan->simple_rows.push_back((q.q_start + i) * cfg.num_q_heads + h);
@@ -928,7 +948,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   // and into its staged copy), and the append launch is dropped.
   const int no_fusion = ctx->options[PIE_OPT_NO_FUSION];
   plan->append_fused = false;
-  if (!(no_fusion & 1) && ctx->cfg.rope_theta <= 0.f && !cross_read && !plan->split.items.empty() &&
+  if (!(no_fusion & 1) && all_rows_out && ctx->cfg.rope_theta <= 0.f && !cross_read && !plan->split.items.empty() &&
       plan->tile.items.empty() && plan->simple_rows.empty()) {
     bool ok = true;
     for (int r = 0; r < R && ok; ++r) {

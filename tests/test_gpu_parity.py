@@ -532,3 +532,42 @@ def test_prefill_under_a_kv_policy_with_a_long_clean_prefix():
         assert np.isfinite(O).all()
         assert np.abs(O - O_ref).max() <= TOL_O["bf16"]
         assert np.abs(L - L_ref).max() <= TOL_LSE
+
+
+@pytest.mark.parametrize("name", ["mixed_prefill_decode", "shared_prefix_tree", "tiny_fp32"])
+@pytest.mark.parametrize("flags", [0, 1, 2])
+def test_outputs_for_the_last_tokens_only(name, flags):
+    """Section 4.2: a forward call fills output Embeds and / or output KvPages.  Requests ask for outputs of
+    their last out_len tokens only (0 = store the rows, attend nothing): those rows match the oracle, all
+    other rows of out / lse keep what the caller put there, and every row is appended bit for bit."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs.small(name)
+    rng = np.random.RandomState(3)
+    ql = wl.q_lens()
+    out_len = np.array([[0, 1, q, max(1, q // 3), q][rng.randint(5)] for q in ql], dtype=np.int32)
+    out_len[0], out_len[-1] = 0, min(1, ql[-1])
+    pool_ref = wl.oracle_pool(True)
+    O_ref, L_ref = orc_forward_with_out_lens(wl, pool_ref, out_len)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl, poison=True)
+        mi, mb = wl.mask_bytes()
+        plan = pie.pie_plan_forward(gp.ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len, mi, mb,
+                                    flags, out_len=out_len)
+        out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))   # (prefilled with NaN)
+        pie.pie_plan_destroy(plan)
+        O, L = out.double().cpu().numpy(), lse.double().cpu().numpy()
+        produced = ~np.isnan(L_ref[:, 0])
+        assert produced.any() and (~produced).any()
+        assert np.isnan(O[~produced]).all() and np.isnan(L[~produced]).all()          # untouched
+        check_close(O[produced], L[produced], O_ref[produced], L_ref[produced], wl.dtype)
+        used = wl.used_pages()
+        Kg, Vg = gp.read_pages(used)
+        for n, pg in enumerate(used):
+            assert same_bits(Kg[n], pool_ref[int(pg)][0]) and same_bits(Vg[n], pool_ref[int(pg)][1])
+
+
+def orc_forward_with_out_lens(wl, pool, out_len):
+    from oracle import pie_oracle as orc
+    return orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                       bits(wl.q()), bits(wl.k_new()), bits(wl.v_new()), wl.masks, out_lens=out_len)

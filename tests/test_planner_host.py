@@ -365,3 +365,45 @@ def test_clean_page_prefix_with_dropped_and_partly_hidden_pages():
     masks[2] = None                                                  # and one inferred causal request
     assert _check_clean_prefix(P, H_q, H_kv, D, np.array(qo), np.array(pi), np.array(idx), np.array(last), masks,
                                pi[-1] + 2) > 0
+
+
+def test_out_len_validation_and_work_lists():
+    """Per-request output length (Section 4.2: output Embeds and / or output KvPages): bounds are checked,
+    requests without output create no attention work, append destinations do not depend on it."""
+    wl = configs.small("mixed_prefill_decode")
+    ql = wl.q_lens()
+    ctx = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+    try:
+        pie.pie_alloc_kvpages(ctx, wl.num_pages)
+        base = (wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len)
+
+        def plan(out_len):
+            p = pie.pie_plan_forward(ctx, *base, out_len=out_len)
+            r = (pie.pie_plan_get_info(p), pie.pie_plan_debug_read(p, 2), pie.pie_plan_debug_read(p, 4).reshape(-1, 16),
+                 pie.pie_plan_debug_read(p, 5).reshape(-1, 16))
+            pie.pie_plan_destroy(p)
+            return r
+
+        for bad in (ql + (np.arange(wl.R) == 3), -(np.arange(wl.R) == 0).astype(np.int32)):
+            with pytest.raises(pie.PieError) as e:
+                plan(bad)
+            assert e.value.status == pie.PIE_ERR_INVALID
+        info_all, app_all, split_all, tile_all = plan(None)
+        info_same, app_same, split_same, tile_same = plan(ql)
+        assert info_same == info_all and np.array_equal(split_same, split_all) and np.array_equal(tile_same, tile_all)
+        out_len = np.minimum(ql, 1)
+        out_len[::3] = 0
+        info, app, split, tile = plan(out_len)
+        assert np.array_equal(app, app_all)
+        G = wl.H_q // wl.H_kv
+        for items in (split, tile):
+            for it in items:
+                r, row0, nrows = int(it[0]), int(it[2]), int(it[3])
+                assert out_len[r] > 0 and row0 + nrows <= out_len[r] * G
+                assert int(it[7]) == wl.qo_indptr[r] + ql[r] - out_len[r] and int(it[8]) == out_len[r]   # query start and length of the view
+        seen = {int(it[0]) for items in (split, tile) for it in items}
+        assert seen == {r for r in range(wl.R) if out_len[r] > 0}
+        nothing = plan(np.zeros(wl.R, np.int32))[0]
+        assert nothing["num_split_items"] == nothing["num_tile_items"] == nothing["num_simple_rows"] == 0
+    finally:
+        pie.pie_destroy(ctx)
