@@ -16,6 +16,8 @@ KvPages; Section 4.2 "Forward API" for masks, positions and the append-then-read
                 causal mask inferred from positions; grouped-query heads (kv = q // G);
   4. copy     - token-range copy of K and V rows between pages, bit for bit.
   5. page masks (`mask_kvpage`) - persistent per-page token masks ANDed into the allowed set.
+  6. next_dist - the sample stage's `get_next_dist` from the logits on: the next-token
+                distribution truncated to its K most probable tokens (Section 4.2 "Sample API").
 
 All floating point is fp64 on exactly widened inputs.  There is no tiling, no online
 softmax and no reordering: a reader can check each function against the definition by eye.
@@ -286,3 +288,29 @@ def merge_partials(o_parts, lse_parts):
     o = (w[..., None] * o_parts).sum(axis=0) / np.where(live, Z, 1.0)[..., None]
     o = np.where(live[..., None], o, 0.0)
     return o, lse
+
+
+# --------------------------------------------------------------------------- sample stage
+def next_dist(logits: np.ndarray, K: int):
+    """`get_next_dist` from the logits on (Section 4.2 "Sample API": the next-token probability
+    distribution, truncated to the top-K tokens, K = 256 by default).
+
+    logits [n, V] in the storage type (float32, or uint16 holding bf16 bit patterns).  Row by row:
+    p = softmax over the WHOLE vocabulary in fp64; the K most probable tokens are returned in order
+    of descending probability, equal logits in order of ascending token id, with their
+    probabilities as they stand in the full distribution (not renormalised over the K kept).
+    Returns ids [n, K] int64, probs [n, K] fp64.
+    """
+    x = widen(np.asarray(logits))
+    n, V = x.shape
+    assert 1 <= K <= V
+    ids = np.zeros((n, K), dtype=np.int64)
+    probs = np.zeros((n, K), dtype=np.float64)
+    for r in range(n):
+        m = x[r].max()
+        e = np.exp(x[r] - m)
+        p = e / e.sum()
+        order = sorted(range(V), key=lambda t: (-x[r, t], t))[:K]   # (by logit: exp is monotone, ties stay ties)
+        ids[r] = order
+        probs[r] = p[order]
+    return ids, probs

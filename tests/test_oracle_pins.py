@@ -509,3 +509,43 @@ def test_out_lens_follow_the_papers_listing_and_the_textbook():
                          s0["Q"][8:], s0["K"][8:], s0["V"][8:])
     np.testing.assert_allclose(Ob[0], O[8], atol=1e-14)
     np.testing.assert_allclose(Lb[0], L[8], atol=1e-14)
+
+
+def test_next_dist_pins():
+    """Top-K truncated next-token distribution (Section 4.2 "Sample API"): closed forms (logits = log of a
+    known distribution), K = V returns the whole distribution summing to 1, shift invariance, equal logits
+    in ascending token order, permutation equivariance, and a scalar-loop definition on small rows."""
+    rng = np.random.RandomState(41)
+    # closed form: logits = ln(p) + c  =>  probs = p, ids = argsort of p
+    p = rng.dirichlet(np.ones(50))
+    for c in (0.0, 7.5, -300.0):
+        ids, pr = orc.next_dist((np.log(p) + c)[None, :].astype(np.float64).astype(np.float32), 50)
+        assert np.array_equal(ids[0], np.argsort(-p, kind="stable"))
+        np.testing.assert_allclose(pr[0], np.sort(p)[::-1], rtol=2e-6 + abs(c) * 2e-7)   # (float32 storage of the logits)
+        assert abs(pr.sum() - 1.0) < 1e-12
+    # scalar-loop definition, with ties, on small rows
+    x = rng.randint(-3, 4, size=(6, 23)).astype(np.float32)
+    ids, pr = orc.next_dist(x, 5)
+    for r in range(6):
+        Z = math.fsum(math.exp(float(v)) for v in x[r])
+        want = sorted(range(23), key=lambda t: (-float(x[r, t]), t))[:5]
+        assert list(ids[r]) == want
+        for k, t in enumerate(want):
+            assert abs(pr[r, k] - math.exp(float(x[r, t])) / Z) < 1e-14
+        assert all(pr[r, k] >= pr[r, k + 1] for k in range(4))
+        for k in range(4):                                                   # equal probabilities: ascending ids
+            if x[r, ids[r, k]] == x[r, ids[r, k + 1]]:
+                assert ids[r, k] < ids[r, k + 1]
+    # permutation equivariance (no ties): permuting the vocabulary permutes the ids
+    y = rng.randn(3, 40).astype(np.float32)
+    perm = rng.permutation(40)
+    ids_a, pr_a = orc.next_dist(y, 7)
+    ids_b, pr_b = orc.next_dist(y[:, perm], 7)
+    assert np.array_equal(perm[ids_b], ids_a)
+    np.testing.assert_allclose(pr_a, pr_b, rtol=1e-13)
+    # bf16 storage: the bit patterns are widened exactly
+    import torch
+    z = torch.from_numpy(y).to(torch.bfloat16)
+    ids_c, pr_c = orc.next_dist(z.view(torch.int16).numpy().view(np.uint16), 7)
+    ids_d, pr_d = orc.next_dist(z.float().numpy(), 7)
+    assert np.array_equal(ids_c, ids_d) and np.array_equal(pr_c, pr_d)
