@@ -231,6 +231,23 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
 int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, const void* k_new,
                      const void* v_new, void* out, float* lse, void* stream);
 
+/* get_next_dist from the logits on (Table 1 `get_next_dist`; Section 4.2 "Sample API": the next-token
+ * probability distribution, truncated to the top-K tokens, K configurable, 256 by default).  The LM head
+ * that turns output Embeds into logits is a plain GEMM and not part of this library.
+ *   logits    device, [n_rows] rows of `vocab` entries, `row_stride` entries apart (>= vocab), of type
+ *             `dtype` (PIE_DTYPE_BF16 or PIE_DTYPE_F32; independent of the context's KV type).  16-byte
+ *             aligned rows are read with vector loads, others entry by entry.  Every row needs at
+ *             least one finite entry; -inf entries get probability 0.
+ *   top_k     1 .. 1024 and <= vocab.
+ *   out_ids   device, [n_rows][top_k] int32: the top_k most probable tokens of every row in order of
+ *             descending probability; equal logits in order of ascending token id (so the result is unique).
+ *   out_probs device, [n_rows][top_k] float: their probabilities in the softmax over the WHOLE vocabulary
+ *             (not renormalised over the kept tokens).
+ * Asynchronous on `stream`; buffers are the caller's.  Errors: PIE_ERR_INVALID (sizes, type, null
+ * pointers), PIE_ERR_NO_DEVICE, PIE_ERR_CUDA. */
+int pie_get_next_dist(pie_ctx* ctx, const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab,
+                      int64_t row_stride, int32_t top_k, int32_t* out_ids, float* out_probs, void* stream);
+
 /* Device-side status word: 0, or PIE_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel
  * gave up since the last call.  Synchronises `stream`, reads and clears the word. */
 int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out);

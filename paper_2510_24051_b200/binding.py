@@ -71,6 +71,7 @@ def _load():
         "pie_forward_host": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
         "pie_get_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int)]),
         "pie_forward_static_scratch": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
+        "pie_get_next_dist": (C.c_int, [vp, vp, i32, i32, i32, C.c_int64, i32, vp, vp, vp]),
         "pie_set_option": (C.c_int, [vp, C.c_int, C.c_int]),
         "pie_sched_create": (C.c_int, [i32, C.POINTER(vp)]),
         "pie_sched_destroy": (C.c_int, [vp]),
@@ -229,6 +230,16 @@ def pie_forward_host(ctx, qo_indptr, page_indptr, page_indices, last_page_len, q
     d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, None, out_len)
     _check(lib.pie_forward_host(ctx, C.byref(d), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse),
                                 _stream(stream)), ctx)
+
+
+def pie_get_next_dist(ctx, logits, top_k, out_ids, out_probs, stream=None):
+    """logits: 2-D torch tensor on the device (bf16 or fp32, rows may be strided); out_ids int32 / out_probs
+    fp32 tensors [n_rows, top_k]."""
+    import torch
+    dtype = {torch.bfloat16: PIE_DTYPE_BF16, torch.float32: PIE_DTYPE_F32}[logits.dtype]
+    assert logits.dim() == 2 and logits.stride(1) == 1
+    _check(lib.pie_get_next_dist(ctx, _ptr(logits), dtype, logits.shape[0], logits.shape[1], logits.stride(0), top_k,
+                                 _ptr(out_ids), _ptr(out_probs), _stream(stream)), ctx)
 
 
 def pie_get_last_device_status(ctx, stream=None):
