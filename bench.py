@@ -189,6 +189,105 @@ def run_reference(args):
     }))
 
 
+def run_next_dist(args, pie, torch, dist, rank, world, local, barrier):
+    """The sample stage next to the path (`get_next_dist`, Section 4.2 "Sample API"): one top-K truncated
+    distribution per request of the batched-decode workload - 64 rows over the 128,256-entry Llama-3
+    vocabulary, bf16 logits ~ N(0, 2.5) with a few tokens far ahead, K = 256.  Buffers rotate so that no
+    logits survive in L2 between steps."""
+    n, V, K = 64, 128256, 256
+    nbuf = 20                                                       # 20 x 16.4 MB > L2
+    g = torch.Generator(device="cuda").manual_seed(0x50494500 + 99 + 1000 * rank)
+    bufs = []
+    for _ in range(nbuf):
+        x = torch.randn(n, V, generator=g, device="cuda") * 2.5
+        x[:, ::977] += 9.0
+        bufs.append(x.to(torch.bfloat16))
+    ctx = pie.pie_create(4, 16, 4, 2, 64, "bf16", 4, 64, local)
+    ids = torch.empty(n, K, dtype=torch.int32, device="cuda")
+    probs = torch.empty(n, K, dtype=torch.float32, device="cuda")
+    sampler = ClockSampler(local)
+    for i in range(args.warmup):
+        pie.pie_get_next_dist(ctx, bufs[i % nbuf], K, ids, probs)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        pie.pie_get_next_dist(ctx, bufs[i % nbuf], K, ids, probs)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    clocks = sampler.stop() if rank == 0 else None
+    e2e = None
+    if not args.no_e2e:
+        host = [b.cpu().pin_memory() for b in bufs[:4]]
+        dev = torch.empty_like(bufs[0])
+        h_ids, h_probs = torch.empty(n, K, dtype=torch.int32).pin_memory(), torch.empty(n, K).pin_memory()
+        n_e2e = max(3, min(args.steps, 30))
+
+        def step(i):
+            dev.copy_(host[i % 4], non_blocking=True)
+            pie.pie_get_next_dist(ctx, dev, K, ids, probs)
+            h_ids.copy_(ids, non_blocking=True)
+            h_probs.copy_(probs, non_blocking=True)
+            torch.cuda.synchronize()
+
+        for i in range(3):
+            step(i)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            step(i)
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([e2e_s], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        e2e = {"value": world * n * n_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": n * V * 2,
+               "d2h_bytes_per_step": n * K * 8, "steps": n_e2e, "ms_per_step": e2e_s / n_e2e * 1e3,
+               "includes": "pinned H2D of the logits, get_next_dist, D2H of ids and probabilities"}
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import pie_oracle as orc
+        rows = bufs[0][:8].cpu().view(torch.int16).numpy().view(np.uint16)
+        t0 = time.perf_counter()
+        orc.next_dist(rows, K)
+        dt = time.perf_counter() - t0
+        cpu = {"value": len(rows) / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+               "sample": f"first {len(rows)} of {n} rows", "seconds": dt}
+    ms_per_step = ms / args.steps
+    alg = n * V * 2 + n * K * 8
+    peaks = load_peaks()
+    line = {
+        "metric": METRIC, "value": world * n / (ms_per_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "next_dist", "rows": n, "vocab": V, "top_k": K,
+                   "l2": f"{nbuf} rotating logit buffers ({nbuf * n * V * 2 / 1e6:.0f} MB) > L2", "launch": "eager"},
+        "hbm_gbs_step": alg / (ms_per_step * 1e-3) / 1e9, "algorithmic_bytes_step": {"logits": n * V * 2, "out": n * K * 8, "total": alg},
+        "kernel_ms": {"next_dist": ms_per_step},
+        "roofline": {"bound": "hbm", "kernel": "next_dist", "achieved": alg / (ms_per_step * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": alg / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                     "algorithmic_bytes": alg, "kernel_ms": ms_per_step, "timing": "timed region / launches (one kernel per step)",
+                     "peak_source": peaks["source"],
+                     "note": "64 rows = 64 thread blocks on 148 SMs; a block is bound by its two passes' arithmetic and the in-block sort"},
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    pie.pie_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -225,6 +324,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.workload == "next_dist":
+        return run_next_dist(args, pie, torch, dist, rank, world, local, barrier)
     wls, l2_note = build_workloads(args.workload, seed_offset=rank)
     wl0 = wls[0]
     ctx = pie.pie_create(wl0.num_pages, wl0.P, wl0.H_q, wl0.H_kv, wl0.D, wl0.dtype, max(wl0.R, 1), max(wl0.T, 1), local)
