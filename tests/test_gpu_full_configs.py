@@ -3,7 +3,6 @@ on sampled requests (the oracle computes any request on its own), plus size-inde
 properties: finite outputs everywhere, bit-exact append on sampled pages."""
 import numpy as np
 import pytest
-import torch
 
 from tests._util import bits, same_bits
 from workloads import configs

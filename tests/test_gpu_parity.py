@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from tests._util import bits, run_oracle, same_bits
-from workloads import configs, synth
+from workloads import configs
 
 pytestmark = pytest.mark.gpu
 

@@ -3,7 +3,6 @@ plan their slices with host-only contexts, and reduce tokens / time the way benc
 import os
 import sys
 
-import numpy as np
 import torch.multiprocessing as mp
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
