@@ -143,8 +143,10 @@ typedef struct pie_batch_desc {
   const int32_t* page_indptr;   /* [R+1], page_indptr[0] == 0                     */
   const int32_t* page_indices;  /* [page_indptr[R]]                               */
   const int32_t* last_page_len; /* [R]                                            */
-  const int64_t* mask_indptr;   /* [R+1] or NULL                                  */
-  const uint8_t* mask;          /* [mask_indptr[R]] or NULL                       */
+  const int64_t* mask_indptr;   /* [R+1] or NULL: request r's explicit mask is mask[mask_indptr[r] ..
+                                   mask_indptr[r+1]); an empty range = causal mask inferred from positions */
+  const uint8_t* mask;          /* q_len x kv_len bool bytes (1 = attend) per request with a mask, or NULL;
+                                   packed bits instead with PIE_PLAN_MASK_BITS                             */
   uint32_t flags;               /* PIE_PLAN_* below, 0 for the default path       */
   const int32_t* positions;     /* [T] explicit position of every new token, or NULL for the
                                    default kv_len - q_len + i.  Used only when the context
@@ -162,7 +164,10 @@ enum {
   PIE_PLAN_FORCE_SIMPLE = 1u,   /* run every request through the plain CUDA-core kernel   */
   PIE_PLAN_NO_TENSOR_TILES = 2u, /* keep prefill / tree requests off the tcgen05 tile path */
   PIE_PLAN_NO_CASCADE = 4u,     /* never attend a shared prefix once for a group of requests */
-  PIE_PLAN_CASCADE_ALWAYS = 8u  /* cascade every shared prefix, however small the saving (tests, tuning) */
+  PIE_PLAN_CASCADE_ALWAYS = 8u, /* cascade every shared prefix, however small the saving (tests, tuning) */
+  PIE_PLAN_MASK_BITS = 16u      /* `mask` holds bits, not bool bytes: for a request with a mask, q_len rows of
+                                   ceil(kv_len / 32) uint32 words (bit j of the row = position j, LSB first; bits
+                                   past kv_len are ignored), `mask` 4-byte aligned, mask_indptr counting WORDS */
 };
 
 typedef struct pie_plan_info {

@@ -14,7 +14,7 @@ import numpy as np
 from . import build as _build
 
 PIE_DTYPE_BF16, PIE_DTYPE_F32 = 0, 1
-PIE_PLAN_FORCE_SIMPLE, PIE_PLAN_NO_TENSOR_TILES, PIE_PLAN_NO_CASCADE, PIE_PLAN_CASCADE_ALWAYS = 1, 2, 4, 8
+PIE_PLAN_FORCE_SIMPLE, PIE_PLAN_NO_TENSOR_TILES, PIE_PLAN_NO_CASCADE, PIE_PLAN_CASCADE_ALWAYS, PIE_PLAN_MASK_BITS = 1, 2, 4, 8, 16
 PIE_OK = 0
 PIE_ERR_INVALID, PIE_ERR_NO_PAGES, PIE_ERR_BAD_PAGE, PIE_ERR_CONFLICT = -1, -2, -3, -4
 PIE_ERR_BATCH_TOO_LARGE, PIE_ERR_MASK, PIE_ERR_CUDA, PIE_ERR_NO_DEVICE = -5, -6, -7, -8
@@ -185,7 +185,10 @@ def pie_copy_kvpage(ctx, src, dst, src_off, dst_off, ntok, stream=None):
 def _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions=None, out_len=None):
     keep = [_i32(qo_indptr), _i32(page_indptr), _i32(page_indices), _i32(last_page_len)]
     mi = None if mask_indptr is None else np.ascontiguousarray(mask_indptr, dtype=np.int64)
-    mk = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
+    if mask is not None and (flags & PIE_PLAN_MASK_BITS):
+        mk = np.ascontiguousarray(mask, dtype=np.uint32)            # packed rows, mask_indptr counts words
+    else:
+        mk = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
     ps = None if positions is None else _i32(positions)
     ol = None if out_len is None else _i32(out_len)
     keep += [mi, mk, ps, ol]

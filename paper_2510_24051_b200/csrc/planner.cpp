@@ -564,6 +564,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   plan->kept.clear();
   const uint32_t full_bits = (P >= 32) ? 0xFFFFFFFFu : ((1u << P) - 1u);
   int64_t n_words = 0, mask_bytes_total = 0;
+  const bool bits_in = (b->flags & PIE_PLAN_MASK_BITS) != 0;   // the caller packed the masks itself
   for (int r = 0; r < R; ++r) {
     PieReq& q = plan->reqs[r];
     int64_t m0 = 0, m1 = 0;
@@ -574,12 +575,14 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       const int32_t* pages = b->page_indices + b->page_indptr[r];
       for (int lp = 0; lp <= q.last_logical && !page_masked; ++lp) page_masked = ctx->page_mask[pages[lp]] != 0xFFFFFFFFu;
     }
-    if (m1 > m0 && (!b->mask || m1 - m0 != (int64_t)q.q_len * q.kv_len)) return PIE_ERR_MASK;
+    // explicit mask: q_len x kv_len bool bytes, or (PIE_PLAN_MASK_BITS) q_len rows of ceil(kv_len / 32) words
+    const int64_t mask_units = bits_in ? (int64_t)q.q_len * ((q.kv_len + 31) / 32) : (int64_t)q.q_len * q.kv_len;
+    if (m1 > m0 && (!b->mask || m1 - m0 != mask_units)) return PIE_ERR_MASK;
     if (m1 > m0 || page_masked) {  // the request gets packed mask rows (given, or causal AND page masks)
       q.mask_row_words = ((q.kv_len + 127) / 128) * 4;
       q.mask_word_off = n_words;
       n_words += (int64_t)q.mask_row_words * q.q_len;
-      mask_bytes_total += m1 - m0;
+      mask_bytes_total += (m1 - m0) * (bits_in ? 4 : 1);
     } else {
       q.mask_row_words = 0;
       q.mask_word_off = 0;
@@ -609,7 +612,17 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       const int row_words = q.mask_row_words;
       uint32_t* w = plan->mask_words.data() + q.mask_word_off;
       const bool given = b->mask_indptr && b->mask_indptr[r + 1] > b->mask_indptr[r];
-      if (given) {
+      if (given && bits_in) {   // rows of ceil(kv_len / 32) words, LSB first: copied into the 128-bit padded rows
+        const int words_in = (q.kv_len + 31) / 32;
+        const uint32_t tail = (q.kv_len & 31) ? ((1u << (q.kv_len & 31)) - 1u) : 0xFFFFFFFFu;   // bits past kv_len are ignored
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(b->mask) + b->mask_indptr[r];
+        for (int i = 0; i < q.q_len; ++i) {
+          uint32_t* row = w + (size_t)i * row_words;
+          std::memcpy(row, src + (int64_t)i * words_in, (size_t)words_in * 4);
+          row[words_in - 1] &= tail;
+          for (int k = words_in; k < row_words; ++k) row[k] = 0u;
+        }
+      } else if (given) {
         const uint8_t* src = b->mask + b->mask_indptr[r];
         for (int i = 0; i < q.q_len; ++i)
           if (!pack_row(src + (int64_t)i * q.kv_len, q.kv_len, w + (size_t)i * row_words, row_words)) bad_mask.store(1);

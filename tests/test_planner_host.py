@@ -407,3 +407,42 @@ def test_out_len_validation_and_work_lists():
         assert nothing["num_split_items"] == nothing["num_tile_items"] == nothing["num_simple_rows"] == 0
     finally:
         pie.pie_destroy(ctx)
+
+
+@pytest.mark.parametrize("name", ["shared_prefix_tree", "long_context_policy", "tiny_fp32"])
+def test_masks_given_as_packed_bits_plan_like_bool_bytes(name):
+    """PIE_PLAN_MASK_BITS: the caller hands over rows of ceil(kv_len / 32) words instead of q_len x kv_len bool
+    bytes.  The plan must be byte for byte the one the bool matrix gives (bits past kv_len are ignored)."""
+    wl = configs.small(name)
+    mi, mb = wl.mask_bytes()
+    assert mi is not None
+    words, ptr = [], [0]
+    kv, ql = wl.kv_lens(), wl.q_lens()
+    rng = np.random.RandomState(2)
+    for r, m in enumerate(wl.masks):
+        if m is None:
+            ptr.append(ptr[-1])
+            continue
+        rw = (kv[r] + 31) // 32
+        bitsm = np.zeros((ql[r], rw * 32), dtype=np.uint8)
+        bitsm[:, :kv[r]] = np.asarray(m, dtype=np.uint8)
+        bitsm[:, kv[r]:] = rng.randint(0, 2, size=(ql[r], rw * 32 - kv[r]))      # garbage past the end
+        packed = np.packbits(bitsm.reshape(ql[r], rw, 32), axis=2, bitorder="little").view(np.uint32).reshape(-1)
+        words.append(packed)
+        ptr.append(ptr[-1] + packed.size)
+    ctx = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+    try:
+        pie.pie_alloc_kvpages(ctx, wl.num_pages)
+        base = (wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len)
+        a = pie.pie_plan_forward(ctx, *base, mi, mb)
+        b = pie.pie_plan_forward(ctx, *base, np.array(ptr, np.int64), np.concatenate(words), pie.PIE_PLAN_MASK_BITS)
+        assert np.array_equal(pie.pie_plan_debug_read(a, 3), pie.pie_plan_debug_read(b, 3))
+        assert pie.pie_plan_get_info(a) == pie.pie_plan_get_info(b)
+        pie.pie_plan_destroy(a)
+        pie.pie_plan_destroy(b)
+        with pytest.raises(pie.PieError) as e:                                   # wrong number of words
+            pie.pie_plan_forward(ctx, *base, np.array(ptr, np.int64) + np.arange(len(ptr)), np.concatenate(words + [np.zeros(len(ptr), np.uint32)]),
+                                 pie.PIE_PLAN_MASK_BITS)
+        assert e.value.status == pie.PIE_ERR_MASK
+    finally:
+        pie.pie_destroy(ctx)
