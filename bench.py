@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (null until a capture exists for that workload).
 NCU_TRAFFIC_BYTES = {
-    "batched_decode": 288_800_000,        # profiles/attn_split_kernel_batched_decode.md
+    "batched_decode": 289_000_000,        # profiles/attn_split_kernel_batched_decode.md
     "shared_prefix_tree": 968_300_000,    # profiles/attn_tc_kernel_shared_prefix_tree.md
 }
 
