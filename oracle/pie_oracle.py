@@ -98,15 +98,17 @@ def default_positions(qo_indptr, page_indptr, last_page_len, P) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- step 1: append
-def append_kv(pool, P, qo_indptr, page_indptr, page_indices, last_page_len, k_new, v_new):
+def append_kv(pool, P, qo_indptr, page_indptr, page_indices, last_page_len, k_new, v_new, skip=None):
     """Store the new K/V rows of every request in its pages (Table 1 `forward`, output
     KvPages; Section 4.2 listings: the new tokens occupy the last q_len positions).
 
     k_new, v_new: [T, H_kv, D] in the storage type.  The pool is updated in place; element
-    bits are copied unchanged.
+    bits are copied unchanged.  Requests with skip[r] set have no output KvPages: nothing is stored.
     """
     R = len(qo_indptr) - 1
     for r in range(R):
+        if skip is not None and skip[r]:
+            continue
         q_len = int(qo_indptr[r + 1] - qo_indptr[r])
         pages = page_indices[page_indptr[r]:page_indptr[r + 1]]
         kv_len = kv_len_of(len(pages), int(last_page_len[r]), P)
@@ -212,7 +214,7 @@ def apply_page_masks(allowed: np.ndarray, pages, P: int, page_masks) -> np.ndarr
 
 def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
             q, k_new, v_new, masks=None, append=True, requests=None, page_masks=None,
-            rope_theta=None, positions=None, out_lens=None):
+            rope_theta=None, positions=None, out_lens=None, no_store=None):
     """One batched `forward`: append, then gather and attend for every request.
 
     q [T, H_q, D], k_new/v_new [T, H_kv, D] in the storage type; masks is None or a list
@@ -225,6 +227,12 @@ def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
     produces outputs for its LAST out_lens[r] query tokens only - 0 = the rows are stored and
     nothing else.  Rows that produce no output come back as NaN (O and LSE); every row is
     appended and keeps its own position and mask row.
+
+    no_store (same passage: a call WITHOUT output KvPages, `forward(kv, iemb[-1:], oemb)` and
+    `forward([], iemb, [], oemb)` in the listing): request r's new rows take part in the attention
+    - they are the last q_len positions of its context - but are stored nowhere.  For such a request
+    the page list and last_page_len describe the EXISTING context only (an empty page list = none),
+    and an explicit mask is [q_len, existing + q_len].
     """
     R = len(qo_indptr) - 1
     T = int(qo_indptr[R])
@@ -238,21 +246,35 @@ def forward(pool, P, H_q, qo_indptr, page_indptr, page_indices, last_page_len,
         q64 = widen(to_storage(rope(q64, pos, rope_theta), np.asarray(q)))
         k_new = to_storage(rope(widen(k_new), pos, rope_theta), k_new)
     if append:
-        append_kv(pool, P, qo_indptr, page_indptr, page_indices, last_page_len, k_new, v_new)
+        append_kv(pool, P, qo_indptr, page_indptr, page_indices, last_page_len, k_new, v_new, skip=no_store)
     O = np.zeros((T, H_q, D), dtype=np.float64)
     LSE = np.full((T, H_q), -np.inf, dtype=np.float64)
     for r in (range(R) if requests is None else requests):
         t0, t1 = int(qo_indptr[r]), int(qo_indptr[r + 1])
         pages = page_indices[page_indptr[r]:page_indptr[r + 1]]
-        kv_len = kv_len_of(len(pages), int(last_page_len[r]), P)
+        unstored = no_store is not None and bool(no_store[r])
+        if unstored:   # the pages hold the existing context; the new rows follow it without being stored
+            kv_in = kv_len_of(len(pages), int(last_page_len[r]), P) if len(pages) else 0
+            kv_len = kv_in + (t1 - t0)
+        else:
+            kv_in = kv_len = kv_len_of(len(pages), int(last_page_len[r]), P)
         allowed = allowed_matrix(t1 - t0, kv_len, None if masks is None else masks[r])
-        allowed = apply_page_masks(allowed, pages, P, page_masks)
+        if page_masks:   # (page masks belong to stored rows: the existing context)
+            allowed = allowed.copy()
+            allowed[:, :kv_in] = apply_page_masks(allowed[:, :kv_in], pages, P, page_masks)
         first = 0 if out_lens is None else (t1 - t0) - int(out_lens[r])   # first query token that produces an output
         O[t0:t0 + first], LSE[t0:t0 + first] = np.nan, np.nan
         if first == t1 - t0:
             continue
         allowed = allowed[first:]
-        K, V = gather_kv(pool, P, pages, kv_len, needed=allowed.any(axis=0))
+        K, V = gather_kv(pool, P, pages, kv_in, needed=allowed[:, :kv_in].any(axis=0))
+        if unstored:
+            shape = (kv_len,) + tuple(np.asarray(k_new).shape[1:])
+            Kc, Vc = np.zeros(shape), np.zeros(shape)
+            if K is not None:
+                Kc[:kv_in], Vc[:kv_in] = K, V
+            Kc[kv_in:], Vc[kv_in:] = widen(k_new[t0:t1]), widen(v_new[t0:t1])
+            K, V = Kc, Vc
         O[t0 + first:t1], LSE[t0 + first:t1] = attend(q64[t0 + first:t1], K, V, allowed)
     return O, LSE
 

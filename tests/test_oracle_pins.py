@@ -549,3 +549,56 @@ def test_next_dist_pins():
     ids_c, pr_c = orc.next_dist(z.view(torch.int16).numpy().view(np.uint16), 7)
     ids_d, pr_d = orc.next_dist(z.float().numpy(), 7)
     assert np.array_equal(ids_c, ids_d) and np.array_equal(pr_c, pr_d)
+
+
+def test_no_store_follows_the_papers_listing_and_the_textbook():
+    """Section 4.2 listing: `forward([], iemb, [], oemb)` - nine tokens in, no KvPages at all, one output -
+    and `forward(kv, iemb[-1:], oemb)` - eight stored tokens plus one that is attended but not stored - give the
+    output of a plain nine-token prefill.  Checked against scalar-loop textbook attention; the pool is untouched."""
+    rng = np.random.RandomState(51)
+    P, H_q, H_kv, D, n = 4, 4, 2, 8, 9
+    Q = rng.randn(n, H_q, D).astype(np.float32)
+    K = rng.randn(n, H_kv, D).astype(np.float32)
+    V = rng.randn(n, H_kv, D).astype(np.float32)
+    Or, Lr = textbook_attention(Q, K, V, causal(n, n))
+
+    def fresh_pool():
+        return {p: (np.full((P, H_kv, D), np.nan, np.float32), np.full((P, H_kv, D), np.nan, np.float32)) for p in range(4)}
+
+    # line 3 of the listing: no pages in, none out, one output
+    pool = fresh_pool()
+    O, L = orc.forward(pool, P, H_q, np.array([0, n]), np.array([0, 0]), np.array([], np.int64), np.array([1]),
+                       Q, K, V, out_lens=[1], no_store=[1])
+    np.testing.assert_allclose(O[-1], Or[-1], atol=1e-12)
+    np.testing.assert_allclose(L[-1], Lr[-1], atol=1e-12)
+    assert np.isnan(O[:-1]).all() and all(np.isnan(a).all() and np.isnan(b).all() for a, b in pool.values())
+    # all nine outputs without storing anything
+    O, L = orc.forward(pool, P, H_q, np.array([0, n]), np.array([0, 0]), np.array([], np.int64), np.array([1]),
+                       Q, K, V, no_store=[1])
+    np.testing.assert_allclose(O, Or, atol=1e-12)
+    np.testing.assert_allclose(L, Lr, atol=1e-12)
+    # lines 6-7: eight tokens stored (pages 3 and 1), then one token attended over them without being stored
+    pages = np.array([3, 1])
+    orc.forward(pool, P, H_q, np.array([0, 8]), np.array([0, 2]), pages, np.array([4]), Q[:8], K[:8], V[:8], out_lens=[0])
+    before = {p: (a.copy(), b.copy()) for p, (a, b) in pool.items()}
+    O, L = orc.forward(pool, P, H_q, np.array([0, 1]), np.array([0, 2]), pages, np.array([4]), Q[8:], K[8:], V[8:],
+                       no_store=[1])
+    np.testing.assert_allclose(O[0], Or[-1], atol=1e-12)
+    np.testing.assert_allclose(L[0], Lr[-1], atol=1e-12)
+    for p in pool:
+        assert np.array_equal(pool[p][0], before[p][0], equal_nan=True) and np.array_equal(pool[p][1], before[p][1], equal_nan=True)
+    # a partly filled last page, an explicit mask over existing + new positions, mixed with a storing request
+    m = rng.rand(3, 6 + 3) < 0.6
+    m[:, 0] = True
+    pool = fresh_pool()
+    orc.forward(pool, P, H_q, np.array([0, 6]), np.array([0, 2]), np.array([2, 0]), np.array([2]), Q[:6], K[:6], V[:6], out_lens=[0])
+    O, L = orc.forward(pool, P, H_q, np.array([0, 3, 4]), np.array([0, 2, 3]), np.array([2, 0, 1]), np.array([2, 1]),
+                       Q[5:9], K[5:9], V[5:9], masks=[m, None], no_store=[1, 0])
+    Kc = np.concatenate([K[:6], K[5:8]])
+    Vc = np.concatenate([V[:6], V[5:8]])
+    Om, Lm = textbook_attention(Q[5:8], Kc, Vc, m)
+    np.testing.assert_allclose(O[:3], Om, atol=1e-12)
+    np.testing.assert_allclose(L[:3], Lm, atol=1e-12)
+    Os, Ls = textbook_attention(Q[8:9], K[8:9], V[8:9], [[True]])
+    np.testing.assert_allclose(O[3], Os[0], atol=1e-12)
+    assert np.array_equal(pool[1][0][0], K[8]) and np.isnan(pool[1][0][1:]).all() and np.isnan(pool[3][0]).all()
