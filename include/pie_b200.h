@@ -158,6 +158,17 @@ typedef struct pie_batch_desc {
                                    q_len rows are appended and keep their positions and mask rows;
                                    out / lse rows of tokens without output are left untouched.
                                    NULL = every token produces an output.             */
+  const uint8_t* no_store;      /* [R] or NULL.  Section 4.2: a forward call may have NO output KvPages
+                                   (`forward(kv, iemb[-1:], oemb)`, `forward([], iemb, [], oemb)` in the
+                                   paper's listing).  no_store[r] != 0: request r's new rows take part in
+                                   the attention as the last q_len positions of its context but are not
+                                   written to its pages.  For such a request the page list and
+                                   last_page_len describe the EXISTING context only (an empty page range =
+                                   none; last_page_len is then ignored) and an explicit mask is
+                                   [q_len x (existing + q_len)].  The plan borrows pages from the context's
+                                   free list for its lifetime (PIE_ERR_NO_PAGES if too few are free; the
+                                   caller's pages are never written); destroy such a plan only after its
+                                   forward calls have completed.                                        */
 } pie_batch_desc;
 
 enum {

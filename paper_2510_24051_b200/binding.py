@@ -30,7 +30,8 @@ class pie_config(C.Structure):
 class pie_batch_desc(C.Structure):
     _fields_ = [("num_requests", C.c_int32), ("qo_indptr", C.c_void_p), ("page_indptr", C.c_void_p),
                 ("page_indices", C.c_void_p), ("last_page_len", C.c_void_p), ("mask_indptr", C.c_void_p),
-                ("mask", C.c_void_p), ("flags", C.c_uint32), ("positions", C.c_void_p), ("out_len", C.c_void_p)]
+                ("mask", C.c_void_p), ("flags", C.c_uint32), ("positions", C.c_void_p), ("out_len", C.c_void_p),
+                ("no_store", C.c_void_p)]
 
 
 class pie_plan_info(C.Structure):
@@ -182,7 +183,8 @@ def pie_copy_kvpage(ctx, src, dst, src_off, dst_off, ntok, stream=None):
     _check(lib.pie_copy_kvpage(ctx, len(a[0]), *[x.ctypes.data for x in a], _stream(stream)), ctx)
 
 
-def _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions=None, out_len=None):
+def _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions=None, out_len=None,
+          no_store=None):
     keep = [_i32(qo_indptr), _i32(page_indptr), _i32(page_indices), _i32(last_page_len)]
     mi = None if mask_indptr is None else np.ascontiguousarray(mask_indptr, dtype=np.int64)
     if mask is not None and (flags & PIE_PLAN_MASK_BITS):
@@ -191,15 +193,16 @@ def _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask
         mk = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
     ps = None if positions is None else _i32(positions)
     ol = None if out_len is None else _i32(out_len)
-    keep += [mi, mk, ps, ol]
+    ns = None if no_store is None else np.ascontiguousarray(no_store, dtype=np.uint8)
+    keep += [mi, mk, ps, ol, ns]
     d = pie_batch_desc(len(keep[0]) - 1, keep[0].ctypes.data, keep[1].ctypes.data, keep[2].ctypes.data,
-                       keep[3].ctypes.data, _ptr(mi), _ptr(mk), flags, _ptr(ps), _ptr(ol))
+                       keep[3].ctypes.data, _ptr(mi), _ptr(mk), flags, _ptr(ps), _ptr(ol), _ptr(ns))
     return d, keep
 
 
 def pie_plan_forward(ctx, qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr=None,
-                     mask=None, flags=0, stream=None, positions=None, out_len=None):
-    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions, out_len)
+                     mask=None, flags=0, stream=None, positions=None, out_len=None, no_store=None):
+    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, positions, out_len, no_store)
     plan = C.c_void_p()
     _check(lib.pie_plan_forward(ctx, C.byref(d), _stream(stream), C.byref(plan)), ctx)
     return plan

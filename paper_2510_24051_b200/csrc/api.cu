@@ -165,6 +165,7 @@ PlanLayout pie_plan_layout(const pie_ctx* ctx, const pie_plan* plan) {
   L.tok = place(plan->tok_req.size() * 4);
   L.pos = place(plan->positions.size() * 4);
   L.simple = place(plan->simple_rows.size() * 4);
+  L.copies = place(plan->pre_copies.size() * 4);
   const PieLaunchList* lls[2] = {&plan->split, &plan->tile};
   for (int k = 0; k < 2; ++k) {
     L.items[k] = place(lls[k]->items.size() * sizeof(PieItem));
@@ -193,6 +194,7 @@ void pie_plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
   cp(L.tok, plan->tok_req.data(), plan->tok_req.size() * 4);
   cp(L.pos, plan->positions.data(), plan->positions.size() * 4);
   cp(L.simple, plan->simple_rows.data(), plan->simple_rows.size() * 4);
+  cp(L.copies, plan->pre_copies.data(), plan->pre_copies.size() * 4);
   const PieLaunchList* lls[2] = {&plan->split, &plan->tile};
   for (int k = 0; k < 2; ++k) {
     cp(L.items[k], lls[k]->items.data(), lls[k]->items.size() * sizeof(PieItem));
@@ -213,6 +215,7 @@ void pie_plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base) {
   plan->d_tok_req = (int32_t*)(base + L.tok);
   plan->d_positions = (int32_t*)(base + L.pos);
   plan->d_simple_rows = (int32_t*)(base + L.simple);
+  plan->d_pre_copies = (int32_t*)(base + L.copies);
   PieLaunchList* lls[2] = {&plan->split, &plan->tile};
   for (int k = 0; k < 2; ++k) {
     lls[k]->d_items = (PieItem*)(base + L.items[k]);
@@ -545,6 +548,7 @@ int pie_copy_kvpage(pie_ctx* ctx, int32_t n, const int32_t* src, const int32_t* 
 static const size_t kParkedPlans = 4;
 
 static void release_plan(pie_plan* plan) {
+  if (plan->ctx) pie_plan_release_scratch(plan);
   if (plan->d_blob || plan->h_image || plan->idle) {
     cudaSetDevice(plan->ctx->cfg.device);
     if (plan->d_blob) cudaFree(plan->d_blob);   // (synchronises: nothing can still be reading the arrays afterwards)
@@ -623,6 +627,7 @@ int pie_plan_destroy(pie_plan* plan) {
     release_plan(plan);
     return PIE_OK;
   }
+  pie_plan_release_scratch(plan);   // pages borrowed for requests without output KvPages go back now
   if (plan->used && plan->d_blob) {
     // a forward may still be reading the device arrays: mark the point behind it on its stream
     cudaSetDevice(ctx->cfg.device);
@@ -688,6 +693,11 @@ int pie_forward(pie_ctx* ctx, const pie_plan* plan, const void* q, const void* k
   if (plan->used && plan->last_stream != s) plan->many_streams = true;
   plan->last_stream = s;
   plan->used = true;
+  if (!plan->pre_copies.empty()) {   // rows of partly filled input pages of requests without output KvPages, into the plan's own pages
+    const int n_ops = (int)plan->pre_copies.size() / 5;
+    const int rc0 = timed_launch(ctx, PIE_KERNEL_COPY, s, [&] { return pie_launch_copy(ctx, n_ops, (const int32_t*)plan->d_pre_copies, s); });
+    if (rc0) return rc0;
+  }
   const void* q_in = q;
   int rc = plan->append_fused ? PIE_OK  // (q stays q_in: the split-KV kernel writes the new rows itself)
                               : timed_launch(ctx, PIE_KERNEL_APPEND, s, [&] { return pie_append_and_q(ctx, plan, q_in, k_new, v_new, s, &q); });

@@ -112,6 +112,11 @@ struct pie_plan {
   std::vector<int32_t> kept;        // pairs (phys, logical|flag)
   std::vector<int32_t> kept_scratch; // planner scratch (per-request slices before packing)
   std::vector<int32_t> clean_kept;   // [R] kept pages of the request before the first one some row sees only in part
+  // requests without output KvPages: pages of the library's own behind their page lists
+  std::vector<int32_t> scratch_pages;                                   // held until the plan is destroyed or rebuilt
+  std::vector<int32_t> pre_copies;                                      // (src, dst, src_off, dst_off, ntok) per copy, run before the append
+  std::vector<int32_t> int_page_indptr, int_page_indices, int_last_page_len;   // the rewritten batch
+  int32_t* d_pre_copies = nullptr;
   std::vector<uint32_t> mask_words;
   std::vector<int32_t> append_dst;  // [T] page*P + slot
   std::vector<int32_t> tok_req;     // [T]
@@ -236,7 +241,7 @@ int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_t
 // workspaces of the two tile launches): offsets, host-side fill of the uploaded part, binding of the
 // plan's device pointers to an image at `base`.
 struct PlanLayout {
-  size_t reqs, kept, mask, app, tok, pos, simple, items[2], cta[2], merges[2], ctr[2], ws_o[2], ws_lse[2];
+  size_t reqs, kept, mask, app, tok, pos, simple, copies, items[2], cta[2], merges[2], ctr[2], ws_o[2], ws_lse[2];
   size_t upload, total;
 };
 
@@ -244,7 +249,8 @@ PlanLayout pie_plan_layout(const pie_ctx* ctx, const pie_plan* plan);
 void pie_plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst);
 void pie_plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base);
 
-int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);  // host part (planner.cc)
+int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);
+void pie_plan_release_scratch(pie_plan* plan);  // host part (planner.cc)
 
 #define PIE_CUDA(ctx, expr)                                   \
   do {                                                        \

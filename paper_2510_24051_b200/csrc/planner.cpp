@@ -447,7 +447,108 @@ void chunk_units(const std::vector<Unit>& units, int n_warps, PieLaunchList& ll)
 
 }  // namespace
 
+static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);
+
+// Scratch pages a plan holds for requests without output KvPages go back to the free list.
+void pie_plan_release_scratch(pie_plan* plan) {
+  pie_ctx* ctx = plan->ctx;
+  for (int32_t id : plan->scratch_pages) {
+    if (ctx->page_mask[id] != 0xFFFFFFFFu) {
+      ctx->page_mask[id] = 0xFFFFFFFFu;
+      --ctx->n_masked_pages;
+    }
+    ctx->allocated[id] = 0;
+    ctx->free_list.push_back(id);
+  }
+  plan->scratch_pages.clear();
+  plan->pre_copies.clear();
+}
+
+// Requests WITHOUT output KvPages (Section 4.2: a forward call takes input KvPages and / or Embeds and fills
+// output Embeds and / or KvPages; `forward(kv, iemb[-1:], oemb)` in its listing): the new rows are attended
+// but must not land in the caller's pages.  The kernels read K/V from pool pages only, so such a request
+// gets pages of the library's own for the lifetime of the plan: the rows of a partly filled last input page
+// are copied into the first of them (a token-range page copy that pie_forward runs before the append), the
+// new rows are appended behind, and the request's page list becomes  full input pages ++ scratch pages.
+// Logical positions do not change, so masks and inferred causality stay as they are.
 int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
+  plan->ctx = ctx;
+  pie_plan_release_scratch(plan);   // (a reused plan object)
+  const int R = b->num_requests;
+  bool any = false;
+  if (b->no_store && R > 0 && R <= ctx->cfg.max_requests)
+    for (int r = 0; r < R; ++r) any = any || b->no_store[r] != 0;
+  if (!any) return build_plan_core(ctx, b, plan);
+  if (!b->qo_indptr || !b->page_indptr || !b->last_page_len || b->qo_indptr[0] != 0 || b->page_indptr[0] != 0) return PIE_ERR_INVALID;
+  const int P = ctx->cfg.page_size;
+  std::vector<int32_t>& ip = plan->int_page_indptr;
+  std::vector<int32_t>& idx = plan->int_page_indices;
+  std::vector<int32_t>& lpl = plan->int_last_page_len;
+  ip.assign(1, 0);
+  idx.clear();
+  lpl.clear();
+  int rc = PIE_OK;
+  for (int r = 0; r < R && rc == PIE_OK; ++r) {
+    const int q_len = b->qo_indptr[r + 1] - b->qo_indptr[r];
+    const int np = b->page_indptr[r + 1] - b->page_indptr[r];
+    if (q_len < 1 || np < 0 || (np > 0 && !b->page_indices)) {
+      rc = PIE_ERR_INVALID;
+      break;
+    }
+    const int32_t* pages = b->page_indices + b->page_indptr[r];
+    if (!b->no_store[r]) {
+      idx.insert(idx.end(), pages, pages + np);
+      lpl.push_back(b->last_page_len[r]);
+    } else {
+      const int last_in = np > 0 ? b->last_page_len[r] : P;
+      if (last_in < 1 || last_in > P) {
+        rc = PIE_ERR_INVALID;
+        break;
+      }
+      for (int k = 0; k < np; ++k)
+        if (pages[k] < 0 || pages[k] >= ctx->cfg.num_pages || !ctx->allocated[pages[k]]) rc = PIE_ERR_BAD_PAGE;
+      if (rc != PIE_OK) break;
+      const int carry = (np > 0 && last_in < P) ? last_in : 0;   // rows of the partly filled last input page
+      const int keep = carry ? np - 1 : np;                      // input pages that stay in the list
+      const int n_scratch = (carry + q_len + P - 1) / P;
+      if ((size_t)n_scratch > ctx->free_list.size()) {
+        rc = PIE_ERR_NO_PAGES;
+        break;
+      }
+      idx.insert(idx.end(), pages, pages + keep);
+      for (int k = 0; k < n_scratch; ++k) {
+        const int32_t id = ctx->free_list.back();
+        ctx->free_list.pop_back();
+        ctx->allocated[id] = 1;
+        plan->scratch_pages.push_back(id);
+        idx.push_back(id);
+        if (k == 0 && carry) {
+          plan->pre_copies.insert(plan->pre_copies.end(), {pages[np - 1], id, 0, 0, carry});
+          const uint32_t pm = ctx->page_mask[pages[np - 1]];   // a page mask travels with the copied rows
+          if (pm != 0xFFFFFFFFu) {
+            ctx->page_mask[id] = pm | ~((1u << carry) - 1u);
+            if (ctx->page_mask[id] != 0xFFFFFFFFu) ++ctx->n_masked_pages;
+          }
+        }
+      }
+      lpl.push_back(carry + q_len - (n_scratch - 1) * P);
+    }
+    ip.push_back((int32_t)idx.size());
+  }
+  if (rc == PIE_OK) {
+    pie_batch_desc bb = *b;
+    bb.page_indptr = ip.data();
+    bb.page_indices = idx.data();
+    bb.last_page_len = lpl.data();
+    bb.no_store = nullptr;
+    rc = build_plan_core(ctx, &bb, plan);
+    // (the fused append would be fine, but the copies must run first: keep the separate launches in order)
+  }
+  if (rc != PIE_OK) pie_plan_release_scratch(plan);
+  return rc;
+}
+
+static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   const pie_config& cfg = ctx->cfg;
   const int P = cfg.page_size, G = ctx->G;
   const int R = b->num_requests;
@@ -1006,7 +1107,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   info.workspace_bytes = ((int64_t)plan->split.n_slots * plan->split.slot_rows +
                           (int64_t)plan->tile.n_slots * plan->tile.slot_rows) * (cfg.head_dim + 1) * 4;
   info.side_by_side_sms = plan->overlap ? plan->tile.grid : 0;
-  info.launches = (plan->append_fused ? 0 : 1) + (info.num_simple_rows ? 1 : 0) + (info.num_split_items ? 1 : 0) +
+  info.launches = (plan->pre_copies.empty() ? 0 : 1) + (plan->append_fused ? 0 : 1) + (info.num_simple_rows ? 1 : 0) + (info.num_split_items ? 1 : 0) +
                   (info.num_tile_items ? 1 : 0) + (plan->split.merges.empty() ? 0 : 1) +
                   (plan->tile.merges.empty() ? 0 : 1);
   return PIE_OK;

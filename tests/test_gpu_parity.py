@@ -571,3 +571,105 @@ def orc_forward_with_out_lens(wl, pool, out_len):
     from oracle import pie_oracle as orc
     return orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
                        bits(wl.q()), bits(wl.k_new()), bits(wl.v_new()), wl.masks, out_lens=out_len)
+
+
+@pytest.mark.parametrize("flags", [0, 1, 2])
+def test_forward_without_output_kvpages(flags):
+    """Section 4.2: a forward call may have no output KvPages - the new rows are attended as the last positions
+    of the context but stored nowhere.  Requests with and without output pages share a batch: contexts that end
+    in the middle of a page or on a page boundary, no context at all, prefill chunks and single tokens, an
+    explicit mask, a page mask on the partly filled last page, outputs for the last token only.  Outputs match
+    the oracle, the caller's pages are bit for bit what the oracle's pool holds (only storing requests appended),
+    and the plan gives its borrowed pages back."""
+    import paper_2510_24051_b200 as pie
+    from oracle import pie_oracle as orc
+    from tests._gpu import TOL_LSE, TOL_O
+    from tests.test_gpu_matrix import _bf16_round
+    rng = np.random.RandomState(77)
+    P, H_q, H_kv, D = 16, 8, 2, 128
+    #          kv_in q_len no_store
+    shapes = [(37, 1, 1), (64, 1, 1), (0, 40, 1), (300, 70, 1), (45, 1, 0), (90, 33, 0), (21, 3, 1), (512, 1, 1)]
+    R = len(shapes)
+    num_pages = 160
+    perm = rng.permutation(100)
+    pool = {p: (np.full((P, H_kv, D), np.nan, np.float32), np.full((P, H_kv, D), np.nan, np.float32)) for p in range(num_pages)}
+    qo, pi, idx, last, masks, out_len, no_store = [0], [0], [], [], [], [], []
+    q_rows, k_rows, v_rows, cur = [], [], [], 0
+    for r, (kv_in, q_len, ns) in enumerate(shapes):
+        total = kv_in + q_len
+        K = _bf16_round(rng.randn(total, H_kv, D).astype(np.float32))
+        V = _bf16_round(rng.randn(total, H_kv, D).astype(np.float32))
+        n_list = (kv_in + P - 1) // P if ns else (total + P - 1) // P
+        pages = perm[cur:cur + n_list]
+        cur += n_list
+        for j in range(kv_in):
+            pool[int(pages[j // P])][0][j % P] = K[j]
+            pool[int(pages[j // P])][1][j % P] = V[j]
+        qo.append(qo[-1] + q_len)
+        pi.append(pi[-1] + n_list)
+        idx.extend(int(p) for p in pages)
+        last.append((kv_in if ns else total) - (n_list - 1) * P if n_list else 1)
+        m = None
+        if r == 3:                                                      # explicit mask over existing + new positions
+            pos = kv_in + np.arange(q_len)
+            m = (np.arange(total)[None, :] <= pos[:, None]) & (rng.rand(q_len, total) < 0.85)
+            m[np.arange(q_len), pos] = True
+        masks.append(m)
+        out_len.append(1 if r == 2 else q_len)
+        no_store.append(ns)
+        q_rows.append(_bf16_round(rng.randn(q_len, H_q, D).astype(np.float32)))
+        k_rows.append(K[kv_in:])
+        v_rows.append(V[kv_in:])
+    q, k_new, v_new = (np.concatenate(x) for x in (q_rows, k_rows, v_rows))
+    qo, pi, idx, last = np.array(qo), np.array(pi), np.array(idx), np.array(last)
+    hidden_page = int(idx[pi[6] + 1])                                   # request 6: second (partly filled) page, slots 1 and 3 hidden
+    pm_bits = 0xFFFFFFFF & ~0b1010
+    page_masks = {hidden_page: np.array([(pm_bits >> s) & 1 for s in range(P)], dtype=bool)}
+    pool_ref = {p: (a.copy(), b.copy()) for p, (a, b) in pool.items()}
+    O_ref, L_ref = orc.forward(pool_ref, P, H_q, qo, pi, idx, last, q, k_new, v_new, masks=masks, out_lens=out_len,
+                               no_store=no_store, page_masks=page_masks)
+    produced = ~np.isnan(L_ref[:, 0])
+    T = len(q)
+    ctx = pie.pie_create(num_pages, P, H_q, H_kv, D, "bf16", R, T, 0)
+    try:
+        ids = pie.pie_alloc_kvpages(ctx, 100)                            # 60 pages stay free for the plan to borrow
+        assert sorted(ids) == list(range(100))
+        tdt = torch.bfloat16
+        Kd = torch.from_numpy(np.stack([pool[int(p)][0] for p in ids])).to(tdt).cuda()
+        Vd = torch.from_numpy(np.stack([pool[int(p)][1] for p in ids])).to(tdt).cuda()
+        pie.pie_kvpage_write(ctx, ids, Kd, Vd)
+        pie.pie_mask_kvpage(ctx, [hidden_page], [pm_bits])
+        ptr = np.zeros(R + 1, np.int64)
+        for r, m in enumerate(masks):
+            ptr[r + 1] = ptr[r] + (0 if m is None else m.size)
+        buf = np.concatenate([m.reshape(-1).astype(np.uint8) for m in masks if m is not None])
+        free0 = pie.pie_num_free_kvpages(ctx)
+        plan = pie.pie_plan_forward(ctx, qo, pi, idx, last, ptr, buf, flags, out_len=out_len, no_store=no_store)
+        assert pie.pie_num_free_kvpages(ctx) < free0
+        out = torch.full((T, H_q, D), float("nan"), dtype=tdt, device="cuda")
+        lse = torch.full((T, H_q), float("nan"), dtype=torch.float32, device="cuda")
+        pie.pie_forward(ctx, plan, *(torch.from_numpy(x).to(tdt).cuda() for x in (q, k_new, v_new)), out, lse)
+        torch.cuda.synchronize()
+        assert pie.pie_get_last_device_status(ctx) == 0
+        pie.pie_plan_destroy(plan)
+        assert pie.pie_num_free_kvpages(ctx) == free0
+        O, L = out.double().cpu().numpy(), lse.double().cpu().numpy()
+        assert np.isnan(O[~produced]).all()
+        assert np.abs(O[produced] - O_ref[produced]).max() <= TOL_O["bf16"]
+        assert np.abs(L[produced] - L_ref[produced]).max() <= TOL_LSE
+        Kg = torch.empty((100, P, H_kv, D), dtype=tdt, device="cuda")
+        Vg = torch.empty_like(Kg)
+        pie.pie_kvpage_read(ctx, np.arange(100, dtype=np.int32), Kg, Vg)
+        torch.cuda.synchronize()
+        Kb, Vb = Kg.cpu().float().numpy(), Vg.cpu().float().numpy()
+        for pg in range(100):
+            assert same_bits(np.nan_to_num(Kb[pg], nan=7.0), np.nan_to_num(pool_ref[pg][0], nan=7.0)), pg
+            assert same_bits(np.nan_to_num(Vb[pg], nan=7.0), np.nan_to_num(pool_ref[pg][1], nan=7.0)), pg
+        # too few free pages for the borrowed ones
+        extra = pie.pie_alloc_kvpages(ctx, pie.pie_num_free_kvpages(ctx) - 1)
+        with pytest.raises(pie.PieError) as e:
+            pie.pie_plan_forward(ctx, qo, pi, idx, last, ptr, buf, flags, out_len=out_len, no_store=no_store)
+        assert e.value.status == pie.PIE_ERR_NO_PAGES and pie.pie_num_free_kvpages(ctx) == 1
+        pie.pie_dealloc_kvpages(ctx, extra)
+    finally:
+        pie.pie_destroy(ctx)

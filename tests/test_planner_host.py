@@ -446,3 +446,46 @@ def test_masks_given_as_packed_bits_plan_like_bool_bytes(name):
         assert e.value.status == pie.PIE_ERR_MASK
     finally:
         pie.pie_destroy(ctx)
+
+
+def test_requests_without_output_kvpages_borrow_and_return_pages(ctx):
+    """no_store requests (Section 4.2: no output KvPages): the plan borrows pages from the free list for the new
+    rows (and for the rows of a partly filled last input page), lists them behind the full input pages, and gives
+    them back when it is destroyed, rebuilt or fails."""
+    P = 16
+    ids = pie.pie_alloc_kvpages(ctx, 6)
+    free0 = pie.pie_num_free_kvpages(ctx)
+    #   r0: 37 existing rows (3 pages, last holds 5) + 1 new, not stored: keeps 2 pages, borrows 1, copies 5 rows
+    #   r1: 32 existing rows (2 full pages) + 20 new, not stored: keeps 2, borrows 2, no copy
+    #   r2: no context, 3 new, not stored: borrows 1
+    #   r3: stores as usual (1 page, 4 rows after the append)
+    args = dict(qo_indptr=[0, 1, 21, 24, 25], page_indptr=[0, 3, 5, 5, 6],
+                page_indices=[ids[0], ids[1], ids[2], ids[3], ids[4], ids[5]], last_page_len=[5, 16, 1, 4])
+    plan = pie.pie_plan_forward(ctx, **args, no_store=[1, 1, 1, 0])
+    assert pie.pie_num_free_kvpages(ctx) == free0 - 4
+    info = pie.pie_plan_get_info(plan)
+    kept = pie.pie_plan_debug_read(plan, 1).reshape(-1, 2)
+    app = pie.pie_plan_debug_read(plan, 2)
+    borrowed = [int(p) for p in kept[:, 0] if int(p) not in ids]
+    assert len(set(borrowed)) == 4 and info["kept_pages"] == 2 + 1 + 2 + 2 + 1 + 1
+    assert list(kept[:2, 0]) == [ids[0], ids[1]] and int(kept[2, 0]) == borrowed[0]          # r0: full pages, then the borrowed one
+    assert int(app[0]) == borrowed[0] * P + 5                                                # its new row lands behind the 5 copied rows
+    assert int(app[-1]) == ids[5] * P + 3                                                    # the storing request writes its own page
+    assert all(int(a) // P in borrowed for a in app[:-1])
+    pie.pie_plan_destroy(plan)
+    assert pie.pie_num_free_kvpages(ctx) == free0
+    # a failing batch (bad last_page_len of a later request) leaves nothing borrowed; so does running out of pages
+    assert status_of(pie.pie_plan_forward, ctx, **dict(args, last_page_len=[5, 16, 1, 40]), no_store=[1, 1, 1, 0]) == pie.PIE_ERR_INVALID
+    assert pie.pie_num_free_kvpages(ctx) == free0
+    hog = pie.pie_alloc_kvpages(ctx, free0 - 3)
+    assert status_of(pie.pie_plan_forward, ctx, **args, no_store=[1, 1, 1, 0]) == pie.PIE_ERR_NO_PAGES
+    assert pie.pie_num_free_kvpages(ctx) == 3
+    pie.pie_dealloc_kvpages(ctx, hog)
+    # a recycled plan object starts clean
+    for _ in range(3):
+        p2 = pie.pie_plan_forward(ctx, **args, no_store=[1, 1, 1, 0])
+        pie.pie_plan_destroy(p2)
+        p3 = pie.pie_plan_forward(ctx, qo_indptr=[0, 1, 3], page_indptr=[0, 3, 5], page_indices=list(ids[:5]), last_page_len=[6, 2])
+        assert pie.pie_num_free_kvpages(ctx) == free0
+        pie.pie_plan_destroy(p3)
+    pie.pie_dealloc_kvpages(ctx, ids)
