@@ -232,8 +232,8 @@ def pie_forward(ctx, plan, q, k_new, v_new, out, lse, stream=None):
 
 
 def pie_forward_host(ctx, qo_indptr, page_indptr, page_indices, last_page_len, q, k_new, v_new, out,
-                     lse, mask_indptr=None, mask=None, flags=0, stream=None, out_len=None):
-    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, None, out_len)
+                     lse, mask_indptr=None, mask=None, flags=0, stream=None, out_len=None, no_store=None):
+    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, None, out_len, no_store)
     _check(lib.pie_forward_host(ctx, C.byref(d), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse),
                                 _stream(stream)), ctx)
 
@@ -277,11 +277,11 @@ PIE_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
 def pie_forward_static_scratch(ctx, qo_indptr, page_indptr, page_indices, last_page_len, q, k_new, v_new,
-                               out, lse, mask_indptr=None, mask=None, flags=0, stream=None, out_len=None):
+                               out, lse, mask_indptr=None, mask=None, flags=0, stream=None, out_len=None, no_store=None):
     """forward for callers that cannot allocate device memory: plan arrays and split partials go
     to the library's fixed device array (at most PIE_STATIC_SCRATCH_BYTES, else
     PIE_ERR_BATCH_TOO_LARGE).  Tensors are device tensors; calls must not overlap on the GPU."""
-    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, None, out_len)
+    d, keep = _desc(qo_indptr, page_indptr, page_indices, last_page_len, mask_indptr, mask, flags, None, out_len, no_store)
     _check(lib.pie_forward_static_scratch(ctx, C.byref(d), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
                                           _ptr(lse), _stream(stream)), ctx)
 
