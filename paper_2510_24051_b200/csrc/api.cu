@@ -818,6 +818,7 @@ int pie_forward_host(pie_ctx* ctx, const pie_batch_desc* batch, const void* q, c
   PIE_CUDA(ctx, cudaMemcpyAsync(out, io + o_out, q_bytes, cudaMemcpyDeviceToHost, s));
   PIE_CUDA(ctx, cudaMemcpyAsync(lse, io + o_lse, lse_bytes, cudaMemcpyDeviceToHost, s));
   PIE_CUDA(ctx, cudaStreamSynchronize(s));
+  pie_plan_release_scratch(plan);   // (pages borrowed for requests without output KvPages: the forward is over)
   return PIE_OK;
 }
 
