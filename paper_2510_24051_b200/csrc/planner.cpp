@@ -105,22 +105,38 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
   const int grid = (int)std::min<int64_t>(grid_max, std::max<int64_t>(1, W / std::max(1, min_pages_per_cta)));
   ll.grid = grid;
 
-  if (allow_whole_units && (int64_t)units.size() >= 4 * (int64_t)grid && max_unit * 8 <= W / grid) {
+  // Whole units also when there are only a few per CTA, as long as dealing them out (largest first then)
+  // leaves the fullest CTA within 12 % of the average: a cut unit costs fp32 partials of up to 256 rows and
+  // the merge launch, which on a short launch is more than that imbalance (8 prefill chunks of 512 tokens:
+  // 137 -> 103 us).
+  const bool many_small = (int64_t)units.size() >= 4 * (int64_t)grid && max_unit * 8 <= W / grid;
+  const bool few_whole = !many_small && allow_whole_units && (int64_t)units.size() >= 2 * (int64_t)grid && W > 0;
+  if (allow_whole_units && (many_small || few_whole)) {
     // least-loaded-first list scheduling (binary heap keyed on (load, cta)), then a counting sort
     std::vector<std::pair<int64_t, int>> heap(grid);
     for (int c = 0; c < grid; ++c) heap[c] = {0, c};
     auto cmp = [](const std::pair<int64_t, int>& a, const std::pair<int64_t, int>& b) { return a > b; };
     std::make_heap(heap.begin(), heap.end(), cmp);
     std::vector<int32_t> owner(units.size());
+    std::vector<int32_t> order(units.size());
+    for (size_t k = 0; k < units.size(); ++k) order[k] = (int32_t)k;
+    if (few_whole)   // largest first (stable: equal units keep the batch order)
+      std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+        return units[a].page_end - units[a].page_begin > units[b].page_end - units[b].page_begin;
+      });
     ll.cta_ptr.assign(grid + 1, 0);
-    for (size_t k = 0; k < units.size(); ++k) {
+    int64_t max_load = 0;
+    for (size_t o = 0; o < units.size(); ++o) {
+      const size_t k = (size_t)order[o];
       std::pop_heap(heap.begin(), heap.end(), cmp);
       auto& top = heap.back();
       owner[k] = top.second;
       ++ll.cta_ptr[top.second + 1];
       top.first += std::max<int64_t>(1, units[k].page_end - units[k].page_begin);
+      max_load = std::max(max_load, top.first);
       std::push_heap(heap.begin(), heap.end(), cmp);
     }
+    if (few_whole && max_load * grid * 100 > W * 112) goto contiguous;   // too uneven: cut the units instead
     for (int c = 0; c < grid; ++c) ll.cta_ptr[c + 1] += ll.cta_ptr[c];
     std::vector<int32_t> fill(ll.cta_ptr.begin(), ll.cta_ptr.end() - 1);
     ll.items.resize(units.size());
@@ -138,6 +154,8 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
     return;
   }
 
+contiguous:
+  ll.cta_ptr.clear();
   // Contiguous shares.  Walking the units in order visits the shares in order too, so the items
   // come out already grouped by CTA; share c covers page visits [c W / grid, (c + 1) W / grid),
   // and its end is recomputed only when the walk crosses it (no division per piece).
@@ -984,7 +1002,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         for (int k = 0; k < cs.n; ++k)
           split_bytes += (double)(plan->reqs[cs.first + k].kept_count - cs.L) * cfg.num_kv_heads * 2.0 * P * cfg.head_dim * 2.0;
       for (const Unit& u : tile_units) tile_flops += (double)(u.page_end - u.page_begin) * P * 4.0 * cfg.head_dim * u.nrows;
-      const double t_split = split_bytes / 6.4e12, t_tile = tile_flops / 0.53e15;  // whole-chip estimates, seconds (rates measured on the mixed workload)
+      const double t_split = split_bytes / 6.4e12, t_tile = tile_flops / 0.60e15;  // whole-chip estimates, seconds (rates measured on the mixed workload)
       const double sat = 0.6 * ctx->n_sms;                                         // SMs that saturate the memory system
       int best_nt = 0;
       double best_t = 1e30;
