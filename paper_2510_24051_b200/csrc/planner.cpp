@@ -1006,7 +1006,10 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       const double sat = 0.6 * ctx->n_sms;                                         // SMs that saturate the memory system
       int best_nt = 0;
       double best_t = 1e30;
-      for (int nt = 8; nt <= ctx->n_sms - 16; nt += 2) {
+      // (on its own the planner only takes budgets that leave the decode kernel its saturating share: below it
+      //  the model's rates are too rough - one 4,096-token prefill next to 64 decodes ran 8 % slower side by side)
+      const int nt_max = ctx->options[PIE_OPT_OVERLAP] == 1 ? ctx->n_sms - 16 : ctx->n_sms - (int)(sat + 0.5);
+      for (int nt = 8; nt <= nt_max; nt += 2) {
         const int ns = ctx->n_sms - nt;
         const double ts = t_split * std::max(1.0, sat / ns), tt = t_tile * ctx->n_sms / nt;
         const double t = std::max(ts, tt);
