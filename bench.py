@@ -514,7 +514,7 @@ def main():
         peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
         roof = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(wl0.name), "useful_flops": flops,
-                "kernel_ms": dom_ms, "peak_source": peaks["source"] + " (sustained)"}
+                "kernel_ms": dom_ms, "timing": dom_timing, "peak_source": peaks["source"] + " (sustained)"}
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
