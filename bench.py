@@ -53,21 +53,28 @@ def load_peaks():
     return dict(FALLBACK_PEAKS, source="fallback")
 
 
-def build_workloads(name, seed_offset=0):
+def build_workloads(name, seed_offset=0, params=()):
     """The list of batches a run cycles through (several page placements when one batch's KV is
-    small enough to live in L2), plus a note saying how L2 reuse is defeated."""
+    small enough to live in L2), plus a note saying how L2 reuse is defeated.  `params` ("key=value"
+    strings, --param) override arguments of the workload's builder for shape sweeps."""
     from workloads import configs
     table = dict(configs.FULL, **configs.EXTRA)
     builder = table[name]
     seed = configs.SEED0 + list(table).index(name) + 1 + 1000 * seed_offset
+    kw = {}
+    for kv in params:
+        k, v = kv.split("=", 1)
+        kw[k] = int(v) if v.lstrip("-").isdigit() else (None if v == "None" else v)
     if name == "batched_decode":
-        probe = builder(seed=seed)
-        n_place = max(1, probe.num_pages // len(probe.page_indices))
-        wls = [builder(seed=seed, placement=i) for i in range(n_place)]
+        probe = builder(seed=seed, **kw)
+        n_place = max(1, min(16, probe.num_pages // len(probe.page_indices)))
+        wls = [builder(seed=seed, placement=i, **kw) for i in range(n_place)]
         note = f"{n_place} rotating page placements ({n_place * probe.algorithmic_bytes()['kv'] / 1e9:.2f} GB of KV) > L2"
     else:
-        wls = [builder(seed=seed)]
+        wls = [builder(seed=seed, **kw)]
         note = f"one placement; KV read per step {wls[0].algorithmic_bytes()['kv'] / 1e9:.2f} GB > L2"
+    if kw:
+        note += "; builder arguments " + ", ".join(f"{k}={v}" for k, v in kw.items())
     return wls, note
 
 
@@ -166,7 +173,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wls, _ = build_workloads(args.workload)
+    wls, _ = build_workloads(args.workload, params=args.param)
     wl = wls[0]
     times, tokens, desc, threads = [], 0, "", 1
     budget = 8.0
@@ -299,6 +306,7 @@ def main():
     ap.add_argument("--opt", action="append", default=[], help="pie_set_option as K=V (tuning runs)")
     ap.add_argument("--graph", type=int, default=0,
                     help="1: replay one captured CUDA graph per step (measured: no gain, the loop is GPU bound), 0: eager launches")
+    ap.add_argument("--param", action="append", default=[], help="builder argument of the workload as key=value (shape sweeps)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -326,7 +334,7 @@ def main():
 
     if args.workload == "next_dist":
         return run_next_dist(args, pie, torch, dist, rank, world, local, barrier)
-    wls, l2_note = build_workloads(args.workload, seed_offset=rank)
+    wls, l2_note = build_workloads(args.workload, seed_offset=rank, params=args.param)
     wl0 = wls[0]
     ctx = pie.pie_create(wl0.num_pages, wl0.P, wl0.H_q, wl0.H_kv, wl0.D, wl0.dtype, max(wl0.R, 1), max(wl0.T, 1), local)
     ids = pie.pie_alloc_kvpages(ctx, wl0.num_pages)
@@ -501,7 +509,7 @@ def main():
             alg += int(wl0.q_lens()[sel].sum()) * b_tok * 2
         achieved = alg / (dom_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(wl0.name),
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None if args.param else NCU_TRAFFIC_BYTES.get(wl0.name),
                 "algorithmic_bytes": alg, "kernel_ms": dom_ms, "timing": dom_timing, "peak_source": peaks["source"]}
     else:
         flops = 0
@@ -513,7 +521,7 @@ def main():
         achieved = flops / (dom_ms * 1e-3) / 1e12
         peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
         roof = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(wl0.name), "useful_flops": flops,
+                "frac": achieved / peak, "traffic": None if args.param else NCU_TRAFFIC_BYTES.get(wl0.name), "useful_flops": flops,
                 "kernel_ms": dom_ms, "timing": dom_timing, "peak_source": peaks["source"] + " (sustained)"}
 
     cpu = None
