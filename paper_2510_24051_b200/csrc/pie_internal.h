@@ -112,6 +112,7 @@ struct pie_plan {
   std::vector<int32_t> kept;        // pairs (phys, logical|flag)
   std::vector<int32_t> kept_scratch; // planner scratch (per-request slices before packing)
   std::vector<int32_t> clean_kept;   // [R] kept pages of the request before the first one some row sees only in part
+  std::vector<int32_t> local_key;    // planner scratch: the batch's decode units as a key of the context's list cache
   // requests without output KvPages: pages of the library's own behind their page lists
   std::vector<int32_t> scratch_pages;                                   // held until the plan is destroyed or rebuilt
   std::vector<int32_t> pre_copies;                                      // (src, dst, src_off, dst_off, ntok) per copy, run before the append
@@ -175,6 +176,18 @@ struct pie_ctx {
   size_t h_stage_bytes = 0;
   pie_plan* host_plan = nullptr;  // reused plan object of pie_forward_host
   std::vector<pie_plan*> parked_plans;  // destroyed plans kept for reuse: host arrays, pinned image, device arrays
+  // The block-local work list of the latest decode batch.  Consecutive steps of a serving loop bring the same
+  // requests with the same page counts (a request grows by a page every page_size steps), and then the list is
+  // the same up to the fields copied from the request records: the planner reuses it instead of dealing the
+  // units to thread blocks again.
+  struct LocalListCache {
+    bool valid = false, balanced = false;
+    int32_t sms = 0, warps = 0, slot_rows = 0;
+    std::vector<int32_t> key;        // (request, kv head, first row, rows, first page, end page) of every unit
+    std::vector<PieItem> items;
+    std::vector<int32_t> cta_ptr;
+    int32_t grid = 0, n_slots = 0;
+  } local_cache;
   std::string cuda_error;
   int options[PIE_NUM_OPTIONS] = {0, 0, 0, 0};
   cudaStream_t side_stream = nullptr;  // second stream of overlapped mixed batches

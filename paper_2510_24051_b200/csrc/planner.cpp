@@ -1072,9 +1072,45 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       // the extra partials cost more in the merge than the better balance gains on a 50 us launch)
       bool plain = true;   // cascade pieces bring partials of another launch: those groups need the merge kernel
       for (const Unit& u : split_units) plain = plain && !u.force_partial;
-      if (!plain || (ctx->options[PIE_OPT_NO_FUSION] & 2) ||
-          !partition_local(split_units, split_sms, pie_split_warps_per_block(ctx), 4, max_rows, plan->split))
-        partition(split_units, n_warps, 4, max_rows, false, plan->split);
+      bool local = plain && !(ctx->options[PIE_OPT_NO_FUSION] & 2);
+      if (local) {
+        // the same units as in the previous batch (a decode loop between two page boundaries): take its list
+        pie_ctx::LocalListCache& lc = ctx->local_cache;
+        const int nw = pie_split_warps_per_block(ctx);
+        std::vector<int32_t>& key = plan->local_key;
+        key.resize(6 * split_units.size());
+        for (size_t k = 0; k < split_units.size(); ++k) {
+          const Unit& u = split_units[k];
+          int32_t* d = key.data() + 6 * k;
+          d[0] = u.req, d[1] = u.kv_head, d[2] = u.row0, d[3] = u.nrows, d[4] = u.page_begin, d[5] = u.page_end;
+        }
+        if (lc.valid && lc.sms == split_sms && lc.warps == nw && lc.slot_rows == max_rows && lc.key == key) {
+          local = lc.balanced;
+          if (local) {
+            PieLaunchList& ll = plan->split;
+            ll.items = lc.items;
+            ll.cta_ptr = lc.cta_ptr;
+            ll.merges.clear();
+            ll.grid = lc.grid;
+            ll.n_slots = lc.n_slots;
+            ll.slot_rows = max_rows;
+            ll.n_static = 0;
+          }
+        } else {
+          local = partition_local(split_units, split_sms, nw, 4, max_rows, plan->split);
+          lc.valid = true;
+          lc.balanced = local;
+          lc.sms = split_sms, lc.warps = nw, lc.slot_rows = max_rows;
+          lc.key.swap(key);
+          if (local) {
+            lc.items = plan->split.items;
+            lc.cta_ptr = plan->split.cta_ptr;
+            lc.grid = plan->split.grid;
+            lc.n_slots = plan->split.n_slots;
+          }
+        }
+      }
+      if (!local) partition(split_units, n_warps, 4, max_rows, false, plan->split);
       plan->split.n_static = (int32_t)plan->split.items.size();
     }
   }

@@ -489,3 +489,58 @@ def test_requests_without_output_kvpages_borrow_and_return_pages(ctx):
         assert pie.pie_num_free_kvpages(ctx) == free0
         pie.pie_plan_destroy(p3)
     pie.pie_dealloc_kvpages(ctx, ids)
+
+
+def test_decode_work_list_reused_between_steps_equals_a_fresh_plan():
+    """Consecutive decode steps bring the same requests with the same page counts; the context then reuses the
+    block-local work list of the previous batch.  Every such plan must be byte for byte what a new context
+    produces: same batch again, every context one token longer (same pages), one request a page longer (other
+    units), and back."""
+    wl = configs.small("batched_decode")
+    P = wl.P
+
+    def variants():
+        base = (np.asarray(wl.qo_indptr), np.asarray(wl.page_indptr), np.asarray(wl.page_indices), np.asarray(wl.last_page_len))
+        yield base
+        yield base
+        grown = base[3].copy()
+        room = grown < P
+        grown[room] += 1                                    # one more token in the same last page
+        yield base[:3] + (grown,)
+        yield base[:3] + (grown,)
+        # request 0 gets one more page: other page counts, other work list
+        pi = base[1].copy()
+        pi[1:] += 1
+        idx = np.concatenate([base[2][:base[1][1]], [wl.num_pages - 1], base[2][base[1][1]:]])
+        last = base[3].copy()
+        last[0] = 1
+        yield (base[0], pi, idx, last)
+        yield base
+
+    def image(ctx, args):
+        plan = pie.pie_plan_forward(ctx, *args)
+        img, info = pie.pie_plan_debug_read(plan, 3), pie.pie_plan_get_info(plan)
+        pie.pie_plan_destroy(plan)
+        return img, info
+
+    def new_ctx(sms):
+        c = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+        pie.pie_set_option(c, pie.PIE_OPT_SPLIT_SMS, sms)
+        pie.pie_alloc_kvpages(c, wl.num_pages)
+        return c
+
+    for sms, local in ((6, True), (0, False)):    # few thread blocks: whole units per block, merged in the block; all: cut across blocks
+        ctx = new_ctx(sms)
+        try:
+            for n, args in enumerate(variants()):
+                fresh_ctx = new_ctx(sms)
+                try:
+                    want = image(fresh_ctx, args)
+                finally:
+                    pie.pie_destroy(fresh_ctx)
+                got = image(ctx, args)
+                assert got[1] == want[1], n
+                assert np.array_equal(got[0], want[0]), n
+                assert (got[1]["num_merge_groups"] == 0) == local
+        finally:
+            pie.pie_destroy(ctx)
