@@ -268,6 +268,12 @@ int pie_get_next_dist(pie_ctx* ctx, const void* logits, int32_t dtype, int32_t n
  * gave up since the last call.  Synchronises `stream`, reads and clears the word. */
 int pie_get_last_device_status(pie_ctx* ctx, void* stream, int* out);
 
+/* Test hook for the failure path.  Every wait inside the kernels is bounded: after about a second it
+ * gives up, sets the status word and the kernel drains.  This call enqueues a one-warp kernel whose only
+ * wait can never complete, so that a test can watch exactly that: pie_get_last_device_status then returns
+ * PIE_ERR_DEVICE_TIMEOUT once, and the context keeps working. */
+int pie_debug_bounded_wait(pie_ctx* ctx, void* stream);
+
 /* forward for callers that must not allocate device memory.  (The paper has no counterpart:
  * this entry point exists for the embedding application, not for the method.)
  *

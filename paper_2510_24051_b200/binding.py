@@ -72,6 +72,7 @@ def _load():
         "pie_forward_host": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
         "pie_get_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int)]),
         "pie_forward_static_scratch": (C.c_int, [vp, C.POINTER(pie_batch_desc), vp, vp, vp, vp, vp, vp]),
+        "pie_debug_bounded_wait": (C.c_int, [vp, vp]),
         "pie_get_next_dist": (C.c_int, [vp, vp, i32, i32, i32, C.c_int64, i32, vp, vp, vp]),
         "pie_set_option": (C.c_int, [vp, C.c_int, C.c_int]),
         "pie_sched_create": (C.c_int, [i32, C.POINTER(vp)]),
@@ -246,6 +247,10 @@ def pie_get_next_dist(ctx, logits, top_k, out_ids, out_probs, stream=None):
     assert logits.dim() == 2 and logits.stride(1) == 1
     _check(lib.pie_get_next_dist(ctx, _ptr(logits), dtype, logits.shape[0], logits.shape[1], logits.stride(0), top_k,
                                  _ptr(out_ids), _ptr(out_probs), _stream(stream)), ctx)
+
+
+def pie_debug_bounded_wait(ctx, stream=None):
+    _check(lib.pie_debug_bounded_wait(ctx, _stream(stream)), ctx)
 
 
 def pie_get_last_device_status(ctx, stream=None):

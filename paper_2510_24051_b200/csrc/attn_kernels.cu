@@ -952,3 +952,28 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   if (!plan.tile.merges.empty() && (rc = pie_launch_merge(ctx, &plan, plan.tile, out, lse, s))) return rc;
   return PIE_OK;
 }
+
+
+// ------------------------------------------------------------------------------ failure path probe
+// A warp waits on a barrier nobody arrives at.  The bounded wait gives up after about a second,
+// writes PIE_ERR_DEVICE_TIMEOUT to the status word and the kernel returns: the context stays usable.
+namespace {
+__global__ void wait_probe_kernel(int* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    pie_ptx::mbar_init(pie_ptx::smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  pie_ptx::mbar_wait(pie_ptx::smem_u32(&bar), 0, status);
+}
+}  // namespace
+
+int pie_debug_bounded_wait(pie_ctx* ctx, void* stream) {
+  if (!ctx) return PIE_ERR_INVALID;
+  if (ctx->host_only) return PIE_ERR_NO_DEVICE;
+  PIE_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  wait_probe_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(ctx->d_status);
+  PIE_CUDA(ctx, cudaGetLastError());
+  return PIE_OK;
+}

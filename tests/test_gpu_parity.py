@@ -673,3 +673,25 @@ def test_forward_without_output_kvpages(flags):
         pie.pie_dealloc_kvpages(ctx, extra)
     finally:
         pie.pie_destroy(ctx)
+
+
+def test_a_wait_that_cannot_complete_gives_up_and_the_context_stays_usable():
+    """Failure path without a fault: a kernel whose only wait has no producer.  The bounded wait runs out
+    after about a second, the status word reports it once, and a forward on the same context still matches
+    the oracle afterwards."""
+    import time
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs.small("mixed_prefill_decode")
+    O_ref, L_ref, _ = run_oracle(wl)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl)
+        t0 = time.perf_counter()
+        pie.pie_debug_bounded_wait(gp.ctx)
+        assert pie.pie_get_last_device_status(gp.ctx) == pie.PIE_ERR_DEVICE_TIMEOUT      # (synchronises the stream)
+        assert 0.5 < time.perf_counter() - t0 < 10.0
+        assert pie.pie_get_last_device_status(gp.ctx) == 0                                # read and cleared
+        plan = gp.plan(wl)
+        out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+        pie.pie_plan_destroy(plan)
+        check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
