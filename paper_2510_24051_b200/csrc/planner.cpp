@@ -1054,9 +1054,11 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
     }
   }
   // split-KV decode.  Long launches: chunks taken dynamically by the warps of the grid (evens out
-  // SMs that get different shares of the memory bandwidth).  Short launches: fixed equal shares,
-  // one per warp - fewer pieces, fewer partials to merge, and the per-chunk overheads matter more
-  // than the balance.
+  // SMs that get different shares of the memory bandwidth: 5-10 % of the launch).  Shorter ones: fixed
+  // shares - whole units per thread block with the merge inside the block when that balances, else one
+  // equal share per warp and the merge launch.  The dynamic list always needs the merge launch
+  // (10-20 us with its partials), so it pays from about 270 us on: 1.2 GB of K/V in 209 us against 192 us with
+  // whole units per block, 2.3 GB in 335 us against 353 us.
   {
     const int n_warps = split_sms * pie_split_warps_per_block(ctx);
     int64_t W = 0;
@@ -1065,7 +1067,11 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       W += u.page_end - u.page_begin;
       max_rows = std::max(max_rows, u.nrows);
     }
-    if (W >= (int64_t)200 * n_warps) {
+    const double kv_bytes = (double)W * 2.0 * P * cfg.head_dim * (cfg.dtype == PIE_DTYPE_BF16 ? 2.0 : 4.0);
+    const bool long_launch = kv_bytes * ctx->n_sms >= 1.6e9 * split_sms;   // (fewer SMs: the same bytes take longer)
+    bool plain_units = true;
+    for (const Unit& u : split_units) plain_units = plain_units && !u.force_partial;
+    if (long_launch || (W >= (int64_t)200 * n_warps && !plain_units)) {
       chunk_units(split_units, n_warps, plan->split);
     } else {
       // fixed equal shares, nothing left to the counter (a dynamic tail of small chunks was measured:
@@ -1110,8 +1116,12 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
           }
         }
       }
-      if (!local) partition(split_units, n_warps, 4, max_rows, false, plan->split);
-      plan->split.n_static = (int32_t)plan->split.items.size();
+      if (!local && W >= (int64_t)200 * n_warps) {
+        chunk_units(split_units, n_warps, plan->split);   // (many visits per warp and no balanced deal of whole units)
+      } else {
+        if (!local) partition(split_units, n_warps, 4, max_rows, false, plan->split);
+        plan->split.n_static = (int32_t)plan->split.items.size();
+      }
     }
   }
 
