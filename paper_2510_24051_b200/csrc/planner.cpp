@@ -105,12 +105,13 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
   const int grid = (int)std::min<int64_t>(grid_max, std::max<int64_t>(1, W / std::max(1, min_pages_per_cta)));
   ll.grid = grid;
 
-  // Whole units also when there are only a few per CTA, as long as dealing them out (largest first then)
-  // leaves the fullest CTA within 12 % of the average: a cut unit costs fp32 partials of up to 256 rows and
-  // the merge launch, which on a short launch is more than that imbalance (8 prefill chunks of 512 tokens:
-  // 137 -> 103 us).
+  // Whole units also when there are only a few per CTA (or fewer units than CTAs), as long as dealing them out
+  // (largest first then) leaves the fullest CTA within 12 % of the average or within 200 page visits (~45 us of
+  // a row-tile CTA) of it: a cut unit costs fp32 partials of up to 256 rows, more and shorter items and the merge
+  // launch, which on a short launch is more than that imbalance (8 prefill chunks of 512 tokens: 137 -> 78 us;
+  // one prompt of 2,048 tokens: 90 -> 46 us although only 64 of 148 CTAs get a unit).
   const bool many_small = (int64_t)units.size() >= 4 * (int64_t)grid && max_unit * 8 <= W / grid;
-  const bool few_whole = !many_small && allow_whole_units && (int64_t)units.size() >= 2 * (int64_t)grid && W > 0;
+  const bool few_whole = !many_small && allow_whole_units && W > 0;
   if (allow_whole_units && (many_small || few_whole)) {
     // least-loaded-first list scheduling (binary heap keyed on (load, cta)), then a counting sort
     std::vector<std::pair<int64_t, int>> heap(grid);
@@ -136,7 +137,7 @@ void partition(const std::vector<Unit>& units, int grid_max, int min_pages_per_c
       max_load = std::max(max_load, top.first);
       std::push_heap(heap.begin(), heap.end(), cmp);
     }
-    if (few_whole && max_load * grid * 100 > W * 112) goto contiguous;   // too uneven: cut the units instead
+    if (few_whole && max_load * grid * 100 > W * 112 && max_load > W / grid + 200) goto contiguous;   // too uneven: cut the units instead
     for (int c = 0; c < grid; ++c) ll.cta_ptr[c + 1] += ll.cta_ptr[c];
     std::vector<int32_t> fill(ll.cta_ptr.begin(), ll.cta_ptr.end() - 1);
     ll.items.resize(units.size());
