@@ -58,8 +58,6 @@ struct Elem<__nv_bfloat16> {
   }
 };
 
-// VEC consecutive entries of the row starting at `base` as keys; returns how many of them lie
-// inside the row (the others get key 0 and are ignored by their index).
 __device__ __forceinline__ float exp2f_fast(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -104,6 +102,8 @@ __device__ __forceinline__ void walk_row(const T* __restrict__ row, int vocab, F
   if (t < vocab) f(to_float(row[t]), t);
 }
 
+// VEC consecutive entries of the row starting at `base` as keys; returns how many of them lie
+// inside the row (the others get key 0 and are ignored by their index).
 template <typename T, bool kAligned>
 __device__ __forceinline__ int load_keys(const T* __restrict__ row, int base, int vocab, uint32_t* keys) {
   constexpr int VEC = Elem<T>::VEC;

@@ -304,9 +304,11 @@ bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int m
   }
   int64_t max_load = 0;
   for (int c = 0; c < n_ctas; ++c) max_load = std::max(max_load, load[c]);
-  // the fullest block may hold up to 8 % above the average: beyond that, cutting units across blocks and paying the
-  // merge launch (+4-5 us on a 55 us launch) is faster (batches at 6 % measured 58.9 vs 60.9 us, at 7 % 60.9 vs 65.8 us)
-  if (max_load * n_ctas * 100 > W * 108) return false;
+  // the fullest block may hold up to 8 % or 100 page visits above the average: beyond that, cutting units across blocks
+  // and paying the merge launch (+4-5 us on a 55 us launch) is faster (batches at 6 % measured 58.9 vs 60.9 us, at 7 %
+  // 60.9 vs 65.8 us; 32 and 48 requests, inside the 100 visits: 37.3 vs 40.2 and 46.5 vs 51.1 us; 16 requests and fewer
+  // lose with whole units: too few blocks get one)
+  if (max_load * n_ctas * 100 > W * 108 && max_load > W / n_ctas + 100) return false;
 
   // (items and warp ranges are written through plain pointers into arrays sized for the worst case,
   //  every unit whole plus one extra piece per warp; a reused plan keeps the arrays, and every field

@@ -496,7 +496,11 @@ def test_decode_work_list_reused_between_steps_equals_a_fresh_plan():
     block-local work list of the previous batch.  Every such plan must be byte for byte what a new context
     produces: same batch again, every context one token longer (same pages), one request a page longer (other
     units), and back."""
-    wl = configs.small("batched_decode")
+    _reused_work_list_case(configs.small("batched_decode"), 6, True)     # few thread blocks: whole units per block, merged in the block
+    _reused_work_list_case(configs.batched_decode(R=16), 0, False)        # long units on all blocks: cut across blocks, merge launch
+
+
+def _reused_work_list_case(wl, sms, local):
     P = wl.P
 
     def variants():
@@ -529,18 +533,17 @@ def test_decode_work_list_reused_between_steps_equals_a_fresh_plan():
         pie.pie_alloc_kvpages(c, wl.num_pages)
         return c
 
-    for sms, local in ((6, True), (0, False)):    # few thread blocks: whole units per block, merged in the block; all: cut across blocks
-        ctx = new_ctx(sms)
-        try:
-            for n, args in enumerate(variants()):
-                fresh_ctx = new_ctx(sms)
-                try:
-                    want = image(fresh_ctx, args)
-                finally:
-                    pie.pie_destroy(fresh_ctx)
-                got = image(ctx, args)
-                assert got[1] == want[1], n
-                assert np.array_equal(got[0], want[0]), n
-                assert (got[1]["num_merge_groups"] == 0) == local
-        finally:
-            pie.pie_destroy(ctx)
+    ctx = new_ctx(sms)
+    try:
+        for n, args in enumerate(variants()):
+            fresh_ctx = new_ctx(sms)
+            try:
+                want = image(fresh_ctx, args)
+            finally:
+                pie.pie_destroy(fresh_ctx)
+            got = image(ctx, args)
+            assert got[1] == want[1], n
+            assert np.array_equal(got[0], want[0]), n
+            assert (got[1]["num_merge_groups"] == 0) == local
+    finally:
+        pie.pie_destroy(ctx)

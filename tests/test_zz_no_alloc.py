@@ -22,7 +22,7 @@ def test_static_scratch_forward_matches_planned_forward(name):
         gp.install(wl)
         q, k, v = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
         plan = gp.plan(wl)
-        assert pie.pie_plan_get_info(plan)["num_merge_groups"] > 0      # the scratch partials are in use
+        assert pie.pie_plan_get_info(plan)["workspace_bytes"] > 0       # the scratch partials are in use (merged in the kernel or by the merge launch)
         ref_out, ref_lse = gp.forward(plan, q, k, v)
         pie.pie_plan_destroy(plan)
         mi, mb = wl.mask_bytes()
