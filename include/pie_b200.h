@@ -93,6 +93,9 @@ int pie_destroy(pie_ctx* ctx);
  * not allocated (PIE_ERR_BAD_PAGE) without freeing any. */
 int pie_alloc_kvpages(pie_ctx* ctx, int32_t n, int32_t* out_ids);
 int pie_dealloc_kvpages(pie_ctx* ctx, int32_t n, const int32_t* ids);
+/* Free pages, counting the pages that forwards of requests without output KvPages (no_store) have
+ * borrowed: both pie_num_free_kvpages and, when the free list is short, pie_alloc_kvpages wait for such
+ * forwards to finish before they answer. */
 int pie_num_free_kvpages(const pie_ctx* ctx, int32_t* out);
 
 /* Write / read whole pages in the canonical layout  K[n][page_size][H_kv][D], V[same]
@@ -167,8 +170,9 @@ typedef struct pie_batch_desc {
                                    none; last_page_len is then ignored) and an explicit mask is
                                    [q_len x (existing + q_len)].  The plan borrows pages from the context's
                                    free list for its lifetime (PIE_ERR_NO_PAGES if too few are free; the
-                                   caller's pages are never written); destroy such a plan only after its
-                                   forward calls have completed.                                        */
+                                   caller's pages are never written).  When the plan is destroyed the
+                                   pages return to the free list behind its latest forward: they are held
+                                   until the work enqueued on that forward's stream has finished.          */
 } pie_batch_desc;
 
 enum {
@@ -289,6 +293,12 @@ int pie_debug_bounded_wait(pie_ctx* ctx, void* stream);
  *
  *   - Arguments, results and errors are those of pie_forward, with `batch` (host) as in
  *     pie_plan_forward; q / k_new / v_new / out / lse are device pointers owned by the caller.
+ *   - The host blocks while the plan image (ordinary pageable host memory) is handed to the copy
+ *     engine; the kernels run asynchronously on `stream` as in pie_forward.
+ *   - Requests without output KvPages (no_store) work as in pie_forward: the pool pages they borrow
+ *     are handed back when the call returns and rejoin the free list once the work enqueued on
+ *     `stream` has finished (one CUDA event per such call, recycled - a host-side object, no device
+ *     memory).
  *   - A batch whose plan arrays plus split partials need more than PIE_STATIC_SCRATCH_BYTES is
  *     refused with PIE_ERR_BATCH_TOO_LARGE and nothing is enqueued.
  *   - The first call on a device looks up the array's device address (one cudaGetSymbolAddress,

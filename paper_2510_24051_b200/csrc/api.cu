@@ -272,6 +272,55 @@ int pie_launch_page_io(pie_ctx* ctx, int n, const int32_t* d_ids, void* K, void*
   return PIE_OK;
 }
 
+// ------------------------------------------------------------------------------------ borrowed pages
+void pie_reclaim_pages(pie_ctx* ctx, bool wait) {
+  if (ctx->held_pages.empty()) return;
+  cudaSetDevice(ctx->cfg.device);
+  size_t kept = 0;
+  for (size_t k = 0; k < ctx->held_pages.size(); ++k) {
+    pie_ctx::HeldPages& h = ctx->held_pages[k];
+    cudaError_t e = wait ? cudaEventSynchronize(h.done) : cudaEventQuery(h.done);
+    if (e == cudaErrorNotReady) {
+      cudaGetLastError();
+      if (kept != k) ctx->held_pages[kept] = std::move(h);
+      ++kept;
+      continue;
+    }
+    if (e != cudaSuccess) cudaGetLastError();   // (a failed device: nothing is running on the pages any more)
+    pie_free_pages(ctx, h.pages);
+    ctx->held_events.push_back(h.done);
+  }
+  ctx->held_pages.resize(kept);
+}
+
+void pie_plan_hold_scratch(pie_plan* plan, cudaStream_t s) {
+  pie_ctx* ctx = plan->ctx;
+  if (plan->scratch_pages.empty() || ctx->host_only) {
+    pie_plan_release_scratch(plan);
+    return;
+  }
+  cudaSetDevice(ctx->cfg.device);
+  cudaEvent_t ev = nullptr;
+  cudaError_t e = cudaSuccess;
+  if (!ctx->held_events.empty()) {
+    ev = ctx->held_events.back();
+    ctx->held_events.pop_back();
+  } else {
+    e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaEventRecord(ev, s);
+  if (e != cudaSuccess) {   // no event to wait behind: wait for the device instead, then the pages are free
+    cudaGetLastError();
+    cudaDeviceSynchronize();
+    if (ev) ctx->held_events.push_back(ev);
+    pie_plan_release_scratch(plan);
+    return;
+  }
+  ctx->held_pages.push_back(pie_ctx::HeldPages{ev, std::move(plan->scratch_pages)});
+  plan->scratch_pages.clear();
+  plan->pre_copies.clear();
+}
+
 // ------------------------------------------------------------------------------------ C ABI
 extern "C" {
 
@@ -385,6 +434,8 @@ int pie_destroy(pie_ctx* ctx) {
       cudaEventDestroy(t.stop);
     }
     for (auto e : ctx->free_events) cudaEventDestroy(e);
+    for (auto& h : ctx->held_pages) cudaEventDestroy(h.done);
+    for (auto e : ctx->held_events) cudaEventDestroy(e);
   }
   delete ctx->host_plan;
   for (pie_plan* plan : ctx->parked_plans) {
@@ -401,6 +452,8 @@ int pie_destroy(pie_ctx* ctx) {
 
 int pie_alloc_kvpages(pie_ctx* ctx, int32_t n, int32_t* out_ids) {
   if (!ctx || n < 0 || (n > 0 && !out_ids)) return PIE_ERR_INVALID;
+  pie_reclaim_pages(ctx, false);
+  if ((size_t)n > ctx->free_list.size()) pie_reclaim_pages(ctx, true);   // pages still borrowed by a running forward
   if ((size_t)n > ctx->free_list.size()) return PIE_ERR_NO_PAGES;
   for (int i = 0; i < n; ++i) {
     int32_t id = ctx->free_list.back();
@@ -446,6 +499,7 @@ int pie_mask_kvpage(pie_ctx* ctx, int32_t n, const int32_t* ids, const uint32_t*
 
 int pie_num_free_kvpages(const pie_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return PIE_ERR_INVALID;
+  pie_reclaim_pages(const_cast<pie_ctx*>(ctx), true);
   *out = (int32_t)ctx->free_list.size();
   return PIE_OK;
 }
@@ -548,7 +602,13 @@ int pie_copy_kvpage(pie_ctx* ctx, int32_t n, const int32_t* src, const int32_t* 
 static const size_t kParkedPlans = 4;
 
 static void release_plan(pie_plan* plan) {
-  if (plan->ctx) pie_plan_release_scratch(plan);
+  if (plan->ctx) {
+    if (plan->used && !plan->ctx->host_only && !plan->scratch_pages.empty()) {
+      cudaSetDevice(plan->ctx->cfg.device);
+      cudaDeviceSynchronize();   // its forwards may still be running on the borrowed pages
+    }
+    pie_plan_release_scratch(plan);
+  }
   if (plan->d_blob || plan->h_image || plan->idle) {
     cudaSetDevice(plan->ctx->cfg.device);
     if (plan->d_blob) cudaFree(plan->d_blob);   // (synchronises: nothing can still be reading the arrays afterwards)
@@ -627,7 +687,18 @@ int pie_plan_destroy(pie_plan* plan) {
     release_plan(plan);
     return PIE_OK;
   }
-  pie_plan_release_scratch(plan);   // pages borrowed for requests without output KvPages go back now
+  // pages borrowed for requests without output KvPages go back once the plan's forwards are over
+  if (plan->used && !plan->scratch_pages.empty() && !ctx->host_only) {
+    if (plan->many_streams) {
+      cudaSetDevice(ctx->cfg.device);
+      cudaDeviceSynchronize();
+      pie_plan_release_scratch(plan);
+    } else {
+      pie_plan_hold_scratch(plan, plan->last_stream);
+    }
+  } else {
+    pie_plan_release_scratch(plan);
+  }
   if (plan->used && plan->d_blob) {
     // a forward may still be reading the device arrays: mark the point behind it on its stream
     cudaSetDevice(ctx->cfg.device);

@@ -795,11 +795,9 @@ template <int D, int P, int NW, int DEPTH>
 int launch_split(pie_ctx* ctx, const AttnParams& p, int n_items, int n_warps, cudaStream_t s) {
   using C = SplitCfg<D, P, NW, DEPTH>;
   auto kern = attn_split_kernel<D, P, NW, DEPTH>;
-  static bool configured[8] = {};
-  int dev = ctx->cfg.device & 7;
-  if (!configured[dev]) {
+  if (!ctx->split_configured) {   // (a context has one shape, hence one instantiation, and one device)
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
-    configured[dev] = true;
+    ctx->split_configured = true;
   }
   const int blocks = (n_warps + NW - 1) / NW;
   PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(blocks), dim3(NW * 32), C::SMEM, s, p, n_items, blocks * NW));
@@ -811,11 +809,9 @@ int launch_tiles(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
   constexpr int NSTAGES = (128 * 1024) / (2 * P * D * 2);
   using C = TileCfg<D, P, NW, NSTAGES>;
   auto kern = attn_tile_kernel<D, P, NW, NSTAGES>;
-  static bool configured[8] = {};
-  int dev = ctx->cfg.device & 7;
-  if (!configured[dev]) {
+  if (!ctx->tile_configured) {
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
-    configured[dev] = true;
+    ctx->tile_configured = true;
   }
   PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3((NW + 1) * 32), C::SMEM, s, p));
   return PIE_OK;
@@ -932,7 +928,14 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   ctx->options[PIE_OPT_OVERLAP] = 2;  // this entry point enqueues its kernels one after the other
   int rc = pie_build_plan(ctx, batch, &plan);
   ctx->options[PIE_OPT_OVERLAP] = saved_overlap;
-  if (rc != PIE_OK) return rc;
+  if (rc != PIE_OK) return rc;   // (a failed build has given its borrowed pages back)
+  // Pages borrowed for requests without output KvPages: on every way out from here they are handed to
+  // the context, which returns them to the free list once the work enqueued on `s` so far is over.
+  struct Holder {
+    pie_plan* plan;
+    cudaStream_t s;
+    ~Holder() { pie_plan_hold_scratch(plan, s); }
+  } holder{&plan, s};
   if (plan.T == 0) return PIE_OK;
   if (!q || !k_new || !v_new || !out || !lse) return PIE_ERR_INVALID;
 
@@ -940,16 +943,20 @@ extern "C" int pie_forward_static_scratch(pie_ctx* ctx, const pie_batch_desc* ba
   if (L.total > (size_t)PIE_STATIC_SCRATCH_BYTES) return PIE_ERR_BATCH_TOO_LARGE;  // plan + partials exceed the static scratch
   // Nothing in the scratch has to start at zero: every plan array is overwritten by this copy
   // and every partial row is written by the attention kernel before a merge reads it.
+  // (The image is ordinary pageable host memory: the copy call returns once the runtime has staged it,
+  //  so the vector may go when this function returns.)
   std::vector<uint8_t> host(L.upload);
   pie_plan_fill(&plan, L, host.data());
   PIE_CUDA(ctx, cudaMemcpyAsync(base, host.data(), host.size(), cudaMemcpyHostToDevice, s));
   pie_plan_bind(&plan, L, base);
+  // rows of partly filled last input pages of requests without output KvPages, into the borrowed pages
+  if (!plan.pre_copies.empty() && (rc = pie_launch_copy(ctx, (int)plan.pre_copies.size() / 5, plan.d_pre_copies, s))) return rc;
   if ((rc = pie_append_and_q(ctx, &plan, q, k_new, v_new, s, &q))) return rc;
   if (!plan.simple_rows.empty() && (rc = pie_launch_simple(ctx, &plan, q, out, lse, s))) return rc;
-  if (!plan.split.items.empty() && (rc = pie_launch_split(ctx, &plan, q, k_new, v_new, out, lse, s))) return rc;
   if (!plan.tile.items.empty() && (rc = pie_launch_tiles(ctx, &plan, q, out, lse, s))) return rc;
-  if (!plan.split.merges.empty() && (rc = pie_launch_merge(ctx, &plan, plan.split, out, lse, s))) return rc;
   if (!plan.tile.merges.empty() && (rc = pie_launch_merge(ctx, &plan, plan.tile, out, lse, s))) return rc;
+  if (!plan.split.items.empty() && (rc = pie_launch_split(ctx, &plan, q, k_new, v_new, out, lse, s))) return rc;
+  if (!plan.split.merges.empty() && (rc = pie_launch_merge(ctx, &plan, plan.split, out, lse, s))) return rc;
   return PIE_OK;
 }
 

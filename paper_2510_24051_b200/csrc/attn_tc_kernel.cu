@@ -793,11 +793,9 @@ template <int D, int P>
 static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_tokens, cudaStream_t s) {
   using C = TcCfg<D, P>;
   auto kern = attn_tc_kernel<D, P>;
-  static bool configured[8] = {};
-  int dev = ctx->cfg.device & 7;
-  if (!configured[dev]) {
+  if (!ctx->tc_configured) {   // (a context has one shape, hence one instantiation, and one device)
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
-    configured[dev] = true;
+    ctx->tc_configured = true;
   }
   CUtensorMap qmap;
   memset(&qmap, 0, sizeof(qmap));

@@ -176,6 +176,12 @@ struct pie_ctx {
   size_t h_stage_bytes = 0;
   pie_plan* host_plan = nullptr;  // reused plan object of pie_forward_host
   std::vector<pie_plan*> parked_plans;  // destroyed plans kept for reuse: host arrays, pinned image, device arrays
+  // Pages a plan borrowed for requests without output KvPages go back to the free list only when the
+  // forward that used them is over: they wait here behind an event recorded on that forward's stream.
+  struct HeldPages { cudaEvent_t done; std::vector<int32_t> pages; };
+  std::vector<HeldPages> held_pages;
+  std::vector<cudaEvent_t> held_events;   // recycled events of held_pages
+  bool tc_configured = false, split_configured = false, tile_configured = false;   // kernel attributes set for this context's device
   // The block-local work list of the latest decode batch.  Consecutive steps of a serving loop bring the same
   // requests with the same page counts (a request grows by a page every page_size steps), and then the list is
   // the same up to the fields copied from the request records: the planner reuses it instead of dealing the
@@ -263,7 +269,14 @@ void pie_plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst);
 void pie_plan_bind(pie_plan* plan, const PlanLayout& L, uint8_t* base);
 
 int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);
-void pie_plan_release_scratch(pie_plan* plan);  // host part (planner.cc)
+// Borrowed pages of a plan (requests without output KvPages), host bookkeeping in planner.cpp:
+// back to the free list at once (no forward has used them, or it is known to be over) ...
+void pie_plan_release_scratch(pie_plan* plan);
+// ... or held until everything enqueued on `s` so far has finished (api.cu).
+void pie_plan_hold_scratch(pie_plan* plan, cudaStream_t s);
+// Returns held pages whose forward is over to the free list; wait = block until all of them are.
+void pie_reclaim_pages(pie_ctx* ctx, bool wait);
+void pie_free_pages(pie_ctx* ctx, const std::vector<int32_t>& ids);
 
 #define PIE_CUDA(ctx, expr)                                   \
   do {                                                        \

@@ -473,9 +473,8 @@ void chunk_units(const std::vector<Unit>& units, int n_warps, PieLaunchList& ll)
 static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan);
 
 // Scratch pages a plan holds for requests without output KvPages go back to the free list.
-void pie_plan_release_scratch(pie_plan* plan) {
-  pie_ctx* ctx = plan->ctx;
-  for (int32_t id : plan->scratch_pages) {
+void pie_free_pages(pie_ctx* ctx, const std::vector<int32_t>& ids) {
+  for (int32_t id : ids) {
     if (ctx->page_mask[id] != 0xFFFFFFFFu) {
       ctx->page_mask[id] = 0xFFFFFFFFu;
       --ctx->n_masked_pages;
@@ -483,6 +482,10 @@ void pie_plan_release_scratch(pie_plan* plan) {
     ctx->allocated[id] = 0;
     ctx->free_list.push_back(id);
   }
+}
+
+void pie_plan_release_scratch(pie_plan* plan) {
+  pie_free_pages(plan->ctx, plan->scratch_pages);
   plan->scratch_pages.clear();
   plan->pre_copies.clear();
 }
@@ -504,6 +507,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
   if (!any) return build_plan_core(ctx, b, plan);
   if (!b->qo_indptr || !b->page_indptr || !b->last_page_len || b->qo_indptr[0] != 0 || b->page_indptr[0] != 0) return PIE_ERR_INVALID;
   const int P = ctx->cfg.page_size;
+  pie_reclaim_pages(ctx, false);   // pages of earlier such batches whose forward is over
   std::vector<int32_t>& ip = plan->int_page_indptr;
   std::vector<int32_t>& idx = plan->int_page_indices;
   std::vector<int32_t>& lpl = plan->int_last_page_len;
@@ -534,6 +538,7 @@ int pie_build_plan(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan) {
       const int carry = (np > 0 && last_in < P) ? last_in : 0;   // rows of the partly filled last input page
       const int keep = carry ? np - 1 : np;                      // input pages that stay in the list
       const int n_scratch = (carry + q_len + P - 1) / P;
+      if ((size_t)n_scratch > ctx->free_list.size()) pie_reclaim_pages(ctx, true);   // wait for the forwards that still hold borrowed pages
       if ((size_t)n_scratch > ctx->free_list.size()) {
         rc = PIE_ERR_NO_PAGES;
         break;
@@ -666,7 +671,13 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       for (int lp = any_written ? 0 : first_written; lp <= q.last_logical; ++lp) {
         int32_t pg = pages[lp];
         uint32_t w = ctx->wmask[pg];
-        if (w == 0 || ctx->writer[pg] == r) continue;
+        if (w == 0) continue;
+        if (ctx->writer[pg] == r) {
+          // the request's own page: listed a second time below the rows it appends, the copy is read by
+          // another warp than the one that would write the new row in a fused append
+          if (lp < first_written) cross_read = true;
+          continue;
+        }
         cross_read = true;  // a page one request appends to is in another request's list
         if (ctx->writer[pg] >= 0 && ctx->writer[pg] < r) continue;  // written by an earlier request: visible
         uint32_t rd = slot_mask(0, lp == q.last_logical ? q.last_page_len : P);

@@ -573,17 +573,10 @@ def orc_forward_with_out_lens(wl, pool, out_len):
                        bits(wl.q()), bits(wl.k_new()), bits(wl.v_new()), wl.masks, out_lens=out_len)
 
 
-@pytest.mark.parametrize("flags", [0, 1, 2])
-def test_forward_without_output_kvpages(flags):
-    """Section 4.2: a forward call may have no output KvPages - the new rows are attended as the last positions
-    of the context but stored nowhere.  Requests with and without output pages share a batch: contexts that end
-    in the middle of a page or on a page boundary, no context at all, prefill chunks and single tokens, an
-    explicit mask, a page mask on the partly filled last page, outputs for the last token only.  Outputs match
-    the oracle, the caller's pages are bit for bit what the oracle's pool holds (only storing requests appended),
-    and the plan gives its borrowed pages back."""
-    import paper_2510_24051_b200 as pie
+def no_store_case():
+    """A batch that mixes requests with and without output KvPages (Section 4.2), its pool contents and the
+    oracle's results: shared by the tests of both forward entry points."""
     from oracle import pie_oracle as orc
-    from tests._gpu import TOL_LSE, TOL_O
     from tests.test_gpu_matrix import _bf16_round
     rng = np.random.RandomState(77)
     P, H_q, H_kv, D = 16, 8, 2, 128
@@ -628,6 +621,26 @@ def test_forward_without_output_kvpages(flags):
     pool_ref = {p: (a.copy(), b.copy()) for p, (a, b) in pool.items()}
     O_ref, L_ref = orc.forward(pool_ref, P, H_q, qo, pi, idx, last, q, k_new, v_new, masks=masks, out_lens=out_len,
                                no_store=no_store, page_masks=page_masks)
+    return dict(P=P, H_q=H_q, H_kv=H_kv, D=D, R=R, num_pages=num_pages, pool=pool, pool_ref=pool_ref, qo=qo, pi=pi, idx=idx,
+                last=last, masks=masks, out_len=out_len, no_store=no_store, q=q, k_new=k_new, v_new=v_new,
+                hidden_page=hidden_page, pm_bits=pm_bits, O_ref=O_ref, L_ref=L_ref)
+
+
+@pytest.mark.parametrize("flags", [0, 1, 2])
+def test_forward_without_output_kvpages(flags):
+    """Section 4.2: a forward call may have no output KvPages - the new rows are attended as the last positions
+    of the context but stored nowhere.  Requests with and without output pages share a batch: contexts that end
+    in the middle of a page or on a page boundary, no context at all, prefill chunks and single tokens, an
+    explicit mask, a page mask on the partly filled last page, outputs for the last token only.  Outputs match
+    the oracle, the caller's pages are bit for bit what the oracle's pool holds (only storing requests appended),
+    and the plan gives its borrowed pages back."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import TOL_LSE, TOL_O
+    c = no_store_case()
+    P, H_q, H_kv, D, R, num_pages = c["P"], c["H_q"], c["H_kv"], c["D"], c["R"], c["num_pages"]
+    pool, pool_ref, qo, pi, idx, last, masks = c["pool"], c["pool_ref"], c["qo"], c["pi"], c["idx"], c["last"], c["masks"]
+    out_len, no_store, q, k_new, v_new = c["out_len"], c["no_store"], c["q"], c["k_new"], c["v_new"]
+    hidden_page, pm_bits, O_ref, L_ref = c["hidden_page"], c["pm_bits"], c["O_ref"], c["L_ref"]
     produced = ~np.isnan(L_ref[:, 0])
     T = len(q)
     ctx = pie.pie_create(num_pages, P, H_q, H_kv, D, "bf16", R, T, 0)

@@ -547,3 +547,17 @@ def _reused_work_list_case(wl, sms, local):
             assert (got[1]["num_merge_groups"] == 0) == local
     finally:
         pie.pie_destroy(ctx)
+
+
+def test_a_request_listing_its_append_page_twice_keeps_the_append_launch(ctx):
+    """A decode batch normally lets the attention kernel write the new K/V row itself (one launch).  A request
+    that lists the page it appends to a second time, below the appended row, would have that copy read by
+    another warp than the one writing the row: the plan then keeps the separate append launch."""
+    ids = pie.pie_alloc_kvpages(ctx, 4)
+    plain = pie.pie_plan_forward(ctx, qo_indptr=[0, 1], page_indptr=[0, 3], page_indices=[ids[0], ids[1], ids[2]], last_page_len=[5])
+    fused = pie.pie_plan_get_info(plain)["launches"]
+    pie.pie_plan_destroy(plain)
+    twice = pie.pie_plan_forward(ctx, qo_indptr=[0, 1], page_indptr=[0, 3], page_indices=[ids[2], ids[1], ids[2]], last_page_len=[5])
+    assert pie.pie_plan_get_info(twice)["launches"] == fused + 1
+    pie.pie_plan_destroy(twice)
+    pie.pie_dealloc_kvpages(ctx, ids)
