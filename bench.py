@@ -1,18 +1,30 @@
 #!/usr/bin/env python
 """Benchmark of the batched `forward` attention handler on synthetic workloads.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME|all] [--impl reference]
 
 One "step" is one pass of the whole hot path over one coalesced batch: pie_forward (append of
 the new K/V rows, attention, merge of split partials) plus, for the long-context workload, the
 pie_copy_kvpage call that follows it.  Plans are built once (host planning time is reported
-separately as `plan_ms`); inputs are resident in HBM when the timed region starts.  The `e2e`
-figure repeats the measurement through pie_forward_host: planning, pinned-host -> device copies
-of Q/K/V and the device -> host read of the outputs are all inside its timed region.
+separately as `plan_ms`); inputs are resident in HBM when the timed region starts.  A timed
+region is exactly K steps between two synchronisations, measured with CUDA events; regions are
+repeated until a workload has at least `--min-seconds` of device time behind it and the median
+region is reported (with the fastest and slowest one beside it).
+
+With no `--workload` the run covers every baseline configuration in one go and prints ONE JSON
+line: the top level describes the headline workload (the largest single-GPU configuration,
+`long_context_policy`) and `workloads` holds one entry per configuration - each with its own
+step time, tokens/s, roofline of its dominant kernel, end-to-end figure, clocks and CPU baseline.
+
+The `e2e` figure goes through pie_forward_host: planning, pinned-host -> device copies of
+Q/K/V and the device -> host read of the outputs are inside its timed region.  For decode
+workloads it is a decode LOOP - every step appends one token to every request, so page lists,
+masks and the plan change from step to step as in a serving loop - and for the others a replay
+of the batch with a fresh plan per step.
 
 With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs its own batch
-of the same shape (requests are independent: no data-path collective); the time is the max over
-ranks and `value` counts all ranks' tokens (weak scaling).
+of the headline shape (requests are independent: no data-path collective); the time is the max
+over ranks and `value` counts all ranks' tokens (weak scaling).
 
 `--impl reference` times the fp64 CPU oracle on the same workload shape instead.
 """
@@ -20,6 +32,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -34,12 +47,17 @@ sys.path.insert(0, ROOT)
 
 METRIC = "attention tokens/s and achieved HBM GB/s / tensor TFLOPS vs B200 peak"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+HEADLINE = "long_context_policy"
+# the default run: the five baseline configurations (config 3 also as its two halves), then
+# two entries of our own (a small decode batch, the sample-stage handler)
+SUITE = ["long_context_policy", "batched_decode", "mixed_prefill_decode", "mixed_prefill_decode_prefill",
+         "mixed_prefill_decode_decode", "shared_prefix_tree", "batched_decode_r16", "next_dist"]
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (null until a capture exists for that workload).
-NCU_TRAFFIC_BYTES = {
-    "batched_decode": 289_000_000,        # profiles/attn_split_kernel_batched_decode.md
-    "shared_prefix_tree": 968_300_000,    # profiles/attn_tc_kernel_shared_prefix_tree.md
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu
+# capture per workload (not measured in this run: a profiler cannot run inside a timed benchmark)
+NCU_TRAFFIC = {
+    "batched_decode": (289_000_000, "ncu capture of the split-KV kernel on this workload, one launch"),
+    "shared_prefix_tree": (968_300_000, "ncu capture of the row-tile kernel on this workload, one launch"),
 }
 
 
@@ -53,20 +71,31 @@ def load_peaks():
     return dict(FALLBACK_PEAKS, source="fallback")
 
 
+def builder_of(name):
+    """(builder, fixed keyword arguments, index for the seed) of a workload name."""
+    from workloads import configs
+    table = dict(configs.FULL, **configs.EXTRA)
+    alias = {
+        "mixed_prefill_decode_prefill": ("mixed_prefill_decode", {"only": "prefill"}),
+        "mixed_prefill_decode_decode": ("mixed_prefill_decode", {"only": "decode"}),
+        "batched_decode_r16": ("batched_decode", {"R": 16}),
+    }
+    base, fixed = alias.get(name, (name, {}))
+    return table[base], dict(fixed), list(table).index(base) + 1
+
+
 def build_workloads(name, seed_offset=0, params=()):
     """The list of batches a run cycles through (several page placements when one batch's KV is
     small enough to live in L2), plus a note saying how L2 reuse is defeated.  `params` ("key=value"
     strings, --param) override arguments of the workload's builder for shape sweeps."""
     from workloads import configs
-    table = dict(configs.FULL, **configs.EXTRA)
-    builder = table[name]
-    seed = configs.SEED0 + list(table).index(name) + 1 + 1000 * seed_offset
-    kw = {}
+    builder, kw, index = builder_of(name)
+    seed = configs.SEED0 + index + 1000 * seed_offset
     for kv in params:
         k, v = kv.split("=", 1)
         kw[k] = int(v) if v.lstrip("-").isdigit() else (None if v == "None" else v)
     seed = kw.pop("seed", seed)
-    if name == "batched_decode":
+    if name.startswith("batched_decode"):
         probe = builder(seed=seed, **kw)
         n_place = max(1, min(16, probe.num_pages // len(probe.page_indices)))
         wls = [builder(seed=seed, placement=i, **kw) for i in range(n_place)]
@@ -74,6 +103,8 @@ def build_workloads(name, seed_offset=0, params=()):
     else:
         wls = [builder(seed=seed, **kw)]
         note = f"one placement; KV read per step {wls[0].algorithmic_bytes()['kv'] / 1e9:.2f} GB > L2"
+    for wl in wls:
+        wl.name = name
     if kw:
         note += "; builder arguments " + ", ".join(f"{k}={v}" for k, v in kw.items())
     return wls, note
@@ -109,29 +140,28 @@ class ClockSampler:
         time.sleep(0.15)
         self.proc.terminate()
         self.thread.join(timeout=2)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for r in self.rows:
             try:
                 sm.append(float(r[0])), mx.append(float(r[1]))
+                pw.append(float(r[2]))
             except (ValueError, IndexError):
                 continue
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "sm_min_mhz": min(sm) if sm else None, "power_w_max": max(pw) if pw else None,
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
 def oracle_sample(wl, budget_s=20.0):
-    """Time the fp64 oracle on a bounded sample of the workload's requests (inputs pre-generated).
-    Returns (tokens, seconds, description, threads)."""
+    """Time the fp64 oracle, as it stands, on a bounded sample of the workload's requests (inputs
+    pre-generated).  Returns (tokens, seconds, description, cores): cores = CPU time the process
+    spent per second of wall time, i.e. the threads that were actually busy (the oracle is one
+    Python thread; only its large matrix products fan out over the BLAS pool)."""
     from oracle import pie_oracle as orc
     from workloads import synth
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
-    except Exception:
-        threads = 1
     qb, kb, vb = (synth.to_numpy_bits(t) for t in (wl.q(), wl.k_new(), wl.v_new()))
     # estimate cost per request from its score-matrix size, then take a prefix that fits the budget
     cost = wl.q_lens() * wl.kept_tokens() * wl.H_q * wl.D * 4.0
@@ -159,14 +189,22 @@ def oracle_sample(wl, budget_s=20.0):
         for lp in range((kv - ql) // wl.P, len(wl.pages_of(r))):
             pool[int(wl.pages_of(r)[lp])]
     times = []
+    cpu0 = time.process_time()
     while not times or (sum(times) < min(budget_s, 10.0) and len(times) < 20):   # repeat short passes
         t0 = time.perf_counter()
         orc.forward(pool, wl.P, wl.H_q, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
                     qb, kb, vb, wl.masks, requests=sample)
         times.append(time.perf_counter() - t0)
+    cores = max(1, int(round((time.process_time() - cpu0) / max(sum(times), 1e-9))))
     dt = statistics.mean(times)
     tokens = int(wl.q_lens()[sample].sum())
-    return tokens, dt, f"first {n} of {wl.R} requests of {wl.name}, mean of {len(times)} passes", threads
+    return tokens, dt, f"first {n} of {wl.R} requests of {wl.name}, mean of {len(times)} passes", cores
+
+
+def cpu_baseline_of(wl, budget_s):
+    tokens, dt, desc, cores = oracle_sample(wl, budget_s=budget_s)
+    return {"value": tokens / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": desc, "seconds": dt,
+            "threads": "one Python thread; numpy's BLAS pool is used by large matrix products only"}
 
 
 def run_reference(args):
@@ -174,15 +212,17 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wls, _ = build_workloads(args.workload, params=args.param)
+    name = HEADLINE if args.workload == "all" else args.workload
+    wls, _ = build_workloads(name, params=args.param)
     wl = wls[0]
     times, tokens, desc, threads = [], 0, "", 1
     budget = 8.0
+    dt = 0.0
     for it in range(args.warmup + args.steps):
         tokens, dt, desc, threads = oracle_sample(wl, budget_s=budget)
         if it >= args.warmup:
             times.append(dt)
-        if (it + 1) * dt > 150:                        # keep the whole run within a few minutes
+        if (it + 1) * max(dt, budget) > 150:           # keep the whole run within a few minutes
             break
     dt = statistics.mean(times) if times else dt
     val = tokens / dt
@@ -197,159 +237,221 @@ def run_reference(args):
     }))
 
 
-def run_next_dist(args, pie, torch, dist, rank, world, local, barrier):
-    """The sample stage next to the path (`get_next_dist`, Section 4.2 "Sample API"): one top-K truncated
-    distribution per request of the batched-decode workload - 64 rows over the 128,256-entry Llama-3
-    vocabulary, bf16 logits ~ N(0, 2.5) with a few tokens far ahead, K = 256.  Buffers rotate so that no
-    logits survive in L2 between steps."""
-    n, V, K = 64, 128256, 256
-    nbuf = 20                                                       # 20 x 16.4 MB > L2
-    g = torch.Generator(device="cuda").manual_seed(0x50494500 + 99 + 1000 * rank)
-    bufs = []
-    for _ in range(nbuf):
-        x = torch.randn(n, V, generator=g, device="cuda") * 2.5
-        x[:, ::977] += 9.0
-        bufs.append(x.to(torch.bfloat16))
-    ctx = pie.pie_create(4, 16, 4, 2, 64, "bf16", 4, 64, local)
-    ids = torch.empty(n, K, dtype=torch.int32, device="cuda")
-    probs = torch.empty(n, K, dtype=torch.float32, device="cuda")
-    sampler = ClockSampler(local)
-    for i in range(args.warmup):
-        pie.pie_get_next_dist(ctx, bufs[i % nbuf], K, ids, probs)
-    barrier()
-    if rank == 0:
-        sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        pie.pie_get_next_dist(ctx, bufs[i % nbuf], K, ids, probs)
-    e1.record()
-    barrier()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    clocks = sampler.stop() if rank == 0 else None
-    e2e = None
-    if not args.no_e2e:
-        host = [b.cpu().pin_memory() for b in bufs[:4]]
-        dev = torch.empty_like(bufs[0])
-        h_ids, h_probs = torch.empty(n, K, dtype=torch.int32).pin_memory(), torch.empty(n, K).pin_memory()
-        n_e2e = max(3, min(args.steps, 30))
+class Env:
+    """torch / binding / process-group handles of this rank."""
 
-        def step(i):
-            dev.copy_(host[i % 4], non_blocking=True)
-            pie.pie_get_next_dist(ctx, dev, K, ids, probs)
-            h_ids.copy_(ids, non_blocking=True)
-            h_probs.copy_(probs, non_blocking=True)
+    def __init__(self):
+        import torch
+        import torch.distributed as dist
+        import paper_2510_24051_b200 as pie
+        self.torch, self.dist, self.pie = torch, dist, pie
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+        torch.cuda.set_device(self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def max_over_ranks(self, x):
+        if self.world == 1:
+            return x
+        t = self.torch.tensor([float(x)], dtype=self.torch.float64, device="cuda")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
+def timed_regions(env, step, steps, min_seconds, max_regions=4000):
+    """Regions of exactly `steps` steps, each between a barrier + synchronize on both sides and timed with
+    CUDA events on the launching stream (max over ranks), repeated until `min_seconds` of device time
+    have been measured.  Returns the per-region milliseconds."""
+    torch = env.torch
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    regions, total, i = [], 0.0, 0
+    while True:
+        env.barrier()
+        ev0.record()
+        for _ in range(steps):
+            step(i)
+            i += 1
+        ev1.record()
+        env.barrier()
+        ms = env.max_over_ranks(ev0.elapsed_time(ev1))
+        regions.append(ms)
+        total += ms
+        if total >= min_seconds * 1e3 or len(regions) >= max_regions:
+            return regions
+
+
+def install_context(env, ctx, wl):
+    pie, torch = env.pie, env.torch
+    used = wl.used_pages()
+    for i in range(0, len(used), 4096):
+        K, V = wl.context_pages(used[i:i + 4096], "cuda")
+        pie.pie_kvpage_write(ctx, used[i:i + 4096], K.contiguous(), V.contiguous())
+        torch.cuda.synchronize()
+        del K, V
+
+
+def e2e_decode_loop(env, args, name, wl0, ctx, hbuf, step_ms):
+    """End to end as a serving loop would call it: every step appends one token to every request, so
+    lengths, page lists, policy masks and therefore the plan change from step to step.  Small batches
+    (KV of a step close to the L2 size) run as several independent loops over different requests,
+    visited in turn, so that no step finds its pages in L2."""
+    from workloads import configs, synth
+    pie, torch = env.pie, env.torch
+    hq, hk, hv, hout, hlse = hbuf
+    n_steps = max(3, min(args.steps, 30 if step_ms > 0.5 else 300))
+    own_ctx = None
+    if name.startswith("batched_decode"):
+        builder, kw, _ = builder_of(name)
+        for kv in args.param:
+            k, v = kv.split("=", 1)
+            if k != "seed":
+                kw[k] = int(v) if v.lstrip("-").isdigit() else v
+        n_streams = max(2, min(8, int(math.ceil(3 * 126e6 / max(wl0.algorithmic_bytes()["kv"], 1)))))
+        visits = (n_steps + n_streams - 1) // n_streams
+        n_steps = visits * n_streams
+        grow = wl0.R * ((visits + wl0.P - 1) // wl0.P + 1)
+        streams, off = [], 0
+        sizes = []
+        for j in range(n_streams):   # (a first pass for the page counts: each loop has its own lengths)
+            probe = builder(seed=wl0.seed + 100 * (j + 1), **kw)
+            sizes.append(len(probe.page_indices))
+        num_pages = sum(sizes) + n_streams * grow
+        perm = synth.permutation(wl0.seed, 10, num_pages)
+        for j in range(n_streams):
+            wl = builder(seed=wl0.seed + 100 * (j + 1), perm_seed=wl0.seed, page_offset=off, **dict(kw, num_pages=num_pages))
+            spare = perm[off + sizes[j]:off + sizes[j] + grow]
+            off += sizes[j] + grow
+            streams.append((wl, configs.decode_loop(wl, visits, spare)))
+        own_ctx = pie.pie_create(num_pages, wl0.P, wl0.H_q, wl0.H_kv, wl0.D, wl0.dtype, wl0.R, wl0.T, env.local)
+        pie.pie_alloc_kvpages(own_ctx, num_pages)
+        for wl, _ in streams:
+            install_context(env, own_ctx, wl)
+        ctx = own_ctx
+        batches = [streams[s % n_streams][1][s // n_streams] for s in range(n_steps)]
+        how = f"decode loop: {n_streams} independent loops of {wl0.R} requests visited in turn, one token appended per visit"
+    else:
+        total = wl0.meta.get("pages_in_lists", len(wl0.page_indices))
+        perm = synth.permutation(wl0.seed, 10, wl0.num_pages)
+        spare = perm[total + (wl0.R if wl0.copies is not None else 0):]
+        batches = configs.decode_loop(wl0, n_steps, spare)
+        how = f"decode loop: one token appended to each of the {wl0.R} requests per step"
+
+    def e2e_step(i):
+        b = batches[i % len(batches)]
+        pie.pie_forward_host(ctx, b["qo_indptr"], b["page_indptr"], b["page_indices"], b["last_page_len"],
+                             hq, hk, hv, hout, hlse, b["mask_indptr"], b["mask"], args.flags)
+        if b["copies"] is not None:
+            c = b["copies"]
+            pie.pie_copy_kvpage(ctx, c["src"], c["dst"], c["src_off"], c["dst_off"], c["ntok"])
             torch.cuda.synchronize()
 
-        for i in range(3):
-            step(i)
-        barrier()
-        t0 = time.perf_counter()
-        for i in range(n_e2e):
-            step(i)
-        e2e_s = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([e2e_s], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
-        e2e = {"value": world * n * n_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": n * V * 2,
-               "d2h_bytes_per_step": n * K * 8, "steps": n_e2e, "ms_per_step": e2e_s / n_e2e * 1e3,
-               "includes": "pinned H2D of the logits, get_next_dist, D2H of ids and probabilities"}
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-    cpu = None
-    if not args.no_cpu_baseline:
-        from oracle import pie_oracle as orc
-        rows = bufs[0][:8].cpu().view(torch.int16).numpy().view(np.uint16)
-        t0 = time.perf_counter()
-        orc.next_dist(rows, K)
-        dt = time.perf_counter() - t0
-        cpu = {"value": len(rows) / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
-               "sample": f"first {len(rows)} of {n} rows", "seconds": dt}
-    ms_per_step = ms / args.steps
-    alg = n * V * 2 + n * K * 8
-    peaks = load_peaks()
-    line = {
-        "metric": METRIC, "value": world * n / (ms_per_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "next_dist", "rows": n, "vocab": V, "top_k": K,
-                   "l2": f"{nbuf} rotating logit buffers ({nbuf * n * V * 2 / 1e6:.0f} MB) > L2", "launch": "eager"},
-        "hbm_gbs_step": alg / (ms_per_step * 1e-3) / 1e9, "algorithmic_bytes_step": {"logits": n * V * 2, "out": n * K * 8, "total": alg},
-        "kernel_ms": {"next_dist": ms_per_step},
-        "roofline": {"bound": "hbm", "kernel": "next_dist", "achieved": alg / (ms_per_step * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": alg / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
-                     "algorithmic_bytes": alg, "kernel_ms": ms_per_step, "timing": "timed region / launches (one kernel per step)",
-                     "peak_source": peaks["source"],
-                     "note": "64 rows = 64 thread blocks on 148 SMs; a block is bound by its two passes' arithmetic and the in-block sort"},
-        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks,
-    }
-    print(json.dumps(line))
-    pie.pie_destroy(ctx)
-    if world > 1:
-        dist.destroy_process_group()
+    for i in range(3):   # (warm-up on the first steps; the timed loop starts over from step 0)
+        e2e_step(i)
+    env.barrier()
+    t0 = time.perf_counter()
+    for i in range(n_steps):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e2e_s = env.max_over_ranks(time.perf_counter() - t0)
+    if own_ctx is not None:
+        pie.pie_destroy(own_ctx)
+    return n_steps, e2e_s, how + "; host planning of every step, pinned H2D of Q/K/V, forward, D2H of O/LSE"
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="batched_decode")
-    ap.add_argument("--flags", type=int, default=0, help="PIE_PLAN_* flags (debug / A-B runs)")
-    ap.add_argument("--opt", action="append", default=[], help="pie_set_option as K=V (tuning runs)")
-    ap.add_argument("--graph", type=int, default=0,
-                    help="1: replay one captured CUDA graph per step (measured: no gain, the loop is GPU bound), 0: eager launches")
-    ap.add_argument("--param", action="append", default=[], help="builder argument of the workload as key=value (shape sweeps)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3)
-    if args.impl == "reference":
-        return run_reference(args)
+def roofline_of(wl0, name, info, ktimes, ms_per_step, peaks, n_gpus, clocks, region_s):
+    """Roofline entry of the workload's dominant kernel: algorithmic bytes (or useful flops) of one launch
+    divided by the kernel's live launch duration, against the measured peak."""
+    launches_per_step = info["launches"] + (1 if wl0.copies is not None else 0)
+    dom = max(("split", "tiles", "simple"), key=lambda k: ktimes[k][0])
+    dom_ms = ktimes[dom][0] / max(ktimes[dom][1], 1)
+    dom_timing = "events around each launch of the kernel"
+    if info.get("side_by_side_sms", 0) > 0:
+        # decode and prefill kernels run at the same time on disjoint SM sets: per-kernel events overlap, so the
+        # step is rated as a whole against the HBM roofline of its decode part (the prefill part is tensor work)
+        dom, dom_ms = "split", ms_per_step
+        dom_timing = "timed region / steps (decode and prefill kernels side by side)"
+    elif launches_per_step == 1 and n_gpus == 1:
+        # the step IS this one kernel: its launch duration is the timed region divided by the launches (the events
+        # around single launches keep consecutive launches from overlapping their prologues and report more)
+        dom_ms = min(dom_ms, ms_per_step)
+        dom_timing = "timed region / launches (one kernel per step)"
+    elif n_gpus == 1 and ms_per_step < dom_ms:
+        # a kernel cannot take longer than the whole step that contains it: bracketing every launch with events
+        # exposes launch latency and prologues that the back-to-back loop overlaps, so the step time is the bound
+        dom_ms = ms_per_step
+        dom_timing = "timed region / steps (upper bound: the step also contains the other kernels)"
+    G = wl0.H_q // wl0.H_kv
+    rows = wl0.q_lens() * G
+    sel = rows <= 16 if dom == "split" else rows > 16
+    b_tok = 2 * wl0.H_kv * wl0.D * wl0.esize
+    traffic, traffic_source = NCU_TRAFFIC.get(name, (None, "not captured"))
+    common = {"kernel_ms": dom_ms, "timing": dom_timing, "peak_source": peaks["source"], "traffic": traffic,
+              "traffic_source": traffic_source}
+    if dom == "tiles" and not sel.any():
+        # shared-prefix cascade: the row-tile kernel attends gathered decode rows to the shared pages and the
+        # split-KV kernel the private pages; together they read every distinct page once
+        dom_ms = sum(ktimes[k][0] / max(ktimes[k][1], 1) for k in ("tiles", "split"))
+        alg = len(np.unique(wl0.page_indices)) * wl0.P * b_tok + int(wl0.q_lens().sum()) * wl0.H_q * (2 * wl0.D * wl0.esize + 4)
+        achieved = alg / (dom_ms * 1e-3) / 1e9
+        return dict(common, bound="hbm", kernel="tiles+split (cascade)", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=achieved / peaks["hbm_gbs"], algorithmic_bytes=alg, kernel_ms=dom_ms)
+    if dom in ("split", "simple"):
+        kv_bytes = int(wl0.kept_tokens()[sel].sum()) * b_tok
+        qo_bytes = int(wl0.q_lens()[sel].sum()) * wl0.H_q * (2 * wl0.D * wl0.esize + 4)
+        mask_bytes = 0 if wl0.masks is None else sum((m.size + 7) // 8 for m, s in zip(wl0.masks, sel) if s and m is not None)
+        alg = kv_bytes + qo_bytes + mask_bytes
+        if dom == "split" and ktimes["append"][1] == 0:   # fused append: the split-KV kernel also moves the new rows
+            alg += int(wl0.q_lens()[sel].sum()) * b_tok * 2
+        achieved = alg / (dom_ms * 1e-3) / 1e9
+        return dict(common, bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=achieved / peaks["hbm_gbs"], algorithmic_bytes=alg)
+    flops = 0
+    for r in np.nonzero(sel)[0]:
+        m = None if wl0.masks is None else wl0.masks[r]
+        ql, kv = int(wl0.q_lens()[r]), int(wl0.kv_lens()[r])
+        n = (ql * kv - ql * (ql - 1) // 2) if m is None else int(m.sum())
+        flops += 4 * wl0.D * wl0.H_q * n
+    achieved = flops / (dom_ms * 1e-3) / 1e12
+    burst = peaks["bf16_tflops"]
+    sustained = peaks.get("bf16_tflops_sustained", burst)
+    # `frac` is always against the dense bf16 peak measured as a burst (cuBLAS at full clocks); the figure against
+    # the peak measured over seconds under the power cap is given beside it.  Which regime this run was in
+    # follows from the length of the timed region and the clocks sampled during it.
+    mhz, mx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    regime = "sustained" if (region_s >= 0.5 and mhz and mx and mhz < 0.9 * mx) else "burst"
+    return dict(common, bound="tensor", kernel=dom, achieved=achieved, peak=burst, unit="TFLOP/s", frac=achieved / burst,
+                peak_sustained=sustained, frac_sustained=achieved / sustained, regime=regime,
+                kernel_ms_x_sm_mhz=(dom_ms * mhz if mhz else None), useful_flops=flops,
+                peak_source=peaks["source"] + " (bf16_tflops burst; bf16_tflops_sustained beside it)")
 
-    import torch
-    import torch.distributed as dist
-    import paper_2510_24051_b200 as pie
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    if args.workload == "next_dist":
-        return run_next_dist(args, pie, torch, dist, rank, world, local, barrier)
-    wls, l2_note = build_workloads(args.workload, seed_offset=rank, params=args.param)
+def bench_workload(env, args, name, cpu_budget_s):
+    """One workload: device-resident timed regions, live per-kernel times, end to end through host buffers,
+    the oracle on a bounded sample.  Returns the workload's entry (rank 0; other ranks get None)."""
+    pie, torch = env.pie, env.torch
+    wls, l2_note = build_workloads(name, seed_offset=env.rank, params=args.param)
     wl0 = wls[0]
-    ctx = pie.pie_create(wl0.num_pages, wl0.P, wl0.H_q, wl0.H_kv, wl0.D, wl0.dtype, max(wl0.R, 1), max(wl0.T, 1), local)
+    ctx = pie.pie_create(wl0.num_pages, wl0.P, wl0.H_q, wl0.H_kv, wl0.D, wl0.dtype, max(wl0.R, 1), max(wl0.T, 1), env.local)
     ids = pie.pie_alloc_kvpages(ctx, wl0.num_pages)
     assert np.array_equal(ids, np.arange(wl0.num_pages))
     for kv in args.opt:
         k, v = kv.split("=")
         pie.pie_set_option(ctx, int(k), int(v))
     for wl in wls:                                     # install the pre-existing context (device generator)
-        used = wl.used_pages()
-        for i in range(0, len(used), 4096):
-            K, V = wl.context_pages(used[i:i + 4096], "cuda")
-            pie.pie_kvpage_write(ctx, used[i:i + 4096], K.contiguous(), V.contiguous())
-            torch.cuda.synchronize()
-            del K, V
+        install_context(env, ctx, wl)
     plans, plan_ms = [], []
     mask_args = [wl.mask_bytes() for wl in wls]
     for wl, (mi, mb) in zip(wls, mask_args):
@@ -403,20 +505,13 @@ def main():
 
     for i in range(args.warmup):
         step(i)
-    barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
+    env.barrier()
+    sampler = ClockSampler(env.local)
+    if env.rank == 0:
         sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for i in range(args.steps):
-        step(i)
-    ev1.record()
-    barrier()
-    ms = ev0.elapsed_time(ev1)
+    regions = timed_regions(env, step, args.steps, args.min_seconds)
     assert pie.pie_get_last_device_status(ctx) == 0, "a device-side wait timed out"
-    from paper_2510_24051_b200 import shard
-    total_tokens, ms = shard.aggregate(wl0.T, ms)          # sum of tokens, slowest rank's time
+    ms = statistics.median(regions)
     launches_per_step = info["launches"] + (1 if copies is not None else 0)
 
     # ---------------------------------------------------------------- per-kernel timing (live)
@@ -426,7 +521,7 @@ def main():
     torch.cuda.synchronize()
     ktimes = pie.pie_get_kernel_times(ctx)
     pie.pie_set_kernel_timing(ctx, 0)
-    clocks = sampler.stop() if rank == 0 else None         # covers both timed loops
+    clocks = sampler.stop() if env.rank == 0 else None         # covers the timed regions and the per-kernel loop
 
     # ---------------------------------------------------------------- end to end (host buffers)
     e2e = None
@@ -434,111 +529,54 @@ def main():
         hq, hk, hv = (t.cpu().pin_memory() for t in (q, k_new, v_new))
         hout = torch.empty_like(hq).pin_memory()
         hlse = torch.empty((wl0.T, wl0.H_q), dtype=torch.float32).pin_memory()
-        # (short steps: more of them, so that one hiccup of the host does not move the figure)
-        n_e2e = max(3, min(args.steps, 30 if ms / args.steps > 0.5 else 300))
-
-        def e2e_step(i):
-            wl = wls[i % len(wls)]
-            mi, mb = mask_args[i % len(wls)]
-            pie.pie_forward_host(ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
-                                 hq, hk, hv, hout, hlse, mi, mb, args.flags)
-            if copies is not None:
-                pie.pie_copy_kvpage(ctx, copies["src"], copies["dst"], copies["src_off"], copies["dst_off"], copies["ntok"])
-                torch.cuda.synchronize()
-
-        for i in range(3):
-            e2e_step(i)
-        barrier()
-        t0 = time.perf_counter()
-        for i in range(n_e2e):
-            e2e_step(i)
-        torch.cuda.synchronize()
-        e2e_s = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([e2e_s], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
         h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
         d2h = hout.numel() * hout.element_size() + hlse.numel() * 4
-        e2e = {"value": world * wl0.T * n_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": e2e_s / n_e2e * 1e3,
-               "includes": "host planning, pinned H2D of Q/K/V, forward, D2H of O/LSE"}
+        decode_only = bool((wl0.q_lens() == 1).all()) and (wl0.masks is None or "window" in wl0.meta)
+        if decode_only:
+            n_e2e, e2e_s, how = e2e_decode_loop(env, args, name, wl0, ctx, (hq, hk, hv, hout, hlse), ms / args.steps)
+        else:
+            # (short steps: more of them, so that one hiccup of the host does not move the figure)
+            n_e2e = max(3, min(args.steps, 30 if ms / args.steps > 0.5 else 300))
 
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+            def e2e_step(i):
+                wl = wls[i % len(wls)]
+                mi, mb = mask_args[i % len(wls)]
+                pie.pie_forward_host(ctx, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len,
+                                     hq, hk, hv, hout, hlse, mi, mb, args.flags)
 
-    # ---------------------------------------------------------------- roofline of the dominant kernel
+            for i in range(3):
+                e2e_step(i)
+            env.barrier()
+            t0 = time.perf_counter()
+            for i in range(n_e2e):
+                e2e_step(i)
+            torch.cuda.synchronize()
+            e2e_s = env.max_over_ranks(time.perf_counter() - t0)
+            how = "the same batch every step; host planning of every step, pinned H2D of Q/K/V, forward, D2H of O/LSE"
+        e2e = {"value": env.world * wl0.T * n_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": e2e_s / n_e2e * 1e3, "includes": how}
+
+    total_tokens = env.world * wl0.T if env.world > 1 else wl0.T    # every rank runs a batch of the same shape
+    for p in plans:
+        pie.pie_plan_destroy(p)
+    pie.pie_destroy(ctx)
+    del q, k_new, v_new, out, lse
+    torch.cuda.empty_cache()
+    if env.rank != 0:
+        return None
+
     peaks = load_peaks()
-    dom = max(("split", "tiles", "simple"), key=lambda k: ktimes[k][0])
-    dom_ms = ktimes[dom][0] / max(ktimes[dom][1], 1)
-    dom_timing = "events around each launch of the kernel"
-    if info.get("side_by_side_sms", 0) > 0:
-        # decode and prefill kernels run at the same time on disjoint SM sets: per-kernel events overlap, so the
-        # step is rated as a whole against the HBM roofline of its decode part (the prefill part is tensor work)
-        dom, dom_ms = "split", ms / args.steps
-        dom_timing = "timed region / steps (decode and prefill kernels side by side)"
-    elif launches_per_step == 1 and args.gpus == 1:
-        # the step IS this one kernel: its launch duration is the timed region divided by the launches (the events
-        # around single launches keep consecutive launches from overlapping their prologues and report more)
-        dom_ms = min(dom_ms, ms / args.steps)
-        dom_timing = "timed region / launches (one kernel per step)"
-    elif args.gpus == 1 and ms / args.steps < dom_ms:
-        # a kernel cannot take longer than the whole step that contains it: bracketing every launch with events
-        # exposes launch latency and prologues that the back-to-back loop overlaps, so the step time is the bound
-        dom_ms = ms / args.steps
-        dom_timing = "timed region / steps (upper bound: the step also contains the other kernels)"
-    G = wl0.H_q // wl0.H_kv
-    rows = wl0.q_lens() * G
-    sel = rows <= 16 if dom == "split" else rows > 16
-    b_tok = 2 * wl0.H_kv * wl0.D * wl0.esize
-    if dom == "tiles" and not sel.any():
-        # shared-prefix cascade: the row-tile kernel attends gathered decode rows to the shared pages and the
-        # split-KV kernel the private pages; together they read every distinct page once
-        dom_ms = sum(ktimes[k][0] / max(ktimes[k][1], 1) for k in ("tiles", "split"))
-        alg = len(np.unique(wl0.page_indices)) * wl0.P * b_tok + int(wl0.q_lens().sum()) * wl0.H_q * (2 * wl0.D * wl0.esize + 4)
-        achieved = alg / (dom_ms * 1e-3) / 1e9
-        roof = {"bound": "hbm", "kernel": "tiles+split (cascade)", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "algorithmic_bytes": alg, "kernel_ms": dom_ms,
-                "peak_source": peaks["source"]}
-    elif dom in ("split", "simple"):
-        kv_bytes = int(wl0.kept_tokens()[sel].sum()) * b_tok
-        qo_bytes = int(wl0.q_lens()[sel].sum()) * wl0.H_q * (2 * wl0.D * wl0.esize + 4)
-        mask_bytes = 0 if wl0.masks is None else sum((m.size + 7) // 8 for m, s in zip(wl0.masks, sel) if s and m is not None)
-        alg = kv_bytes + qo_bytes + mask_bytes
-        if dom == "split" and ktimes["append"][1] == 0:   # fused append: the split-KV kernel also moves the new rows
-            alg += int(wl0.q_lens()[sel].sum()) * b_tok * 2
-        achieved = alg / (dom_ms * 1e-3) / 1e9
-        roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None if args.param else NCU_TRAFFIC_BYTES.get(wl0.name),
-                "algorithmic_bytes": alg, "kernel_ms": dom_ms, "timing": dom_timing, "peak_source": peaks["source"]}
-    else:
-        flops = 0
-        for r in np.nonzero(sel)[0]:
-            m = None if wl0.masks is None else wl0.masks[r]
-            ql, kv = int(wl0.q_lens()[r]), int(wl0.kv_lens()[r])
-            n = (ql * kv - ql * (ql - 1) // 2) if m is None else int(m.sum())
-            flops += 4 * wl0.D * wl0.H_q * n
-        achieved = flops / (dom_ms * 1e-3) / 1e12
-        peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
-        roof = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None if args.param else NCU_TRAFFIC_BYTES.get(wl0.name), "useful_flops": flops,
-                "kernel_ms": dom_ms, "timing": dom_timing, "peak_source": peaks["source"] + " (sustained)"}
-
-    cpu = None
-    if world == 1 and not args.no_cpu_baseline:
-        tokens, dt, desc, threads = oracle_sample(wl0)
-        cpu = {"value": tokens / dt, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc,
-               "seconds": dt}
-
     ms_per_step = ms / args.steps
+    roof = roofline_of(wl0, name, info, ktimes, ms_per_step, peaks, args.gpus, clocks, sum(regions) * 1e-3)
+    cpu = None
+    if env.world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline_of(wl0, cpu_budget_s)
     alg_bytes = wl0.algorithmic_bytes()
-    line = {
-        "metric": METRIC, "value": total_tokens / (ms_per_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": wl0.dtype, "data": "synthetic",
-        "config": {"workload": wl0.name, "requests": wl0.R, "query_tokens": wl0.T, "heads": f"{wl0.H_q}/{wl0.H_kv}",
+    return {
+        "timed": True, "value": total_tokens / (ms_per_step * 1e-3), "unit": "tokens/s", "ms_per_step": ms_per_step,
+        "ms_per_step_min": min(regions) / args.steps, "ms_per_step_max": max(regions) / args.steps,
+        "regions": len(regions), "timed_seconds": sum(regions) * 1e-3, "dtype": wl0.dtype,
+        "config": {"workload": name, "requests": wl0.R, "query_tokens": wl0.T, "heads": f"{wl0.H_q}/{wl0.H_kv}",
                    "head_dim": wl0.D, "page_size": wl0.P, "pool_pages": wl0.num_pages, "l2": l2_note,
                    "plan_flags": args.flags, "launch": "cuda graph replay" if use_graph else "eager"},
         "hbm_gbs_step": alg_bytes["total"] / (ms_per_step * 1e-3) / 1e9,
@@ -546,14 +584,154 @@ def main():
         "plan_ms": statistics.median(plan_ms), "plan_first_ms": plan_first_ms, "plan_info": info,
         "kernel_ms": {k: (v[0] / v[1] if v[1] else 0.0) for k, v in ktimes.items()},
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
-        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        "gpu_launches": launches_per_step * args.steps * len(regions), "clocks": clocks,
     }
-    print(json.dumps(line))
-    for p in plans:
-        pie.pie_plan_destroy(p)
+
+
+def bench_next_dist(env, args):
+    """The sample stage next to the path (`get_next_dist`, Section 4.2 "Sample API"): one top-K truncated
+    distribution per request of the batched-decode workload - 64 rows over the 128,256-entry Llama-3
+    vocabulary, bf16 logits ~ N(0, 2.5) with a few tokens far ahead, K = 256.  Buffers rotate so that no
+    logits survive in L2 between steps."""
+    pie, torch = env.pie, env.torch
+    n, V, K = 64, 128256, 256
+    nbuf = 20                                                       # 20 x 16.4 MB > L2
+    g = torch.Generator(device="cuda").manual_seed(0x50494500 + 99 + 1000 * env.rank)
+    bufs = []
+    for _ in range(nbuf):
+        x = torch.randn(n, V, generator=g, device="cuda") * 2.5
+        x[:, ::977] += 9.0
+        bufs.append(x.to(torch.bfloat16))
+    ctx = pie.pie_create(4, 16, 4, 2, 64, "bf16", 4, 64, env.local)
+    ids = torch.empty(n, K, dtype=torch.int32, device="cuda")
+    probs = torch.empty(n, K, dtype=torch.float32, device="cuda")
+
+    def step(i):
+        pie.pie_get_next_dist(ctx, bufs[i % nbuf], K, ids, probs)
+
+    for i in range(args.warmup):
+        step(i)
+    env.barrier()
+    sampler = ClockSampler(env.local)
+    if env.rank == 0:
+        sampler.start()
+    regions = timed_regions(env, step, args.steps, args.min_seconds)
+    clocks = sampler.stop() if env.rank == 0 else None
+    ms = statistics.median(regions)
+    e2e = None
+    if not args.no_e2e:
+        host = [b.cpu().pin_memory() for b in bufs[:4]]
+        dev = torch.empty_like(bufs[0])
+        h_ids, h_probs = torch.empty(n, K, dtype=torch.int32).pin_memory(), torch.empty(n, K).pin_memory()
+        n_e2e = max(3, min(args.steps, 30))
+
+        def e2e_step(i):
+            dev.copy_(host[i % 4], non_blocking=True)
+            pie.pie_get_next_dist(ctx, dev, K, ids, probs)
+            h_ids.copy_(ids, non_blocking=True)
+            h_probs.copy_(probs, non_blocking=True)
+            torch.cuda.synchronize()
+
+        for i in range(3):
+            e2e_step(i)
+        env.barrier()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            e2e_step(i)
+        e2e_s = env.max_over_ranks(time.perf_counter() - t0)
+        e2e = {"value": env.world * n * n_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": n * V * 2,
+               "d2h_bytes_per_step": n * K * 8, "steps": n_e2e, "ms_per_step": e2e_s / n_e2e * 1e3,
+               "includes": "pinned H2D of the logits, get_next_dist, D2H of ids and probabilities"}
+    cpu = None
+    if env.rank == 0 and env.world == 1 and not args.no_cpu_baseline:
+        from oracle import pie_oracle as orc
+        rows = bufs[0][:8].cpu().view(torch.int16).numpy().view(np.uint16)
+        t0 = time.perf_counter()
+        orc.next_dist(rows, K)
+        dt = time.perf_counter() - t0
+        cpu = {"value": len(rows) / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+               "sample": f"first {len(rows)} of {n} rows", "seconds": dt}
     pie.pie_destroy(ctx)
-    if world > 1:
-        dist.destroy_process_group()
+    del bufs
+    torch.cuda.empty_cache()
+    if env.rank != 0:
+        return None
+    ms_per_step = ms / args.steps
+    alg = n * V * 2 + n * K * 8
+    peaks = load_peaks()
+    achieved = alg / (ms_per_step * 1e-3) / 1e9
+    return {
+        "timed": True, "value": env.world * n / (ms_per_step * 1e-3), "unit": "tokens/s", "ms_per_step": ms_per_step,
+        "ms_per_step_min": min(regions) / args.steps, "ms_per_step_max": max(regions) / args.steps,
+        "regions": len(regions), "timed_seconds": sum(regions) * 1e-3, "dtype": "bf16",
+        "config": {"workload": "next_dist", "rows": n, "vocab": V, "top_k": K,
+                   "l2": f"{nbuf} rotating logit buffers ({nbuf * n * V * 2 / 1e6:.0f} MB) > L2", "launch": "eager"},
+        "hbm_gbs_step": achieved, "algorithmic_bytes_step": {"logits": n * V * 2, "out": n * K * 8, "total": alg},
+        "kernel_ms": {"next_dist": ms_per_step},
+        "roofline": {"bound": "hbm", "kernel": "next_dist", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None, "traffic_source": "not captured",
+                     "algorithmic_bytes": alg, "kernel_ms": ms_per_step, "timing": "timed region / launches",
+                     "peak_source": peaks["source"]},
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * len(regions) * args.nd_launches, "clocks": clocks,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="all",
+                    help="one workload by name, or 'all' (default): every baseline configuration in one run")
+    ap.add_argument("--min-seconds", type=float, default=0.5, help="device time to collect per workload (regions of --steps steps are repeated)")
+    ap.add_argument("--flags", type=int, default=0, help="PIE_PLAN_* flags (debug / A-B runs)")
+    ap.add_argument("--opt", action="append", default=[], help="pie_set_option as K=V (tuning runs)")
+    ap.add_argument("--graph", type=int, default=0,
+                    help="1: replay one captured CUDA graph per step (measured: no gain, the loop is GPU bound), 0: eager launches")
+    ap.add_argument("--param", action="append", default=[], help="builder argument of the workload as key=value (shape sweeps)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    args.nd_launches = 1
+    if args.impl == "reference":
+        return run_reference(args)
+
+    env = Env()
+    # N > 1: every rank runs the headline batch (weak scaling); the other entries are single-GPU figures
+    names = (SUITE if env.world == 1 else [HEADLINE]) if args.workload == "all" else [args.workload]
+    entries = {}
+    t_start = time.perf_counter()
+    for name in names:
+        t0 = time.perf_counter()
+        head = name == names[0]
+        if name == "next_dist":
+            entry = bench_next_dist(env, args)
+        else:
+            entry = bench_workload(env, args, name, cpu_budget_s=15.0 if head else 4.0)
+        if entry is not None:
+            entry["wall_seconds"] = time.perf_counter() - t0
+            entries[name] = entry
+    if env.rank == 0:
+        head = entries[names[0]]
+        line = {"metric": METRIC, "value": head["value"], "unit": "tokens/s", "n_gpus": env.world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": head["dtype"], "data": "synthetic"}
+        for k in ("config", "hbm_gbs_step", "algorithmic_bytes_step", "useful_flops_step", "plan_ms", "plan_first_ms",
+                  "plan_info", "kernel_ms", "roofline", "cpu_baseline", "e2e", "gpu_launches", "clocks", "regions",
+                  "timed_seconds", "ms_per_step_min", "ms_per_step_max"):
+            if k in head:
+                line[k] = head[k]
+        if "shared_prefix_tree" in entries:
+            line["roofline_tensor"] = dict(entries["shared_prefix_tree"]["roofline"], workload="shared_prefix_tree")
+        if args.workload == "all":
+            if env.world == 1:
+                entries["tiny_fp32"] = {"timed": False, "note": "correctness-only configuration (fp32, 4 requests): covered by the parity tests"}
+            line["workloads"] = entries
+        line["wall_seconds"] = time.perf_counter() - t_start
+        print(json.dumps(line))
+    env.close()
 
 
 if __name__ == "__main__":

@@ -115,7 +115,9 @@ int ensure_buffer(pie_ctx* ctx, void** buf, size_t* cap, size_t need) {
   if (*buf) PIE_CUDA(ctx, cudaFree(*buf));
   *buf = nullptr;
   *cap = 0;
-  size_t want = std::max(need, (size_t)1 << 20);
+  // half as much again: a serving loop's batches grow step by step, and every regrowth is a cudaFree +
+  // cudaMalloc (a device-wide synchronisation of several hundred microseconds)
+  size_t want = std::max(need + need / 2, (size_t)1 << 20);
   PIE_CUDA(ctx, cudaMalloc(buf, want));
   *cap = want;
   return PIE_OK;

@@ -167,15 +167,18 @@ def _csr(lengths):
 
 
 def _assemble(name, seed, H_q, H_kv, D, P, dtype, num_pages, q_lens, kv_lens, masks,
-              placement=0, perm_stream=10, meta=None):
-    """Private pages for every request, taken in order from a seeded shuffle of the pool."""
+              placement=0, perm_stream=10, meta=None, perm_seed=None, page_offset=None):
+    """Private pages for every request, taken in order from a seeded shuffle of the pool:
+    the `placement`-th run of the batch's page count, or the run that starts at `page_offset`
+    of the shuffle seeded by `perm_seed` (several batches with different seeds in one pool)."""
     q_lens = np.asarray(q_lens, dtype=np.int64)
     kv_lens = np.asarray(kv_lens, dtype=np.int64)
     npages = (kv_lens + P - 1) // P
     total = int(npages.sum())
-    assert (placement + 1) * total <= num_pages, "pool too small for this placement"
-    perm = synth.permutation(seed, perm_stream, num_pages)
-    ids = perm[placement * total:(placement + 1) * total]
+    first = placement * total if page_offset is None else int(page_offset)
+    assert first + total <= num_pages, "pool too small for this placement"
+    perm = synth.permutation(seed if perm_seed is None else perm_seed, perm_stream, num_pages)
+    ids = perm[first:first + total]
     page_indptr = _csr(npages)
     owner = np.full(num_pages, -1, dtype=np.int64)
     logical = np.zeros(num_pages, dtype=np.int64)
@@ -214,11 +217,12 @@ def tiny_fp32(seed=SEED0 + 1, column_wise=False, P=16, dtype="f32", H_q=4, H_kv=
 
 # ------------------------------------------------------------------------------- config 2
 def batched_decode(seed=SEED0 + 2, R=64, lo=512, hi=4096, num_pages=65536, placement=0,
-                   H_q=32, H_kv=8, D=64, P=16, dtype="bf16"):
+                   H_q=32, H_kv=8, D=64, P=16, dtype="bf16", perm_seed=None, page_offset=None):
     """Single-token decodes over scattered pages, causal, one appended row per request."""
     kv = synth.uniform_ints(seed, 11, R, lo, hi)
     return _assemble("batched_decode", seed, H_q, H_kv, D, P, dtype, num_pages,
-                     np.ones(R, dtype=np.int64), kv, None, placement=placement)
+                     np.ones(R, dtype=np.int64), kv, None, placement=placement,
+                     perm_seed=perm_seed, page_offset=page_offset)
 
 
 # ------------------------------------------------------------------------------- config 3
@@ -349,7 +353,48 @@ def long_context_policy(seed=SEED0 + 5, R=256, lo=16384, hi=32768, sink=4, windo
                  "ntok": wl.last_page_len.astype(np.int32).copy()}
     wl.page_owner[dst] = 100000 + np.arange(R)
     wl.name = "long_context_policy"
+    wl.meta = {"sink": sink, "window": window, "keep_frac": keep_frac, "pages_in_lists": total}
     return wl
+
+
+def decode_loop(wl, n_steps, spare_pages):
+    """The batches of a decode loop that starts from the decode workload `wl` (every request one
+    query token): step s has every request s tokens longer than in `wl`, a request that crosses a
+    page boundary takes its next page from `spare_pages`, and application KV policies (the
+    long-context workload) are re-evaluated at the new length.  Returns one dict per step with
+    the CSR arrays (int32), the mask arrays of Workload.mask_bytes() and, for workloads with
+    page copies, the copy arrays of that step."""
+    assert (wl.q_lens() == 1).all(), "a decode loop needs single-token requests"
+    P, R = wl.P, wl.R
+    spare = [int(p) for p in spare_pages]
+    lists = [[int(p) for p in wl.pages_of(r)] for r in range(R)]
+    kv0 = wl.kv_lens()
+    policy = wl.masks is not None
+    if policy:
+        assert "window" in wl.meta, "only the sink / window / kept-pages policy can be re-evaluated"
+    steps = []
+    for s in range(n_steps):
+        kv = kv0 + s
+        for r in range(R):
+            need = (int(kv[r]) + P - 1) // P
+            while len(lists[r]) < need:
+                lists[r].append(spare.pop())
+        npages = np.array([len(x) for x in lists], dtype=np.int64)
+        b = {"qo_indptr": wl.qo_indptr.astype(np.int32), "page_indptr": _csr(npages),
+             "page_indices": np.fromiter((p for x in lists for p in x), dtype=np.int32, count=int(npages.sum())),
+             "last_page_len": (kv - (npages - 1) * P).astype(np.int32), "mask_indptr": None, "mask": None,
+             "copies": None}
+        if policy:
+            rows = [policy_mask(wl.seed, 22, r, int(kv[r]), P, wl.meta["sink"], wl.meta["window"],
+                                wl.meta["keep_frac"]) for r in range(R)]
+            ptr = np.zeros(R + 1, dtype=np.int64)
+            ptr[1:] = np.cumsum([len(x) for x in rows])
+            b["mask_indptr"], b["mask"] = ptr, np.concatenate(rows).astype(np.uint8)
+        if wl.copies is not None:
+            b["copies"] = dict(wl.copies, src=np.array([x[-1] for x in lists], dtype=np.int32),
+                               ntok=b["last_page_len"].copy())
+        steps.append(b)
+    return steps
 
 
 # ------------------------------------------------------------------------------- shared-prefix decode
