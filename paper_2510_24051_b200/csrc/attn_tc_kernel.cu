@@ -78,6 +78,22 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
                "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
                : "memory");
 }
+// Tiled TMA store of a 3-D box from shared memory (bulk async-group completion).
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map), "r"(src), "r"(x), "r"(y),
+               "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// every bulk store of this thread has finished READING shared memory / has completed altogether
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// barrier among the 128 threads of one softmax warpgroup (ids 1 and 2; 0 is __syncthreads)
+template <int ID>
+__device__ __forceinline__ void wg_sync() { asm volatile("bar.sync %0, 128;" ::"n"(ID) : "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 // 32-byte global store (the address must be 32-byte aligned)
 __device__ __forceinline__ void st_global_v8(void* p, const uint32_t* w) {
   asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]),
@@ -168,17 +184,20 @@ struct TcCfg {
   static constexpr int KVTILE = kTileN * D * 2;
   static constexpr int STAGES = D == 128 ? 2 : 4;
   static constexpr int NBAR = 4 * STAGES + 19;
-  static constexpr int SMEM = 2 * QTILE + 2 * STAGES * KVTILE + NBAR * 8 + 64;
+  static constexpr int OSLAB = kTileM * 128;           // output staging: one 64-column slab of a 128-row tile per warpgroup
+  static constexpr int SMEM = 2 * QTILE + 2 * STAGES * KVTILE + 2 * OSLAB + NBAR * 8 + 64;
 };
 
 template <int D, int P>
-__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qmap, const int kflags) {
+__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qmap,
+                                                              const __grid_constant__ CUtensorMap omap, const int kflags) {
   using C = TcCfg<D, P>;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* sQ = smem;
   uint8_t* sK = smem + 2 * C::QTILE;
   uint8_t* sV = sK + C::STAGES * C::KVTILE;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + C::STAGES * C::KVTILE);
+  uint8_t* sO = sV + C::STAGES * C::KVTILE;   // [2][128 rows][128 B], 128-byte swizzle like the Q tiles
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sO + 2 * C::OSLAB);
   uint64_t* k_full = bars;
   uint64_t* k_empty = k_full + C::STAGES;
   uint64_t* v_full = k_empty + C::STAGES;
@@ -196,6 +215,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool use_qmap = kflags & 1;      // Q tiles come through the tensor map
   const bool out_wide = kflags & 2;      // the output pointer allows 32-byte stores
+  const bool use_omap = kflags & 4;      // full output tiles leave through shared memory and a TMA store
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) {
       mbar_init(smem_u32(k_full + s), 1);
@@ -485,12 +505,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
     uint32_t my_items = 0;   // phase of o_done
     uint32_t s_ph = 0;       // bit h: phase of s_full[t][h]
     uint32_t n_arr = 0;      // p_full arrivals so far = PV groups of this Q tile issued or about to be
+    // The record of the next item is fetched before the wait for the last PV of the current one, so that its
+    // latency is not added to the gap between two items (where the tensor pipe is idle).
+    PieItem item_nxt = PieItem{};
+    if (it0 < it1) item_nxt = p.items[it0];
     for (int it = it0; it < it1; ++it) {
-      const PieItem item = p.items[it];
+      const PieItem item = item_nxt;
       const int npages = item.page_end - item.page_begin;
       const int nhalf = (npages + C::PPH - 1) / C::PPH;
       const int nt = item.nrows > kTileM ? 2 : 1;
-      if (t >= nt) continue;
+      if (t >= nt) {
+        if (it + 1 < it1) item_nxt = p.items[it + 1];
+        continue;
+      }
       const int gr = item.row0 + t * kTileM + rho;
       const bool valid = gr < item.row0 + item.nrows;
       const int tok = valid ? gr / p.G : 0;
@@ -687,60 +714,122 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
         const int n_lean = min(nhalf, max(0, clean_halves - 2));   // (the look-ahead of the general loop starts two halves early)
         for (int i = 0; i < n_lean; ++i) do_half(i, std::false_type{});
         for (int i = n_lean; i < nhalf; ++i) do_half(i, std::true_type{});
+        if (it + 1 < it1) item_nxt = p.items[it + 1];
         mbar_wait(smem_u32(o_done + t), my_items & 1, p.status);
         ++my_items;
         tc_fence_after();
       }
 
+      if (nhalf == 0 && it + 1 < it1) item_nxt = p.items[it + 1];
       // ---- epilogue: normalise, store
       const bool live = m_ref != kNegInf && l_sum > 0.f;   // a row with no allowed position: O = 0, LSE = -inf
       const float inv = live ? 1.f / l_sum : 0.f;
       const float lse = live ? (m_ref + log2f(l_sum)) * kLn2 : kNegInf;
+      // A full tile of final rows leaves through shared memory: every thread converts its row, 64 columns at a
+      // time, into the warpgroup's staging slab (the swizzled image of the box 64 dims x G heads x 128 / G tokens
+      // of the output tensor) and one thread hands the slab to a TMA store.  The accumulator is free for the next
+      // item as soon as it has been read into registers, and the stores to global memory run while the warpgroup
+      // is already in the next item's softmax - the epilogue sits between the last MMA of an item and the first
+      // of the next, so every cycle of it is idle tensor-pipe time.  (All conditions are uniform over the
+      // warpgroup: the barriers below always see their 128 threads.)
+      const bool via_tma = use_omap && nhalf > 0 && item.partial_slot < 0 && item.nrows >= (t + 1) * kTileM;
+      if (via_tma) {
+        const uint32_t stg = smem_u32(sO + t * C::OSLAB) + rho * 128;
+        const bool lead = (warp & 3) == 0;
+        const int tok0 = item.q_start + (item.row0 + t * kTileM) / p.G;
+        auto sync_wg = [&]() {
+          if (t == 0) wg_sync<1>();
+          else wg_sync<2>();
+        };
 #pragma unroll
-      for (int c0 = 0; c0 < D; c0 += 32) {
-        uint32_t o[32];
-        if (nhalf > 0) {
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          uint32_t o[32];
           tmem_ld32(tO + c0, o);
           tmem_wait_ld();
-        } else {
+          if (c0 + 32 == D) {   // O_t is in registers: the next item's PV may overwrite it
+            tc_fence_before();
+            mbar_arrive(smem_u32(o_free + t));
+          }
+          uint32_t w[16];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) o[c] = 0u;
-        }
-        if (valid) {
-          if (item.partial_slot < 0) {
-            // 32-byte stores: every thread writes its own row, so the store path is bound by the number
-            // of (thread, instruction) pairs, not by bytes
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D + c0;
-            uint32_t w[16];
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) w[c >> 1] = pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
-            if (out_wide) {
-              st_global_v8(dst, w);
-              st_global_v8(dst + 16, w + 8);
-            } else {
-#pragma unroll
-              for (int c = 0; c < 16; c += 4) reinterpret_cast<uint4*>(dst)[c >> 2] = make_uint4(w[c], w[c + 1], w[c + 2], w[c + 3]);
+          for (int c = 0; c < 32; c += 2) w[c >> 1] = pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+          if ((c0 & 63) == 0) {   // the slab's previous store must have read it before it is overwritten
+            if (lead) {
+              if (elect_one()) bulk_wait_read();
+              __syncwarp();
             }
-          } else {
-            float* dst = p.ws_o + ((int64_t)item.partial_slot * 256 + (gr - item.row0)) * D + c0;
+            sync_wg();
+          }
 #pragma unroll
-            for (int c = 0; c < 32; c += 8) {
-              uint32_t w[8];
-#pragma unroll
-              for (int k = 0; k < 8; ++k) w[k] = __float_as_uint(__uint_as_float(o[c + k]) * inv);
-              st_global_v8(dst + c, w);
+          for (int k = 0; k < 4; ++k) {
+            const int ch = ((c0 & 63) >> 3) + k;   // 16-byte chunk of the row inside the slab
+            st_shared_v4(stg + ((ch ^ (rho & 7)) << 4), w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
+          }
+          if ((c0 & 63) == 32) {
+            fence_async_smem();
+            sync_wg();
+            if (lead) {
+              if (elect_one()) {
+                tma_store_3d(&omap, smem_u32(sO + t * C::OSLAB), c0 & ~63, item.kv_head * p.G, tok0);
+                bulk_commit();
+              }
+              __syncwarp();
             }
           }
         }
+        p.lse[oi] = lse;
+      } else {
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          uint32_t o[32];
+          if (nhalf > 0) {
+            tmem_ld32(tO + c0, o);
+            tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) o[c] = 0u;
+          }
+          if (valid) {
+            if (item.partial_slot < 0) {
+              // 32-byte stores: every thread writes its own row, so the store path is bound by the number
+              // of (thread, instruction) pairs, not by bytes
+              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D + c0;
+              uint32_t w[16];
+#pragma unroll
+              for (int c = 0; c < 32; c += 2) w[c >> 1] = pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+              if (out_wide) {
+                st_global_v8(dst, w);
+                st_global_v8(dst + 16, w + 8);
+              } else {
+#pragma unroll
+                for (int c = 0; c < 16; c += 4) reinterpret_cast<uint4*>(dst)[c >> 2] = make_uint4(w[c], w[c + 1], w[c + 2], w[c + 3]);
+              }
+            } else {
+              float* dst = p.ws_o + ((int64_t)item.partial_slot * 256 + (gr - item.row0)) * D + c0;
+#pragma unroll
+              for (int c = 0; c < 32; c += 8) {
+                uint32_t w[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) w[k] = __float_as_uint(__uint_as_float(o[c + k]) * inv);
+                st_global_v8(dst + c, w);
+              }
+            }
+          }
+        }
+        if (valid) {
+          if (item.partial_slot < 0) p.lse[oi] = lse;
+          else p.ws_lse[(int64_t)item.partial_slot * 256 + (gr - item.row0)] = lse;
+        }
+        if (nhalf > 0) {
+          tc_fence_before();
+          mbar_arrive(smem_u32(o_free + t));
+        }
       }
-      if (valid) {
-        if (item.partial_slot < 0) p.lse[oi] = lse;
-        else p.ws_lse[(int64_t)item.partial_slot * 256 + (gr - item.row0)] = lse;
-      }
-      if (nhalf > 0) {
-        tc_fence_before();
-        mbar_arrive(smem_u32(o_free + t));
-      }
+    }
+    // the last output tiles must have left shared memory (and reached global memory) before the block ends
+    if ((warp & 3) == 0) {
+      if (elect_one()) bulk_wait_all();
+      __syncwarp();
     }
   }
 
@@ -776,7 +865,7 @@ static EncodeTiledFn encode_tiled_fn() {
 // Tensor map of Q [tokens][q heads][D] (bf16) whose box is one Q tile: 64 dims x G heads x 128/G
 // tokens, 128-byte swizzle.  Returns false when the shape does not fit (128 not a multiple of G,
 // unaligned pointer): the kernel then loads Q with plain asynchronous copies.
-static bool make_q_map(const pie_ctx* ctx, const void* q, int64_t n_tokens, int G, CUtensorMap* map) {
+static bool make_q_map(const pie_ctx* ctx, const void* q, int64_t n_tokens, int G, CUtensorMap* map) {   // (also the map of the output tensor: same shape)
   const int D = ctx->cfg.head_dim, Hq = ctx->cfg.num_q_heads;
   if (G <= 0 || kTileM % G != 0 || n_tokens <= 0 || (reinterpret_cast<uintptr_t>(q) & 15) != 0) return false;
   EncodeTiledFn enc = encode_tiled_fn();
@@ -797,10 +886,12 @@ static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_toke
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
     ctx->tc_configured = true;
   }
-  CUtensorMap qmap;
+  CUtensorMap qmap, omap;
   memset(&qmap, 0, sizeof(qmap));
-  const int kflags = (make_q_map(ctx, p.q, n_tokens, p.G, &qmap) ? 1 : 0) | ((reinterpret_cast<uintptr_t>(p.out) & 31) == 0 ? 2 : 0);
-  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3(kThreads), C::SMEM, s, p, qmap, kflags));
+  memset(&omap, 0, sizeof(omap));
+  const int kflags = (make_q_map(ctx, p.q, n_tokens, p.G, &qmap) ? 1 : 0) | ((reinterpret_cast<uintptr_t>(p.out) & 31) == 0 ? 2 : 0) |
+                     (make_q_map(ctx, p.out, n_tokens, p.G, &omap) ? 4 : 0);
+  PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(grid), dim3(kThreads), C::SMEM, s, p, qmap, omap, kflags));
   return PIE_OK;
 }
 
