@@ -177,7 +177,7 @@ typedef struct pie_batch_desc {
 
 enum {
   PIE_PLAN_FORCE_SIMPLE = 1u,   /* run every request through the plain CUDA-core kernel   */
-  PIE_PLAN_NO_TENSOR_TILES = 2u, /* keep prefill / tree requests off the tcgen05 tile path */
+  PIE_PLAN_NO_TENSOR_TILES = 2u, /* keep prefill / tree requests off the tcgen05 tile path (ignored with 8-token pages) */
   PIE_PLAN_NO_CASCADE = 4u,     /* never attend a shared prefix once for a group of requests */
   PIE_PLAN_CASCADE_ALWAYS = 8u, /* cascade every shared prefix, however small the saving (tests, tuning) */
   PIE_PLAN_MASK_BITS = 16u      /* `mask` holds bits, not bool bytes: for a request with a mask, q_len rows of

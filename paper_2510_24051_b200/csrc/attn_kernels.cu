@@ -103,50 +103,73 @@ __device__ __forceinline__ void rows_init(RowState<D>& st, const AttnParams& p, 
   for (int nb = 0; nb < D / 8; ++nb) st.o[nb][0] = st.o[nb][1] = st.o[nb][2] = st.o[nb][3] = 0.f;
 }
 
-// Attend the warp's rows to one KvPage block resident in shared memory (K block then V block,
-// each [slab][slot][128 B] with the 16-byte chunks XOR-swizzled by slot & 7).
-template <int D, int P>
-__device__ __forceinline__ void page_compute(RowState<D>& st, uint8_t* stage, const PieReq& rq, uint32_t lpf,
-                                             float scale_log2, int lane) {
-  constexpr int KSTEPS = D / 16, SUBS = P / 16, BLK = P * D * 2, SLAB = P * 128;
+// Attend the warp's rows to one visit resident in shared memory: PPV pages, each a K block then a V
+// block ([slab][slot][128 B] with the 16-byte chunks XOR-swizzled by slot & 7), handled in steps of 16
+// tokens (one m16n8k16 k-step of P V).  Pages of 16 or 32 tokens are one visit each; pages of 8 tokens
+// come in pairs, so that a step is filled by two pages (lpf[i] = logical page | needs-mask flag of page i,
+// 0xFFFFFFFF when the visit has no page i: the odd page at the end of a piece).
+#define PIE_NO_PAGE 0xFFFFFFFFu
+template <int D, int P, int PPV>
+__device__ __forceinline__ void visit_compute(RowState<D>& st, uint8_t* stage, const PieReq& rq, const uint32_t* lpf,
+                                              float scale_log2, int lane) {
+  constexpr int KSTEPS = D / 16, VT = P * PPV, SUBS = VT / 16, BLK = P * D * 2, SLAB = P * 128, PAGE = 2 * BLK;
+  constexpr int PIECES = P >= 16 ? 1 : 16 / P, PW = 16 / PIECES;   // a 16-token step is made of PIECES runs of PW tokens, each inside one page
+  static_assert(VT % 16 == 0, "a visit is a whole number of 16-token steps");
   const int cpair = (lane & 3) * 2;
-  const int lp = (int)(lpf & ~PIE_KEPT_NEEDS_MASK);
-  const bool needs_mask = (lpf & PIE_KEPT_NEEDS_MASK) != 0;
-  const uint32_t kbase = smem_u32(stage), vbase = kbase + BLK;
+  const uint32_t sbase = smem_u32(stage);
 
-  if (lp == rq.last_logical && rq.last_page_len < P) {
-    // slots past the end of the context may hold anything: clear their V rows so that a zero
-    // probability times a NaN bit pattern cannot leak into the output
-    constexpr int CH = D * 2 / 16;
-    const int nz = (P - rq.last_page_len) * CH;
-    for (int c = lane; c < nz; c += 32) {
-      const int t = rq.last_page_len + c / CH, ch = c % CH;
-      *reinterpret_cast<uint4*>(stage + BLK + pie_chunk_offset(SLAB, t, ch)) = make_uint4(0, 0, 0, 0);
+#pragma unroll
+  for (int i = 0; i < PPV; ++i) {
+    // slots past the end of the context (and a page the visit does not have) may hold anything: clear their V
+    // rows so that a zero probability times a NaN bit pattern cannot leak into the output
+    int first_bad = P;
+    if (lpf[i] == PIE_NO_PAGE) first_bad = 0;
+    else if ((int)(lpf[i] & ~PIE_KEPT_NEEDS_MASK) == rq.last_logical && rq.last_page_len < P) first_bad = rq.last_page_len;
+    if (first_bad < P) {
+      constexpr int CH = D * 2 / 16;
+      const int nz = (P - first_bad) * CH;
+      for (int c = lane; c < nz; c += 32) {
+        const int t = first_bad + c / CH, ch = c % CH;
+        *reinterpret_cast<uint4*>(stage + i * PAGE + BLK + pie_chunk_offset(SLAB, t, ch)) = make_uint4(0, 0, 0, 0);
+      }
+      // these generic-proxy writes must be ordered before the bulk copy that later refills the stage
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
     }
-    // these generic-proxy writes must be ordered before the bulk copy that later refills the stage
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
   }
   if (!st.any_rows) return;
 
 #pragma unroll
   for (int sub = 0; sub < SUBS; ++sub) {
-    const int j0 = lp * P + sub * 16;
-    uint32_t bits[2] = {0xFFFFu, 0xFFFFu};
-    if (needs_mask) {
+    uint32_t bits[2] = {0u, 0u};
+    bool needs_mask = false;
 #pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        if (!st.valid[r]) bits[r] = 0;
-        else if (st.explicit_mask) bits[r] = (__ldg(st.mrow[r] + (j0 >> 5)) >> (j0 & 31)) & 0xFFFFu;
-        else bits[r] = st.lim[r] >= j0 + 15 ? 0xFFFFu : (st.lim[r] < j0 ? 0u : ((1u << (st.lim[r] - j0 + 1)) - 1u));
+    for (int pc = 0; pc < PIECES; ++pc) {
+      const int pg = (sub * 16 + pc * PW) / P, off = (sub * 16 + pc * PW) % P;
+      const uint32_t l = lpf[pg], full = (1u << PW) - 1u;
+      uint32_t piece[2] = {full, full};
+      if (l == PIE_NO_PAGE) {
+        needs_mask = true;
+        piece[0] = piece[1] = 0u;
+      } else if (l & PIE_KEPT_NEEDS_MASK) {
+        needs_mask = true;
+        const int j0 = (int)(l & ~PIE_KEPT_NEEDS_MASK) * P + off;
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          if (!st.valid[r]) piece[r] = 0u;
+          else if (st.explicit_mask) piece[r] = (__ldg(st.mrow[r] + (j0 >> 5)) >> (j0 & 31)) & full;
+          else piece[r] = st.lim[r] >= j0 + PW - 1 ? full : (st.lim[r] < j0 ? 0u : ((1u << (st.lim[r] - j0 + 1)) - 1u));
+        }
       }
-      if (__all_sync(0xFFFFFFFFu, (bits[0] | bits[1]) == 0)) continue;  // nothing visible to this warp
+      bits[0] |= piece[0] << (pc * PW);
+      bits[1] |= piece[1] << (pc * PW);
     }
+    if (needs_mask && __all_sync(0xFFFFFFFFu, (bits[0] | bits[1]) == 0)) continue;  // nothing visible to this warp
     // ---- S = Q K^T for 16 tokens
     float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     {
-      const int t = sub * 16 + ((lane >> 4) << 3) + (lane & 7);
-      const uint32_t rowaddr = kbase + t * 128;
+      const int t = sub * 16 + ((lane >> 4) << 3) + (lane & 7);   // token of the visit whose K row this lane addresses
+      const uint32_t rowaddr = sbase + (t / P) * PAGE + (t % P) * 128;
       const int csel = (lane >> 3) & 1;
 #pragma unroll
       for (int ks = 0; ks < KSTEPS; ++ks) {
@@ -205,7 +228,7 @@ __device__ __forceinline__ void page_compute(RowState<D>& st, uint8_t* stage, co
     // ---- O += P V
     {
       const int t = sub * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
-      const uint32_t rowaddr = vbase + t * 128;
+      const uint32_t rowaddr = sbase + (t / P) * PAGE + BLK + (t % P) * 128;
       const int csel = lane >> 4;
 #pragma unroll
       for (int db = 0; db < KSTEPS; ++db) {
@@ -217,6 +240,13 @@ __device__ __forceinline__ void page_compute(RowState<D>& st, uint8_t* stage, co
       }
     }
   }
+}
+
+// One page per visit (pages of 16 or 32 tokens).
+template <int D, int P>
+__device__ __forceinline__ void page_compute(RowState<D>& st, uint8_t* stage, const PieReq& rq, uint32_t lpf,
+                                             float scale_log2, int lane) {
+  visit_compute<D, P, 1>(st, stage, rq, &lpf, scale_log2, lane);
 }
 
 // Normalise and store the warp's rows: final bf16 output + LSE, or an fp32 partial for the merge.
@@ -321,9 +351,11 @@ __device__ __forceinline__ void rows_merge_store(RowState<D>& st, const AttnPara
 // that neither the atomic nor the chunk record is ever waited for.
 template <int D, int P, int NW, int DEPTH>
 struct SplitCfg {
-  static constexpr int STAGE = 2 * P * D * 2;
+  static constexpr int PPV = P == 8 ? 2 : 1;   // pages per visit: 8-token pages are handled in pairs (16 tokens fill an MMA step)
+  static constexpr int PAGE = 2 * P * D * 2;   // K block + V block of one (page, kv head)
+  static constexpr int STAGE = PPV * PAGE;
   static constexpr int QUEUE = 8;  // chunk ids a warp has started fetching but not finished (<= DEPTH + 2)
-  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * 16 + NW * QUEUE * 4 + PIE_MAX_LOCAL_GROUPS * 4 + 64;
+  static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * (8 + 8 * PPV) + NW * QUEUE * 4 + PIE_MAX_LOCAL_GROUPS * 4 + 64;
 };
 
 template <int D, int P, int NW, int DEPTH>
@@ -334,10 +366,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   uint8_t* stages = smem + warp * DEPTH * C::STAGE;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + NW * DEPTH * C::STAGE) + warp * DEPTH;
-  volatile uint32_t* meta = reinterpret_cast<uint32_t*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 8) + warp * DEPTH;
-  volatile int* meta_phys = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 12) + warp * DEPTH;
-  volatile int* queue = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 16) + warp * C::QUEUE;
-  int* local_cnt = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 16 + NW * C::QUEUE * 4);  // block-local merge groups
+  constexpr int PPV = C::PPV;
+  volatile uint32_t* meta = reinterpret_cast<uint32_t*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * 8) + warp * DEPTH * PPV;
+  volatile int* meta_phys = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * (8 + 4 * PPV)) + warp * DEPTH * PPV;
+  volatile int* queue = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * (8 + 8 * PPV)) + warp * C::QUEUE;
+  int* local_cnt = reinterpret_cast<int*>(smem + NW * DEPTH * C::STAGE + NW * DEPTH * (8 + 8 * PPV) + NW * C::QUEUE * 4);  // block-local merge groups
   if (threadIdx.x < PIE_MAX_LOCAL_GROUPS) local_cnt[threadIdx.x] = 0;
   __syncthreads();   // the only block-wide sync of the kernel (counters are zero before any warp counts itself in)
   if (!p.late_trigger) pie_pdl_launch_dependents();
@@ -405,12 +438,12 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
     if (!pf_live || nx_idx >= 0 || exhausted) return;
     const int left = pf_end - pf_k;
     if (!grab_pending) {
-      if (left <= 4) {
+      if (left <= 4 * PPV) {
         if (own_next < own_end) grabbed = own_next++;
         else if (lane == 0) grabbed = atomicAdd(p.work_ctr, 1);
         grab_pending = true;
       }
-    } else if (left <= 2) {
+    } else if (left <= 2 * PPV) {
       const int idx = __shfl_sync(0xFFFFFFFFu, grabbed, 0);
       grab_pending = false;
       load_next_record(idx);
@@ -419,38 +452,58 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
   // (The stage was last read with ldmatrix by this same warp, and those reads have returned
   // their registers before the warp gets here, so the overwrite needs no proxy fence; the one
   // generic-proxy write to a stage, clearing rows of a last page, fences for itself.)
-  auto issue = [&](int n, int2 rec, int head) {
+  auto issue = [&](int n, const int2* rec, int cnt, int head) {   // one visit: cnt <= PPV pages
     const uint32_t s = n % DEPTH;
-    meta[s] = (uint32_t)rec.y;  // logical page | needs-mask flag, read back by the warp after the wait
-    meta_phys[s] = rec.x;       // physical page (the fused append writes its row back to it)
-    mbar_expect_tx(smem_u32(full_bar + s), C::STAGE);
-    bulk_g2s(smem_u32(stages + s * C::STAGE), p.pool + ((int64_t)rec.x * p.n_kv_heads + head) * C::STAGE, C::STAGE,
-             smem_u32(full_bar + s));
+#pragma unroll
+    for (int i = 0; i < PPV; ++i) {
+      meta[s * PPV + i] = i < cnt ? (uint32_t)rec[i].y : PIE_NO_PAGE;  // logical page | needs-mask flag, read back by the warp after the wait
+      meta_phys[s * PPV + i] = rec[i].x;                                // physical page (the fused append writes its row back to it)
+    }
+    mbar_expect_tx(smem_u32(full_bar + s), cnt * C::PAGE);
+#pragma unroll
+    for (int i = 0; i < PPV; ++i)
+      if (i < cnt)
+        bulk_g2s(smem_u32(stages + s * C::STAGE + i * C::PAGE), p.pool + ((int64_t)rec[i].x * p.n_kv_heads + head) * C::PAGE, C::PAGE,
+                 smem_u32(full_bar + s));
+  };
+  auto load_visit = [&](int2* rec) {   // records of the visit at the prefetch cursor; returns its page count
+    const int cnt = min(PPV, pf_end - pf_k);
+#pragma unroll
+    for (int i = 0; i < PPV; ++i) {
+      rec[i] = make_int2(0, 0);
+      if (i < cnt) rec[i] = __ldg(&p.kept[pf_k + i]);
+    }
+    return cnt;
   };
 
   // Prologue.  The plan arrays are not written by the kernels that precede this one in the stream, so
   // a warp with a fixed share walks its first DEPTH page records BEFORE waiting for those kernels:
   // under programmatic dependent launch this runs while the previous kernel drains.  The work
   // counter, the pool, Q and every output are touched only after the wait.
-  int2 pre_rec[DEPTH];
+  int2 pre_rec[DEPTH][PPV];
   int n_pre = 0;
   if (own_next < own_end) {
     pf_settle();  // enters the first item of the fixed share (no counter access)
-    n_pre = min(DEPTH, pf_end - pf_k);
+    n_pre = min(DEPTH, (pf_end - pf_k + PPV - 1) / PPV);
 #pragma unroll
     for (int i = 0; i < DEPTH; ++i)
-      if (i < n_pre) pre_rec[i] = __ldg(&p.kept[pf_k + i]);
+#pragma unroll
+      for (int j = 0; j < PPV; ++j) {
+        pre_rec[i][j] = make_int2(0, 0);
+        if (i < n_pre && pf_k + i * PPV + j < pf_end) pre_rec[i][j] = __ldg(&p.kept[pf_k + i * PPV + j]);
+      }
   }
   pie_pdl_wait();  // the append (and whatever produced Q) is complete from here on
 #pragma unroll
   for (int i = 0; i < DEPTH; ++i)
-    if (i < n_pre && lane == 0) issue(i, pre_rec[i], pf_head);
-  pf_k += n_pre;
+    if (i < n_pre && lane == 0) issue(i, pre_rec[i], min(PPV, pf_end - pf_k - i * PPV), pf_head);
+  pf_k = min(pf_k + n_pre * PPV, pf_end);
   pf_settle();  // (may take from the counter now)
   for (int n = n_pre; n < DEPTH && pf_live; ++n) {  // rest of the ring
-    const int2 rec = __ldg(&p.kept[pf_k]);
-    if (lane == 0) issue(n, rec, pf_head);
-    ++pf_k;
+    int2 rec[PPV];
+    const int cnt = load_visit(rec);
+    if (lane == 0) issue(n, rec, cnt, pf_head);
+    pf_k += cnt;
     pf_lookahead();
     pf_settle();
   }
@@ -483,28 +536,34 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
                                                        ((int64_t)item.q_start * p.n_kv_heads + item.kv_head) * (D * 2)) + (lane % CH));
     RowState<D> st;
     rows_init<D>(st, p, item, rq, item.row0, lane);
-    for (int k = item.page_begin; k < item.page_end; ++k, ++n) {
+    for (int k = item.page_begin; k < item.page_end; k += PPV, ++n) {
       const uint32_t s = n % DEPTH, ph = (n / DEPTH) & 1;
-      int2 rec_next = make_int2(0, 0);
-      if (pf_live) rec_next = __ldg(&p.kept[pf_k]);  // latency hides behind the wait
+      int2 rec_next[PPV];
+      int cnt_next = 0;
+      if (pf_live) cnt_next = load_visit(rec_next);  // latency hides behind the wait
       mbar_wait(smem_u32(full_bar + s), ph, p.status);
-      const uint32_t lpf = meta[s];
-      if (do_append && (int)(lpf & ~PIE_KEPT_NEEDS_MASK) == item.last_logical) {
-        if (lane < 2 * CH) {
-          const int off = (lane < CH ? 0 : C::STAGE / 2) + pie_chunk_offset(P * 128, item.last_page_len - 1, lane % CH);
-          *reinterpret_cast<uint4*>(stages + s * C::STAGE + off) = new_chunk;
-          const int phys = meta_phys[s];
-          *reinterpret_cast<uint4*>(const_cast<uint8_t*>(p.pool) + ((int64_t)phys * p.n_kv_heads + item.kv_head) * C::STAGE + off) = new_chunk;
+      uint32_t lpf[PPV];
+#pragma unroll
+      for (int i = 0; i < PPV; ++i) lpf[i] = meta[s * PPV + i];
+#pragma unroll
+      for (int i = 0; i < PPV; ++i) {
+        if (do_append && lpf[i] != PIE_NO_PAGE && (int)(lpf[i] & ~PIE_KEPT_NEEDS_MASK) == item.last_logical) {
+          if (lane < 2 * CH) {
+            const int off = (lane < CH ? 0 : C::PAGE / 2) + pie_chunk_offset(P * 128, item.last_page_len - 1, lane % CH);
+            *reinterpret_cast<uint4*>(stages + s * C::STAGE + i * C::PAGE + off) = new_chunk;
+            const int phys = meta_phys[s * PPV + i];
+            *reinterpret_cast<uint4*>(const_cast<uint8_t*>(p.pool) + ((int64_t)phys * p.n_kv_heads + item.kv_head) * C::PAGE + off) = new_chunk;
+          }
+          // the generic-proxy write must be ordered before the bulk copy that later refills the stage
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
         }
-        // the generic-proxy write must be ordered before the bulk copy that later refills the stage
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
       }
-      page_compute<D, P>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
+      visit_compute<D, P, PPV>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
       __syncwarp();
       if (pf_live) {
-        if (lane == 0) issue(n + DEPTH, rec_next, pf_head);
-        ++pf_k;
+        if (lane == 0) issue(n + DEPTH, rec_next, cnt_next, pf_head);
+        pf_k += cnt_next;
         pf_lookahead();
         pf_settle();
       }
@@ -821,8 +880,8 @@ int launch_tiles(pie_ctx* ctx, const AttnParams& p, int grid, cudaStream_t s) {
 
 bool pie_split_supported(const pie_ctx* ctx) {
   const pie_config& c = ctx->cfg;
-  return c.dtype == PIE_DTYPE_BF16 && (c.page_size == 16 || c.page_size == 32) && (c.head_dim == 64 || c.head_dim == 128) &&
-         ctx->G <= 16;
+  return c.dtype == PIE_DTYPE_BF16 && (c.page_size == 8 || c.page_size == 16 || c.page_size == 32) &&
+         (c.head_dim == 64 || c.head_dim == 128) && ctx->G <= 16;
 }
 
 // Warps per block of the split-KV kernel (the planner sizes its shares with this).
@@ -837,6 +896,8 @@ int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, const vo
   p.v_new = v_new;
   const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size, n = plan->split.grid, ni = (int)plan->split.items.size();
   // ring depth: about 192 KB of copies in flight per SM
+  if (D == 64 && P == 8) return launch_split<64, 8, 8, 6>(ctx, p, ni, n, s);     // (a visit is two pages: the same 4 / 8 KB as with 16-token pages)
+  if (D == 128 && P == 8) return launch_split<128, 8, 8, 3>(ctx, p, ni, n, s);
   if (D == 64 && P == 16) return launch_split<64, 16, 8, 6>(ctx, p, ni, n, s);
   if (D == 128 && P == 16) return launch_split<128, 16, 8, 3>(ctx, p, ni, n, s);
   if (D == 64 && P == 32) return launch_split<64, 32, 8, 3>(ctx, p, ni, n, s);

@@ -281,24 +281,27 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
         mbar_wait(smem_u32(v_empty + s), ph ^ 1, p.status);
         unsigned hit = 0;
         if (ragged) hit = __ballot_sync(0xFFFFFFFFu, lane < nvalid && (int)((uint32_t)rec.y & ~PIE_KEPT_NEEDS_MASK) == item.last_logical);
-        const uint32_t vbar = hit ? smem_u32(v_land) : smem_u32(v_full + s);
+        const bool odd_end = P == 8 && (nvalid & 1);   // half of the tile's last 16-token step has no page
+        const uint32_t vbar = (hit || odd_end) ? smem_u32(v_land) : smem_u32(v_full + s);
         if (lane == 0) mbar_expect_tx(vbar, nvalid * C::BLK);
         __syncwarp();
         if (lane < ncopies)
           bulk_g2s(smem_u32(sV + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
                    base + (int64_t)ph_pg * p.page_bytes + C::BLK + sl * C::SLAB_PAGE, C::SLAB_PAGE, vbar);
         __syncwarp();
-        if (hit) {
+        if (hit || odd_end) {
           mbar_wait(smem_u32(v_land), land_cnt & 1, p.status);
           ++land_cnt;
-          const int pgi = __ffs(hit) - 1;
           constexpr int CH = D * 2 / 16;
-          const int nz = (P - item.last_page_len) * CH;
-          for (int c = lane; c < nz; c += 32) {
-            const int tkn = pgi * P + item.last_page_len + c / CH, ch = c % CH;
-            *reinterpret_cast<uint4*>(sV + s * C::KVTILE + (ch >> 3) * C::SLAB_TILE + tkn * 128 + (((ch & 7) ^ (tkn & 7)) << 4)) =
-                make_uint4(0, 0, 0, 0);
-          }
+          auto clear_rows = [&](int first, int n) {   // V rows [first, first + n) of the tile
+            for (int c = lane; c < n * CH; c += 32) {
+              const int tkn = first + c / CH, ch = c % CH;
+              *reinterpret_cast<uint4*>(sV + s * C::KVTILE + (ch >> 3) * C::SLAB_TILE + tkn * 128 + (((ch & 7) ^ (tkn & 7)) << 4)) =
+                  make_uint4(0, 0, 0, 0);
+            }
+          };
+          if (hit) clear_rows((__ffs(hit) - 1) * P + item.last_page_len, P - item.last_page_len);
+          if (odd_end) clear_rows(nvalid * P, P);
           fence_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(v_full + s));
@@ -340,7 +343,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
         if (npages == 0) continue;  // the softmax warpgroups write zeros / -inf on their own
         const int ntiles = (npages + C::PPT - 1) / C::PPT;
         const int nhalf = (npages + C::PPH - 1) / C::PPH;           // halves of the item
-        const int last_cols = (npages - (nhalf - 1) * C::PPH) * P;  // columns of the last half
+        // columns of the last half, as a whole number of 16-token MMA steps (with 8-token pages the last step may
+        // be half empty: its scores are masked off like any column past the end, its V rows are cleared)
+        const int last_cols = ((npages - (nhalf - 1) * C::PPH) * P + 15) & ~15;
         const int nt = nrows > kTileM ? 2 : 1;
         // Phase of q_full / o_free of Q tile t: bit t of item_ph counts the items the tile took part in.
         const uint32_t ph_item = item_ph;
@@ -843,7 +848,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
 }  // namespace
 bool pie_tc_supported(const pie_ctx* ctx) {
   const pie_config& c = ctx->cfg;
-  return c.dtype == PIE_DTYPE_BF16 && (c.page_size == 16 || c.page_size == 32) && (c.head_dim == 64 || c.head_dim == 128);
+  return c.dtype == PIE_DTYPE_BF16 && (c.page_size == 8 || c.page_size == 16 || c.page_size == 32) &&
+         (c.head_dim == 64 || c.head_dim == 128);
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda)
@@ -897,6 +903,8 @@ static int launch_tc(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_toke
 
 int pie_launch_tc_tiles(pie_ctx* ctx, const AttnParams& p, int grid, int64_t n_tokens, cudaStream_t s) {
   const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size;
+  if (D == 128 && P == 8) return launch_tc<128, 8>(ctx, p, grid, n_tokens, s);
+  if (D == 64 && P == 8) return launch_tc<64, 8>(ctx, p, grid, n_tokens, s);
   if (D == 128 && P == 16) return launch_tc<128, 16>(ctx, p, grid, n_tokens, s);
   if (D == 64 && P == 16) return launch_tc<64, 16>(ctx, p, grid, n_tokens, s);
   if (D == 128 && P == 32) return launch_tc<128, 32>(ctx, p, grid, n_tokens, s);

@@ -889,7 +889,8 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
   const bool tiles_ok = pie_split_supported(ctx) && !(b->flags & PIE_PLAN_FORCE_SIMPLE);
   std::vector<Unit> split_units, tile_units;
   plan->simple_rows.clear();
-  plan->tile_tc = pie_tc_supported(ctx) && !(b->flags & PIE_PLAN_NO_TENSOR_TILES);
+  // (8-token pages: the mma.sync row-tile kernel behind PIE_PLAN_NO_TENSOR_TILES has no instantiation, the flag is ignored)
+  plan->tile_tc = pie_tc_supported(ctx) && (!(b->flags & PIE_PLAN_NO_TENSOR_TILES) || P == 8);
   const int TILE_ROWS = plan->tile_tc ? 256 : 64;   // two 128-row tcgen05 tiles, or four 16-row warps
 
   // Shared-prefix cascade (decode-shaped requests): consecutive requests whose page lists start

@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 def _random_batch(seed):
     from tests.test_gpu_matrix import _bf16_round
     rng = np.random.RandomState(1000 + seed)
-    P = int(rng.choice([16, 32]))
+    P = int(rng.choice([8, 16, 32]))
     H_q, H_kv = [(8, 2), (32, 8), (4, 4), (6, 2), (16, 1)][rng.randint(5)]
     D = int(rng.choice([64, 128]))
     R = rng.randint(3, 11)
@@ -112,7 +112,7 @@ def test_random_batches_with_requests_that_do_not_store(seed):
     from tests._util import same_bits
     from tests.test_gpu_matrix import _bf16_round
     rng = np.random.RandomState(5000 + seed)
-    P = int(rng.choice([16, 32]))
+    P = int(rng.choice([8, 16, 32]))
     H_q, H_kv = [(8, 2), (32, 8), (4, 4), (6, 2)][rng.randint(4)]
     D = int(rng.choice([64, 128]))
     R = rng.randint(3, 9)

@@ -42,6 +42,39 @@ def test_small_configs_match_oracle(name, flags):
         gp.close()
 
 
+def test_tiny_config_with_column_wise_drops_matches_oracle():
+    """The tiny fp32 configuration with the same dropped tokens for all eight rows of request 3 (the other
+    reading of "30 % of its earlier tokens masked off")."""
+    from tests._gpu import check_close, run_workload
+    wl = configs.tiny_fp32(column_wise=True)
+    O_ref, L_ref, _ = run_oracle(wl, poison=True)
+    O, L, _ = run_workload(wl, poison=True)
+    check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
+
+
+@pytest.mark.parametrize("name", SMALL[1:])
+@pytest.mark.parametrize("flags", [0, 2])
+def test_small_configs_with_8_token_pages(name, flags):
+    """KvPages of 8 tokens (the small end of the 8 - 32 tokens of Section 4.1) on the tensor-core kernels: the
+    decode kernel takes them in pairs, the row-tile kernel as 16 page blocks per KV tile.  Outputs against the
+    oracle, append bit exact, NaN-poisoned tails harmless."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import check_close, run_workload
+    wl = configs.small(name, P=8)
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    O, L, info, gp = run_workload(wl, poison=True, flags=flags, keep=True)
+    try:
+        assert info["num_simple_rows"] == 0 and info["num_split_items"] + info["num_tile_items"] > 0
+        check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        used = wl.used_pages()
+        K, V = gp.read_pages(used)
+        for n, p in enumerate(used):
+            Ko, Vo = pool[int(p)]
+            assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {p}"
+    finally:
+        gp.close()
+
+
 @pytest.mark.parametrize("name", SMALL[1:])
 def test_peaked_scores_match_oracle(name):
     """Q scaled x4: the softmax concentrates and |O| = O(1), so a wrong kernel cannot hide
