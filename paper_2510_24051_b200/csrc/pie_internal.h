@@ -181,7 +181,7 @@ struct pie_ctx {
   struct HeldPages { cudaEvent_t done; std::vector<int32_t> pages; };
   std::vector<HeldPages> held_pages;
   std::vector<cudaEvent_t> held_events;   // recycled events of held_pages
-  bool tc_configured = false, split_configured = false, tile_configured = false;   // kernel attributes set for this context's device
+  bool tc_configured = false, split_configured = false, tile_configured = false, nd_configured = false;   // kernel attributes set for this context's device
   // The block-local work list of the latest decode batch.  Consecutive steps of a serving loop bring the same
   // requests with the same page counts (a request grows by a page every page_size steps), and then the list is
   // the same up to the fields copied from the request records: the planner reuses it instead of dealing the

@@ -67,6 +67,26 @@ def test_next_dist_with_many_equal_logits_and_masked_vocabulary():
     np.testing.assert_allclose(p, 1.0 / 20011, rtol=1e-5)
 
 
+def test_next_dist_on_decode_batches_with_a_cluster_of_blocks_per_row():
+    """Aligned bf16 rows of at least 8,192 logits in batches up to twice the SM count run with a cluster of thread
+    blocks per row (parts of the row in shared memory, candidates gathered through distributed shared memory):
+    the benchmark's shape (2 blocks per row), a few rows (4 blocks per row), a vocabulary that is not a multiple
+    of 8 inside a wider row stride, and quantised / constant / partly masked rows, where the candidates overflow
+    and the first block redoes the row the general way."""
+    _check(_logits(64, 128256, torch.bfloat16, seed=11).cuda(), 256)
+    _check(_logits(5, 32768, torch.bfloat16, seed=12).cuda(), 256)
+    wide = torch.zeros(3, 50264, dtype=torch.bfloat16)
+    wide[:, :50260] = _logits(3, 50260, torch.bfloat16, seed=13)
+    _check(wide.cuda()[:, :50260], 100)
+    g = torch.Generator().manual_seed(6)
+    x = torch.randint(-6, 7, (4, 20016), generator=g).float() * 0.5
+    x[1, 100:15000] = float("-inf")
+    x[2, :] = 1.25
+    _check(x.to(torch.bfloat16).cuda(), 256)
+    p = _check(x[2:3].to(torch.bfloat16).cuda(), 16)
+    np.testing.assert_allclose(p, 1.0 / 20016, rtol=1e-5)
+
+
 def test_next_dist_argument_errors():
     import paper_2510_24051_b200 as pie
     ctx = _ctx()
