@@ -62,14 +62,17 @@ def test_random_batches_match_oracle(seed):
     O_ref, L_ref = orc.forward(**dict(args, pool=pool_ref), out_lens=out_len)
     produced = ~np.isnan(L_ref[:, 0])
     T = len(args["q"])
-    tdt = torch.bfloat16
     ptr = np.zeros(len(seqs) + 1, np.int64)
     for r, m in enumerate(args["masks"]):
         ptr[r + 1] = ptr[r] + (0 if m is None else m.size)
     given = [m.reshape(-1).astype(np.uint8) for m in args["masks"] if m is not None]
     buf = np.concatenate(given) if given else np.zeros(0, np.uint8)
-    for flags in (0, pie.PIE_PLAN_NO_TENSOR_TILES, pie.PIE_PLAN_FORCE_SIMPLE):
-        ctx = pie.pie_create(total, P, H_q, H_kv, D, "bf16", len(seqs), T, 0)
+    runs = [("bf16", 0), ("bf16", pie.PIE_PLAN_NO_TENSOR_TILES), ("bf16", pie.PIE_PLAN_FORCE_SIMPLE)]
+    if seed % 4 == 3:
+        runs.append(("f32", 0))          # the same values in an fp32 pool (the plain kernel), at the fp32 tolerance
+    for dtype, flags in runs:
+        tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+        ctx = pie.pie_create(total, P, H_q, H_kv, D, dtype, len(seqs), T, 0)
         try:
             ids = pie.pie_alloc_kvpages(ctx, total)
             K = torch.from_numpy(np.stack([args["pool"][int(p)][0] for p in ids])).to(tdt).cuda()
@@ -88,7 +91,7 @@ def test_random_batches_match_oracle(seed):
             assert np.isnan(O[~produced]).all() and np.isnan(L[~produced]).all()
             if produced.any():
                 assert np.isfinite(O[produced]).all()
-                assert np.abs(O[produced] - O_ref[produced]).max() <= TOL_O["bf16"], (seed, flags)
+                assert np.abs(O[produced] - O_ref[produced]).max() <= TOL_O[dtype], (seed, dtype, flags)
                 assert np.abs(L[produced] - L_ref[produced]).max() <= TOL_LSE, (seed, flags)
             Kg = torch.empty((total, P, H_kv, D), dtype=tdt, device="cuda")
             Vg = torch.empty_like(Kg)
