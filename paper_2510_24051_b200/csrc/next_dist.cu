@@ -402,9 +402,9 @@ next_dist_kernel(const T* __restrict__ logits, int64_t row_stride, int vocab, in
     // (plain fp32 arithmetic per entry: exp2 of a fused multiply-add, one comparison with tau as a float; the
     //  integer key is only made for the few entries that pass)
     float s_acc = 0.f;
-    const float tau_f = value_of_key(tau), kLog2e = 1.4426950408889634f, neg_max_l2 = -row_max_f * kLog2e;
+    const float tau_f = value_of_key(tau), kLog2e = 1.4426950408889634f;
     walk_row<T, kAligned>(row, vocab, [&](float x, int token) {
-      s_acc += exp2f_fast(fmaf(x, kLog2e, neg_max_l2));   // (about 2^-21 relative: the kept tokens below use expf)
+      s_acc += exp2f_fast((x - row_max_f) * kLog2e);   // (the difference first: exact enough for logits of any magnitude)
       if (x >= tau_f) {
         const uint32_t at = atomicAdd(&sh_cnt, 1u);
         if (at < (uint32_t)kMaxCand) pool[at] = ((unsigned long long)key_of_bits(__float_as_uint(x)) << 32) | (0xFFFFFFFFu - (uint32_t)token);
@@ -522,7 +522,7 @@ next_dist_cluster_kernel(const __nv_bfloat16* __restrict__ logits, int64_t row_s
       acc *= f;
       m_t = x;
     }
-    if (m_t != kNegInf) acc += exp2f_fast(fmaf(x, kLog2e, -m_t * kLog2e));
+    if (m_t != kNegInf) acc += exp2f_fast((x - m_t) * kLog2e);
   };
   for (int c = 0; c < n_chunks; ++c) {
     mbar_wait(smem_u32(&sh.bar[c]), 0, status);
@@ -542,15 +542,16 @@ next_dist_cluster_kernel(const __nv_bfloat16* __restrict__ logits, int64_t row_s
         m_t = gmax;
       }
       if (m_t != kNegInf) {
-        uint64_t shift2;
-        asm("mov.b64 %0, {%1,%1};" : "=l"(shift2) : "f"(-m_t * kLog2e));
+        uint64_t negm2;   // (x - m first, then the scale: the rounded product m * log2(e) would cost accuracy at large |m|)
+        asm("mov.b64 %0, {%1,%1};" : "=l"(negm2) : "f"(-m_t));
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           uint64_t x2, y2, p2;
           float e0, e1;
           asm("mov.b64 %0, {%1,%2};" : "=l"(x2) : "r"(w[e] << 16), "r"(w[e] & 0xFFFF0000u));
-          asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(y2) : "l"(x2), "l"(scale2), "l"(shift2));
+          asm("add.rn.f32x2 %0, %1, %2;" : "=l"(y2) : "l"(x2), "l"(negm2));
+          asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(y2) : "l"(scale2));
           asm("mov.b64 {%0,%1}, %2;" : "=f"(e0), "=f"(e1) : "l"(y2));
           asm("mov.b64 %0, {%1,%2};" : "=l"(p2) : "f"(exp2f_fast(e0)), "f"(exp2f_fast(e1)));
           if (e & 1) asm("add.rn.f32x2 %0, %0, %1;" : "+l"(acc_b) : "l"(p2));

@@ -85,6 +85,9 @@ def test_next_dist_on_decode_batches_with_a_cluster_of_blocks_per_row():
     _check(x.to(torch.bfloat16).cuda(), 256)
     p = _check(x[2:3].to(torch.bfloat16).cuda(), 16)
     np.testing.assert_allclose(p, 1.0 / 20016, rtol=1e-5)
+    big = (_logits(4, 32768, torch.float32, seed=14) + 300.0).to(torch.bfloat16)      # logits far from zero
+    _check(big.cuda(), 256)
+    _check(big.float().cuda(), 256)                                                   # (the one-block kernel)
 
 
 def test_next_dist_argument_errors():
