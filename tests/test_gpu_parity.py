@@ -365,15 +365,16 @@ def test_output_pointer_that_is_only_16_byte_aligned():
         pie.pie_plan_destroy(plan)
 
 
+@pytest.mark.parametrize("P", [16, 8])
 @pytest.mark.parametrize("name", ["batched_decode", "long_context_policy"])
-def test_decode_fusions_equal_the_separate_launches(name):
+def test_decode_fusions_equal_the_separate_launches(name, P):
     """Decode batches let the split-KV kernel write the new K/V rows itself and (short launches)
     merge the pieces of a (request, kv head) inside one thread block; PIE_OPT_NO_FUSION switches
     either off.  The append fusion must not change a bit of O, LSE or the pool; the merge fusion
     only changes the fp32 summation order, so it is held to the oracle tolerance."""
     import paper_2510_24051_b200 as pie
     from tests._gpu import GpuPool, check_close
-    wl = configs.small(name)
+    wl = configs.small(name, P=P)
     O_ref, L_ref, pool = run_oracle(wl, poison=True)
     res = {}
     for no_fusion in (0, 1, 2, 3):
@@ -398,15 +399,15 @@ def test_decode_fusions_equal_the_separate_launches(name):
     assert res[3][0] == 3 and res[0][0] <= 2              # append + split-KV + merge against split-KV (+ merge if dynamic)
 
 
-@pytest.mark.parametrize("flags", [8, 4, 0, 8 | 2])
-def test_shared_prefix_cascade_matches_oracle(flags):
+@pytest.mark.parametrize("flags,P", [(8, 16), (4, 16), (0, 16), (8 | 2, 16), (8, 8), (8, 32)])
+def test_shared_prefix_cascade_matches_oracle(flags, P):
     """Branches that decode from a shared prompt: with the cascade the prompt's pages are attended
     once per group (row-tile kernel over the gathered rows) and each request's private pages by the
     split-KV kernel, merged on LSE (Section 4.2: forked contexts share KvPages).  Flags: 8 = cascade
     however small the saving, 4 = never, 0 = the planner's own choice (this small batch: none)."""
     import paper_2510_24051_b200 as pie
     from tests._gpu import check_close, run_workload
-    wl = configs.small("shared_prefix_decode")
+    wl = configs.small("shared_prefix_decode", P=P)
     O_ref, L_ref, pool = run_oracle(wl, poison=True)
     O, L, info, gp = run_workload(wl, poison=True, flags=flags, keep=True)
     try:
@@ -421,14 +422,14 @@ def test_shared_prefix_cascade_matches_oracle(flags):
         gp.close()
 
 
-@pytest.mark.parametrize("sms", [6, 16])
-def test_block_local_merge_matches_oracle(sms):
+@pytest.mark.parametrize("sms,P", [(6, 16), (16, 16), (6, 8)])
+def test_block_local_merge_matches_oracle(sms, P):
     """Short decode launches deal whole (request, kv head) units to thread blocks and cut them only
     between warps of one block, which then merges the pieces itself: no merge launch.  Few SMs
     make the small batch balance well enough for that path to be chosen."""
     import paper_2510_24051_b200 as pie
     from tests._gpu import GpuPool, check_close
-    wl = configs.small("batched_decode")
+    wl = configs.small("batched_decode", P=P)
     O_ref, L_ref, pool = run_oracle(wl, poison=True)
     with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
         pie.pie_set_option(gp.ctx, pie.PIE_OPT_SPLIT_SMS, sms)
