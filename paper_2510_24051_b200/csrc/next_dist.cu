@@ -764,9 +764,12 @@ int pie_get_next_dist(pie_ctx* ctx, const void* logits, int32_t dtype, int32_t n
       attr[0].val.clusterDim.z = 1;
       cfg.attrs = attr;
       cfg.numAttrs = 1;
-      PIE_CUDA(ctx, cudaLaunchKernelEx(&cfg, next_dist_cluster_kernel, (const __nv_bfloat16*)logits, row_stride, (int)vocab, (int)top_k, gpp,
-                                       out_ids, out_probs, ctx->d_status));
-      return PIE_OK;
+      // (a device that cannot place such clusters - fewer SMs per GPC, a partitioned GPU - refuses the launch:
+      //  the one-block kernel below then does the work)
+      if (cudaLaunchKernelEx(&cfg, next_dist_cluster_kernel, (const __nv_bfloat16*)logits, row_stride, (int)vocab, (int)top_k, gpp, out_ids,
+                             out_probs, ctx->d_status) == cudaSuccess)
+        return PIE_OK;
+      cudaGetLastError();
     }
   }
   if (dtype == PIE_DTYPE_BF16) {

@@ -886,7 +886,9 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
   }
 
   // ---- route requests to kernels and partition the work
-  const bool tiles_ok = pie_split_supported(ctx) && !(b->flags & PIE_PLAN_FORCE_SIMPLE);
+  // (head groups above 16 - multi-query models - do not fit the split-KV kernel's 16 rows per warp: every request
+  //  of such a context has more than 16 rows and runs on the row-tile kernel)
+  const bool tiles_ok = (pie_split_supported(ctx) || (pie_tc_supported(ctx) && G > 16)) && !(b->flags & PIE_PLAN_FORCE_SIMPLE);
   std::vector<Unit> split_units, tile_units;
   plan->simple_rows.clear();
   // (8-token pages: the mma.sync row-tile kernel behind PIE_PLAN_NO_TENSOR_TILES has no instantiation, the flag is ignored)

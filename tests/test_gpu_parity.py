@@ -336,6 +336,21 @@ def test_head_groups_that_do_not_divide_the_row_tile(heads):
         check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
 
 
+@pytest.mark.parametrize("heads", [(32, 1), (64, 2), (24, 1)])
+def test_head_groups_above_16_run_on_the_row_tile_kernel(heads):
+    """Multi-query style grouping (32 or 24 query heads per kv head): more rows per token than a decode warp
+    holds, so every request, single-token decodes included, takes the tensor-core row-tile kernel."""
+    from tests._gpu import check_close, run_workload
+    H_q, H_kv = heads
+    for name in ("batched_decode", "mixed_prefill_decode"):
+        wl = configs.small(name, H_q=H_q, H_kv=H_kv)
+        O_ref, L_ref, _ = run_oracle(wl, poison=True)
+        for flags in (0, 2):
+            O, L, info = run_workload(wl, poison=True, flags=flags)
+            assert info["num_tile_items"] > 0 and info["num_simple_rows"] == 0 and info["num_split_items"] == 0
+            check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
+
+
 def test_output_pointer_that_is_only_16_byte_aligned():
     """The kernels use 32-byte stores when the output pointer allows it; a view that starts 16 bytes
     into an allocation must give the same bits."""
