@@ -1,8 +1,10 @@
 // get_next_dist from the logits on (Table 1 `get_next_dist`; Section 4.2 "Sample API": the
 // next-token probability distribution, truncated to the top-K tokens, K = 256 by default).
 //
-// One thread block per row of logits, two passes over the row (the second finds it in L2: a row
-// is 256 - 512 KB).
+// Two kernels.  Aligned bf16 rows of at least 8,192 logits run with a CLUSTER of thread blocks per row
+// (next_dist_cluster_kernel, described where it is defined).  Everything else - fp32 logits, unaligned or short
+// rows - runs with one thread block per row (next_dist_kernel), two passes over the row (the second finds it in
+// L2: a row is 256 - 512 KB):
 //  1. Every thread takes the maximum of its own entries; every warp sorts its 32 maxima and offers
 //     its ceil(K / 32)-th largest.  The smallest offer, tau, has at least K entries of the row at
 //     or above it (that many thread maxima alone), so the K-th largest entry of the row is >= tau
@@ -12,7 +14,7 @@
 //     descending, token id ascending), which is exactly the order of the result; the first K are
 //     written with their probabilities exp(x - max) / sum, not renormalised.
 // Rows with so many equal entries around the K-th place that more than 4,096 entries pass the
-// filter (quantised logits, constant rows) take the general way instead: radix selection of the
+// filter (quantised logits, constant rows) take the general way instead (radix_path): radix selection of the
 // K-th largest key, eight bits per pass, then the entries above it and, in ascending token order,
 // as many entries equal to it as are still missing.
 #include <cuda_bf16.h>
