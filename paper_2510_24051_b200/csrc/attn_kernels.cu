@@ -759,6 +759,113 @@ __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* 
   if (lane == 0) lse_out[oi] = Z > 0.f ? M + logf(Z) : kNegInf;
 }
 
+// The same for groups of row-tile partials (up to 256 rows per group, few sources each: the pieces of a cut unit,
+// or a request's private part plus the shared-prefix cascade).  One thread block per group, its record read
+// once; every warp takes four rows at a time: lane 8 k + c fetches the LSE of (row k, source c) while every lane
+// already fetches its columns of all sources of the four rows - one round trip to memory per four rows instead
+// of a chain of four per row.  Sources are combined in slot order (own slots, then the cascade's), as above.
+template <typename T, int D>
+__global__ void __launch_bounds__(256) merge_tiles_kernel(const PieMerge* __restrict__ merges, const PieReq* __restrict__ reqs,
+                                                          const float* __restrict__ ws_o, const float* __restrict__ ws_lse,
+                                                          T* __restrict__ out, float* __restrict__ lse_out, int slot_rows,
+                                                          int n_q_heads, int G, const float* __restrict__ x_ws_o,
+                                                          const float* __restrict__ x_ws_lse, int x_slot_rows) {
+  constexpr int EPL = D / 32, RPW = 4, MAXS = 4;
+  pie_pdl_launch_dependents();
+  pie_pdl_wait();
+  const PieMerge mg = merges[blockIdx.x];
+  const PieReq rq = reqs[mg.req];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int ntot = mg.nslots + mg.x_nslots;
+  auto lse_at = [&](int c, int row) -> const float* {
+    return c < mg.nslots ? ws_lse + (int64_t)(mg.slot0 + c) * slot_rows + row
+                         : x_ws_lse + (int64_t)(mg.x_slot0 + c - mg.nslots) * x_slot_rows + mg.x_row0 + row;
+  };
+  auto row_at = [&](int c, int row) -> const float* {
+    return c < mg.nslots ? ws_o + ((int64_t)(mg.slot0 + c) * slot_rows + row) * D + lane * EPL
+                         : x_ws_o + ((int64_t)(mg.x_slot0 + c - mg.nslots) * x_slot_rows + mg.x_row0 + row) * D + lane * EPL;
+  };
+  auto store_row = [&](int row, const float* acc, float M, float Z) {
+    const int gr = mg.row0 + row;
+    const int tok = gr / G, head = mg.kv_head * G + gr % G;
+    const int64_t oi = (int64_t)(rq.q_start + tok) * n_q_heads + head;
+    const float inv = Z > 0.f ? 1.f / Z : 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) out[oi * D + lane * EPL + e] = (T)(acc[e] * inv);
+    if (lane == 0) lse_out[oi] = Z > 0.f ? M + logf(Z) : kNegInf;
+  };
+  for (int row0 = warp * RPW; row0 < mg.nrows; row0 += (blockDim.x >> 5) * RPW) {
+    const int nr = min(RPW, mg.nrows - row0);   // (warp uniform)
+    if (ntot <= MAXS) {
+      float v[RPW][MAXS][EPL];
+#pragma unroll
+      for (int k = 0; k < RPW; ++k)
+#pragma unroll
+        for (int c = 0; c < MAXS; ++c) {
+          if (k < nr && c < ntot) {
+            const float* src = row_at(c, row0 + k);
+            if constexpr (EPL == 4) {
+              const float4 x = __ldcg(reinterpret_cast<const float4*>(src));
+              v[k][c][0] = x.x, v[k][c][1] = x.y, v[k][c][2] = x.z, v[k][c][3] = x.w;
+            } else {
+              const float2 x = __ldcg(reinterpret_cast<const float2*>(src));
+              v[k][c][0] = x.x, v[k][c][1] = x.y;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) v[k][c][e] = 0.f;
+          }
+        }
+      const int lk = lane >> 3, lc = lane & 7;   // this lane's (row, source) pair
+      float l = kNegInf;
+      if (lk < nr && lc < ntot) l = *lse_at(lc, row0 + lk);
+      float M = l;
+      for (int sft = 4; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));   // over the 8 lanes of the row
+      const float w = M != kNegInf ? __expf(l - M) : 0.f;   // exp(-inf) = 0
+#pragma unroll
+      for (int k = 0; k < RPW; ++k) {
+        float acc[EPL], Z = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+#pragma unroll
+        for (int c = 0; c < MAXS; ++c) {
+          const float wu = __shfl_sync(0xFFFFFFFFu, w, k * 8 + c);
+          Z += wu;
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) acc[e] += wu * v[k][c][e];
+        }
+        const float Mk = __shfl_sync(0xFFFFFFFFu, M, k * 8);
+        if (k < nr) store_row(row0 + k, acc, Mk, Z);
+      }
+    } else {
+      for (int k = 0; k < nr; ++k) {   // many sources: row by row
+        const int row = row0 + k;
+        float M = kNegInf;
+        for (int c = lane; c < ntot; c += 32) M = fmaxf(M, *lse_at(c, row));
+        for (int sft = 16; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));
+        float Z = 0.f, acc[EPL];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+        for (int base = 0; base < ntot; base += 32) {
+          const int c = base + lane;
+          float w = 0.f;
+          if (c < ntot && M != kNegInf) w = __expf(*lse_at(c, row) - M);
+          Z += w;
+          const int cnt = min(32, ntot - base);
+          for (int u = 0; u < cnt; ++u) {
+            const float wu = __shfl_sync(0xFFFFFFFFu, w, u);
+            const float* src = row_at(base + u, row);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[e] += wu * src[e];
+          }
+        }
+        for (int sft = 16; sft > 0; sft >>= 1) Z += __shfl_xor_sync(0xFFFFFFFFu, Z, sft);
+        store_row(row, acc, M, Z);
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------ simple kernel
 template <typename T>
 __device__ __forceinline__ float to_f32(T v);
@@ -919,12 +1026,13 @@ int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* ou
 
 int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s) {
   const int D = ctx->cfg.head_dim;
+  const bool tiles = ll.slot_rows >= 32;      // groups of row-tile partials: one block per group
   const int wpb = ll.slot_rows >= 8 ? 8 : 4;  // warps (= rows) per block
-  const dim3 n((unsigned)ll.merges.size(), (unsigned)((ll.slot_rows + wpb - 1) / wpb));
-#define PIE_MERGE(T, DD)                                                                                          \
-  PIE_CUDA(ctx, pie_launch_pdl(merge_kernel<T, DD>, n, dim3(wpb * 32), 0, s, (const PieMerge*)ll.d_merges,      \
-                               (const PieReq*)plan->d_reqs, (const float*)ll.d_ws_o, (const float*)ll.d_ws_lse, \
-                               (T*)out, lse, ll.slot_rows, ctx->cfg.num_q_heads, ctx->G,                         \
+  const dim3 n((unsigned)ll.merges.size(), tiles ? 1u : (unsigned)((ll.slot_rows + wpb - 1) / wpb));
+#define PIE_MERGE(T, DD)                                                                                                   \
+  PIE_CUDA(ctx, pie_launch_pdl(tiles ? merge_tiles_kernel<T, DD> : merge_kernel<T, DD>, n, dim3(tiles ? 256 : wpb * 32), 0, s, \
+                               (const PieMerge*)ll.d_merges, (const PieReq*)plan->d_reqs, (const float*)ll.d_ws_o,         \
+                               (const float*)ll.d_ws_lse, (T*)out, lse, ll.slot_rows, ctx->cfg.num_q_heads, ctx->G,        \
                                (const float*)plan->tile.d_ws_o, (const float*)plan->tile.d_ws_lse, plan->tile.slot_rows))
   if (ctx->cfg.dtype == PIE_DTYPE_BF16) {
     if (D == 64) PIE_MERGE(__nv_bfloat16, 64);

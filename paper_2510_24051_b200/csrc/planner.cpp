@@ -895,14 +895,19 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
   plan->tile_tc = pie_tc_supported(ctx) && (!(b->flags & PIE_PLAN_NO_TENSOR_TILES) || P == 8);
   const int TILE_ROWS = plan->tile_tc ? 256 : 64;   // two 128-row tcgen05 tiles, or four 16-row warps
 
-  // Shared-prefix cascade (decode-shaped requests): consecutive requests whose page lists start
-  // with the same physical pages - parallel samples, beams, branches of one prompt - have their
-  // rows gathered and attended to that prefix ONCE, as row tiles of a virtual request on the
-  // row-tile kernel; every request then attends only its private pages on the split-KV kernel,
-  // and the merge combines the two partials.  The prefix is read from HBM once per group instead
-  // of once per request.  (Requests with many rows of their own, e.g. token trees, already fill
-  // whole row tiles and find the shared pages in L2: gathering them would only add partials.)
-  struct Cascade { int32_t first, n, L, vreq; };
+  // Shared-prefix cascade: consecutive requests whose page lists start with the same physical
+  // pages - parallel samples, beams, branches of one prompt - have their rows gathered and
+  // attended to that prefix ONCE, as row tiles of a virtual request on the row-tile kernel; every
+  // request then attends only its private pages, and the merge combines the two partials.
+  //  * Decode-shaped requests (at most 16 rows): private pages on the split-KV kernel.  The prefix
+  //    is read from HBM once per group instead of once per request.
+  //  * Requests with more rows that still fill at most half a row tile (a token tree of 32 nodes
+  //    under 4 grouped heads: 128 rows): private pages as row-tile items of their own.  Here the
+  //    gain is the tile: a lone request would leave half of the 256-row item, and one of the two
+  //    softmax warpgroups, without work over the whole prefix.
+  // (Requests that fill a row tile on their own, e.g. token trees of 64 nodes, find the shared
+  //  pages in L2: gathering them would only add partials.)
+  struct Cascade { int32_t first, n, L, vreq; bool big; };
   std::vector<Cascade> cascades;
   std::vector<int32_t> casc_of(R, -1);
   if (tiles_ok && !(b->flags & PIE_PLAN_NO_CASCADE) && all_rows_out) {   // (the gathered rows of a group must be consecutive query tokens)
@@ -917,7 +922,8 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
     for (int r = 0; r < R;) {
       const PieReq& q0 = plan->reqs[r];
       const int rows = q0.q_len * G;
-      if (rows == 0 || rows > 16 || TILE_ROWS % rows != 0 || q0.kept_count < 2 || r + 1 >= R || plan->reqs[r + 1].kept_count < 2 ||
+      const bool big = rows > 16;
+      if (rows == 0 || (big && 2 * rows > TILE_ROWS) || TILE_ROWS % rows != 0 || q0.kept_count < 2 || r + 1 >= R || plan->reqs[r + 1].kept_count < 2 ||
           plan->kept[2 * (size_t)plan->reqs[r + 1].kept_start] != plan->kept[2 * (size_t)q0.kept_start]) {  // (no neighbour with the same first page: no run starts here)
         ++r;
         continue;
@@ -932,16 +938,21 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         if (c < min_L) break;
         L = c;
       }
-      if (e - r >= min_n && L >= min_L) {
-        cascades.push_back(Cascade{r, e - r, L, 0});
-        saved += (int64_t)(e - r - 1) * L * cfg.num_kv_heads;
+      // (a group of larger requests must fill at least one row tile and share at least 1,024 tokens: below that
+      //  the partials and the merge cost more than the filled tile gains)
+      const bool accept = !big ? (e - r >= min_n && L >= min_L)
+                               : (e - r >= 2 && L >= min_L && (always || ((e - r) * rows >= TILE_ROWS && (int64_t)L * P >= 1024)));
+      if (accept) {
+        cascades.push_back(Cascade{r, e - r, L, 0, big});
+        if (!big) saved += (int64_t)(e - r - 1) * L * cfg.num_kv_heads;
         r = e;
       } else {
         ++r;
       }
     }
-    // worth a second launch and a merge only when enough page reads disappear
-    if (!always && saved < 2048) cascades.clear();
+    // decode-shaped groups are worth a second launch and a merge only when enough page reads disappear
+    if (!always && saved < 2048)
+      cascades.erase(std::remove_if(cascades.begin(), cascades.end(), [](const Cascade& c) { return !c.big; }), cascades.end());
     for (size_t c = 0; c < cascades.size(); ++c) {
       Cascade& cs = cascades[c];
       const PieReq& q0 = plan->reqs[cs.first];
@@ -974,6 +985,9 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
           split_units.push_back(Unit{r, g, 0, rows, q.kept_start, q.kept_start + q.kept_count});
       // (requests of a cascade get their split units below, once the cascade's slots are known)
     } else {
+      // (a request of a cascade attends only the pages behind the shared prefix here and writes a partial; the
+      //  cascade's slots are added to its merge group once the partition has assigned them)
+      const int skip = casc_of[r] >= 0 ? cascades[casc_of[r]].L : 0;
       for (int g = 0; g < cfg.num_kv_heads; ++g)
         for (int row0 = 0; row0 < rows; row0 += TILE_ROWS) {
           int nrows = std::min(TILE_ROWS, rows - row0);
@@ -983,7 +997,9 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
             int lim = q.kv_len - q.q_len + i1;
             end = std::min(end, lim / P + 1);
           }
-          tile_units.push_back(Unit{r, g, row0, nrows, q.kept_start, q.kept_start + end});
+          Unit u{r, g, row0, nrows, q.kept_start + skip, q.kept_start + std::max(end, skip)};
+          u.force_partial = skip > 0;
+          tile_units.push_back(u);
         }
     }
   }
@@ -1017,8 +1033,8 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       // beats one kernel after the other.
       double split_bytes = 0, tile_flops = 0;
       for (const Unit& u : split_units) split_bytes += (double)(u.page_end - u.page_begin) * 2.0 * P * cfg.head_dim * 2.0;
-      for (const Cascade& cs : cascades)   // the private pages of cascaded requests (their split units are made below)
-        for (int k = 0; k < cs.n; ++k)
+      for (const Cascade& cs : cascades)   // the private pages of cascaded decode-shaped requests (their split units are made below)
+        for (int k = 0; k < (cs.big ? 0 : cs.n); ++k)
           split_bytes += (double)(plan->reqs[cs.first + k].kept_count - cs.L) * cfg.num_kv_heads * 2.0 * P * cfg.head_dim * 2.0;
       for (const Unit& u : tile_units) tile_flops += (double)(u.page_end - u.page_begin) * P * 4.0 * cfg.head_dim * u.nrows;
       const double t_split = split_bytes / 6.4e12, t_tile = tile_flops / 0.60e15;  // whole-chip estimates, seconds (rates measured on the mixed workload)
@@ -1051,8 +1067,22 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
   // cascaded requests then name as further sources of their merge groups
   UnitSlots tile_slots;
   partition(tile_units, tile_sms, plan->tile_tc ? 32 : 8, TILE_ROWS, true, plan->tile, &tile_slots);
+  // merge groups of the larger cascaded requests (row-tile items over their private pages): add the slots of
+  // the cascade pieces that hold the same rows
+  for (PieMerge& m : plan->tile.merges) {
+    if (m.req >= R || casc_of[m.req] < 0) continue;
+    const Cascade& cs = cascades[casc_of[m.req]];
+    const PieReq& v = plan->reqs[cs.vreq];
+    const int tiles_per_head = (v.q_len * G + TILE_ROWS - 1) / TILE_ROWS;
+    const int vr0 = (plan->reqs[m.req].q_start - v.q_start) * G + m.row0;   // first virtual row of the group's rows
+    const auto& sl = tile_slots[(size_t)casc_unit0[casc_of[m.req]] + (size_t)m.kv_head * tiles_per_head + vr0 / TILE_ROWS];
+    m.x_slot0 = sl.first;
+    m.x_nslots = sl.second;
+    m.x_row0 = vr0 % TILE_ROWS;
+  }
   for (size_t c = 0; c < cascades.size(); ++c) {
     const Cascade& cs = cascades[c];
+    if (cs.big) continue;
     const PieReq& v = plan->reqs[cs.vreq];
     const int tiles_per_head = (v.q_len * G + TILE_ROWS - 1) / TILE_ROWS;
     for (int k = 0; k < cs.n; ++k) {

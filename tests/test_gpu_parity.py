@@ -437,6 +437,38 @@ def test_shared_prefix_cascade_matches_oracle(flags, P):
         gp.close()
 
 
+@pytest.mark.parametrize("case", ["small_forced", "mid_auto", "mid_auto_8_token_pages", "causal_chunks"])
+def test_shared_prefix_cascade_of_requests_with_row_tiles_of_their_own(case):
+    """Branches that verify a token tree of 32 nodes over a shared prompt bring 128 rows each - half a row tile.
+    The cascade gathers the group's rows over the shared pages (full tiles, no masks) and runs every request's
+    private suffix + tree pages as a row-tile item of its own; both write partials that the merge combines.  Also
+    with inferred causal masks (short prefill chunks of forked requests)."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import check_close, run_workload
+    flags = 0
+    if case == "small_forced":
+        wl, flags = configs.small("shared_prefix_tree"), pie.PIE_PLAN_CASCADE_ALWAYS
+    elif case == "mid_auto":
+        wl = configs.shared_prefix_tree(groups=2, branches=4, prefix=1024, suffix=48, tree=32, num_pages=512)
+    elif case == "mid_auto_8_token_pages":
+        wl = configs.shared_prefix_tree(groups=2, branches=5, prefix=1024, suffix=40, tree=32, num_pages=1024, P=8)
+    else:
+        wl = configs.shared_prefix_tree(groups=2, branches=4, prefix=1040, suffix=16, tree=16, num_pages=512)
+        wl.masks = None                                   # 16 new tokens per branch under the inferred causal mask: 64 rows
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    O, L, info, gp = run_workload(wl, poison=True, flags=flags, keep=True)
+    try:
+        assert info["num_merge_groups"] == wl.R * wl.H_kv and info["num_split_items"] == 0
+        check_close(O, L, O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        used = wl.used_pages()
+        K, V = gp.read_pages(used)
+        for n, p in enumerate(used):
+            Ko, Vo = pool[int(p)]
+            assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {p}"
+    finally:
+        gp.close()
+
+
 @pytest.mark.parametrize("sms,P", [(6, 16), (16, 16), (6, 8)])
 def test_block_local_merge_matches_oracle(sms, P):
     """Short decode launches deal whole (request, kv head) units to thread blocks and cut them only

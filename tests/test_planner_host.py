@@ -211,9 +211,19 @@ def test_shared_prefix_cascade_planning():
     off = plan_info(full, pie.PIE_PLAN_NO_CASCADE)
     assert auto["num_tile_items"] > 0 and off["num_tile_items"] == 0
     assert auto["num_merge_groups"] == full.R * full.H_kv
-    # the tree workload keeps its requests whole: many rows each, shared pages served from L2
-    tree_wl = configs.small("shared_prefix_tree")
-    assert plan_info(tree_wl, pie.PIE_PLAN_CASCADE_ALWAYS) == plan_info(tree_wl, pie.PIE_PLAN_NO_CASCADE)
+    # token trees of 64 nodes fill a row tile per request (256 rows): they stay whole, shared pages served from L2
+    tree64 = configs.shared_prefix_tree(groups=2, branches=3, prefix=256, suffix=32, tree=64, num_pages=256)
+    assert plan_info(tree64, pie.PIE_PLAN_CASCADE_ALWAYS) == plan_info(tree64, pie.PIE_PLAN_NO_CASCADE)
+    # trees of 32 nodes fill half a tile (128 rows): their rows are gathered over the shared prefix as well, and the
+    # private pages run as row-tile items of their own - when the group fills a tile and shares >= 1,024 tokens
+    tree32 = configs.small("shared_prefix_tree")
+    forced = plan_info(tree32, pie.PIE_PLAN_CASCADE_ALWAYS)
+    assert forced["num_merge_groups"] == tree32.R * tree32.H_kv and forced["num_split_items"] == 0
+    assert forced["launches"] == 3                                             # append, row tiles, merge
+    assert plan_info(tree32, 0) == plan_info(tree32, pie.PIE_PLAN_NO_CASCADE)  # 256 shared tokens: too few
+    mid = configs.shared_prefix_tree(groups=2, branches=4, prefix=1024, suffix=48, tree=32, num_pages=512)
+    auto = plan_info(mid, 0)
+    assert auto["num_merge_groups"] == mid.R * mid.H_kv and plan_info(mid, pie.PIE_PLAN_NO_CASCADE)["num_merge_groups"] == 0
 
 
 @pytest.mark.parametrize("name", ["long_context_policy", "shared_prefix_tree", "mixed_prefill_decode", "batched_decode"])
