@@ -1037,7 +1037,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         for (int k = 0; k < (cs.big ? 0 : cs.n); ++k)
           split_bytes += (double)(plan->reqs[cs.first + k].kept_count - cs.L) * cfg.num_kv_heads * 2.0 * P * cfg.head_dim * 2.0;
       for (const Unit& u : tile_units) tile_flops += (double)(u.page_end - u.page_begin) * P * 4.0 * cfg.head_dim * u.nrows;
-      const double t_split = split_bytes / 6.4e12, t_tile = tile_flops / 0.60e15;  // whole-chip estimates, seconds (rates measured on the mixed workload)
+      const double t_split = split_bytes / 6.4e12, t_tile = tile_flops / 0.76e15;  // whole-chip estimates, seconds (rates measured on the mixed workload: its decode requests alone, its prefill chunks alone)
       const double sat = 0.6 * ctx->n_sms;                                         // SMs that saturate the memory system
       int best_nt = 0;
       double best_t = 1e30;
