@@ -615,9 +615,8 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
     uint32_t max_id = 0;   // (negative ids wrap to large values)
     for (int k = 0; k < np; ++k) max_id = std::max(max_id, (uint32_t)pages[k]);
     if (max_id >= (uint32_t)cfg.num_pages) return PIE_ERR_BAD_PAGE;
-    uint8_t all_allocated = 1;
-    for (int k = 0; k < np; ++k) all_allocated &= ctx->allocated[pages[k]];
-    if (!all_allocated) return PIE_ERR_BAD_PAGE;
+    // (whether every page is allocated is looked up further down, in the same pass over the page lists that looks
+    //  for pages another request of the batch writes: one random access per listed page instead of two)
     PieReq& q = plan->reqs[r];
     q.q_start = b->qo_indptr[r];
     q.q_len = q_len;
@@ -651,6 +650,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         if (ctx->wmask[pg] == 0) {
           touched.push_back(pg);
           ctx->writer[pg] = r;
+          ctx->allocated[pg] |= 2;   // "written in this batch", next to the allocation flag (cleared again below)
         } else {
           if (ctx->writer[pg] >= 0) {  // second writer of this page: start the per-writer record
             shared.push_back(SharedWrite{pg, ctx->writer[pg], ctx->wmask[pg]});
@@ -661,13 +661,26 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         ctx->wmask[pg] |= m;
       }
     }
-    for (int r = 0; r < R && status == PIE_OK; ++r) {
+    bool bad_page = false;   // (reported before a conflict, as when the pages were checked first)
+    for (int r = 0; r < R && !bad_page; ++r) {
       const PieReq& q = plan->reqs[r];
       const int32_t* pages = b->page_indices + b->page_indptr[r];
-      // (common case first: none of the pages the request only reads is written by anybody)
+      // one look per listed page: allocated?  written by a request of this batch?
+      // (common case: none of the pages the request only reads is written by anybody)
       const int first_written = (q.kv_len - q.q_len) / P;
-      uint32_t any_written = 0;
-      for (int lp = 0; lp < first_written; ++lp) any_written |= ctx->wmask[pages[lp]];
+      uint8_t all_a = 0xFF, any_a = 0;
+      for (int lp = 0; lp < first_written; ++lp) {
+        const uint8_t a = ctx->allocated[pages[lp]];
+        all_a &= a;
+        any_a |= a;
+      }
+      for (int lp = first_written; lp <= q.last_logical; ++lp) all_a &= ctx->allocated[pages[lp]];
+      if (!(all_a & 1)) {
+        bad_page = true;
+        break;
+      }
+      if (status != PIE_OK) continue;
+      const bool any_written = (any_a & 2) != 0;
       for (int lp = any_written ? 0 : first_written; lp <= q.last_logical; ++lp) {
         int32_t pg = pages[lp];
         uint32_t w = ctx->wmask[pg];
@@ -689,7 +702,12 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         if (w & rd) { status = PIE_ERR_CONFLICT; break; }
       }
     }
-    for (int32_t pg : touched) { ctx->wmask[pg] = 0; ctx->writer[pg] = -1; }
+    for (int32_t pg : touched) {
+      ctx->wmask[pg] = 0;
+      ctx->writer[pg] = -1;
+      ctx->allocated[pg] &= 1;
+    }
+    if (bad_page) return PIE_ERR_BAD_PAGE;
     if (status != PIE_OK) return status;
   }
 
