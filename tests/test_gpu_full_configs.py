@@ -99,11 +99,22 @@ def test_full_long_context_policy_with_copy():
         gp.close()
 
 
-def test_large_single_requests():
-    """Index arithmetic at the large end: a 131,071-token decode (8,192 pages, many split chunks and a
+def test_long_context_policy_with_8_token_pages():
+    """A launch long enough for the dynamic chunk list (1.7 GB of kept K/V) on 8-token pages: chunks of odd page
+    counts, pairs of pages per ring stage, partials through the merge kernel."""
+    wl = configs.long_context_policy(R=64, P=8)
+    kv = wl.kv_lens()
+    info, gp = _sampled_check(wl, sample=[0, int(np.argmax(kv)), 63])
+    gp.close()
+    assert info["num_merge_groups"] == wl.R * wl.H_kv and info["num_split_items"] > 4 * wl.R * wl.H_kv
+
+
+@pytest.mark.parametrize("P", [16, 8])
+def test_large_single_requests(P):
+    """Index arithmetic at the large end: a 131,071-token decode (8,192 pages of 16 tokens, many split chunks and a
     ragged last page) and a 300-token prefill chunk over a 20,000-token prefix in one batch."""
     from workloads.configs import _assemble
-    wl = _assemble("large", 0x50494500 + 77, 32, 8, 128, 16, "bf16", 9600, [1, 300], [131071, 20300], None)
+    wl = _assemble("large", 0x50494500 + 77, 32, 8, 128, P, "bf16", 9600 * 16 // P, [1, 300], [131071, 20300], None)
     info, gp = _sampled_check(wl, sample=[0, 1])
     gp.close()
     assert info["num_split_items"] > 100 and info["num_tile_items"] > 0
