@@ -194,6 +194,8 @@ typedef struct pie_plan_info {
   int32_t num_merge_groups;     /* groups whose split partials the merge combines  */
   int32_t launches;             /* kernels one pie_forward enqueues                */
   int32_t side_by_side_sms;     /* SMs given to the row-tile kernel when it runs next to the decode kernel (0: one after the other) */
+  int32_t split_unit_kv_heads;  /* adjacent kv heads that one split-KV work item covers: 1, or 2 (one copy of twice the size per page) */
+  int32_t reserved0;
   int64_t kept_pages;           /* pages left in the lists after dropping fully masked ones */
   int64_t mask_words;           /* 32-bit words of packed mask                     */
   int64_t workspace_bytes;      /* device scratch for split partials               */
@@ -354,14 +356,16 @@ int pie_sched_next_batch(pie_sched* s, int32_t* out_type, int32_t cap, int64_t* 
  *                      after the other; 1 = side by side whenever both kinds are present;
  *                      2 = never.  With 1 and PIE_OPT_SPLIT_SMS and PIE_OPT_TILE_SMS both set,
  *                      those are the two SM sets.
- *   PIE_OPT_NO_FUSION  bit mask of fusions of the decode path to switch off (default 0: both on;
+ *   PIE_OPT_NO_FUSION  bit mask of fusions of the decode path to switch off (default 0: all on;
  *                      results are identical up to fp32 summation order, pool contents bit-identical).
  *                      Bit 0: always launch the append kernel.  By default a decode batch (every
  *                      request one new token, all on the split-KV kernel, no request listing a
  *                      page another one appends to) lets the attention kernel write the new K/V
  *                      rows itself.  Bit 1: always merge split partials with the merge kernel.  By
  *                      default short decode launches keep all pieces of a (request, kv head)
- *                      inside one thread block, which merges them itself. */
+ *                      inside one thread block, which merges them itself.  Bit 2: one kv head per
+ *                      decode unit.  By default, with 64-wide heads and pages of 8 or 16 tokens, a
+ *                      unit is a pair of adjacent kv heads (one copy of twice the size per page). */
 enum { PIE_OPT_SPLIT_SMS = 0, PIE_OPT_TILE_SMS = 1, PIE_OPT_OVERLAP = 2, PIE_OPT_NO_FUSION = 3, PIE_NUM_OPTIONS = 4 };
 int pie_set_option(pie_ctx* ctx, int option, int value);
 

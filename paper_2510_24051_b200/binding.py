@@ -37,7 +37,7 @@ class pie_batch_desc(C.Structure):
 class pie_plan_info(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "num_requests", "num_query_tokens", "num_split_items", "num_tile_items", "num_simple_rows",
-        "num_merge_groups", "launches", "side_by_side_sms")] + [
+        "num_merge_groups", "launches", "side_by_side_sms", "split_unit_kv_heads", "reserved0")] + [
         (n, C.c_int64) for n in ("kept_pages", "mask_words", "workspace_bytes")]
 
     def as_dict(self):

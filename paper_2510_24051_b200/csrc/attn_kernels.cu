@@ -62,6 +62,7 @@ struct RowState {
   int lim[2];              // last visible position under the inferred causal mask (-1: no row)
   const uint32_t* mrow[2]; // packed explicit mask row
   bool valid[2];
+  int hsel[2];             // head of the row inside its unit (units of two adjacent kv heads; else 0)
   bool explicit_mask;
   bool any_rows;
 };
@@ -81,6 +82,7 @@ __device__ __forceinline__ void rows_init(RowState<D>& st, const AttnParams& p, 
     const int tok = st.valid[r] ? gr / p.G : 0;
     const int head = item.kv_head * p.G + (st.valid[r] ? gr % p.G : 0);
     st.lim[r] = st.valid[r] ? rq.kv_len - rq.q_len + tok : -1;
+    st.hsel[r] = st.valid[r] ? (gr % p.G) / p.G_head : -1;
     st.mrow[r] = p.mask + rq.mask_word_off + (int64_t)tok * rq.mask_row_words;
     qptr[r] = reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)(rq.q_start + tok) * p.n_q_heads + head) * D;
     st.m_run[r] = kNegInf;
@@ -108,11 +110,15 @@ __device__ __forceinline__ void rows_init(RowState<D>& st, const AttnParams& p, 
 // tokens (one m16n8k16 k-step of P V).  Pages of 16 or 32 tokens are one visit each; pages of 8 tokens
 // come in pairs, so that a step is filled by two pages (lpf[i] = logical page | needs-mask flag of page i,
 // 0xFFFFFFFF when the visit has no page i: the odd page at the end of a piece).
+// HP = 2: the unit is a PAIR of adjacent kv heads (their blocks of a page are contiguous in the pool, so one
+// copy of twice the size brings both).  Rows of the first head take their scores from the first head's K
+// and their probabilities meet only its V; likewise for the second: two sets of MMAs, one softmax.
 #define PIE_NO_PAGE 0xFFFFFFFFu
-template <int D, int P, int PPV>
+template <int D, int P, int PPV, int HP>
 __device__ __forceinline__ void visit_compute(RowState<D>& st, uint8_t* stage, const PieReq& rq, const uint32_t* lpf,
                                               float scale_log2, int lane) {
   constexpr int KSTEPS = D / 16, VT = P * PPV, SUBS = VT / 16, BLK = P * D * 2, SLAB = P * 128, PAGE = 2 * BLK;
+  constexpr int VP = HP * PAGE;   // bytes of one page in the stage: the blocks of its HP heads
   constexpr int PIECES = P >= 16 ? 1 : 16 / P, PW = 16 / PIECES;   // a 16-token step is made of PIECES runs of PW tokens, each inside one page
   static_assert(VT % 16 == 0, "a visit is a whole number of 16-token steps");
   const int cpair = (lane & 3) * 2;
@@ -128,10 +134,12 @@ __device__ __forceinline__ void visit_compute(RowState<D>& st, uint8_t* stage, c
     if (first_bad < P) {
       constexpr int CH = D * 2 / 16;
       const int nz = (P - first_bad) * CH;
-      for (int c = lane; c < nz; c += 32) {
-        const int t = first_bad + c / CH, ch = c % CH;
-        *reinterpret_cast<uint4*>(stage + i * PAGE + BLK + pie_chunk_offset(SLAB, t, ch)) = make_uint4(0, 0, 0, 0);
-      }
+#pragma unroll
+      for (int hh = 0; hh < HP; ++hh)
+        for (int c = lane; c < nz; c += 32) {
+          const int t = first_bad + c / CH, ch = c % CH;
+          *reinterpret_cast<uint4*>(stage + i * VP + hh * PAGE + BLK + pie_chunk_offset(SLAB, t, ch)) = make_uint4(0, 0, 0, 0);
+        }
       // these generic-proxy writes must be ordered before the bulk copy that later refills the stage
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
@@ -166,19 +174,29 @@ __device__ __forceinline__ void visit_compute(RowState<D>& st, uint8_t* stage, c
     }
     if (needs_mask && __all_sync(0xFFFFFFFFu, (bits[0] | bits[1]) == 0)) continue;  // nothing visible to this warp
     // ---- S = Q K^T for 16 tokens
-    float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float sacc[2][4];
     {
+      float sh[HP][2][4];
       const int t = sub * 16 + ((lane >> 4) << 3) + (lane & 7);   // token of the visit whose K row this lane addresses
-      const uint32_t rowaddr = sbase + (t / P) * PAGE + (t % P) * 128;
+      const uint32_t rowaddr = sbase + (t / P) * VP + (t % P) * 128;
       const int csel = (lane >> 3) & 1;
 #pragma unroll
-      for (int ks = 0; ks < KSTEPS; ++ks) {
-        const int c = (ks & 3) * 2 + csel;
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(rowaddr + (ks >> 2) * SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16(sacc[0], st.qf[ks], b0, b1);
-        mma_bf16(sacc[1], st.qf[ks], b2, b3);
+      for (int hh = 0; hh < HP; ++hh) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sh[hh][0][e] = sh[hh][1][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+          const int c = (ks & 3) * 2 + csel;
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4(rowaddr + hh * PAGE + (ks >> 2) * SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
+          mma_bf16(sh[hh][0], st.qf[ks], b0, b1);
+          mma_bf16(sh[hh][1], st.qf[ks], b2, b3);
+        }
       }
+#pragma unroll
+      for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sacc[nb][e] = (HP > 1 && st.hsel[e >> 1] == 1) ? sh[HP - 1][nb][e] : sh[0][nb][e];
     }
     // ---- mask, online softmax (base-2 domain)
     float mx[2] = {kNegInf, kNegInf};
@@ -228,15 +246,23 @@ __device__ __forceinline__ void visit_compute(RowState<D>& st, uint8_t* stage, c
     // ---- O += P V
     {
       const int t = sub * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
-      const uint32_t rowaddr = sbase + (t / P) * PAGE + BLK + (t % P) * 128;
+      const uint32_t rowaddr = sbase + (t / P) * VP + BLK + (t % P) * 128;
       const int csel = lane >> 4;
 #pragma unroll
-      for (int db = 0; db < KSTEPS; ++db) {
-        const int c = (db & 3) * 2 + csel;
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4_t(rowaddr + (db >> 2) * SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16(st.o[2 * db], pa, b0, b1);
-        mma_bf16(st.o[2 * db + 1], pa, b2, b3);
+      for (int hh = 0; hh < HP; ++hh) {
+        uint32_t ph[4] = {pa[0], pa[1], pa[2], pa[3]};
+        if (HP > 1) {   // the probabilities of the other head's rows do not meet this head's V
+          if (st.hsel[0] != hh) ph[0] = ph[2] = 0u;
+          if (st.hsel[1] != hh) ph[1] = ph[3] = 0u;
+        }
+#pragma unroll
+        for (int db = 0; db < KSTEPS; ++db) {
+          const int c = (db & 3) * 2 + csel;
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(rowaddr + hh * PAGE + (db >> 2) * SLAB + ((c ^ (t & 7)) << 4), b0, b1, b2, b3);
+          mma_bf16(st.o[2 * db], ph, b0, b1);
+          mma_bf16(st.o[2 * db + 1], ph, b2, b3);
+        }
       }
     }
   }
@@ -246,7 +272,7 @@ __device__ __forceinline__ void visit_compute(RowState<D>& st, uint8_t* stage, c
 template <int D, int P>
 __device__ __forceinline__ void page_compute(RowState<D>& st, uint8_t* stage, const PieReq& rq, uint32_t lpf,
                                              float scale_log2, int lane) {
-  visit_compute<D, P, 1>(st, stage, rq, &lpf, scale_log2, lane);
+  visit_compute<D, P, 1, 1>(st, stage, rq, &lpf, scale_log2, lane);
 }
 
 // Normalise and store the warp's rows: final bf16 output + LSE, or an fp32 partial for the merge.
@@ -349,18 +375,19 @@ __device__ __forceinline__ void rows_merge_store(RowState<D>& st, const AttnPara
 // private ring and refills a stage as soon as it has consumed it: no producer warp, no empty
 // barrier, no block-level sync.  The chunk after the current one is taken a few pages early so
 // that neither the atomic nor the chunk record is ever waited for.
-template <int D, int P, int NW, int DEPTH>
+template <int D, int P, int NW, int DEPTH, int HP>
 struct SplitCfg {
   static constexpr int PPV = P == 8 ? 2 : 1;   // pages per visit: 8-token pages are handled in pairs (16 tokens fill an MMA step)
   static constexpr int PAGE = 2 * P * D * 2;   // K block + V block of one (page, kv head)
-  static constexpr int STAGE = PPV * PAGE;
+  static constexpr int VP = HP * PAGE;         // one copy: the blocks of the unit's HP adjacent kv heads of one page
+  static constexpr int STAGE = PPV * VP;
   static constexpr int QUEUE = 8;  // chunk ids a warp has started fetching but not finished (<= DEPTH + 2)
   static constexpr int SMEM = NW * DEPTH * STAGE + NW * DEPTH * (8 + 8 * PPV) + NW * QUEUE * 4 + PIE_MAX_LOCAL_GROUPS * 4 + 64;
 };
 
-template <int D, int P, int NW, int DEPTH>
+template <int D, int P, int NW, int DEPTH, int HP>
 __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams p, int n_items, int n_warps) {
-  using C = SplitCfg<D, P, NW, DEPTH>;
+  using C = SplitCfg<D, P, NW, DEPTH, HP>;
   static_assert(DEPTH + 2 <= C::QUEUE, "queue too small");
   extern __shared__ __align__(1024) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -459,11 +486,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
       meta[s * PPV + i] = i < cnt ? (uint32_t)rec[i].y : PIE_NO_PAGE;  // logical page | needs-mask flag, read back by the warp after the wait
       meta_phys[s * PPV + i] = rec[i].x;                                // physical page (the fused append writes its row back to it)
     }
-    mbar_expect_tx(smem_u32(full_bar + s), cnt * C::PAGE);
+    mbar_expect_tx(smem_u32(full_bar + s), cnt * C::VP);
 #pragma unroll
     for (int i = 0; i < PPV; ++i)
       if (i < cnt)
-        bulk_g2s(smem_u32(stages + s * C::STAGE + i * C::PAGE), p.pool + ((int64_t)rec[i].x * p.n_kv_heads + head) * C::PAGE, C::PAGE,
+        bulk_g2s(smem_u32(stages + s * C::STAGE + i * C::VP), p.pool + ((int64_t)rec[i].x * p.n_kv_heads + head * HP) * C::PAGE, C::VP,
                  smem_u32(full_bar + s));
   };
   auto load_visit = [&](int2* rec) {   // records of the visit at the prefetch cursor; returns its page count
@@ -525,15 +552,17 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
     rq.last_logical = item.last_logical;
     rq.last_page_len = item.last_page_len;
     // Fused append (decode batches): this piece ends with the request's last page, so this warp
-    // also owns the request's one new K/V row of its kv head.  The row's 16-byte chunks are
-    // fetched now (lanes [0, CH): K, [CH, 2 CH): V) and written, once the page has landed, into
-    // the staged copy and into the pool at the same offset (the stage is an image of the block).
+    // also owns the request's one new K/V row of its kv head(s).  The row's 16-byte chunks are
+    // fetched now (per head CH lanes for K, then CH for V) and written, once the page has landed, into
+    // the staged copy and into the pool at the same offset (the stage is an image of the blocks).
     constexpr int CH = D * 2 / 16;
+    static_assert(2 * CH * HP <= 32, "one lane per 16-byte chunk of the new row");
     const bool do_append = (item.flags & PIE_ITEM_APPEND) != 0;
+    const int a_head = lane / (2 * CH), a_v = (lane / CH) & 1;   // which head of the unit, K or V
     uint4 new_chunk = make_uint4(0, 0, 0, 0);
-    if (do_append && lane < 2 * CH)
-      new_chunk = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(lane < CH ? p.k_new : p.v_new) +
-                                                       ((int64_t)item.q_start * p.n_kv_heads + item.kv_head) * (D * 2)) + (lane % CH));
+    if (do_append && lane < 2 * CH * HP)
+      new_chunk = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(a_v ? p.v_new : p.k_new) +
+                                                       ((int64_t)item.q_start * p.n_kv_heads + item.kv_head * HP + a_head) * (D * 2)) + (lane % CH));
     RowState<D> st;
     rows_init<D>(st, p, item, rq, item.row0, lane);
     for (int k = item.page_begin; k < item.page_end; k += PPV, ++n) {
@@ -548,18 +577,18 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
 #pragma unroll
       for (int i = 0; i < PPV; ++i) {
         if (do_append && lpf[i] != PIE_NO_PAGE && (int)(lpf[i] & ~PIE_KEPT_NEEDS_MASK) == item.last_logical) {
-          if (lane < 2 * CH) {
-            const int off = (lane < CH ? 0 : C::PAGE / 2) + pie_chunk_offset(P * 128, item.last_page_len - 1, lane % CH);
-            *reinterpret_cast<uint4*>(stages + s * C::STAGE + i * C::PAGE + off) = new_chunk;
+          if (lane < 2 * CH * HP) {
+            const int off = a_head * C::PAGE + (a_v ? C::PAGE / 2 : 0) + pie_chunk_offset(P * 128, item.last_page_len - 1, lane % CH);
+            *reinterpret_cast<uint4*>(stages + s * C::STAGE + i * C::VP + off) = new_chunk;
             const int phys = meta_phys[s * PPV + i];
-            *reinterpret_cast<uint4*>(const_cast<uint8_t*>(p.pool) + ((int64_t)phys * p.n_kv_heads + item.kv_head) * C::PAGE + off) = new_chunk;
+            *reinterpret_cast<uint4*>(const_cast<uint8_t*>(p.pool) + ((int64_t)phys * p.n_kv_heads + item.kv_head * HP) * C::PAGE + off) = new_chunk;
           }
           // the generic-proxy write must be ordered before the bulk copy that later refills the stage
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
         }
       }
-      visit_compute<D, P, PPV>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
+      visit_compute<D, P, PPV, HP>(st, stages + s * C::STAGE, rq, lpf, p.scale_log2, lane);
       __syncwarp();
       if (pf_live) {
         if (lane == 0) issue(n + DEPTH, rec_next, cnt_next, pf_head);
@@ -951,19 +980,21 @@ AttnParams make_params(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& 
   p.page_bytes = ctx->geom.page_bytes;
   p.n_q_heads = ctx->cfg.num_q_heads;
   p.n_kv_heads = ctx->cfg.num_kv_heads;
-  p.G = ctx->G;
+  p.G_head = ctx->G;
+  p.G = ctx->G * ll.heads_per_unit;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)ctx->cfg.head_dim);
   p.late_trigger = plan->overlap ? 1 : 0;
   return p;
 }
 
-template <int D, int P, int NW, int DEPTH>
+template <int D, int P, int NW, int DEPTH, int HP = 1>
 int launch_split(pie_ctx* ctx, const AttnParams& p, int n_items, int n_warps, cudaStream_t s) {
-  using C = SplitCfg<D, P, NW, DEPTH>;
-  auto kern = attn_split_kernel<D, P, NW, DEPTH>;
-  if (!ctx->split_configured) {   // (a context has one shape, hence one instantiation, and one device)
+  using C = SplitCfg<D, P, NW, DEPTH, HP>;
+  auto kern = attn_split_kernel<D, P, NW, DEPTH, HP>;
+  bool& configured = HP == 1 ? ctx->split_configured : ctx->split_pair_configured;
+  if (!configured) {   // (a context has one shape and one device, hence one instantiation per unit width)
     PIE_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
-    ctx->split_configured = true;
+    configured = true;
   }
   const int blocks = (n_warps + NW - 1) / NW;
   PIE_CUDA(ctx, pie_launch_pdl(kern, dim3(blocks), dim3(NW * 32), C::SMEM, s, p, n_items, blocks * NW));
@@ -991,6 +1022,13 @@ bool pie_split_supported(const pie_ctx* ctx) {
          (c.head_dim == 64 || c.head_dim == 128) && ctx->G <= 16;
 }
 
+// Units of two adjacent kv heads (copies of twice the size): the shapes whose blocks are 2 or 4 KB.
+bool pie_split_pair_supported(const pie_ctx* ctx) {
+  const pie_config& c = ctx->cfg;
+  return pie_split_supported(ctx) && c.head_dim == 64 && (c.page_size == 8 || c.page_size == 16) && c.num_kv_heads % 2 == 0 &&
+         2 * ctx->G <= 16;
+}
+
 // Warps per block of the split-KV kernel (the planner sizes its shares with this).
 int pie_split_warps_per_block(const pie_ctx* ctx) {
   return (ctx->cfg.page_size == 32 && ctx->cfg.head_dim == 128) ? 4 : 8;
@@ -1004,6 +1042,11 @@ int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, const vo
   const int D = ctx->cfg.head_dim, P = ctx->cfg.page_size, n = plan->split.grid, ni = (int)plan->split.items.size();
   // ring depth: 128 - 192 KB of copies in flight per SM (measured on the 64-request decode batch with 4 KB stages:
   // depths 3 and 4 run 1.5 % faster than 5 and 6 - a deeper ring only lengthens the queue in front of every copy)
+  if (plan->split.heads_per_unit == 2) {   // units of two adjacent kv heads: copies of 8 KB instead of 4 KB (of 4 KB instead of 2 KB)
+    if (D == 64 && P == 16) return launch_split<64, 16, 8, 3, 2>(ctx, p, ni, n, s);
+    if (D == 64 && P == 8) return launch_split<64, 8, 8, 3, 2>(ctx, p, ni, n, s);
+    return PIE_ERR_UNSUPPORTED;
+  }
   if (D == 64 && P == 8) return launch_split<64, 8, 8, 4>(ctx, p, ni, n, s);     // (a visit is two pages: the same 4 / 8 KB as with 16-token pages)
   if (D == 128 && P == 8) return launch_split<128, 8, 8, 3>(ctx, p, ni, n, s);
   if (D == 64 && P == 16) return launch_split<64, 16, 8, 4>(ctx, p, ni, n, s);
@@ -1032,7 +1075,7 @@ int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll
 #define PIE_MERGE(T, DD)                                                                                                   \
   PIE_CUDA(ctx, pie_launch_pdl(tiles ? merge_tiles_kernel<T, DD> : merge_kernel<T, DD>, n, dim3(tiles ? 256 : wpb * 32), 0, s, \
                                (const PieMerge*)ll.d_merges, (const PieReq*)plan->d_reqs, (const float*)ll.d_ws_o,         \
-                               (const float*)ll.d_ws_lse, (T*)out, lse, ll.slot_rows, ctx->cfg.num_q_heads, ctx->G,        \
+                               (const float*)ll.d_ws_lse, (T*)out, lse, ll.slot_rows, ctx->cfg.num_q_heads, ctx->G * ll.heads_per_unit, \
                                (const float*)plan->tile.d_ws_o, (const float*)plan->tile.d_ws_lse, plan->tile.slot_rows))
   if (ctx->cfg.dtype == PIE_DTYPE_BF16) {
     if (D == 64) PIE_MERGE(__nv_bfloat16, 64);

@@ -95,6 +95,7 @@ struct PieLaunchList {           // one tile-kernel launch (split-KV decode, or 
   int32_t n_slots = 0;
   int32_t slot_rows = 0;
   int32_t n_static = 0;          // split-KV: items [n_static, size) are taken from the work counter
+  int32_t heads_per_unit = 1;    // split-KV: 2 = every item covers kv heads 2 kv_head and 2 kv_head + 1 (rows of the first, then of the second)
   // device copies
   PieItem* d_items = nullptr;
   int32_t* d_cta_ptr = nullptr;
@@ -181,7 +182,7 @@ struct pie_ctx {
   struct HeldPages { cudaEvent_t done; std::vector<int32_t> pages; };
   std::vector<HeldPages> held_pages;
   std::vector<cudaEvent_t> held_events;   // recycled events of held_pages
-  bool tc_configured = false, split_configured = false, tile_configured = false, nd_configured = false;   // kernel attributes set for this context's device
+  bool tc_configured = false, split_configured = false, split_pair_configured = false, tile_configured = false, nd_configured = false;   // kernel attributes set for this context's device
   // The block-local work list of the latest decode batch.  Consecutive steps of a serving loop bring the same
   // requests with the same page counts (a request grows by a page every page_size steps), and then the list is
   // the same up to the fields copied from the request records: the planner reuses it instead of dealing the
@@ -229,7 +230,9 @@ struct AttnParams {
   const void* v_new;
   int* status;
   int64_t page_bytes;
-  int32_t n_q_heads, n_kv_heads, G;
+  int32_t n_q_heads, n_kv_heads;
+  int32_t G;         // rows per query token of an item: query heads per kv head, times the kv heads of a unit
+  int32_t G_head;    // query heads per kv head
   float scale_log2;  // log2(e) / sqrt(D)
   // 1: signal dependent launches only when a block is done.  Side by side with another kernel an
   // early signal would let the NEXT kernel of the stream (a merge) occupy the SMs meant for the
@@ -251,6 +254,7 @@ int pie_launch_split(pie_ctx* ctx, const pie_plan* plan, const void* q, const vo
 int pie_launch_tiles(pie_ctx* ctx, const pie_plan* plan, const void* q, void* out, float* lse, cudaStream_t s);
 int pie_launch_merge(pie_ctx* ctx, const pie_plan* plan, const PieLaunchList& ll, void* out, float* lse, cudaStream_t s);
 bool pie_split_supported(const pie_ctx* ctx);
+bool pie_split_pair_supported(const pie_ctx* ctx);   // ... with units of two adjacent kv heads
 int pie_split_warps_per_block(const pie_ctx* ctx);
 bool pie_tc_supported(const pie_ctx* ctx);
 // n_tokens: rows of the Q tensor (the batch's query tokens), for the bounds of the Q tensor map

@@ -989,6 +989,22 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       for (int k = 0; k < cs.n; ++k) casc_of[cs.first + k] = (int32_t)c;
     }
   }
+  // Decode units of two adjacent kv heads: the two heads' blocks of a page are neighbours in the pool, so
+  // one copy of twice the size brings both, and blocks of 2 - 4 KB are fetched at a visibly lower rate than
+  // blocks of 8 KB.  Possible when the rows of both heads fit the 16 rows of a warp for every decode-shaped
+  // request of the batch (cascaded requests keep one head per unit: their shared partials are per kv head).
+  int hp = 1;
+  if (tiles_ok && pie_split_pair_supported(ctx) && cascades.empty() && !(ctx->options[PIE_OPT_NO_FUSION] & 4)) {
+    bool any = false, fits = true;
+    for (int r = 0; r < R; ++r) {
+      const PieReq& q = plan->reqs[r];
+      const int rows = q.q_len * G;
+      if (rows == 0 || q.kept_count == 0 || rows > 16) continue;
+      any = true;
+      fits = fits && 2 * rows <= 16;
+    }
+    if (any && fits) hp = 2;
+  }
   std::vector<int32_t> casc_unit0(cascades.size(), 0);  // first tile unit of every cascade
   for (int r = 0; r < R; ++r) {
     const PieReq& q = plan->reqs[r];
@@ -999,8 +1015,8 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         for (int h = 0; h < cfg.num_q_heads; ++h) plan->simple_rows.push_back((q.q_start + i) * cfg.num_q_heads + h);
     } else if (rows <= 16) {
       if (casc_of[r] < 0)
-        for (int g = 0; g < cfg.num_kv_heads; ++g)
-          split_units.push_back(Unit{r, g, 0, rows, q.kept_start, q.kept_start + q.kept_count});
+        for (int g = 0; g < cfg.num_kv_heads / hp; ++g)   // (hp = 2: g is the pair of kv heads 2g, 2g + 1; rows of the first head, then of the second)
+          split_units.push_back(Unit{r, g, 0, rows * hp, q.kept_start, q.kept_start + q.kept_count});
       // (requests of a cascade get their split units below, once the cascade's slots are known)
     } else {
       // (a request of a cascade attends only the pages behind the shared prefix here and writes a partial; the
@@ -1050,7 +1066,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       // 1 / SMs.  Take the budget that minimises the later finish, and run side by side only if that
       // beats one kernel after the other.
       double split_bytes = 0, tile_flops = 0;
-      for (const Unit& u : split_units) split_bytes += (double)(u.page_end - u.page_begin) * 2.0 * P * cfg.head_dim * 2.0;
+      for (const Unit& u : split_units) split_bytes += (double)(u.page_end - u.page_begin) * hp * 2.0 * P * cfg.head_dim * 2.0;
       for (const Cascade& cs : cascades)   // the private pages of cascaded decode-shaped requests (their split units are made below)
         for (int k = 0; k < (cs.big ? 0 : cs.n); ++k)
           split_bytes += (double)(plan->reqs[cs.first + k].kept_count - cs.L) * cfg.num_kv_heads * 2.0 * P * cfg.head_dim * 2.0;
@@ -1132,7 +1148,8 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       W += u.page_end - u.page_begin;
       max_rows = std::max(max_rows, u.nrows);
     }
-    const double kv_bytes = (double)W * 2.0 * P * cfg.head_dim * (cfg.dtype == PIE_DTYPE_BF16 ? 2.0 : 4.0);
+    plan->split.heads_per_unit = hp;
+    const double kv_bytes = (double)W * hp * 2.0 * P * cfg.head_dim * (cfg.dtype == PIE_DTYPE_BF16 ? 2.0 : 4.0);
     const bool long_launch = kv_bytes * ctx->n_sms >= 1.6e9 * split_sms;   // (fewer SMs: the same bytes take longer)
     bool plain_units = true;
     for (const Unit& u : split_units) plain_units = plain_units && !u.force_partial;
@@ -1241,6 +1258,8 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
   info.workspace_bytes = ((int64_t)plan->split.n_slots * plan->split.slot_rows +
                           (int64_t)plan->tile.n_slots * plan->tile.slot_rows) * (cfg.head_dim + 1) * 4;
   info.side_by_side_sms = plan->overlap ? plan->tile.grid : 0;
+  info.split_unit_kv_heads = plan->split.items.empty() ? 1 : plan->split.heads_per_unit;
+  info.reserved0 = 0;
   info.launches = (plan->pre_copies.empty() ? 0 : 1) + (plan->append_fused ? 0 : 1) + (info.num_simple_rows ? 1 : 0) + (info.num_split_items ? 1 : 0) +
                   (info.num_tile_items ? 1 : 0) + (plan->split.merges.empty() ? 0 : 1) +
                   (plan->tile.merges.empty() ? 0 : 1);

@@ -484,7 +484,7 @@ def test_block_local_merge_matches_oracle(sms, P):
         plan = gp.plan(wl)
         info = pie.pie_plan_get_info(plan)
         assert info["num_merge_groups"] == 0 and info["launches"] == 1        # fused append, in-kernel merge
-        assert info["num_split_items"] > wl.R * wl.H_kv                        # units were cut
+        assert info["num_split_items"] > wl.R * wl.H_kv // info["split_unit_kv_heads"]   # units were cut
         out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
         out2, lse2 = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
         assert torch.equal(out.view(torch.int16), out2.view(torch.int16)) and torch.equal(lse, lse2)
@@ -789,3 +789,50 @@ def test_a_wait_that_cannot_complete_gives_up_and_the_context_stays_usable():
         out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
         pie.pie_plan_destroy(plan)
         check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+
+
+@pytest.mark.parametrize("kv_heads_per_unit", [2, 1])
+@pytest.mark.parametrize("P", [16, 8])
+@pytest.mark.parametrize("shape", ["decode", "two_tokens_masked"])
+def test_decode_units_of_one_or_two_kv_heads_match_oracle(shape, P, kv_heads_per_unit):
+    """64-wide heads with pages of 8 or 16 tokens: by default a decode unit covers two adjacent kv heads (one copy of
+    twice the size per page; rows of the first head take K and V of the first head only, rows of the second of the
+    second), with the option bit one kv head as everywhere else.  Both against the oracle: single-token decodes
+    (the kernel also writes the new rows of both heads) and requests of two query tokens - 16 rows per pair - where
+    some carry an explicit mask with dropped earlier tokens and ragged last pages."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    from workloads import synth
+    seed = 0x5EED0 + P
+    if shape == "decode":
+        q_lens = [1] * 9
+        kv_lens = [1, 15, 16, 17, 33, 250, 511, 640, 97]
+        masks = None
+    else:
+        q_lens = [2, 1, 2, 2, 1, 2]
+        kv_lens = [2, 40, 130, 257, 16, 600]
+        masks = [None] * len(q_lens)
+        for r in (2, 3, 5):
+            ql, kl = q_lens[r], kv_lens[r]
+            pos = kl - ql + np.arange(ql)
+            causal = np.arange(kl)[None, :] <= pos[:, None]
+            drop = synth.uniform_unit(seed, 30 + r, (ql, kl)) < (0.6 if r == 5 else 0.3)
+            if r == 5:
+                drop[:, 64:192] = True                    # whole pages that no row attends to are dropped from the lists
+            masks[r] = causal & ~(drop & (np.arange(kl)[None, :] < pos[:, None]))
+    wl = configs._assemble("decode_units", seed, 32, 8, 64, P, "bf16", 512, q_lens, kv_lens, masks)
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        pie.pie_set_option(gp.ctx, pie.PIE_OPT_NO_FUSION, 0 if kv_heads_per_unit == 2 else 4)
+        gp.install(wl, poison=True)
+        plan = gp.plan(wl)
+        info = pie.pie_plan_get_info(plan)
+        assert info["split_unit_kv_heads"] == kv_heads_per_unit and info["num_tile_items"] == 0 and info["num_simple_rows"] == 0
+        assert info["launches"] == (1 if shape == "decode" else 2) + (info["num_merge_groups"] > 0)
+        out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+        pie.pie_plan_destroy(plan)
+        check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        K, V = gp.read_pages(wl.used_pages())
+        for n, pg in enumerate(wl.used_pages()):
+            Ko, Vo = pool[int(pg)]
+            assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {pg}"

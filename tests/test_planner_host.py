@@ -571,3 +571,50 @@ def test_a_request_listing_its_append_page_twice_keeps_the_append_launch(ctx):
     assert pie.pie_plan_get_info(twice)["launches"] == fused + 1
     pie.pie_plan_destroy(twice)
     pie.pie_dealloc_kvpages(ctx, ids)
+
+
+def _split_items(plan):
+    return pie.pie_plan_debug_read(plan, 4).view(np.int32).reshape(-1, 16)
+
+
+def test_decode_units_cover_two_adjacent_kv_heads_when_their_rows_fit_one_warp():
+    """With 64-wide heads and pages of 8 or 16 tokens a decode unit is a pair of adjacent kv heads (their blocks of
+    a page are neighbours in the pool: one copy of twice the size).  The pair needs both heads' rows inside the 16
+    rows of a warp for every decode-shaped request of the batch; other shapes, an odd number of kv heads, or the
+    option bit keep one kv head per unit."""
+    def units_of(P, H_q, H_kv, D, q_lens, opt=0):
+        c = pie.pie_create(64, P, H_q, H_kv, D, "bf16", 8, 64, device=-1)
+        try:
+            pie.pie_set_option(c, pie.PIE_OPT_NO_FUSION, opt)
+            ids = pie.pie_alloc_kvpages(c, 3 * len(q_lens))
+            qo = np.concatenate([[0], np.cumsum(q_lens)])
+            plan = pie.pie_plan_forward(c, qo_indptr=qo, page_indptr=3 * np.arange(len(q_lens) + 1), page_indices=ids,
+                                        last_page_len=[min(P, max(q_lens))] * len(q_lens))
+            info, items = pie.pie_plan_get_info(plan), _split_items(plan)
+            pie.pie_plan_destroy(plan)
+            return info, items
+        finally:
+            pie.pie_destroy(c)
+
+    G = 4
+    for P in (8, 16):
+        info, items = units_of(P, 32, 8, 64, [1, 1, 2])
+        assert info["split_unit_kv_heads"] == 2
+        assert set(items[:, 1].tolist()) == {0, 1, 2, 3}                     # kv head pairs
+        for it in items:
+            assert it[2] == 0 and it[3] == 2 * G * it[8]                     # rows of both heads of every query token (field 8: q_len)
+        # every (request, pair) is covered exactly once over the request's kept pages
+        for r in range(3):
+            for pair in range(4):
+                spans = sorted((it[4], it[5]) for it in items if it[0] == r and it[1] == pair)
+                assert spans[0][0] == 3 * r and spans[-1][1] == 3 * r + 3
+                assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+        info, items = units_of(P, 32, 8, 64, [1, 1, 2], opt=4)               # switched off
+        assert info["split_unit_kv_heads"] == 1 and set(items[:, 1].tolist()) == set(range(8))
+        info, items = units_of(P, 32, 8, 64, [1, 3, 2])                      # 12 rows per head: a pair would need 24
+        assert info["split_unit_kv_heads"] == 1 and items[:, 3].max() == 12
+    assert units_of(32, 32, 8, 64, [1, 1])[0]["split_unit_kv_heads"] == 1      # blocks of 8 KB already
+    assert units_of(16, 32, 8, 128, [1, 1])[0]["split_unit_kv_heads"] == 1
+    assert units_of(16, 12, 3, 64, [1, 1])[0]["split_unit_kv_heads"] == 1      # no partner for the last kv head
+    assert units_of(16, 32, 2, 64, [1, 1])[0]["split_unit_kv_heads"] == 1      # 16 query heads per kv head fill the warp
+    assert units_of(16, 16, 2, 64, [1, 1])[0]["split_unit_kv_heads"] == 2
