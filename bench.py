@@ -56,7 +56,7 @@ SUITE = ["long_context_policy", "batched_decode", "mixed_prefill_decode", "mixed
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu
 # capture per workload (not measured in this run: a profiler cannot run inside a timed benchmark)
 NCU_TRAFFIC = {
-    "batched_decode": (289_600_000, "ncu capture of the split-KV kernel on this workload, two launches"),
+    "batched_decode": (287_950_000, "ncu capture of the split-KV kernel on this workload, two launches"),
     "shared_prefix_tree": (980_300_000, "ncu capture of the row-tile kernel on this workload, two launches"),
     "mixed_prefill_decode_prefill": (82_500_000, "ncu capture of the row-tile kernel on this workload, two launches"),
     "next_dist": (16_480_000, "ncu capture of the cluster kernel on this workload, two launches"),
