@@ -173,7 +173,7 @@ PlanLayout pie_plan_layout(const pie_ctx* ctx, const pie_plan* plan) {
     L.items[k] = place(lls[k]->items.size() * sizeof(PieItem));
     L.cta[k] = place(lls[k]->cta_ptr.size() * 4);
     L.merges[k] = place(lls[k]->merges.size() * sizeof(PieMerge));
-    L.ctr[k] = place(8);
+    L.ctr[k] = place(8 + (lls[k]->grid_merge ? (size_t)lls[k]->n_slots * 4 : 0));
   }
   L.upload = off;
   const size_t D = ctx->cfg.head_dim;
@@ -205,6 +205,7 @@ void pie_plan_fill(const pie_plan* plan, const PlanLayout& L, uint8_t* dst) {
     {
       const int32_t ctr0[2] = {lls[k]->n_static, 0};  // next dynamic item, finished warps; the kernel re-arms them
       std::memcpy(dst + L.ctr[k], ctr0, 8);
+      if (lls[k]->grid_merge) std::memset(dst + L.ctr[k] + 8, 0, (size_t)lls[k]->n_slots * 4);   // pieces written so far, per group
     }
   }
 }

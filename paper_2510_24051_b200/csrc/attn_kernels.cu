@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 
 #include <cstring>
+#include <type_traits>
 
 #include "pie_internal.h"
 #include "ptx_helpers.cuh"
@@ -311,59 +312,86 @@ __device__ __forceinline__ void rows_store(RowState<D>& st, const AttnParams& p,
   }
 }
 
-// The warp holding the first piece of a block-local group: combine its own rows (still in
-// registers) with the fp32 partials of the other pieces, slots slot0 + 1 .. slot0 + np - 1, and
-// store the final rows.  lse = ln sum_c exp(lse_c), o = sum_c exp(lse_c - lse) o_c, pieces in
-// slot order (the same fixed order as the merge kernel, so results do not depend on timing).
+// In-kernel merge of fp32 partial rows by one warp (the split-KV kernel's block-local and cross-block
+// merges).  Sources: slot0, then slot0 + first, slot0 + first + stride, ... (n in all), combined in that
+// order: lse = ln sum_c exp(lse_c), o = sum_c exp(lse_c - lse) o_c - whichever warp ends up doing it reads
+// the same values in the same order, so results do not depend on timing.  dst_slot < 0: final rows (bf16
+// output and LSE); else the combination is itself a partial and goes to that slot (which may be slot0:
+// a lane reads exactly the addresses it later writes).  A merge is a handful of round trips to L2 and
+// nothing else, so the rows of kBatch sources are fetched at once, all loads issued before the first is
+// used.  Not inlined: its registers are allocated apart from the attention loop's.
+struct MergeArgs {
+  const float* ws_o;
+  const float* ws_lse;
+  float* ws_o_w;
+  float* ws_lse_w;
+  __nv_bfloat16* out;
+  float* lse;
+  int slot0, n, first, stride, dst_slot;
+  int nrows, slot_rows, row0, kv_head, G, n_q_heads, q_start;
+};
 template <int D>
-__device__ __forceinline__ void rows_merge_store(RowState<D>& st, const AttnParams& p, const PieItem& item, const PieReq& rq,
-                                                 int np, int slot_rows, int lane) {
+__device__ __noinline__ void merge_slots(const MergeArgs a, int lane) {
+  constexpr int kBatch = D == 64 ? 4 : 2;
   const int r_lo = lane >> 2, cpair = (lane & 3) * 2;
-#pragma unroll
+  auto slot_of = [&](int c) { return c == 0 ? a.slot0 : a.slot0 + a.first + a.stride * (c - 1); };
+#pragma unroll 1
   for (int r = 0; r < 2; ++r) {
-    st.l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, st.l_run[r], 1);
-    st.l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, st.l_run[r], 2);
-  }
+    const int row = r_lo + r * 8;   // row inside the unit
+    if (row >= a.nrows) continue;
+    float2 v[kBatch][D / 8];
+    float l[kBatch];
+    auto load = [&](int c0) {
 #pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    if (!st.valid[r]) continue;
-    const int row = r_lo + r * 8;   // row inside the unit (item.row0 == 0 for split-KV units)
-    const int gr = item.row0 + row;
-    const int tok = gr / p.G, head = item.kv_head * p.G + gr % p.G;
-    const float L = st.l_run[r];
-    const float inv = L > 0.f ? 1.f / L : 0.f;
-    const float lse0 = L > 0.f ? (st.m_run[r] + log2f(L)) * kLn2 : kNegInf;
-    float M = lse0;
-    for (int c = 1; c < np; ++c) M = fmaxf(M, __ldcg(p.ws_lse + (int64_t)(item.partial_slot + c) * slot_rows + row));
-    float w0 = 0.f, Z = 0.f;
-    if (M != kNegInf) w0 = __expf(lse0 - M);
-    Z = w0;
-    const float s0 = w0 * inv;      // own rows are un-normalised: weight times 1 / l
+      for (int u = 0; u < kBatch; ++u)
+        if (c0 + u < a.n) {
+          const int64_t si = (int64_t)slot_of(c0 + u) * a.slot_rows + row;
+          l[u] = __ldcg(a.ws_lse + si);
+          const float* src = a.ws_o + si * D;
 #pragma unroll
-    for (int nb = 0; nb < D / 8; ++nb) {
-      st.o[nb][2 * r] *= s0;
-      st.o[nb][2 * r + 1] *= s0;
-    }
-    for (int c = 1; c < np; ++c) {
-      const int64_t si = (int64_t)(item.partial_slot + c) * slot_rows + row;
-      float wc = 0.f;
-      if (M != kNegInf) wc = __expf(__ldcg(p.ws_lse + si) - M);
-      Z += wc;
-      const float* src = p.ws_o + si * D;
+          for (int nb = 0; nb < D / 8; ++nb) v[u][nb] = __ldcg(reinterpret_cast<const float2*>(src + nb * 8 + cpair));
+        }
+    };
+    load(0);
+    float M = kNegInf;
+#pragma unroll 4
+    for (int c = 0; c < a.n; ++c) M = fmaxf(M, __ldcg(a.ws_lse + (int64_t)slot_of(c) * a.slot_rows + row));
+    float Z = 0.f, acc[D / 8][2];
 #pragma unroll
-      for (int nb = 0; nb < D / 8; ++nb) {
-        const float2 v = __ldcg(reinterpret_cast<const float2*>(src + nb * 8 + cpair));
-        st.o[nb][2 * r] += wc * v.x;
-        st.o[nb][2 * r + 1] += wc * v.y;
-      }
+    for (int nb = 0; nb < D / 8; ++nb) acc[nb][0] = acc[nb][1] = 0.f;
+    for (int c0 = 0; c0 < a.n; c0 += kBatch) {
+      if (c0 > 0) load(c0);
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u)
+        if (c0 + u < a.n) {
+          float wc = 0.f;
+          if (M != kNegInf) wc = __expf(l[u] - M);
+          Z += wc;
+#pragma unroll
+          for (int nb = 0; nb < D / 8; ++nb) {
+            acc[nb][0] += wc * v[u][nb].x;
+            acc[nb][1] += wc * v[u][nb].y;
+          }
+        }
     }
     const float invZ = Z > 0.f ? 1.f / Z : 0.f;
-    const int64_t oi = ((int64_t)(rq.q_start + tok) * p.n_q_heads + head);
-    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + oi * D;
+    const float lse = Z > 0.f ? M + logf(Z) : kNegInf;
+    if (a.dst_slot < 0) {
+      const int gr = a.row0 + row;
+      const int tok = gr / a.G, head = a.kv_head * a.G + gr % a.G;
+      const int64_t oi = ((int64_t)(a.q_start + tok) * a.n_q_heads + head);
+      __nv_bfloat16* dst = a.out + oi * D;
 #pragma unroll
-    for (int nb = 0; nb < D / 8; ++nb)
-      *reinterpret_cast<uint32_t*>(dst + nb * 8 + cpair) = pack_bf16(st.o[nb][2 * r] * invZ, st.o[nb][2 * r + 1] * invZ);
-    if ((lane & 3) == 0) p.lse[oi] = Z > 0.f ? M + logf(Z) : kNegInf;
+      for (int nb = 0; nb < D / 8; ++nb)
+        *reinterpret_cast<uint32_t*>(dst + nb * 8 + cpair) = pack_bf16(acc[nb][0] * invZ, acc[nb][1] * invZ);
+      if ((lane & 3) == 0) a.lse[oi] = lse;
+    } else {
+      const int64_t si = (int64_t)a.dst_slot * a.slot_rows + row;
+      float* dst = a.ws_o_w + si * D;
+#pragma unroll
+      for (int nb = 0; nb < D / 8; ++nb) *reinterpret_cast<float2*>(dst + nb * 8 + cpair) = make_float2(acc[nb][0] * invZ, acc[nb][1] * invZ);
+      if ((lane & 3) == 0) a.ws_lse_w[si] = lse;
+    }
   }
 }
 
@@ -597,35 +625,65 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
         pf_settle();
       }
     }
-    if (!(item.flags & PIE_ITEM_LOCAL_PIECE)) {
-      rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);
+    const uint32_t fl = item.flags;
+    if (!(fl & (PIE_ITEM_LOCAL_PIECE | PIE_ITEM_GRID_PIECE))) {
+      rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);   // final rows, or an fp32 partial for the merge launch
     } else {
-      const int gid = (item.flags >> 8) & 0xFF, np = (item.flags >> 16) & 0xFF;
-      if (!(item.flags & PIE_ITEM_LOCAL_MERGER)) {
-        rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);   // fp32 partial
-        __threadfence_block();   // the merging warp runs on this SM: block scope is enough
-        __syncwarp();
-        if (lane == 0) atomicAdd(local_cnt + gid, 1);
-      } else {
-        // wait (bounded) until the other pieces of the group have been written
-        if (lane == 0) {
-          volatile int* cnt = local_cnt + gid;
-          uint64_t t0 = 0;
-          for (uint32_t spin = 1; *cnt < np - 1; ++spin) {
-            if ((spin & 255u) == 0) {
-              if (*reinterpret_cast<volatile int*>(p.status) != 0) break;
-              const uint64_t now = global_ns();
-              if (t0 == 0) t0 = now;
-              if (now - t0 > 1000000000ull) {
-                atomicExch(p.status, (int)PIE_ERR_DEVICE_TIMEOUT);
-                break;
+      bool block_partial = true;   // this warp writes what its block holds of the unit
+      rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);   // fp32 partial (the merging warp's own piece too)
+      MergeArgs margs;
+      margs.ws_o = p.ws_o, margs.ws_lse = p.ws_lse, margs.ws_o_w = p.ws_o, margs.ws_lse_w = p.ws_lse;
+      margs.out = reinterpret_cast<__nv_bfloat16*>(p.out), margs.lse = p.lse;
+      margs.nrows = item.nrows, margs.slot_rows = p.slot_rows, margs.row0 = item.row0, margs.kv_head = item.kv_head;
+      margs.G = p.G, margs.n_q_heads = p.n_q_heads, margs.q_start = rq.q_start;
+      if (fl & PIE_ITEM_LOCAL_PIECE) {
+        const int gid = PIE_ITEM_LOCAL_GID(fl), np = PIE_ITEM_LOCAL_NP(fl);
+        if (!(fl & PIE_ITEM_LOCAL_MERGER)) {
+          __threadfence_block();   // the merging warp runs on this SM: block scope is enough
+          __syncwarp();
+          if (lane == 0) atomicAdd(local_cnt + gid, 1);
+          block_partial = false;
+        } else {
+          // wait (bounded) until the other pieces of the group have been written
+          if (lane == 0) {
+            volatile int* cnt = local_cnt + gid;
+            uint64_t t0 = 0;
+            for (uint32_t spin = 1; *cnt < np - 1; ++spin) {
+              if ((spin & 255u) == 0) {
+                if (*reinterpret_cast<volatile int*>(p.status) != 0) break;
+                const uint64_t now = global_ns();
+                if (t0 == 0) t0 = now;
+                if (now - t0 > 1000000000ull) {
+                  atomicExch(p.status, (int)PIE_ERR_DEVICE_TIMEOUT);
+                  break;
+                }
               }
             }
           }
+          __syncwarp();
+          __threadfence_block();
+          margs.slot0 = item.partial_slot, margs.n = np, margs.first = 1, margs.stride = 1;
+          margs.dst_slot = (fl & PIE_ITEM_GRID_PIECE) ? item.partial_slot : -1;
+          merge_slots<D>(margs, lane);
         }
+      }
+      if ((fl & PIE_ITEM_GRID_PIECE) && block_partial) {
+        // make the block partial visible device-wide and count it; the warp that finds all other blocks of the
+        // unit counted combines them (no warp waits for another block)
+        const int nb = PIE_ITEM_GRID_NB(fl), kb = PIE_ITEM_GRID_KB(fl), n0 = PIE_ITEM_GRID_N0(fl);
+        const int slot0 = item.partial_slot - (kb == 0 ? 0 : n0 + NW * (kb - 1));
+        __threadfence();
         __syncwarp();
-        __threadfence_block();
-        rows_merge_store<D>(st, p, item, rq, np, p.slot_rows, lane);
+        int32_t* cnt = p.work_ctr + 2 + slot0;
+        int seen = 0;
+        if (lane == 0) seen = atomicAdd(cnt, 1);
+        seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
+        if (seen == nb - 1) {
+          __threadfence();
+          if (lane == 0) *cnt = 0;   // re-armed for the next launch
+          margs.slot0 = slot0, margs.n = nb, margs.first = n0, margs.stride = NW, margs.dst_slot = -1;
+          merge_slots<D>(margs, lane);
+        }
       }
     }
   }
@@ -753,29 +811,46 @@ __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* 
     return c < mg.nslots ? ws_o + ((int64_t)(mg.slot0 + c) * slot_rows + row) * D + lane * EPL
                          : x_ws_o + ((int64_t)(mg.x_slot0 + c - mg.nslots) * x_slot_rows + mg.x_row0 + row) * D + lane * EPL;
   };
+  // The first sources' rows are fetched together with the LSEs (their addresses need neither the
+  // maximum nor the weights), the others in batches of the same size: one round trip to memory per
+  // batch instead of one after the LSEs and then one per four sources.
+  constexpr int BATCH = 8;
+  typedef typename std::conditional<EPL == 4, float4, float2>::type Vec;
+  Vec pre[BATCH];
+#pragma unroll
+  for (int u = 0; u < BATCH; ++u)
+    if (u < ntot) pre[u] = *reinterpret_cast<const Vec*>(row_of(u));
   float M = kNegInf;
   for (int c = lane; c < ntot; c += 32) M = fmaxf(M, lse_of(c));
   for (int sft = 16; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));
   float Z = 0.f, acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  auto add = [&](float wu, const Vec& v) {
+    if constexpr (EPL == 4) acc[0] += wu * v.x, acc[1] += wu * v.y, acc[2] += wu * v.z, acc[3] += wu * v.w;
+    else acc[0] += wu * v.x, acc[1] += wu * v.y;
+  };
   for (int base = 0; base < ntot; base += 32) {
     const int c = base + lane;
     float w = 0.f;
     if (c < ntot && M != kNegInf) w = __expf(lse_of(c) - M);  // exp(-inf) = 0
     Z += w;
     const int cnt = min(32, ntot - base);
-#pragma unroll 4
-    for (int u = 0; u < cnt; ++u) {
-      const float wu = __shfl_sync(0xFFFFFFFFu, w, u);
-      const float* src = row_of(base + u);
-      if constexpr (EPL == 4) {
-        const float4 v = *reinterpret_cast<const float4*>(src);
-        acc[0] += wu * v.x, acc[1] += wu * v.y, acc[2] += wu * v.z, acc[3] += wu * v.w;
-      } else {
-        const float2 v = *reinterpret_cast<const float2*>(src);
-        acc[0] += wu * v.x, acc[1] += wu * v.y;
-      }
+    int u0 = 0;
+    if (base == 0) {
+#pragma unroll
+      for (int u = 0; u < BATCH; ++u)
+        if (u < cnt) add(__shfl_sync(0xFFFFFFFFu, w, u), pre[u]);
+      u0 = BATCH;
+    }
+    for (int ub = u0; ub < cnt; ub += BATCH) {
+      Vec v[BATCH];
+#pragma unroll
+      for (int u = 0; u < BATCH; ++u)
+        if (ub + u < cnt) v[u] = *reinterpret_cast<const Vec*>(row_of(base + ub + u));
+#pragma unroll
+      for (int u = 0; u < BATCH; ++u)
+        if (ub + u < cnt) add(__shfl_sync(0xFFFFFFFFu, w, ub + u), v[u]);
     }
   }
   for (int sft = 16; sft > 0; sft >>= 1) Z += __shfl_xor_sync(0xFFFFFFFFu, Z, sft);

@@ -62,15 +62,30 @@ static_assert(sizeof(PieItem) == 64, "PieItem is one 64-byte line");
 // The split-KV warp that owns this item also writes the request's one new K/V row (decode batches
 // whose append is fused into the attention kernel): into the pool and into its staged copy of the page.
 #define PIE_ITEM_APPEND 1u
-// Split-KV, fixed shares: a (request, kv head) cut into pieces that all belong to warps of ONE
-// thread block is merged inside the kernel.  Every piece but the first writes its fp32 partial and
-// counts itself in on a shared-memory counter (block-scope fence, no device-wide one); the warp
-// with the first piece - its last item, so it finishes last - waits for the count and combines
-// the partials with its own registers.  flags: bits 8-15 = the group's counter in the block,
-// bits 16-23 = number of pieces.
+// Split-KV, fixed shares: the pieces of a cut unit that lie in ONE thread block are merged inside the
+// kernel.  Every piece but the block's first writes its fp32 partial and counts itself in on a
+// shared-memory counter (block-scope fence, no device-wide one); the warp with the first piece - its
+// last item, so it finishes last - waits for the count and combines the partials with its own
+// registers.  PIE_ITEM_LOCAL_GID = the group's counter in the block, PIE_ITEM_LOCAL_NP = its pieces.
 #define PIE_ITEM_LOCAL_PIECE 2u
 #define PIE_ITEM_LOCAL_MERGER 4u
 #define PIE_MAX_LOCAL_GROUPS 8
+// A unit cut across thread blocks: what a block holds of it (one piece, or the combination of its
+// pieces made as above) is written as ONE fp32 partial, into the slot of the block's first piece,
+// made visible device-wide and counted on the unit's counter in global memory (behind the launch's
+// two work counters, indexed by the unit's first slot); the warp that finds all other blocks counted
+// combines the block partials in slot order.  No warp waits for another block.  PIE_ITEM_GRID_NB =
+// blocks the unit spans, PIE_ITEM_GRID_KB = index of this block among them, PIE_ITEM_GRID_N0 =
+// pieces in the first of these blocks (every block between the first and the last holds one piece
+// per warp, so block partial k > 0 sits n0 + warps_per_block (k - 1) slots behind the first).
+#define PIE_ITEM_GRID_PIECE 8u
+#define PIE_ITEM_LOCAL_GID(f) (((f) >> 4) & 7u)
+#define PIE_ITEM_LOCAL_NP(f) (((f) >> 7) & 15u)
+#define PIE_ITEM_GRID_NB(f) (((f) >> 11) & 255u)
+#define PIE_ITEM_GRID_KB(f) (((f) >> 19) & 255u)
+#define PIE_ITEM_GRID_N0(f) (((f) >> 27) & 15u)
+#define PIE_ITEM_LOCAL_BITS(gid, np) (((uint32_t)(gid) << 4) | ((uint32_t)(np) << 7))
+#define PIE_ITEM_GRID_BITS(nb, kb, n0) (((uint32_t)(nb) << 11) | ((uint32_t)(kb) << 19) | ((uint32_t)(n0) << 27))
 // Row-tile items: flags >> PIE_ITEM_CLEAN_SHIFT = number of leading pages of the item that every
 // row of the tile sees in full (no page record and no mask word needs to be looked at for them).
 #define PIE_ITEM_CLEAN_SHIFT 8
@@ -95,12 +110,13 @@ struct PieLaunchList {           // one tile-kernel launch (split-KV decode, or 
   int32_t n_slots = 0;
   int32_t slot_rows = 0;
   int32_t n_static = 0;          // split-KV: items [n_static, size) are taken from the work counter
+  bool grid_merge = false;       // split-KV: cut units are merged inside the kernel by their last piece (one counter per slot behind d_work_ctr)
   int32_t heads_per_unit = 1;    // split-KV: 2 = every item covers kv heads 2 kv_head and 2 kv_head + 1 (rows of the first, then of the second)
   // device copies
   PieItem* d_items = nullptr;
   int32_t* d_cta_ptr = nullptr;
   PieMerge* d_merges = nullptr;
-  int32_t* d_work_ctr = nullptr; // [2] dynamic-scheduling counters (split-KV kernel), zero between launches
+  int32_t* d_work_ctr = nullptr; // [2] dynamic-scheduling counters (split-KV kernel), re-armed by the kernel; then [n_slots] group counters if grid_merge
   float* d_ws_o = nullptr;       // [n_slots][slot_rows][D]
   float* d_ws_lse = nullptr;     // [n_slots][slot_rows]
 };
@@ -113,6 +129,7 @@ struct pie_plan {
   std::vector<int32_t> kept;        // pairs (phys, logical|flag)
   std::vector<int32_t> kept_scratch; // planner scratch (per-request slices before packing)
   std::vector<int32_t> clean_kept;   // [R] kept pages of the request before the first one some row sees only in part
+  std::vector<int32_t> slot_group;   // planner scratch: partial slot -> its merge group
   std::vector<int32_t> local_key;    // planner scratch: the batch's decode units as a key of the context's list cache
   // requests without output KvPages: pages of the library's own behind their page lists
   std::vector<int32_t> scratch_pages;                                   // held until the plan is destroyed or rebuilt

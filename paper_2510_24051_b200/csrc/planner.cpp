@@ -375,7 +375,7 @@ bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int m
         for (int k = 0; k < np; ++k) {
           PieItem& it = items[first_item + k];
           it.partial_slot = n_slots + k;
-          it.flags |= PIE_ITEM_LOCAL_PIECE | (k == 0 ? PIE_ITEM_LOCAL_MERGER : 0u) | ((uint32_t)local_groups << 8) | ((uint32_t)np << 16);
+          it.flags |= PIE_ITEM_LOCAL_PIECE | (k == 0 ? PIE_ITEM_LOCAL_MERGER : 0u) | PIE_ITEM_LOCAL_BITS(local_groups, np);
         }
         n_slots += np;
         ++local_groups;
@@ -1149,6 +1149,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       max_rows = std::max(max_rows, u.nrows);
     }
     plan->split.heads_per_unit = hp;
+    plan->split.grid_merge = false;
     const double kv_bytes = (double)W * hp * 2.0 * P * cfg.head_dim * (cfg.dtype == PIE_DTYPE_BF16 ? 2.0 : 4.0);
     const bool long_launch = kv_bytes * ctx->n_sms >= 1.6e9 * split_sms;   // (fewer SMs: the same bytes take longer)
     bool plain_units = true;
@@ -1201,7 +1202,71 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       if (!local && W >= (int64_t)200 * n_warps) {
         chunk_units(split_units, n_warps, plan->split);   // (many visits per warp and no balanced deal of whole units)
       } else {
-        if (!local) partition(split_units, n_warps, 4, max_rows, false, plan->split);
+        if (!local) {
+          partition(split_units, n_warps, 4, max_rows, false, plan->split);
+          // Units cut across thread blocks are merged inside the kernel too, in two levels: the pieces that lie
+          // in one block by that block (as above: shared-memory counter, the warp with the block's first piece
+          // combines them), the resulting one partial per block by whichever block writes its partial last (a
+          // device-wide fence and one atomic per block and unit, no waiting).  Both the merge launch and this
+          // cost a chain of round trips to L2 at the end of the step - about 8 us the launch, 5 - 6 us the
+          // in-kernel merge, which however sits on the critical path of every block instead of behind the
+          // last one: measured on 4 / 8 / 16 / 32 single-token requests (4 - 16 page visits per warp) 17.5 /
+          // 21.4 / 26.5 / 41.3 us against 22.7 / 26.3 / 27.1 / 39.9 us with the merge launch (attention alone:
+          // 11.6 / 14.3 / 18.6 / 33.0 us).  Taken up to 8 page visits per warp.
+          PieLaunchList& ll = plan->split;
+          bool two_level = plain && !(ctx->options[PIE_OPT_NO_FUSION] & 2) && !ll.merges.empty() && W <= (int64_t)8 * (P == 8 ? 2 : 1) * n_warps;   // (8-token pages come two per visit)
+          if (two_level) {
+            const int nw = pie_split_warps_per_block(ctx);
+            std::vector<int32_t>& scr = plan->slot_group;   // [n_slots] item of a slot, then [items] warp of an item, then [items] new flags
+            const size_t ni = ll.items.size(), ns = (size_t)ll.n_slots;
+            scr.assign(ns + 2 * ni, 0);
+            int32_t* slot_item = scr.data();
+            int32_t* item_warp = scr.data() + ns;
+            int32_t* new_flags = scr.data() + ns + ni;
+            for (int w = 0; w + 1 < (int)ll.cta_ptr.size(); ++w)
+              for (int32_t k = ll.cta_ptr[w]; k < ll.cta_ptr[w + 1]; ++k) item_warp[k] = w;
+            for (size_t k = 0; k < ni; ++k)
+              if (ll.items[k].partial_slot >= 0) slot_item[ll.items[k].partial_slot] = (int32_t)k;
+            int cur_block = -1, gids = 0;   // counters used so far in the block the walk is in (groups come in warp order)
+            for (const PieMerge& m : ll.merges) {
+              // runs of pieces that share a block
+              int nb = 0, n0 = 0;
+              for (int a = 0; a < m.nslots;) {
+                const int blk = item_warp[slot_item[m.slot0 + a]] / nw;
+                int b = a + 1;
+                while (b < m.nslots && item_warp[slot_item[m.slot0 + b]] / nw == blk) ++b;
+                if (nb == 0) n0 = b - a;
+                else if (b < m.nslots && b - a != nw) two_level = false;   // (cannot happen with contiguous shares: a block inside a unit has one piece per warp)
+                ++nb;
+                a = b;
+              }
+              if (nb > 255 || n0 > 15) two_level = false;
+              if (!two_level) break;
+              int kb = 0;
+              for (int a = 0; a < m.nslots; ++kb) {
+                const int blk = item_warp[slot_item[m.slot0 + a]] / nw;
+                int b = a + 1;
+                while (b < m.nslots && item_warp[slot_item[m.slot0 + b]] / nw == blk) ++b;
+                if (blk != cur_block) cur_block = blk, gids = 0;
+                uint32_t f = nb > 1 ? (PIE_ITEM_GRID_PIECE | PIE_ITEM_GRID_BITS(nb, kb, n0)) : 0u;
+                if (b - a > 1) {
+                  if (gids >= PIE_MAX_LOCAL_GROUPS) two_level = false;
+                  f |= PIE_ITEM_LOCAL_PIECE | PIE_ITEM_LOCAL_BITS(gids, b - a);
+                  ++gids;
+                }
+                for (int k = a; k < b; ++k)   // (only the block's first piece carries the unit-level fields)
+                  new_flags[slot_item[m.slot0 + k]] = (int32_t)(k == a ? (f | (b - a > 1 ? PIE_ITEM_LOCAL_MERGER : 0u)) : (f & ~(PIE_ITEM_GRID_PIECE | PIE_ITEM_GRID_BITS(255, 255, 15))));
+                a = b;
+              }
+              if (!two_level) break;
+            }
+            if (two_level) {
+              for (size_t k = 0; k < ni; ++k) ll.items[k].flags |= (uint32_t)new_flags[k];
+              ll.merges.clear();
+              ll.grid_merge = true;
+            }
+          }
+        }
         plan->split.n_static = (int32_t)plan->split.items.size();
       }
     }

@@ -836,3 +836,33 @@ def test_decode_units_of_one_or_two_kv_heads_match_oracle(shape, P, kv_heads_per
         for n, pg in enumerate(wl.used_pages()):
             Ko, Vo = pool[int(pg)]
             assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {pg}"
+
+
+@pytest.mark.parametrize("R,D,P,lo", [(4, 64, 16, 512), (8, 64, 8, 512), (3, 128, 16, 512), (2, 128, 32, 3900)])
+def test_very_short_decode_launches_merge_across_blocks_inside_the_kernel(R, D, P, lo):
+    """A handful of single-token requests over contexts of 512 - 4,096 tokens: every (request, kv head) unit is cut
+    across the warps of several thread blocks.  One launch: the pieces a block holds are merged by one of its warps,
+    the block partials by whichever block writes its partial last.  Against the oracle, bitwise equal from run to
+    run (the combine order is fixed), counters re-armed (the second call with the same plan), pool bit-exact."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs.batched_decode(R=R, D=D, P=P, lo=lo, num_pages=4096 * 16 // P)
+    O_ref, L_ref, pool = run_oracle(wl, poison=True)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        gp.install(wl, poison=True)
+        plan = gp.plan(wl)
+        info = pie.pie_plan_get_info(plan)
+        assert info["launches"] == 1 and info["num_merge_groups"] == 0 and info["num_split_items"] > 4 * R * wl.H_kv
+        flags = pie.pie_plan_debug_read(plan, 4).view(np.int32).reshape(-1, 16)[:, 13]
+        assert (flags & 8).any() and (flags & 4).any()
+        q, k, v = wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda")
+        out, lse = gp.forward(plan, q, k, v)
+        for _ in range(3):
+            out2, lse2 = gp.forward(plan, q, k, v)
+            assert torch.equal(out.view(torch.int16), out2.view(torch.int16)) and torch.equal(lse, lse2)
+        pie.pie_plan_destroy(plan)
+        check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
+        K, V = gp.read_pages(wl.used_pages())
+        for n, pg in enumerate(wl.used_pages()):
+            Ko, Vo = pool[int(pg)]
+            assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {pg}"

@@ -506,11 +506,12 @@ def test_decode_work_list_reused_between_steps_equals_a_fresh_plan():
     block-local work list of the previous batch.  Every such plan must be byte for byte what a new context
     produces: same batch again, every context one token longer (same pages), one request a page longer (other
     units), and back."""
-    _reused_work_list_case(configs.small("batched_decode"), 6, True)     # few thread blocks: whole units per block, merged in the block
-    _reused_work_list_case(configs.batched_decode(R=16), 0, False)        # long units on all blocks: cut across blocks, merge launch
+    _reused_work_list_case(configs.small("batched_decode"), 6, "block")   # few thread blocks: whole units per block, merged in the block
+    _reused_work_list_case(configs.batched_decode(R=8), 0, "two_level")    # few long units on all blocks, a very short launch: merged in the kernel, blocks first
+    _reused_work_list_case(configs.batched_decode(R=32), 0, "launch")      # the same with more work per warp: merge launch
 
 
-def _reused_work_list_case(wl, sms, local):
+def _reused_work_list_case(wl, sms, mode):
     P = wl.P
 
     def variants():
@@ -534,8 +535,9 @@ def _reused_work_list_case(wl, sms, local):
     def image(ctx, args):
         plan = pie.pie_plan_forward(ctx, *args)
         img, info = pie.pie_plan_debug_read(plan, 3), pie.pie_plan_get_info(plan)
+        flags = pie.pie_plan_debug_read(plan, 4).view(np.int32).reshape(-1, 16)[:, 13]
         pie.pie_plan_destroy(plan)
-        return img, info
+        return img, info, flags
 
     def new_ctx(sms):
         c = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
@@ -554,7 +556,13 @@ def _reused_work_list_case(wl, sms, local):
             got = image(ctx, args)
             assert got[1] == want[1], n
             assert np.array_equal(got[0], want[0]), n
-            assert (got[1]["num_merge_groups"] == 0) == local
+            # pieces merged by a warp of their block carry flag 2; block partials of a unit cut across blocks, merged
+            # by the block that writes its partial last, flag 8; without flags the merge launch combines the pieces
+            if mode == "launch":
+                assert got[1]["num_merge_groups"] > 0 and got[1]["launches"] == 2 and not (got[2] & 10).any()
+            else:
+                assert got[1]["num_merge_groups"] == 0 and got[1]["launches"] == 1
+                assert (got[2] & 2).any() and bool((got[2] & 8).any()) == (mode == "two_level")
     finally:
         pie.pie_destroy(ctx)
 
@@ -618,3 +626,55 @@ def test_decode_units_cover_two_adjacent_kv_heads_when_their_rows_fit_one_warp()
     assert units_of(16, 12, 3, 64, [1, 1])[0]["split_unit_kv_heads"] == 1      # no partner for the last kv head
     assert units_of(16, 32, 2, 64, [1, 1])[0]["split_unit_kv_heads"] == 1      # 16 query heads per kv head fill the warp
     assert units_of(16, 16, 2, 64, [1, 1])[0]["split_unit_kv_heads"] == 2
+
+
+def test_two_level_merge_fields_describe_the_block_partials():
+    """A very short decode launch cuts every unit across many warps of several thread blocks.  The pieces a block
+    holds are merged by the warp with the block's first piece (flags 2 / 4: counter and piece count of the group),
+    which writes ONE partial per block into that piece's slot; the unit-level fields on it (flag 8: blocks spanned,
+    index of this block, pieces in the first block) must let any block find the slots of all block partials:
+    slot0, then slot0 + n0 + 8 (k - 1)."""
+    wl = configs.batched_decode(R=4)
+    c = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+    try:
+        pie.pie_alloc_kvpages(c, wl.num_pages)
+        plan = pie.pie_plan_forward(c, wl.qo_indptr, wl.page_indptr, wl.page_indices, wl.last_page_len)
+        info, items = pie.pie_plan_get_info(plan), _split_items(plan)
+        pie.pie_plan_destroy(plan)
+    finally:
+        pie.pie_destroy(c)
+    assert info["launches"] == 1 and info["num_merge_groups"] == 0
+    NW = 8
+    units = {}
+    for it in items:
+        units.setdefault((it[0], it[1]), []).append(it)
+    n_cut = 0
+    for pieces in units.values():
+        assert all(a[5] == b[4] for a, b in zip(pieces, pieces[1:]))                 # contiguous page ranges, in order
+        if len(pieces) == 1:
+            assert pieces[0][6] == -1 and pieces[0][13] & 14 == 0
+            continue
+        n_cut += 1
+        slot0 = pieces[0][6]
+        assert [p[6] for p in pieces] == list(range(slot0, slot0 + len(pieces)))     # consecutive slots
+        # block partials: pieces with flag 8, or a lone block-local group
+        heads = [p for p in pieces if p[13] & 8]
+        if not heads:
+            f = int(pieces[0][13])
+            assert f & 2 and f & 4 and ((f >> 7) & 15) == len(pieces)
+            continue
+        nb = (int(heads[0][13]) >> 11) & 255
+        n0 = (int(heads[0][13]) >> 27) & 15
+        assert len(heads) == nb and nb > 1
+        covered = 0
+        for k, h in enumerate(heads):
+            f = int(h[13])
+            assert ((f >> 11) & 255, (f >> 19) & 255, (f >> 27) & 15) == (nb, k, n0)
+            assert h[6] == (slot0 if k == 0 else slot0 + n0 + NW * (k - 1))
+            in_block = ((f >> 7) & 15) if f & 2 else 1                               # pieces this block holds
+            assert bool(f & 4) == (in_block > 1) and in_block == (n0 if k == 0 else (NW if k + 1 < nb else in_block))
+            followers = pieces[h[6] - slot0 + 1: h[6] - slot0 + in_block]
+            assert all((int(q[13]) & 14) == 2 and ((int(q[13]) >> 4) & 7) == ((f >> 4) & 7) for q in followers)
+            covered += in_block
+        assert covered == len(pieces)
+    assert n_cut == len(units) == wl.R * wl.H_kv // 2
