@@ -290,6 +290,28 @@ class Env:
         if self.world > 1:
             self.dist.destroy_process_group()
 
+    def device_info(self):
+        """Which GPU this ran on, and its plain device-to-device copy rate right now (1 GiB, read + write
+        bytes, median of 10 after 3 untimed): context for the fractions, which are rated against the pool's
+        measured peaks - GPUs of one pool differ, on scattered page reads by more than on this copy."""
+        torch = self.torch
+        props = torch.cuda.get_device_properties(self.local)
+        x = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+        y = torch.empty_like(x)
+        ts = []
+        for i in range(13):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            y.copy_(x)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        del x, y
+        torch.cuda.empty_cache()
+        return {"name": props.name, "uuid": str(getattr(props, "uuid", "")), "sms": props.multi_processor_count,
+                "copy_gbs_now": 2 * (1 << 30) / (statistics.median(ts) * 1e-3) / 1e9}
+
 
 def timed_regions(env, step, steps, min_seconds, max_regions=4000):
     """Regions of exactly `steps` steps, each between a barrier + synchronize on both sides and timed with
@@ -743,6 +765,7 @@ def main():
     names = (SUITE if env.world == 1 else [HEADLINE]) if args.workload == "all" else [args.workload]
     entries = {}
     t_start = time.perf_counter()
+    device = env.device_info()
     for name in names:
         t0 = time.perf_counter()
         head = name == names[0]
@@ -769,6 +792,7 @@ def main():
             if env.world == 1:
                 entries["tiny_fp32"] = {"timed": False, "note": "correctness-only configuration (fp32, 4 requests): covered by the parity tests"}
             line["workloads"] = entries
+        line["device"] = device
         line["wall_seconds"] = time.perf_counter() - t_start
         print(json.dumps(line))
     env.close()

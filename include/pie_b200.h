@@ -367,7 +367,10 @@ int pie_sched_next_batch(pie_sched* s, int32_t* out_type, int32_t cap, int64_t* 
  *                      (a few requests, at most 8 page visits per warp) cut units across thread
  *                      blocks and still merge inside the kernel: every block combines what it
  *                      holds of a unit, the block that writes its partial last combines the
- *                      blocks' partials (fixed order: results do not depend on timing).  Bit 2: one kv head per
+ *                      blocks' partials (fixed order: results do not depend on timing).  Bit 3:
+ *                      partials of merges inside a thread block always go through global memory.
+ *                      By default a group whose pieces are the last work of their warps leaves
+ *                      them in the warps' idle staging buffers in shared memory.  Bit 2: one kv head per
  *                      decode unit.  By default, with 64-wide heads and pages of 8 or 16 tokens, a
  *                      unit is a pair of adjacent kv heads (one copy of twice the size per page). */
 enum { PIE_OPT_SPLIT_SMS = 0, PIE_OPT_TILE_SMS = 1, PIE_OPT_OVERLAP = 2, PIE_OPT_NO_FUSION = 3, PIE_NUM_OPTIONS = 4 };

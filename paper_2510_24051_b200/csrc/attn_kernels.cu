@@ -312,6 +312,30 @@ __device__ __forceinline__ void rows_store(RowState<D>& st, const AttnParams& p,
   }
 }
 
+// The same partial, written into shared memory (the warp's own, now idle, ring of stages) for a merge by
+// another warp of the block: [16 rows][D] fp32, then 16 LSEs.
+template <int D>
+__device__ __forceinline__ void rows_store_smem(RowState<D>& st, float* base, int lane) {
+  const int r_lo = lane >> 2, cpair = (lane & 3) * 2;
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    st.l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, st.l_run[r], 1);
+    st.l_run[r] += __shfl_xor_sync(0xFFFFFFFFu, st.l_run[r], 2);
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (!st.valid[r]) continue;
+    const int row = r_lo + r * 8;
+    const float L = st.l_run[r];
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    float* dst = base + row * D;
+#pragma unroll
+    for (int nb = 0; nb < D / 8; ++nb)
+      *reinterpret_cast<float2*>(dst + nb * 8 + cpair) = make_float2(st.o[nb][2 * r] * inv, st.o[nb][2 * r + 1] * inv);
+    if ((lane & 3) == 0) base[16 * D + row] = L > 0.f ? (st.m_run[r] + log2f(L)) * kLn2 : kNegInf;
+  }
+}
+
 // In-kernel merge of fp32 partial rows by one warp (the split-KV kernel's block-local and cross-block
 // merges).  Sources: slot0, then slot0 + first, slot0 + first + stride, ... (n in all), combined in that
 // order: lse = ln sum_c exp(lse_c), o = sum_c exp(lse_c - lse) o_c - whichever warp ends up doing it reads
@@ -329,8 +353,10 @@ struct MergeArgs {
   float* lse;
   int slot0, n, first, stride, dst_slot;
   int nrows, slot_rows, row0, kv_head, G, n_q_heads, q_start;
+  const float* sm_base;   // SMEM variant: source c is the partial that warp (own + c) left in its ring
+  int sm_stride;          // floats between the rings of consecutive warps
 };
-template <int D>
+template <int D, bool SMEM>
 __device__ __noinline__ void merge_slots(const MergeArgs a, int lane) {
   constexpr int kBatch = D == 64 ? 4 : 2;
   const int r_lo = lane >> 2, cpair = (lane & 3) * 2;
@@ -345,17 +371,25 @@ __device__ __noinline__ void merge_slots(const MergeArgs a, int lane) {
 #pragma unroll
       for (int u = 0; u < kBatch; ++u)
         if (c0 + u < a.n) {
-          const int64_t si = (int64_t)slot_of(c0 + u) * a.slot_rows + row;
-          l[u] = __ldcg(a.ws_lse + si);
-          const float* src = a.ws_o + si * D;
+          if constexpr (SMEM) {
+            const float* src = a.sm_base + (size_t)(c0 + u) * a.sm_stride;
+            l[u] = src[16 * D + row];
 #pragma unroll
-          for (int nb = 0; nb < D / 8; ++nb) v[u][nb] = __ldcg(reinterpret_cast<const float2*>(src + nb * 8 + cpair));
+            for (int nb = 0; nb < D / 8; ++nb) v[u][nb] = *reinterpret_cast<const float2*>(src + row * D + nb * 8 + cpair);
+          } else {
+            const int64_t si = (int64_t)slot_of(c0 + u) * a.slot_rows + row;
+            l[u] = __ldcg(a.ws_lse + si);
+            const float* src = a.ws_o + si * D;
+#pragma unroll
+            for (int nb = 0; nb < D / 8; ++nb) v[u][nb] = __ldcg(reinterpret_cast<const float2*>(src + nb * 8 + cpair));
+          }
         }
     };
     load(0);
     float M = kNegInf;
 #pragma unroll 4
-    for (int c = 0; c < a.n; ++c) M = fmaxf(M, __ldcg(a.ws_lse + (int64_t)slot_of(c) * a.slot_rows + row));
+    for (int c = 0; c < a.n; ++c)
+      M = fmaxf(M, SMEM ? a.sm_base[(size_t)c * a.sm_stride + 16 * D + row] : __ldcg(a.ws_lse + (int64_t)slot_of(c) * a.slot_rows + row));
     float Z = 0.f, acc[D / 8][2];
 #pragma unroll
     for (int nb = 0; nb < D / 8; ++nb) acc[nb][0] = acc[nb][1] = 0.f;
@@ -630,8 +664,14 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
       rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);   // final rows, or an fp32 partial for the merge launch
     } else {
       bool block_partial = true;   // this warp writes what its block holds of the unit
-      rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);   // fp32 partial (the merging warp's own piece too)
+      // fp32 partial (the merging warp's own piece too): in global memory, or - when this is the last item of every
+      // warp of the block-local group, so that their rings are idle - in the warp's ring, where the merging warp
+      // finds it without a round trip to L2
+      const bool in_smem = (fl & PIE_ITEM_LOCAL_SMEM) != 0;
+      if (in_smem) rows_store_smem<D>(st, reinterpret_cast<float*>(stages), lane);
+      else rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);
       MergeArgs margs;
+      margs.sm_base = reinterpret_cast<const float*>(stages), margs.sm_stride = DEPTH * C::STAGE / 4;
       margs.ws_o = p.ws_o, margs.ws_lse = p.ws_lse, margs.ws_o_w = p.ws_o, margs.ws_lse_w = p.ws_lse;
       margs.out = reinterpret_cast<__nv_bfloat16*>(p.out), margs.lse = p.lse;
       margs.nrows = item.nrows, margs.slot_rows = p.slot_rows, margs.row0 = item.row0, margs.kv_head = item.kv_head;
@@ -664,7 +704,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
           __threadfence_block();
           margs.slot0 = item.partial_slot, margs.n = np, margs.first = 1, margs.stride = 1;
           margs.dst_slot = (fl & PIE_ITEM_GRID_PIECE) ? item.partial_slot : -1;
-          merge_slots<D>(margs, lane);
+          if (in_smem) merge_slots<D, true>(margs, lane);
+          else merge_slots<D, false>(margs, lane);
         }
       }
       if ((fl & PIE_ITEM_GRID_PIECE) && block_partial) {
@@ -682,7 +723,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
           __threadfence();
           if (lane == 0) *cnt = 0;   // re-armed for the next launch
           margs.slot0 = slot0, margs.n = nb, margs.first = n0, margs.stride = NW, margs.dst_slot = -1;
-          merge_slots<D>(margs, lane);
+          merge_slots<D, false>(margs, lane);
         }
       }
     }

@@ -79,6 +79,9 @@ static_assert(sizeof(PieItem) == 64, "PieItem is one 64-byte line");
 // pieces in the first of these blocks (every block between the first and the last holds one piece
 // per warp, so block partial k > 0 sits n0 + warps_per_block (k - 1) slots behind the first).
 #define PIE_ITEM_GRID_PIECE 8u
+// A block-local group all of whose pieces are the LAST items of their warps: the partials are left in the
+// warps' own (idle) rings in shared memory instead of global memory.
+#define PIE_ITEM_LOCAL_SMEM 0x80000000u
 #define PIE_ITEM_LOCAL_GID(f) (((f) >> 4) & 7u)
 #define PIE_ITEM_LOCAL_NP(f) (((f) >> 7) & 15u)
 #define PIE_ITEM_GRID_NB(f) (((f) >> 11) & 255u)

@@ -390,6 +390,29 @@ bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int m
   return true;
 }
 
+// Block-local merge groups (PIE_ITEM_LOCAL_*) all of whose pieces are the last items of their warps leave
+// their partials in shared memory: mark them.  `ll.cta_ptr` holds one item range per warp; the pieces of a
+// group are consecutive items, the merging one first.
+void mark_smem_groups(PieLaunchList& ll) {
+  const int n_w = (int)ll.cta_ptr.size() - 1;
+  auto is_last = [&](int32_t idx, int& w) {   // (groups come in warp order: w only moves forward)
+    while (w < n_w && ll.cta_ptr[w + 1] <= idx) ++w;
+    return w < n_w && ll.cta_ptr[w + 1] == idx + 1;
+  };
+  int w = 0;
+  for (size_t k = 0; k < ll.items.size(); ++k) {
+    const uint32_t f = ll.items[k].flags;
+    if (!(f & PIE_ITEM_LOCAL_MERGER)) continue;
+    const int np = (int)PIE_ITEM_LOCAL_NP(f);
+    bool all_last = k + np <= ll.items.size();
+    int wk = w;
+    for (int c = 0; c < np && all_last; ++c) all_last = is_last((int32_t)(k + c), wk);
+    w = wk;
+    if (all_last)
+      for (int c = 0; c < np; ++c) ll.items[k + c].flags |= PIE_ITEM_LOCAL_SMEM;
+  }
+}
+
 // Split-KV decode: cut every unit into chunks that the warps of the grid take from a global
 // counter at run time.  Units in the first 80 % of the page visits get large chunks (about a
 // third of a warp's fair share), the rest small ones, and the large chunks come first in the
@@ -1187,6 +1210,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
           }
         } else {
           local = partition_local(split_units, split_sms, nw, 4, max_rows, plan->split);
+          if (local && !(ctx->options[PIE_OPT_NO_FUSION] & 8)) mark_smem_groups(plan->split);
           lc.valid = true;
           lc.balanced = local;
           lc.sms = split_sms, lc.warps = nw, lc.slot_rows = max_rows;
@@ -1264,6 +1288,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
               for (size_t k = 0; k < ni; ++k) ll.items[k].flags |= (uint32_t)new_flags[k];
               ll.merges.clear();
               ll.grid_merge = true;
+              if (!(ctx->options[PIE_OPT_NO_FUSION] & 8)) mark_smem_groups(ll);
             }
           }
         }
