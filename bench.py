@@ -116,7 +116,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+         "clocks_event_reasons.sw_power_cap,clocks.mem,clocks.max.mem,temperature.memory")
 
     def __init__(self, device):
         self.rows, self.proc, self.device = [], None, device
@@ -143,6 +143,7 @@ class ClockSampler:
         self.proc.terminate()
         self.thread.join(timeout=2)
         sm, mx, pw, reasons = [], [], [], set()
+        mem, mem_max, mem_temp = [], [], []
         for r in self.rows:
             try:
                 sm.append(float(r[0])), mx.append(float(r[1]))
@@ -152,8 +153,15 @@ class ClockSampler:
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
+            for dst, v in zip((mem, mem_max, mem_temp), r[7:10]):   # (memory clock and temperature: not every driver reports them)
+                try:
+                    dst.append(float(v))
+                except ValueError:
+                    pass
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "sm_min_mhz": min(sm) if sm else None, "power_w_max": max(pw) if pw else None,
+                "mem_mhz_min": min(mem) if mem else None, "mem_max_mhz": max(mem_max) if mem_max else None,
+                "mem_temp_c_max": max(mem_temp) if mem_temp else None,
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 

@@ -440,6 +440,8 @@ int pie_destroy(pie_ctx* ctx) {
     for (auto& h : ctx->held_pages) cudaEventDestroy(h.done);
     for (auto e : ctx->held_events) cudaEventDestroy(e);
   }
+  pie_workers_destroy(ctx->workers);
+  ctx->workers = nullptr;
   delete ctx->host_plan;
   for (pie_plan* plan : ctx->parked_plans) {
     if (!ctx->host_only) {

@@ -132,6 +132,7 @@ struct pie_plan {
   std::vector<int32_t> kept;        // pairs (phys, logical|flag)
   std::vector<int32_t> kept_scratch; // planner scratch (per-request slices before packing)
   std::vector<int32_t> clean_kept;   // [R] kept pages of the request before the first one some row sees only in part
+  std::vector<int32_t> req_note;     // planner scratch: per request, the outcome of a pass over its page list
   std::vector<int32_t> slot_group;   // planner scratch: partial slot -> its merge group
   std::vector<int32_t> local_key;    // planner scratch: the batch's decode units as a key of the context's list cache
   // requests without output KvPages: pages of the library's own behind their page lists
@@ -171,8 +172,14 @@ struct pie_plan {
 };
 
 struct pie_plan;
+// Host worker threads of a context (planner.cpp): started on the first batch that is worth them, parked on a
+// condition variable between batches, joined by pie_destroy.
+struct PieWorkers;
+void pie_workers_destroy(PieWorkers* w);
+
 struct pie_ctx {
   pie_config cfg{};
+  PieWorkers* workers = nullptr;
   PoolGeom geom{};
   int32_t G = 1;
   int32_t n_sms = 148;

@@ -7,13 +7,109 @@
 // work partition that gives every SM an equal share of page visits.
 #include <algorithm>
 #include <atomic>
+#include <chrono>
 #include <cstring>
+#include <condition_variable>
+#include <functional>
+#include <mutex>
 #include <thread>
 #if defined(__SSE2__)
 #include <emmintrin.h>
 #endif
 
 #include "pie_internal.h"
+
+// A context's worker threads: `run(n, fn)` calls fn(0) .. fn(n - 1), each once, on the calling thread and the
+// workers, and returns when all are done.  (Starting threads for every batch cost more than the packing of
+// a long-context batch's masks gained: ~0.4 ms against ~0.7 ms.)
+struct PieWorkers {
+  std::vector<std::thread> threads;
+  std::mutex m;
+  std::condition_variable wake, done;
+  const std::function<void(int)>* fn = nullptr;
+  std::atomic<int> next{0}, generation{0}, busy{0};
+  std::atomic<bool> stop{false};
+  int n_tasks = 0;
+
+  explicit PieWorkers(int n_workers) {
+    for (int t = 0; t < n_workers; ++t) threads.emplace_back([this] { loop(); });
+  }
+  ~PieWorkers() {
+    {
+      std::lock_guard<std::mutex> lk(m);
+      stop.store(true);
+    }
+    wake.notify_all();
+    for (auto& t : threads) t.join();
+  }
+  // Waiting: a short spin first (the planner calls run() several times per batch, some tens of microseconds
+  // apart: a sleeping thread takes longer than that to wake up), then the condition variable.
+  template <class Pred>
+  static bool spin_for(Pred pred) {
+    const auto t0 = std::chrono::steady_clock::now();
+    for (int k = 0;; ++k) {
+      if (pred()) return true;
+#if defined(__SSE2__)
+      _mm_pause();
+#endif
+      if ((k & 63) == 63 && std::chrono::steady_clock::now() - t0 > std::chrono::microseconds(200)) return false;
+    }
+  }
+  void drain() {
+    for (int k = next.fetch_add(1); k < n_tasks; k = next.fetch_add(1)) (*fn)(k);
+  }
+  void loop() {
+    int seen = 0;
+    for (;;) {
+      auto ready = [&] { return stop.load(std::memory_order_acquire) || generation.load(std::memory_order_acquire) != seen; };
+      if (!spin_for(ready)) {
+        std::unique_lock<std::mutex> lk(m);
+        wake.wait(lk, ready);
+      }
+      if (stop.load()) return;
+      seen = generation.load(std::memory_order_acquire);
+      drain();
+      if (busy.fetch_sub(1, std::memory_order_acq_rel) == 1) {
+        std::lock_guard<std::mutex> lk(m);
+        done.notify_one();
+      }
+    }
+  }
+  void run(int n, const std::function<void(int)>& f) {
+    fn = &f;
+    n_tasks = n;
+    next.store(0);
+    busy.store((int)threads.size());
+    {
+      std::lock_guard<std::mutex> lk(m);   // (a worker between its check and its wait holds the mutex: no wake-up is lost)
+      generation.fetch_add(1, std::memory_order_release);
+    }
+    wake.notify_all();
+    drain();
+    auto idle = [&] { return busy.load(std::memory_order_acquire) == 0; };
+    if (!spin_for(idle)) {
+      std::unique_lock<std::mutex> lk(m);
+      done.wait(lk, idle);
+    }
+  }
+};
+void pie_workers_destroy(PieWorkers* w) { delete w; }
+
+// fn(0) .. fn(n - 1): on the context's worker threads when `parallel`, else in order on this thread.
+// (Half the hardware threads, at most 8: with all of them the sibling threads of a core slow each other
+//  and the serial parts of the planner.)
+static int pie_host_threads(int n) {
+  return (int)std::min<int64_t>({(int64_t)std::max(1u, std::thread::hardware_concurrency() / 2), 8, (int64_t)n});
+}
+static void pie_run_tasks(pie_ctx* ctx, int n, bool parallel, const std::function<void(int)>& fn) {
+  const int nt = parallel ? pie_host_threads(n) : 1;
+  if (nt <= 1) {
+    for (int k = 0; k < n; ++k) fn(k);
+    return;
+  }
+  if (!ctx->workers) ctx->workers = new PieWorkers(nt - 1);
+  ctx->workers->run(n, fn);
+}
 
 namespace {
 
@@ -55,6 +151,45 @@ bool pack_row(const uint8_t* src, int64_t n, uint32_t* dst, int row_words) {
   }
   for (; k < row_words; ++k) dst[k] = 0u;
   return bad == 0;
+}
+
+// One bit per page: does the OR of all mask rows (`any_w`, `row_words` words, a multiple of four) have a bit
+// in the page's P positions?  Bits for pages [first, first + 64) (first a multiple of 64; P = 8, 16 or 32).
+// Which pages an application keeps is not predictable, so the kept-page list is built by walking the set
+// bits of these words instead of testing page after page.
+uint64_t page_any_bits(const uint32_t* any_w, int row_words, int P, int first) {
+  uint64_t out = 0;
+  const int w0 = (int)(((int64_t)first * P) >> 5), nw = 2 * P;   // 64 pages span 64 P / 32 words
+#if defined(__SSE2__)
+  const __m128i zero = _mm_setzero_si128();
+  for (int k = 0; k < nw; k += 4) {   // 128 bits: 16 / 8 / 4 pages
+    if (w0 + k + 4 > row_words) break;
+    const __m128i v = _mm_loadu_si128((const __m128i*)(any_w + w0 + k));
+    uint32_t none;
+    int per;
+    if (P == 8) {
+      none = (uint32_t)_mm_movemask_epi8(_mm_cmpeq_epi8(v, zero));
+      per = 16;
+    } else if (P == 16) {
+      const __m128i z = _mm_cmpeq_epi16(v, zero);
+      none = (uint32_t)_mm_movemask_epi8(_mm_packs_epi16(z, z)) & 0xFFu;
+      per = 8;
+    } else {
+      none = (uint32_t)_mm_movemask_ps(_mm_castsi128_ps(_mm_cmpeq_epi32(v, zero)));
+      per = 4;
+    }
+    const uint64_t some = (uint64_t)(~none & ((1u << per) - 1u));
+    out |= some << ((k / 4) * per);
+  }
+#else
+  const uint32_t full = P == 32 ? 0xFFFFFFFFu : ((1u << P) - 1u);
+  for (int i = 0; i < 64; ++i) {
+    const int64_t bit = (int64_t)(first + i) * P;
+    if ((bit >> 5) >= row_words) break;
+    if ((any_w[bit >> 5] >> (bit & 31)) & full) out |= 1ull << i;
+  }
+#endif
+  return out;
 }
 
 struct Unit {
@@ -623,21 +758,30 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
   if (T > cfg.max_query_tokens) return PIE_ERR_BATCH_TOO_LARGE;
   plan->T = T;
 
-  // ---- per-request validation
+  // ---- per-request validation (the passes over the page lists - here and in the next step - run on the
+  // context's worker threads when the batch lists many pages; the first failing request, in batch order,
+  // decides the error)
   plan->reqs.assign(R, PieReq{});
-  for (int r = 0; r < R; ++r) {
+  const bool many_pages = b->page_indptr[R] >= 65536;
+  std::vector<int32_t>& req_note = plan->req_note;
+  req_note.assign((size_t)R, PIE_OK);
+  pie_run_tasks(ctx, R, many_pages, [&](int r) {
     const int q_len = b->qo_indptr[r + 1] - b->qo_indptr[r];
     const int np = b->page_indptr[r + 1] - b->page_indptr[r];
     const int last = b->last_page_len[r];
-    if (last < 1 || last > P) return PIE_ERR_INVALID;
     const int64_t kv_len64 = (int64_t)(np - 1) * P + last;
-    if (kv_len64 > 0x3FFFFFFF) return PIE_ERR_INVALID;
-    if (kv_len64 < q_len) return PIE_ERR_INVALID;
-    if (b->out_len && (b->out_len[r] < 0 || b->out_len[r] > q_len)) return PIE_ERR_INVALID;
+    if (last < 1 || last > P || kv_len64 > 0x3FFFFFFF || kv_len64 < q_len ||
+        (b->out_len && (b->out_len[r] < 0 || b->out_len[r] > q_len))) {
+      req_note[r] = PIE_ERR_INVALID;
+      return;
+    }
     const int32_t* pages = b->page_indices + b->page_indptr[r];
     uint32_t max_id = 0;   // (negative ids wrap to large values)
     for (int k = 0; k < np; ++k) max_id = std::max(max_id, (uint32_t)pages[k]);
-    if (max_id >= (uint32_t)cfg.num_pages) return PIE_ERR_BAD_PAGE;
+    if (max_id >= (uint32_t)cfg.num_pages) {
+      req_note[r] = PIE_ERR_BAD_PAGE;
+      return;
+    }
     // (whether every page is allocated is looked up further down, in the same pass over the page lists that looks
     //  for pages another request of the batch writes: one random access per listed page instead of two)
     PieReq& q = plan->reqs[r];
@@ -646,7 +790,9 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
     q.kv_len = (int32_t)kv_len64;
     q.last_logical = np - 1;
     q.last_page_len = last;
-  }
+  });
+  for (int r = 0; r < R; ++r)
+    if (req_note[r] != PIE_OK) return req_note[r];
 
   bool cross_read = false;  // some request lists a page that another request of the batch appends to
   // ---- conflict rule: no slot is written twice, and no request reads a slot that a later request
@@ -684,12 +830,11 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         ctx->wmask[pg] |= m;
       }
     }
-    bool bad_page = false;   // (reported before a conflict, as when the pages were checked first)
-    for (int r = 0; r < R && !bad_page; ++r) {
+    // one look per listed page: allocated?  written by a request of this batch?
+    // (note bit 0: some page is not allocated; bit 1: some page the request only reads is written by somebody)
+    pie_run_tasks(ctx, R, many_pages, [&](int r) {
       const PieReq& q = plan->reqs[r];
       const int32_t* pages = b->page_indices + b->page_indptr[r];
-      // one look per listed page: allocated?  written by a request of this batch?
-      // (common case: none of the pages the request only reads is written by anybody)
       const int first_written = (q.kv_len - q.q_len) / P;
       uint8_t all_a = 0xFF, any_a = 0;
       for (int lp = 0; lp < first_written; ++lp) {
@@ -698,12 +843,20 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         any_a |= a;
       }
       for (int lp = first_written; lp <= q.last_logical; ++lp) all_a &= ctx->allocated[pages[lp]];
-      if (!(all_a & 1)) {
+      req_note[r] = ((all_a & 1) ? 0 : 1) | ((any_a & 2) ? 2 : 0);
+    });
+    bool bad_page = false;   // (reported before a conflict, as when the pages were checked first)
+    for (int r = 0; r < R && !bad_page; ++r) {
+      const PieReq& q = plan->reqs[r];
+      const int32_t* pages = b->page_indices + b->page_indptr[r];
+      const int first_written = (q.kv_len - q.q_len) / P;
+      if (req_note[r] & 1) {
         bad_page = true;
         break;
       }
       if (status != PIE_OK) continue;
-      const bool any_written = (any_a & 2) != 0;
+      // (common case: none of the pages the request only reads is written by anybody)
+      const bool any_written = (req_note[r] & 2) != 0;
       for (int lp = any_written ? 0 : first_written; lp <= q.last_logical; ++lp) {
         int32_t pg = pages[lp];
         uint32_t w = ctx->wmask[pg];
@@ -769,7 +922,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
   // "all pages kept"); the slices are then packed together in request order
   int n_threads = 1;
   if (mask_bytes_total > (4 << 20)) {
-    n_threads = (int)std::min<int64_t>({(int64_t)std::max(1u, std::thread::hardware_concurrency()), 16, (int64_t)R});
+    n_threads = pie_host_threads(R);
   }
   // (one thread: the requests are visited in order, so each writes straight behind its predecessor
   //  in the final list and nothing is packed afterwards)
@@ -822,7 +975,8 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
         }
       }
       // OR and AND of all rows, word by word (contiguous passes over the rows), then one look per page
-      std::vector<uint32_t> col(2 * (size_t)row_words);
+      static thread_local std::vector<uint32_t> col;
+      col.resize(2 * (size_t)row_words);
       uint32_t* const any_w = col.data();
       uint32_t* const all_w = col.data() + row_words;
       for (int k = 0; k < row_words; ++k) {
@@ -836,15 +990,20 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
           all_w[k] &= row[k];
         }
       }
-      for (int lp = 0; lp < np; ++lp) {
-        const int bit = lp * P;
-        const uint32_t any = (any_w[bit >> 5] >> (bit & 31)) & full_bits;
-        const uint32_t all = (all_w[bit >> 5] >> (bit & 31)) & full_bits;
-        if (!any) continue;  // no query row attends to this page: it is never fetched
-        kept[2 * nk] = pages[lp];
-        kept[2 * nk + 1] = (int32_t)((uint32_t)lp | (all == full_bits ? 0u : PIE_KEPT_NEEDS_MASK));
-        if (all != full_bits && first_flagged < 0) first_flagged = nk;
-        ++nk;
+      for (int lp0 = 0; lp0 < np; lp0 += 64) {
+        // (a page no query row attends to is never fetched: only the others are visited)
+        uint64_t some = page_any_bits(any_w, row_words, P, lp0);
+        if (np - lp0 < 64) some &= (1ull << (np - lp0)) - 1ull;
+        while (some) {
+          const int lp = lp0 + __builtin_ctzll(some);
+          some &= some - 1;
+          const int bit = lp * P;
+          const uint32_t all = (all_w[bit >> 5] >> (bit & 31)) & full_bits;
+          kept[2 * nk] = pages[lp];
+          kept[2 * nk + 1] = (int32_t)((uint32_t)lp | (all == full_bits ? 0u : PIE_KEPT_NEEDS_MASK));
+          if (all != full_bits && first_flagged < 0) first_flagged = nk;
+          ++nk;
+        }
       }
     } else {
       const int lim0 = q.kv_len - q.q_len;  // last position the first query token sees
@@ -861,17 +1020,7 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
       kept_at += (size_t)nk;
     }
   };
-  if (n_threads <= 1) {
-    for (int r = 0; r < R; ++r) do_request(r);
-  } else {
-    std::atomic<int> next{0};
-    std::vector<std::thread> pool;
-    for (int t = 0; t < n_threads; ++t)
-      pool.emplace_back([&] {
-        for (int r = next.fetch_add(1); r < R; r = next.fetch_add(1)) do_request(r);
-      });
-    for (auto& th : pool) th.join();
-  }
+  pie_run_tasks(ctx, R, n_threads > 1, do_request);
   if (bad_mask.load()) return PIE_ERR_MASK;
   if (n_threads <= 1) {
     plan->kept.resize(2 * kept_at);
