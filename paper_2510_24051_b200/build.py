@@ -18,7 +18,7 @@ OBJDIR = os.path.join(HERE, "build")
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-    "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",
+    "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr", "-Xptxas", "-v",
     "-I", INCLUDE, "-I", CSRC,
 ]
 
@@ -63,6 +63,8 @@ def build(force=False, verbose=False, extra_flags=()):
             sys.stderr.write(" ".join(cmd) + "\n" + r.stdout + r.stderr)
         if r.returncode:
             raise RuntimeError(f"nvcc failed on {src}")
+        with open(obj + ".ptxas.txt", "w") as f:   # registers, spills and stack of every kernel (kernel_resources)
+            f.write(r.stderr)
         return obj
 
     with concurrent.futures.ThreadPoolExecutor(max_workers=8) as ex:
@@ -77,6 +79,34 @@ def build(force=False, verbose=False, extra_flags=()):
     return LIB
 
 
+def kernel_resources():
+    """What ptxas reported for every kernel of the last build: {mangled name: {"registers", "spill_stores",
+    "spill_loads", "stack"}} (bytes).  A kernel of the hot path that spills is a performance bug: a merge
+    routine inlined at the end of the decode kernel's item loop once cost that loop half its speed."""
+    import re
+    out = {}
+    for src in sources():
+        path = os.path.join(OBJDIR, os.path.basename(src) + ".o.ptxas.txt")
+        if not os.path.exists(path):
+            continue
+        name = None
+        for line in open(path):
+            m = re.search(r"Compiling entry function '([^']+)'", line)
+            if m:
+                name = m.group(1)
+                out[name] = {}
+                continue
+            if name is None:
+                continue
+            m = re.search(r"(\d+) bytes stack frame, (\d+) bytes spill stores, (\d+) bytes spill loads", line)
+            if m and "stack" not in out[name]:
+                out[name].update(stack=int(m.group(1)), spill_stores=int(m.group(2)), spill_loads=int(m.group(3)))
+            m = re.search(r"Used (\d+) registers", line)
+            if m:
+                out[name]["registers"] = int(m.group(1))
+                name = None
+    return out
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv,
-                extra_flags=("-Xptxas", "-v") if "-v" in sys.argv else ()))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -343,7 +343,7 @@ __device__ __forceinline__ void rows_store_smem(RowState<D>& st, float* base, in
 // output and LSE); else the combination is itself a partial and goes to that slot (which may be slot0:
 // a lane reads exactly the addresses it later writes).  A merge is a handful of round trips to L2 and
 // nothing else, so the rows of kBatch sources are fetched at once, all loads issued before the first is
-// used.  Not inlined: its registers are allocated apart from the attention loop's.
+// used.
 struct MergeArgs {
   const float* ws_o;
   const float* ws_lse;
@@ -357,7 +357,7 @@ struct MergeArgs {
   int sm_stride;          // floats between the rings of consecutive warps
 };
 template <int D, bool SMEM>
-__device__ __noinline__ void merge_slots(const MergeArgs a, int lane) {
+__device__ __forceinline__ void merge_slots(const MergeArgs& a, int lane) {
   constexpr int kBatch = D == 64 ? 4 : 2;
   const int r_lo = lane >> 2, cpair = (lane & 3) * 2;
   auto slot_of = [&](int c) { return c == 0 ? a.slot0 : a.slot0 + a.first + a.stride * (c - 1); };
@@ -425,6 +425,66 @@ __device__ __noinline__ void merge_slots(const MergeArgs a, int lane) {
 #pragma unroll
       for (int nb = 0; nb < D / 8; ++nb) *reinterpret_cast<float2*>(dst + nb * 8 + cpair) = make_float2(acc[nb][0] * invZ, acc[nb][1] * invZ);
       if ((lane & 3) == 0) a.ws_lse_w[si] = lse;
+    }
+  }
+}
+
+// What a split-KV warp still owes for a piece of a unit that is merged inside the kernel (PIE_ITEM_LOCAL_MERGER /
+// PIE_ITEM_GRID_PIECE), once the piece's rows have been written as an fp32 partial.  It runs after the warp's
+// last item: nothing of the attention loop is live any more, so this code does not weigh on the loop's registers
+// (inlined at the end of every item it cost the loop spills and up to half its speed; as a call of its own, too).
+template <int D, int NW>
+__device__ __forceinline__ void split_piece_finish(const AttnParams& p, int item_idx, const float* ring, int ring_floats, int* local_cnt,
+                                                   int lane) {
+  const PieItem item = p.items[item_idx];
+  const uint32_t fl = item.flags;
+  MergeArgs margs;
+  margs.sm_base = ring, margs.sm_stride = ring_floats;
+  margs.ws_o = p.ws_o, margs.ws_lse = p.ws_lse, margs.ws_o_w = p.ws_o, margs.ws_lse_w = p.ws_lse;
+  margs.out = reinterpret_cast<__nv_bfloat16*>(p.out), margs.lse = p.lse;
+  margs.nrows = item.nrows, margs.slot_rows = p.slot_rows, margs.row0 = item.row0, margs.kv_head = item.kv_head;
+  margs.G = p.G, margs.n_q_heads = p.n_q_heads, margs.q_start = item.q_start;
+  if (fl & PIE_ITEM_LOCAL_MERGER) {
+    const int gid = PIE_ITEM_LOCAL_GID(fl), np = PIE_ITEM_LOCAL_NP(fl);
+    // wait (bounded) until the other pieces of the group have been written
+    if (lane == 0) {
+      volatile int* cnt = local_cnt + gid;
+      uint64_t t0 = 0;
+      for (uint32_t spin = 1; *cnt < np - 1; ++spin) {
+        if ((spin & 255u) == 0) {
+          if (*reinterpret_cast<volatile int*>(p.status) != 0) break;
+          const uint64_t now = global_ns();
+          if (t0 == 0) t0 = now;
+          if (now - t0 > 1000000000ull) {
+            atomicExch(p.status, (int)PIE_ERR_DEVICE_TIMEOUT);
+            break;
+          }
+        }
+      }
+    }
+    __syncwarp();
+    __threadfence_block();
+    margs.slot0 = item.partial_slot, margs.n = np, margs.first = 1, margs.stride = 1;
+    margs.dst_slot = (fl & PIE_ITEM_GRID_PIECE) ? item.partial_slot : -1;
+    if (fl & PIE_ITEM_LOCAL_SMEM) merge_slots<D, true>(margs, lane);
+    else merge_slots<D, false>(margs, lane);
+  }
+  if (fl & PIE_ITEM_GRID_PIECE) {
+    // make the block partial visible device-wide and count it; the warp that finds all other blocks of the
+    // unit counted combines them (no warp waits for another block)
+    const int nb = PIE_ITEM_GRID_NB(fl), kb = PIE_ITEM_GRID_KB(fl), n0 = PIE_ITEM_GRID_N0(fl);
+    const int slot0 = item.partial_slot - (kb == 0 ? 0 : n0 + NW * (kb - 1));
+    __threadfence();
+    __syncwarp();
+    int32_t* cnt = p.work_ctr + 2 + slot0;
+    int seen = 0;
+    if (lane == 0) seen = atomicAdd(cnt, 1);
+    seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
+    if (seen == nb - 1) {
+      __threadfence();
+      if (lane == 0) *cnt = 0;   // re-armed for the next launch
+      margs.slot0 = slot0, margs.n = nb, margs.first = n0, margs.stride = NW, margs.dst_slot = -1;
+      merge_slots<D, false>(margs, lane);
     }
   }
 }
@@ -599,6 +659,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
 
   // ---- consumer side
   int n = 0;  // visits consumed so far (ring position)
+  int owed0 = 0, owed1 = 0, n_owed = 0;   // items whose merge duties are carried out after the last item
   while (q_head < q_tail) {
     const int idx = queue[q_head % C::QUEUE];
     ++q_head;
@@ -659,75 +720,26 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_split_kernel(const AttnParams
         pf_settle();
       }
     }
+    // Rows out: final, or an fp32 partial - in global memory, or, for a block-local group all of whose pieces are
+    // the last items of their warps (so that their rings are idle), in the warp's ring, where the merging warp
+    // finds it without a round trip to L2.
     const uint32_t fl = item.flags;
-    if (!(fl & (PIE_ITEM_LOCAL_PIECE | PIE_ITEM_GRID_PIECE))) {
-      rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);   // final rows, or an fp32 partial for the merge launch
-    } else {
-      bool block_partial = true;   // this warp writes what its block holds of the unit
-      // fp32 partial (the merging warp's own piece too): in global memory, or - when this is the last item of every
-      // warp of the block-local group, so that their rings are idle - in the warp's ring, where the merging warp
-      // finds it without a round trip to L2
-      const bool in_smem = (fl & PIE_ITEM_LOCAL_SMEM) != 0;
-      if (in_smem) rows_store_smem<D>(st, reinterpret_cast<float*>(stages), lane);
-      else rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);
-      MergeArgs margs;
-      margs.sm_base = reinterpret_cast<const float*>(stages), margs.sm_stride = DEPTH * C::STAGE / 4;
-      margs.ws_o = p.ws_o, margs.ws_lse = p.ws_lse, margs.ws_o_w = p.ws_o, margs.ws_lse_w = p.ws_lse;
-      margs.out = reinterpret_cast<__nv_bfloat16*>(p.out), margs.lse = p.lse;
-      margs.nrows = item.nrows, margs.slot_rows = p.slot_rows, margs.row0 = item.row0, margs.kv_head = item.kv_head;
-      margs.G = p.G, margs.n_q_heads = p.n_q_heads, margs.q_start = rq.q_start;
-      if (fl & PIE_ITEM_LOCAL_PIECE) {
-        const int gid = PIE_ITEM_LOCAL_GID(fl), np = PIE_ITEM_LOCAL_NP(fl);
-        if (!(fl & PIE_ITEM_LOCAL_MERGER)) {
-          __threadfence_block();   // the merging warp runs on this SM: block scope is enough
-          __syncwarp();
-          if (lane == 0) atomicAdd(local_cnt + gid, 1);
-          block_partial = false;
-        } else {
-          // wait (bounded) until the other pieces of the group have been written
-          if (lane == 0) {
-            volatile int* cnt = local_cnt + gid;
-            uint64_t t0 = 0;
-            for (uint32_t spin = 1; *cnt < np - 1; ++spin) {
-              if ((spin & 255u) == 0) {
-                if (*reinterpret_cast<volatile int*>(p.status) != 0) break;
-                const uint64_t now = global_ns();
-                if (t0 == 0) t0 = now;
-                if (now - t0 > 1000000000ull) {
-                  atomicExch(p.status, (int)PIE_ERR_DEVICE_TIMEOUT);
-                  break;
-                }
-              }
-            }
-          }
-          __syncwarp();
-          __threadfence_block();
-          margs.slot0 = item.partial_slot, margs.n = np, margs.first = 1, margs.stride = 1;
-          margs.dst_slot = (fl & PIE_ITEM_GRID_PIECE) ? item.partial_slot : -1;
-          if (in_smem) merge_slots<D, true>(margs, lane);
-          else merge_slots<D, false>(margs, lane);
-        }
-      }
-      if ((fl & PIE_ITEM_GRID_PIECE) && block_partial) {
-        // make the block partial visible device-wide and count it; the warp that finds all other blocks of the
-        // unit counted combines them (no warp waits for another block)
-        const int nb = PIE_ITEM_GRID_NB(fl), kb = PIE_ITEM_GRID_KB(fl), n0 = PIE_ITEM_GRID_N0(fl);
-        const int slot0 = item.partial_slot - (kb == 0 ? 0 : n0 + NW * (kb - 1));
-        __threadfence();
-        __syncwarp();
-        int32_t* cnt = p.work_ctr + 2 + slot0;
-        int seen = 0;
-        if (lane == 0) seen = atomicAdd(cnt, 1);
-        seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
-        if (seen == nb - 1) {
-          __threadfence();
-          if (lane == 0) *cnt = 0;   // re-armed for the next launch
-          margs.slot0 = slot0, margs.n = nb, margs.first = n0, margs.stride = NW, margs.dst_slot = -1;
-          merge_slots<D, false>(margs, lane);
-        }
-      }
+    if (fl & PIE_ITEM_LOCAL_SMEM) rows_store_smem<D>(st, reinterpret_cast<float*>(stages), lane);
+    else rows_store<D>(st, p, item, rq, item.row0, p.slot_rows, lane);
+    if ((fl & PIE_ITEM_LOCAL_PIECE) && !(fl & PIE_ITEM_LOCAL_MERGER)) {
+      __threadfence_block();   // the merging warp runs on this SM: block scope is enough
+      __syncwarp();
+      if (lane == 0) atomicAdd(local_cnt + PIE_ITEM_LOCAL_GID(fl), 1);
+    } else if (fl & (PIE_ITEM_LOCAL_MERGER | PIE_ITEM_GRID_PIECE)) {
+      // merging and cross-block counting wait until the warp has no item left (at most two pieces per warp owe
+      // any: the one that ends a unit begun in an earlier block, and the warp's last item)
+      if (n_owed == 0) owed0 = idx;
+      else owed1 = idx;
+      ++n_owed;
     }
   }
+  if (n_owed > 0) split_piece_finish<D, NW>(p, owed0, reinterpret_cast<const float*>(stages), DEPTH * C::STAGE / 4, local_cnt, lane);
+  if (n_owed > 1) split_piece_finish<D, NW>(p, owed1, reinterpret_cast<const float*>(stages), DEPTH * C::STAGE / 4, local_cnt, lane);
 
   if (p.late_trigger) pie_pdl_launch_dependents();
   // ---- the last warp of the grid to finish re-arms the counters for the next launch
