@@ -301,7 +301,7 @@ class Env:
     def device_info(self):
         """Which GPU this ran on, and its plain device-to-device copy rate right now (1 GiB, read + write
         bytes, median of 10 after 3 untimed): context for the fractions, which are rated against the pool's
-        measured peaks - GPUs of one pool differ, on scattered page reads by more than on this copy."""
+        measured peaks."""
         torch = self.torch
         props = torch.cuda.get_device_properties(self.local)
         x = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
