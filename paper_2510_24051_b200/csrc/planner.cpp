@@ -96,10 +96,10 @@ struct PieWorkers {
 void pie_workers_destroy(PieWorkers* w) { delete w; }
 
 // fn(0) .. fn(n - 1): on the context's worker threads when `parallel`, else in order on this thread.
-// (Half the hardware threads, at most 8: with all of them the sibling threads of a core slow each other
+// (Half the hardware threads, at most 16: with all of them the sibling threads of a core slow each other
 //  and the serial parts of the planner.)
 static int pie_host_threads(int n) {
-  return (int)std::min<int64_t>({(int64_t)std::max(1u, std::thread::hardware_concurrency() / 2), 8, (int64_t)n});
+  return (int)std::min<int64_t>({(int64_t)std::max(1u, std::thread::hardware_concurrency() / 2), 16, (int64_t)n});
 }
 static void pie_run_tasks(pie_ctx* ctx, int n, bool parallel, const std::function<void(int)>& fn) {
   const int nt = parallel ? pie_host_threads(n) : 1;
