@@ -867,7 +867,7 @@ __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* 
   // The first sources' rows are fetched together with the LSEs (their addresses need neither the
   // maximum nor the weights), the others in batches of the same size: one round trip to memory per
   // batch instead of one after the LSEs and then one per four sources.
-  constexpr int BATCH = 8;
+  constexpr int BATCH = EPL == 4 ? 4 : 8;   // (16 registers of loads in flight: more would cost large merge grids their occupancy)
   typedef typename std::conditional<EPL == 4, float4, float2>::type Vec;
   Vec pre[BATCH];
 #pragma unroll
