@@ -369,9 +369,15 @@ bool partition_local(const std::vector<Unit>& units, int ctas_max, int NW, int m
     return true;
   }
   auto size_of = [&](int32_t k) { return (int64_t)std::max(1, units[k].page_end - units[k].page_begin); };
-  int64_t W = 0;
-  for (size_t k = 0; k < units.size(); ++k) W += size_of((int32_t)k);
+  int64_t W = 0, largest = 0;
+  for (size_t k = 0; k < units.size(); ++k) {
+    W += size_of((int32_t)k);
+    largest = std::max(largest, size_of((int32_t)k));
+  }
   const int n_ctas = (int)std::min<int64_t>(ctas_max, std::max<int64_t>(1, W / std::max(1, min_pages_per_warp * NW)));
+  // (some block holds the largest unit whole: when that alone is beyond what the test at the end accepts, there is
+  //  nothing to deal - the common case of a few long requests)
+  if (largest * n_ctas * 100 > W * 108 && largest > W / n_ctas + 100) return false;
   // Largest first.  Units arrive in runs of equal size (the kv heads of one request), so the runs
   // are sorted, not the units: equivalent to a stable sort of the units by size, descending.
   const int n_units = (int)units.size();
