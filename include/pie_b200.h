@@ -363,9 +363,9 @@ int pie_sched_next_batch(pie_sched* s, int32_t* out_type, int32_t cap, int64_t* 
  *                      page another one appends to) lets the attention kernel write the new K/V
  *                      rows itself.  Bit 1: always merge split partials with the merge kernel.  By
  *                      default short decode launches keep all pieces of a (request, kv head)
- *                      inside one thread block, which merges them itself, and very short ones
- *                      (a few requests, at most 8 page visits per warp) cut units across thread
- *                      blocks and still merge inside the kernel: every block combines what it
+ *                      inside one thread block, which merges them itself, and those where whole
+ *                      units cannot fill the blocks evenly (a few long requests) cut units across
+ *                      thread blocks and still merge inside the kernel: every block combines what it
  *                      holds of a unit, the block that writes its partial last combines the
  *                      blocks' partials (fixed order: results do not depend on timing).  Bit 3:
  *                      partials of merges inside a thread block always go through global memory.

@@ -1386,14 +1386,12 @@ static int build_plan_core(pie_ctx* ctx, const pie_batch_desc* b, pie_plan* plan
           // Units cut across thread blocks are merged inside the kernel too, in two levels: the pieces that lie
           // in one block by that block (as above: shared-memory counter, the warp with the block's first piece
           // combines them), the resulting one partial per block by whichever block writes its partial last (a
-          // device-wide fence and one atomic per block and unit, no waiting).  Both the merge launch and this
-          // cost a chain of round trips to L2 at the end of the step - about 8 us the launch, 5 - 6 us the
-          // in-kernel merge, which however sits on the critical path of every block instead of behind the
-          // last one: measured on 4 / 8 / 16 / 32 single-token requests (4 - 16 page visits per warp) 17.5 /
-          // 21.4 / 26.5 / 41.3 us against 22.7 / 26.3 / 27.1 / 39.9 us with the merge launch (attention alone:
-          // 11.6 / 14.3 / 18.6 / 33.0 us).  Taken up to 8 page visits per warp.
+          // device-wide fence and one atomic per block and unit, no waiting).  Measured against the merge launch on
+          // 4 / 8 / 16 / 24 / 32 single-token requests of 512 - 4,096 tokens (4 - 16 page visits per warp): 17.3 / 21.3 /
+          // 24.2 / 31.2 / 39.0 us against 22.9 / 25.9 / 27.0 / 32.8 / 39.8 us; 8 requests of 8 - 16 k tokens 41.9
+          // against 47.3 us (attention alone: 11.6 / 14.3 / 18.6 us for 4 / 8 / 16 requests).
           PieLaunchList& ll = plan->split;
-          bool two_level = plain && !(ctx->options[PIE_OPT_NO_FUSION] & 2) && !ll.merges.empty() && W <= (int64_t)8 * (P == 8 ? 2 : 1) * n_warps;   // (8-token pages come two per visit)
+          bool two_level = plain && !(ctx->options[PIE_OPT_NO_FUSION] & 2) && !ll.merges.empty();   // (8-token pages come two per visit)
           if (two_level) {
             const int nw = pie_split_warps_per_block(ctx);
             std::vector<int32_t>& scr = plan->slot_group;   // [n_slots] item of a slot, then [items] warp of an item, then [items] new flags

@@ -507,8 +507,9 @@ def test_decode_work_list_reused_between_steps_equals_a_fresh_plan():
     produces: same batch again, every context one token longer (same pages), one request a page longer (other
     units), and back."""
     _reused_work_list_case(configs.small("batched_decode"), 6, "block")   # few thread blocks: whole units per block, merged in the block
-    _reused_work_list_case(configs.batched_decode(R=8), 0, "two_level")    # few long units on all blocks, a very short launch: merged in the kernel, blocks first
-    _reused_work_list_case(configs.batched_decode(R=32), 0, "launch")      # the same with more work per warp: merge launch
+    _reused_work_list_case(configs.batched_decode(R=8), 0, "two_level")    # few long units on all blocks: merged in the kernel, blocks first
+    _reused_work_list_case(configs.batched_decode(R=32), 0, "two_level")
+    _reused_work_list_case(configs.batched_decode(R=32), 0, "launch")      # the same with in-kernel merges switched off: merge launch
 
 
 def _reused_work_list_case(wl, sms, mode):
@@ -542,6 +543,7 @@ def _reused_work_list_case(wl, sms, mode):
     def new_ctx(sms):
         c = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
         pie.pie_set_option(c, pie.PIE_OPT_SPLIT_SMS, sms)
+        pie.pie_set_option(c, pie.PIE_OPT_NO_FUSION, 2 if mode == "launch" else 0)
         pie.pie_alloc_kvpages(c, wl.num_pages)
         return c
 

@@ -14,13 +14,15 @@ import torch
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["batched_decode", "long_context_policy", "mixed_prefill_decode"])
+@pytest.mark.parametrize("name", ["batched_decode", "long_context_policy", "mixed_prefill_decode", "four_long_decodes"])
 def test_static_scratch_forward_matches_planned_forward(name):
     import paper_2510_24051_b200 as pie
     from tests._gpu import GpuPool, check_close
     from tests._util import run_oracle
     from workloads import configs
-    wl = configs.small(name)
+    # (four_long_decodes: units cut across thread blocks and merged inside the kernel - the counters of that merge
+    #  live in the scratch too, re-armed by the kernel and overwritten by the next call's upload)
+    wl = configs.batched_decode(R=4, num_pages=4096) if name == "four_long_decodes" else configs.small(name)
     O_ref, L_ref, _ = run_oracle(wl)
     with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
         gp.install(wl)
