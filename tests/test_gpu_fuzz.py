@@ -49,13 +49,60 @@ def _random_batch(seed):
     return P, H_q, H_kv, D, seqs, np.array(out_len, dtype=np.int32)
 
 
+def _random_decode_batch(seed):
+    """Decode-shaped batches only (one or two new tokens per request, contexts up to 6,000 tokens, 1 - 24 requests):
+    what the split-KV kernel's planner variants see - units of one or two kv heads, whole units per thread block with
+    merges inside the block, units cut across blocks with the two-level merge, the kernel writing the new rows."""
+    from tests.test_gpu_matrix import _bf16_round
+    rng = np.random.RandomState(5000 + seed)
+    P = int(rng.choice([8, 16, 32]))
+    H_q, H_kv = [(8, 2), (32, 8), (4, 4), (16, 2), (16, 1), (12, 4)][rng.randint(6)]
+    D = int(rng.choice([64, 128]))
+    R = int(rng.choice([1, 2, 3, 5, 8, 13, 24]))
+    two = rng.rand() < 0.3                       # some batches bring two tokens per request (no fused append then)
+    long_ctx = 6000 if R <= 5 else 1500
+    seqs = []
+    for r in range(R):
+        q_len = 2 if two and rng.rand() < 0.5 else 1
+        ctx = int(rng.randint(0, long_ctx))
+        kv_len = ctx + q_len
+        pos = kv_len - q_len + np.arange(q_len)
+        form = rng.choice(["inferred", "pages", "tokens"], p=[0.6, 0.25, 0.15])
+        mask = None
+        if form != "inferred":
+            mask = np.arange(kv_len)[None, :] <= pos[:, None]
+            npg = (kv_len + P - 1) // P
+            if form == "pages" and npg > 2:
+                for pg in rng.choice(npg - 1, size=max(1, npg // 3), replace=False):
+                    mask[:, pg * P:(pg + 1) * P] = False
+            elif form == "tokens":
+                mask &= rng.rand(q_len, kv_len) < 0.7
+            mask[np.arange(q_len), pos] = True
+        s = dict(Q=_bf16_round(rng.randn(q_len, H_q, D).astype(np.float32)),
+                 K=_bf16_round(rng.randn(kv_len, H_kv, D).astype(np.float32)),
+                 V=_bf16_round(rng.randn(kv_len, H_kv, D).astype(np.float32)))
+        if mask is not None:
+            s["mask"] = mask
+        seqs.append(s)
+    return P, H_q, H_kv, D, seqs, np.array([len(s["Q"]) for s in seqs], dtype=np.int32)
+
+
+@pytest.mark.parametrize("seed", range(14))
+def test_random_decode_batches_match_oracle(seed):
+    _run_random_batch(seed, _random_decode_batch(seed), decode_only=True)
+
+
 @pytest.mark.parametrize("seed", range(16))
 def test_random_batches_match_oracle(seed):
+    _run_random_batch(seed, _random_batch(seed))
+
+
+def _run_random_batch(seed, batch, decode_only=False):
     import paper_2510_24051_b200 as pie
     from oracle import pie_oracle as orc
     from tests._gpu import TOL_LSE, TOL_O
     from tests._util import SmallBatch, same_bits
-    P, H_q, H_kv, D, seqs, out_len = _random_batch(seed)
+    P, H_q, H_kv, D, seqs, out_len = batch
     args = SmallBatch(seqs, H_q).paged(P, "random", seed=seed)
     total = len(args["pool"])
     pool_ref = {p: (a.copy(), b.copy()) for p, (a, b) in args["pool"].items()}
@@ -67,13 +114,16 @@ def test_random_batches_match_oracle(seed):
         ptr[r + 1] = ptr[r] + (0 if m is None else m.size)
     given = [m.reshape(-1).astype(np.uint8) for m in args["masks"] if m is not None]
     buf = np.concatenate(given) if given else np.zeros(0, np.uint8)
-    runs = [("bf16", 0), ("bf16", pie.PIE_PLAN_NO_TENSOR_TILES), ("bf16", pie.PIE_PLAN_FORCE_SIMPLE)]
+    runs = [("bf16", 0, 0), ("bf16", pie.PIE_PLAN_NO_TENSOR_TILES, 0), ("bf16", pie.PIE_PLAN_FORCE_SIMPLE, 0)]
+    if decode_only:   # default fusions, then each switched off: append launch, merge launch, one kv head per unit, partials in global memory
+        runs = [("bf16", 0, 0), ("bf16", 0, 1 | 2), ("bf16", 0, 4 | 8)]
     if seed % 4 == 3:
-        runs.append(("f32", 0))          # the same values in an fp32 pool (the plain kernel), at the fp32 tolerance
-    for dtype, flags in runs:
+        runs.append(("f32", 0, 0))       # the same values in an fp32 pool (the plain kernel), at the fp32 tolerance
+    for dtype, flags, no_fusion in runs:
         tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
         ctx = pie.pie_create(total, P, H_q, H_kv, D, dtype, len(seqs), T, 0)
         try:
+            pie.pie_set_option(ctx, pie.PIE_OPT_NO_FUSION, no_fusion)
             ids = pie.pie_alloc_kvpages(ctx, total)
             K = torch.from_numpy(np.stack([args["pool"][int(p)][0] for p in ids])).to(tdt).cuda()
             V = torch.from_numpy(np.stack([args["pool"][int(p)][1] for p in ids])).to(tdt).cuda()
