@@ -90,9 +90,13 @@ def test_conflict_rule(ctx):
     assert status_of(pie.pie_copy_kvpage, ctx, [ids[0]], [200], [0], [0], [8]) == pie.PIE_ERR_BAD_PAGE
 
 
-@pytest.mark.parametrize("name", ["tiny_fp32", "shared_prefix_tree", "long_context_policy", "mixed_prefill_decode"])
+@pytest.mark.parametrize("name", ["tiny_fp32", "shared_prefix_tree", "long_context_policy", "mixed_prefill_decode",
+                                  "long_context_policy_full", "long_context_policy_p8", "long_context_policy_p32"])
 def test_plan_arrays_match_numpy(name):
-    wl = configs.small(name)
+    # (the full-size batches list enough pages and mask bytes for the planner's worker threads, and walk the
+    #  one-bit-per-page words of all three page sizes)
+    big = {"long_context_policy_full": dict(), "long_context_policy_p8": dict(R=64, P=8), "long_context_policy_p32": dict(P=32)}
+    wl = configs.long_context_policy(**big[name]) if name in big else configs.small(name)
     ctx = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
     try:
         pie.pie_alloc_kvpages(ctx, wl.num_pages)
