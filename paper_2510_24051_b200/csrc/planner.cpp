@@ -307,11 +307,19 @@ contiguous:
     }
   };
   int c = 0;                                             // share that holds the walk's position
-  int64_t c_end = grid == 1 ? W : W / grid;              // its end
+  // end of share c = floor((c + 1) W / grid) = (c + 1) q + floor((c + 1) r / grid): stepped, one division per list
+  const int64_t q_share = W / grid, r_share = W % grid;
+  int64_t c_end = grid == 1 ? W : q_share, acc = r_share;
   auto advance_to = [&](int64_t x) {                     // make c the share that holds page visit x
     while (c + 1 < grid && x >= c_end) {
       ++c;
-      c_end = (c + 1 == grid) ? W : ((int64_t)(c + 1) * W) / grid;
+      acc += r_share;
+      c_end += q_share;
+      if (acc >= grid) {
+        acc -= grid;
+        ++c_end;
+      }
+      if (c + 1 == grid) c_end = W;
     }
   };
   int64_t off = 0;
