@@ -684,3 +684,37 @@ def test_two_level_merge_fields_describe_the_block_partials():
             covered += in_block
         assert covered == len(pieces)
     assert n_cut == len(units) == wl.R * wl.H_kv // 2
+
+
+def test_worker_threads_come_and_go_with_their_context():
+    """A batch with many listed pages starts the context's planner threads; pie_destroy joins them.  Many contexts
+    in a row (and two alive at once) plan the same batch to the same bytes, with and without having planned a small
+    batch - which runs on the calling thread alone - in between."""
+    wl = configs.long_context_policy(R=96)
+    small = configs.small("batched_decode")
+    mi, mb = wl.mask_bytes()
+
+    def image(c, w, masks=(None, None)):
+        plan = pie.pie_plan_forward(c, w.qo_indptr, w.page_indptr, w.page_indices, w.last_page_len, *masks)
+        img = pie.pie_plan_debug_read(plan, 3).copy()
+        pie.pie_plan_destroy(plan)
+        return img
+
+    want = None
+    keep = None
+    for k in range(12):
+        c = pie.pie_create(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype, wl.R, wl.T, device=-1)
+        pie.pie_alloc_kvpages(c, wl.num_pages)
+        if k % 3 == 1:
+            image(c, small)
+        got = image(c, wl, (mi, mb))
+        if want is None:
+            want = got
+        assert np.array_equal(got, want), k
+        assert np.array_equal(image(c, wl, (mi, mb)), want), k      # recycled plan, parked workers woken again
+        if k == 4:
+            keep = c                                                 # stays alive next to the following contexts
+        else:
+            pie.pie_destroy(c)
+    assert np.array_equal(image(keep, wl, (mi, mb)), want)
+    pie.pie_destroy(keep)
