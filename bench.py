@@ -393,9 +393,16 @@ def e2e_decode_loop(env, args, name, wl0, ctx, hbuf, step_ms):
         batches = [streams[s % n_streams][1][s // n_streams] for s in range(n_steps)]
         how = f"decode loop: {n_streams} independent loops of {wl0.R} requests visited in turn, one token appended per visit"
     else:
-        total = wl0.meta.get("pages_in_lists", len(wl0.page_indices))
+        # pages the loop may grow into: those of the pool that the batch does not hold (lists may share pages)
+        taken = np.zeros(wl0.num_pages, dtype=bool)
+        taken[np.asarray(wl0.page_indices)] = True
+        total = wl0.meta.get("pages_in_lists", 0)     # (the long-context batch lists only its kept pages: all of a request's pages are its own)
         perm = synth.permutation(wl0.seed, 10, wl0.num_pages)
-        spare = perm[total + (wl0.R if wl0.copies is not None else 0):]
+        taken[perm[:total + (wl0.R if wl0.copies is not None else 0)]] = True
+        if wl0.copies is not None:
+            taken[np.asarray(wl0.copies["dst"])] = True
+        spare = perm[~taken[perm]]
+        n_steps = min(n_steps, max(3, (len(spare) // max(wl0.R, 1)) * wl0.P - wl0.P))   # (never more page crossings than spare pages)
         batches = configs.decode_loop(wl0, n_steps, spare)
         how = f"decode loop: one token appended to each of the {wl0.R} requests per step"
 
