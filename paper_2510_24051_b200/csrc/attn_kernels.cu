@@ -918,16 +918,17 @@ __global__ void merge_kernel(const PieMerge* __restrict__ merges, const PieReq* 
 
 // The same for groups of row-tile partials (up to 256 rows per group, few sources each: the pieces of a cut unit,
 // or a request's private part plus the shared-prefix cascade).  One thread block per group, its record read
-// once; every warp takes four rows at a time: lane 8 k + c fetches the LSE of (row k, source c) while every lane
-// already fetches its columns of all sources of the four rows - one round trip to memory per four rows instead
-// of a chain of four per row.  Sources are combined in slot order (own slots, then the cascade's), as above.
+// once; every warp takes eight rows at a time (four when there are three or four sources): one lane per (row,
+// source) pair fetches the pair's LSE while every lane already fetches its columns of all sources of those rows -
+// one round trip to memory per eight rows instead of a chain of four per row.  Sources are combined in slot order
+// (own slots, then the cascade's), as above.
 template <typename T, int D>
 __global__ void __launch_bounds__(256) merge_tiles_kernel(const PieMerge* __restrict__ merges, const PieReq* __restrict__ reqs,
                                                           const float* __restrict__ ws_o, const float* __restrict__ ws_lse,
                                                           T* __restrict__ out, float* __restrict__ lse_out, int slot_rows,
                                                           int n_q_heads, int G, const float* __restrict__ x_ws_o,
                                                           const float* __restrict__ x_ws_lse, int x_slot_rows) {
-  constexpr int EPL = D / 32, RPW = 4, MAXS = 4;
+  constexpr int EPL = D / 32;
   pie_pdl_launch_dependents();
   pie_pdl_wait();
   const PieMerge mg = merges[blockIdx.x];
@@ -951,14 +952,17 @@ __global__ void __launch_bounds__(256) merge_tiles_kernel(const PieMerge* __rest
     for (int e = 0; e < EPL; ++e) out[oi * D + lane * EPL + e] = (T)(acc[e] * inv);
     if (lane == 0) lse_out[oi] = Z > 0.f ? M + logf(Z) : kNegInf;
   };
-  for (int row0 = warp * RPW; row0 < mg.nrows; row0 += (blockDim.x >> 5) * RPW) {
-    const int nr = min(RPW, mg.nrows - row0);   // (warp uniform)
-    if (ntot <= MAXS) {
-      float v[RPW][MAXS][EPL];
+  // Few sources: RPW rows per warp and step, 32 / RPW lanes per row fetch the row's LSEs (one per source).
+  auto run_few = [&](auto rpw_c, auto ns_c) {
+    constexpr int RPW = decltype(rpw_c)::value, NS = decltype(ns_c)::value, LPR = 32 / RPW;
+    static_assert(NS <= LPR, "one lane per (row, source) pair");
+    for (int row0 = warp * RPW; row0 < mg.nrows; row0 += (blockDim.x >> 5) * RPW) {
+      const int nr = min(RPW, mg.nrows - row0);   // (warp uniform)
+      float v[RPW][NS][EPL];
 #pragma unroll
       for (int k = 0; k < RPW; ++k)
 #pragma unroll
-        for (int c = 0; c < MAXS; ++c) {
+        for (int c = 0; c < NS; ++c) {
           if (k < nr && c < ntot) {
             const float* src = row_at(c, row0 + k);
             if constexpr (EPL == 4) {
@@ -973,11 +977,12 @@ __global__ void __launch_bounds__(256) merge_tiles_kernel(const PieMerge* __rest
             for (int e = 0; e < EPL; ++e) v[k][c][e] = 0.f;
           }
         }
-      const int lk = lane >> 3, lc = lane & 7;   // this lane's (row, source) pair
+      const int lk = lane / LPR, lc = lane % LPR;   // this lane's (row, source) pair
       float l = kNegInf;
       if (lk < nr && lc < ntot) l = *lse_at(lc, row0 + lk);
       float M = l;
-      for (int sft = 4; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));   // over the 8 lanes of the row
+#pragma unroll
+      for (int sft = LPR / 2; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));   // over the lanes of the row
       const float w = M != kNegInf ? __expf(l - M) : 0.f;   // exp(-inf) = 0
 #pragma unroll
       for (int k = 0; k < RPW; ++k) {
@@ -985,41 +990,47 @@ __global__ void __launch_bounds__(256) merge_tiles_kernel(const PieMerge* __rest
 #pragma unroll
         for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
 #pragma unroll
-        for (int c = 0; c < MAXS; ++c) {
-          const float wu = __shfl_sync(0xFFFFFFFFu, w, k * 8 + c);
+        for (int c = 0; c < NS; ++c) {
+          const float wu = __shfl_sync(0xFFFFFFFFu, w, k * LPR + c);
           Z += wu;
 #pragma unroll
           for (int e = 0; e < EPL; ++e) acc[e] += wu * v[k][c][e];
         }
-        const float Mk = __shfl_sync(0xFFFFFFFFu, M, k * 8);
+        const float Mk = __shfl_sync(0xFFFFFFFFu, M, k * LPR);
         if (k < nr) store_row(row0 + k, acc, Mk, Z);
       }
-    } else {
-      for (int k = 0; k < nr; ++k) {   // many sources: row by row
-        const int row = row0 + k;
-        float M = kNegInf;
-        for (int c = lane; c < ntot; c += 32) M = fmaxf(M, *lse_at(c, row));
-        for (int sft = 16; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));
-        float Z = 0.f, acc[EPL];
+    }
+  };
+  if (ntot <= 2) {   // (a request's private part plus the cascade's shared part, a unit cut once: the common cases)
+    run_few(std::integral_constant<int, 8>{}, std::integral_constant<int, 2>{});
+    return;
+  }
+  if (ntot <= 4) {
+    run_few(std::integral_constant<int, 4>{}, std::integral_constant<int, 4>{});
+    return;
+  }
+  for (int row = warp; row < mg.nrows; row += blockDim.x >> 5) {   // many sources: row by row
+    float M = kNegInf;
+    for (int c = lane; c < ntot; c += 32) M = fmaxf(M, *lse_at(c, row));
+    for (int sft = 16; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, sft));
+    float Z = 0.f, acc[EPL];
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-        for (int base = 0; base < ntot; base += 32) {
-          const int c = base + lane;
-          float w = 0.f;
-          if (c < ntot && M != kNegInf) w = __expf(*lse_at(c, row) - M);
-          Z += w;
-          const int cnt = min(32, ntot - base);
-          for (int u = 0; u < cnt; ++u) {
-            const float wu = __shfl_sync(0xFFFFFFFFu, w, u);
-            const float* src = row_at(base + u, row);
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+    for (int base = 0; base < ntot; base += 32) {
+      const int c = base + lane;
+      float w = 0.f;
+      if (c < ntot && M != kNegInf) w = __expf(*lse_at(c, row) - M);
+      Z += w;
+      const int cnt = min(32, ntot - base);
+      for (int u = 0; u < cnt; ++u) {
+        const float wu = __shfl_sync(0xFFFFFFFFu, w, u);
+        const float* src = row_at(base + u, row);
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) acc[e] += wu * src[e];
-          }
-        }
-        for (int sft = 16; sft > 0; sft >>= 1) Z += __shfl_xor_sync(0xFFFFFFFFu, Z, sft);
-        store_row(row, acc, M, Z);
+        for (int e = 0; e < EPL; ++e) acc[e] += wu * src[e];
       }
     }
+    for (int sft = 16; sft > 0; sft >>= 1) Z += __shfl_xor_sync(0xFFFFFFFFu, Z, sft);
+    store_row(row, acc, M, Z);
   }
 }
 
