@@ -632,12 +632,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
               for (int c = 0; c < 32; ++c)
                 if (!((bits[(k * 32 + c) / P] >> ((k * 32 + c) % P)) & 1u)) x[c] = kNegInf;
             }
-            // Lean copy: no maximum is taken while the sums stay small.  The exponentials are computed
+            // Lean form (the whole of the lean copy; in the general copy the first attempt on every chunk, masked
+            // scores being -inf by now - the halves around an item's first masked page and the diagonal of a
+            // causal chunk are a quarter of a short item): no maximum is taken while the sums stay small.  The exponentials are computed
             // against the current reference straight away; the chunk's sum bounds its largest term, so a
             // sum below 2^16 proves that no score runs ahead of the reference by more than 16 binades
             // (fp32 sums and bf16 P keep their relative precision at any such lag).  Otherwise - or when a
             // row of the warp has no reference yet - the chunk is redone the careful way below.
-            if constexpr (!kMasked) {
+            if constexpr (!kMasked || P != 8) {   // (with 8-token pages the general loop has no registers left for it)
               if (__all_sync(0xFFFFFFFFu, m_ref != kNegInf)) {
                 const uint64_t negm2 = pack_f32x2(-m_ref, -m_ref);
                 uint64_t ca = pack_f32x2(0.f, 0.f), cb = pack_f32x2(0.f, 0.f);
