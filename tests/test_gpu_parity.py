@@ -866,3 +866,29 @@ def test_very_short_decode_launches_merge_across_blocks_inside_the_kernel(R, D, 
         for n, pg in enumerate(wl.used_pages()):
             Ko, Vo = pool[int(pg)]
             assert same_bits(K[n], Ko) and same_bits(V[n], Vo), f"page {pg}"
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("tile_sms,D", [(4, 64), (8, 128), (40, 128)])
+def test_row_tile_units_cut_across_blocks_are_merged_like_the_oracle(tile_sms, D):
+    """One prefill chunk over a long context is two row-tile units (two kv heads) for far more thread blocks: the
+    units are cut into pieces whose fp32 partials the tile merge combines - from two sources per row (eight rows per
+    warp and step), from four (four rows), and from sixteen (row by row)."""
+    import paper_2510_24051_b200 as pie
+    from tests._gpu import GpuPool, check_close
+    wl = configs._assemble("one_long_prefill", configs.SEED0 + 31, 8, 2, D, 16, "bf16", 1024,
+                           np.array([64]), np.array([8192]), None)
+    O_ref, L_ref, _ = run_oracle(wl, poison=True)
+    with GpuPool(wl.num_pages, wl.P, wl.H_q, wl.H_kv, wl.D, wl.dtype) as gp:
+        pie.pie_set_option(gp.ctx, pie.PIE_OPT_TILE_SMS, tile_sms)
+        gp.install(wl, poison=True)
+        plan = gp.plan(wl)
+        info = pie.pie_plan_get_info(plan)
+        pieces = min(tile_sms, 2 * 512 // 32)
+        assert info["num_merge_groups"] == 2 and info["num_split_items"] == 0
+        assert pieces <= info["num_tile_items"] <= pieces + 2          # two units over `pieces` equal shares
+        out, lse = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+        out2, lse2 = gp.forward(plan, wl.q("cuda"), wl.k_new("cuda"), wl.v_new("cuda"))
+        assert torch.equal(out.view(torch.int16), out2.view(torch.int16)) and torch.equal(lse, lse2)
+        pie.pie_plan_destroy(plan)
+        check_close(out.double().cpu().numpy(), lse.double().cpu().numpy(), O_ref, L_ref, wl.dtype, wl.qo_indptr)
