@@ -170,7 +170,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTileM = 128;    // rows per Q tile
 constexpr int kTileN = 128;    // tokens per KV tile (one stage of the K / V rings)
 constexpr int kHalf = 64;      // columns per half tile: the unit handed between softmax and MMA
-constexpr int kThreads = 384;   // 8 softmax warps, K producer, MMA issuer, Q loader, V producer
+constexpr int kThreads = 352;
 
 template <int D, int P>
 struct TcCfg {
@@ -183,7 +183,7 @@ struct TcCfg {
   static constexpr int QTILE = kTileM * D * 2;
   static constexpr int KVTILE = kTileN * D * 2;
   static constexpr int STAGES = D == 128 ? 2 : 4;
-  static constexpr int NBAR = 8 * STAGES + 19;   // (the K / V rings have a full and an empty barrier per 64-token half of a stage)
+  static constexpr int NBAR = 4 * STAGES + 19;
   static constexpr int OSLAB = kTileM * 128;           // output staging: one 64-column slab of a 128-row tile per warpgroup
   static constexpr int SMEM = 2 * QTILE + 2 * STAGES * KVTILE + 2 * OSLAB + NBAR * 8 + 64;
 };
@@ -198,14 +198,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
   uint8_t* sV = sK + C::STAGES * C::KVTILE;
   uint8_t* sO = sV + C::STAGES * C::KVTILE;   // [2][128 rows][128 B], 128-byte swizzle like the Q tiles
   uint64_t* bars = reinterpret_cast<uint64_t*>(sO + 2 * C::OSLAB);
-  // K / V rings: a stage holds a 128-token tile, but is handed over - and refilled - in halves of 64 tokens
-  // ([2 * stage + half]): a half is requested again as soon as the MMAs that read it are done, half a tile earlier
-  // than the whole stage could be, which is what keeps the next tile from arriving late with only two stages
   uint64_t* k_full = bars;
-  uint64_t* k_empty = k_full + 2 * C::STAGES;
-  uint64_t* v_full = k_empty + 2 * C::STAGES;
-  uint64_t* v_empty = v_full + 2 * C::STAGES;
-  uint64_t* q_full = v_empty + 2 * C::STAGES;  // [2]      Q tile t is in shared memory
+  uint64_t* k_empty = k_full + C::STAGES;
+  uint64_t* v_full = k_empty + C::STAGES;
+  uint64_t* v_empty = v_full + C::STAGES;
+  uint64_t* q_full = v_empty + C::STAGES;  // [2]      Q tile t is in shared memory
   uint64_t* q_free = q_full + 2;           // [2]      every S MMA of the item that reads Q tile t is complete
   uint64_t* s_full = q_free + 2;           // [2][2]   S_t^h is complete in TMEM
   uint64_t* p_full = s_full + 4;           // [2][2]   P_t^h is written (128 arrivals)
@@ -220,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
   const bool out_wide = kflags & 2;      // the output pointer allows 32-byte stores
   const bool use_omap = kflags & 4;      // full output tiles leave through shared memory and a TMA store
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 2 * C::STAGES; ++s) {
+    for (int s = 0; s < C::STAGES; ++s) {
       mbar_init(smem_u32(k_full + s), 1);
       mbar_init(smem_u32(k_empty + s), 1);
       mbar_init(smem_u32(v_full + s), 1);
@@ -253,63 +250,61 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
 
   const int it0 = p.cta_ptr[blockIdx.x], it1 = p.cta_ptr[blockIdx.x + 1];
 
-  if (warp == 8 || warp == 11) {
-    // ================================================================ producers: warp 8 the K tiles, warp 11 the V tiles
-    // Each walks the block's tiles in order, one 64-token half at a time: wait until the half of the stage is
-    // free, announce the bytes, one bulk copy per (page, slab) of the half.
-    const bool is_v = warp == 11;
-    uint64_t* const full = is_v ? v_full : k_full;
-    uint64_t* const empty = is_v ? v_empty : k_empty;
-    uint8_t* const ring = is_v ? sV : sK;
+  if (warp == 8) {
+    // ================================================================ producer
     uint32_t tile_cnt = 0, land_cnt = 0;
     for (int it = it0; it < it1; ++it) {
       const PieItem item = p.items[it];
-      const uint8_t* base = p.pool + (int64_t)item.kv_head * (2 * C::BLK) + (is_v ? C::BLK : 0);
+      const uint8_t* base = p.pool + (int64_t)item.kv_head * (2 * C::BLK);
       const int npages = item.page_end - item.page_begin;
       const int ntiles = (npages + C::PPT - 1) / C::PPT;
       const bool ragged = item.last_page_len < P;   // slots past the end of the context may hold anything
       for (int j = 0; j < ntiles; ++j, ++tile_cnt) {
         const uint32_t s = tile_cnt % C::STAGES, ph = (tile_cnt / C::STAGES) & 1;
         const int nvalid = min(C::PPT, npages - j * C::PPT);
+        const int ncopies = nvalid * C::NSLAB;
         int2 rec = make_int2(0, -1);
         if (lane < nvalid) rec = __ldg(&p.kept[item.page_begin + j * C::PPT + lane]);
         const int pg = lane / C::NSLAB, sl = lane % C::NSLAB;   // copy `lane`: page pg of the tile, slab sl
         const int ph_pg = __shfl_sync(0xFFFFFFFFu, rec.x, pg);   // (at most PPT * NSLAB <= 32 copies per tile)
-        for (int hh = 0; hh < 2; ++hh) {
-          const int nv = max(0, min(C::PPH, nvalid - hh * C::PPH));   // pages of this half (a half without pages still completes its barrier)
-          const bool mine = pg >= hh * C::PPH && pg < hh * C::PPH + nv;
-          mbar_wait(smem_u32(empty + 2 * s + hh), ph ^ 1, p.status);
-          // V: a half that holds the request's partly filled last page lands on a private barrier first: the rows
-          // past the end of the context are cleared (they may hold NaN patterns, and 0 x NaN would poison O)
-          // before the half is handed to the MMA thread.
-          unsigned hit = 0;
-          if (is_v && ragged)
-            hit = __ballot_sync(0xFFFFFFFFu, lane < nvalid && lane / C::PPH == hh && (int)((uint32_t)rec.y & ~PIE_KEPT_NEEDS_MASK) == item.last_logical);
-          const bool odd_end = is_v && P == 8 && (nvalid & 1) && (nvalid - 1) / C::PPH == hh;   // half of the tile's last 16-token step has no page
-          const uint32_t bar = (hit || odd_end) ? smem_u32(v_land) : smem_u32(full + 2 * s + hh);
-          if (lane == 0) mbar_expect_tx(bar, nv * C::BLK);
+        // ---- K
+        mbar_wait(smem_u32(k_empty + s), ph ^ 1, p.status);
+        if (lane == 0) mbar_expect_tx(smem_u32(k_full + s), nvalid * C::BLK);
+        __syncwarp();
+        if (lane < ncopies)
+          bulk_g2s(smem_u32(sK + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
+                   base + (int64_t)ph_pg * p.page_bytes + sl * C::SLAB_PAGE, C::SLAB_PAGE, smem_u32(k_full + s));
+        __syncwarp();
+        // ---- V.  A tile that holds the request's partly filled last page lands on a private
+        // barrier first: the rows past the end of the context are cleared (they may hold NaN
+        // patterns, and 0 x NaN would poison O) before the tile is handed to the MMA thread.
+        mbar_wait(smem_u32(v_empty + s), ph ^ 1, p.status);
+        unsigned hit = 0;
+        if (ragged) hit = __ballot_sync(0xFFFFFFFFu, lane < nvalid && (int)((uint32_t)rec.y & ~PIE_KEPT_NEEDS_MASK) == item.last_logical);
+        const bool odd_end = P == 8 && (nvalid & 1);   // half of the tile's last 16-token step has no page
+        const uint32_t vbar = (hit || odd_end) ? smem_u32(v_land) : smem_u32(v_full + s);
+        if (lane == 0) mbar_expect_tx(vbar, nvalid * C::BLK);
+        __syncwarp();
+        if (lane < ncopies)
+          bulk_g2s(smem_u32(sV + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
+                   base + (int64_t)ph_pg * p.page_bytes + C::BLK + sl * C::SLAB_PAGE, C::SLAB_PAGE, vbar);
+        __syncwarp();
+        if (hit || odd_end) {
+          mbar_wait(smem_u32(v_land), land_cnt & 1, p.status);
+          ++land_cnt;
+          constexpr int CH = D * 2 / 16;
+          auto clear_rows = [&](int first, int n) {   // V rows [first, first + n) of the tile
+            for (int c = lane; c < n * CH; c += 32) {
+              const int tkn = first + c / CH, ch = c % CH;
+              *reinterpret_cast<uint4*>(sV + s * C::KVTILE + (ch >> 3) * C::SLAB_TILE + tkn * 128 + (((ch & 7) ^ (tkn & 7)) << 4)) =
+                  make_uint4(0, 0, 0, 0);
+            }
+          };
+          if (hit) clear_rows((__ffs(hit) - 1) * P + item.last_page_len, P - item.last_page_len);
+          if (odd_end) clear_rows(nvalid * P, P);
+          fence_async_smem();
           __syncwarp();
-          if (mine)
-            bulk_g2s(smem_u32(ring + s * C::KVTILE + sl * C::SLAB_TILE + pg * C::SLAB_PAGE),
-                     base + (int64_t)ph_pg * p.page_bytes + sl * C::SLAB_PAGE, C::SLAB_PAGE, bar);
-          __syncwarp();
-          if (hit || odd_end) {
-            mbar_wait(smem_u32(v_land), land_cnt & 1, p.status);
-            ++land_cnt;
-            constexpr int CH = D * 2 / 16;
-            auto clear_rows = [&](int first, int n) {   // V rows [first, first + n) of the tile
-              for (int c = lane; c < n * CH; c += 32) {
-                const int tkn = first + c / CH, ch = c % CH;
-                *reinterpret_cast<uint4*>(sV + s * C::KVTILE + (ch >> 3) * C::SLAB_TILE + tkn * 128 + (((ch & 7) ^ (tkn & 7)) << 4)) =
-                    make_uint4(0, 0, 0, 0);
-              }
-            };
-            if (hit) clear_rows((__ffs(hit) - 1) * P + item.last_page_len, P - item.last_page_len);
-            if (odd_end) clear_rows(nvalid * P, P);
-            fence_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(v_full + 2 * s + hh));
-          }
+          if (lane == 0) mbar_arrive(smem_u32(v_full + s));
         }
       }
     }
@@ -378,12 +373,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
         // prologue: both halves of S_t for the first KV tile
         {
           const uint32_t s = tile_cnt % C::STAGES, ph = (tile_cnt / C::STAGES) & 1;
-          for (int h = 0; h < min(2, nhalf); ++h) {
-            mbar_wait(smem_u32(k_full + 2 * s + h), ph, p.status);
-            tc_fence_after();
+          mbar_wait(smem_u32(k_full + s), ph, p.status);
+          tc_fence_after();
+          for (int h = 0; h < min(2, nhalf); ++h)
             for (int t = 0; t < nt; ++t) issue_s(t, h, s);
-          }
-          for (int h = 0; h < 2; ++h) umma_commit(smem_u32(k_empty + 2 * s + h));   // (a half without tokens is handed back too)
+          umma_commit(smem_u32(k_empty + s));
           if (ntiles == 1)
             for (int t = 0; t < nt; ++t) umma_commit(smem_u32(q_free + t));
         }
@@ -391,15 +385,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
           const uint32_t cnt = tile_cnt + j;
           const uint32_t s = cnt % C::STAGES, ph = (cnt / C::STAGES) & 1;
           const uint32_t sn = (cnt + 1) % C::STAGES, phn = ((cnt + 1) / C::STAGES) & 1;
+          mbar_wait(smem_u32(v_full + s), ph, p.status);
           if (nt == 2 && j > 0 && 2 * j + 5 <= nhalf) {
             // ---- interior tile: this tile and the next both have two full halves
+            mbar_wait(smem_u32(k_full + sn), phn, p.status);
             const uint64_t vd0 = v_desc0 + (uint64_t)(s * (C::KVTILE >> 4));
             const uint64_t kd0 = k_desc0 + (uint64_t)(sn * (C::KVTILE >> 4));
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
 #pragma unroll
               for (int t = 0; t < 2; ++t) {
-                if (t == 0) mbar_wait(smem_u32(v_full + 2 * s + h), ph, p.status);   // this half of the V tile has landed
                 mbar_wait(bar_p + 8 * (2 * t + h), (half_ph >> (2 * t + h)) & 1, p.status);
                 tc_fence_after();
                 const uint32_t dO = tmem + 256 + t * D, dS = tmem + t * 128 + h * kHalf;
@@ -407,11 +402,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
                 for (int ks = 0; ks < kHalf / 16; ++ks)   // 16 token rows = 2048 bytes per k-step
                   umma_ts(dO, dS + ks * 8, vd0 + (uint64_t)((h * (kHalf / 16) + ks) * 128), idesc_pv, 1u);
                 umma_commit(bar_pv + 8 * t);
-                if (t == 1) umma_commit(smem_u32(v_empty + 2 * s + h));
-                if (t == 0) {   // ... and this half of the next K tile
-                  mbar_wait(smem_u32(k_full + 2 * sn + h), phn, p.status);
-                  tc_fence_after();
-                }
+                if (h == 1 && t == 1) umma_commit(smem_u32(v_empty + s));
                 const uint64_t qd = q_desc0 + (uint64_t)(t * (C::QTILE >> 4));
                 const uint64_t kd = kd0 + (uint64_t)(h * ((kHalf * 128) >> 4));
 #pragma unroll
@@ -420,7 +411,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
                   umma_ss(dS, qd + off, kd + off, idesc_s, ks > 0);
                 }
                 umma_commit(bar_s + 8 * (2 * t + h));
-                if (t == 1) umma_commit(smem_u32(k_empty + 2 * sn + h));
+                if (h == 1 && t == 1) umma_commit(smem_u32(k_empty + sn));
               }
             }
             half_ph ^= 0xFu;
@@ -429,13 +420,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
           // ---- first / last tiles of an item, ragged halves, single Q tile
           const int nh = min(2, nhalf - 2 * j);                            // halves of this tile
           const int nhn = j + 1 < ntiles ? min(2, nhalf - 2 * j - 2) : 0;   // halves of the next one
+          bool k_ready = false;
           for (int h = 0; h < nh; ++h) {
             const int i = 2 * j + h;
             const int ksteps = (i + 1 < nhalf ? kHalf : last_cols) / 16;
             for (int t = 0; t < nt; ++t) {
-              if (t == 0) mbar_wait(smem_u32(v_full + 2 * s + h), ph, p.status);
               mbar_wait(bar_p + 8 * (2 * t + h), (half_ph >> (2 * t + h)) & 1, p.status);
               half_ph ^= 1u << (2 * t + h);
+              if (h < nhn && !k_ready) {
+                mbar_wait(smem_u32(k_full + sn), phn, p.status);
+                k_ready = true;
+              }
               if (i == 0) mbar_wait(smem_u32(o_free + t), ((ph_item >> t) & 1) ^ 1, p.status);  // the previous epilogue has drained O_t
               tc_fence_after();
               const uint64_t vd = v_desc0 + (uint64_t)(s * (C::KVTILE >> 4) + h * (kHalf / 16) * 128);
@@ -443,22 +438,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const AttnParams p
               for (int ks = 0; ks < ksteps; ++ks)
                 umma_ts(dO, aP + ks * 8, vd + (uint64_t)(ks * 128), idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
               umma_commit(bar_pv + 8 * t);
-              if (t == nt - 1) umma_commit(smem_u32(v_empty + 2 * s + h));
+              if (h == nh - 1 && t == nt - 1) umma_commit(smem_u32(v_empty + s));
               if (i + 1 == nhalf) umma_commit(smem_u32(o_done + t));
               if (h < nhn) {   // S_t^h of the next tile goes into the columns this PV frees
-                if (t == 0) {
-                  mbar_wait(smem_u32(k_full + 2 * sn + h), phn, p.status);
-                  tc_fence_after();
-                }
                 issue_s(t, i + 2, sn);
-                if (t == nt - 1) umma_commit(smem_u32(k_empty + 2 * sn + h));
+                if (h == nhn - 1 && t == nt - 1) umma_commit(smem_u32(k_empty + sn));
               }
             }
           }
-          // (halves without tokens - of this tile's V, of the next tile's K - are handed back all the same)
-          for (int h = nh; h < 2; ++h) umma_commit(smem_u32(v_empty + 2 * s + h));
-          if (j + 1 < ntiles)
-            for (int h = nhn; h < 2; ++h) umma_commit(smem_u32(k_empty + 2 * sn + h));
           if (j + 2 == ntiles)   // the S MMAs of the last tile are all issued: Q may be replaced once they are done
             for (int t = 0; t < nt; ++t) umma_commit(smem_u32(q_free + t));
         }
